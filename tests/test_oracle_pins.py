@@ -1,0 +1,359 @@
+"""Pins for the CPU oracle: closed forms, invariants, special cases, brute force.
+
+None of these retype the oracle's formula with the same library calls: the brute
+force uses scalar Python loops, the closed forms come from linearity / the
+definition of softmax, and the special cases reduce to plain base-cache attention.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import lrkv_oracle as O
+from paper_2609_34054_b200 import inputs as I
+
+RNG = np.random.default_rng(1234)
+
+
+def _tiny(T=7, d=12, n_q=4, n_kv=2, hd=6, N=3, rk=2, rv=2, B=3):
+    r = lambda *s: RNG.standard_normal(s)
+    return dict(H=r(T, d), W_k=0.3 * r(d, n_kv * hd), W_v=0.3 * r(d, n_kv * hd),
+                A_k=0.3 * r(N, d, rk), B_k=0.3 * r(N, rk, n_kv * hd),
+                A_v=0.3 * r(N, d, rv), B_v=0.3 * r(N, rv, n_kv * hd),
+                q=r(B, n_q, hd), agent_id=np.array([0, 2, 1][:B]), ctx_len=np.array([T, 1, 4][:B]),
+                n_kv=n_kv)
+
+
+def _decode(p, s_k=2.0, s_v=2.0, **kw):
+    args = dict(p)
+    n_kv = args.pop("n_kv")
+    heads = kw.pop("heads", None)
+    args.update(kw)
+    return O.lr_decode_reference(args["q"], args["agent_id"], args["ctx_len"], args["H"], args["W_k"], args["W_v"],
+                                 args["A_k"], args["B_k"], args["A_v"], args["B_v"], s_k, s_v, n_kv, heads=heads)
+
+
+# ---------------------------------------------------------------- brute force (P11)
+
+def _brute_decode(p, s_k, s_v):
+    """Scalar-loop evaluation of Eq. 1 (left form) + softmax attention."""
+    H, q = p["H"], p["q"]
+    T, d = H.shape
+    Bn, n_q, hd = q.shape
+    n_kv = p["n_kv"]
+    G = n_q // n_kv
+    out = np.zeros((Bn, n_q, hd))
+    for b in range(Bn):
+        a = int(p["agent_id"][b])
+        t_max = int(p["ctx_len"][b])
+        for h in range(n_q):
+            g = h // G
+            # adapted K and V rows of this head, element by element
+            K = [[0.0] * hd for _ in range(t_max)]
+            V = [[0.0] * hd for _ in range(t_max)]
+            for t in range(t_max):
+                for c in range(hd):
+                    col = g * hd + c
+                    accK = accV = 0.0
+                    for i in range(d):
+                        wk = p["W_k"][i, col]
+                        wv = p["W_v"][i, col]
+                        for j in range(p["A_k"].shape[2]):
+                            wk += s_k * p["A_k"][a, i, j] * p["B_k"][a, j, col]
+                        for j in range(p["A_v"].shape[2]):
+                            wv += s_v * p["A_v"][a, i, j] * p["B_v"][a, j, col]
+                        accK += H[t, i] * wk
+                        accV += H[t, i] * wv
+                    K[t][c], V[t][c] = accK, accV
+            z = [sum(q[b, h, c] * K[t][c] for c in range(hd)) / math.sqrt(hd) for t in range(t_max)]
+            m = max(z)
+            e = [math.exp(v - m) for v in z]
+            den = sum(e)
+            for c in range(hd):
+                out[b, h, c] = sum(e[t] * V[t][c] for t in range(t_max)) / den
+    return out
+
+
+def test_brute_force_tiny():
+    p = _tiny()
+    np.testing.assert_allclose(_decode(p, 2.0, 0.5), _brute_decode(p, 2.0, 0.5), rtol=1e-10, atol=1e-12)
+
+
+def test_brute_force_tiny_gqa_odd_group():
+    p = _tiny(T=5, d=8, n_q=6, n_kv=2, hd=4, N=3, rk=1, rv=2)
+    np.testing.assert_allclose(_decode(p, 1.0, 1.0), _brute_decode(p, 1.0, 1.0), rtol=1e-10, atol=1e-12)
+
+
+# ------------------------------------------------------ P1: reductions to base-only
+
+def _base_only(p):
+    out = np.zeros_like(p["q"])
+    for b in range(p["q"].shape[0]):
+        K = p["H"] @ p["W_k"]
+        V = p["H"] @ p["W_v"]
+        out[b] = O.attend_decode_one(p["q"][b], K, V, int(p["ctx_len"][b]), p["n_kv"])
+    return out
+
+
+def test_zero_scale_zero_B_zero_rank_reduce_to_base_attention():
+    p = _tiny()
+    base = _base_only(p)
+    np.testing.assert_allclose(_decode(p, 0.0, 0.0), base, rtol=1e-12)
+    pz = dict(p, B_k=np.zeros_like(p["B_k"]), B_v=np.zeros_like(p["B_v"]))
+    np.testing.assert_allclose(_decode(pz), base, rtol=1e-12)
+    p0 = dict(p, A_k=p["A_k"][:, :, :0], B_k=p["B_k"][:, :0], A_v=p["A_v"][:, :, :0], B_v=p["B_v"][:, :0])
+    np.testing.assert_allclose(_decode(p0), base, rtol=1e-12)
+    # and the adapters do matter when present
+    assert np.max(np.abs(_decode(p) - base)) > 1e-2
+
+
+# ------------------------------------------------------ P2: merged == decomposed
+
+def test_merged_equals_decomposed_eq1():
+    p = _tiny(T=33, d=40)
+    for a in range(3):
+        m = O.adapted_projection(p["H"], p["W_k"], p["A_k"][a], p["B_k"][a], 1.7)
+        dcp = O.decomposed_projection(p["H"], p["W_k"], p["A_k"][a], p["B_k"][a], 1.7)
+        np.testing.assert_allclose(m, dcp, rtol=1e-11, atol=1e-12)
+        rec = O.reconstruct(O.base_cache(p["H"], p["W_k"]), O.lr_cache(p["H"], p["A_k"][a]), p["B_k"][a], 1.7)
+        np.testing.assert_allclose(m, rec, rtol=1e-11, atol=1e-12)
+
+
+def test_literal_eq1_without_scale():
+    # s = 1 must be the paper's literal X(W0 + AB)
+    p = _tiny()
+    X, W0, A, B = p["H"], p["W_v"], p["A_v"][1], p["B_v"][1]
+    lit = np.zeros((X.shape[0], W0.shape[1]))
+    for t in range(X.shape[0]):
+        for c in range(W0.shape[1]):
+            lit[t, c] = sum(X[t, i] * (W0[i, c] + sum(A[i, j] * B[j, c] for j in range(A.shape[1])))
+                            for i in range(X.shape[1]))
+    np.testing.assert_allclose(O.adapted_projection(X, W0, A, B, 1.0), lit, rtol=1e-11, atol=1e-12)
+
+
+def test_lr_cache_shape_and_transposition():
+    # A is d x r (tall), B is r x d_out (wide): a transposed operand cannot even multiply
+    p = _tiny(d=12, rk=2)
+    L = O.lr_cache(p["H"], p["A_k"][0])
+    assert L.shape == (p["H"].shape[0], 2)
+    e = np.zeros((1, 12)); e[0, 3] = 1.0
+    np.testing.assert_allclose(O.lr_cache(e, p["A_k"][0])[0], p["A_k"][0][3])
+    np.testing.assert_allclose(O.base_cache(e, p["W_k"])[0], p["W_k"][3])
+
+
+# ---------------------------------------------------------- P3: softmax properties
+
+def test_softmax_rows_sum_to_one_and_convexity():
+    z = RNG.standard_normal(1000) * 30
+    w = O.softmax_weights(z)
+    assert abs(w.sum() - 1.0) < 1e-12 and w.min() >= 0
+    assert np.argmax(w) == np.argmax(z)
+    p = _tiny(T=50)
+    p["ctx_len"] = np.array([50, 17, 3])
+    out = _decode(p)
+    G = p["q"].shape[1] // p["n_kv"]
+    hd = p["q"].shape[2]
+    for b in range(3):
+        a = p["agent_id"][b]
+        V = O.adapted_projection(p["H"], p["W_v"], p["A_v"][a], p["B_v"][a], 2.0)[: p["ctx_len"][b]]
+        for h in range(p["q"].shape[1]):
+            Vg = V[:, (h // G) * hd:(h // G + 1) * hd]
+            assert np.all(out[b, h] <= Vg.max(0) + 1e-12) and np.all(out[b, h] >= Vg.min(0) - 1e-12)
+
+
+def test_softmax_shift_invariance_and_two_point_closed_form():
+    z = np.array([0.3, -1.2])
+    w = O.softmax_weights(z)
+    assert abs(w[0] - 1.0 / (1.0 + math.exp(-1.5))) < 1e-15
+    np.testing.assert_allclose(O.softmax_weights(z + 100.0), w, rtol=1e-12)
+
+
+def test_scale_default_is_inverse_sqrt_head_dim():
+    # two keys, one query: weight of key 0 is logistic(sigma * q.(k0-k1))
+    hd = 16
+    q = RNG.standard_normal((1, hd)); K = RNG.standard_normal((2, hd)); V = np.eye(2, hd)
+    out = O.attend_decode_one(q, K, V, 2, 1)
+    w0 = 1.0 / (1.0 + math.exp(-float(q[0] @ (K[0] - K[1])) / 4.0))
+    np.testing.assert_allclose(out[0, :2], [w0, 1 - w0], rtol=1e-12)
+    out2 = O.attend_decode_one(q, K, V, 2, 1, sigma=0.5)
+    w0 = 1.0 / (1.0 + math.exp(-float(q[0] @ (K[0] - K[1])) * 0.5))
+    np.testing.assert_allclose(out2[0, :2], [w0, 1 - w0], rtol=1e-12)
+
+
+# ------------------------------------------------------------------ P4, P5, P6, P7
+
+def test_ctx_len_one_returns_value_row():
+    p = _tiny()
+    p["ctx_len"] = np.array([1, 1, 1])
+    out = _decode(p)
+    G = p["q"].shape[1] // p["n_kv"]; hd = p["q"].shape[2]
+    for b in range(3):
+        a = p["agent_id"][b]
+        v0 = p["H"][0] @ (p["W_v"] + 2.0 * p["A_v"][a] @ p["B_v"][a])
+        for h in range(p["q"].shape[1]):
+            np.testing.assert_allclose(out[b, h], v0[(h // G) * hd:(h // G + 1) * hd], rtol=1e-11)
+
+
+def test_zero_query_gives_mean_value_by_linearity():
+    p = _tiny(T=9)
+    p["q"] = np.zeros_like(p["q"]); p["ctx_len"] = np.array([9, 9, 9])
+    out = _decode(p)
+    G = p["q"].shape[1] // p["n_kv"]; hd = p["q"].shape[2]
+    for b in range(3):
+        a = p["agent_id"][b]
+        mean_v = p["H"].mean(0) @ (p["W_v"] + 2.0 * p["A_v"][a] @ p["B_v"][a])
+        for h in range(p["q"].shape[1]):
+            np.testing.assert_allclose(out[b, h], mean_v[(h // G) * hd:(h // G + 1) * hd], rtol=1e-10)
+
+
+def test_identical_rows_give_that_rows_value():
+    p = _tiny(T=6)
+    p["H"] = np.tile(p["H"][:1], (6, 1)); p["ctx_len"] = np.array([6, 3, 5])
+    out = _decode(p)
+    p1 = dict(p, ctx_len=np.array([1, 1, 1]))
+    np.testing.assert_allclose(out, _decode(p1), rtol=1e-11)
+
+
+def test_decode_invariant_to_token_permutation():
+    p = _tiny(T=11)
+    p["ctx_len"] = np.array([11, 11, 11])
+    perm = RNG.permutation(11)
+    np.testing.assert_allclose(_decode(p), _decode(dict(p, H=p["H"][perm])), rtol=1e-10)
+
+
+# --------------------------------------------------------------- P8: prefill/decode
+
+def test_prefill_row_equals_decode_at_that_length_and_is_causal():
+    p = _tiny(T=12)
+    T, S = 7, 5
+    q = RNG.standard_normal((S, 4, 6))
+    args = (p["H"], p["W_k"], p["W_v"], p["A_k"], p["B_k"], p["A_v"], p["B_v"], 2.0, 2.0, p["n_kv"])
+    pre = O.lr_prefill_reference(q, 1, T, *args)
+    for i in range(S):
+        dec = O.lr_decode_reference(q[i:i + 1], [1], [T + i + 1], *args)
+        np.testing.assert_allclose(pre[i], dec[0], rtol=1e-11)
+    # causality: changing a later new token's hidden state leaves earlier rows untouched
+    H2 = p["H"].copy(); H2[T + 3] += 1.0
+    pre2 = O.lr_prefill_reference(q, 1, T, H2, *args[1:])
+    np.testing.assert_array_equal(pre[:3], pre2[:3])
+    assert np.max(np.abs(pre[3:] - pre2[3:])) > 1e-6
+    # context rows are visible to every query
+    H3 = p["H"].copy(); H3[0] += 1.0
+    pre3 = O.lr_prefill_reference(q, 1, T, H3, *args[1:])
+    assert all(np.max(np.abs(pre[i] - pre3[i])) > 1e-9 for i in range(S))
+
+
+def test_attend_prefill_matches_row_restriction():
+    K = RNG.standard_normal((9, 8)); V = RNG.standard_normal((9, 8)); q = RNG.standard_normal((4, 2, 4))
+    full = O.attend_prefill(q, K, V, 5, 2)
+    part = O.attend_prefill(q, K, V, 5, 2, rows=[0, 3])
+    np.testing.assert_array_equal(full[[0, 3]], part[[0, 3]])
+    assert np.isnan(part[1]).all()
+
+
+# ---------------------------------------------------------------- P9: agent isolation
+
+def test_agent_isolation_and_identical_adapters():
+    p = _tiny()
+    ref = _decode(p)
+    p2 = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in p.items()}
+    p2["A_k"][1] += 5.0; p2["B_v"][1] -= 3.0          # request 2 uses agent 1
+    out = _decode(p2)
+    np.testing.assert_array_equal(out[[0, 1]], ref[[0, 1]])
+    assert np.max(np.abs(out[2] - ref[2])) > 1e-3
+    # identical adapters => identical results for the same query/ctx
+    p3 = dict(p, A_k=np.tile(p["A_k"][:1], (3, 1, 1)), B_k=np.tile(p["B_k"][:1], (3, 1, 1)),
+              A_v=np.tile(p["A_v"][:1], (3, 1, 1)), B_v=np.tile(p["B_v"][:1], (3, 1, 1)),
+              q=np.tile(p["q"][:1], (3, 1, 1)), ctx_len=np.array([7, 7, 7]))
+    o3 = _decode(p3)
+    np.testing.assert_array_equal(o3[0], o3[1]); np.testing.assert_array_equal(o3[0], o3[2])
+
+
+def test_concatenated_precompute_columns_equal_single_agent_products():
+    # Section 3.1: applying every A_k to the same hidden states == one product with [A_1 | ... | A_N]
+    p = _tiny(T=20)
+    A_cat = np.concatenate([p["A_k"][k] for k in range(3)], axis=1)
+    L_cat = O.lr_cache(p["H"], A_cat)
+    for k in range(3):
+        np.testing.assert_allclose(L_cat[:, 2 * k:2 * k + 2], O.lr_cache(p["H"], p["A_k"][k]), rtol=1e-12)
+
+
+# ------------------------------------------------------- staged (cache-content) form
+
+def test_attend_from_caches_equals_first_principles():
+    p = _tiny(T=10)
+    a = 2
+    kb, vb = O.base_cache(p["H"], p["W_k"]), O.base_cache(p["H"], p["W_v"])
+    Lk, Lv = O.lr_cache(p["H"], p["A_k"][a]), O.lr_cache(p["H"], p["A_v"][a])
+    got = O.attend_from_caches(p["q"][0], kb, vb, Lk, Lv, p["B_k"][a], p["B_v"][a], 2.0, 0.7, p["n_kv"])
+    ref = O.lr_decode_reference(p["q"][:1], [a], [10], p["H"], p["W_k"], p["W_v"], p["A_k"], p["B_k"],
+                                p["A_v"], p["B_v"], 2.0, 0.7, p["n_kv"])[0]
+    np.testing.assert_allclose(got, ref, rtol=1e-10)
+    np.testing.assert_allclose(got, _brute_decode(dict(p, q=p["q"][:1], agent_id=[a], ctx_len=[10]), 2.0, 0.7)[0],
+                               rtol=1e-10)
+
+
+def test_head_sampling_matches_full():
+    p = _tiny()
+    full = _decode(p)
+    part = _decode(p, heads=[1])
+    G = 2
+    np.testing.assert_array_equal(part[:, G:], full[:, G:])
+    assert np.isnan(part[:, :G]).all()
+
+
+# --------------------------------------------------- P12: rebase / schedule equivalence
+
+def test_rebase_same_hidden_states_is_identity_and_order_independent():
+    p = _tiny(T=16)
+    cache = O.base_cache(p["H"], p["W_k"])
+    again = cache.copy(); again[4:12] = O.base_cache(p["H"][4:12], p["W_k"])
+    np.testing.assert_array_equal(cache, again)
+    # lazy-prefill order (one write over the segment after the turn) vs double-batching
+    # order (token by token during the turn) leave the same cache state
+    X_neut = RNG.standard_normal((8, p["H"].shape[1]))
+    lp = cache.copy(); lp[4:12] = O.base_cache(X_neut, p["W_k"])
+    db = cache.copy()
+    for t in range(8):
+        db[4 + t] = O.base_cache(X_neut[t:t + 1], p["W_k"])[0]
+    np.testing.assert_allclose(lp, db, rtol=1e-13)
+
+
+# ------------------------------------------------ P10: cache-size closed form vs paper
+
+def _golden_table9():
+    path = os.path.join(os.path.dirname(__file__), "golden", "table9_peak_memory.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    return [(float(a), float(b), float(c)) for a, b, c in rows]
+
+
+def test_lr_cache_bytes_against_paper_memory_table():
+    # paper setup: Llama-3.1-8B (32 layers, 8 kv heads x 128), three agents, QV LoRA r=8 => only V has LR
+    base, lr = O.cache_bytes_per_token(n_kv=8, hd=128, n_agents=3, rank_k=0, rank_v=8)
+    assert base == 4096 and lr == 48
+    assert abs(lr / base - 3 * 8 / (2 * 1024)) < 1e-15          # = 1.17 %
+    rows = _golden_table9()
+    tokens_k, full, pre = rows[-1]
+    assert (pre - full) / full < 0.02                            # "within 2 %" at 66.4k tokens
+    predicted_gb = tokens_k * 1e3 * 32 * lr / 1e9
+    # the persistent LR caches must fit inside the measured gap (which also holds temporaries)
+    assert 0.0 < predicted_gb <= (pre - full) + 0.005
+    # and the gap grows with length roughly like a per-token cost (monotone)
+    gaps = [c - b for _, b, c in rows]
+    assert all(g2 >= g1 - 0.011 for g1, g2 in zip(gaps, gaps[1:]))
+
+
+# -------------------------------------------------- sensitivity on the C1 distribution
+
+def test_c1_adapter_term_is_visible_to_the_tolerance():
+    geo = I.C1
+    w = I.layer_weights(geo, seed=0)
+    H = I.hidden_states(64, geo, seed=0).float().numpy()
+    q = I.queries(geo.n_agents, geo, seed=0).float().numpy()
+    f = {k: v.float().numpy() for k, v in w.items()}
+    args = (H, f["W_k"], f["W_v"], f["A_k"], f["B_k"], f["A_v"], f["B_v"])
+    with_lr = O.lr_decode_reference(q, [0, 1, 2], [64] * 3, *args, geo.scale_k, geo.scale_v, geo.n_kv)
+    no_lr = O.lr_decode_reference(q, [0, 1, 2], [64] * 3, *args, 0.0, 0.0, geo.n_kv)
+    diff = np.abs(with_lr - no_lr)
+    assert np.max(diff - (2e-2 + 1e-2 * np.abs(no_lr))) > 0.0, "adapters invisible at the stated tolerance"
