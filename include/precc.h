@@ -1,0 +1,182 @@
+/*
+ * precc -- shared base KV cache + per-agent low-rank (LR) KV cache path for
+ * multi-LoRA agents, hand-written for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, for ONE decoder layer, the cache path of PReCache:
+ *
+ *   Eq. 1            Y_i = X (W0 + A_i B_i) = X W0 + (X A_i) B_i
+ *   Section 2.2      base cache X W0 (shared by all agents) + LR cache X A_i (width r, per agent)
+ *   Section 3.1      PreLRShared: when a segment is first processed, X A_k is built for EVERY agent k
+ *   Section 3.2      ReBaseShared: the base cache is rebuilt as X_neut W0 from adapter-free hidden states
+ *   Section 4.1 /    attention of the current agent over the base cache plus its own LR cache without
+ *   Appendix D.2     materialising the agent's K or V (the adapter is folded into the query side and
+ *                    into the output side by associativity)
+ *
+ * with the usual LoRA scale s = alpha / r:  K_a = K_base + s_k (H A_a^K) B_a^K,  V_a likewise.
+ * The path is position-free (no rotary embedding is applied inside the library).
+ *
+ * Conventions
+ *   - All tensors are bf16 in DEVICE memory unless stated; all accumulation is fp32; stores round to
+ *     nearest even.  Index arrays are int32 in DEVICE memory unless stated.
+ *   - Every buffer is owned by the caller.  The library allocates no device memory; it keeps no
+ *     pointer after the work it enqueued on `stream` has completed.  `stream` is a cudaStream_t
+ *     passed as void* (NULL = the default stream).  All calls are asynchronous with respect to the
+ *     host and can be captured into a CUDA graph (none synchronises, none allocates).
+ *   - Return value: PRECC_OK or an error code.  On a host-detected error nothing is launched and no
+ *     output is touched.  Text for the last error of a context: precc_last_error().
+ *   - A context may be used from one host thread at a time.
+ *
+ * HBM layouts (PRECC_PAGE = 16 tokens per block; token slot s lives in block s / 16 at offset s % 16)
+ *   base K, base V : [n_blocks][n_kv_heads][16][head_dim]
+ *   LR K, LR V     : [n_agents][n_blocks][16][rank]          (one row per token, shared by all kv heads)
+ *   q, out         : [rows][n_q_heads][head_dim]
+ *   B_k, B_v       : [n_agents][rank][n_kv_heads*head_dim]   (the paper's B_i, r x d_out)
+ *   packed A       : [n_agents*(rank_k+rank_v)][d_model]      rows ordered [projection K,V][agent][r]
+ *   packed W       : [2*n_kv_heads*head_dim][d_model]         rows ordered [projection K,V][kv head][c]
+ *   A "contiguous" cache is the same layout addressed without a block table (logical block i of a
+ *   sequence = physical block first_block + i).
+ *
+ * Supported shapes (anything else returns PRECC_ERR_UNSUPPORTED):
+ *   head_dim in {64,128}; n_q_heads % n_kv_heads == 0 with group size <= 8;
+ *   (rank_k, rank_v) in {(0,0), (0,r), (r,r)} with r in {8,16,32,64}; d_model % 64 == 0;
+ *   n_agents <= 64.
+ */
+#ifndef PRECC_H_
+#define PRECC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PRECC_PAGE 16
+
+enum {
+  PRECC_OK = 0,
+  PRECC_ERR_INVALID_ARG = 1,   /* null pointer, negative size, inconsistent sizes */
+  PRECC_ERR_UNSUPPORTED = 2,   /* shape outside the supported set above */
+  PRECC_ERR_MISALIGNED = 3,    /* a tensor pointer is not 16-byte aligned */
+  PRECC_ERR_WORKSPACE = 4,     /* workspace missing or too small */
+  PRECC_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed (text in precc_last_error) */
+  PRECC_ERR_DEVICE_STATUS = 6  /* a kernel recorded a problem (see precc_poll_status) */
+};
+
+/* Bits of the device status word read by precc_poll_status(). */
+#define PRECC_STATUS_BAD_INDEX 1u /* an agent id / block id / slot was out of range and was skipped  */
+#define PRECC_STATUS_TIMEOUT 2u   /* a bounded wait inside a kernel expired (results are invalid)    */
+
+typedef struct precc_ctx precc_ctx;
+
+/* One decoder layer's KV-path geometry (host struct, read during the call only). */
+typedef struct {
+  int32_t d_model;
+  int32_t n_q_heads, n_kv_heads, head_dim;
+  int32_t n_agents;
+  int32_t rank_k, rank_v;      /* 0 = that projection carries no adapter (the paper's default adapts Q,V: rank_k = 0) */
+  float lora_scale_k;          /* s for the key side; 1.0 is Eq. 1 literally */
+  float lora_scale_v;          /* s for the value side */
+  float softmax_scale;         /* <= 0 selects 1/sqrt(head_dim) */
+} precc_layer_desc;
+
+/* Caller-owned caches of one layer (device pointers, layouts above). lr_k / lr_v may be NULL when
+ * the corresponding rank is 0. */
+typedef struct {
+  void* k_base;
+  void* v_base;
+  void* lr_k;
+  void* lr_v;
+  int64_t n_blocks;            /* physical blocks in each of the four arrays */
+} precc_cache;
+
+/* Create a context for CUDA device `device` (host allocation only, plus a 4-byte device status
+ * word obtained with cudaMalloc here and released in precc_destroy). */
+int32_t precc_create(precc_ctx** out, int32_t device);
+int32_t precc_destroy(precc_ctx* ctx);
+/* Text of the last error seen by `ctx` (owned by ctx, valid until the next call on it). */
+const char* precc_last_error(const precc_ctx* ctx);
+const char* precc_error_name(int32_t code);
+/* Number of SMs of the context's device (the split schedule of decode depends on it). */
+int32_t precc_sm_count(const precc_ctx* ctx);
+
+/* Read the device status word accumulated by kernels launched through `ctx`, then clear it.
+ * Synchronises `stream`.  *status_out receives an OR of PRECC_STATUS_* bits.  Returns PRECC_OK when the
+ * word is zero, PRECC_ERR_DEVICE_STATUS otherwise. */
+int32_t precc_poll_status(precc_ctx* ctx, void* stream, uint32_t* status_out);
+
+/* Transpose-pack a row-major [d_model][n_cols] matrix (paper layout d_in x d_out) into rows
+ * [dst_row0, dst_row0 + n_cols) of a [dst_rows][d_model] matrix, i.e. dst[dst_row0 + c][i] = src[i][c].
+ * Used to build the packed A (all agents' down-projections side by side, Section 3.1) and the
+ * packed W.  src, dst device; d_model % 8 == 0. */
+int32_t precc_pack_kmajor(precc_ctx* ctx, const void* src, int32_t d_model, int32_t n_cols,
+                          void* dst, int32_t dst_rows, int32_t dst_row0, void* stream);
+
+/* LR-cache precompute (Section 3.1, PreLRShared): L_k^p = H A_k^p for every agent k whose bit is set
+ * in agent_mask and both projections p, written to the LR caches at the tokens' slots.
+ *   H            [M][d_model]
+ *   A_packed     [n_agents*(rank_k+rank_v)][d_model]  (precc_pack_kmajor output)
+ *   slot_mapping [M] physical token slots, or NULL for slots start_slot .. start_slot+M-1
+ *   agent_mask   bit k = write agent k (all agents: PreLRShared; all but the current one: the
+ *                adapter-free pass of ReBaseShared; only the current one: its adapted pass)
+ * Slots outside [0, 16*n_blocks) are skipped and PRECC_STATUS_BAD_INDEX is recorded.  M == 0 is a no-op. */
+int32_t precc_lr_precompute(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
+                            const void* A_packed, const int32_t* slot_mapping, int64_t start_slot,
+                            uint64_t agent_mask, const precc_cache* cache, void* stream);
+
+/* Base-cache (re-)projection (Section 3.2, ReBaseShared; also the in-turn append): K_base[slot] = H W_k,
+ * V_base[slot] = H W_v for each of the M rows; existing slots are overwritten.
+ *   H [M][d_model];  W_packed [2*n_kv_heads*head_dim][d_model];  slot_mapping / start_slot as above. */
+int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
+                             const void* W_packed, const int32_t* slot_mapping, int64_t start_slot,
+                             const precc_cache* cache, void* stream);
+
+/* Workspace size for precc_lr_attend_decode with at most max_batch requests of at most max_ctx tokens
+ * on a device with `sm_count` SMs.  The workspace must be zeroed once (precc_workspace_init) before its
+ * first use; calls leave it ready for the next call.  Two calls that may run concurrently need
+ * separate workspaces. */
+size_t precc_decode_workspace_bytes(const precc_layer_desc* desc, int32_t max_batch, int32_t max_ctx,
+                                    int32_t sm_count);
+int32_t precc_workspace_init(precc_ctx* ctx, void* workspace, size_t workspace_bytes, void* stream);
+
+/* LR-reconstructed decode attention (Sections 3.1, 4.1): for request b with agent a = agent_id[b] and
+ * every q head h (kv head g = h / (n_q_heads/n_kv_heads)):
+ *   z_t  = softmax_scale * ( q_h . K_base[t,g] + s_k (q_h B^K_{a,g}^T) . L^K_a[t] ),   t < ctx_len[b]
+ *   out_h = sum_t softmax(z)_t V_base[t,g] + s_v (sum_t softmax(z)_t L^V_a[t]) B^V_{a,g}
+ * which equals plain attention with K_a = K_base + s_k L^K_a B^K_a and V_a likewise (Eq. 1).
+ *   q, out        [B][n_q_heads][head_dim]
+ *   agent_id      [B] in [0, n_agents);  ctx_len [B] >= 1 (a request with ctx_len < 1 gets zeros)
+ *   block_table   [B][table_stride] logical block -> physical block, or NULL
+ *   first_block   [B] physical block of logical block 0 when block_table is NULL (NULL = 0 for all)
+ *   max_ctx       HOST upper bound on every ctx_len[b]; with B and the SM count it fixes the split of
+ *                 the context across thread blocks, so results are bit-identical for any block
+ *                 placement given the same (B, max_ctx)
+ *   B_k, B_v      [n_agents][rank][n_kv_heads*head_dim]
+ * B == 0 is a no-op. */
+int32_t precc_lr_attend_decode(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,
+                               const int32_t* agent_id, const int32_t* ctx_len,
+                               const int32_t* block_table, int32_t table_stride,
+                               const int32_t* first_block, int32_t max_ctx,
+                               const void* B_k, const void* B_v, const precc_cache* cache,
+                               void* out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* LR-reconstructed attention for the S new tokens of a turn (Section 3.1: the current agent computes
+ * only over the newly added context and reuses base + own LR cache for the rest).  The caches must
+ * already cover the new tokens (precc_rebase_project + precc_lr_precompute on them first).  Query i
+ * (0 <= i < S) attends logical positions 0 .. ctx_len + i: the old context fully, the new tokens
+ * causally.  Same formula as decode.
+ *   q, out       [S][n_q_heads][head_dim]
+ *   agent        the current agent (host value);  ctx_len  T, tokens before the new ones (host value)
+ *   block_table  [table_stride] logical -> physical block for this sequence, or NULL
+ *   first_block  physical block of logical block 0 when block_table is NULL
+ * No workspace is needed.  S == 0 is a no-op. */
+int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S,
+                                int32_t agent, int32_t ctx_len, const int32_t* block_table,
+                                int32_t table_stride, int32_t first_block,
+                                const void* B_k, const void* B_v, const precc_cache* cache,
+                                void* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRECC_H_ */

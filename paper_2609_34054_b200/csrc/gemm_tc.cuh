@@ -1,0 +1,225 @@
+// Skinny projection GEMM on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
+//
+//   C[M, N_out] = X[M, K] . Wt[N_out, K]^T        (both operands K-major bf16, fp32 accumulate)
+//
+// with a scatter epilogue that writes bf16 rows straight into the paged caches:
+//   mode 0  LR precompute (Section 3.1):  column -> (projection, agent, r index), LR cache rows
+//   mode 1  base projection (Section 3.2): column -> (projection, kv head, c), base cache rows
+//
+// One 128 x BN output tile per thread block.  Warp roles: warp 0 = TMA producer (one lane),
+// warp 1 = TMEM owner + MMA issuer (one lane), warps 2..5 = epilogue (one TMEM lane = one row each).
+// A STAGES-deep ring of {X tile 128x64, Wt tile BNx64} in 128-byte-swizzled shared memory is handed
+// from producer to issuer with mbarriers; tcgen05.commit releases a stage when its MMAs have read it.
+// Every wait is bounded: on expiry the waiter records PRECC_STATUS_TIMEOUT and carries on, so the
+// kernel always terminates and frees its TMEM.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace precc {
+
+struct GemmParams {
+  int M, N_out, K;
+  int BN, stages, tmem_cols;
+  int mode;                       // 0 = LR caches, 1 = base caches
+  const int32_t* slot_mapping;    // [M] or null
+  int64_t start_slot;
+  int64_t n_blocks;
+  __nv_bfloat16* dst0;            // lr_k or k_base
+  __nv_bfloat16* dst1;            // lr_v or v_base
+  int n_agents, rank_k, rank_v;
+  unsigned long long agent_mask;
+  int n_kv, hd;
+  uint32_t* status;
+};
+
+constexpr int GEMM_BM = 128;
+constexpr int GEMM_BK = 64;                 // 64 bf16 = one 128-byte swizzle row
+constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait (about a second of SM clock).  Returns false after recording a timeout.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (clock64() - t0 > 2000000000LL) break;
+  }
+  atomicOr(status, StatusBits::TIMEOUT);
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
+// 1024 bytes apart (start >> 4 | LBO(ignored) | SBO = 1024 >> 4 | version 1 | layout SWIZZLE_128B).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(GEMM_BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const GemmParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  // 1024-byte alignment for the 128-byte swizzle atoms
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  const int b_bytes = p.BN * GEMM_BK * 2;
+  const int stage_bytes = GEMM_A_BYTES + b_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes);
+  const uint32_t full0 = smem_u32(bars);
+  const uint32_t empty0 = full0 + 8 * p.stages;
+  const uint32_t tfull = empty0 + 8 * p.stages;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * p.stages + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * GEMM_BM, n0 = blockIdx.y * p.BN;
+  const int nkb = p.K / GEMM_BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(tfull, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_holder)), "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = *tmem_holder;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb % p.stages;
+        if (kb >= p.stages) mbar_wait(empty0 + 8 * s, ((kb / p.stages) - 1) & 1, p.status);
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        mbar_expect_tx(full0 + 8 * s, stage_bytes);
+        tma_load_2d(sa, &map_x, kb * GEMM_BK, m0, full0 + 8 * s);
+        tma_load_2d(sa + GEMM_A_BYTES, &map_w, kb * GEMM_BK, n0, full0 + 8 * s);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(p.BN);
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb % p.stages;
+        mbar_wait(full0 + 8 * s, (kb / p.stages) & 1, p.status);
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + GEMM_A_BYTES);
+#pragma unroll
+        for (int k = 0; k < GEMM_BK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
+          umma_bf16(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
+        umma_commit(empty0 + 8 * s);             // stage reusable once these MMAs have read it
+      }
+      umma_commit(tfull);                        // accumulator complete
+    }
+  } else {
+    // ---- epilogue: TMEM lane = tile row; this warp may touch lanes 32*(warp%4) .. +31
+    const int lane_base = (warp & 3) * 32;
+    const int row = lane_base + lane;
+    const int gm = m0 + row;
+    bool row_ok = gm < p.M;
+    long long slot = 0;
+    if (row_ok) {
+      slot = p.slot_mapping ? (long long)p.slot_mapping[gm] : p.start_slot + gm;
+      if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
+    }
+    const long long blk = slot / PAGE;
+    const int off = (int)(slot % PAGE);
+    mbar_wait(tfull, 0, p.status);
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const int n_k = p.n_agents * p.rank_k;
+    const int w = p.n_kv * p.hd;
+    for (int c0 = 0; c0 < p.BN; c0 += 16) {
+      uint32_t r[16];
+      tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + c0, r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int gc = n0 + c0 + 8 * h;
+        if (!row_ok || gc >= p.N_out) continue;
+        __nv_bfloat16* dst;
+        if (p.mode == 0) {
+          const bool is_v = gc >= n_k;
+          const int rr = is_v ? p.rank_v : p.rank_k;
+          const int cc = is_v ? gc - n_k : gc;
+          const int agent = cc / rr, ri = cc % rr;
+          if (!((p.agent_mask >> agent) & 1ull)) continue;
+          dst = (is_v ? p.dst1 : p.dst0) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
+        } else {
+          const bool is_v = gc >= w;
+          const int cc = is_v ? gc - w : gc;
+          const int g = cc / p.hd, c = cc % p.hd;
+          dst = (is_v ? p.dst1 : p.dst0) + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
+        }
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(r[8 * h + 0]), __uint_as_float(r[8 * h + 1]));
+        v.y = pack_bf16(__uint_as_float(r[8 * h + 2]), __uint_as_float(r[8 * h + 3]));
+        v.z = pack_bf16(__uint_as_float(r[8 * h + 4]), __uint_as_float(r[8 * h + 5]));
+        v.w = pack_bf16(__uint_as_float(r[8 * h + 6]), __uint_as_float(r[8 * h + 7]));
+        *reinterpret_cast<uint4*>(dst) = v;
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+  }
+}
+
+}  // namespace precc

@@ -1,0 +1,461 @@
+// C-ABI entry points of libprecc: argument validation, launch configuration, kernel dispatch.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/precc.h"
+#include "decode.cuh"
+#include "gemm_tc.cuh"
+#include "prefill.cuh"
+
+using namespace precc;
+
+struct precc_ctx {
+  int device = 0;
+  int sm_count = 0;
+  int max_smem_optin = 0;
+  uint32_t* status = nullptr;          // device status word
+  char err[512] = {0};
+  CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                           const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                           CUtensorMapL2promotion, CUtensorMapFloatOOBfill) = nullptr;
+};
+
+namespace {
+
+int32_t fail(precc_ctx* ctx, int32_t code, const char* fmt, ...) {
+  if (ctx) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+#define PRECC_CUDA(ctx, expr)                                                                   \
+  do {                                                                                          \
+    cudaError_t e__ = (expr);                                                                   \
+    if (e__ != cudaSuccess) return fail(ctx, PRECC_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool rank_ok(int r) { return r == 8 || r == 16 || r == 32 || r == 64; }
+
+int32_t check_desc(precc_ctx* ctx, const precc_layer_desc* d) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!d) return fail(ctx, PRECC_ERR_INVALID_ARG, "layer descriptor is null");
+  if (d->d_model <= 0 || d->n_q_heads <= 0 || d->n_kv_heads <= 0 || d->n_agents <= 0 || d->rank_k < 0 || d->rank_v < 0)
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "non-positive size in layer descriptor");
+  if (d->head_dim != 64 && d->head_dim != 128) return fail(ctx, PRECC_ERR_UNSUPPORTED, "head_dim %d not in {64,128}", d->head_dim);
+  if (d->n_q_heads % d->n_kv_heads) return fail(ctx, PRECC_ERR_UNSUPPORTED, "n_q_heads %% n_kv_heads != 0");
+  if (d->n_q_heads / d->n_kv_heads > 8) return fail(ctx, PRECC_ERR_UNSUPPORTED, "group size %d > 8", d->n_q_heads / d->n_kv_heads);
+  if (d->d_model % 64) return fail(ctx, PRECC_ERR_UNSUPPORTED, "d_model %d not a multiple of 64", d->d_model);
+  if (d->n_agents > 64) return fail(ctx, PRECC_ERR_UNSUPPORTED, "n_agents %d > 64", d->n_agents);
+  const int rk = d->rank_k, rv = d->rank_v;
+  const bool combo = (rk == 0 && rv == 0) || (rk == 0 && rank_ok(rv)) || (rk == rv && rank_ok(rv));
+  if (!combo) return fail(ctx, PRECC_ERR_UNSUPPORTED, "ranks (%d,%d) not in {(0,0),(0,r),(r,r)}, r in {8,16,32,64}", rk, rv);
+  return PRECC_OK;
+}
+
+int32_t check_cache(precc_ctx* ctx, const precc_layer_desc* d, const precc_cache* c, bool need_base, bool need_lr) {
+  if (!c) return fail(ctx, PRECC_ERR_INVALID_ARG, "cache is null");
+  if (c->n_blocks <= 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "cache.n_blocks must be positive");
+  if (c->n_blocks > (int64_t)1 << 26) return fail(ctx, PRECC_ERR_UNSUPPORTED, "cache.n_blocks too large");
+  if (need_base && (!c->k_base || !c->v_base)) return fail(ctx, PRECC_ERR_INVALID_ARG, "base cache pointer is null");
+  if (need_lr && ((d->rank_k > 0 && !c->lr_k) || (d->rank_v > 0 && !c->lr_v))) return fail(ctx, PRECC_ERR_INVALID_ARG, "LR cache pointer is null");
+  if (!aligned16(c->k_base) || !aligned16(c->v_base) || !aligned16(c->lr_k) || !aligned16(c->lr_v))
+    return fail(ctx, PRECC_ERR_MISALIGNED, "cache pointer not 16-byte aligned");
+  return PRECC_OK;
+}
+
+float softmax_scale_log2(const precc_layer_desc* d) {
+  const float sc = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / std::sqrt((float)d->head_dim);
+  return sc * 1.4426950408889634f;
+}
+
+// ------------------------------------------------------------------------------------------ pack
+__global__ void pack_kmajor_kernel(const __nv_bfloat16* __restrict__ src, int d, int n, __nv_bfloat16* __restrict__ dst, int row0) {
+  __shared__ __nv_bfloat16 tile[32][33];
+  const int c0 = blockIdx.x * 32, i0 = blockIdx.y * 32;
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int i = i0 + r, c = c0 + threadIdx.x;
+    tile[r][threadIdx.x] = (i < d && c < n) ? src[(size_t)i * n + c] : __float2bfloat16(0.f);
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int c = c0 + r, i = i0 + threadIdx.x;
+    if (c < n && i < d) dst[(size_t)(row0 + c) * d + i] = tile[threadIdx.x][r];
+  }
+}
+
+// ------------------------------------------------------------------------------------ GEMM launch
+int32_t make_map(precc_ctx* ctx, CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)GEMM_BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, PRECC_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  return PRECC_OK;
+}
+
+int pick_bn(int n_out, int m_tiles, int sm_count) {
+  if (n_out <= 256) return (n_out + 15) / 16 * 16;
+  const int cands[3] = {256, 128, 64};
+  for (int bn : cands)
+    if ((long long)m_tiles * ((n_out + bn - 1) / bn) >= sm_count) return bn;
+  return 64;
+}
+
+int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
+  const int m_tiles = (M + GEMM_BM - 1) / GEMM_BM;
+  const int bn = pick_bn(n_out, m_tiles, ctx->sm_count);
+  const int n_tiles = (n_out + bn - 1) / bn;
+  const int stage_bytes = GEMM_A_BYTES + bn * GEMM_BK * 2;
+  int stages = (ctx->max_smem_optin - 4096) / stage_bytes;
+  if (stages > 8) stages = 8;
+  if (stages > K / GEMM_BK) stages = K / GEMM_BK;
+  if (stages < 1) return fail(ctx, PRECC_ERR_CUDA, "not enough shared memory for one GEMM stage");
+  int tmem_cols = 32;
+  while (tmem_cols < bn) tmem_cols <<= 1;
+  const size_t smem = (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 1024;
+  CUtensorMap map_x, map_w;
+  int32_t rc = make_map(ctx, &map_x, X, M, K, GEMM_BM);
+  if (rc) return rc;
+  rc = make_map(ctx, &map_w, Wt, n_out, K, bn);
+  if (rc) return rc;
+  gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
+  gp.status = ctx->status;
+  PRECC_CUDA(ctx, cudaFuncSetAttribute(proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  proj_gemm_kernel<<<dim3(m_tiles, n_tiles), GEMM_THREADS, smem, stream>>>(map_x, map_w, gp);
+  PRECC_CUDA(ctx, cudaGetLastError());
+  return PRECC_OK;
+}
+
+// ---------------------------------------------------------------------------- attention dispatch
+template <template <int, int, int> class F, typename... Args>
+int32_t dispatch_shape(precc_ctx* ctx, int hd, int rk, int rv, Args&&... args) {
+#define PRECC_CASE(HD, RK, RV) \
+  if (hd == HD && rk == RK && rv == RV) return F<HD, RK, RV>::run(ctx, args...);
+#define PRECC_RANKS(HD)                                                                              \
+  PRECC_CASE(HD, 0, 0) PRECC_CASE(HD, 0, 8) PRECC_CASE(HD, 0, 16) PRECC_CASE(HD, 0, 32) PRECC_CASE(HD, 0, 64) \
+  PRECC_CASE(HD, 8, 8) PRECC_CASE(HD, 16, 16) PRECC_CASE(HD, 32, 32) PRECC_CASE(HD, 64, 64)
+  PRECC_RANKS(64)
+  PRECC_RANKS(128)
+#undef PRECC_RANKS
+#undef PRECC_CASE
+  return fail(ctx, PRECC_ERR_UNSUPPORTED, "no kernel for head_dim %d ranks (%d,%d)", hd, rk, rv);
+}
+
+// Split schedule of decode: pages per thread block and blocks per (request, kv head).
+struct DecodePlan { int chunk_tiles, max_splits, stages, smem; };
+
+template <int HD, int RK, int RV>
+DecodePlan plan_decode(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
+  using C = DecodeCfg<HD, RK, RV>;
+  DecodePlan pl;
+  // ring depth: as deep as possible (<= 4) while two blocks still fit on an SM
+  int stages = 4;
+  while (stages > 2 && 2 * (C::smem_bytes(stages) + 1024) > max_smem) --stages;
+  pl.stages = stages;
+  pl.smem = C::smem_bytes(stages);
+  const int per_sm = (2 * (pl.smem + 1024) <= max_smem) ? 2 : 1;
+  const long long slots = (long long)sm_count * per_sm;
+  const int max_tiles = (max_ctx + PAGE - 1) / PAGE;
+  const long long units = (long long)B * n_kv;
+  // blocks per (request, kv head): fill the machine once; with plenty of work use 4 waves of
+  // blocks so that requests of different length balance out
+  long long want = (slots + units - 1) / units;
+  const long long total_tiles = units * max_tiles;
+  if (total_tiles >= slots * 4 * 64) want = (4 * slots + units - 1) / units;
+  int chunk = (int)((max_tiles + want - 1) / want);
+  if (chunk < DEC_WARPS) chunk = DEC_WARPS;
+  pl.chunk_tiles = chunk;
+  pl.max_splits = (max_tiles + chunk - 1) / chunk;
+  return pl;
+}
+
+struct DecodeArgs {
+  const precc_layer_desc* d; const void* q; int B; const int32_t* agent_id; const int32_t* ctx_len;
+  const int32_t* block_table; int table_stride; const int32_t* first_block; int max_ctx;
+  const void* B_k; const void* B_v; const precc_cache* cache; void* out; void* ws; size_t ws_bytes; cudaStream_t stream;
+};
+
+template <int HD, int RK, int RV>
+struct DecodeRun {
+  static size_t ws_bytes(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
+    const DecodePlan pl = plan_decode<HD, RK, RV>(sm_count, max_smem, B, n_kv, max_ctx);
+    const size_t tickets = ((size_t)B * n_kv * 4 + 255) / 256 * 256;
+    return tickets + (size_t)B * n_kv * pl.max_splits * DecodeCfg<HD, RK, RV>::PART_STRIDE * 4;
+  }
+  static int32_t run(precc_ctx* ctx, const DecodeArgs& a) {
+    const precc_layer_desc* d = a.d;
+    const DecodePlan pl = plan_decode<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
+    const size_t need = ws_bytes(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
+    if (!a.ws || a.ws_bytes < need) return fail(ctx, PRECC_ERR_WORKSPACE, "decode workspace: need %zu bytes, got %zu", need, a.ws_bytes);
+    DecodeParams p;
+    p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out;
+    p.agent_id = a.agent_id; p.ctx_len = a.ctx_len; p.block_table = a.block_table; p.first_block = a.first_block;
+    p.k_base = (const __nv_bfloat16*)a.cache->k_base; p.v_base = (const __nv_bfloat16*)a.cache->v_base;
+    p.lr_k = (const __nv_bfloat16*)a.cache->lr_k; p.lr_v = (const __nv_bfloat16*)a.cache->lr_v;
+    p.B_k = (const __nv_bfloat16*)a.B_k; p.B_v = (const __nv_bfloat16*)a.B_v;
+    const size_t tickets = ((size_t)a.B * d->n_kv_heads * 4 + 255) / 256 * 256;
+    p.tickets = (int32_t*)a.ws;
+    p.part = (float*)((char*)a.ws + tickets);
+    p.status = ctx->status;
+    p.n_blocks = a.cache->n_blocks; p.table_stride = a.table_stride;
+    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = d->n_q_heads / d->n_kv_heads; p.n_agents = d->n_agents;
+    p.chunk_tiles = pl.chunk_tiles; p.max_splits = pl.max_splits; p.stages = pl.stages;
+    p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
+    auto kern = lr_attend_decode_kernel<HD, RK, RV>;
+    PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem));
+    kern<<<dim3(pl.max_splits, d->n_kv_heads, a.B), DEC_THREADS, pl.smem, a.stream>>>(p);
+    PRECC_CUDA(ctx, cudaGetLastError());
+    return PRECC_OK;
+  }
+};
+
+struct PrefillArgs {
+  const precc_layer_desc* d; const void* q; int S; int agent; int T; const int32_t* block_table; int first_block;
+  const void* B_k; const void* B_v; const precc_cache* cache; void* out; cudaStream_t stream;
+};
+
+template <int HD, int RK, int RV>
+struct PrefillRun {
+  static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
+    using C = PrefillCfg<HD, RK, RV>;
+    const precc_layer_desc* d = a.d;
+    int stages = 3;
+    while (stages > 2 && 2 * (C::smem_bytes(stages) + 1024) > ctx->max_smem_optin) --stages;
+    const int smem = C::smem_bytes(stages);
+    PrefillParams p;
+    const size_t kvw = (size_t)d->n_kv_heads * HD;
+    p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;
+    p.k_base = (const __nv_bfloat16*)a.cache->k_base; p.v_base = (const __nv_bfloat16*)a.cache->v_base;
+    p.lr_k = RK ? (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * a.cache->n_blocks * PAGE * RK : nullptr;
+    p.lr_v = RV ? (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * a.cache->n_blocks * PAGE * RV : nullptr;
+    p.B_k = RK ? (const __nv_bfloat16*)a.B_k + (size_t)a.agent * RK * kvw : nullptr;
+    p.B_v = RV ? (const __nv_bfloat16*)a.B_v + (size_t)a.agent * RV * kvw : nullptr;
+    p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
+    p.S = a.S; p.T = a.T; p.first_block = a.first_block;
+    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = d->n_q_heads / d->n_kv_heads; p.stages = stages;
+    p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
+    auto kern = lr_attend_prefill_kernel<HD, RK, RV>;
+    PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int row_tiles = (a.S * p.group + PF_ROWS - 1) / PF_ROWS;
+    kern<<<dim3(row_tiles, d->n_kv_heads), PF_THREADS, smem, a.stream>>>(p);
+    PRECC_CUDA(ctx, cudaGetLastError());
+    return PRECC_OK;
+  }
+};
+
+struct WsQuery { int sm_count, max_smem, B, n_kv, max_ctx; size_t* out; };
+template <int HD, int RK, int RV>
+struct DecodeWs {
+  static int32_t run(precc_ctx*, const WsQuery& w) {
+    *w.out = DecodeRun<HD, RK, RV>::ws_bytes(w.sm_count, w.max_smem, w.B, w.n_kv, w.max_ctx);
+    return PRECC_OK;
+  }
+};
+
+}  // namespace
+
+// =========================================================================================== ABI
+extern "C" {
+
+int32_t precc_create(precc_ctx** out, int32_t device) {
+  if (!out) return PRECC_ERR_INVALID_ARG;
+  *out = nullptr;
+  precc_ctx* ctx = new (std::nothrow) precc_ctx();
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  ctx->device = device;
+  cudaError_t e = cudaSetDevice(device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->status, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
+  if (e == cudaSuccess) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e == cudaSuccess && (qres != cudaDriverEntryPointSuccess || !fn)) e = cudaErrorUnknown;
+    ctx->encode_tiled = reinterpret_cast<decltype(ctx->encode_tiled)>(fn);
+  }
+  if (e != cudaSuccess) {
+    fprintf(stderr, "precc_create: %s\n", cudaGetErrorString(e));
+    if (ctx->status) cudaFree(ctx->status);
+    delete ctx;
+    return PRECC_ERR_CUDA;
+  }
+  *out = ctx;
+  return PRECC_OK;
+}
+
+int32_t precc_destroy(precc_ctx* ctx) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (ctx->status) cudaFree(ctx->status);
+  delete ctx;
+  return PRECC_OK;
+}
+
+const char* precc_last_error(const precc_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+const char* precc_error_name(int32_t code) {
+  switch (code) {
+    case PRECC_OK: return "PRECC_OK";
+    case PRECC_ERR_INVALID_ARG: return "PRECC_ERR_INVALID_ARG";
+    case PRECC_ERR_UNSUPPORTED: return "PRECC_ERR_UNSUPPORTED";
+    case PRECC_ERR_MISALIGNED: return "PRECC_ERR_MISALIGNED";
+    case PRECC_ERR_WORKSPACE: return "PRECC_ERR_WORKSPACE";
+    case PRECC_ERR_CUDA: return "PRECC_ERR_CUDA";
+    case PRECC_ERR_DEVICE_STATUS: return "PRECC_ERR_DEVICE_STATUS";
+    default: return "PRECC_ERR_?";
+  }
+}
+
+int32_t precc_sm_count(const precc_ctx* ctx) { return ctx ? ctx->sm_count : 0; }
+
+int32_t precc_poll_status(precc_ctx* ctx, void* stream, uint32_t* status_out) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint32_t h = 0;
+  PRECC_CUDA(ctx, cudaMemcpyAsync(&h, ctx->status, sizeof(h), cudaMemcpyDeviceToHost, st));
+  PRECC_CUDA(ctx, cudaMemsetAsync(ctx->status, 0, sizeof(h), st));
+  PRECC_CUDA(ctx, cudaStreamSynchronize(st));
+  if (status_out) *status_out = h;
+  if (h) return fail(ctx, PRECC_ERR_DEVICE_STATUS, "device status 0x%x%s%s", h, (h & PRECC_STATUS_BAD_INDEX) ? " bad-index" : "",
+                     (h & PRECC_STATUS_TIMEOUT) ? " timeout" : "");
+  return PRECC_OK;
+}
+
+int32_t precc_pack_kmajor(precc_ctx* ctx, const void* src, int32_t d_model, int32_t n_cols, void* dst, int32_t dst_rows,
+                          int32_t dst_row0, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (n_cols == 0) return PRECC_OK;
+  if (!src || !dst || d_model <= 0 || n_cols < 0 || dst_row0 < 0 || dst_row0 + n_cols > dst_rows)
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "pack_kmajor: bad arguments");
+  if (d_model % 8) return fail(ctx, PRECC_ERR_UNSUPPORTED, "pack_kmajor: d_model %% 8 != 0");
+  dim3 grid((n_cols + 31) / 32, (d_model + 31) / 32), block(32, 8);
+  pack_kmajor_kernel<<<grid, block, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)src, d_model, n_cols, (__nv_bfloat16*)dst, dst_row0);
+  PRECC_CUDA(ctx, cudaGetLastError());
+  return PRECC_OK;
+}
+
+int32_t precc_lr_precompute(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* A_packed,
+                            const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_cache* cache,
+                            void* stream) {
+  int32_t rc = check_desc(ctx, desc);
+  if (rc) return rc;
+  if (M < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "M < 0");
+  const int n_out = desc->n_agents * (desc->rank_k + desc->rank_v);
+  if (M == 0 || n_out == 0) return PRECC_OK;
+  rc = check_cache(ctx, desc, cache, false, true);
+  if (rc) return rc;
+  if (!H || !A_packed) return fail(ctx, PRECC_ERR_INVALID_ARG, "H or A_packed is null");
+  if (!aligned16(H) || !aligned16(A_packed)) return fail(ctx, PRECC_ERR_MISALIGNED, "H / A_packed not 16-byte aligned");
+  if (!slot_mapping && (start_slot < 0 || start_slot + M > cache->n_blocks * PRECC_PAGE))
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "slots [%lld, %lld) outside the cache", (long long)start_slot, (long long)start_slot + M);
+  GemmParams gp{};
+  gp.mode = 0; gp.slot_mapping = slot_mapping; gp.start_slot = start_slot; gp.n_blocks = cache->n_blocks;
+  gp.dst0 = (__nv_bfloat16*)cache->lr_k; gp.dst1 = (__nv_bfloat16*)cache->lr_v;
+  gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = agent_mask;
+  gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
+  return launch_gemm(ctx, H, M, desc->d_model, A_packed, n_out, gp, (cudaStream_t)stream);
+}
+
+int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* W_packed,
+                             const int32_t* slot_mapping, int64_t start_slot, const precc_cache* cache, void* stream) {
+  int32_t rc = check_desc(ctx, desc);
+  if (rc) return rc;
+  if (M < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "M < 0");
+  if (M == 0) return PRECC_OK;
+  rc = check_cache(ctx, desc, cache, true, false);
+  if (rc) return rc;
+  if (!H || !W_packed) return fail(ctx, PRECC_ERR_INVALID_ARG, "H or W_packed is null");
+  if (!aligned16(H) || !aligned16(W_packed)) return fail(ctx, PRECC_ERR_MISALIGNED, "H / W_packed not 16-byte aligned");
+  if (!slot_mapping && (start_slot < 0 || start_slot + M > cache->n_blocks * PRECC_PAGE))
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "slots [%lld, %lld) outside the cache", (long long)start_slot, (long long)start_slot + M);
+  GemmParams gp{};
+  gp.mode = 1; gp.slot_mapping = slot_mapping; gp.start_slot = start_slot; gp.n_blocks = cache->n_blocks;
+  gp.dst0 = (__nv_bfloat16*)cache->k_base; gp.dst1 = (__nv_bfloat16*)cache->v_base;
+  gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = ~0ull;
+  gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
+  return launch_gemm(ctx, H, M, desc->d_model, W_packed, 2 * desc->n_kv_heads * desc->head_dim, gp, (cudaStream_t)stream);
+}
+
+size_t precc_decode_workspace_bytes(const precc_layer_desc* desc, int32_t max_batch, int32_t max_ctx, int32_t sm_count) {
+  if (!desc || max_batch <= 0 || max_ctx <= 0 || sm_count <= 0) return 0;
+  size_t out = 0;
+  // the ring depth depends on the opt-in shared memory of the device; sm_100 offers 227 KB
+  WsQuery w{sm_count, 232448, max_batch, desc->n_kv_heads, max_ctx, &out};
+  precc_ctx tmp;
+  if (dispatch_shape<DecodeWs>(&tmp, desc->head_dim, desc->rank_k, desc->rank_v, w) != PRECC_OK) return 0;
+  return out;
+}
+
+int32_t precc_workspace_init(precc_ctx* ctx, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes == 0) return fail(ctx, PRECC_ERR_WORKSPACE, "workspace is null or empty");
+  PRECC_CUDA(ctx, cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream));
+  return PRECC_OK;
+}
+
+int32_t precc_lr_attend_decode(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B, const int32_t* agent_id,
+                               const int32_t* ctx_len, const int32_t* block_table, int32_t table_stride,
+                               const int32_t* first_block, int32_t max_ctx, const void* B_k, const void* B_v,
+                               const precc_cache* cache, void* out, void* workspace, size_t workspace_bytes, void* stream) {
+  int32_t rc = check_desc(ctx, desc);
+  if (rc) return rc;
+  if (B < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "B < 0");
+  if (B == 0) return PRECC_OK;
+  rc = check_cache(ctx, desc, cache, true, true);
+  if (rc) return rc;
+  if (!q || !out || !agent_id || !ctx_len) return fail(ctx, PRECC_ERR_INVALID_ARG, "q / out / agent_id / ctx_len is null");
+  if ((desc->rank_k > 0 && !B_k) || (desc->rank_v > 0 && !B_v)) return fail(ctx, PRECC_ERR_INVALID_ARG, "B_k / B_v is null");
+  if (!aligned16(q) || !aligned16(out) || !aligned16(B_k) || !aligned16(B_v) || !aligned16(workspace))
+    return fail(ctx, PRECC_ERR_MISALIGNED, "q / out / B_k / B_v / workspace not 16-byte aligned");
+  if (max_ctx < 1) return fail(ctx, PRECC_ERR_INVALID_ARG, "max_ctx < 1");
+  if (block_table && (long long)table_stride * PRECC_PAGE < max_ctx)
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "block table stride %d too short for max_ctx %d", table_stride, max_ctx);
+  if (B > 65535) return fail(ctx, PRECC_ERR_UNSUPPORTED, "B > 65535");
+  if (ctx->max_smem_optin != 232448) {
+    // the workspace query assumes the sm_100 shared-memory size
+    return fail(ctx, PRECC_ERR_UNSUPPORTED, "device opt-in shared memory %d != 232448 (not an sm_100 part?)", ctx->max_smem_optin);
+  }
+  DecodeArgs a{desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, B_v, cache, out,
+               workspace, workspace_bytes, (cudaStream_t)stream};
+  return dispatch_shape<DecodeRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
+}
+
+int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
+                                int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
+                                const void* B_k, const void* B_v, const precc_cache* cache, void* out, void* stream) {
+  int32_t rc = check_desc(ctx, desc);
+  if (rc) return rc;
+  if (S < 0 || ctx_len < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "S < 0 or ctx_len < 0");
+  if (S == 0) return PRECC_OK;
+  rc = check_cache(ctx, desc, cache, true, true);
+  if (rc) return rc;
+  if (!q || !out) return fail(ctx, PRECC_ERR_INVALID_ARG, "q / out is null");
+  if (agent < 0 || agent >= desc->n_agents) return fail(ctx, PRECC_ERR_INVALID_ARG, "agent %d outside [0,%d)", agent, desc->n_agents);
+  if ((desc->rank_k > 0 && !B_k) || (desc->rank_v > 0 && !B_v)) return fail(ctx, PRECC_ERR_INVALID_ARG, "B_k / B_v is null");
+  if (!aligned16(q) || !aligned16(out) || !aligned16(B_k) || !aligned16(B_v)) return fail(ctx, PRECC_ERR_MISALIGNED, "q / out / B_k / B_v not 16-byte aligned");
+  const long long need_blocks = ((long long)ctx_len + S + PRECC_PAGE - 1) / PRECC_PAGE;
+  if (block_table && table_stride < need_blocks) return fail(ctx, PRECC_ERR_INVALID_ARG, "block table has %d entries, need %lld", table_stride, need_blocks);
+  if (!block_table && (first_block < 0 || first_block + need_blocks > cache->n_blocks))
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "blocks [%d, %lld) outside the cache", first_block, first_block + need_blocks);
+  if ((long long)S * (desc->n_q_heads / desc->n_kv_heads) > (long long)PF_ROWS * 65535) return fail(ctx, PRECC_ERR_UNSUPPORTED, "S too large");
+  PrefillArgs a{desc, q, S, agent, ctx_len, block_table, first_block, B_k, B_v, cache, out, (cudaStream_t)stream};
+  return dispatch_shape<PrefillRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
+}
+
+}  // extern "C"

@@ -1,0 +1,311 @@
+"""GPU parity: the CUDA path (through the C-ABI binding) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lrkv_oracle as O
+from paper_2609_34054_b200 import inputs as I
+from paper_2609_34054_b200.binding import Precc, PreccError
+
+from harness import ATOL, RTOL, Layer, assert_close, base_rows, f64, lr_rows
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def px():
+    p = Precc(0)
+    yield p
+    assert p.poll_status() == 0, "a kernel recorded a device status"
+    p.close()
+
+
+def _ref_decode(L: Layer, H, q, agent_id, ctx_len, heads=None, softmax_scale=None):
+    w, g = L.w_np, L.geo
+    return O.lr_decode_reference(f64(q), agent_id, ctx_len, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"],
+                                 w["B_v"], L.desc.lora_scale_k, L.desc.lora_scale_v, g.n_kv, softmax_scale, heads)
+
+
+def _cache_tol(ref):
+    # one bf16 rounding of an fp32-accumulated value
+    return 2.0 ** -8 * np.abs(ref) + 1e-3
+
+
+# ------------------------------------------------------------------ C1: the whole chain
+
+def test_c1_chain_precompute_rebase_decode(px):
+    geo = I.C1
+    T = I.C1_T
+    L = Layer(px, geo, seed=0, n_blocks=T // 16)
+    H = I.hidden_states(T, geo, seed=0)
+    L.append(H)
+    torch.cuda.synchronize()
+    Hn = f64(H)
+    kb, vb = base_rows(L.cache.k_base), base_rows(L.cache.v_base)
+    rk, rv = O.base_cache(Hn, L.w_np["W_k"]), O.base_cache(Hn, L.w_np["W_v"])
+    assert (np.abs(kb - rk) <= _cache_tol(rk)).all() and (np.abs(vb - rv) <= _cache_tol(rv)).all()
+    for a in range(geo.n_agents):
+        for cache_t, A in ((L.cache.lr_k, L.w_np["A_k"]), (L.cache.lr_v, L.w_np["A_v"])):
+            ref = O.lr_cache(Hn, A[a])
+            assert (np.abs(lr_rows(cache_t, a) - ref) <= _cache_tol(ref)).all()
+    q = I.queries(geo.n_agents, geo, seed=0)
+    agent_id, ctx_len = [0, 1, 2], [T, T, T]
+    out = L.decode(q, agent_id, ctx_len)
+    ref = _ref_decode(L, H, q, agent_id, ctx_len)
+    assert_close(f64(out), ref, "C1 decode")
+    # sensitivity: the adapter term must be visible at this tolerance
+    base_only = O.lr_decode_reference(f64(q), agent_id, ctx_len, Hn, L.w_np["W_k"], L.w_np["W_v"], L.w_np["A_k"],
+                                      L.w_np["B_k"], L.w_np["A_v"], L.w_np["B_v"], 0.0, 0.0, geo.n_kv)
+    assert (np.abs(f64(out) - base_only) > ATOL + RTOL * np.abs(base_only)).any()
+    # peaked variant (larger logits): outputs are O(0.1..1), so the bar bites
+    qp = I.queries(geo.n_agents, geo, seed=0, tag="L0.q.peaked", gain=4.0)
+    assert_close(f64(L.decode(qp, agent_id, ctx_len)), _ref_decode(L, H, qp, agent_id, ctx_len), "C1 decode peaked")
+
+
+SMALL = [
+    # d, n_q, n_kv, hd, N, rk, rv, T, ctx list
+    (256, 8, 2, 128, 3, 8, 8, 100, [100, 1, 37]),
+    (256, 8, 2, 64, 2, 16, 16, 200, [200, 16, 17]),
+    (128, 28, 4, 128, 3, 16, 16, 90, [90, 33, 64]),          # group of 7 (Qwen-like)
+    (192, 8, 8, 64, 2, 0, 0, 50, [50, 49, 2]),               # no adapters: plain attention
+    (192, 16, 4, 128, 2, 0, 32, 77, [77, 5, 48]),            # adapters on V only (paper default QV)
+    (256, 4, 1, 128, 2, 64, 64, 130, [130, 129, 15]),
+    (128, 4, 2, 64, 5, 32, 32, 48, [48, 47, 1]),
+    (128, 2, 2, 64, 2, 0, 8, 33, [33, 32, 31]),
+    (128, 6, 2, 128, 2, 0, 64, 70, [70, 3, 69]),
+]
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: "d%d_q%d_kv%d_hd%d_N%d_r%d-%d_T%d" % c[:8])
+def test_small_shapes_decode_and_prefill(px, cfg):
+    d, n_q, n_kv, hd, N, rk, rv, T, ctxs = cfg
+    geo = I.Geometry(d, n_q, n_kv, hd, N, rk, rv, alpha=2.0 * max(rk, rv, 1))
+    nb = (T + 15) // 16 + 2
+    L = Layer(px, geo, seed=7, n_blocks=nb, fill=float("nan"))   # unwritten slots hold NaN: must never leak
+    H = I.hidden_states(T, geo, seed=7)
+    L.append(H)
+    agent_id = [i % N for i in range(len(ctxs))]
+    q = I.queries(len(ctxs), geo, seed=7, gain=2.0)
+    out = L.decode(q, agent_id, ctxs)
+    assert_close(f64(out), _ref_decode(L, H, q, agent_id, ctxs), "decode")
+    # new-turn prefill: last S tokens are the turn
+    S = min(T - 1, 21)
+    Tc = T - S
+    qs = I.queries(S, geo, seed=7, tag="q.turn", gain=2.0)
+    w = L.w_np
+    for agent in range(min(N, 2)):
+        got = L.prefill(qs, agent, Tc)
+        ref = O.lr_prefill_reference(f64(qs), agent, Tc, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                     L.desc.lora_scale_k, L.desc.lora_scale_v, n_kv)
+        assert_close(f64(got), ref, f"prefill agent {agent}")
+
+
+def test_softmax_scale_and_lora_scales_are_honoured(px):
+    geo = I.Geometry(128, 4, 2, 64, 2, 16, 16, alpha=32.0)
+    H = I.hidden_states(40, geo, seed=3)
+    q = I.queries(2, geo, seed=3, gain=2.0)
+    L = Layer(px, geo, seed=3, n_blocks=3, softmax_scale=0.31, scale_k=0.5, scale_v=3.0)
+    L.append(H)
+    out = L.decode(q, [0, 1], [40, 40])
+    assert_close(f64(out), _ref_decode(L, H, q, [0, 1], [40, 40], softmax_scale=0.31), "custom scales")
+    L1 = Layer(px, geo, seed=3, n_blocks=3, scale_k=1.0, scale_v=1.0)     # Eq. 1 literally
+    L1.append(H)
+    assert_close(f64(L1.decode(q, [0, 1], [40, 40])), _ref_decode(L1, H, q, [0, 1], [40, 40]), "s = 1")
+
+
+def test_decode_many_splits_long_context(px):
+    geo = I.Geometry(128, 8, 2, 128, 2, 16, 16, alpha=32.0)
+    T = 6000 + 5
+    L = Layer(px, geo, seed=11, n_blocks=(T + 15) // 16)
+    H = I.hidden_states(T, geo, seed=11)
+    L.append(H)
+    q = I.queries(3, geo, seed=11, gain=4.0)
+    ctx = [T, 4097, 333]
+    assert_close(f64(L.decode(q, [1, 0, 1], ctx)), _ref_decode(L, H, q, [1, 0, 1], ctx), "long decode")
+    # closed forms through the whole GPU path: q = 0 gives the mean adapted value row
+    q0 = torch.zeros_like(q)
+    out0 = f64(L.decode(q0, [1, 0, 1], ctx))
+    w = L.w_np
+    for b, a in enumerate([1, 0, 1]):
+        mean_v = f64(H)[:ctx[b]].mean(0) @ (w["W_v"] + geo.scale_v * w["A_v"][a] @ w["B_v"][a])
+        for h in range(geo.n_q):
+            g = h // geo.group
+            np.testing.assert_allclose(out0[b, h], mean_v[g * geo.hd:(g + 1) * geo.hd], atol=5e-3, rtol=2e-2)
+
+
+def test_decode_is_deterministic_and_workspace_reusable(px):
+    geo = I.Geometry(128, 8, 2, 64, 2, 8, 8, alpha=16.0)
+    T = 3000
+    L = Layer(px, geo, seed=5, n_blocks=(T + 15) // 16)
+    L.append(I.hidden_states(T, geo, seed=5))
+    q = I.queries(2, geo, seed=5)
+    ws = px.decode_workspace(L.desc, 2, T)
+    outs = [L.decode(q, [0, 1], [T, 1234], max_ctx=T, ws=ws) for _ in range(3)]
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+
+
+# ------------------------------------------------------------------ paging: bit-exact
+
+def test_paged_equals_contiguous_bitwise(px):
+    geo = I.Geometry(256, 8, 2, 128, 3, 16, 16, alpha=32.0)
+    ctx = [700, 50, 333]
+    T = max(ctx)
+    nb_seq = (T + 15) // 16
+    H = I.hidden_states(T, geo, seed=21)
+    q = I.queries(3, geo, seed=21)
+    # contiguous: one shared sequence starting at block 0
+    Lc = Layer(px, geo, seed=21, n_blocks=nb_seq)
+    Lc.append(H)
+    ref = Lc.decode(q, [0, 1, 2], ctx, max_ctx=T)
+    # paged: same rows scattered over a larger pool through a random block permutation
+    pool = 3 * nb_seq
+    perm = I.permutation(pool, 21, "perm")[:nb_seq]
+    slots = (perm.long()[:, None] * 16 + torch.arange(16)[None, :]).reshape(-1)[:T].to(torch.int32).cuda()
+    Lp = Layer(px, geo, seed=21, n_blocks=pool, fill=float("nan"))
+    Lp.append(H, slot_mapping=slots)
+    table = perm.view(1, -1).repeat(3, 1).contiguous()
+    got = Lp.decode(q, [0, 1, 2], ctx, max_ctx=T, block_table=table)
+    assert torch.equal(got, ref)
+    # written rows are bit-identical to the contiguous write, all other slots keep their fill
+    tok = lambda c: c.permute(0, 2, 1, 3).reshape(-1, geo.kv_width)[:T].view(torch.int16)
+    pidx = perm.long().cuda()
+    assert torch.equal(tok(Lp.cache.k_base[pidx]), tok(Lc.cache.k_base))
+    assert torch.equal(tok(Lp.cache.v_base[pidx]), tok(Lc.cache.v_base))
+    for a in range(geo.n_agents):
+        assert torch.equal(Lp.cache.lr_k[a][pidx].reshape(-1, 16)[:T].view(torch.int16),
+                           Lc.cache.lr_k[a].reshape(-1, 16)[:T].view(torch.int16))
+    untouched = torch.ones(pool, dtype=torch.bool)
+    untouched[perm.long()] = False
+    assert torch.isnan(Lp.cache.k_base[untouched.cuda()]).all() and torch.isnan(Lp.cache.lr_v[:, untouched.cuda()]).all()
+    # the tail of the last block (slots >= T) is untouched too
+    last = int(perm[-1])
+    assert torch.isnan(Lp.cache.v_base[last, :, T % 16:]).all()
+    # first_block addressing: the same sequence placed at an offset inside a bigger contiguous cache
+    Lo = Layer(px, geo, seed=21, n_blocks=nb_seq + 9)
+    Lo.append(H, start_slot=5 * 16)
+    got2 = Lo.decode(q, [0, 1, 2], ctx, max_ctx=T, first_block=[5, 5, 5])
+    assert torch.equal(got2, ref)
+    # prefill: paged == contiguous, bitwise
+    qs = I.queries(40, geo, seed=21, tag="turn")
+    assert torch.equal(Lp.prefill(qs, 1, T - 40, block_table=perm), Lc.prefill(qs, 1, T - 40))
+    assert torch.equal(Lo.prefill(qs, 1, T - 40, first_block=5), Lc.prefill(qs, 1, T - 40))
+
+
+def test_agent_isolation_bitwise_and_agent_mask(px):
+    geo = I.Geometry(128, 8, 2, 64, 3, 16, 16, alpha=32.0)
+    T = 150
+    H = I.hidden_states(T, geo, seed=9)
+    q = I.queries(1, geo, seed=9)
+    L = Layer(px, geo, seed=9, n_blocks=10)
+    L.append(H)
+    ref = L.decode(q, [1], [T])
+    # clobber the other agents' LR caches and B matrices: agent 1's result must not move a bit
+    for a in (0, 2):
+        L.cache.lr_k[a].fill_(float("nan")); L.cache.lr_v[a].fill_(float("nan"))
+        L.B_k[a].fill_(float("nan")); L.B_v[a].fill_(float("nan"))
+    assert torch.equal(L.decode(q, [1], [T]), ref)
+    # agent mask: write only agents 0 and 2 -> agent 1's rows keep their fill
+    L2 = Layer(px, geo, seed=9, n_blocks=10, fill=float("nan"))
+    L2.append(H, agent_mask=0b101)
+    torch.cuda.synchronize()
+    rows = slice(0, (T + 15) // 16)
+    assert torch.isnan(L2.cache.lr_k[1]).all() and torch.isnan(L2.cache.lr_v[1]).all()
+    assert torch.isfinite(L2.cache.lr_k[0].reshape(-1, 16)[:T]).all() and torch.isfinite(L2.cache.lr_v[2].reshape(-1, 16)[:T]).all()
+
+
+def test_rebase_overwrites_segment_and_identity(px):
+    geo = I.Geometry(256, 8, 2, 128, 2, 8, 8, alpha=16.0)
+    T, S = 96, 40
+    H = I.hidden_states(T, geo, seed=13)
+    L = Layer(px, geo, seed=13, n_blocks=6)
+    L.append(H)
+    torch.cuda.synchronize()
+    before_k, before_lr = L.cache.k_base.clone(), L.cache.lr_k.clone()
+    # re-projecting the same hidden states leaves the cache bitwise unchanged
+    L.px.rebase_project(L.desc, H[T - S:].cuda(), L.W_packed, L.cache, T - S)
+    torch.cuda.synchronize()
+    assert torch.equal(L.cache.k_base, before_k)
+    # adapter-free pass over the turn: base rows and the other agent's LR rows are rebuilt from X_neut,
+    # the current agent's LR rows stay as they were (Section 3.2)
+    X_neut = I.hidden_states(S, geo, seed=13, tag="neut")
+    cur = 1
+    L.px.rebase_project(L.desc, X_neut.cuda(), L.W_packed, L.cache, T - S)
+    L.px.lr_precompute(L.desc, X_neut.cuda(), L.A_packed, L.cache, T - S, None, ~(1 << cur))
+    torch.cuda.synchronize()
+    kb = base_rows(L.cache.k_base)
+    ref_new = O.base_cache(f64(X_neut), L.w_np["W_k"])
+    assert (np.abs(kb[T - S:T] - ref_new) <= _cache_tol(ref_new)).all()
+    assert torch.equal(L.cache.k_base.permute(0, 2, 1, 3).reshape(-1, 256)[:T - S],
+                       before_k.permute(0, 2, 1, 3).reshape(-1, 256)[:T - S])
+    assert torch.equal(L.cache.lr_k[cur], before_lr[cur])
+    ref_lr = O.lr_cache(f64(X_neut), L.w_np["A_k"][0])
+    assert (np.abs(lr_rows(L.cache.lr_k, 0)[T - S:T] - ref_lr) <= _cache_tol(ref_lr)).all()
+    # token-by-token writes (double-batching order) == one segment write (lazy-prefill order), bitwise
+    L2 = Layer(px, geo, seed=13, n_blocks=6)
+    L2.append(H)
+    for t in range(S):
+        L2.px.rebase_project(L2.desc, X_neut[t:t + 1].cuda(), L2.W_packed, L2.cache, T - S + t)
+    torch.cuda.synchronize()
+    assert torch.equal(L2.cache.k_base, L.cache.k_base) and torch.equal(L2.cache.v_base, L.cache.v_base)
+
+
+def test_prefill_row_matches_decode(px):
+    geo = I.Geometry(256, 8, 2, 128, 2, 16, 16, alpha=32.0)
+    T, S = 200, 70
+    H = I.hidden_states(T + S, geo, seed=17)
+    L = Layer(px, geo, seed=17, n_blocks=(T + S + 15) // 16)
+    L.append(H)
+    qs = I.queries(S, geo, seed=17, gain=3.0)
+    pre = f64(L.prefill(qs, 0, T))
+    for i in (0, 1, 15, 16, 17, S - 1):
+        dec = f64(L.decode(qs[i:i + 1], [0], [T + i + 1]))[0]
+        np.testing.assert_allclose(pre[i], dec, atol=1e-2, rtol=2e-2)
+
+
+# ------------------------------------------------------------------ host-side validation
+
+def test_invalid_arguments_are_rejected_without_launch(px):
+    geo = I.Geometry(128, 8, 2, 64, 2, 16, 16, alpha=32.0)
+    L = Layer(px, geo, seed=1, n_blocks=4, fill=7.0)
+    H = I.hidden_states(32, geo, seed=1).cuda()
+    snapshot = L.cache.k_base.clone()
+    with pytest.raises(PreccError, match="INVALID_ARG"):
+        px.rebase_project(L.desc, H, L.W_packed, L.cache, start_slot=4 * 16 - 8)      # runs past the cache
+    with pytest.raises(PreccError, match="MISALIGNED"):
+        px.rebase_project(L.desc, H.view(-1)[1:1 + 31 * 128].view(31, 128), L.W_packed, L.cache)
+    bad = I.Geometry(128, 8, 2, 96, 2, 16, 16, alpha=32.0)
+    from paper_2609_34054_b200.binding import layer_desc
+    with pytest.raises(PreccError, match="UNSUPPORTED"):
+        px.rebase_project(layer_desc(bad), H, L.W_packed, L.cache)
+    with pytest.raises(PreccError, match="UNSUPPORTED"):
+        px.lr_precompute(layer_desc(I.Geometry(128, 8, 2, 64, 2, 16, 8, alpha=1.0)), H, L.A_packed, L.cache)
+    q = I.queries(1, geo, seed=1).cuda()
+    out = torch.zeros_like(q)
+    aid = torch.zeros(1, dtype=torch.int32, device="cuda"); cl = torch.full((1,), 32, dtype=torch.int32, device="cuda")
+    tiny_ws = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(PreccError, match="WORKSPACE"):
+        px.lr_attend_decode(L.desc, q, aid, cl, 32, L.B_k, L.B_v, L.cache, out, tiny_ws)
+    with pytest.raises(PreccError, match="INVALID_ARG"):
+        px.lr_attend_prefill(L.desc, q, 5, 10, L.B_k, L.B_v, L.cache, out)             # agent out of range
+    torch.cuda.synchronize()
+    assert torch.equal(L.cache.k_base, snapshot) and (out == 0).all()
+    # empty problems are no-ops
+    px.rebase_project(L.desc, H[:0], L.W_packed, L.cache)
+    px.lr_precompute(L.desc, H[:0], L.A_packed, L.cache)
+    assert px.poll_status() == 0
+
+
+def test_device_side_bad_indices_are_flagged_not_fatal(px):
+    geo = I.Geometry(128, 8, 2, 64, 2, 16, 16, alpha=32.0)
+    L = Layer(px, geo, seed=2, n_blocks=4, fill=1.0)
+    H = I.hidden_states(16, geo, seed=2).cuda()
+    slots = torch.arange(16, dtype=torch.int32)
+    slots[3] = 10_000                   # outside the cache: skipped and recorded
+    px.rebase_project(L.desc, H, L.W_packed, L.cache, 0, slots.cuda())
+    assert px.poll_status() & 1
+    assert (L.cache.k_base[0, :, 3] == 1.0).all()
+    q = I.queries(2, geo, seed=2)
+    out = L.decode(q, [0, 9], [16, 16])  # agent 9 does not exist: zeros + flag
+    assert px.poll_status() & 1
+    assert (out[1] == 0).all() and torch.isfinite(out[0]).all()
+    assert px.poll_status() == 0
