@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the shared-base + LR KV-cache path on B200.
+
+Workload (one "step" = one pass of the hot path over one synthetic trajectory, single stream):
+a Llama-3.2-1B-shaped stack (16 layers, d_model 2048, 32 q / 8 kv heads, head_dim 64), 4 agents,
+LoRA rank 16 on K and V (scale alpha/r = 2), shared trajectory of 8192 tokens:
+  phase A  per layer: base K/V projection of the 8192 hidden states into the shared cache
+           (precc_rebase_project) and the LR precompute for all 4 agents (precc_lr_precompute);
+  phase B  per agent, 128 decode steps, each one LR-reconstructed decode attention per layer
+           (precc_lr_attend_decode, batch 1, context 8192): 4 x 128 x 16 = 8192 launches,
+           replayed from one CUDA graph.
+The metric is the decode attention's algorithmic HBM bytes per second: per launch
+ctx*(2*n_kv*hd + r_k + r_v)*2 + q/out + the agent's B slices, summed over the launches of the step and
+divided by the WHOLE step time (phase A included).  Inputs are resident in HBM for `value`; `e2e`
+repeats the step with the hidden states and queries copied from pinned host memory and the outputs
+copied back inside the timed region.
+
+`--impl reference` times the CPU oracle (oracle/lrkv_oracle.py, numpy float64) on a bounded sample
+of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "lr_kv_decode_attention_GBps"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per decode launch of this workload, from the ncu
+# capture summarised under profiles/ (None until a capture exists)
+NCU_DECODE_TRAFFIC_BYTES = None
+
+
+def decode_bytes_per_launch(geo, ctx: int, batch: int = 1, distinct_agents: int = 1) -> int:
+    """Algorithmic HBM bytes of one decode-attention launch (LR rows counted once, not per kv head)."""
+    per_tok = (2 * geo.kv_width + geo.rank_k + geo.rank_v) * 2
+    qo = 2 * geo.n_q * geo.hd * 2
+    bmat = (geo.rank_k + geo.rank_v) * geo.kv_width * 2
+    table = (ctx + 15) // 16 * 4
+    return batch * (ctx * per_tok + qo + table) + distinct_agents * bmat
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            with open(p) as f:
+                return float(json.load(f)["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ CPU arm
+
+def oracle_sample(n_requests: int, seed: int = 0):
+    """Time the oracle on `n_requests` decode requests of layer 0 (all 8 kv heads, context 8192)."""
+    import numpy as np
+    from oracle import lrkv_oracle as O
+    from paper_2609_34054_b200 import inputs as I
+    geo, T = I.C2, I.C2_T
+    w = {k: v.float().numpy() for k, v in I.layer_weights(geo, seed, "L0").items()}
+    H = I.hidden_states(T, geo, seed, "L0.H").float().numpy()
+    q = I.queries(n_requests, geo, seed, "L0.q").float().numpy()
+    agent_id = [i % geo.n_agents for i in range(n_requests)]
+    t0 = time.perf_counter()
+    out = O.lr_decode_reference(q, agent_id, [T] * n_requests, H, w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                geo.scale_k, geo.scale_v, geo.n_kv)
+    dt = time.perf_counter() - t0
+    assert np.isfinite(out).all()
+    return n_requests * decode_bytes_per_launch(geo, T) / dt / 1e9, dt
+
+
+def cpu_threads() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    per_step = 8
+    for _ in range(args.warmup):
+        oracle_sample(per_step)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample(per_step)
+    dt = time.perf_counter() - t0
+    from paper_2609_34054_b200 import inputs as I
+    val = args.steps * per_step * decode_bytes_per_launch(I.C2, I.C2_T) / dt / 1e9
+    sample = f"{per_step} decode requests of layer 0 per step (all 8 kv heads, context 8192), merged-weight K/V + naive softmax in float64"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "C2 llama-3.2-1B-shaped stack, T=8192, N=4 agents, r=16 (bounded sample)", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+
+class Workload:
+    def __init__(self, px, seed: int, layers: int, steps: int, T: int):
+        import torch
+        from paper_2609_34054_b200 import inputs as I
+        from paper_2609_34054_b200.binding import Cache, layer_desc
+        self.torch, self.px = torch, px
+        geo = self.geo = I.C2
+        self.layers, self.dsteps, self.T = layers, steps, T
+        self.desc = layer_desc(geo)
+        nb = (T + 15) // 16
+        self.H_host, self.H, self.A_packed, self.W_packed, self.B_k, self.B_v, self.cache = [], [], [], [], [], [], []
+        for l in range(layers):
+            w = I.layer_weights(geo, seed, f"L{l}")
+            dev = {k: v.cuda() for k, v in w.items()}
+            self.A_packed.append(px.pack_adapters(geo, dev["A_k"], dev["A_v"]))
+            self.W_packed.append(px.pack_base_weights(geo, dev["W_k"], dev["W_v"]))
+            self.B_k.append(dev["B_k"]); self.B_v.append(dev["B_v"])
+            h = I.hidden_states(T, geo, seed, f"L{l}.H").pin_memory()
+            self.H_host.append(h)
+            self.H.append(h.cuda())
+            self.cache.append(Cache(geo, nb))
+        # queries of every (agent, decode step, layer): [N, steps, layers, n_q, hd]
+        self.q_host = I.normal_bf16((geo.n_agents, steps, layers, geo.n_q, geo.hd), 1.0, seed, "q").pin_memory()
+        self.q = self.q_host.cuda()
+        self.out = torch.zeros_like(self.q)
+        self.out_host = torch.empty_like(self.q_host).pin_memory()
+        self.agent_ids = [torch.full((1,), a, dtype=torch.int32, device="cuda") for a in range(geo.n_agents)]
+        self.ctx = torch.full((1,), T, dtype=torch.int32, device="cuda")
+        self.ws = px.decode_workspace(self.desc, 1, T)
+        self.graph = None
+        self.launches_a = 2 * layers
+        self.launches_b = geo.n_agents * steps * layers
+
+    def phase_a(self):
+        px = self.px
+        for l in range(self.layers):
+            px.rebase_project(self.desc, self.H[l], self.W_packed[l], self.cache[l], 0)
+            px.lr_precompute(self.desc, self.H[l], self.A_packed[l], self.cache[l], 0)
+
+    def phase_b_eager(self):
+        px, geo = self.px, self.geo
+        for a in range(geo.n_agents):
+            for s in range(self.dsteps):
+                for l in range(self.layers):
+                    px.lr_attend_decode(self.desc, self.q[a, s, l:l + 1], self.agent_ids[a], self.ctx, self.T,
+                                        self.B_k[l], self.B_v[l], self.cache[l], self.out[a, s, l:l + 1], self.ws)
+
+    def capture(self):
+        torch = self.torch
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            self.phase_a()
+            px, geo = self.px, self.geo
+            for l in range(self.layers):          # one eager launch per layer sets the kernel attributes
+                px.lr_attend_decode(self.desc, self.q[0, 0, l:l + 1], self.agent_ids[0], self.ctx, self.T,
+                                    self.B_k[l], self.B_v[l], self.cache[l], self.out[0, 0, l:l + 1], self.ws)
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.phase_b_eager()
+        self.graph = g
+
+    def phase_b(self):
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.phase_b_eager()
+
+    def step(self):
+        self.phase_a()
+        self.phase_b()
+
+    def step_host(self):
+        """The same step with inputs arriving from pinned host memory and outputs returned to it."""
+        for l in range(self.layers):
+            self.H[l].copy_(self.H_host[l], non_blocking=True)
+        self.q.copy_(self.q_host, non_blocking=True)
+        self.step()
+        self.out_host.copy_(self.out, non_blocking=True)
+
+    def h2d_bytes(self):
+        return sum(h.numel() * 2 for h in self.H_host) + self.q_host.numel() * 2
+
+    def d2h_bytes(self):
+        return self.out_host.numel() * 2
+
+    def decode_bytes_per_step(self):
+        return self.launches_b * decode_bytes_per_launch(self.geo, self.T)
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_34054_b200 import inputs as I
+    from paper_2609_34054_b200.binding import Precc
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the precc path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    px = Precc(local)
+    wl = Workload(px, seed=rank, layers=args.layers, steps=args.decode_steps, T=args.ctx)
+    wl.step()                                        # first pass builds the caches (also a warm-up)
+    torch.cuda.synchronize()
+    if not args.no_graph:
+        wl.capture()
+    assert px.poll_status() == 0
+
+    def timed(fn, steps, warmup, phases=False):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        pa = pb = 0.0
+        marks = []
+        ev[0].record()
+        for _ in range(steps):
+            if phases:
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                e0.record(); wl.phase_a(); e1.record(); wl.phase_b(); e2.record()
+                marks.append((e0, e1, e2))
+            else:
+                fn()
+        ev[1].record()
+        barrier()
+        ms = ev[0].elapsed_time(ev[1])
+        for e0, e1, e2 in marks:
+            pa += e0.elapsed_time(e1); pb += e1.elapsed_time(e2)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, pa, pb
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms, pa, pb = timed(wl.step, args.steps, args.warmup, phases=True)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_e2e, _, _ = timed(wl.step_host, max(1, min(args.steps, 3)), 1)
+    e2e_steps = max(1, min(args.steps, 3))
+    status = px.poll_status()
+    if status:
+        raise SystemExit(f"bench.py: device status 0x{status:x}")
+
+    geo = wl.geo
+    step_bytes = wl.decode_bytes_per_step()
+    value = world * step_bytes * args.steps / (ms * 1e-3) / 1e9
+    e2e_value = world * step_bytes * e2e_steps / (ms_e2e * 1e-3) / 1e9
+    per_launch = decode_bytes_per_launch(geo, wl.T)
+    launch_us = pb / args.steps / wl.launches_b * 1e3
+    achieved = per_launch / (launch_us * 1e-6) / 1e9
+    peak, peak_kind = measured_peak()
+    flops_a = wl.layers * 2.0 * wl.T * geo.d_model * (2 * geo.kv_width + geo.n_agents * (geo.rank_k + geo.rank_v))
+
+    if rank == 0:
+        cpu_val, cpu_dt = oracle_sample(args.cpu_requests) if world == 1 and not args.no_cpu else (None, None)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {
+                "workload": f"C2 llama-3.2-1B-shaped stack: {wl.layers} layers d=2048 32q/8kv hd=64, N=4 agents r=16 on K,V, "
+                            f"T={wl.T}: base projection + LR precompute, then {wl.dsteps} decode steps per agent (batch 1)",
+                "parallelism": "replicas" if world > 1 else "single GPU",
+                "l2_policy": f"decode cycles over {wl.layers} layers' caches = "
+                             f"{wl.layers * per_launch / 1e6:.0f} MB > 126 MB L2; no explicit flush",
+                "decode_launch": "CUDA graph replay" if not args.no_graph else "eager ctypes launches",
+            },
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(), "d2h_bytes_per_step": wl.d2h_bytes(),
+                    "ms_per_step": ms_e2e / e2e_steps},
+            "gpu_launches": (wl.launches_a + wl.launches_b) * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "lr_attend_decode_kernel<64,16,16>", "achieved": achieved, "peak": peak,
+                         "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
+                         "traffic": NCU_DECODE_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": per_launch,
+                         "avg_launch_us": launch_us},
+            "phases": {"precompute_ms_per_step": pa / args.steps, "decode_ms_per_step": pb / args.steps,
+                       "projection_tflops": flops_a / (pa / args.steps * 1e-3) / 1e12,
+                       "decode_only_GBps": step_bytes / (pb / args.steps * 1e-3) / 1e9},
+        }
+        if cpu_val is not None:
+            line["cpu_baseline"] = {"value": cpu_val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                    "sample": f"{args.cpu_requests} decode requests of layer 0 (all kv heads, context {I.C2_T}), "
+                                              f"{cpu_dt:.1f} s of numpy float64"}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="precc", choices=["precc", "reference"])
+    ap.add_argument("--layers", type=int, default=16)
+    ap.add_argument("--decode-steps", type=int, default=128)
+    ap.add_argument("--ctx", type=int, default=8192)
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-requests", type=int, default=40)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -100,6 +100,13 @@ const char* precc_error_name(int32_t code);
 /* Number of SMs of the context's device (the split schedule of decode depends on it). */
 int32_t precc_sm_count(const precc_ctx* ctx);
 
+/* Tracing (optional).  Give the context a caller-owned DEVICE buffer of n_blocks * 16 uint64 entries;
+ * while it is set, each thread block of precc_lr_attend_decode whose grid has at most n_blocks blocks
+ * records the GPU nanosecond timer at points of its life at entry [block][point]: 0 start, 1 indices
+ * read, 2 stream issued, 3 query fold ready, 4 first tile landed, 5 stream done, 6 record published,
+ * 7 done, and for the merging block 8 partials gathered, 9 weights ready, 10 merged (others stay 0).  Pass NULL to switch tracing off (the default).  There is no paper counterpart. */
+int32_t precc_set_trace_buffer(precc_ctx* ctx, void* buffer, size_t n_blocks);
+
 /* Read the device status word accumulated by kernels launched through `ctx`, then clear it.
  * Synchronises `stream`.  *status_out receives an OR of PRECC_STATUS_* bits.  Returns PRECC_OK when the
  * word is zero, PRECC_ERR_DEVICE_STATUS otherwise. */

@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libprecc.so")
 
 EXPORTS = [
-    "precc_create", "precc_destroy", "precc_last_error", "precc_error_name", "precc_sm_count",
+    "precc_create", "precc_destroy", "precc_last_error", "precc_error_name", "precc_sm_count", "precc_set_trace_buffer",
     "precc_poll_status", "precc_pack_kmajor", "precc_lr_precompute", "precc_rebase_project",
     "precc_decode_workspace_bytes", "precc_workspace_init", "precc_lr_attend_decode",
     "precc_lr_attend_prefill",
@@ -60,6 +60,7 @@ def load_library() -> C.CDLL:
     lib.precc_error_name.argtypes = [i32]
     lib.precc_error_name.restype = C.c_char_p
     lib.precc_sm_count.argtypes = [vp]
+    lib.precc_set_trace_buffer.argtypes = [vp, vp, sz]
     lib.precc_poll_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     lib.precc_pack_kmajor.argtypes = [vp, vp, i32, i32, vp, i32, i32, vp]
     lib.precc_lr_precompute.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, u64, C.POINTER(CacheDesc), vp]
@@ -157,6 +158,13 @@ class Precc:
                              f"{self.lib.precc_last_error(self.h).decode()}")
 
     # ------------------------------------------------------------------ plumbing
+    def set_trace_buffer(self, buf: Optional[torch.Tensor]):
+        """int64 CUDA tensor [n_blocks, 8] receiving per-block phase timestamps of decode, or None."""
+        if buf is None:
+            self._check(self.lib.precc_set_trace_buffer(self.h, None, 0), "precc_set_trace_buffer")
+        else:
+            self._check(self.lib.precc_set_trace_buffer(self.h, _ptr(buf), buf.shape[0]), "precc_set_trace_buffer")
+
     def poll_status(self) -> int:
         st = C.c_uint32(0)
         self.lib.precc_poll_status(self.h, _stream(), C.byref(st))

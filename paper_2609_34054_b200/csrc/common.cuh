@@ -70,6 +70,13 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// Programmatic dependent launch: when a kernel is launched with the programmatic-serialization
+// attribute it may start while its predecessor in the stream drains; pdl_wait() blocks until the
+// predecessor has completed and its writes are visible (a no-op for ordinary launches), and
+// pdl_launch_dependents() lets the successor begin its own launch early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 // XOR swizzle of 16-byte chunks inside a tile whose rows hold CPR chunks (CPR in {1,2,4,8,16}):
 // eight consecutive rows of the same logical chunk land in eight different 16-byte bank groups.
 template <int CPR>

@@ -1,19 +1,27 @@
 // LR-reconstructed decode attention (split-KV).
 //
-// For request b (agent a), kv head g and its G <= 8 query heads the kernel evaluates plain softmax
+// For request b (agent a), kv head g and its G <= 8 query heads the kernels evaluate plain softmax
 // attention with K_a = K_base + s_k L^K_a B^K_a and V_a = V_base + s_v L^V_a B^V_a (Eq. 1) without
 // building K_a or V_a: the key-side adapter is folded into r extra query coordinates
 // (q~ = s_k q B^K_{a,g}^T, contraction length head_dim + r_k) and the value-side adapter into r extra
 // output coordinates (U = P L^V_a, then out += s_v U B^V_{a,g}).
 //
-// Work split: grid (split j, kv head g, request b).  A thread block owns `chunk_tiles` consecutive
-// 16-token pages of one (b, g); its warps take pages round-robin, each with a private cp.async ring
-// (no block-wide barrier inside the stream loop).  Tokens sit on the MMA M axis:
+// Streaming core (decode_stream_block): a thread block owns consecutive 16-token pages of one (b, g);
+// its warps take pages round-robin, each with a private cp.async ring (no block-wide barrier inside
+// the stream loop).  Tokens sit on the MMA M axis:
 //   S^T[16 tok x 8 q]   = K'[16 x (hd+r_k)] . Q'^T          (mma.sync m16n8k16, bf16 -> fp32)
 //   O^T[(hd+r_v) x 8 q] += V'^T[(hd+r_v) x 16 tok] . P^T     (P^T obtained with movmatrix)
-// so no MMA row is wasted on padding.  Per-block partial (m, l, O') goes to the workspace; the last
-// block to finish a (b, g) (atomic ticket) merges the partials in split order and applies the
-// B^V epilogue.  Nothing waits on another block.
+// so no MMA row is wasted on padding.  The block's result (m, l, O') is left in shared memory.
+//
+// Two ways to combine the blocks of one (b, g):
+//   cluster kernel  the splits of a (b, g) form one thread-block cluster (up to 16 blocks); after a
+//                   cluster barrier every block merges its own slice of the output columns by reading
+//                   its peers' results over distributed shared memory.  No global scratch, no atomics:
+//                   the short-latency path for small batches.
+//   ticket kernel   blocks publish their result to a global workspace; the last block to finish a
+//                   (b, g) (atomic ticket) merges the records in split order.  Any number of splits.
+// Neither waits on another block with a spin: the cluster barrier is a hardware barrier among
+// co-scheduled blocks, the ticket path never waits at all.
 #pragma once
 #include "common.cuh"
 
@@ -32,9 +40,10 @@ struct DecodeParams {
   const __nv_bfloat16* lr_v;
   const __nv_bfloat16* B_k;
   const __nv_bfloat16* B_v;
-  float* part;        // [B][n_kv][max_splits][PART_STRIDE]
-  int32_t* tickets;   // [B][n_kv], zero between calls
+  float* part;        // ticket kernel: [B][n_kv][max_splits][PART_STRIDE]
+  int32_t* tickets;   // ticket kernel: [B][n_kv], zero between calls
   uint32_t* status;
+  unsigned long long* trace;   // optional [blocks][16] phase timestamps (ns), or null
   int64_t n_blocks;
   int table_stride;
   int n_q, n_kv, group, n_agents;
@@ -42,8 +51,9 @@ struct DecodeParams {
   float scale_log2, s_k, s_v;
 };
 
-constexpr int DEC_WARPS = 4;
-constexpr int DEC_THREADS = DEC_WARPS * 32;
+constexpr int DEC_WARPS = 4;            // ticket kernel
+constexpr int DEC_MAX_SPLITS = 512;
+constexpr int DEC_MAX_CLUSTER = 16;
 
 template <int HD, int RK, int RV>
 struct DecodeCfg {
@@ -53,18 +63,61 @@ struct DecodeCfg {
   static constexpr int STAGE_BYTES = 2 * KV_BYTES + LK_BYTES + LV_BYTES;
   static constexpr int OW = HD + RV;                 // accumulated output width
   static constexpr int PART_STRIDE = 8 * OW + 16;     // floats: m[8], l[8], O'[8][OW]
-  static constexpr int QX_BYTES = 8 * (RK > 0 ? RK : 8) * 2;
-  static constexpr int MERGE_FLOATS = DEC_WARPS * (OW * 8 + 16);
-  static constexpr int smem_bytes(int stages) {
-    int ring = DEC_WARPS * stages * STAGE_BYTES;
-    int merge = MERGE_FLOATS * 4;
-    return (ring > merge ? ring : merge) + QX_BYTES + 64;
+  // shared memory of a block with `warps` warps and `stages` ring slots per warp
+  __host__ __device__ static constexpr int ring_bytes(int warps, int stages) { return warps * stages * STAGE_BYTES; }
+  __host__ __device__ static constexpr int merge_bytes(int warps) { return warps * (OW * 8 + 16) * 4; }
+  __host__ __device__ static constexpr int ticket_smem(int stages) {
+    int a = ring_bytes(DEC_WARPS, stages), b = merge_bytes(DEC_WARPS);
+    int c = (16 + 8 * OW + 16 * DEC_MAX_SPLITS + DEC_WARPS * 8 * OW) * 4 + RV * HD * 2;   // final merge without staging
+    int m = a > b ? a : b;
+    return (m > c ? m : c) + 64;
+  }
+  // cluster kernel tail: own result | merged slice + denominators | B_v column slice (at most hd/2 columns)
+  static constexpr int CL_TAIL_BYTES = PART_STRIDE * 4 + (8 * (HD + RV) + 8) * 4 + RV * HD;
+  __host__ __device__ static constexpr int cluster_smem(int warps, int stages) {
+    int a = ring_bytes(warps, stages), b = merge_bytes(warps);
+    int m = a > b ? a : b;
+    return (m > CL_TAIL_BYTES ? m : CL_TAIL_BYTES) + 64;
   }
 };
 
-template <int HD, int RK, int RV>
-__global__ void __launch_bounds__(DEC_THREADS)
-lr_attend_decode_kernel(const DecodeParams p) {
+struct DecodeTrace {
+  unsigned long long* buf;
+  __device__ __forceinline__ void operator()(int k) const {
+    if (buf && threadIdx.x == 0) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+      buf[k] = t;
+    }
+  }
+};
+
+// Query fragments of one (b, g): B operand of the score MMA (k = head-dim coordinate, n = query head).
+template <int HD>
+__device__ __forceinline__ void load_q_frags(const DecodeParams& p, int b, int g, uint32_t (&qb)[HD / 16][2]) {
+  const int lane = threadIdx.x & 31;
+  const int qrow = lane >> 2, qk = (lane & 3) * 2;
+  const __nv_bfloat16* qsrc = p.q + ((size_t)b * p.n_q + (size_t)g * p.group + qrow) * HD;
+#pragma unroll
+  for (int kc = 0; kc < HD / 16; ++kc) {
+    if (qrow < p.group) {
+      qb[kc][0] = __ldg(reinterpret_cast<const uint32_t*>(qsrc + kc * 16 + qk));
+      qb[kc][1] = __ldg(reinterpret_cast<const uint32_t*>(qsrc + kc * 16 + 8 + qk));
+    } else {
+      qb[kc][0] = 0u; qb[kc][1] = 0u;
+    }
+  }
+}
+
+// Streams pages [tile0, tile_end) of (b, g) through the NW warps of the block and leaves the block's
+// result in shared memory as floats  res = [ m[8] | l[8] | O'[G][OW] ]  at the start of `smem`
+// (m = running maximum in the log2 domain, l = softmax denominator, O' = unnormalised output with the
+// r_v LR-V coordinates appended).  Ends with a __syncthreads().  A block with no pages yields
+// m = NEG_BIG, l = 0, O' = 0.
+template <int HD, int RK, int RV, int NW>
+__device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsigned char* smem, int b, int g, int ctx,
+                                                    int agent, int tile0, int tile_end,
+                                                    const uint32_t (&qb)[HD / 16][2], const DecodeTrace& mark) {
   using C = DecodeCfg<HD, RK, RV>;
   constexpr int OW = C::OW;
   constexpr int KC = HD / 16;                         // k-chunks of the base part
@@ -74,43 +127,22 @@ lr_attend_decode_kernel(const DecodeParams p) {
   constexpr int CPR_KV = HD / 8;
   constexpr int CPR_LK = RK > 0 ? RK / 8 : 1;
   constexpr int CPR_LV = RV > 0 ? RV / 8 : 1;
+  constexpr int NT = NW * 32;
 
-  extern __shared__ __align__(128) unsigned char smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int G = p.group;
+  const int qk = (lane & 3) * 2;
+  // this warp's pages: tile0 + warp + NW * i
+  const int my_n = (tile_end - tile0 - warp + NW - 1) / NW;   // may be <= 0
+  const uint32_t ring_u32 = smem_u32(smem + (size_t)warp * p.stages * C::STAGE_BYTES);
 
-  const int ctx = p.ctx_len[b];
-  const int agent = p.agent_id[b];
-  __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
-  if (ctx < 1 || agent < 0 || agent >= p.n_agents) {
-    if (split == 0) {
-      for (int i = threadIdx.x; i < G * HD; i += DEC_THREADS) out_bg[i] = __float2bfloat16(0.f);
-      if (threadIdx.x == 0 && ctx >= 1) atomicOr(p.status, StatusBits::BAD_INDEX);
-    }
-    return;
-  }
-  const int n_tiles = (ctx + PAGE - 1) / PAGE;
-  const int n_splits = (n_tiles + p.chunk_tiles - 1) / p.chunk_tiles;
-  if (split >= n_splits) return;
-  const int tile0 = split * p.chunk_tiles;
-  const int tile_end = min(n_tiles, tile0 + p.chunk_tiles);
-  // this warp's tiles: tile0 + warp + DEC_WARPS * i
-  const int my_n = (tile_end - tile0 - warp + DEC_WARPS - 1) / DEC_WARPS;   // may be <= 0
-
-  unsigned char* ring = smem + (size_t)warp * p.stages * C::STAGE_BYTES;
-  const uint32_t ring_u32 = smem_u32(ring);
-  const int ring_total = DEC_WARPS * p.stages * C::STAGE_BYTES;
-  const int merge_total = C::MERGE_FLOATS * 4;
-  __nv_bfloat16* qx = reinterpret_cast<__nv_bfloat16*>(smem + (ring_total > merge_total ? ring_total : merge_total));
-
-  // ---- physical block ids, fetched 32 tiles at a time, one batch ahead
+  // ---- physical block ids, fetched 32 pages at a time, one batch ahead
   auto load_phys = [&](int batch) -> int {
-    int i = batch * 32 + lane;
-    int t = tile0 + warp + DEC_WARPS * i;
+    const int i = batch * 32 + lane;
     if (i >= my_n) return 0;
-    int ph = p.block_table ? p.block_table[(size_t)b * p.table_stride + t]
-                           : (p.first_block ? p.first_block[b] : 0) + t;
+    const int t = tile0 + warp + NW * i;
+    int ph = p.block_table ? __ldg(p.block_table + (size_t)b * p.table_stride + t)
+                           : (p.first_block ? __ldg(p.first_block + b) : 0) + t;
     if (ph < 0 || ph >= p.n_blocks) { atomicOr(p.status, StatusBits::BAD_INDEX); ph = 0; }
     return ph;
   };
@@ -124,7 +156,7 @@ lr_attend_decode_kernel(const DecodeParams p) {
     if (i < my_n) {
       if ((i & 31) == 0 && i > 0) { phys_cur = phys_nxt; phys_nxt = load_phys((i >> 5) + 1); }
       const int ph = __shfl_sync(0xffffffffu, phys_cur, i & 31);
-      const int t = tile0 + warp + DEC_WARPS * i;
+      const int t = tile0 + warp + NW * i;
       const int valid = min(PAGE, ctx - t * PAGE);
       const uint32_t st = ring_u32 + (uint32_t)(i % p.stages) * C::STAGE_BYTES;
       const unsigned char* ksrc = reinterpret_cast<const unsigned char*>(p.k_base + ((size_t)ph * p.n_kv + g) * PAGE * HD);
@@ -134,6 +166,8 @@ lr_attend_decode_kernel(const DecodeParams p) {
         const int row = c / CPR_KV, ch = c % CPR_KV;
         const int off = swz_off<CPR_KV>(row, ch);
         cp_async16(st + off, ksrc + c * 16, 16);
+        // value rows past the context are zero-filled: their weight is zero, but 0 * garbage
+        // (an unwritten slot may hold NaN) must not reach the accumulators
         cp_async16(st + C::KV_BYTES + off, vsrc + c * 16, row < valid ? 16 : 0);
       }
       if constexpr (RK > 0) {
@@ -156,59 +190,59 @@ lr_attend_decode_kernel(const DecodeParams p) {
     cp_async_commit();
   };
 
-  // ---- start the stream before anything else
-  for (int i = 0; i < p.stages - 1; ++i) issue_tile(i);
-
-  // ---- query fragments: B operand (k = head-dim coordinate, n = query head)
-  const int qrow = lane >> 2;                 // query head within the group held as column n
-  const int qk = (lane & 3) * 2;
-  uint32_t qb[KC][2];
-  {
-    const __nv_bfloat16* qsrc = p.q + ((size_t)b * p.n_q + (size_t)g * G + qrow) * HD;
-#pragma unroll
-    for (int kc = 0; kc < KC; ++kc) {
-      if (qrow < G) {
-        qb[kc][0] = *reinterpret_cast<const uint32_t*>(qsrc + kc * 16 + qk);
-        qb[kc][1] = *reinterpret_cast<const uint32_t*>(qsrc + kc * 16 + 8 + qk);
-      } else {
-        qb[kc][0] = 0u; qb[kc][1] = 0u;
-      }
+  // ---- B_k fragments for the query fold are requested first (a few small loads), so that they do
+  //      not queue behind the page stream; large ranks would need too many registers and load later
+  constexpr bool PRELOAD_BK = RK > 0 && KX * KC * 4 <= 32;
+  const __nv_bfloat16* Bk = RK > 0 ? p.B_k + ((size_t)agent * RK) * ((size_t)p.n_kv * HD) + (size_t)g * HD : nullptr;
+  const size_t bk_rs = (size_t)p.n_kv * HD;     // row stride of B_k
+  auto load_bk = [&](int jt, int kc, uint32_t (&a)[4]) {
+    const __nv_bfloat16* r0 = Bk + (size_t)(jt * 16 + (lane >> 2)) * bk_rs + qk + kc * 16;
+    a[0] = __ldg(reinterpret_cast<const uint32_t*>(r0));
+    a[2] = __ldg(reinterpret_cast<const uint32_t*>(r0 + 8));
+    if (RK >= 16) {
+      a[1] = __ldg(reinterpret_cast<const uint32_t*>(r0 + 8 * bk_rs));
+      a[3] = __ldg(reinterpret_cast<const uint32_t*>(r0 + 8 * bk_rs + 8));
+    } else {
+      a[1] = 0u; a[3] = 0u;
     }
+  };
+  uint32_t bk_pre[PRELOAD_BK ? KX * KC : 1][4];
+  if constexpr (PRELOAD_BK) {
+#pragma unroll
+    for (int jt = 0; jt < KX; ++jt)
+#pragma unroll
+      for (int kc = 0; kc < KC; ++kc) load_bk(jt, kc, bk_pre[jt * KC + kc]);
   }
-  // ---- folded key-side adapter: q~[h][j] = s_k * sum_c q[h][c] * B_k[a][j][g*hd + c]
+  // ---- start the stream: every ring slot is filled at once
+  for (int i = 0; i < p.stages; ++i) issue_tile(i);
+  mark(2);
+
+  // ---- folded key-side adapter q~ = s_k q B_k[a][:, g]^T, computed per warp on the tensor cores as
+  //      q~^T[j x q] = B_k[j x c] . q^T[c x q]; the accumulator fragment, transposed with movmatrix,
+  //      is exactly the B operand (k = j, n = query) needed by the score MMA.
   uint32_t qxb[KX > 0 ? KX : 1][2];
   if constexpr (RK > 0) {
-    const __nv_bfloat16* Bk = p.B_k + ((size_t)agent * RK) * ((size_t)p.n_kv * HD) + (size_t)g * HD;
-    for (int e = threadIdx.x; e < 8 * RK; e += DEC_THREADS) {
-      const int h = e / RK, j = e % RK;
-      float acc = 0.f;
-      if (h < G) {
-        const uint4* qv = reinterpret_cast<const uint4*>(p.q + ((size_t)b * p.n_q + (size_t)g * G + h) * HD);
-        const uint4* bv = reinterpret_cast<const uint4*>(Bk + (size_t)j * p.n_kv * HD);
-#pragma unroll 4
-        for (int c = 0; c < HD / 8; ++c) {
-          uint4 x = __ldg(qv + c), y = __ldg(bv + c);
-          const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            acc += bf16_bits_to_float(xs[k] & 0xffff) * bf16_bits_to_float(ys[k] & 0xffff);
-            acc += bf16_bits_to_float(xs[k] >> 16) * bf16_bits_to_float(ys[k] >> 16);
-          }
+    for (int jt = 0; jt < KX; ++jt) {
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int kc = 0; kc < KC; ++kc) {
+        if constexpr (PRELOAD_BK) {
+          mma_bf16_16816(c, bk_pre[jt * KC + kc], qb[kc][0], qb[kc][1]);
+        } else {
+          uint32_t a[4];
+          load_bk(jt, kc, a);
+          mma_bf16_16816(c, a, qb[kc][0], qb[kc][1]);
         }
       }
-      qx[h * RK + j] = __float2bfloat16(acc * p.s_k);
-    }
-    __syncthreads();
-#pragma unroll
-    for (int kc = 0; kc < KX; ++kc) {
-      qxb[kc][0] = *reinterpret_cast<const uint32_t*>(qx + qrow * RK + kc * 16 + qk);
-      qxb[kc][1] = (RK >= 16) ? *reinterpret_cast<const uint32_t*>(qx + qrow * RK + kc * 16 + 8 + qk) : 0u;
+      qxb[jt][0] = movmatrix_t(pack_bf16(c[0] * p.s_k, c[1] * p.s_k));
+      qxb[jt][1] = movmatrix_t(pack_bf16(c[2] * p.s_k, c[3] * p.s_k));
     }
   }
 
   // ---- online-softmax state: this lane's two query columns (2*(lane&3), +1)
   float m0 = NEG_BIG, m1 = NEG_BIG, l0 = 0.f, l1 = 0.f;
-  float o[MT + (MX > 0 ? MX : 0)][4];
+  float o[MT + MX][4];
 #pragma unroll
   for (int i = 0; i < MT + MX; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
 
@@ -217,16 +251,17 @@ lr_attend_decode_kernel(const DecodeParams p) {
   const int v_row = (lane & 7) + (lane >> 4) * 8;         // V'^T A-operand (transposed load)
   const int v_cpar = (lane >> 3) & 1;
 
+  mark(3);
   for (int i = 0; i < my_n; ++i) {
     switch (p.stages) {
-      case 2: cp_async_wait<0>(); break;
-      case 3: cp_async_wait<1>(); break;
-      default: cp_async_wait<2>(); break;
+      case 2: cp_async_wait<1>(); break;
+      case 3: cp_async_wait<2>(); break;
+      default: cp_async_wait<3>(); break;
     }
-    __syncwarp();                      // tile i visible to all lanes; the slot of tile i-1 is free
-    issue_tile(i + p.stages - 1);
+    __syncwarp();                      // page i is visible to all lanes
+    if (i == 0) mark(4);
     const uint32_t st = ring_u32 + (uint32_t)(i % p.stages) * C::STAGE_BYTES;
-    const int t = tile0 + warp + DEC_WARPS * i;
+    const int t = tile0 + warp + NW * i;
     const int valid = ctx - t * PAGE;   // >= 1; tokens >= valid are masked
 
     float s[4] = {0.f, 0.f, 0.f, 0.f};
@@ -289,6 +324,8 @@ lr_attend_decode_kernel(const DecodeParams p) {
       ldsm_x2_t(a[0], a[2], st + 2 * C::KV_BYTES + C::LK_BYTES + swz_off<1>(a_row, 0));
       mma_bf16_16816(o[MT], a, pb0, pb1);
     }
+    __syncwarp();                      // all lanes are done with this slot
+    issue_tile(i + p.stages);
   }
   cp_async_wait<0>();
 #pragma unroll
@@ -296,12 +333,14 @@ lr_attend_decode_kernel(const DecodeParams p) {
     l0 += __shfl_xor_sync(0xffffffffu, l0, d);
     l1 += __shfl_xor_sync(0xffffffffu, l1, d);
   }
+  mark(5);
 
   // ---- merge the warps of this block: smem [warp][ m[8] | l[8] | O'[OW][8] ]
   __syncthreads();
   float* mg = reinterpret_cast<float*>(smem);
+  constexpr int WREC = OW * 8 + 16;
   {
-    float* w = mg + warp * (OW * 8 + 16);
+    float* w = mg + warp * WREC;
     if (lane < 4) { w[2 * lane] = m0; w[2 * lane + 1] = m1; w[8 + 2 * lane] = l0; w[8 + 2 * lane + 1] = l1; }
     const int r = lane >> 2, cq = (lane & 3) * 2;
 #pragma unroll
@@ -312,108 +351,320 @@ lr_attend_decode_kernel(const DecodeParams p) {
     }
   }
   __syncthreads();
-  // block result, written q-major into the partial record (or kept for the direct epilogue)
-  float* rec = p.part + (((size_t)b * p.n_kv + g) * p.max_splits + split) * C::PART_STRIDE;
-  __shared__ float fin_m[8], fin_l[8];
-  if (threadIdx.x < 8) {
-    const int h = threadIdx.x;
-    float M = NEG_BIG;
-    for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, mg[w * (OW * 8 + 16) + h]);
-    float L = 0.f;
-    for (int w = 0; w < DEC_WARPS; ++w) L += mg[w * (OW * 8 + 16) + 8 + h] * fast_exp2(mg[w * (OW * 8 + 16) + h] - M);
-    fin_m[h] = M; fin_l[h] = L;
-  }
-  __syncthreads();
-  // fin_o lives behind the per-warp records? no: reuse a separate region after them is not available,
-  // so accumulate into registers and write straight to the destination.
-  const bool direct = (n_splits == 1);
-  float* dst_o = direct ? nullptr : rec + 16;
-  // When direct, stage the merged O' in shared memory (region of warp 0 is consumed first, so use a
-  // dedicated area placed after all warp records is impossible; instead each thread keeps its values).
-  // Element e = h*OW + c handled by thread e % DEC_THREADS.
-  constexpr int PER_THREAD = (8 * OW + DEC_THREADS - 1) / DEC_THREADS;
-  float acc[PER_THREAD];
+  // every thread merges its own elements and derives the warp weights of its query row itself
+  // (a few redundant shared-memory reads instead of a serial phase and a barrier); element
+  // G*OW + h is the pair (m, l) of row h
+  const int n_el = G * OW;
+  constexpr int PER_THREAD = (8 * OW + 8 + NT - 1) / NT;
+  float acc[PER_THREAD], acc_m[PER_THREAD];
 #pragma unroll
   for (int k = 0; k < PER_THREAD; ++k) {
-    const int e = threadIdx.x + k * DEC_THREADS;
-    float v = 0.f;
-    if (e < 8 * OW) {
-      const int h = e / OW, c = e % OW;
-      const float M = fin_m[h];
-      for (int w = 0; w < DEC_WARPS; ++w) {
-        const float* wr = mg + w * (OW * 8 + 16);
-        v += wr[16 + c * 8 + h] * fast_exp2(wr[h] - M);
+    const int e = threadIdx.x + k * NT;
+    float v = 0.f, M = NEG_BIG;
+    if (e < n_el + 8) {
+      const bool is_ml = e >= n_el;
+      const int h = is_ml ? e - n_el : e / OW;
+      const int src = is_ml ? 8 + h : 16 + (e % OW) * 8 + h;
+      float mw[NW], xw[NW];
+#pragma unroll
+      for (int w = 0; w < NW; ++w) { mw[w] = mg[w * WREC + h]; xw[w] = mg[w * WREC + src]; }
+#pragma unroll
+      for (int w = 0; w < NW; ++w) M = fmaxf(M, mw[w]);
+#pragma unroll
+      for (int w = 0; w < NW; ++w) v += xw[w] * fast_exp2(mw[w] - M);   // warp order: deterministic
+    }
+    acc[k] = v; acc_m[k] = M;
+  }
+  __syncthreads();   // all reads of the warp records are done; the region is reused for the result
+#pragma unroll
+  for (int k = 0; k < PER_THREAD; ++k) {
+    const int e = threadIdx.x + k * NT;
+    if (e < n_el) mg[16 + e] = acc[k];
+    else if (e < n_el + 8) { mg[e - n_el] = acc_m[k]; mg[8 + e - n_el] = acc[k]; }
+  }
+  __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Ticket kernel: grid (split, kv head, request), DEC_WARPS warps.
+template <int HD, int RK, int RV>
+__global__ void __launch_bounds__(DEC_WARPS * 32)
+lr_attend_decode_kernel(const DecodeParams p) {
+  using C = DecodeCfg<HD, RK, RV>;
+  constexpr int OW = C::OW;
+  constexpr int NT = DEC_WARPS * 32;
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int G = p.group;
+  const int cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+  const DecodeTrace mark{p.trace ? p.trace + (size_t)cta_lin * 16 : nullptr};
+  mark(0);
+  pdl_wait();                 // nothing of the predecessor's output is touched before this point
+  pdl_launch_dependents();
+  uint32_t qb[HD / 16][2];    // independent of the index arrays: same round trip
+  load_q_frags<HD>(p, b, g, qb);
+  const int ctx = __ldg(p.ctx_len + b);
+  const int agent = __ldg(p.agent_id + b);
+  __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
+  if (ctx < 1 || agent < 0 || agent >= p.n_agents) {
+    if (split == 0) {
+      for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
+      if (threadIdx.x == 0 && ctx >= 1) atomicOr(p.status, StatusBits::BAD_INDEX);
+    }
+    return;
+  }
+  const int n_tiles = (ctx + PAGE - 1) / PAGE;
+  const int n_splits = (n_tiles + p.chunk_tiles - 1) / p.chunk_tiles;
+  if (split >= n_splits) return;
+  const int tile0 = split * p.chunk_tiles;
+  const int tile_end = min(n_tiles, tile0 + p.chunk_tiles);
+  mark(1);
+  decode_stream_block<HD, RK, RV, DEC_WARPS>(p, smem, b, g, ctx, agent, tile0, tile_end, qb, mark);
+
+  float* res = reinterpret_cast<float*>(smem);          // [m[8] | l[8] | O'[G][OW]]
+  const int n_el = G * OW;
+  const int rec_f = 16 + n_el;                          // used floats per record (multiple of 4)
+  const int region = C::ticket_smem(p.stages) - 64;     // bytes of shared memory usable below
+  const int bv_bytes = RV * HD * 2;
+  unsigned char* bv_s = smem + region - bv_bytes;       // B_v[a][:, g] slice, [RV][HD] bf16
+  const __nv_bfloat16* Bv = RV > 0 ? p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD : nullptr;
+  auto stage_bv = [&]() {
+    if constexpr (RV > 0) {
+      for (int c = threadIdx.x; c < RV * (HD / 8); c += NT) {
+        const int j = c / (HD / 8), ch = c % (HD / 8);
+        cp_async16(smem_u32(bv_s) + c * 16, Bv + (size_t)j * p.n_kv * HD + ch * 8, 16);
       }
     }
-    acc[k] = v;
-  }
-  __syncthreads();   // all reads of the warp records are done; smem can be reused
-  float* fo = reinterpret_cast<float*>(smem);   // merged O' [8][OW], then m[8], l[8]
-  if (!direct) {
-#pragma unroll
-    for (int k = 0; k < PER_THREAD; ++k) {
-      const int e = threadIdx.x + k * DEC_THREADS;
-      if (e < 8 * OW) dst_o[e] = acc[k];
-    }
-    if (threadIdx.x < 8) { rec[threadIdx.x] = fin_m[threadIdx.x]; rec[8 + threadIdx.x] = fin_l[threadIdx.x]; }
-    __threadfence();
+  };
+  float* fo = res + 16;                                 // final O' [G][OW]
+  __shared__ float fin_l[8];
+  if (n_splits > 1) {
+    float* rec = p.part + (((size_t)b * p.n_kv + g) * p.max_splits + split) * C::PART_STRIDE;
+    for (int i = threadIdx.x; i < rec_f / 4; i += NT)
+      reinterpret_cast<float4*>(rec)[i] = reinterpret_cast<const float4*>(res)[i];
     __syncthreads();
     __shared__ int is_last;
     if (threadIdx.x == 0) {
-      const int old = atomicAdd(p.tickets + (size_t)b * p.n_kv + g, 1);
+      // acq_rel at gpu scope: publishes this block's record (the barrier above orders the other
+      // threads' stores before it) and, for the last arriver, acquires everybody else's
+      int old;
+      asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(p.tickets + (size_t)b * p.n_kv + g) : "memory");
       is_last = (old == n_splits - 1);
       if (is_last) p.tickets[(size_t)b * p.n_kv + g] = 0;   // ready for the next call
     }
     __syncthreads();
+    mark(6);
     if (!is_last) return;
-    __threadfence();
-    // merge all splits in split order (deterministic whichever block arrives last)
+    // The last block merges all splits in split order, so the result does not depend on which
+    // block that is.  Records (and the B_v slice) are staged with one batch of async copies, so the
+    // L2 round trip is paid once.
     const float* base = p.part + (((size_t)b * p.n_kv + g) * p.max_splits) * C::PART_STRIDE;
-    if (threadIdx.x < 8) {
-      const int h = threadIdx.x;
+    float* recs = res + 16 + 8 * OW;                    // [n_splits][rec_f] (staged) or [n_splits][16]
+    const bool staged = (16 + 8 * OW + n_splits * rec_f + DEC_WARPS * n_el) * 4 + bv_bytes <= region;
+    stage_bv();
+    if (staged) {
+      const int cpr = rec_f / 4;                        // 16-byte chunks per record
+      for (int c = threadIdx.x; c < n_splits * cpr; c += NT) {
+        const int s2 = c / cpr, ch = c % cpr;
+        cp_async16(smem_u32(recs) + c * 16, base + (size_t)s2 * C::PART_STRIDE + ch * 4, 16);
+      }
+    } else {
+      for (int i = threadIdx.x; i < n_splits * 16; i += NT)
+        recs[i] = __ldcg(base + (size_t)(i >> 4) * C::PART_STRIDE + (i & 15));
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
+    __syncthreads();
+    mark(8);
+    const int wstr = staged ? rec_f : 16;               // stride of the (m | l) heads kept in shared memory
+    // weights: warp w owns query rows w, w+4 (< G); lanes stride over the splits
+    for (int h = warp; h < G; h += DEC_WARPS) {
       float M = NEG_BIG;
-      for (int s2 = 0; s2 < n_splits; ++s2) M = fmaxf(M, __ldcg(base + (size_t)s2 * C::PART_STRIDE + h));
+      for (int s2 = lane; s2 < n_splits; s2 += 32) M = fmaxf(M, recs[s2 * wstr + h]);
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, d));
       float L = 0.f;
-      for (int s2 = 0; s2 < n_splits; ++s2)
-        L += __ldcg(base + (size_t)s2 * C::PART_STRIDE + 8 + h) * fast_exp2(__ldcg(base + (size_t)s2 * C::PART_STRIDE + h) - M);
-      fin_m[h] = M; fin_l[h] = L;
+      for (int s2 = lane; s2 < n_splits; s2 += 32) {
+        const float wv = fast_exp2(recs[s2 * wstr + h] - M);
+        L += recs[s2 * wstr + 8 + h] * wv;
+        recs[s2 * wstr + h] = wv;
+      }
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) L += __shfl_xor_sync(0xffffffffu, L, d);   // fixed tree: deterministic
+      if (lane == 0) fin_l[h] = L;
     }
     __syncthreads();
-#pragma unroll
-    for (int k = 0; k < PER_THREAD; ++k) {
-      const int e = threadIdx.x + k * DEC_THREADS;
-      if (e < 8 * OW) {
-        const int h = e / OW;
-        const float M = fin_m[h];
-        float v = 0.f;
-        for (int s2 = 0; s2 < n_splits; ++s2) {
-          const float* r2 = base + (size_t)s2 * C::PART_STRIDE;
-          v += __ldcg(r2 + 16 + e) * fast_exp2(__ldcg(r2 + h) - M);
-        }
-        fo[e] = v;
+    mark(9);
+    // merge: a thread owns one float4 column of O' and a quarter of the splits (s = q, q+4, ...),
+    // four loads in flight; the quarters are then added in a fixed order
+    const int n_f4 = n_el / 4;
+    float* wsum = recs + (size_t)n_splits * wstr;       // [4][n_el]
+    for (int item = threadIdx.x; item < 4 * n_f4; item += NT) {
+      const int col = item % n_f4, qd = item / n_f4;
+      const int h = (col * 4) / OW;
+      float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+      auto fetch = [&](int s2) -> float4 {
+        if (staged) return *reinterpret_cast<const float4*>(recs + (size_t)s2 * rec_f + 16 + col * 4);
+        return __ldcg(reinterpret_cast<const float4*>(base + (size_t)s2 * C::PART_STRIDE + 16 + col * 4));
+      };
+      int s2 = qd;
+      for (; s2 + 4 < n_splits; s2 += 8) {
+        const float4 x0 = fetch(s2), x1 = fetch(s2 + 4);
+        const float w0 = recs[s2 * wstr + h], w1 = recs[(s2 + 4) * wstr + h];
+        a0.x += x0.x * w0; a0.y += x0.y * w0; a0.z += x0.z * w0; a0.w += x0.w * w0;
+        a1.x += x1.x * w1; a1.y += x1.y * w1; a1.z += x1.z * w1; a1.w += x1.w * w1;
       }
+      if (s2 < n_splits) {
+        const float4 x0 = fetch(s2);
+        const float w0 = recs[s2 * wstr + h];
+        a0.x += x0.x * w0; a0.y += x0.y * w0; a0.z += x0.z * w0; a0.w += x0.w * w0;
+      }
+      *reinterpret_cast<float4*>(wsum + (size_t)qd * n_el + col * 4) =
+          make_float4(a0.x + a1.x, a0.y + a1.y, a0.z + a1.z, a0.w + a1.w);
     }
+    __syncthreads();
+    for (int e = threadIdx.x; e < n_el; e += NT)
+      fo[e] = ((wsum[e] + wsum[n_el + e]) + wsum[2 * n_el + e]) + wsum[3 * n_el + e];
   } else {
-#pragma unroll
-    for (int k = 0; k < PER_THREAD; ++k) {
-      const int e = threadIdx.x + k * DEC_THREADS;
-      if (e < 8 * OW) fo[e] = acc[k];
-    }
+    stage_bv();
+    cp_async_commit();
+    if (threadIdx.x < 8) fin_l[threadIdx.x] = res[8 + threadIdx.x];
+    cp_async_wait<0>();
   }
   __syncthreads();
-  // ---- epilogue: out[h][c] = (O[h][c] + s_v * sum_j U[h][j] * B_v[a][j][g*hd + c]) / l[h]
-  const __nv_bfloat16* Bv = RV > 0 ? p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD : nullptr;
-  for (int e = threadIdx.x; e < G * HD; e += DEC_THREADS) {
+  mark(10);
+  const __nv_bfloat16* bvs = reinterpret_cast<const __nv_bfloat16*>(bv_s);
+  for (int e = threadIdx.x; e < G * HD; e += NT) {
     const int h = e / HD, c = e % HD;
     float v = fo[h * OW + c];
     if constexpr (RV > 0) {
       float u = 0.f;
 #pragma unroll 8
-      for (int j = 0; j < RV; ++j) u += fo[h * OW + HD + j] * __bfloat162float(Bv[(size_t)j * p.n_kv * HD + c]);
+      for (int j = 0; j < RV; ++j) u += fo[h * OW + HD + j] * __bfloat162float(bvs[j * HD + c]);
       v += p.s_v * u;
     }
     out_bg[e] = __float2bfloat16(v / fin_l[h]);
   }
+  mark(7);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Cluster kernel: grid (cluster size CS, kv head, request), cluster (CS,1,1), NW warps.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float dsmem_ld(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];\n" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+
+template <int HD, int RK, int RV, int NW>
+__global__ void __launch_bounds__(NW * 32)
+lr_attend_decode_cluster_kernel(const DecodeParams p) {
+  using C = DecodeCfg<HD, RK, RV>;
+  constexpr int OW = C::OW;
+  constexpr int NT = NW * 32;
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int rank = blockIdx.x, CS = gridDim.x;          // the cluster spans grid.x
+  const int g = blockIdx.y, b = blockIdx.z;
+  const int G = p.group;
+  const int cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+  const DecodeTrace mark{p.trace ? p.trace + (size_t)cta_lin * 16 : nullptr};
+  mark(0);
+  pdl_wait();
+  pdl_launch_dependents();
+  uint32_t qb[HD / 16][2];
+  load_q_frags<HD>(p, b, g, qb);
+  const int ctx = __ldg(p.ctx_len + b);
+  const int agent = __ldg(p.agent_id + b);
+  __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
+  if (ctx < 1 || agent < 0 || agent >= p.n_agents) {   // the same decision in every block of the cluster
+    if (rank == 0) {
+      for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
+      if (threadIdx.x == 0 && ctx >= 1) atomicOr(p.status, StatusBits::BAD_INDEX);
+    }
+    return;
+  }
+  const int n_tiles = (ctx + PAGE - 1) / PAGE;
+  const int tile0 = min(n_tiles, rank * p.chunk_tiles);
+  const int tile_end = min(n_tiles, tile0 + p.chunk_tiles);
+  mark(1);
+  // B_v column slice of this block: requested now (before the page stream), parked in registers
+  constexpr int BV_PER_THREAD = RV > 0 ? (RV * (HD / 2) + NT - 1) / NT : 1;
+  __nv_bfloat16 bv_pre[BV_PER_THREAD];
+  if constexpr (RV > 0) {
+    const int cols_ = HD / CS;
+    const __nv_bfloat16* Bv = p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD + rank * cols_;
+#pragma unroll
+    for (int k = 0; k < BV_PER_THREAD; ++k) {
+      const int i = threadIdx.x + k * NT;
+      bv_pre[k] = (i < RV * cols_) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);
+    }
+  }
+  decode_stream_block<HD, RK, RV, NW>(p, smem, b, g, ctx, agent, tile0, tile_end, qb, mark);
+
+  // own result res = [m[8] | l[8] | O'[G][OW]] sits at the start of shared memory in every block
+  float* res = reinterpret_cast<float*>(smem);
+  float* mine = res + C::PART_STRIDE;                   // merged slice [G][cols + RV], then l[8]
+  __nv_bfloat16* bvs = reinterpret_cast<__nv_bfloat16*>(mine + 8 * (HD + RV) + 8);   // B_v[:, my columns], [RV][cols]
+  const int cols = HD / CS;                             // output columns finished by this block
+  const int c0 = rank * cols;
+  if constexpr (RV > 0) {                               // B_v column slice (bv_pre was requested before the stream)
+    for (int k = 0; k < BV_PER_THREAD; ++k) {
+      const int i = threadIdx.x + k * NT;
+      if (i < RV * cols) bvs[i] = bv_pre[k];
+    }
+  }
+  mark(6);
+  cluster_sync_all();                                   // every block's result is complete and visible
+  // One pass over distributed shared memory: a thread owns one merged element (for every h < G my
+  // `cols` base columns and all r_v LR-V coordinates, plus the denominators) and reads the peers'
+  // running maxima and values with all loads in flight at once; peers are added in rank order.
+  const uint32_t res_u32 = smem_u32(res);
+  const int sw = cols + RV;
+  for (int e = threadIdx.x; e < G * sw + G; e += NT) {
+    const bool is_l = e >= G * sw;
+    const int h = is_l ? e - G * sw : e / sw;
+    const int k = e % sw;
+    const int src = is_l ? 8 + h : 16 + h * OW + (k < cols ? c0 + k : HD + (k - cols));
+    float mr[DEC_MAX_CLUSTER], xr[DEC_MAX_CLUSTER];
+#pragma unroll
+    for (int r = 0; r < DEC_MAX_CLUSTER; ++r) {
+      if (r < CS) { mr[r] = dsmem_ld(dsmem_addr(res_u32 + h * 4, r)); xr[r] = dsmem_ld(dsmem_addr(res_u32 + src * 4, r)); }
+      else { mr[r] = NEG_BIG; xr[r] = 0.f; }
+    }
+    float M = NEG_BIG;
+#pragma unroll
+    for (int r = 0; r < DEC_MAX_CLUSTER; ++r) M = fmaxf(M, mr[r]);
+    float v = 0.f;
+#pragma unroll
+    for (int r = 0; r < DEC_MAX_CLUSTER; ++r) v += xr[r] * fast_exp2(mr[r] - M);
+    mine[is_l ? 8 * (HD + RV) + h : e] = v;
+  }
+  __syncthreads();
+  mark(10);
+  const float* fin_l = mine + 8 * (HD + RV);
+  for (int e = threadIdx.x; e < G * cols; e += NT) {
+    const int h = e / cols, c = e % cols;
+    float v = mine[h * sw + c];
+    if constexpr (RV > 0) {
+      float u[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int j = 0; j < RV; ++j) u[j & 3] += mine[h * sw + cols + j] * __bfloat162float(bvs[j * cols + c]);
+      v += p.s_v * ((u[0] + u[1]) + (u[2] + u[3]));
+    }
+    out_bg[h * HD + c0 + c] = __float2bfloat16(v / fin_l[h]);
+  }
+  mark(7);
+  cluster_sync_all();                                   // nobody leaves while a peer may still read its result
 }
 
 }  // namespace precc

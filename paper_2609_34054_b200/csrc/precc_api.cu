@@ -20,6 +20,8 @@ struct precc_ctx {
   int sm_count = 0;
   int max_smem_optin = 0;
   uint32_t* status = nullptr;          // device status word
+  unsigned long long* trace = nullptr; // optional caller-owned trace buffer
+  size_t trace_blocks = 0;
   char err[512] = {0};
   CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                            const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -156,18 +158,19 @@ int32_t dispatch_shape(precc_ctx* ctx, int hd, int rk, int rv, Args&&... args) {
   return fail(ctx, PRECC_ERR_UNSUPPORTED, "no kernel for head_dim %d ranks (%d,%d)", hd, rk, rv);
 }
 
-// Split schedule of decode: pages per thread block and blocks per (request, kv head).
-struct DecodePlan { int chunk_tiles, max_splits, stages, smem; };
+// Split schedule of decode.  cluster > 0: the cluster kernel with that many blocks per (request, kv head);
+// otherwise the ticket kernel with up to max_splits blocks per (request, kv head).
+struct DecodePlan { int cluster, warps, chunk_tiles, max_splits, stages, smem; };
 
 template <int HD, int RK, int RV>
-DecodePlan plan_decode(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
+DecodePlan plan_ticket(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
   using C = DecodeCfg<HD, RK, RV>;
-  DecodePlan pl;
+  DecodePlan pl{};
   // ring depth: as deep as possible (<= 4) while two blocks still fit on an SM
   int stages = 4;
-  while (stages > 2 && 2 * (C::smem_bytes(stages) + 1024) > max_smem) --stages;
+  while (stages > 2 && 2 * (C::ticket_smem(stages) + 1024) > max_smem) --stages;
   pl.stages = stages;
-  pl.smem = C::smem_bytes(stages);
+  pl.smem = C::ticket_smem(stages);
   const int per_sm = (2 * (pl.smem + 1024) <= max_smem) ? 2 : 1;
   const long long slots = (long long)sm_count * per_sm;
   const int max_tiles = (max_ctx + PAGE - 1) / PAGE;
@@ -179,8 +182,40 @@ DecodePlan plan_decode(int sm_count, int max_smem, int B, int n_kv, int max_ctx)
   if (total_tiles >= slots * 4 * 64) want = (4 * slots + units - 1) / units;
   int chunk = (int)((max_tiles + want - 1) / want);
   if (chunk < DEC_WARPS) chunk = DEC_WARPS;
+  if ((max_tiles + chunk - 1) / chunk > DEC_MAX_SPLITS) chunk = (max_tiles + DEC_MAX_SPLITS - 1) / DEC_MAX_SPLITS;
   pl.chunk_tiles = chunk;
   pl.max_splits = (max_tiles + chunk - 1) / chunk;
+  return pl;
+}
+
+// The cluster kernel serves the latency-bound regime: few (request, kv head) units, each worth
+// splitting, the whole grid co-resident in one wave.  Returns cluster = 0 when it does not apply.
+template <int HD, int RK, int RV>
+DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
+  using C = DecodeCfg<HD, RK, RV>;
+  DecodePlan pl{};
+  const int max_tiles = (max_ctx + PAGE - 1) / PAGE;
+  const long long units = (long long)B * n_kv;
+  if (units * 2 > sm_count || max_tiles <= 16) return pl;  // too many units, or nothing worth splitting
+  if (units * max_tiles > 32768) return pl;              // bandwidth-bound: all SMs matter more than the short tail
+  // two blocks per SM must fit (a 16-block cluster needs 16 free slots inside one GPC, and not every
+  // GPC has 16 SMs): 8 warps with a 2-deep ring if that fits, else 4 warps with the deepest ring that does
+  const int budget = max_smem / 2 - 1024;
+  int warps = 8, stages = 2;
+  if (C::cluster_smem(8, 2) > budget) {
+    warps = 4; stages = 4;
+    while (stages > 2 && C::cluster_smem(4, stages) > budget) --stages;
+    if (C::cluster_smem(4, stages) > budget) return pl;
+  }
+  int cs = DEC_MAX_CLUSTER;
+  while (cs > 1 && (units * cs > sm_count || max_tiles < cs * warps)) cs >>= 1;
+  if (cs < 2) return pl;
+  pl.cluster = cs;
+  pl.warps = warps;
+  pl.stages = stages;
+  pl.smem = C::cluster_smem(warps, stages);
+  pl.chunk_tiles = (max_tiles + cs - 1) / cs;
+  pl.max_splits = cs;
   return pl;
 }
 
@@ -193,15 +228,45 @@ struct DecodeArgs {
 template <int HD, int RK, int RV>
 struct DecodeRun {
   static size_t ws_bytes(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
-    const DecodePlan pl = plan_decode<HD, RK, RV>(sm_count, max_smem, B, n_kv, max_ctx);
+    const DecodePlan pl = plan_ticket<HD, RK, RV>(sm_count, max_smem, B, n_kv, max_ctx);
     const size_t tickets = ((size_t)B * n_kv * 4 + 255) / 256 * 256;
     return tickets + (size_t)B * n_kv * pl.max_splits * DecodeCfg<HD, RK, RV>::PART_STRIDE * 4;
   }
+  // Can `need` clusters of `cs` blocks be resident at once?  Asked once per (shape, warps, cluster size).
+  template <int NW>
+  static bool cluster_fits(precc_ctx* ctx, const DecodePlan& pl, int need) {
+    static int cached[DEC_MAX_CLUSTER + 1] = {0};      // 0 = unknown, else max active clusters + 1
+    if (cached[pl.cluster] == 0) {
+      auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW>;
+      int n = 0;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess ||
+          cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+        cudaGetLastError();
+        cached[pl.cluster] = 1;
+        return false;
+      }
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(pl.cluster, ctx->sm_count / pl.cluster, 1);
+      cfg.blockDim = dim3(NW * 32);
+      cfg.dynamicSmemBytes = pl.smem;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = pl.cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+      cached[pl.cluster] = n + 1;
+    }
+    return cached[pl.cluster] - 1 >= need;
+  }
   static int32_t run(precc_ctx* ctx, const DecodeArgs& a) {
     const precc_layer_desc* d = a.d;
-    const DecodePlan pl = plan_decode<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
-    const size_t need = ws_bytes(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
-    if (!a.ws || a.ws_bytes < need) return fail(ctx, PRECC_ERR_WORKSPACE, "decode workspace: need %zu bytes, got %zu", need, a.ws_bytes);
+    DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
+    if (pl.cluster && !(pl.warps == 8 ? cluster_fits<8>(ctx, pl, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, pl, a.B * d->n_kv_heads))) pl.cluster = 0;
+    if (!pl.cluster) {
+      pl = plan_ticket<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
+      const size_t need = ws_bytes(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
+      if (!a.ws || a.ws_bytes < need) return fail(ctx, PRECC_ERR_WORKSPACE, "decode workspace: need %zu bytes, got %zu", need, a.ws_bytes);
+    }
     DecodeParams p;
     p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out;
     p.agent_id = a.agent_id; p.ctx_len = a.ctx_len; p.block_table = a.block_table; p.first_block = a.first_block;
@@ -210,16 +275,35 @@ struct DecodeRun {
     p.B_k = (const __nv_bfloat16*)a.B_k; p.B_v = (const __nv_bfloat16*)a.B_v;
     const size_t tickets = ((size_t)a.B * d->n_kv_heads * 4 + 255) / 256 * 256;
     p.tickets = (int32_t*)a.ws;
-    p.part = (float*)((char*)a.ws + tickets);
+    p.part = a.ws ? (float*)((char*)a.ws + tickets) : nullptr;
     p.status = ctx->status;
+    p.trace = (ctx->trace && (size_t)pl.max_splits * d->n_kv_heads * a.B <= ctx->trace_blocks) ? ctx->trace : nullptr;
     p.n_blocks = a.cache->n_blocks; p.table_stride = a.table_stride;
     p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = d->n_q_heads / d->n_kv_heads; p.n_agents = d->n_agents;
     p.chunk_tiles = pl.chunk_tiles; p.max_splits = pl.max_splits; p.stages = pl.stages;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
-    auto kern = lr_attend_decode_kernel<HD, RK, RV>;
-    PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem));
-    kern<<<dim3(pl.max_splits, d->n_kv_heads, a.B), DEC_THREADS, pl.smem, a.stream>>>(p);
-    PRECC_CUDA(ctx, cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.max_splits, d->n_kv_heads, a.B);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (pl.cluster) {
+      cfg.blockDim = dim3(pl.warps * 32);
+      attr[1].id = cudaLaunchAttributeClusterDimension;
+      attr[1].val.clusterDim.x = pl.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+      cfg.numAttrs = 2;
+      if (pl.warps == 8) PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 8>, p));
+      else PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 4>, p));
+    } else {
+      auto kern = lr_attend_decode_kernel<HD, RK, RV>;
+      cfg.blockDim = dim3(DEC_WARPS * 32);
+      PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem));
+      PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, p));
+    }
     return PRECC_OK;
   }
 };
@@ -323,6 +407,14 @@ const char* precc_error_name(int32_t code) {
 }
 
 int32_t precc_sm_count(const precc_ctx* ctx) { return ctx ? ctx->sm_count : 0; }
+
+int32_t precc_set_trace_buffer(precc_ctx* ctx, void* buffer, size_t n_blocks) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (buffer && (reinterpret_cast<uintptr_t>(buffer) & 7u)) return fail(ctx, PRECC_ERR_MISALIGNED, "trace buffer not 8-byte aligned");
+  ctx->trace = static_cast<unsigned long long*>(buffer);
+  ctx->trace_blocks = buffer ? n_blocks : 0;
+  return PRECC_OK;
+}
 
 int32_t precc_poll_status(precc_ctx* ctx, void* stream, uint32_t* status_out) {
   if (!ctx) return PRECC_ERR_INVALID_ARG;

@@ -44,7 +44,7 @@ struct PrefillCfg {
   static constexpr int LV_BYTES = PF_TOK * RV * 2;
   static constexpr int STAGE_BYTES = 2 * KV_BYTES + LK_BYTES + LV_BYTES;
   static constexpr int OW = HD + RV;
-  static constexpr int smem_bytes(int stages) {
+  __host__ __device__ static constexpr int smem_bytes(int stages) {
     int stream = Q_BYTES + QX_BYTES + stages * STAGE_BYTES;
     int epi = PF_ROWS * (OW + 1) * 4;
     return (stream > epi ? stream : epi) + 16;
