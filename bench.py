@@ -60,6 +60,22 @@ def measured_peak():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+def reduce_max_ms(ms: float, device="cpu") -> float:
+    """Max over ranks of a per-rank duration (identity when torch.distributed is not initialised)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(bytes_per_rank_step: float, steps: int, ms_max: float, world: int) -> float:
+    """Replicas: every rank processes the same number of units; GB/s of the whole job."""
+    return world * bytes_per_rank_step * steps / (ms_max * 1e-3) / 1e9
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
 
@@ -302,10 +318,7 @@ def run_gpu(args):
         ms = ev[0].elapsed_time(ev[1])
         for e0, e1, e2 in marks:
             pa += e0.elapsed_time(e1); pb += e1.elapsed_time(e2)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = reduce_max_ms(ms, "cuda")
         return ms, pa, pb
 
     sampler = ClockSampler(local)
@@ -321,8 +334,8 @@ def run_gpu(args):
 
     geo = wl.geo
     step_bytes = wl.decode_bytes_per_step()
-    value = world * step_bytes * args.steps / (ms * 1e-3) / 1e9
-    e2e_value = world * step_bytes * e2e_steps / (ms_e2e * 1e-3) / 1e9
+    value = whole_job_value(step_bytes, args.steps, ms, world)
+    e2e_value = whole_job_value(step_bytes, e2e_steps, ms_e2e, world)
     per_launch = decode_bytes_per_launch(geo, wl.T)
     launch_us = pb / args.steps / wl.launches_b * 1e3
     achieved = per_launch / (launch_us * 1e-6) / 1e9
