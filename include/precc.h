@@ -167,6 +167,32 @@ int32_t precc_lr_attend_decode(precc_ctx* ctx, const precc_layer_desc* desc, con
                                const void* B_k, const void* B_v, const precc_cache* cache,
                                void* out, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same decode attention for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a property of the library, not of the method).  Some users of this library run
+ * where cudaMalloc is off limits: a serving engine that handed every free byte of HBM to its KV-cache
+ * pool at start-up, code running while a stream is being captured (allocation is illegal there), or a
+ * latency-critical decode loop that must not take cudaMalloc's device-wide synchronisation.  For them the
+ * split-merge scratch of precc_lr_attend_decode lives in an array compiled into the library
+ * (PRECC_STATIC_SCRATCH_BYTES of device memory, held by every GPU that loads the library until the
+ * process exits) instead of a caller workspace.  Arguments and results are those of
+ * precc_lr_attend_decode without `workspace`.
+ *   - If precc_decode_workspace_bytes(desc, B, max_ctx, sm_count) exceeds PRECC_STATIC_SCRATCH_BYTES the
+ *     call returns PRECC_ERR_WORKSPACE (the message names both sizes) and launches nothing.
+ *   - The call allocates nothing: no cudaMalloc / cudaFree, no allocating library routine.
+ *   - The first call on a device looks up the device address of the array (the context's device must be
+ *     the current device).  Make that first call outside any stream capture.
+ *   - Every call on a device shares the one array.  The part that must start at zero is cleared on
+ *     `stream` at the start of each call; the rest keeps the previous call's contents.  Two calls that
+ *     may overlap on the GPU (different streams, or different contexts on the same device) race on it:
+ *     serialise them, or give one of them precc_lr_attend_decode with its own workspace. */
+#define PRECC_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t precc_lr_attend_decode_static(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,
+                                      const int32_t* agent_id, const int32_t* ctx_len,
+                                      const int32_t* block_table, int32_t table_stride,
+                                      const int32_t* first_block, int32_t max_ctx,
+                                      const void* B_k, const void* B_v, const precc_cache* cache,
+                                      void* out, void* stream);
+
 /* LR-reconstructed attention for the S new tokens of a turn (Section 3.1: the current agent computes
  * only over the newly added context and reuses base + own LR cache for the rest).  The caches must
  * already cover the new tokens (precc_rebase_project + precc_lr_precompute on them first).  Query i

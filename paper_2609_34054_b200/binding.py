@@ -21,7 +21,7 @@ EXPORTS = [
     "precc_create", "precc_destroy", "precc_last_error", "precc_error_name", "precc_sm_count", "precc_set_trace_buffer",
     "precc_poll_status", "precc_pack_kmajor", "precc_lr_precompute", "precc_rebase_project",
     "precc_decode_workspace_bytes", "precc_workspace_init", "precc_lr_attend_decode",
-    "precc_lr_attend_prefill",
+    "precc_lr_attend_decode_static", "precc_lr_attend_prefill",
 ]
 
 
@@ -70,6 +70,8 @@ def load_library() -> C.CDLL:
     lib.precc_workspace_init.argtypes = [vp, vp, sz, vp]
     lib.precc_lr_attend_decode.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, i32, vp, i32, vp, vp,
                                            C.POINTER(CacheDesc), vp, vp, sz, vp]
+    lib.precc_lr_attend_decode_static.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, i32, vp, i32, vp, vp,
+                                                  C.POINTER(CacheDesc), vp, vp]
     lib.precc_lr_attend_prefill.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp,
                                             C.POINTER(CacheDesc), vp, vp]
     for name in EXPORTS:
@@ -225,6 +227,20 @@ class Precc:
             self.h, C.byref(desc), _ptr(q), q.shape[0], _ptr(agent_id), _ptr(ctx_len), _ptr(block_table), stride,
             _ptr(first_block), max_ctx, _ptr(B_k), _ptr(B_v), C.byref(cd), _ptr(out), _ptr(workspace),
             workspace.numel(), _stream()), "precc_lr_attend_decode")
+
+    def lr_attend_decode_static(self, desc: LayerDesc, q: torch.Tensor, agent_id: torch.Tensor, ctx_len: torch.Tensor,
+                                max_ctx: int, B_k, B_v, cache: Cache, out: torch.Tensor,
+                                block_table: Optional[torch.Tensor] = None, first_block: Optional[torch.Tensor] = None):
+        """Decode attention for callers that may not allocate device memory (an engine whose KV pool owns
+        all of HBM, code inside a stream capture, a loop that cannot afford cudaMalloc's synchronisation):
+        the split-merge scratch is an array built into the library, so no workspace is passed.  All calls
+        on a device share that array; do not let two of them overlap on the GPU."""
+        cd = cache.desc()
+        stride = block_table.shape[1] if block_table is not None else 0
+        self._check(self.lib.precc_lr_attend_decode_static(
+            self.h, C.byref(desc), _ptr(q), q.shape[0], _ptr(agent_id), _ptr(ctx_len), _ptr(block_table), stride,
+            _ptr(first_block), max_ctx, _ptr(B_k), _ptr(B_v), C.byref(cd), _ptr(out), _stream()),
+            "precc_lr_attend_decode_static")
 
     def lr_attend_prefill(self, desc: LayerDesc, q: torch.Tensor, agent: int, ctx_len: int, B_k, B_v, cache: Cache,
                           out: torch.Tensor, block_table: Optional[torch.Tensor] = None, first_block: int = 0):

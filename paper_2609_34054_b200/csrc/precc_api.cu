@@ -28,7 +28,15 @@ struct precc_ctx {
                            CUtensorMapL2promotion, CUtensorMapFloatOOBfill) = nullptr;
 };
 
+// Scratch for precc_lr_attend_decode_static: lives in the library image, one copy per GPU that loads it.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[PRECC_STATIC_SCRATCH_BYTES];
+
 namespace {
+
+// Device address of g_static_scratch on each device, looked up on the first static call there.
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {nullptr};
 
 int32_t fail(precc_ctx* ctx, int32_t code, const char* fmt, ...) {
   if (ctx) {
@@ -526,6 +534,37 @@ int32_t precc_lr_attend_decode(precc_ctx* ctx, const precc_layer_desc* desc, con
   DecodeArgs a{desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, B_v, cache, out,
                workspace, workspace_bytes, (cudaStream_t)stream};
   return dispatch_shape<DecodeRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
+}
+
+int32_t precc_lr_attend_decode_static(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,
+                                      const int32_t* agent_id, const int32_t* ctx_len, const int32_t* block_table,
+                                      int32_t table_stride, const int32_t* first_block, int32_t max_ctx, const void* B_k,
+                                      const void* B_v, const precc_cache* cache, void* out, void* stream) {
+  int32_t rc = check_desc(ctx, desc);
+  if (rc) return rc;
+  if (B < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "B < 0");
+  if (B == 0) return PRECC_OK;
+  if (max_ctx < 1) return fail(ctx, PRECC_ERR_INVALID_ARG, "max_ctx < 1");
+  const size_t need = precc_decode_workspace_bytes(desc, B, max_ctx, ctx->sm_count);
+  if (need == 0) return fail(ctx, PRECC_ERR_UNSUPPORTED, "no decode kernel for this shape");
+  if (need > PRECC_STATIC_SCRATCH_BYTES)
+    return fail(ctx, PRECC_ERR_WORKSPACE, "this call needs %zu bytes of scratch but the built-in array holds %u; "
+                "use precc_lr_attend_decode with a caller workspace", need, (unsigned)PRECC_STATIC_SCRATCH_BYTES);
+  if (ctx->device < 0 || ctx->device >= kMaxDevices) return fail(ctx, PRECC_ERR_UNSUPPORTED, "device index %d >= %d", ctx->device, kMaxDevices);
+  void* scratch = g_static_scratch_addr[ctx->device];
+  if (!scratch) {
+    // once per device, with that device current: the symbol's address differs from GPU to GPU
+    int cur = -1;
+    PRECC_CUDA(ctx, cudaGetDevice(&cur));
+    if (cur != ctx->device) return fail(ctx, PRECC_ERR_INVALID_ARG, "current device %d is not the context's device %d", cur, ctx->device);
+    PRECC_CUDA(ctx, cudaGetSymbolAddress(&scratch, g_static_scratch));
+    g_static_scratch_addr[ctx->device] = scratch;
+  }
+  // the arrival counters at the head of the scratch must be zero when the kernel starts
+  const size_t counters = ((size_t)B * desc->n_kv_heads * 4 + 255) / 256 * 256;
+  PRECC_CUDA(ctx, cudaMemsetAsync(scratch, 0, counters, (cudaStream_t)stream));
+  return precc_lr_attend_decode(ctx, desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, B_v,
+                                cache, out, scratch, PRECC_STATIC_SCRATCH_BYTES, stream);
 }
 
 int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
