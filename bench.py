@@ -76,6 +76,18 @@ def whole_job_value(bytes_per_rank_step: float, steps: int, ms_max: float, world
     return world * bytes_per_rank_step * steps / (ms_max * 1e-3) / 1e9
 
 
+def measured_tensor_peaks():
+    """Dense bf16 TFLOP/s (burst, sustained) from MEASURED_PEAKS.json, else the fallback figures."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            d = json.load(f)
+        return {"bf16_tflops_burst": float(d["bf16_tflops"]), "bf16_tflops_sustained": float(d["bf16_tflops_sustained"]),
+                "peak_kind": "measured"}
+    except Exception:
+        return {"bf16_tflops_burst": 1590.0, "bf16_tflops_sustained": 1400.0, "peak_kind": "fallback"}
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
 
@@ -175,6 +187,111 @@ def run_reference(args):
     print(json.dumps(line))
     return 0
 
+
+
+# ------------------------------------------------------------------------- other rows of the metric
+
+def _event_us(torch, fn, iters, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters * 1e3
+
+
+def extra_serving_decode(px, batch: int, ctx_min: int, ctx_max: int, seed: int = 0):
+    """C4-shaped decode: `batch` requests, agents uniform over 8, contexts uniform in [ctx_min, ctx_max],
+    paged-16 caches with every logical block on its own physical block (a seeded CPU pool of 4096 blocks
+    tiled over the physical pool: values repeat, addresses do not, so every launch streams from HBM)."""
+    import torch
+    from paper_2609_34054_b200 import inputs as I
+    from paper_2609_34054_b200.binding import Cache, layer_desc
+    geo = I.C4
+    agent_id, ctx_len = I.serving_batch(batch, ctx_min, ctx_max, geo.n_agents, seed)
+    need = [(int(t) + 15) // 16 for t in ctx_len]
+    n_phys = sum(need)
+    pool = I.direct_caches(4096, geo, seed, "C4.pool")
+    reps = (n_phys + 4095) // 4096
+    tile = lambda t, dim: torch.cat([t.cuda()] * reps, dim=dim).narrow(dim, 0, n_phys).contiguous()
+    cache = Cache.from_tensors(geo, tile(pool["k_base"], 0), tile(pool["v_base"], 0), tile(pool["lr_k"], 1), tile(pool["lr_v"], 1))
+    table = I.block_tables(ctx_len, n_phys, seed).cuda()
+    w = I.layer_weights(geo, seed, "C4")
+    desc = layer_desc(geo)
+    q = I.queries(batch, geo, seed, "C4.q").cuda()
+    out = torch.empty_like(q)
+    mx = int(ctx_len.max())
+    ws = px.decode_workspace(desc, batch, mx)
+    Bk, Bv, aid, cl = w["B_k"].cuda(), w["B_v"].cuda(), agent_id.cuda(), ctx_len.cuda()
+    us = _event_us(torch, lambda: px.lr_attend_decode(desc, q, aid, cl, mx, Bk, Bv, cache, out, ws, table), iters=10)
+    per_tok = (2 * geo.kv_width + geo.rank_k + geo.rank_v) * 2
+    byt = int(ctx_len.sum()) * per_tok + batch * 2 * geo.n_q * geo.hd * 2 + sum(need) * 4 + geo.n_agents * (geo.rank_k + geo.rank_v) * geo.kv_width * 2
+    peak, kind = measured_peak()
+    gbs = byt / us / 1e3
+    return {"workload": f"C4 serving decode: B={batch}, ctx~U[{ctx_min},{ctx_max}], 28q/4kv hd=128, N=8 r=16, paged-16",
+            "kernel": "lr_attend_decode_kernel<128,16,16> (ticket)", "us_per_launch": us, "algorithmic_bytes": byt,
+            "GBps": gbs, "frac_of_peak": gbs / peak, "peak_kind": kind, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+            "l2_policy": f"{byt / 1e6:.0f} MB of distinct cache per launch >> 126 MB L2"}
+
+
+def extra_turn(px, T: int, S: int, seed: int = 0):
+    """C3-shaped turn of one layer: LR precompute over the context (throughput), then the turn itself
+    (base append + LR precompute of the S new tokens + prefill attention) and the ReBase re-projection."""
+    import torch
+    from paper_2609_34054_b200 import inputs as I
+    from paper_2609_34054_b200.binding import Cache, layer_desc
+    geo = I.C3
+    desc = layer_desc(geo)
+    w = {k: v.cuda() for k, v in I.layer_weights(geo, seed, "C3").items()}
+    A_packed = px.pack_adapters(geo, w["A_k"], w["A_v"])
+    W_packed = px.pack_base_weights(geo, w["W_k"], w["W_v"])
+    cache = Cache(geo, (T + S + 15) // 16)
+    H_ctx = [I.hidden_states(T, geo, seed + i, "C3.H_ctx").cuda() for i in range(2)]     # 2 x 268 MB: rotates past L2
+    H_new = [I.hidden_states(S, geo, seed + i, "C3.H_new_adpt").cuda() for i in range(32)]
+    H_neut = [I.hidden_states(S, geo, seed + i, "C3.H_new_neut").cuda() for i in range(32)]
+    q = I.queries(S, geo, seed, "C3.q").cuda()
+    out = torch.empty_like(q)
+    it = [0]
+
+    def ctx_pre():
+        px.lr_precompute(desc, H_ctx[it[0] % 2], A_packed, cache, 0); it[0] += 1
+
+    def ctx_base():
+        px.rebase_project(desc, H_ctx[it[0] % 2], W_packed, cache, 0); it[0] += 1
+    us_pre = _event_us(torch, ctx_pre, 10)
+    us_base = _event_us(torch, ctx_base, 6)
+    n_lr = geo.n_agents * (geo.rank_k + geo.rank_v)
+    fl_pre = 2.0 * T * geo.d_model * n_lr
+    cur = 1
+
+    def turn():
+        h = H_new[it[0] % 32]; it[0] += 1
+        px.rebase_project(desc, h, W_packed, cache, T)
+        px.lr_precompute(desc, h, A_packed, cache, T)
+        px.lr_attend_prefill(desc, q, cur, T, w["B_k"], w["B_v"], cache, out)
+
+    def rebase():
+        h = H_neut[it[0] % 32]; it[0] += 1
+        px.rebase_project(desc, h, W_packed, cache, T)
+        px.lr_precompute(desc, h, A_packed, cache, T, None, ~(1 << cur))
+    us_turn = _event_us(torch, turn, 5)
+    us_attn = _event_us(torch, lambda: px.lr_attend_prefill(desc, q, cur, T, w["B_k"], w["B_v"], cache, out), 5)
+    us_reb = _event_us(torch, rebase, 10)
+    fl_attn = 4.0 * geo.n_q * S * (geo.hd + (geo.rank_k + geo.rank_v) / 2) * (T + S / 2)
+    return {"workload": f"C3 turn, one layer: d=4096 32q/8kv hd=128, N=4 r=32, T={T}, S={S}",
+            "lr_precompute_context": {"us": us_pre, "tflops": fl_pre / us_pre / 1e6, "n_out": n_lr,
+                                      "GBps": 2.0 * (T * geo.d_model + T * n_lr) / us_pre / 1e3},
+            "base_projection_context": {"us": us_base, "tflops": 2.0 * T * geo.d_model * 2 * geo.kv_width / us_base / 1e6},
+            "turn_us_per_layer": us_turn, "turn_ttft_ms_32_layers": us_turn * C3_LAYERS_FOR_TTFT / 1e3,
+            "prefill_attention": {"us": us_attn, "tflops": fl_attn / us_attn / 1e6},
+            "rebase_us_per_layer": us_reb, "peaks": measured_tensor_peaks()}
+
+
+C3_LAYERS_FOR_TTFT = 32
 
 # ------------------------------------------------------------------------------------------ GPU arm
 
@@ -291,6 +408,12 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     px = Precc(local)
+    if args.extra_only:
+        res = extra_serving_decode(px, args.c4_batch, args.c4_ctx_min, args.c4_ctx_max) if args.extra_only == "c4" \
+            else extra_turn(px, args.c3_ctx, args.c3_new)
+        assert px.poll_status() == 0
+        print(json.dumps(res))
+        return 0
     wl = Workload(px, seed=rank, layers=args.layers, steps=args.decode_steps, T=args.ctx)
     wl.step()                                        # first pass builds the caches (also a warm-up)
     torch.cuda.synchronize()
@@ -368,6 +491,11 @@ def run_gpu(args):
                        "projection_tflops": flops_a / (pa / args.steps * 1e-3) / 1e12,
                        "decode_only_GBps": step_bytes / (pb / args.steps * 1e-3) / 1e9},
         }
+        if world == 1 and not args.no_extra:
+            del wl
+            torch.cuda.empty_cache()
+            line["extra"] = {"serving_decode": extra_serving_decode(px, 64, 4096, 32768),
+                             "turn": extra_turn(px, 32768, 512)}
         if cpu_val is not None:
             line["cpu_baseline"] = {"value": cpu_val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                                     "sample": f"{args.cpu_requests} decode requests of layer 0 (all kv heads, context {I.C2_T}), "
@@ -381,7 +509,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="precc", choices=["precc", "reference"])
     ap.add_argument("--layers", type=int, default=16)
@@ -389,7 +517,14 @@ def main():
     ap.add_argument("--ctx", type=int, default=8192)
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--cpu-requests", type=int, default=40)
+    ap.add_argument("--cpu-requests", type=int, default=120)
+    ap.add_argument("--no-extra", action="store_true", help="skip the C4 decode and C3 turn measurements")
+    ap.add_argument("--extra-only", choices=["c3", "c4"], help="run only that measurement (used for profiling)")
+    ap.add_argument("--c4-batch", type=int, default=64)
+    ap.add_argument("--c4-ctx-min", type=int, default=4096)
+    ap.add_argument("--c4-ctx-max", type=int, default=32768)
+    ap.add_argument("--c3-ctx", type=int, default=32768)
+    ap.add_argument("--c3-new", type=int, default=512)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
