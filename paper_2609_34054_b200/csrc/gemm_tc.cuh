@@ -63,6 +63,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (clock64() - t0 > 2000000000LL) break;
+    // once any wait in the grid has expired the results are void anyway: do not queue up more seconds
+    if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
   }
   atomicOr(status, StatusBits::TIMEOUT);
   return false;

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -12,6 +13,7 @@
 #include "decode.cuh"
 #include "gemm_tc.cuh"
 #include "prefill.cuh"
+#include "prefill_tc.cuh"
 
 using namespace precc;
 
@@ -22,6 +24,7 @@ struct precc_ctx {
   uint32_t* status = nullptr;          // device status word
   unsigned long long* trace = nullptr; // optional caller-owned trace buffer
   size_t trace_blocks = 0;
+  bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
   char err[512] = {0};
   CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                            const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -113,6 +116,22 @@ int32_t make_map(precc_ctx* ctx, CUtensorMap* map, const void* base, int rows, i
   const cuuint32_t estr[2] = {1, 1};
   CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, PRECC_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  return PRECC_OK;
+}
+
+// 2-D bf16 tensor map: `rows` x `cols` (cols contiguous), box `box_rows` x `box_cols`, swizzle = box row bytes.
+int32_t make_map2(precc_ctx* ctx, CUtensorMap* map, const void* base, long long rows, int cols, int box_rows, int box_cols) {
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const int bytes = box_cols * 2;
+  const CUtensorMapSwizzle sw = bytes >= 128 ? CU_TENSOR_MAP_SWIZZLE_128B : bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                : bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(ctx, PRECC_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
   return PRECC_OK;
@@ -323,7 +342,51 @@ struct PrefillArgs {
 
 template <int HD, int RK, int RV>
 struct PrefillRun {
+  // tensor-core kernel (tcgen05 + TMEM + TMA) for the shapes it supports
+  static int32_t run_tc(precc_ctx* ctx, const PrefillArgs& a) {
+    using C = PrefillTcCfg<HD, RK, RV>;
+    const precc_layer_desc* d = a.d;
+    const int G = d->n_q_heads / d->n_kv_heads;
+    int stages = 4;
+    while (stages > 2 && C::smem_bytes(stages) > ctx->max_smem_optin) --stages;
+    const int smem = C::smem_bytes(stages);
+    const size_t kvw = (size_t)d->n_kv_heads * HD;
+    const long long kv_rows = (long long)a.cache->n_blocks * d->n_kv_heads * PAGE;
+    const long long lr_rows = (long long)a.cache->n_blocks * PAGE;
+    CUtensorMap mk, mv, mlk, mlv;
+    int32_t rc = make_map2(ctx, &mk, a.cache->k_base, kv_rows, HD, PAGE, 64);
+    if (rc) return rc;
+    rc = make_map2(ctx, &mv, a.cache->v_base, kv_rows, HD, PAGE, 64);
+    if (rc) return rc;
+    mlk = mk; mlv = mv;     // placeholders when a rank is zero (never dereferenced)
+    if (RK) { rc = make_map2(ctx, &mlk, (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * lr_rows * RK, lr_rows, RK, PAGE, RK); if (rc) return rc; }
+    if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, PAGE, RV); if (rc) return rc; }
+    PrefillTcParams p;
+    p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;
+    p.B_k = RK ? (const __nv_bfloat16*)a.B_k + (size_t)a.agent * RK * kvw : nullptr;
+    p.B_v = RV ? (const __nv_bfloat16*)a.B_v + (size_t)a.agent * RV * kvw : nullptr;
+    p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
+    p.S = a.S; p.T = a.T; p.first_block = a.first_block;
+    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.stages = stages;
+    p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
+    auto kern = lr_attend_prefill_tc_kernel<HD, RK, RV>;
+    PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int row_tiles = (a.S + p.tok_per_tile - 1) / p.tok_per_tile;
+    kern<<<dim3(row_tiles, d->n_kv_heads), PTC_THREADS, smem, a.stream>>>(mk, mv, mlk, mlv, p);
+    PRECC_CUDA(ctx, cudaGetLastError());
+    return PRECC_OK;
+  }
   static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
+    if constexpr (PrefillTcCfg<HD, RK, RV>::supported) {
+      const long long kv_rows = (long long)a.cache->n_blocks * a.d->n_kv_heads * PAGE;
+      const bool aligned128 = ((reinterpret_cast<uintptr_t>(a.cache->k_base) | reinterpret_cast<uintptr_t>(a.cache->v_base) |
+                                reinterpret_cast<uintptr_t>(a.cache->lr_k) | reinterpret_cast<uintptr_t>(a.cache->lr_v)) & 127u) == 0;
+      if (kv_rows < (1ll << 31) && aligned128 && !ctx->force_simple_prefill) return run_tc(ctx, a);
+    }
+    return run_simple(ctx, a);
+  }
+  // mma.sync kernel: ranks 8 and 64, oversized or unaligned caches
+  static int32_t run_simple(precc_ctx* ctx, const PrefillArgs& a) {
     using C = PrefillCfg<HD, RK, RV>;
     const precc_layer_desc* d = a.d;
     int stages = 3;
@@ -382,6 +445,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
     if (e == cudaSuccess && (qres != cudaDriverEntryPointSuccess || !fn)) e = cudaErrorUnknown;
     ctx->encode_tiled = reinterpret_cast<decltype(ctx->encode_tiled)>(fn);
   }
+  if (const char* v = getenv("PRECC_PREFILL")) ctx->force_simple_prefill = (strcmp(v, "simple") == 0);
   if (e != cudaSuccess) {
     fprintf(stderr, "precc_create: %s\n", cudaGetErrorString(e));
     if (ctx->status) cudaFree(ctx->status);

@@ -1,0 +1,467 @@
+// LR-reconstructed attention for the new tokens of a turn on the 5th-generation tensor cores.
+//
+// One thread block = up to 128 query rows of one kv head (row = new token i * G + head-in-group) against
+// the whole visible context, 128 tokens per step:
+//   S  = Q K_base^T + Q~ L_K^T                 tcgen05.mma, A/B from shared memory, S in TMEM (2 buffers)
+//   P  = exp2(S*scale - m)                     4 softmax warps, one TMEM lane (= query row) per thread,
+//                                              written back over S as packed bf16
+//   O' += P [V_base | L_V]                      tcgen05.mma with A = P from TMEM, O' (hd + r_v columns) in TMEM
+// and finally out = (O + s_v U B_v) / l on the CUDA cores.  The key-side fold Q~ = s_k Q B_k^T is
+// computed once per block by the softmax threads.  Pages of the caches arrive by TMA (one box per page
+// and 64-column slab, 128/64/32-byte swizzle) into a ring of stages guarded by mbarriers.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 =
+// softmax / correction / epilogue.  The running maximum is only raised when it grows by more than 8
+// (log2 domain), so O' is rescaled a handful of times per row instead of at every step; P stays
+// below 2^8.  Every mbarrier wait is bounded and falls through with PRECC_STATUS_TIMEOUT.
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace precc {
+
+struct PrefillTcParams {
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  const int32_t* block_table;
+  const __nv_bfloat16* B_k;    // already offset to the agent: [r_k][n_kv*hd]
+  const __nv_bfloat16* B_v;
+  uint32_t* status;
+  int64_t n_blocks;
+  int S, T, first_block;
+  int n_q, n_kv, group;
+  int tok_per_tile;            // 128 / group
+  int stages;
+  float scale_log2, s_k, s_v;
+};
+
+constexpr int PTC_THREADS = 192;
+constexpr int PTC_TOK = 128;      // tokens per step
+constexpr float PTC_RAISE = 8.f;  // the running maximum is raised only when it grows by more than this
+
+template <int HD, int RK, int RV>
+struct PrefillTcCfg {
+  static constexpr int SLABS = HD / 64;                      // 64-column slabs of a base row
+  static constexpr int SLAB_BYTES = PTC_TOK * 128;            // 128 rows x 128 bytes
+  static constexpr int Q_BYTES = SLABS * SLAB_BYTES;
+  static constexpr int QX_BYTES = RK > 0 ? PTC_TOK * RK * 2 : 0;
+  static constexpr int KV_BYTES = SLABS * SLAB_BYTES;
+  static constexpr int LK_BYTES = PTC_TOK * RK * 2;
+  static constexpr int LV_BYTES = PTC_TOK * RV * 2;
+  static constexpr int STAGE_BYTES = 2 * KV_BYTES + LK_BYTES + LV_BYTES;
+  static constexpr int PAGE_TX = PAGE * (2 * HD + RK + RV) * 2;   // bytes one page contributes to a stage
+  static constexpr int TMEM_O = 2 * PTC_TOK;                  // O' starts after the two S buffers
+  __host__ __device__ static constexpr int smem_bytes(int stages) { return Q_BYTES + QX_BYTES + stages * STAGE_BYTES + 256 + 1024; }
+  static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 16 || RK == 32) && (RV == 0 || RV == 16 || RV == 32);
+};
+
+// layout_type field of a shared-memory matrix descriptor for rows of `row_bytes`
+__device__ __forceinline__ constexpr uint64_t umma_layout_for(int row_bytes) {
+  return row_bytes >= 128 ? 2ull : (row_bytes == 64 ? 4ull : 6ull);
+}
+// K-major operand: rows of `row_bytes` (one swizzle span), 8-row groups `8*row_bytes` apart.
+__device__ __forceinline__ uint64_t umma_desc_kmajor(uint32_t saddr, int row_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>((8 * row_bytes) >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= umma_layout_for(row_bytes) << 61;
+  return d;
+}
+// MN-major operand (rows = k index, `row_bytes` of contiguous MN elements per row): 8-row groups
+// `8*row_bytes` apart (stride offset), successive MN blocks `mn_block_stride` bytes apart (leading offset).
+__device__ __forceinline__ uint64_t umma_desc_mnmajor(uint32_t saddr, int row_bytes, int mn_block_stride) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
+  d |= static_cast<uint64_t>((mn_block_stride >> 4) & 0x3FFF) << 16;
+  d |= static_cast<uint64_t>((8 * row_bytes) >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= umma_layout_for(row_bytes) << 61;
+  return d;
+}
+// D fp32, A/B bf16, M = 128, N = n; b_mn = 1 when B is MN-major.
+__device__ __forceinline__ uint32_t umma_idesc(int n, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(b_mn) << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(128 >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+
+template <int HD, int RK, int RV>
+__global__ void __launch_bounds__(PTC_THREADS, 1)
+lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                            const __grid_constant__ CUtensorMap map_lk, const __grid_constant__ CUtensorMap map_lv,
+                            const PrefillTcParams p) {
+  using C = PrefillTcCfg<HD, RK, RV>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  const uint32_t q_u32 = smem_u32(smem);
+  const uint32_t qx_u32 = q_u32 + C::Q_BYTES;
+  const uint32_t ring_u32 = qx_u32 + C::QX_BYTES;
+  unsigned char* ring = smem + C::Q_BYTES + C::QX_BYTES;
+  const int ST = p.stages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)ST * C::STAGE_BYTES);
+  const uint32_t bar0 = smem_u32(bars);
+  // barrier map: kv_full[ST] | kv_empty[ST] | s_full[2] | p_full[2] | pv_done | q_ready
+  const uint32_t kv_full = bar0, kv_empty = bar0 + 8 * ST, s_full = bar0 + 16 * ST, p_full = s_full + 16,
+                 pv_done = p_full + 16, q_ready = pv_done + 8;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * ST + 6);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = blockIdx.y, G = p.group;
+  const int tok0 = blockIdx.x * p.tok_per_tile;
+  const int n_tok = min(p.tok_per_tile, p.S - tok0);             // new tokens handled by this block
+  const int t_end = p.T + tok0 + n_tok;                          // context + causal reach of the last row
+  const int n_tiles = (t_end + PTC_TOK - 1) / PTC_TOK;
+  const int full_vis = p.T + tok0 + 1;                           // tokens visible to every row of the block
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < ST; ++s) { mbar_init(kv_full + 8 * s, 1); mbar_init(kv_empty + 8 * s, 1); }
+    mbar_init(s_full, 1); mbar_init(s_full + 8, 1);
+    mbar_init(p_full, 4); mbar_init(p_full + 8, 4);
+    mbar_init(pv_done, 1);
+    mbar_init(q_ready, 4);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_holder)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    for (int j = 0; j < n_tiles; ++j) {
+      const int s = j % ST;
+      if (j >= ST) mbar_wait(kv_empty + 8 * s, ((j / ST) - 1) & 1, p.status);
+      // the last stage doubles as the staging area of B_k until the query fold is done
+      if (RK > 0 && j == ST - 1) mbar_wait(q_ready, 0, p.status);
+      const int t0 = j * PTC_TOK;
+      const int live = min(PTC_TOK / PAGE, (t_end - t0 + PAGE - 1) / PAGE);
+      const uint32_t st = ring_u32 + (uint32_t)s * C::STAGE_BYTES;
+      const uint32_t full = kv_full + 8 * s;
+      if (lane == 0) mbar_expect_tx(full, live * C::PAGE_TX);
+      __syncwarp();
+      if (lane < live) {
+        const int lt = j * (PTC_TOK / PAGE) + lane;
+        int ph = p.block_table ? __ldg(p.block_table + lt) : p.first_block + lt;
+        if (ph < 0 || ph >= p.n_blocks) { atomicOr(p.status, StatusBits::BAD_INDEX); ph = 0; }
+        const int row_kv = (ph * p.n_kv + g) * PAGE;
+#pragma unroll
+        for (int sl = 0; sl < C::SLABS; ++sl) {
+          tma_load_2d(st + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_k, sl * 64, row_kv, full);
+          tma_load_2d(st + C::KV_BYTES + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_v, sl * 64, row_kv, full);
+        }
+        if constexpr (RK > 0) tma_load_2d(st + 2 * C::KV_BYTES + lane * PAGE * RK * 2, &map_lk, 0, ph * PAGE, full);
+        if constexpr (RV > 0) tma_load_2d(st + 2 * C::KV_BYTES + C::LK_BYTES + lane * PAGE * RV * 2, &map_lv, 0, ph * PAGE, full);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    const uint32_t id_s = umma_idesc(PTC_TOK, 0);
+    const uint32_t id_o = umma_idesc(HD, 1);
+    const uint32_t id_u = umma_idesc(RV > 0 ? RV : 16, 1);
+    auto issue_qk = [&](int j) {
+      const int s = j % ST;
+      mbar_wait(kv_full + 8 * s, (j / ST) & 1, p.status);
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t st = ring_u32 + (uint32_t)s * C::STAGE_BYTES;
+        const uint32_t d = tmem_base + (j & 1) * PTC_TOK;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint32_t off = (ks / 4) * C::SLAB_BYTES + (ks % 4) * 32;
+          umma_bf16(d, umma_desc_kmajor(q_u32 + off, 128), umma_desc_kmajor(st + off, 128), id_s, ks ? 1u : 0u);
+        }
+        if constexpr (RK > 0) {
+#pragma unroll
+          for (int ks = 0; ks < RK / 16; ++ks)
+            umma_bf16(d, umma_desc_kmajor(qx_u32 + ks * 32, RK * 2), umma_desc_kmajor(st + 2 * C::KV_BYTES + ks * 32, RK * 2), id_s, 1u);
+        }
+        umma_commit(s_full + 8 * (j & 1));
+      }
+      __syncwarp();
+    };
+    mbar_wait(q_ready, 0, p.status);
+    tc_fence_after();
+    issue_qk(0);
+    for (int j = 0; j < n_tiles; ++j) {
+      if (j + 1 < n_tiles) issue_qk(j + 1);
+      const int s = j % ST;
+      const uint32_t st = ring_u32 + (uint32_t)s * C::STAGE_BYTES;
+      const int n_live = min(PTC_TOK, t_end - j * PTC_TOK);       // tokens of this step that exist
+      if (n_live < PTC_TOK && (n_live % PAGE) != 0) {
+        // the last page is only partly written: value rows past the end may hold anything, and
+        // 0 * NaN would poison the accumulators, so clear them before the MMA reads the page
+        const int r0 = n_live, r1 = (n_live + PAGE - 1) / PAGE * PAGE;
+        unsigned char* base = ring + (size_t)s * C::STAGE_BYTES;
+        for (int r = r0; r < r1; ++r) {
+          for (int sl = 0; sl < C::SLABS; ++sl)
+            for (int c = lane; c < 8; c += 32) *reinterpret_cast<uint4*>(base + C::KV_BYTES + sl * C::SLAB_BYTES + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+          if constexpr (RV > 0)
+            for (int c = lane; c < RV / 8; c += 32) *reinterpret_cast<uint4*>(base + 2 * C::KV_BYTES + C::LK_BYTES + r * RV * 2 + c * 16) = make_uint4(0, 0, 0, 0);
+        }
+        fence_async_smem();
+        __syncwarp();
+      }
+      mbar_wait(p_full + 8 * (j & 1), (j >> 1) & 1, p.status);
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t a = tmem_base + (j & 1) * PTC_TOK;          // P overlays S (packed bf16, 2 per column)
+        const int n_ks = (n_live + 15) / 16;
+        for (int ks = 0; ks < n_ks; ++ks) {
+          const uint32_t acc = (j | ks) ? 1u : 0u;
+          umma_bf16_ts(tmem_base + C::TMEM_O, a + ks * 8,
+                       umma_desc_mnmajor(st + C::KV_BYTES + ks * 16 * 128, 128, C::SLAB_BYTES), id_o, acc);
+          if constexpr (RV > 0)
+            umma_bf16_ts(tmem_base + C::TMEM_O + HD, a + ks * 8,
+                         umma_desc_mnmajor(st + 2 * C::KV_BYTES + C::LK_BYTES + ks * 16 * RV * 2, RV * 2, 0), id_u, acc);
+        }
+        umma_commit(kv_empty + 8 * s);
+        umma_commit(pv_done);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax / correction / epilogue
+    const int quad = warp & 3;                                    // TMEM lane quadrant this warp may touch
+    const int row = quad * 32 + lane;                             // query row of this thread
+    const int tid = (warp - 2) * 32 + lane;                       // 0..127 among the softmax threads
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+    const int i_new = tok0 + row / G, hg = row % G;
+    const bool row_ok = row < n_tok * G;
+    const int lim = row_ok ? p.T + i_new : -1;                    // last visible token of this row
+    // ---- B_k slice into the last stage, Q row into the swizzled K-major tile, then the fold Q~
+    unsigned char* bk_s = ring + (size_t)(ST - 1) * C::STAGE_BYTES;
+    if constexpr (RK > 0) {
+      for (int c = tid; c < RK * (HD / 8); c += 128) {
+        const int j = c / (HD / 8), ch = c % (HD / 8);
+        *reinterpret_cast<uint4*>(bk_s + (j * HD + ch * 8) * 2) =
+            __ldg(reinterpret_cast<const uint4*>(p.B_k + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
+      }
+    }
+    uint4 qv[HD / 8];
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + ((size_t)i_new * p.n_q + (size_t)g * G + hg) * HD);
+#pragma unroll
+      for (int c = 0; c < HD / 8; ++c) qv[c] = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int c = 0; c < HD / 8; ++c) {
+        const int sl = c / 8, ch = c % 8;
+        *reinterpret_cast<uint4*>(smem + sl * C::SLAB_BYTES + row * 128 + ((ch ^ (row & 7)) * 16)) = qv[c];
+      }
+    }
+    asm volatile("bar.sync 1, 128;\n" ::: "memory");                // B_k slice visible to the softmax threads
+    if constexpr (RK > 0) {
+      constexpr int CPR = RK / 8;
+#pragma unroll 1
+      for (int j0 = 0; j0 < RK; j0 += 8) {
+        uint32_t packed[4];
+#pragma unroll
+        for (int jj = 0; jj < 8; jj += 2) {
+          float a0 = 0.f, a1 = 0.f;
+          const uint32_t* b0 = reinterpret_cast<const uint32_t*>(bk_s + (size_t)(j0 + jj) * HD * 2);
+          const uint32_t* b1 = b0 + HD / 2;
+#pragma unroll
+          for (int c = 0; c < HD / 8; ++c) {
+            const uint32_t xs[4] = {qv[c].x, qv[c].y, qv[c].z, qv[c].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float x0 = bf16_bits_to_float(xs[k] & 0xffff), x1 = bf16_bits_to_float(xs[k] >> 16);
+              const uint32_t y = b0[c * 4 + k], z = b1[c * 4 + k];
+              a0 += x0 * bf16_bits_to_float(y & 0xffff) + x1 * bf16_bits_to_float(y >> 16);
+              a1 += x0 * bf16_bits_to_float(z & 0xffff) + x1 * bf16_bits_to_float(z >> 16);
+            }
+          }
+          packed[jj / 2] = pack_bf16(a0 * p.s_k, a1 * p.s_k);
+        }
+        const int ch = j0 / 8;
+        *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, ch)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+      }
+    }
+    fence_async_smem();                                           // generic-proxy writes -> visible to the MMA unit
+    __syncwarp();
+    if (lane == 0) mbar_arrive(q_ready);
+
+    float m_used = NEG_BIG, l_sum = 0.f;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int b = j & 1;
+      const int t0 = j * PTC_TOK;
+      mbar_wait(s_full + 8 * b, (j >> 1) & 1, p.status);
+      tc_fence_after();
+      uint32_t sv[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(lane_addr + b * PTC_TOK + c * 32, sv[c]);
+      tmem_wait_ld();
+      const bool need_mask = t0 + PTC_TOK > full_vis;
+      float tmax = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+          float z = __uint_as_float(sv[c][k]) * p.scale_log2;
+          if (need_mask && t0 + c * 32 + k > lim) z = -INFINITY;
+          sv[c][k] = __float_as_uint(z);
+          tmax = fmaxf(tmax, z);
+        }
+      float m_new = m_used;
+      if (tmax > m_used + PTC_RAISE) m_new = tmax;
+      const bool raise = m_new != m_used;
+      if (__any_sync(0xffffffffu, raise)) {
+        const float alpha = fast_exp2(m_used - m_new);             // 1 for rows that keep their maximum
+        if (j > 0) {
+          mbar_wait(pv_done, (j - 1) & 1, p.status);               // O' is complete through step j-1
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < (HD + RV) / 32; ++c) {
+            uint32_t ov[32];
+            tmem_ld32(lane_addr + C::TMEM_O + c * 32, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * alpha);
+            tmem_st32(lane_addr + C::TMEM_O + c * 32, ov);
+          }
+          if constexpr ((HD + RV) % 32 != 0) {                     // 16 trailing columns
+            uint32_t ov[16];
+            tmem_ld16(lane_addr + C::TMEM_O + (HD + RV) / 32 * 32, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 16; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * alpha);
+            tmem_st16(lane_addr + C::TMEM_O + (HD + RV) / 32 * 32, ov);
+          }
+          tmem_wait_st();
+        }
+        l_sum *= alpha;
+        m_used = m_new;
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int k = 0; k < 32; k += 2) {
+          const float p0 = fast_exp2(__uint_as_float(sv[c][k]) - m_used);
+          const float p1 = fast_exp2(__uint_as_float(sv[c][k + 1]) - m_used);
+          l_sum += p0 + p1;
+          pk[k / 2] = pack_bf16(p0, p1);
+        }
+        tmem_st16(lane_addr + b * PTC_TOK + c * 16, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full + 8 * b);
+      // observe every phase of pv_done (a parity wait must never lag two phases behind); by now the
+      // previous step's MMAs have normally retired, so this does not stall the pipeline
+      if (j > 0) mbar_wait(pv_done, (j - 1) & 1, p.status);
+    }
+    // ---- epilogue: out = (O + s_v U B_v) / l
+    mbar_wait(pv_done, (n_tiles - 1) & 1, p.status);
+    tc_fence_after();
+    unsigned char* bv_s = ring;                                   // stage 0 is free now
+    if constexpr (RV > 0) {
+      for (int c = tid; c < RV * (HD / 8); c += 128) {
+        const int j = c / (HD / 8), ch = c % (HD / 8);
+        *reinterpret_cast<uint4*>(bv_s + (j * HD + ch * 8) * 2) =
+            __ldg(reinterpret_cast<const uint4*>(p.B_v + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
+      }
+    }
+    asm volatile("bar.sync 1, 128;\n" ::: "memory");
+    float u[RV > 0 ? RV : 1];
+    if constexpr (RV > 0) {
+      uint32_t uv[16];
+#pragma unroll
+      for (int c = 0; c < RV / 16; ++c) {
+        tmem_ld16(lane_addr + C::TMEM_O + HD + c * 16, uv);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) u[c * 16 + k] = __uint_as_float(uv[k]) * p.s_v;
+      }
+    }
+    const float inv = 1.f / l_sum;
+    __nv_bfloat16* orow = p.out + ((size_t)i_new * p.n_q + (size_t)g * G + hg) * HD;
+#pragma unroll 1
+    for (int c = 0; c < HD / 32; ++c) {
+      uint32_t ov[32];
+      tmem_ld32(lane_addr + C::TMEM_O + c * 32, ov);
+      tmem_wait_ld();
+      float o[32];
+#pragma unroll
+      for (int k = 0; k < 32; ++k) o[k] = __uint_as_float(ov[k]);
+      if constexpr (RV > 0) {
+#pragma unroll
+        for (int jv = 0; jv < RV; ++jv) {
+          const uint32_t* bvr = reinterpret_cast<const uint32_t*>(bv_s + (size_t)jv * HD * 2) + c * 16;
+          const float uj = u[jv];
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const uint32_t y = bvr[k];
+            o[2 * k] += uj * bf16_bits_to_float(y & 0xffff);
+            o[2 * k + 1] += uj * bf16_bits_to_float(y >> 16);
+          }
+        }
+      }
+      if (row_ok) {
+#pragma unroll
+        for (int k = 0; k < 32; k += 8) {
+          uint4 w;
+          w.x = pack_bf16(o[k] * inv, o[k + 1] * inv); w.y = pack_bf16(o[k + 2] * inv, o[k + 3] * inv);
+          w.z = pack_bf16(o[k + 4] * inv, o[k + 5] * inv); w.w = pack_bf16(o[k + 6] * inv, o[k + 7] * inv);
+          *reinterpret_cast<uint4*>(orow + c * 32 + k) = w;
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+}  // namespace precc
