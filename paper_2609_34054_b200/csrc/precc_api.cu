@@ -347,9 +347,14 @@ struct PrefillRun {
     using C = PrefillTcCfg<HD, RK, RV>;
     const precc_layer_desc* d = a.d;
     const int G = d->n_q_heads / d->n_kv_heads;
-    int stages = 4;
-    while (stages > 2 && C::smem_bytes(stages) > ctx->max_smem_optin) --stages;
-    const int smem = C::smem_bytes(stages);
+    // as deep as shared memory allows, keys first (they are needed one step earlier)
+    int ks = 2, vs = 2;
+    while (ks + vs < 8) {
+      if (ks <= vs && C::smem_bytes(ks + 1, vs) <= ctx->max_smem_optin) ++ks;
+      else if (C::smem_bytes(ks, vs + 1) <= ctx->max_smem_optin) ++vs;
+      else break;
+    }
+    const int smem = C::smem_bytes(ks, vs);
     const size_t kvw = (size_t)d->n_kv_heads * HD;
     const long long kv_rows = (long long)a.cache->n_blocks * d->n_kv_heads * PAGE;
     const long long lr_rows = (long long)a.cache->n_blocks * PAGE;
@@ -367,7 +372,7 @@ struct PrefillRun {
     p.B_v = RV ? (const __nv_bfloat16*)a.B_v + (size_t)a.agent * RV * kvw : nullptr;
     p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
     p.S = a.S; p.T = a.T; p.first_block = a.first_block;
-    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.stages = stages;
+    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.k_stages = ks; p.v_stages = vs;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
     auto kern = lr_attend_prefill_tc_kernel<HD, RK, RV>;
     PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));

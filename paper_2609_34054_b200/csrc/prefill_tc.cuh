@@ -10,11 +10,15 @@
 // computed once per block by the softmax threads.  Pages of the caches arrive by TMA (one box per page
 // and 64-column slab, 128/64/32-byte swizzle) into a ring of stages guarded by mbarriers.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 =
-// softmax / correction / epilogue.  The running maximum is only raised when it grows by more than 8
+// Warp roles (352 threads): warp 0 = TMA producer of the key ring, warp 10 = TMA producer of the value
+// ring (keys are released right after S is computed, values only after O' is updated, so the two rings
+// run at different distances ahead), warp 1 = TMEM owner + MMA issuer, warps 2..9 = softmax /
+// correction / epilogue, two threads per query row.  The running maximum is only raised when it grows by more than 8
 // (log2 domain), so O' is rescaled a handful of times per row instead of at every step; P stays
 // below 2^8.  Every mbarrier wait is bounded and falls through with PRECC_STATUS_TIMEOUT.
 #pragma once
+#include <type_traits>
+
 #include "gemm_tc.cuh"
 
 namespace precc {
@@ -30,11 +34,11 @@ struct PrefillTcParams {
   int S, T, first_block;
   int n_q, n_kv, group;
   int tok_per_tile;            // 128 / group
-  int stages;
+  int k_stages, v_stages;      // depth of the key ring and of the value ring
   float scale_log2, s_k, s_v;
 };
 
-constexpr int PTC_THREADS = 192;
+constexpr int PTC_THREADS = 352;
 constexpr int PTC_TOK = 128;      // tokens per step
 constexpr float PTC_RAISE = 8.f;  // the running maximum is raised only when it grows by more than this
 
@@ -47,10 +51,12 @@ struct PrefillTcCfg {
   static constexpr int KV_BYTES = SLABS * SLAB_BYTES;
   static constexpr int LK_BYTES = PTC_TOK * RK * 2;
   static constexpr int LV_BYTES = PTC_TOK * RV * 2;
-  static constexpr int STAGE_BYTES = 2 * KV_BYTES + LK_BYTES + LV_BYTES;
-  static constexpr int PAGE_TX = PAGE * (2 * HD + RK + RV) * 2;   // bytes one page contributes to a stage
+  static constexpr int KSTAGE = KV_BYTES + LK_BYTES;          // {K_base slabs | L_K} of 128 tokens
+  static constexpr int VSTAGE = KV_BYTES + LV_BYTES;          // {V_base slabs | L_V}
+  static constexpr int K_PAGE_TX = PAGE * (HD + RK) * 2;      // bytes one page contributes to a key stage
+  static constexpr int V_PAGE_TX = PAGE * (HD + RV) * 2;
   static constexpr int TMEM_O = 2 * PTC_TOK;                  // O' starts after the two S buffers
-  __host__ __device__ static constexpr int smem_bytes(int stages) { return Q_BYTES + QX_BYTES + stages * STAGE_BYTES + 256 + 1024; }
+  __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 256 + 2048 + 1024; }
   static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 16 || RK == 32) && (RV == 0 || RV == 16 || RV == 32);
 };
 
@@ -137,15 +143,17 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const uint32_t q_u32 = smem_u32(smem);
   const uint32_t qx_u32 = q_u32 + C::Q_BYTES;
-  const uint32_t ring_u32 = qx_u32 + C::QX_BYTES;
-  unsigned char* ring = smem + C::Q_BYTES + C::QX_BYTES;
-  const int ST = p.stages;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)ST * C::STAGE_BYTES);
+  const uint32_t kring_u32 = qx_u32 + C::QX_BYTES;
+  const int KS = p.k_stages, VS = p.v_stages;
+  unsigned char* kring = smem + C::Q_BYTES + C::QX_BYTES;
+  unsigned char* vring = kring + (size_t)KS * C::KSTAGE;
+  const uint32_t vring_u32 = kring_u32 + KS * C::KSTAGE;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(vring + (size_t)VS * C::VSTAGE);
   const uint32_t bar0 = smem_u32(bars);
-  // barrier map: kv_full[ST] | kv_empty[ST] | s_full[2] | p_full[2] | pv_done | q_ready
-  const uint32_t kv_full = bar0, kv_empty = bar0 + 8 * ST, s_full = bar0 + 16 * ST, p_full = s_full + 16,
-                 pv_done = p_full + 16, q_ready = pv_done + 8;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * ST + 6);
+  // barrier map: k_full[KS] | k_empty[KS] | v_full[VS] | v_empty[VS] | s_full[2] | p_full[2] | pv_done | q_ready
+  const uint32_t k_full = bar0, k_empty = k_full + 8 * KS, v_full = k_empty + 8 * KS, v_empty = v_full + 8 * VS,
+                 s_full = v_empty + 8 * VS, p_full = s_full + 16, pv_done = p_full + 16, q_ready = pv_done + 8;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * KS + 2 * VS + 6);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.y, G = p.group;
@@ -156,11 +164,12 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   const int full_vis = p.T + tok0 + 1;                           // tokens visible to every row of the block
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < ST; ++s) { mbar_init(kv_full + 8 * s, 1); mbar_init(kv_empty + 8 * s, 1); }
+    for (int s = 0; s < KS; ++s) { mbar_init(k_full + 8 * s, 1); mbar_init(k_empty + 8 * s, 1); }
+    for (int s = 0; s < VS; ++s) { mbar_init(v_full + 8 * s, 1); mbar_init(v_empty + 8 * s, 1); }
     mbar_init(s_full, 1); mbar_init(s_full + 8, 1);
-    mbar_init(p_full, 4); mbar_init(p_full + 8, 4);
+    mbar_init(p_full, 8); mbar_init(p_full + 8, 8);
     mbar_init(pv_done, 1);
-    mbar_init(q_ready, 4);
+    mbar_init(q_ready, 8);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     fence_async_smem();
   }
@@ -173,31 +182,36 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+  if (warp == 0 || warp == 10) {
+    // ------------------------------------------------------------------ TMA producers (keys / values)
+    const bool is_k = warp == 0;
+    const int NS = is_k ? KS : VS;
+    const uint32_t fullb = is_k ? k_full : v_full, emptyb = is_k ? k_empty : v_empty;
     for (int j = 0; j < n_tiles; ++j) {
-      const int s = j % ST;
-      if (j >= ST) mbar_wait(kv_empty + 8 * s, ((j / ST) - 1) & 1, p.status);
-      // the last stage doubles as the staging area of B_k until the query fold is done
-      if (RK > 0 && j == ST - 1) mbar_wait(q_ready, 0, p.status);
+      const int s = j % NS;
+      if (j >= NS) mbar_wait(emptyb + 8 * s, ((j / NS) - 1) & 1, p.status);
+      // the last key stage doubles as the staging area of B_k until the query fold is done
+      if (RK > 0 && is_k && j == KS - 1) mbar_wait(q_ready, 0, p.status);
       const int t0 = j * PTC_TOK;
       const int live = min(PTC_TOK / PAGE, (t_end - t0 + PAGE - 1) / PAGE);
-      const uint32_t st = ring_u32 + (uint32_t)s * C::STAGE_BYTES;
-      const uint32_t full = kv_full + 8 * s;
-      if (lane == 0) mbar_expect_tx(full, live * C::PAGE_TX);
+      const uint32_t st = is_k ? kring_u32 + (uint32_t)s * C::KSTAGE : vring_u32 + (uint32_t)s * C::VSTAGE;
+      const uint32_t full = fullb + 8 * s;
+      if (lane == 0) mbar_expect_tx(full, live * (is_k ? C::K_PAGE_TX : C::V_PAGE_TX));
       __syncwarp();
       if (lane < live) {
         const int lt = j * (PTC_TOK / PAGE) + lane;
         int ph = p.block_table ? __ldg(p.block_table + lt) : p.first_block + lt;
         if (ph < 0 || ph >= p.n_blocks) { atomicOr(p.status, StatusBits::BAD_INDEX); ph = 0; }
         const int row_kv = (ph * p.n_kv + g) * PAGE;
+        if (is_k) {
 #pragma unroll
-        for (int sl = 0; sl < C::SLABS; ++sl) {
-          tma_load_2d(st + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_k, sl * 64, row_kv, full);
-          tma_load_2d(st + C::KV_BYTES + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_v, sl * 64, row_kv, full);
+          for (int sl = 0; sl < C::SLABS; ++sl) tma_load_2d(st + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_k, sl * 64, row_kv, full);
+          if constexpr (RK > 0) tma_load_2d(st + C::KV_BYTES + lane * PAGE * RK * 2, &map_lk, 0, ph * PAGE, full);
+        } else {
+#pragma unroll
+          for (int sl = 0; sl < C::SLABS; ++sl) tma_load_2d(st + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_v, sl * 64, row_kv, full);
+          if constexpr (RV > 0) tma_load_2d(st + C::KV_BYTES + lane * PAGE * RV * 2, &map_lv, 0, ph * PAGE, full);
         }
-        if constexpr (RK > 0) tma_load_2d(st + 2 * C::KV_BYTES + lane * PAGE * RK * 2, &map_lk, 0, ph * PAGE, full);
-        if constexpr (RV > 0) tma_load_2d(st + 2 * C::KV_BYTES + C::LK_BYTES + lane * PAGE * RV * 2, &map_lv, 0, ph * PAGE, full);
       }
       __syncwarp();
     }
@@ -206,23 +220,33 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const uint32_t id_s = umma_idesc(PTC_TOK, 0);
     const uint32_t id_o = umma_idesc(HD, 1);
     const uint32_t id_u = umma_idesc(RV > 0 ? RV : 16, 1);
+    // One thread issues every MMA of the block, so its instruction count per MMA matters: all
+    // descriptors are prepared once (the address field holds addr >> 4, so moving to another stage,
+    // slab or k-step is one 64-bit add of a small constant).
+    const uint64_t qd0 = umma_desc_kmajor(q_u32, 128);
+    const uint64_t qxd0 = RK > 0 ? umma_desc_kmajor(qx_u32, RK * 2) : 0;
+    const uint64_t kd0 = umma_desc_kmajor(kring_u32, 128);
+    const uint64_t lkd0 = RK > 0 ? umma_desc_kmajor(kring_u32 + C::KV_BYTES, RK * 2) : 0;
+    const uint64_t vd0 = umma_desc_mnmajor(vring_u32, 128, C::SLAB_BYTES);
+    const uint64_t lvd0 = RV > 0 ? umma_desc_mnmajor(vring_u32 + C::KV_BYTES, RV * 2, 0) : 0;
     auto issue_qk = [&](int j) {
-      const int s = j % ST;
-      mbar_wait(kv_full + 8 * s, (j / ST) & 1, p.status);
+      const int s = j % KS;
+      mbar_wait(k_full + 8 * s, (j / KS) & 1, p.status);
       tc_fence_after();
       if (lane == 0) {
-        const uint32_t st = ring_u32 + (uint32_t)s * C::STAGE_BYTES;
+        const uint64_t so = (uint64_t)((s * C::KSTAGE) >> 4);
         const uint32_t d = tmem_base + (j & 1) * PTC_TOK;
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
-          const uint32_t off = (ks / 4) * C::SLAB_BYTES + (ks % 4) * 32;
-          umma_bf16(d, umma_desc_kmajor(q_u32 + off, 128), umma_desc_kmajor(st + off, 128), id_s, ks ? 1u : 0u);
+          constexpr int dummy = 0; (void)dummy;
+          const uint64_t off = (uint64_t)(((ks / 4) * C::SLAB_BYTES + (ks % 4) * 32) >> 4);
+          umma_bf16(d, qd0 + off, kd0 + so + off, id_s, ks ? 1u : 0u);
         }
         if constexpr (RK > 0) {
 #pragma unroll
-          for (int ks = 0; ks < RK / 16; ++ks)
-            umma_bf16(d, umma_desc_kmajor(qx_u32 + ks * 32, RK * 2), umma_desc_kmajor(st + 2 * C::KV_BYTES + ks * 32, RK * 2), id_s, 1u);
+          for (int ks = 0; ks < RK / 16; ++ks) umma_bf16(d, qxd0 + (uint64_t)(ks * 2), lkd0 + so + (uint64_t)(ks * 2), id_s, 1u);
         }
+        umma_commit(k_empty + 8 * s);            // the key stage is free as soon as S is computed
         umma_commit(s_full + 8 * (j & 1));
       }
       __syncwarp();
@@ -232,19 +256,19 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     issue_qk(0);
     for (int j = 0; j < n_tiles; ++j) {
       if (j + 1 < n_tiles) issue_qk(j + 1);
-      const int s = j % ST;
-      const uint32_t st = ring_u32 + (uint32_t)s * C::STAGE_BYTES;
+      const int s = j % VS;
       const int n_live = min(PTC_TOK, t_end - j * PTC_TOK);       // tokens of this step that exist
+      mbar_wait(v_full + 8 * s, (j / VS) & 1, p.status);
       if (n_live < PTC_TOK && (n_live % PAGE) != 0) {
         // the last page is only partly written: value rows past the end may hold anything, and
         // 0 * NaN would poison the accumulators, so clear them before the MMA reads the page
         const int r0 = n_live, r1 = (n_live + PAGE - 1) / PAGE * PAGE;
-        unsigned char* base = ring + (size_t)s * C::STAGE_BYTES;
+        unsigned char* base = vring + (size_t)s * C::VSTAGE;
         for (int r = r0; r < r1; ++r) {
           for (int sl = 0; sl < C::SLABS; ++sl)
-            for (int c = lane; c < 8; c += 32) *reinterpret_cast<uint4*>(base + C::KV_BYTES + sl * C::SLAB_BYTES + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+            for (int c = lane; c < 8; c += 32) *reinterpret_cast<uint4*>(base + sl * C::SLAB_BYTES + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
           if constexpr (RV > 0)
-            for (int c = lane; c < RV / 8; c += 32) *reinterpret_cast<uint4*>(base + 2 * C::KV_BYTES + C::LK_BYTES + r * RV * 2 + c * 16) = make_uint4(0, 0, 0, 0);
+            for (int c = lane; c < RV / 8; c += 32) *reinterpret_cast<uint4*>(base + C::KV_BYTES + r * RV * 2 + c * 16) = make_uint4(0, 0, 0, 0);
         }
         fence_async_smem();
         __syncwarp();
@@ -253,104 +277,127 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       tc_fence_after();
       if (lane == 0) {
         const uint32_t a = tmem_base + (j & 1) * PTC_TOK;          // P overlays S (packed bf16, 2 per column)
-        const int n_ks = (n_live + 15) / 16;
-        for (int ks = 0; ks < n_ks; ++ks) {
-          const uint32_t acc = (j | ks) ? 1u : 0u;
-          umma_bf16_ts(tmem_base + C::TMEM_O, a + ks * 8,
-                       umma_desc_mnmajor(st + C::KV_BYTES + ks * 16 * 128, 128, C::SLAB_BYTES), id_o, acc);
-          if constexpr (RV > 0)
-            umma_bf16_ts(tmem_base + C::TMEM_O + HD, a + ks * 8,
-                         umma_desc_mnmajor(st + 2 * C::KV_BYTES + C::LK_BYTES + ks * 16 * RV * 2, RV * 2, 0), id_u, acc);
+        const uint64_t so = (uint64_t)((s * C::VSTAGE) >> 4);
+        const uint32_t od = tmem_base + C::TMEM_O;
+        if (n_live == PTC_TOK) {
+#pragma unroll
+          for (int ks = 0; ks < PTC_TOK / 16; ++ks) {
+            const uint32_t acc = (j | ks) ? 1u : 0u;
+            umma_bf16_ts(od, a + ks * 8, vd0 + so + (uint64_t)(ks * 128), id_o, acc);
+            if constexpr (RV > 0) umma_bf16_ts(od + HD, a + ks * 8, lvd0 + so + (uint64_t)(ks * RV * 2), id_u, acc);
+          }
+        } else {
+          const int n_ks = (n_live + 15) / 16;
+          for (int ks = 0; ks < n_ks; ++ks) {
+            const uint32_t acc = (j | ks) ? 1u : 0u;
+            umma_bf16_ts(od, a + ks * 8, vd0 + so + (uint64_t)(ks * 128), id_o, acc);
+            if constexpr (RV > 0) umma_bf16_ts(od + HD, a + ks * 8, lvd0 + so + (uint64_t)(ks * RV * 2), id_u, acc);
+          }
         }
-        umma_commit(kv_empty + 8 * s);
+        umma_commit(v_empty + 8 * s);
         umma_commit(pv_done);
       }
       __syncwarp();
     }
-  } else {
+  } else if (warp >= 2 && warp <= 9) {
     // ------------------------------------------------------------------ softmax / correction / epilogue
+    // Two threads per query row: warps 2..5 take the first 64 tokens of a step, warps 6..9 the other
+    // 64 (a warp may only touch the TMEM lane quadrant warp % 4, so the pair shares a quadrant).  Two
+    // warps per scheduler let one warp's exponentials overlap the other's TMEM traffic.
     const int quad = warp & 3;                                    // TMEM lane quadrant this warp may touch
+    const int half = (warp - 2) >> 2;                             // which 64 tokens / which output columns
     const int row = quad * 32 + lane;                             // query row of this thread
-    const int tid = (warp - 2) * 32 + lane;                       // 0..127 among the softmax threads
+    const int tid = (warp - 2) * 32 + lane;                       // 0..255 among the softmax threads
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
     const int i_new = tok0 + row / G, hg = row % G;
     const bool row_ok = row < n_tok * G;
     const int lim = row_ok ? p.T + i_new : -1;                    // last visible token of this row
-    // ---- B_k slice into the last stage, Q row into the swizzled K-major tile, then the fold Q~
-    unsigned char* bk_s = ring + (size_t)(ST - 1) * C::STAGE_BYTES;
+    float* xch = reinterpret_cast<float*>(bars + 2 * KS + 2 * VS + 8);   // [2][2][128] row maxima exchanged by the pair
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;\n" ::"r"(2 + quad) : "memory"); };
+    // ---- B_k slice into the last key stage, Q row into the swizzled K-major tile, then the fold Q~
+    unsigned char* bk_s = kring + (size_t)(KS - 1) * C::KSTAGE;
     if constexpr (RK > 0) {
-      for (int c = tid; c < RK * (HD / 8); c += 128) {
+      for (int c = tid; c < RK * (HD / 8); c += 256) {
         const int j = c / (HD / 8), ch = c % (HD / 8);
         *reinterpret_cast<uint4*>(bk_s + (j * HD + ch * 8) * 2) =
             __ldg(reinterpret_cast<const uint4*>(p.B_k + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
       }
     }
-    uint4 qv[HD / 8];
     {
+      uint4 qv[HD / 8];
       const uint4* src = reinterpret_cast<const uint4*>(p.q + ((size_t)i_new * p.n_q + (size_t)g * G + hg) * HD);
 #pragma unroll
       for (int c = 0; c < HD / 8; ++c) qv[c] = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
 #pragma unroll
       for (int c = 0; c < HD / 8; ++c) {
         const int sl = c / 8, ch = c % 8;
-        *reinterpret_cast<uint4*>(smem + sl * C::SLAB_BYTES + row * 128 + ((ch ^ (row & 7)) * 16)) = qv[c];
+        if ((c & 1) == half) *reinterpret_cast<uint4*>(smem + sl * C::SLAB_BYTES + row * 128 + ((ch ^ (row & 7)) * 16)) = qv[c];
       }
-    }
-    asm volatile("bar.sync 1, 128;\n" ::: "memory");                // B_k slice visible to the softmax threads
-    if constexpr (RK > 0) {
-      constexpr int CPR = RK / 8;
+      asm volatile("bar.sync 1, 256;\n" ::: "memory");              // B_k slice visible to the softmax threads
+      if constexpr (RK > 0) {
+        constexpr int CPR = RK / 8;
 #pragma unroll 1
-      for (int j0 = 0; j0 < RK; j0 += 8) {
-        uint32_t packed[4];
+        for (int j0 = half * (RK / 2); j0 < (half + 1) * (RK / 2); j0 += 8) {
+          uint32_t packed[4];
 #pragma unroll
-        for (int jj = 0; jj < 8; jj += 2) {
-          float a0 = 0.f, a1 = 0.f;
-          const uint32_t* b0 = reinterpret_cast<const uint32_t*>(bk_s + (size_t)(j0 + jj) * HD * 2);
-          const uint32_t* b1 = b0 + HD / 2;
+          for (int jj = 0; jj < 8; jj += 2) {
+            float a0 = 0.f, a1 = 0.f;
+            const uint32_t* b0 = reinterpret_cast<const uint32_t*>(bk_s + (size_t)(j0 + jj) * HD * 2);
+            const uint32_t* b1 = b0 + HD / 2;
 #pragma unroll
-          for (int c = 0; c < HD / 8; ++c) {
-            const uint32_t xs[4] = {qv[c].x, qv[c].y, qv[c].z, qv[c].w};
+            for (int c = 0; c < HD / 8; ++c) {
+              const uint32_t xs[4] = {qv[c].x, qv[c].y, qv[c].z, qv[c].w};
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const float x0 = bf16_bits_to_float(xs[k] & 0xffff), x1 = bf16_bits_to_float(xs[k] >> 16);
-              const uint32_t y = b0[c * 4 + k], z = b1[c * 4 + k];
-              a0 += x0 * bf16_bits_to_float(y & 0xffff) + x1 * bf16_bits_to_float(y >> 16);
-              a1 += x0 * bf16_bits_to_float(z & 0xffff) + x1 * bf16_bits_to_float(z >> 16);
+              for (int k = 0; k < 4; ++k) {
+                const float x0 = bf16_bits_to_float(xs[k] & 0xffff), x1 = bf16_bits_to_float(xs[k] >> 16);
+                const uint32_t y = b0[c * 4 + k], z = b1[c * 4 + k];
+                a0 += x0 * bf16_bits_to_float(y & 0xffff) + x1 * bf16_bits_to_float(y >> 16);
+                a1 += x0 * bf16_bits_to_float(z & 0xffff) + x1 * bf16_bits_to_float(z >> 16);
+              }
             }
+            packed[jj / 2] = pack_bf16(a0 * p.s_k, a1 * p.s_k);
           }
-          packed[jj / 2] = pack_bf16(a0 * p.s_k, a1 * p.s_k);
+          *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, j0 / 8)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
         }
-        const int ch = j0 / 8;
-        *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, ch)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
       }
     }
     fence_async_smem();                                           // generic-proxy writes -> visible to the MMA unit
     __syncwarp();
     if (lane == 0) mbar_arrive(q_ready);
 
+    constexpr int OCH = (HD + RV) / 16;                           // 16-column chunks of O'
+    constexpr int OCH0 = (OCH + 1) / 2;                           // chunks rescaled by the first thread of a pair
+    const int och_lo = half ? OCH0 : 0, och_hi = half ? OCH : OCH0;
     float m_used = NEG_BIG, l_sum = 0.f;
-    for (int j = 0; j < n_tiles; ++j) {
+    // One step of the online softmax for this thread's 64 scores.  MASKED is a compile-time flag so
+    // that the common step (far from the causal edge) carries no per-element compare/select.
+    auto step = [&](int j, auto masked_tag) {
+      constexpr bool MASKED = decltype(masked_tag)::value;
       const int b = j & 1;
-      const int t0 = j * PTC_TOK;
-      mbar_wait(s_full + 8 * b, (j >> 1) & 1, p.status);
-      tc_fence_after();
-      uint32_t sv[4][32];
+      const int t0 = j * PTC_TOK + half * 64;
+      uint32_t sv[2][32];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(lane_addr + b * PTC_TOK + c * 32, sv[c]);
+      for (int c = 0; c < 2; ++c) tmem_ld32(lane_addr + b * PTC_TOK + half * 64 + c * 32, sv[c]);
       tmem_wait_ld();
-      const bool need_mask = t0 + PTC_TOK > full_vis;
-      float tmax = -INFINITY;
+      // row maximum of the raw scores (the scale is positive, so it commutes with max); eight
+      // independent chains, because a warp has the scheduler almost to itself
+      const int nvis = lim - t0 + 1;                              // visible tokens among this thread's 64
+      float tm[8];
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
+      for (int k = 0; k < 8; ++k) tm[k] = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
 #pragma unroll
         for (int k = 0; k < 32; ++k) {
-          float z = __uint_as_float(sv[c][k]) * p.scale_log2;
-          if (need_mask && t0 + c * 32 + k > lim) z = -INFINITY;
-          sv[c][k] = __float_as_uint(z);
-          tmax = fmaxf(tmax, z);
+          if (MASKED && c * 32 + k >= nvis) sv[c][k] = 0xff800000u;   // -inf
+          tm[k & 7] = fmaxf(tm[k & 7], __uint_as_float(sv[c][k]));
         }
+      float tmax = fmaxf(fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])), fmaxf(fmaxf(tm[4], tm[5]), fmaxf(tm[6], tm[7]))) * p.scale_log2;
+      xch[(b * 2 + half) * 128 + row] = tmax;
+      pair_sync();
+      tmax = fmaxf(tmax, xch[(b * 2 + (half ^ 1)) * 128 + row]);
       float m_new = m_used;
-      if (tmax > m_used + PTC_RAISE) m_new = tmax;
+      if (tmax > m_used + PTC_RAISE) m_new = tmax;                 // both threads of the pair decide alike
       const bool raise = m_new != m_used;
       if (__any_sync(0xffffffffu, raise)) {
         const float alpha = fast_exp2(m_used - m_new);             // 1 for rows that keep their maximum
@@ -358,39 +405,34 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           mbar_wait(pv_done, (j - 1) & 1, p.status);               // O' is complete through step j-1
           tc_fence_after();
 #pragma unroll 1
-          for (int c = 0; c < (HD + RV) / 32; ++c) {
-            uint32_t ov[32];
-            tmem_ld32(lane_addr + C::TMEM_O + c * 32, ov);
-            tmem_wait_ld();
-#pragma unroll
-            for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * alpha);
-            tmem_st32(lane_addr + C::TMEM_O + c * 32, ov);
-          }
-          if constexpr ((HD + RV) % 32 != 0) {                     // 16 trailing columns
+          for (int c = och_lo; c < och_hi; ++c) {
             uint32_t ov[16];
-            tmem_ld16(lane_addr + C::TMEM_O + (HD + RV) / 32 * 32, ov);
+            tmem_ld16(lane_addr + C::TMEM_O + c * 16, ov);
             tmem_wait_ld();
 #pragma unroll
             for (int k = 0; k < 16; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * alpha);
-            tmem_st16(lane_addr + C::TMEM_O + (HD + RV) / 32 * 32, ov);
+            tmem_st16(lane_addr + C::TMEM_O + c * 16, ov);
           }
           tmem_wait_st();
         }
         l_sum *= alpha;
         m_used = m_new;
       }
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      const float neg_m = -m_used;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t pk[16];
 #pragma unroll
         for (int k = 0; k < 32; k += 2) {
-          const float p0 = fast_exp2(__uint_as_float(sv[c][k]) - m_used);
-          const float p1 = fast_exp2(__uint_as_float(sv[c][k + 1]) - m_used);
-          l_sum += p0 + p1;
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c][k]), p.scale_log2, neg_m));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c][k + 1]), p.scale_log2, neg_m));
+          ls[(k >> 1) & 3] += p0 + p1;
           pk[k / 2] = pack_bf16(p0, p1);
         }
-        tmem_st16(lane_addr + b * PTC_TOK + c * 16, pk);
+        tmem_st16(lane_addr + b * PTC_TOK + half * 32 + c * 16, pk);
       }
+      l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
@@ -398,19 +440,27 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       // observe every phase of pv_done (a parity wait must never lag two phases behind); by now the
       // previous step's MMAs have normally retired, so this does not stall the pipeline
       if (j > 0) mbar_wait(pv_done, (j - 1) & 1, p.status);
+    };
+    for (int j = 0; j < n_tiles; ++j) {
+      mbar_wait(s_full + 8 * (j & 1), (j >> 1) & 1, p.status);
+      tc_fence_after();
+      if (j * PTC_TOK + PTC_TOK > full_vis) step(j, std::true_type{});     // only the last few steps reach the causal edge
+      else step(j, std::false_type{});
     }
-    // ---- epilogue: out = (O + s_v U B_v) / l
+    // ---- epilogue: out = (O + s_v U B_v) / l ; each thread of a pair writes half of the row
     mbar_wait(pv_done, (n_tiles - 1) & 1, p.status);
     tc_fence_after();
-    unsigned char* bv_s = ring;                                   // stage 0 is free now
+    unsigned char* bv_s = vring;                                  // value stage 0 is free now
     if constexpr (RV > 0) {
-      for (int c = tid; c < RV * (HD / 8); c += 128) {
+      for (int c = tid; c < RV * (HD / 8); c += 256) {
         const int j = c / (HD / 8), ch = c % (HD / 8);
         *reinterpret_cast<uint4*>(bv_s + (j * HD + ch * 8) * 2) =
             __ldg(reinterpret_cast<const uint4*>(p.B_v + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
       }
     }
-    asm volatile("bar.sync 1, 128;\n" ::: "memory");
+    xch[half * 128 + row] = l_sum;
+    asm volatile("bar.sync 1, 256;\n" ::: "memory");
+    const float inv = 1.f / (xch[row] + xch[128 + row]);
     float u[RV > 0 ? RV : 1];
     if constexpr (RV > 0) {
       uint32_t uv[16];
@@ -422,23 +472,22 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         for (int k = 0; k < 16; ++k) u[c * 16 + k] = __uint_as_float(uv[k]) * p.s_v;
       }
     }
-    const float inv = 1.f / l_sum;
     __nv_bfloat16* orow = p.out + ((size_t)i_new * p.n_q + (size_t)g * G + hg) * HD;
 #pragma unroll 1
-    for (int c = 0; c < HD / 32; ++c) {
-      uint32_t ov[32];
-      tmem_ld32(lane_addr + C::TMEM_O + c * 32, ov);
+    for (int c = half * (HD / 32); c < (half + 1) * (HD / 32); ++c) {   // 16-column chunks of this thread's half
+      uint32_t ov[16];
+      tmem_ld16(lane_addr + C::TMEM_O + c * 16, ov);
       tmem_wait_ld();
-      float o[32];
+      float o[16];
 #pragma unroll
-      for (int k = 0; k < 32; ++k) o[k] = __uint_as_float(ov[k]);
+      for (int k = 0; k < 16; ++k) o[k] = __uint_as_float(ov[k]);
       if constexpr (RV > 0) {
 #pragma unroll
         for (int jv = 0; jv < RV; ++jv) {
-          const uint32_t* bvr = reinterpret_cast<const uint32_t*>(bv_s + (size_t)jv * HD * 2) + c * 16;
+          const uint32_t* bvr = reinterpret_cast<const uint32_t*>(bv_s + (size_t)jv * HD * 2) + c * 8;
           const float uj = u[jv];
 #pragma unroll
-          for (int k = 0; k < 16; ++k) {
+          for (int k = 0; k < 8; ++k) {
             const uint32_t y = bvr[k];
             o[2 * k] += uj * bf16_bits_to_float(y & 0xffff);
             o[2 * k + 1] += uj * bf16_bits_to_float(y >> 16);
@@ -447,11 +496,11 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       }
       if (row_ok) {
 #pragma unroll
-        for (int k = 0; k < 32; k += 8) {
+        for (int k = 0; k < 16; k += 8) {
           uint4 w;
           w.x = pack_bf16(o[k] * inv, o[k + 1] * inv); w.y = pack_bf16(o[k + 2] * inv, o[k + 3] * inv);
           w.z = pack_bf16(o[k + 4] * inv, o[k + 5] * inv); w.w = pack_bf16(o[k + 6] * inv, o[k + 7] * inv);
-          *reinterpret_cast<uint4*>(orow + c * 32 + k) = w;
+          *reinterpret_cast<uint4*>(orow + c * 16 + k) = w;
         }
       }
     }
