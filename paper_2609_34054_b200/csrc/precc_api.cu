@@ -365,7 +365,7 @@ struct PrefillRun {
     if (rc) return rc;
     mlk = mk; mlv = mv;     // placeholders when a rank is zero (never dereferenced)
     if (RK) { rc = make_map2(ctx, &mlk, (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * lr_rows * RK, lr_rows, RK, PAGE, RK); if (rc) return rc; }
-    if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, PAGE, RV); if (rc) return rc; }
+    if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, PAGE, 64); if (rc) return rc; }
     PrefillTcParams p;
     p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;
     p.B_k = RK ? (const __nv_bfloat16*)a.B_k + (size_t)a.agent * RK * kvw : nullptr;

@@ -10,10 +10,10 @@
 // computed once per block by the softmax threads.  Pages of the caches arrive by TMA (one box per page
 // and 64-column slab, 128/64/32-byte swizzle) into a ring of stages guarded by mbarriers.
 //
-// Warp roles (352 threads): warp 0 = TMA producer of the key ring, warp 10 = TMA producer of the value
-// ring (keys are released right after S is computed, values only after O' is updated, so the two rings
-// run at different distances ahead), warp 1 = TMEM owner + MMA issuer, warps 2..9 = softmax /
-// correction / epilogue, two threads per query row.  The running maximum is only raised when it grows by more than 8
+// Warp roles: warp 0 = TMA producer of the key ring, the last warp = TMA producer of the value ring
+// (keys are released right after S is computed, values only after O' is updated, so the two rings run
+// at different distances ahead), warp 1 = TMEM owner + MMA issuer, the 16 warps in between = softmax /
+// correction / epilogue, four threads per query row.  The running maximum is only raised when it grows by more than 8
 // (log2 domain), so O' is rescaled a handful of times per row instead of at every step; P stays
 // below 2^8.  Every mbarrier wait is bounded and falls through with PRECC_STATUS_TIMEOUT.
 #pragma once
@@ -38,7 +38,11 @@ struct PrefillTcParams {
   float scale_log2, s_k, s_v;
 };
 
-constexpr int PTC_THREADS = 352;
+constexpr int PTC_PARTS_MAX = 4;
+constexpr int PTC_PARTS = 2;                         // softmax threads per query row
+constexpr int PTC_SOFTMAX_WARPS = 4 * PTC_PARTS;
+constexpr int PTC_FIRST_SM_WARP = 3;                 // warps 0..2: key producer, QK^T issuer, PV issuer
+constexpr int PTC_THREADS = (PTC_FIRST_SM_WARP + PTC_SOFTMAX_WARPS + 1) * 32;
 constexpr int PTC_TOK = 128;      // tokens per step
 constexpr float PTC_RAISE = 8.f;  // the running maximum is raised only when it grows by more than this
 
@@ -52,11 +56,13 @@ struct PrefillTcCfg {
   static constexpr int LK_BYTES = PTC_TOK * RK * 2;
   static constexpr int LV_BYTES = PTC_TOK * RV * 2;
   static constexpr int KSTAGE = KV_BYTES + LK_BYTES;          // {K_base slabs | L_K} of 128 tokens
-  static constexpr int VSTAGE = KV_BYTES + LV_BYTES;          // {V_base slabs | L_V}
+  static constexpr int VSLABS = SLABS + (RV > 0 ? 1 : 0);     // L_V rides as one more 64-column slab (zero padded)
+  static constexpr int OW = VSLABS * 64;                      // columns of O' in TMEM: [O | U | padding]
+  static constexpr int VSTAGE = VSLABS * SLAB_BYTES;          // {V_base slabs | L_V slab}
   static constexpr int K_PAGE_TX = PAGE * (HD + RK) * 2;      // bytes one page contributes to a key stage
-  static constexpr int V_PAGE_TX = PAGE * (HD + RV) * 2;
+  static constexpr int V_PAGE_TX = PAGE * VSLABS * 128;
   static constexpr int TMEM_O = 2 * PTC_TOK;                  // O' starts after the two S buffers
-  __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 256 + 2048 + 1024; }
+  __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 320 + 2 * PTC_PARTS_MAX * 512 + 1024; }
   static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 16 || RK == 32) && (RV == 0 || RV == 16 || RV == 32);
 };
 
@@ -150,10 +156,11 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   const uint32_t vring_u32 = kring_u32 + KS * C::KSTAGE;
   uint64_t* bars = reinterpret_cast<uint64_t*>(vring + (size_t)VS * C::VSTAGE);
   const uint32_t bar0 = smem_u32(bars);
-  // barrier map: k_full[KS] | k_empty[KS] | v_full[VS] | v_empty[VS] | s_full[2] | p_full[2] | pv_done | q_ready
+  // barrier map: k_full[KS] | k_empty[KS] | v_full[VS] | v_empty[VS] | s_full[2] | p_full[2] | pv_done | q_ready | s_free[2]
   const uint32_t k_full = bar0, k_empty = k_full + 8 * KS, v_full = k_empty + 8 * KS, v_empty = v_full + 8 * VS,
-                 s_full = v_empty + 8 * VS, p_full = s_full + 16, pv_done = p_full + 16, q_ready = pv_done + 8;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * KS + 2 * VS + 6);
+                 s_full = v_empty + 8 * VS, p_full = s_full + 16, pv_done = p_full + 16, q_ready = pv_done + 8,
+                 s_free = q_ready + 8;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * KS + 2 * VS + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.y, G = p.group;
@@ -167,9 +174,10 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     for (int s = 0; s < KS; ++s) { mbar_init(k_full + 8 * s, 1); mbar_init(k_empty + 8 * s, 1); }
     for (int s = 0; s < VS; ++s) { mbar_init(v_full + 8 * s, 1); mbar_init(v_empty + 8 * s, 1); }
     mbar_init(s_full, 1); mbar_init(s_full + 8, 1);
-    mbar_init(p_full, 8); mbar_init(p_full + 8, 8);
+    mbar_init(p_full, PTC_SOFTMAX_WARPS); mbar_init(p_full + 8, PTC_SOFTMAX_WARPS);
     mbar_init(pv_done, 1);
-    mbar_init(q_ready, 8);
+    mbar_init(s_free, 1); mbar_init(s_free + 8, 1);
+    mbar_init(q_ready, PTC_SOFTMAX_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     fence_async_smem();
   }
@@ -182,7 +190,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
-  if (warp == 0 || warp == 10) {
+  if (warp == 0 || warp == PTC_FIRST_SM_WARP + PTC_SOFTMAX_WARPS) {
     // ------------------------------------------------------------------ TMA producers (keys / values)
     const bool is_k = warp == 0;
     const int NS = is_k ? KS : VS;
@@ -210,27 +218,28 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         } else {
 #pragma unroll
           for (int sl = 0; sl < C::SLABS; ++sl) tma_load_2d(st + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_v, sl * 64, row_kv, full);
-          if constexpr (RV > 0) tma_load_2d(st + C::KV_BYTES + lane * PAGE * RV * 2, &map_lv, 0, ph * PAGE, full);
+          if constexpr (RV > 0) tma_load_2d(st + C::SLABS * C::SLAB_BYTES + lane * PAGE * 128, &map_lv, 0, ph * PAGE, full);
         }
       }
       __syncwarp();
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ S = Q' K'^T issuer
+    // One thread issues these MMAs and another (warp 2) the P V' ones: an MMA costs its issuing thread
+    // on the order of a hundred cycles, so two issue streams are needed to keep the tensor pipe fed.
+    // All descriptors are prepared once (the address field holds addr >> 4, so moving to another
+    // stage, slab or k-step is one 64-bit add of a small constant).
     const uint32_t id_s = umma_idesc(PTC_TOK, 0);
-    const uint32_t id_o = umma_idesc(HD, 1);
-    const uint32_t id_u = umma_idesc(RV > 0 ? RV : 16, 1);
-    // One thread issues every MMA of the block, so its instruction count per MMA matters: all
-    // descriptors are prepared once (the address field holds addr >> 4, so moving to another stage,
-    // slab or k-step is one 64-bit add of a small constant).
     const uint64_t qd0 = umma_desc_kmajor(q_u32, 128);
     const uint64_t qxd0 = RK > 0 ? umma_desc_kmajor(qx_u32, RK * 2) : 0;
     const uint64_t kd0 = umma_desc_kmajor(kring_u32, 128);
     const uint64_t lkd0 = RK > 0 ? umma_desc_kmajor(kring_u32 + C::KV_BYTES, RK * 2) : 0;
-    const uint64_t vd0 = umma_desc_mnmajor(vring_u32, 128, C::SLAB_BYTES);
-    const uint64_t lvd0 = RV > 0 ? umma_desc_mnmajor(vring_u32 + C::KV_BYTES, RV * 2, 0) : 0;
-    auto issue_qk = [&](int j) {
+    mbar_wait(q_ready, 0, p.status);
+    for (int j = 0; j < n_tiles; ++j) {
       const int s = j % KS;
+      // S buffer j&1 still holds P of step j-2 until that step's P V' has been executed (one barrier
+      // per buffer, so this wait is never more than one phase behind)
+      if (j >= 2) mbar_wait(s_free + 8 * (j & 1), ((j >> 1) - 1) & 1, p.status);
       mbar_wait(k_full + 8 * s, (j / KS) & 1, p.status);
       tc_fence_after();
       if (lane == 0) {
@@ -238,7 +247,6 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         const uint32_t d = tmem_base + (j & 1) * PTC_TOK;
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
-          constexpr int dummy = 0; (void)dummy;
           const uint64_t off = (uint64_t)(((ks / 4) * C::SLAB_BYTES + (ks % 4) * 32) >> 4);
           umma_bf16(d, qd0 + off, kd0 + so + off, id_s, ks ? 1u : 0u);
         }
@@ -250,12 +258,12 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         umma_commit(s_full + 8 * (j & 1));
       }
       __syncwarp();
-    };
-    mbar_wait(q_ready, 0, p.status);
-    tc_fence_after();
-    issue_qk(0);
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ O' += P V' issuer
+    const uint32_t id_o = umma_idesc(C::OW, 1);
+    const uint64_t vd0 = umma_desc_mnmajor(vring_u32, 128, C::SLAB_BYTES);
     for (int j = 0; j < n_tiles; ++j) {
-      if (j + 1 < n_tiles) issue_qk(j + 1);
       const int s = j % VS;
       const int n_live = min(PTC_TOK, t_end - j * PTC_TOK);       // tokens of this step that exist
       mbar_wait(v_full + 8 * s, (j / VS) & 1, p.status);
@@ -264,12 +272,9 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         // 0 * NaN would poison the accumulators, so clear them before the MMA reads the page
         const int r0 = n_live, r1 = (n_live + PAGE - 1) / PAGE * PAGE;
         unsigned char* base = vring + (size_t)s * C::VSTAGE;
-        for (int r = r0; r < r1; ++r) {
-          for (int sl = 0; sl < C::SLABS; ++sl)
+        for (int r = r0; r < r1; ++r)
+          for (int sl = 0; sl < C::VSLABS; ++sl)
             for (int c = lane; c < 8; c += 32) *reinterpret_cast<uint4*>(base + sl * C::SLAB_BYTES + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
-          if constexpr (RV > 0)
-            for (int c = lane; c < RV / 8; c += 32) *reinterpret_cast<uint4*>(base + C::KV_BYTES + r * RV * 2 + c * 16) = make_uint4(0, 0, 0, 0);
-        }
         fence_async_smem();
         __syncwarp();
       }
@@ -281,83 +286,81 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         const uint32_t od = tmem_base + C::TMEM_O;
         if (n_live == PTC_TOK) {
 #pragma unroll
-          for (int ks = 0; ks < PTC_TOK / 16; ++ks) {
-            const uint32_t acc = (j | ks) ? 1u : 0u;
-            umma_bf16_ts(od, a + ks * 8, vd0 + so + (uint64_t)(ks * 128), id_o, acc);
-            if constexpr (RV > 0) umma_bf16_ts(od + HD, a + ks * 8, lvd0 + so + (uint64_t)(ks * RV * 2), id_u, acc);
-          }
+          for (int ks = 0; ks < PTC_TOK / 16; ++ks) umma_bf16_ts(od, a + ks * 8, vd0 + so + (uint64_t)(ks * 128), id_o, (j | ks) ? 1u : 0u);
         } else {
           const int n_ks = (n_live + 15) / 16;
-          for (int ks = 0; ks < n_ks; ++ks) {
-            const uint32_t acc = (j | ks) ? 1u : 0u;
-            umma_bf16_ts(od, a + ks * 8, vd0 + so + (uint64_t)(ks * 128), id_o, acc);
-            if constexpr (RV > 0) umma_bf16_ts(od + HD, a + ks * 8, lvd0 + so + (uint64_t)(ks * RV * 2), id_u, acc);
-          }
+          for (int ks = 0; ks < n_ks; ++ks) umma_bf16_ts(od, a + ks * 8, vd0 + so + (uint64_t)(ks * 128), id_o, (j | ks) ? 1u : 0u);
         }
         umma_commit(v_empty + 8 * s);
+        umma_commit(s_free + 8 * (j & 1));
         umma_commit(pv_done);
       }
       __syncwarp();
     }
-  } else if (warp >= 2 && warp <= 9) {
+  } else if (warp >= PTC_FIRST_SM_WARP && warp < PTC_FIRST_SM_WARP + PTC_SOFTMAX_WARPS) {
     // ------------------------------------------------------------------ softmax / correction / epilogue
-    // Two threads per query row: warps 2..5 take the first 64 tokens of a step, warps 6..9 the other
-    // 64 (a warp may only touch the TMEM lane quadrant warp % 4, so the pair shares a quadrant).  Two
-    // warps per scheduler let one warp's exponentials overlap the other's TMEM traffic.
+    // PTC_PARTS threads per query row, each owning 128/PTC_PARTS tokens of a step (a warp may only touch
+    // the TMEM lane quadrant warp % 4, so the threads of a row sit in warps whose ids agree modulo 4).
+    // Several warps per scheduler let one warp's exponentials overlap another's TMEM traffic.
+    constexpr int NP = PTC_PARTS;
+    constexpr int COLS = PTC_TOK / NP;                            // score columns per thread (32)
+    constexpr int NSM = PTC_SOFTMAX_WARPS * 32;                   // softmax threads
     const int quad = warp & 3;                                    // TMEM lane quadrant this warp may touch
-    const int half = (warp - 2) >> 2;                             // which 64 tokens / which output columns
+    const int part = (warp - PTC_FIRST_SM_WARP) >> 2;             // which tokens / which output columns
     const int row = quad * 32 + lane;                             // query row of this thread
-    const int tid = (warp - 2) * 32 + lane;                       // 0..255 among the softmax threads
+    const int tid = (warp - PTC_FIRST_SM_WARP) * 32 + lane;
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
     const int i_new = tok0 + row / G, hg = row % G;
     const bool row_ok = row < n_tok * G;
     const int lim = row_ok ? p.T + i_new : -1;                    // last visible token of this row
-    float* xch = reinterpret_cast<float*>(bars + 2 * KS + 2 * VS + 8);   // [2][2][128] row maxima exchanged by the pair
-    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;\n" ::"r"(2 + quad) : "memory"); };
+    float* xch = reinterpret_cast<float*>(bars + 2 * KS + 2 * VS + 10);   // [2][NP][128] row maxima exchanged by a row's threads
+    auto row_sync = [&]() { asm volatile("bar.sync %0, %1;\n" ::"r"(2 + quad), "r"(32 * NP) : "memory"); };
     // ---- B_k slice into the last key stage, Q row into the swizzled K-major tile, then the fold Q~
     unsigned char* bk_s = kring + (size_t)(KS - 1) * C::KSTAGE;
     if constexpr (RK > 0) {
-      for (int c = tid; c < RK * (HD / 8); c += 256) {
+      for (int c = tid; c < RK * (HD / 8); c += NSM) {
         const int j = c / (HD / 8), ch = c % (HD / 8);
         *reinterpret_cast<uint4*>(bk_s + (j * HD + ch * 8) * 2) =
             __ldg(reinterpret_cast<const uint4*>(p.B_k + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
       }
     }
     {
-      uint4 qv[HD / 8];
       const uint4* src = reinterpret_cast<const uint4*>(p.q + ((size_t)i_new * p.n_q + (size_t)g * G + hg) * HD);
 #pragma unroll
-      for (int c = 0; c < HD / 8; ++c) qv[c] = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-#pragma unroll
       for (int c = 0; c < HD / 8; ++c) {
-        const int sl = c / 8, ch = c % 8;
-        if ((c & 1) == half) *reinterpret_cast<uint4*>(smem + sl * C::SLAB_BYTES + row * 128 + ((ch ^ (row & 7)) * 16)) = qv[c];
+        if ((c % NP) == part) {
+          const int sl = c / 8, ch = c % 8;
+          *reinterpret_cast<uint4*>(smem + sl * C::SLAB_BYTES + row * 128 + ((ch ^ (row & 7)) * 16)) =
+              row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+        }
       }
-      asm volatile("bar.sync 1, 256;\n" ::: "memory");              // B_k slice visible to the softmax threads
+      asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");      // B_k slice and the Q tile are visible
       if constexpr (RK > 0) {
         constexpr int CPR = RK / 8;
 #pragma unroll 1
-        for (int j0 = half * (RK / 2); j0 < (half + 1) * (RK / 2); j0 += 8) {
-          uint32_t packed[4];
+        for (int j0 = part * 8; j0 < RK; j0 += NP * 8) {           // this thread folds coordinates j0 .. j0+7
+          float acc[8];
 #pragma unroll
-          for (int jj = 0; jj < 8; jj += 2) {
-            float a0 = 0.f, a1 = 0.f;
-            const uint32_t* b0 = reinterpret_cast<const uint32_t*>(bk_s + (size_t)(j0 + jj) * HD * 2);
-            const uint32_t* b1 = b0 + HD / 2;
+          for (int jj = 0; jj < 8; ++jj) acc[jj] = 0.f;
+#pragma unroll 2
+          for (int c = 0; c < HD / 8; ++c) {
+            const int sl = c / 8, ch = c % 8;
+            const uint4 qq = *reinterpret_cast<const uint4*>(smem + sl * C::SLAB_BYTES + row * 128 + ((ch ^ (row & 7)) * 16));
+            const uint32_t xs[4] = {qq.x, qq.y, qq.z, qq.w};
 #pragma unroll
-            for (int c = 0; c < HD / 8; ++c) {
-              const uint32_t xs[4] = {qv[c].x, qv[c].y, qv[c].z, qv[c].w};
+            for (int jj = 0; jj < 8; ++jj) {
+              const uint32_t* bb = reinterpret_cast<const uint32_t*>(bk_s + (size_t)(j0 + jj) * HD * 2) + c * 4;
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
-                const float x0 = bf16_bits_to_float(xs[k] & 0xffff), x1 = bf16_bits_to_float(xs[k] >> 16);
-                const uint32_t y = b0[c * 4 + k], z = b1[c * 4 + k];
-                a0 += x0 * bf16_bits_to_float(y & 0xffff) + x1 * bf16_bits_to_float(y >> 16);
-                a1 += x0 * bf16_bits_to_float(z & 0xffff) + x1 * bf16_bits_to_float(z >> 16);
+                const uint32_t y = bb[k];
+                acc[jj] += bf16_bits_to_float(xs[k] & 0xffff) * bf16_bits_to_float(y & 0xffff) +
+                           bf16_bits_to_float(xs[k] >> 16) * bf16_bits_to_float(y >> 16);
               }
             }
-            packed[jj / 2] = pack_bf16(a0 * p.s_k, a1 * p.s_k);
           }
-          *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, j0 / 8)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+          *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, j0 / 8)) =
+              make_uint4(pack_bf16(acc[0] * p.s_k, acc[1] * p.s_k), pack_bf16(acc[2] * p.s_k, acc[3] * p.s_k),
+                         pack_bf16(acc[4] * p.s_k, acc[5] * p.s_k), pack_bf16(acc[6] * p.s_k, acc[7] * p.s_k));
         }
       }
     }
@@ -365,39 +368,36 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     __syncwarp();
     if (lane == 0) mbar_arrive(q_ready);
 
-    constexpr int OCH = (HD + RV) / 16;                           // 16-column chunks of O'
-    constexpr int OCH0 = (OCH + 1) / 2;                           // chunks rescaled by the first thread of a pair
-    const int och_lo = half ? OCH0 : 0, och_hi = half ? OCH : OCH0;
+    constexpr int OCH = (HD + RV) / 16;                           // 16-column chunks of O' that carry data
     float m_used = NEG_BIG, l_sum = 0.f;
-    // One step of the online softmax for this thread's 64 scores.  MASKED is a compile-time flag so
+    // One step of the online softmax for this thread's COLS scores.  MASKED is a compile-time flag so
     // that the common step (far from the causal edge) carries no per-element compare/select.
     auto step = [&](int j, auto masked_tag) {
       constexpr bool MASKED = decltype(masked_tag)::value;
       const int b = j & 1;
-      const int t0 = j * PTC_TOK + half * 64;
-      uint32_t sv[2][32];
+      const int t0 = j * PTC_TOK + part * COLS;
+      constexpr int NCH = COLS / 32;
+      uint32_t sv[NCH][32];
 #pragma unroll
-      for (int c = 0; c < 2; ++c) tmem_ld32(lane_addr + b * PTC_TOK + half * 64 + c * 32, sv[c]);
+      for (int c = 0; c < NCH; ++c) tmem_ld32(lane_addr + b * PTC_TOK + part * COLS + c * 32, sv[c]);
       tmem_wait_ld();
-      // row maximum of the raw scores (the scale is positive, so it commutes with max); eight
-      // independent chains, because a warp has the scheduler almost to itself
-      const int nvis = lim - t0 + 1;                              // visible tokens among this thread's 64
-      float tm[8];
+      // row maximum of the raw scores (the scale is positive, so it commutes with max)
+      const int nvis = lim - t0 + 1;                              // visible tokens among this thread's
+      float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int k = 0; k < 8; ++k) tm[k] = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 2; ++c)
+      for (int c = 0; c < NCH; ++c)
 #pragma unroll
         for (int k = 0; k < 32; ++k) {
           if (MASKED && c * 32 + k >= nvis) sv[c][k] = 0xff800000u;   // -inf
-          tm[k & 7] = fmaxf(tm[k & 7], __uint_as_float(sv[c][k]));
+          tm[k & 3] = fmaxf(tm[k & 3], __uint_as_float(sv[c][k]));
         }
-      float tmax = fmaxf(fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])), fmaxf(fmaxf(tm[4], tm[5]), fmaxf(tm[6], tm[7]))) * p.scale_log2;
-      xch[(b * 2 + half) * 128 + row] = tmax;
-      pair_sync();
-      tmax = fmaxf(tmax, xch[(b * 2 + (half ^ 1)) * 128 + row]);
+      float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])) * p.scale_log2;
+      xch[(b * NP + part) * 128 + row] = tmax;
+      row_sync();
+#pragma unroll
+      for (int q2 = 0; q2 < NP; ++q2) tmax = fmaxf(tmax, xch[(b * NP + q2) * 128 + row]);
       float m_new = m_used;
-      if (tmax > m_used + PTC_RAISE) m_new = tmax;                 // both threads of the pair decide alike
+      if (tmax > m_used + PTC_RAISE) m_new = tmax;                 // all threads of the row decide alike
       const bool raise = m_new != m_used;
       if (__any_sync(0xffffffffu, raise)) {
         const float alpha = fast_exp2(m_used - m_new);             // 1 for rows that keep their maximum
@@ -405,7 +405,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           mbar_wait(pv_done, (j - 1) & 1, p.status);               // O' is complete through step j-1
           tc_fence_after();
 #pragma unroll 1
-          for (int c = och_lo; c < och_hi; ++c) {
+          for (int c = part; c < OCH; c += NP) {
             uint32_t ov[16];
             tmem_ld16(lane_addr + C::TMEM_O + c * 16, ov);
             tmem_wait_ld();
@@ -421,7 +421,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
       const float neg_m = -m_used;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < NCH; ++c) {
         uint32_t pk[16];
 #pragma unroll
         for (int k = 0; k < 32; k += 2) {
@@ -430,7 +430,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           ls[(k >> 1) & 3] += p0 + p1;
           pk[k / 2] = pack_bf16(p0, p1);
         }
-        tmem_st16(lane_addr + b * PTC_TOK + half * 32 + c * 16, pk);
+        tmem_st16(lane_addr + b * PTC_TOK + part * (COLS / 2) + c * 16, pk);
       }
       l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       tmem_wait_st();
@@ -447,20 +447,23 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       if (j * PTC_TOK + PTC_TOK > full_vis) step(j, std::true_type{});     // only the last few steps reach the causal edge
       else step(j, std::false_type{});
     }
-    // ---- epilogue: out = (O + s_v U B_v) / l ; each thread of a pair writes half of the row
+    // ---- epilogue: out = (O + s_v U B_v) / l ; the threads of a row share its output columns
     mbar_wait(pv_done, (n_tiles - 1) & 1, p.status);
     tc_fence_after();
     unsigned char* bv_s = vring;                                  // value stage 0 is free now
     if constexpr (RV > 0) {
-      for (int c = tid; c < RV * (HD / 8); c += 256) {
+      for (int c = tid; c < RV * (HD / 8); c += NSM) {
         const int j = c / (HD / 8), ch = c % (HD / 8);
         *reinterpret_cast<uint4*>(bv_s + (j * HD + ch * 8) * 2) =
             __ldg(reinterpret_cast<const uint4*>(p.B_v + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
       }
     }
-    xch[half * 128 + row] = l_sum;
-    asm volatile("bar.sync 1, 256;\n" ::: "memory");
-    const float inv = 1.f / (xch[row] + xch[128 + row]);
+    xch[part * 128 + row] = l_sum;
+    asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+    float l_tot = 0.f;
+#pragma unroll
+    for (int q2 = 0; q2 < NP; ++q2) l_tot += xch[q2 * 128 + row];
+    const float inv = 1.f / l_tot;
     float u[RV > 0 ? RV : 1];
     if constexpr (RV > 0) {
       uint32_t uv[16];
@@ -474,7 +477,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     }
     __nv_bfloat16* orow = p.out + ((size_t)i_new * p.n_q + (size_t)g * G + hg) * HD;
 #pragma unroll 1
-    for (int c = half * (HD / 32); c < (half + 1) * (HD / 32); ++c) {   // 16-column chunks of this thread's half
+    for (int c = part; c < HD / 16; c += NP) {                    // 16-column chunks of this thread
       uint32_t ov[16];
       tmem_ld16(lane_addr + C::TMEM_O + c * 16, ov);
       tmem_wait_ld();
