@@ -37,7 +37,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch of this workload, from the ncu
 # capture summarised under profiles/ (None until a capture exists)
-NCU_DECODE_TRAFFIC_BYTES = None
+NCU_DECODE_TRAFFIC_BYTES = 17370112   # profiles/decode_cluster_c2_layer.md
 
 
 def decode_bytes_per_launch(geo, ctx: int, batch: int = 1, distinct_agents: int = 1) -> int:
@@ -483,7 +483,7 @@ def run_gpu(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(), "d2h_bytes_per_step": wl.d2h_bytes(),
                     "ms_per_step": ms_e2e / e2e_steps},
             "gpu_launches": (wl.launches_a + wl.launches_b) * args.steps,
-            "roofline": {"bound": "hbm", "kernel": "lr_attend_decode_kernel<64,16,16>", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": "lr_attend_decode_cluster_kernel<64,16,16,8>", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
                          "traffic": NCU_DECODE_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": per_launch,
                          "avg_launch_us": launch_us},
