@@ -6,10 +6,12 @@
 //   mode 0  LR precompute (Section 3.1):  column -> (projection, agent, r index), LR cache rows
 //   mode 1  base projection (Section 3.2): column -> (projection, kv head, c), base cache rows
 //
-// One 128 x BN output tile per thread block.  Warp roles: warp 0 = TMA producer (one lane),
-// warp 1 = TMEM owner + MMA issuer (one lane), warps 2..5 = epilogue (one TMEM lane = one row each).
-// A STAGES-deep ring of {X tile 128x64, Wt tile BNx64} in 128-byte-swizzled shared memory is handed
-// from producer to issuer with mbarriers; tcgen05.commit releases a stage when its MMAs have read it.
+// Persistent blocks, 128 x BN output tiles.  Warp roles: warp 0 = TMA producer (one lane), warp 1 =
+// TMEM owner + MMA issuer (one lane), warps 2..5 = epilogue (one TMEM lane = one row each).  A
+// STAGES-deep ring of {X tile 128x64, Wt tile BNx64} in 128-byte-swizzled shared memory is handed from
+// producer to issuer with mbarriers; tcgen05.commit releases a stage when its MMAs have read it.  The
+// accumulator is double-buffered in TMEM (2 x BN columns), so a tile's epilogue overlaps the next
+// tile's MMAs.
 // Every wait is bounded: on expiry the waiter records PRECC_STATUS_TIMEOUT and carries on, so the
 // kernel always terminates and frees its TMEM.
 #pragma once
@@ -117,18 +119,22 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const int b_bytes = p.BN * GEMM_BK * 2;
   const int stage_bytes = GEMM_A_BYTES + b_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes);
+  // barrier map: full[stages] | empty[stages] | acc_full[2] | acc_empty[2]
   const uint32_t full0 = smem_u32(bars);
   const uint32_t empty0 = full0 + 8 * p.stages;
-  const uint32_t tfull = empty0 + 8 * p.stages;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * p.stages + 1);
+  const uint32_t acc_full = empty0 + 8 * p.stages;
+  const uint32_t acc_empty = acc_full + 16;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * p.stages + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * GEMM_BM, n0 = blockIdx.y * p.BN;
   const int nkb = p.K / GEMM_BK;
+  const int n_tiles_n = (p.N_out + p.BN - 1) / p.BN;
+  const int n_tiles = ((p.M + GEMM_BM - 1) / GEMM_BM) * n_tiles_n;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    mbar_init(tfull, 1);
+    mbar_init(acc_full, 1); mbar_init(acc_full + 8, 1);
+    mbar_init(acc_empty, 4); mbar_init(acc_empty + 8, 4);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
   }
@@ -141,79 +147,103 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
   const uint32_t tmem_base = *tmem_holder;
 
+  // Persistent: this block takes tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the column tile index
+  // runs fastest, so blocks working at the same time share their row tile of X in L2.  The shared
+  // memory ring runs straight through tile boundaries and the accumulator is double-buffered in TMEM,
+  // so the epilogue of one tile overlaps the MMAs of the next.
   if (warp == 0) {
     if (lane == 0) {
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % p.stages;
-        if (kb >= p.stages) mbar_wait(empty0 + 8 * s, ((kb / p.stages) - 1) & 1, p.status);
-        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        mbar_expect_tx(full0 + 8 * s, stage_bytes);
-        tma_load_2d(sa, &map_x, kb * GEMM_BK, m0, full0 + 8 * s);
-        tma_load_2d(sa + GEMM_A_BYTES, &map_w, kb * GEMM_BK, n0, full0 + 8 * s);
+      int it = 0;
+      for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        const int m0 = (t / n_tiles_n) * GEMM_BM, n0 = (t % n_tiles_n) * p.BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % p.stages;
+          if (it >= p.stages) mbar_wait(empty0 + 8 * s, ((it / p.stages) - 1) & 1, p.status);
+          const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+          mbar_expect_tx(full0 + 8 * s, stage_bytes);
+          tma_load_2d(sa, &map_x, kb * GEMM_BK, m0, full0 + 8 * s);
+          tma_load_2d(sa + GEMM_A_BYTES, &map_w, kb * GEMM_BK, n0, full0 + 8 * s);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(p.BN);
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % p.stages;
-        mbar_wait(full0 + 8 * s, (kb / p.stages) & 1, p.status);
+      const uint64_t da0 = umma_desc_sw128(smem_u32(smem));
+      const uint64_t db0 = umma_desc_sw128(smem_u32(smem) + GEMM_A_BYTES);
+      int it = 0, i = 0;
+      for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
+        const int buf = i & 1;
+        if (i >= 2) mbar_wait(acc_empty + 8 * buf, ((i >> 1) - 1) & 1, p.status);   // epilogue has drained this buffer
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint64_t da = umma_desc_sw128(sa), db = umma_desc_sw128(sa + GEMM_A_BYTES);
+        const uint32_t d = tmem_base + buf * p.BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % p.stages;
+          mbar_wait(full0 + 8 * s, (it / p.stages) & 1, p.status);
+          asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+          const uint64_t so = (uint64_t)((s * stage_bytes) >> 4);
 #pragma unroll
-        for (int k = 0; k < GEMM_BK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
-          umma_bf16(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
-        umma_commit(empty0 + 8 * s);             // stage reusable once these MMAs have read it
+          for (int k = 0; k < GEMM_BK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
+            umma_bf16(d, da0 + so + 2 * k, db0 + so + 2 * k, idesc, (kb | k) ? 1u : 0u);
+          umma_commit(empty0 + 8 * s);             // stage reusable once these MMAs have read it
+        }
+        umma_commit(acc_full + 8 * buf);           // accumulator of this tile complete
       }
-      umma_commit(tfull);                        // accumulator complete
     }
   } else {
     // ---- epilogue: TMEM lane = tile row; this warp may touch lanes 32*(warp%4) .. +31
     const int lane_base = (warp & 3) * 32;
     const int row = lane_base + lane;
-    const int gm = m0 + row;
-    bool row_ok = gm < p.M;
-    long long slot = 0;
-    if (row_ok) {
-      slot = p.slot_mapping ? (long long)p.slot_mapping[gm] : p.start_slot + gm;
-      if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
-    }
-    const long long blk = slot / PAGE;
-    const int off = (int)(slot % PAGE);
-    mbar_wait(tfull, 0, p.status);
-    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     const int n_k = p.n_agents * p.rank_k;
     const int w = p.n_kv * p.hd;
-    for (int c0 = 0; c0 < p.BN; c0 += 16) {
-      uint32_t r[16];
-      tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + c0, r);
-      asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int gc = n0 + c0 + 8 * h;
-        if (!row_ok || gc >= p.N_out) continue;
-        __nv_bfloat16* dst;
-        if (p.mode == 0) {
-          const bool is_v = gc >= n_k;
-          const int rr = is_v ? p.rank_v : p.rank_k;
-          const int cc = is_v ? gc - n_k : gc;
-          const int agent = cc / rr, ri = cc % rr;
-          if (!((p.agent_mask >> agent) & 1ull)) continue;
-          dst = (is_v ? p.dst1 : p.dst0) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
-        } else {
-          const bool is_v = gc >= w;
-          const int cc = is_v ? gc - w : gc;
-          const int g = cc / p.hd, c = cc % p.hd;
-          dst = (is_v ? p.dst1 : p.dst0) + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
-        }
-        uint4 v;
-        v.x = pack_bf16(__uint_as_float(r[8 * h + 0]), __uint_as_float(r[8 * h + 1]));
-        v.y = pack_bf16(__uint_as_float(r[8 * h + 2]), __uint_as_float(r[8 * h + 3]));
-        v.z = pack_bf16(__uint_as_float(r[8 * h + 4]), __uint_as_float(r[8 * h + 5]));
-        v.w = pack_bf16(__uint_as_float(r[8 * h + 6]), __uint_as_float(r[8 * h + 7]));
-        *reinterpret_cast<uint4*>(dst) = v;
+    int i = 0;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
+      const int buf = i & 1;
+      const int m0 = (t / n_tiles_n) * GEMM_BM, n0 = (t % n_tiles_n) * p.BN;
+      const int gm = m0 + row;
+      bool row_ok = gm < p.M;
+      long long slot = 0;
+      if (row_ok) {
+        slot = p.slot_mapping ? (long long)p.slot_mapping[gm] : p.start_slot + gm;
+        if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
       }
+      const long long blk = slot / PAGE;
+      const int off = (int)(slot % PAGE);
+      mbar_wait(acc_full + 8 * buf, (i >> 1) & 1, p.status);
+      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+      for (int c0 = 0; c0 < p.BN; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + buf * p.BN + c0, r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int gc = n0 + c0 + 8 * h;
+          if (!row_ok || gc >= p.N_out) continue;
+          __nv_bfloat16* dst;
+          if (p.mode == 0) {
+            const bool is_v = gc >= n_k;
+            const int rr = is_v ? p.rank_v : p.rank_k;
+            const int cc = is_v ? gc - n_k : gc;
+            const int agent = cc / rr, ri = cc % rr;
+            if (!((p.agent_mask >> agent) & 1ull)) continue;
+            dst = (is_v ? p.dst1 : p.dst0) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
+          } else {
+            const bool is_v = gc >= w;
+            const int cc = is_v ? gc - w : gc;
+            const int g = cc / p.hd, c = cc % p.hd;
+            dst = (is_v ? p.dst1 : p.dst0) + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
+          }
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(r[8 * h + 0]), __uint_as_float(r[8 * h + 1]));
+          v.y = pack_bf16(__uint_as_float(r[8 * h + 2]), __uint_as_float(r[8 * h + 3]));
+          v.z = pack_bf16(__uint_as_float(r[8 * h + 4]), __uint_as_float(r[8 * h + 5]));
+          v.w = pack_bf16(__uint_as_float(r[8 * h + 6]), __uint_as_float(r[8 * h + 7]));
+          *reinterpret_cast<uint4*>(dst) = v;
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(acc_empty + 8 * buf) : "memory");
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");

@@ -155,8 +155,8 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   if (stages > K / GEMM_BK) stages = K / GEMM_BK;
   if (stages < 1) return fail(ctx, PRECC_ERR_CUDA, "not enough shared memory for one GEMM stage");
   int tmem_cols = 32;
-  while (tmem_cols < bn) tmem_cols <<= 1;
-  const size_t smem = (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 1024;
+  while (tmem_cols < 2 * bn) tmem_cols <<= 1;      // two accumulator buffers
+  const size_t smem = (size_t)stages * stage_bytes + (2 * stages + 6) * 8 + 1024;
   CUtensorMap map_x, map_w;
   int32_t rc = make_map(ctx, &map_x, X, M, K, GEMM_BM);
   if (rc) return rc;
@@ -165,7 +165,8 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
   gp.status = ctx->status;
   PRECC_CUDA(ctx, cudaFuncSetAttribute(proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  proj_gemm_kernel<<<dim3(m_tiles, n_tiles), GEMM_THREADS, smem, stream>>>(map_x, map_w, gp);
+  const int total_tiles = m_tiles * n_tiles;
+  proj_gemm_kernel<<<dim3(total_tiles < ctx->sm_count ? total_tiles : ctx->sm_count), GEMM_THREADS, smem, stream>>>(map_x, map_w, gp);
   PRECC_CUDA(ctx, cudaGetLastError());
   return PRECC_OK;
 }
