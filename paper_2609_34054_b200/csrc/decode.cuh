@@ -206,37 +206,51 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
       a[1] = 0u; a[3] = 0u;
     }
   };
+  // Only warp 0 loads B_k and folds; the other warps pick the folded fragments up from shared memory
+  // (every warp needs the same ones, and the load/store unit is what limits the start of the stream).
   uint32_t bk_pre[PRELOAD_BK ? KX * KC : 1][4];
   if constexpr (PRELOAD_BK) {
+    if (warp == 0) {
 #pragma unroll
-    for (int jt = 0; jt < KX; ++jt)
+      for (int jt = 0; jt < KX; ++jt)
 #pragma unroll
-      for (int kc = 0; kc < KC; ++kc) load_bk(jt, kc, bk_pre[jt * KC + kc]);
+        for (int kc = 0; kc < KC; ++kc) load_bk(jt, kc, bk_pre[jt * KC + kc]);
+    }
   }
   // ---- start the stream: every ring slot is filled at once
   for (int i = 0; i < p.stages; ++i) issue_tile(i);
   mark(2);
 
-  // ---- folded key-side adapter q~ = s_k q B_k[a][:, g]^T, computed per warp on the tensor cores as
+  // ---- folded key-side adapter q~ = s_k q B_k[a][:, g]^T, computed on the tensor cores as
   //      q~^T[j x q] = B_k[j x c] . q^T[c x q]; the accumulator fragment, transposed with movmatrix,
   //      is exactly the B operand (k = j, n = query) needed by the score MMA.
   uint32_t qxb[KX > 0 ? KX : 1][2];
   if constexpr (RK > 0) {
+    __shared__ uint32_t qx_share[KX > 0 ? KX : 1][2][32];
+    if (warp == 0) {
 #pragma unroll
-    for (int jt = 0; jt < KX; ++jt) {
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int jt = 0; jt < KX; ++jt) {
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int kc = 0; kc < KC; ++kc) {
-        if constexpr (PRELOAD_BK) {
-          mma_bf16_16816(c, bk_pre[jt * KC + kc], qb[kc][0], qb[kc][1]);
-        } else {
-          uint32_t a[4];
-          load_bk(jt, kc, a);
-          mma_bf16_16816(c, a, qb[kc][0], qb[kc][1]);
+        for (int kc = 0; kc < KC; ++kc) {
+          if constexpr (PRELOAD_BK) {
+            mma_bf16_16816(c, bk_pre[jt * KC + kc], qb[kc][0], qb[kc][1]);
+          } else {
+            uint32_t a[4];
+            load_bk(jt, kc, a);
+            mma_bf16_16816(c, a, qb[kc][0], qb[kc][1]);
+          }
         }
+        qxb[jt][0] = movmatrix_t(pack_bf16(c[0] * p.s_k, c[1] * p.s_k));
+        qxb[jt][1] = movmatrix_t(pack_bf16(c[2] * p.s_k, c[3] * p.s_k));
+        qx_share[jt][0][lane] = qxb[jt][0];
+        qx_share[jt][1][lane] = qxb[jt][1];
       }
-      qxb[jt][0] = movmatrix_t(pack_bf16(c[0] * p.s_k, c[1] * p.s_k));
-      qxb[jt][1] = movmatrix_t(pack_bf16(c[2] * p.s_k, c[3] * p.s_k));
+    }
+    __syncthreads();
+    if (warp != 0) {
+#pragma unroll
+      for (int jt = 0; jt < KX; ++jt) { qxb[jt][0] = qx_share[jt][0][lane]; qxb[jt][1] = qx_share[jt][1][lane]; }
     }
   }
 
