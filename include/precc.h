@@ -138,6 +138,17 @@ int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const
                              const void* W_packed, const int32_t* slot_mapping, int64_t start_slot,
                              const precc_cache* cache, void* stream);
 
+/* Both of the above in one pass over H (Section 3.1: the hidden states of a newly processed segment
+ * feed the base cache and every agent's LR cache; Section 3.2: the adapter-free pass writes the neutral
+ * base rows and the other agents' LR rows).  H is read from HBM once and one kernel runs instead of two.
+ *   WA_packed  [2*n_kv_heads*head_dim + n_agents*(rank_k+rank_v)][d_model]: the packed W rows followed by
+ *              the packed A rows (precc_pack_kmajor into one buffer)
+ *   agent_mask selects the LR caches written; the base rows are always written.
+ * Results are bit-identical to precc_rebase_project followed by precc_lr_precompute. */
+int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
+                           const void* WA_packed, const int32_t* slot_mapping, int64_t start_slot,
+                           uint64_t agent_mask, const precc_cache* cache, void* stream);
+
 /* Workspace size for precc_lr_attend_decode with at most max_batch requests of at most max_ctx tokens
  * on a device with `sm_count` SMs.  The workspace must be zeroed once (precc_workspace_init) before its
  * first use; calls leave it ready for the next call.  Two calls that may run concurrently need
@@ -152,7 +163,9 @@ int32_t precc_workspace_init(precc_ctx* ctx, void* workspace, size_t workspace_b
  *   out_h = sum_t softmax(z)_t V_base[t,g] + s_v (sum_t softmax(z)_t L^V_a[t]) B^V_{a,g}
  * which equals plain attention with K_a = K_base + s_k L^K_a B^K_a and V_a likewise (Eq. 1).
  *   q, out        [B][n_q_heads][head_dim]
- *   agent_id      [B] in [0, n_agents);  ctx_len [B] >= 1 (a request with ctx_len < 1 gets zeros)
+ *   agent_id      [B] in [0, n_agents), or -1 for the adapter-free view of Section 3.2 (double batching:
+ *                 the request attends to its base cache only; no LR row and no B matrix is touched);
+ *                 ctx_len [B] >= 1 (a request with ctx_len < 1 gets zeros)
  *   block_table   [B][table_stride] logical block -> physical block, or NULL
  *   first_block   [B] physical block of logical block 0 when block_table is NULL (NULL = 0 for all)
  *   max_ctx       HOST upper bound on every ctx_len[b]; with B and the SM count it fixes the split of
@@ -199,7 +212,8 @@ int32_t precc_lr_attend_decode_static(precc_ctx* ctx, const precc_layer_desc* de
  * (0 <= i < S) attends logical positions 0 .. ctx_len + i: the old context fully, the new tokens
  * causally.  Same formula as decode.
  *   q, out       [S][n_q_heads][head_dim]
- *   agent        the current agent (host value);  ctx_len  T, tokens before the new ones (host value)
+ *   agent        the current agent, or -1 for the adapter-free pass over the neutral base cache (host
+ *                value);  ctx_len  T, tokens before the new ones (host value)
  *   block_table  [table_stride] logical -> physical block for this sequence, or NULL
  *   first_block  physical block of logical block 0 when block_table is NULL
  * No workspace is needed.  S == 0 is a no-op. */

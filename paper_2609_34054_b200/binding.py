@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libprecc.so")
 
 EXPORTS = [
     "precc_create", "precc_destroy", "precc_last_error", "precc_error_name", "precc_sm_count", "precc_set_trace_buffer",
-    "precc_poll_status", "precc_pack_kmajor", "precc_lr_precompute", "precc_rebase_project",
+    "precc_poll_status", "precc_pack_kmajor", "precc_lr_precompute", "precc_rebase_project", "precc_turn_project",
     "precc_decode_workspace_bytes", "precc_workspace_init", "precc_lr_attend_decode",
     "precc_lr_attend_decode_static", "precc_lr_attend_prefill",
 ]
@@ -65,6 +65,7 @@ def load_library() -> C.CDLL:
     lib.precc_pack_kmajor.argtypes = [vp, vp, i32, i32, vp, i32, i32, vp]
     lib.precc_lr_precompute.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, u64, C.POINTER(CacheDesc), vp]
     lib.precc_rebase_project.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, C.POINTER(CacheDesc), vp]
+    lib.precc_turn_project.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, u64, C.POINTER(CacheDesc), vp]
     lib.precc_decode_workspace_bytes.argtypes = [C.POINTER(LayerDesc), i32, i32, i32]
     lib.precc_decode_workspace_bytes.restype = sz
     lib.precc_workspace_init.argtypes = [vp, vp, sz, vp]
@@ -194,6 +195,26 @@ class Precc:
         self.pack_kmajor(W_k, dst, 0)
         self.pack_kmajor(W_v, dst, geo.kv_width)
         return dst
+
+    def pack_turn_weights(self, geo: Geometry, W_k, W_v, A_k, A_v) -> torch.Tensor:
+        """Packed W rows followed by packed A rows: the operand of ``turn_project``."""
+        n_lr = geo.n_agents * (geo.rank_k + geo.rank_v)
+        dst = torch.empty((2 * geo.kv_width + n_lr, geo.d_model), dtype=torch.bfloat16, device=W_k.device)
+        self.pack_kmajor(W_k, dst, 0)
+        self.pack_kmajor(W_v, dst, geo.kv_width)
+        at = 2 * geo.kv_width
+        for A, r in ((A_k, geo.rank_k), (A_v, geo.rank_v)):
+            for k in range(geo.n_agents if r else 0):
+                self.pack_kmajor(A[k], dst, at)
+                at += r
+        return dst
+
+    def turn_project(self, desc: LayerDesc, H: torch.Tensor, WA_packed: torch.Tensor, cache: Cache,
+                     start_slot: int = 0, slot_mapping: Optional[torch.Tensor] = None, agent_mask: int = (1 << 64) - 1):
+        cd = cache.desc()
+        self._check(self.lib.precc_turn_project(self.h, C.byref(desc), _ptr(H), H.shape[0], _ptr(WA_packed),
+                                                _ptr(slot_mapping), start_slot, agent_mask & ((1 << 64) - 1),
+                                                C.byref(cd), _stream()), "precc_turn_project")
 
     # ------------------------------------------------------------------ the four entry points
     def lr_precompute(self, desc: LayerDesc, H: torch.Tensor, A_packed: torch.Tensor, cache: Cache,

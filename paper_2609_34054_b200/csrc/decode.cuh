@@ -116,7 +116,7 @@ __device__ __forceinline__ void load_q_frags(const DecodeParams& p, int b, int g
 // m = NEG_BIG, l = 0, O' = 0.
 template <int HD, int RK, int RV, int NW>
 __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsigned char* smem, int b, int g, int ctx,
-                                                    int agent, int tile0, int tile_end,
+                                                    int agent, bool use_lr, int tile0, int tile_end,
                                                     const uint32_t (&qb)[HD / 16][2], const DecodeTrace& mark) {
   using C = DecodeCfg<HD, RK, RV>;
   constexpr int OW = C::OW;
@@ -170,7 +170,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
         // (an unwritten slot may hold NaN) must not reach the accumulators
         cp_async16(st + C::KV_BYTES + off, vsrc + c * 16, row < valid ? 16 : 0);
       }
-      if constexpr (RK > 0) {
+      if (RK > 0 && use_lr) {
         const unsigned char* src = reinterpret_cast<const unsigned char*>(lrk_a + (size_t)ph * PAGE * RK);
 #pragma unroll
         for (int c = lane; c < PAGE * CPR_LK; c += 32) {
@@ -178,7 +178,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
           cp_async16(st + 2 * C::KV_BYTES + swz_off<CPR_LK>(row, ch), src + c * 16, 16);
         }
       }
-      if constexpr (RV > 0) {
+      if (RV > 0 && use_lr) {
         const unsigned char* src = reinterpret_cast<const unsigned char*>(lrv_a + (size_t)ph * PAGE * RV);
 #pragma unroll
         for (int c = lane; c < PAGE * CPR_LV; c += 32) {
@@ -210,7 +210,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   // (every warp needs the same ones, and the load/store unit is what limits the start of the stream).
   uint32_t bk_pre[PRELOAD_BK ? KX * KC : 1][4];
   if constexpr (PRELOAD_BK) {
-    if (warp == 0) {
+    if (warp == 0 && use_lr) {
 #pragma unroll
       for (int jt = 0; jt < KX; ++jt)
 #pragma unroll
@@ -227,7 +227,9 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   uint32_t qxb[KX > 0 ? KX : 1][2];
   if constexpr (RK > 0) {
     __shared__ uint32_t qx_share[KX > 0 ? KX : 1][2][32];
-    if (warp == 0) {
+#pragma unroll
+    for (int jt = 0; jt < KX; ++jt) { qxb[jt][0] = 0u; qxb[jt][1] = 0u; }
+    if (warp == 0 && use_lr) {
 #pragma unroll
       for (int jt = 0; jt < KX; ++jt) {
         float c[4] = {0.f, 0.f, 0.f, 0.f};
@@ -248,7 +250,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
       }
     }
     __syncthreads();
-    if (warp != 0) {
+    if (warp != 0 && use_lr) {
 #pragma unroll
       for (int jt = 0; jt < KX; ++jt) { qxb[jt][0] = qx_share[jt][0][lane]; qxb[jt][1] = qx_share[jt][1][lane]; }
     }
@@ -285,7 +287,8 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
       ldsm_x4(a, st + swz_off<CPR_KV>(a_row, 2 * kc + a_cpar));
       mma_bf16_16816(s, a, qb[kc][0], qb[kc][1]);
     }
-    if constexpr (RK >= 16) {
+    if (!use_lr) {
+    } else if constexpr (RK >= 16) {
 #pragma unroll
       for (int kc = 0; kc < KX; ++kc) {
         uint32_t a[4];
@@ -326,7 +329,8 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
       ldsm_x4_t(a, st + C::KV_BYTES + swz_off<CPR_KV>(v_row, 2 * mt + v_cpar));
       mma_bf16_16816(o[mt], a, pb0, pb1);
     }
-    if constexpr (RV >= 16) {
+    if (!use_lr) {
+    } else if constexpr (RV >= 16) {
 #pragma unroll
       for (int mx = 0; mx < MX; ++mx) {
         uint32_t a[4];
@@ -419,9 +423,11 @@ lr_attend_decode_kernel(const DecodeParams p) {
   uint32_t qb[HD / 16][2];    // independent of the index arrays: same round trip
   load_q_frags<HD>(p, b, g, qb);
   const int ctx = __ldg(p.ctx_len + b);
-  const int agent = __ldg(p.agent_id + b);
+  const int agent_raw = __ldg(p.agent_id + b);
+  const bool use_lr = agent_raw >= 0;          // agent id -1: adapter-free view, base cache only
+  const int agent = use_lr ? agent_raw : 0;
   __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
-  if (ctx < 1 || agent < 0 || agent >= p.n_agents) {
+  if (ctx < 1 || agent_raw < -1 || agent_raw >= p.n_agents) {
     if (split == 0) {
       for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
       if (threadIdx.x == 0 && ctx >= 1) atomicOr(p.status, StatusBits::BAD_INDEX);
@@ -434,7 +440,7 @@ lr_attend_decode_kernel(const DecodeParams p) {
   const int tile0 = split * p.chunk_tiles;
   const int tile_end = min(n_tiles, tile0 + p.chunk_tiles);
   mark(1);
-  decode_stream_block<HD, RK, RV, DEC_WARPS>(p, smem, b, g, ctx, agent, tile0, tile_end, qb, mark);
+  decode_stream_block<HD, RK, RV, DEC_WARPS>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, qb, mark);
 
   float* res = reinterpret_cast<float*>(smem);          // [m[8] | l[8] | O'[G][OW]]
   const int n_el = G * OW;
@@ -598,9 +604,11 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   uint32_t qb[HD / 16][2];
   load_q_frags<HD>(p, b, g, qb);
   const int ctx = __ldg(p.ctx_len + b);
-  const int agent = __ldg(p.agent_id + b);
+  const int agent_raw = __ldg(p.agent_id + b);
+  const bool use_lr = agent_raw >= 0;          // agent id -1: adapter-free view, base cache only
+  const int agent = use_lr ? agent_raw : 0;
   __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
-  if (ctx < 1 || agent < 0 || agent >= p.n_agents) {   // the same decision in every block of the cluster
+  if (ctx < 1 || agent_raw < -1 || agent_raw >= p.n_agents) {   // the same decision in every block of the cluster
     if (rank == 0) {
       for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
       if (threadIdx.x == 0 && ctx >= 1) atomicOr(p.status, StatusBits::BAD_INDEX);
@@ -623,7 +631,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
       bv_pre[k] = (i < RV * cols_) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);
     }
   }
-  decode_stream_block<HD, RK, RV, NW>(p, smem, b, g, ctx, agent, tile0, tile_end, qb, mark);
+  decode_stream_block<HD, RK, RV, NW>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, qb, mark);
 
   // own result res = [m[8] | l[8] | O'[G][OW]] sits at the start of shared memory in every block
   float* res = reinterpret_cast<float*>(smem);

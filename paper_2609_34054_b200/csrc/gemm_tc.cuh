@@ -5,6 +5,8 @@
 // with a scatter epilogue that writes bf16 rows straight into the paged caches:
 //   mode 0  LR precompute (Section 3.1):  column -> (projection, agent, r index), LR cache rows
 //   mode 1  base projection (Section 3.2): column -> (projection, kv head, c), base cache rows
+//   mode 2  both at once: the first 2*n_kv*hd columns go to the base caches, the rest to the LR caches
+//           (the hidden states of a newly processed segment are read once, Section 3.1)
 //
 // Persistent blocks, 128 x BN output tiles.  Warp roles: warp 0 = TMA producer (one lane), warp 1 =
 // TMEM owner + MMA issuer (one lane), warps 2..5 = epilogue (one TMEM lane = one row each).  A
@@ -24,12 +26,14 @@ namespace precc {
 struct GemmParams {
   int M, N_out, K;
   int BN, stages, tmem_cols;
-  int mode;                       // 0 = LR caches, 1 = base caches
+  int mode;                       // 0 = LR caches, 1 = base caches, 2 = base columns then LR columns
   const int32_t* slot_mapping;    // [M] or null
   int64_t start_slot;
   int64_t n_blocks;
-  __nv_bfloat16* dst0;            // lr_k or k_base
-  __nv_bfloat16* dst1;            // lr_v or v_base
+  __nv_bfloat16* base_k;          // modes 1, 2
+  __nv_bfloat16* base_v;
+  __nv_bfloat16* lr_k;            // modes 0, 2
+  __nv_bfloat16* lr_v;
   int n_agents, rank_k, rank_v;
   unsigned long long agent_mask;
   int n_kv, hd;
@@ -220,18 +224,20 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
           const int gc = n0 + c0 + 8 * h;
           if (!row_ok || gc >= p.N_out) continue;
           __nv_bfloat16* dst;
-          if (p.mode == 0) {
-            const bool is_v = gc >= n_k;
+          const bool to_base = p.mode == 1 || (p.mode == 2 && gc < 2 * w);
+          if (!to_base) {
+            const int gl = p.mode == 2 ? gc - 2 * w : gc;
+            const bool is_v = gl >= n_k;
             const int rr = is_v ? p.rank_v : p.rank_k;
-            const int cc = is_v ? gc - n_k : gc;
+            const int cc = is_v ? gl - n_k : gl;
             const int agent = cc / rr, ri = cc % rr;
             if (!((p.agent_mask >> agent) & 1ull)) continue;
-            dst = (is_v ? p.dst1 : p.dst0) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
+            dst = (is_v ? p.lr_v : p.lr_k) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
           } else {
             const bool is_v = gc >= w;
             const int cc = is_v ? gc - w : gc;
             const int g = cc / p.hd, c = cc % p.hd;
-            dst = (is_v ? p.dst1 : p.dst0) + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
+            dst = (is_v ? p.base_v : p.base_k) + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
           }
           uint4 v;
           v.x = pack_bf16(__uint_as_float(r[8 * h + 0]), __uint_as_float(r[8 * h + 1]));

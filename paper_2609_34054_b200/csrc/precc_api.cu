@@ -536,7 +536,7 @@ int32_t precc_lr_precompute(precc_ctx* ctx, const precc_layer_desc* desc, const 
     return fail(ctx, PRECC_ERR_INVALID_ARG, "slots [%lld, %lld) outside the cache", (long long)start_slot, (long long)start_slot + M);
   GemmParams gp{};
   gp.mode = 0; gp.slot_mapping = slot_mapping; gp.start_slot = start_slot; gp.n_blocks = cache->n_blocks;
-  gp.dst0 = (__nv_bfloat16*)cache->lr_k; gp.dst1 = (__nv_bfloat16*)cache->lr_v;
+  gp.lr_k = (__nv_bfloat16*)cache->lr_k; gp.lr_v = (__nv_bfloat16*)cache->lr_v;
   gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = agent_mask;
   gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
   return launch_gemm(ctx, H, M, desc->d_model, A_packed, n_out, gp, (cudaStream_t)stream);
@@ -556,10 +556,33 @@ int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const
     return fail(ctx, PRECC_ERR_INVALID_ARG, "slots [%lld, %lld) outside the cache", (long long)start_slot, (long long)start_slot + M);
   GemmParams gp{};
   gp.mode = 1; gp.slot_mapping = slot_mapping; gp.start_slot = start_slot; gp.n_blocks = cache->n_blocks;
-  gp.dst0 = (__nv_bfloat16*)cache->k_base; gp.dst1 = (__nv_bfloat16*)cache->v_base;
+  gp.base_k = (__nv_bfloat16*)cache->k_base; gp.base_v = (__nv_bfloat16*)cache->v_base;
   gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = ~0ull;
   gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
   return launch_gemm(ctx, H, M, desc->d_model, W_packed, 2 * desc->n_kv_heads * desc->head_dim, gp, (cudaStream_t)stream);
+}
+
+int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
+                           const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_cache* cache,
+                           void* stream) {
+  int32_t rc = check_desc(ctx, desc);
+  if (rc) return rc;
+  if (M < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "M < 0");
+  if (M == 0) return PRECC_OK;
+  const int n_lr = desc->n_agents * (desc->rank_k + desc->rank_v);
+  rc = check_cache(ctx, desc, cache, true, n_lr > 0);
+  if (rc) return rc;
+  if (!H || !WA_packed) return fail(ctx, PRECC_ERR_INVALID_ARG, "H or WA_packed is null");
+  if (!aligned16(H) || !aligned16(WA_packed)) return fail(ctx, PRECC_ERR_MISALIGNED, "H / WA_packed not 16-byte aligned");
+  if (!slot_mapping && (start_slot < 0 || start_slot + M > cache->n_blocks * PRECC_PAGE))
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "slots [%lld, %lld) outside the cache", (long long)start_slot, (long long)start_slot + M);
+  GemmParams gp{};
+  gp.mode = 2; gp.slot_mapping = slot_mapping; gp.start_slot = start_slot; gp.n_blocks = cache->n_blocks;
+  gp.base_k = (__nv_bfloat16*)cache->k_base; gp.base_v = (__nv_bfloat16*)cache->v_base;
+  gp.lr_k = (__nv_bfloat16*)cache->lr_k; gp.lr_v = (__nv_bfloat16*)cache->lr_v;
+  gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = agent_mask;
+  gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
+  return launch_gemm(ctx, H, M, desc->d_model, WA_packed, 2 * desc->n_kv_heads * desc->head_dim + n_lr, gp, (cudaStream_t)stream);
 }
 
 size_t precc_decode_workspace_bytes(const precc_layer_desc* desc, int32_t max_batch, int32_t max_ctx, int32_t sm_count) {
@@ -647,16 +670,17 @@ int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, co
   rc = check_cache(ctx, desc, cache, true, true);
   if (rc) return rc;
   if (!q || !out) return fail(ctx, PRECC_ERR_INVALID_ARG, "q / out is null");
-  if (agent < 0 || agent >= desc->n_agents) return fail(ctx, PRECC_ERR_INVALID_ARG, "agent %d outside [0,%d)", agent, desc->n_agents);
-  if ((desc->rank_k > 0 && !B_k) || (desc->rank_v > 0 && !B_v)) return fail(ctx, PRECC_ERR_INVALID_ARG, "B_k / B_v is null");
+  if (agent < -1 || agent >= desc->n_agents) return fail(ctx, PRECC_ERR_INVALID_ARG, "agent %d outside [-1,%d)", agent, desc->n_agents);
+  const bool neutral = agent < 0;       // adapter-free view: base cache only
+  if (!neutral && ((desc->rank_k > 0 && !B_k) || (desc->rank_v > 0 && !B_v))) return fail(ctx, PRECC_ERR_INVALID_ARG, "B_k / B_v is null");
   if (!aligned16(q) || !aligned16(out) || !aligned16(B_k) || !aligned16(B_v)) return fail(ctx, PRECC_ERR_MISALIGNED, "q / out / B_k / B_v not 16-byte aligned");
   const long long need_blocks = ((long long)ctx_len + S + PRECC_PAGE - 1) / PRECC_PAGE;
   if (block_table && table_stride < need_blocks) return fail(ctx, PRECC_ERR_INVALID_ARG, "block table has %d entries, need %lld", table_stride, need_blocks);
   if (!block_table && (first_block < 0 || first_block + need_blocks > cache->n_blocks))
     return fail(ctx, PRECC_ERR_INVALID_ARG, "blocks [%d, %lld) outside the cache", first_block, first_block + need_blocks);
   if ((long long)S * (desc->n_q_heads / desc->n_kv_heads) > (long long)PF_ROWS * 65535) return fail(ctx, PRECC_ERR_UNSUPPORTED, "S too large");
-  PrefillArgs a{desc, q, S, agent, ctx_len, block_table, first_block, B_k, B_v, cache, out, (cudaStream_t)stream};
-  return dispatch_shape<PrefillRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
+  PrefillArgs a{desc, q, S, neutral ? 0 : agent, ctx_len, block_table, first_block, B_k, B_v, cache, out, (cudaStream_t)stream};
+  return dispatch_shape<PrefillRun>(ctx, desc->head_dim, neutral ? 0 : desc->rank_k, neutral ? 0 : desc->rank_v, a);
 }
 
 }  // extern "C"

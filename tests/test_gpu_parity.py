@@ -262,6 +262,58 @@ def test_prefill_row_matches_decode(px):
         np.testing.assert_allclose(pre[i], dec, atol=1e-2, rtol=2e-2)
 
 
+# ------------------------------------------------------------------ fused projection, adapter-free view
+
+def test_turn_project_equals_the_two_separate_projections_bitwise(px):
+    geo = I.Geometry(256, 8, 2, 128, 3, 16, 16, alpha=32.0)
+    T = 200
+    H = I.hidden_states(T, geo, seed=31)
+    La = Layer(px, geo, seed=31, n_blocks=14, fill=float("nan"))
+    La.append(H, start_slot=16, agent_mask=0b101)
+    Lb = Layer(px, geo, seed=31, n_blocks=14, fill=float("nan"))
+    dev = {k: v.cuda() for k, v in Lb.w.items()}
+    WA = px.pack_turn_weights(geo, dev["W_k"], dev["W_v"], dev["A_k"], dev["A_v"])
+    px.turn_project(Lb.desc, H.cuda(), WA, Lb.cache, 16, None, 0b101)
+    torch.cuda.synchronize()
+    for name in ("k_base", "v_base", "lr_k", "lr_v"):
+        a, b = getattr(La.cache, name).view(torch.int16), getattr(Lb.cache, name).view(torch.int16)
+        assert torch.equal(a, b), name
+
+
+def test_adapter_free_view_in_a_mixed_batch(px):
+    """Double batching: adapted requests and adapter-free requests (agent id -1) in one launch."""
+    geo = I.Geometry(256, 8, 2, 128, 2, 16, 16, alpha=32.0)
+    T = 333
+    H = I.hidden_states(T, geo, seed=33)
+    L = Layer(px, geo, seed=33, n_blocks=(T + 15) // 16)
+    L.append(H)
+    L.cache.lr_k[1].fill_(float("nan"))          # the neutral requests must never touch an LR row
+    q = I.queries(4, geo, seed=33, gain=2.0)
+    agent_id, ctx = [0, -1, 0, -1], [T, T, 100, 17]
+    out = f64(L.decode(q, agent_id, ctx))
+    w = L.w_np
+    args = (f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"])
+    adapted = O.lr_decode_reference(f64(q), [0, 0, 0, 0], ctx, *args, geo.scale_k, geo.scale_v, geo.n_kv)
+    neutral = O.lr_decode_reference(f64(q), [0, 0, 0, 0], ctx, *args, 0.0, 0.0, geo.n_kv)
+    assert_close(out[[0, 2]], adapted[[0, 2]], "adapted requests")
+    assert_close(out[[1, 3]], neutral[[1, 3]], "adapter-free requests")
+    # prefill: agent -1 is plain attention over the base cache
+    qs = I.queries(30, geo, seed=33, tag="turn", gain=2.0)
+    got = f64(L.prefill(qs, -1, T - 30))
+    ref = O.lr_prefill_reference(f64(qs), 0, T - 30, *args, 0.0, 0.0, geo.n_kv)
+    assert_close(got, ref, "adapter-free prefill")
+    # a long, split context too (cluster path for the adapted one, same launch)
+    T2 = 3000
+    H2 = I.hidden_states(T2, geo, seed=34)
+    L2 = Layer(px, geo, seed=34, n_blocks=(T2 + 15) // 16)
+    L2.append(H2)
+    q2 = I.queries(2, geo, seed=34, gain=3.0)
+    out2 = f64(L2.decode(q2, [-1, 1], [T2, T2]))
+    a2 = (f64(H2), L2.w_np["W_k"], L2.w_np["W_v"], L2.w_np["A_k"], L2.w_np["B_k"], L2.w_np["A_v"], L2.w_np["B_v"])
+    assert_close(out2[:1], O.lr_decode_reference(f64(q2[:1]), [0], [T2], *a2, 0.0, 0.0, geo.n_kv), "neutral long")
+    assert_close(out2[1:], O.lr_decode_reference(f64(q2[1:]), [1], [T2], *a2, geo.scale_k, geo.scale_v, geo.n_kv), "adapted long")
+
+
 # ------------------------------------------------------------------ host-side validation
 
 def test_invalid_arguments_are_rejected_without_launch(px):
@@ -305,7 +357,7 @@ def test_device_side_bad_indices_are_flagged_not_fatal(px):
     assert px.poll_status() & 1
     assert (L.cache.k_base[0, :, 3] == 1.0).all()
     q = I.queries(2, geo, seed=2)
-    out = L.decode(q, [0, 9], [16, 16])  # agent 9 does not exist: zeros + flag
+    out = L.decode(q, [0, 9], [16, 16])  # agent 9 does not exist: zeros + flag (-1 would be the adapter-free view)
     assert px.poll_status() & 1
     assert (out[1] == 0).all() and torch.isfinite(out[0]).all()
     assert px.poll_status() == 0
