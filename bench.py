@@ -249,6 +249,7 @@ def extra_turn(px, T: int, S: int, seed: int = 0):
     w = {k: v.cuda() for k, v in I.layer_weights(geo, seed, "C3").items()}
     A_packed = px.pack_adapters(geo, w["A_k"], w["A_v"])
     W_packed = px.pack_base_weights(geo, w["W_k"], w["W_v"])
+    WA_packed = px.pack_turn_weights(geo, w["W_k"], w["W_v"], w["A_k"], w["A_v"])
     cache = Cache(geo, (T + S + 15) // 16)
     H_ctx = [I.hidden_states(T, geo, seed + i, "C3.H_ctx").cuda() for i in range(2)]     # 2 x 268 MB: rotates past L2
     H_new = [I.hidden_states(S, geo, seed + i, "C3.H_new_adpt").cuda() for i in range(32)]
@@ -270,15 +271,22 @@ def extra_turn(px, T: int, S: int, seed: int = 0):
 
     def turn():
         h = H_new[it[0] % 32]; it[0] += 1
-        px.rebase_project(desc, h, W_packed, cache, T)
-        px.lr_precompute(desc, h, A_packed, cache, T)
+        px.turn_project(desc, h, WA_packed, cache, T)
         px.lr_attend_prefill(desc, q, cur, T, w["B_k"], w["B_v"], cache, out)
+
+    def turn_proj():
+        h = H_new[it[0] % 32]; it[0] += 1
+        px.turn_project(desc, h, WA_packed, cache, T)
+
+    def ctx_fused():
+        px.turn_project(desc, H_ctx[it[0] % 2], WA_packed, cache, 0); it[0] += 1
 
     def rebase():
         h = H_neut[it[0] % 32]; it[0] += 1
-        px.rebase_project(desc, h, W_packed, cache, T)
-        px.lr_precompute(desc, h, A_packed, cache, T, None, ~(1 << cur))
+        px.turn_project(desc, h, WA_packed, cache, T, None, ~(1 << cur))
     us_turn = _event_us(torch, turn, 5)
+    us_tproj = _event_us(torch, turn_proj, 10)
+    us_cfused = _event_us(torch, ctx_fused, 6)
     us_attn = _event_us(torch, lambda: px.lr_attend_prefill(desc, q, cur, T, w["B_k"], w["B_v"], cache, out), 5)
     us_reb = _event_us(torch, rebase, 10)
     fl_attn = 4.0 * geo.n_q * S * (geo.hd + (geo.rank_k + geo.rank_v) / 2) * (T + S / 2)
@@ -286,6 +294,8 @@ def extra_turn(px, T: int, S: int, seed: int = 0):
             "lr_precompute_context": {"us": us_pre, "tflops": fl_pre / us_pre / 1e6, "n_out": n_lr,
                                       "GBps": 2.0 * (T * geo.d_model + T * n_lr) / us_pre / 1e3},
             "base_projection_context": {"us": us_base, "tflops": 2.0 * T * geo.d_model * 2 * geo.kv_width / us_base / 1e6},
+            "fused_projection_context": {"us": us_cfused, "tflops": 2.0 * T * geo.d_model * (2 * geo.kv_width + n_lr) / us_cfused / 1e6},
+            "turn_projection_us": us_tproj,
             "turn_us_per_layer": us_turn, "turn_ttft_ms_32_layers": us_turn * C3_LAYERS_FOR_TTFT / 1e3,
             "prefill_attention": {"us": us_attn, "tflops": fl_attn / us_attn / 1e6},
             "rebase_us_per_layer": us_reb, "peaks": measured_tensor_peaks()}
