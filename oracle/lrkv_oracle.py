@@ -17,9 +17,11 @@ What it computes (paper notation, Section 2.1):
   W_eff = W0 + s A_i B_i.  s = 1 is Eq. 1 literally.
 * Attention of the current agent over the shared context (Section 3.1): plain
   softmax attention with the agent's own adapted K and V, scale sigma = 1/sqrt(hd),
-  grouped-query mapping q-head h -> kv-head h // (n_q / n_kv).  No positional
-  rotation is applied (the hot path is position-free; Appendix D.2 notes that a
-  rotated key needs the LR term expanded first, which is outside this path).
+  grouped-query mapping q-head h -> kv-head h // (n_q / n_kv).  The main path is
+  position-free.  The rotary variant (Appendix D.2: a rotated key needs the rank-r
+  term expanded to full width before the rotation) is ``rope_rotate`` /
+  ``lr_decode_reference_rope``: K_a[t] = RoPE_t(H_t (W_k + s A B)), rotate-half
+  pairing (c, c + hd/2), angle t * theta^(-2c/hd); values are never rotated.
 * Decode attends over exactly ``ctx_len`` cached tokens (the caller has already
   appended the current token).  New-turn prefill of S tokens that sit at
   positions T .. T+S-1: query i sees positions 0 .. T+i (context fully visible,
@@ -30,7 +32,10 @@ attention; merged == decomposed; softmax rows sum to one and outputs are convex
 combinations of V rows; ctx_len = 1, q = 0 and identical-rows closed forms;
 permutation invariance; prefill row i == decode at ctx T+i+1; agent isolation;
 pure-Python float brute force on tiny shapes; the LR/base byte ratio against the
-paper's memory table.  No function here is unpinned.
+paper's memory table; for the rotary functions: norm preservation, identity at
+position 0, dependence on relative position only, an explicit 2x2 rotation, the
+linearity that makes expand-then-rotate equal the merged weight, and brute force.
+No function here is unpinned.
 """
 from __future__ import annotations
 
@@ -207,6 +212,46 @@ def attend_from_caches(q_b, k_base, v_base, L_k, L_v, B_k_a, B_v_a, s_k: float, 
         V = reconstruct(as_f64(v_base)[:, cols], L_v, as_f64(B_v_a)[:, cols], s_v)
         for h in range(g * G, (g + 1) * G):
             out[h] = attend_rows(q_b[h], K, V, sg)
+    return out
+
+
+# ------------------------------------------------------------ rotary keys (Appendix D.2)
+
+def rope_tables(max_pos: int, hd: int, theta: float = 10000.0):
+    """cos/sin tables [max_pos, hd/2] of the rotate-half rotary embedding: angle(t, c) = t * theta^(-2c/hd)."""
+    inv = theta ** (-np.arange(hd // 2, dtype=F64) * 2.0 / hd)
+    ang = np.arange(max_pos, dtype=F64)[:, None] * inv[None, :]
+    return np.cos(ang), np.sin(ang)
+
+
+def rope_rotate(x, pos, n_heads: int, cos, sin) -> np.ndarray:
+    """Rotate rows x [t, n_heads*hd] head by head: coordinates (c, c + hd/2) of a head turn by the angle
+    of the row's position (rotate-half convention: x' = x cos + rotate_half(x) sin)."""
+    x = as_f64(x)
+    t, w = x.shape
+    hd = w // n_heads
+    xs = x.reshape(t, n_heads, 2, hd // 2)
+    c = as_f64(cos)[np.asarray(pos)][:, None, :]
+    s_ = as_f64(sin)[np.asarray(pos)][:, None, :]
+    lo, hi = xs[:, :, 0], xs[:, :, 1]
+    out = np.stack([lo * c - hi * s_, hi * c + lo * s_], axis=2)
+    return out.reshape(t, w)
+
+
+def lr_decode_reference_rope(q, agent_id, ctx_len, H, W_k, W_v, A_k, B_k, A_v, B_v, s_k: float, s_v: float,
+                             n_kv: int, cos, sin, sigma=None) -> np.ndarray:
+    """Decode with rotary keys from first principles: the agent's key row of token t is
+    RoPE_t(H_t (W_k + s_k A B)), i.e. the rank-r contribution is expanded to full width BEFORE the
+    rotation (Appendix D.2); values are not rotated; q arrives already rotated.  Token t sits at position t."""
+    q = as_f64(q)
+    Bn, n_q, hd = q.shape
+    out = np.empty(q.shape, dtype=F64)
+    H = as_f64(H)
+    for b in range(Bn):
+        a, t = int(agent_id[b]), int(ctx_len[b])
+        K = rope_rotate(H[:t] @ merged_weight(W_k, A_k[a], B_k[a], s_k), np.arange(t), n_kv, cos, sin)
+        V = H[:t] @ merged_weight(W_v, A_v[a], B_v[a], s_v)
+        out[b] = attend_decode_one(q[b], K, V, t, n_kv, sigma)
     return out
 
 

@@ -357,3 +357,70 @@ def test_c1_adapter_term_is_visible_to_the_tolerance():
     no_lr = O.lr_decode_reference(q, [0, 1, 2], [64] * 3, *args, 0.0, 0.0, geo.n_kv)
     diff = np.abs(with_lr - no_lr)
     assert np.max(diff - (2e-2 + 1e-2 * np.abs(no_lr))) > 0.0, "adapters invisible at the stated tolerance"
+
+
+# -------------------------------------------------------------- rotary keys (Appendix D.2)
+
+def test_rope_is_a_rotation_and_depends_on_relative_position_only():
+    hd, n_heads = 8, 2
+    cos, sin = O.rope_tables(64, hd)
+    x = RNG.standard_normal((5, n_heads * hd)); y = RNG.standard_normal((5, n_heads * hd))
+    pos = np.array([0, 3, 17, 40, 63])
+    rx = O.rope_rotate(x, pos, n_heads, cos, sin)
+    np.testing.assert_allclose(np.linalg.norm(rx.reshape(5, n_heads, hd), axis=2),
+                               np.linalg.norm(x.reshape(5, n_heads, hd), axis=2), rtol=1e-12)
+    np.testing.assert_allclose(rx[0], x[0], rtol=1e-15)                      # position 0: identity
+    # <R_m q, R_n k> depends on m - n only
+    q1, k1 = x[:1], y[:1]
+    a = O.rope_rotate(q1, [10], n_heads, cos, sin) @ O.rope_rotate(k1, [4], n_heads, cos, sin).T
+    b = O.rope_rotate(q1, [36], n_heads, cos, sin) @ O.rope_rotate(k1, [30], n_heads, cos, sin).T
+    np.testing.assert_allclose(a, b, rtol=1e-10)
+    # explicit 2x2 rotation of one coordinate pair, angle = t * theta^(-2c/hd)
+    t, c = 17, 1
+    ang = t * 10000.0 ** (-2.0 * c / hd)
+    lo, hi = x[2, c], x[2, c + hd // 2]
+    np.testing.assert_allclose([rx[2, c], rx[2, c + hd // 2]],
+                               [lo * math.cos(ang) - hi * math.sin(ang), hi * math.cos(ang) + lo * math.sin(ang)], rtol=1e-12)
+
+
+def test_rope_commutes_with_the_low_rank_split_but_not_with_the_fold():
+    p = _tiny(T=9, d=10, n_q=4, n_kv=2, hd=8, N=2, rk=2, rv=2, B=2)
+    cos, sin = O.rope_tables(16, 8)
+    pos = np.arange(9)
+    a = 1
+    merged = O.rope_rotate(O.adapted_projection(p["H"], p["W_k"], p["A_k"][a], p["B_k"][a], 2.0), pos, 2, cos, sin)
+    split = O.rope_rotate(O.base_cache(p["H"], p["W_k"]), pos, 2, cos, sin) + \
+        2.0 * O.rope_rotate(O.lr_cache(p["H"], p["A_k"][a]) @ p["B_k"][a], pos, 2, cos, sin)
+    np.testing.assert_allclose(merged, split, rtol=1e-11, atol=1e-12)        # RoPE is linear: expand, then rotate
+    # rotating the base only and adding the un-rotated rank-r term (what the position-free fold would do) is wrong
+    wrong = O.rope_rotate(O.base_cache(p["H"], p["W_k"]), pos, 2, cos, sin) + 2.0 * O.lr_cache(p["H"], p["A_k"][a]) @ p["B_k"][a]
+    assert np.max(np.abs(wrong[1:] - merged[1:])) > 1e-3
+    np.testing.assert_allclose(wrong[0], merged[0], rtol=1e-12)              # except at position 0
+
+
+def test_rope_decode_reference_brute_force():
+    p = _tiny(T=6, d=8, n_q=4, n_kv=2, hd=4, N=2, rk=2, rv=1, B=2)
+    cos, sin = O.rope_tables(8, 4)
+    p["agent_id"], p["ctx_len"] = np.array([1, 0]), np.array([6, 3])
+    got = O.lr_decode_reference_rope(p["q"], p["agent_id"], p["ctx_len"], p["H"], p["W_k"], p["W_v"], p["A_k"], p["B_k"],
+                                     p["A_v"], p["B_v"], 1.5, 0.5, 2, cos, sin)
+    hd, G = 4, 2
+    for b in range(2):
+        a, T = int(p["agent_id"][b]), int(p["ctx_len"][b])
+        for h in range(4):
+            g = h // G
+            z, V = [], []
+            for t in range(T):
+                k = [sum(p["H"][t, i] * (p["W_k"][i, g * hd + c] + 1.5 * sum(p["A_k"][a, i, j] * p["B_k"][a, j, g * hd + c] for j in range(2)))
+                         for i in range(8)) for c in range(hd)]
+                kr = list(k)
+                for c in range(hd // 2):
+                    ang = t * 10000.0 ** (-2.0 * c / hd)
+                    kr[c] = k[c] * math.cos(ang) - k[c + hd // 2] * math.sin(ang)
+                    kr[c + hd // 2] = k[c + hd // 2] * math.cos(ang) + k[c] * math.sin(ang)
+                z.append(sum(p["q"][b, h, c] * kr[c] for c in range(hd)) / math.sqrt(hd))
+                V.append([sum(p["H"][t, i] * (p["W_v"][i, g * hd + c] + 0.5 * p["A_v"][a, i, 0] * p["B_v"][a, 0, g * hd + c])
+                              for i in range(8)) for c in range(hd)])
+            m = max(z); e = [math.exp(v - m) for v in z]; den = sum(e)
+            for c in range(hd):
+                assert abs(got[b, h, c] - sum(e[t] * V[t][c] for t in range(T)) / den) < 1e-11
