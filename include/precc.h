@@ -13,7 +13,8 @@
  *                    into the output side by associativity)
  *
  * with the usual LoRA scale s = alpha / r:  K_a = K_base + s_k (H A_a^K) B_a^K,  V_a likewise.
- * The path is position-free (no rotary embedding is applied inside the library).
+ * The main path is position-free (no rotary embedding is applied).  The *_rope entry points at the
+ * end of this header are the rotary-key variant of Appendix D.2.
  *
  * Conventions
  *   - All tensors are bf16 in DEVICE memory unless stated; all accumulation is fp32; stores round to
@@ -222,6 +223,51 @@ int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, co
                                 int32_t table_stride, int32_t first_block,
                                 const void* B_k, const void* B_v, const precc_cache* cache,
                                 void* out, void* stream);
+
+/* ---------------------------------------------------------------- rotary keys (Appendix D.2)
+ * With a rotary position embedding the agent's key row of token t is RoPE_t(H_t (W_k + s_k A B)): the
+ * rotation sits between the rank-r term and the query, so the rank-r term must be expanded to full
+ * width and rotated before it meets q.  In this variant
+ *   - the base K cache holds ROTATED rows RoPE_t(H_t W_k) (written by the *_project_rope calls),
+ *   - the LR-K cache holds UNROTATED rows H_t A_a^K (precc_lr_precompute / the LR columns of
+ *     precc_turn_project_rope, unchanged),
+ *   - decode expands L^K B^K_{a,g} page by page on chip, rotates it by the tokens' positions and adds it
+ *     to the rotated base rows; K_a is never written to memory.  V is not rotated.
+ *   - q must already be rotated by the caller (the query projection is outside this library).
+ * Convention: rotate-half pairing, coordinates (c, c + head_dim/2) of a head turn by angle(t, c):
+ *   x'[c] = x[c] cos - x[c + hd/2] sin,   x'[c + hd/2] = x[c + hd/2] cos + x[c] sin.
+ * Prefill over rotary keys has no entry point yet. */
+typedef struct precc_rope {
+  const float* table;        /* device fp32 [max_pos][head_dim/2][2]: (cos, sin) of angle(t, c); 16-byte aligned */
+  int32_t max_pos;           /* rows of `table` */
+  const int32_t* positions;  /* projection calls: device [M] position of each projected row, or NULL for
+                                start_pos + i.  Ignored by decode, where cached token t sits at position t. */
+  int64_t start_pos;
+} precc_rope;
+
+/* precc_rebase_project with the key columns rotated by each row's position before the store.  A
+ * position outside [0, max_pos) raises PRECC_STATUS_BAD_INDEX and that row is not written. */
+int32_t precc_rebase_project_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
+                                  const void* W_packed, const int32_t* slot_mapping, int64_t start_slot,
+                                  const precc_rope* rope, const precc_cache* cache, void* stream);
+
+/* precc_turn_project with rotated base K rows; the LR rows are written unrotated. */
+int32_t precc_turn_project_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
+                                const void* WA_packed, const int32_t* slot_mapping, int64_t start_slot,
+                                uint64_t agent_mask, const precc_rope* rope, const precc_cache* cache,
+                                void* stream);
+
+/* precc_lr_attend_decode over rotated base keys.  Same arguments plus `rope` (max_pos >= max_ctx; a
+ * context longer than max_pos raises PRECC_STATUS_BAD_INDEX and clamps the position).  The workspace
+ * of precc_decode_workspace_bytes suffices.  With rank_k == 0, or for agent id -1, the result equals
+ * precc_lr_attend_decode (the rotated base cache is all there is). */
+int32_t precc_lr_attend_decode_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,
+                                    const int32_t* agent_id, const int32_t* ctx_len,
+                                    const int32_t* block_table, int32_t table_stride,
+                                    const int32_t* first_block, int32_t max_ctx,
+                                    const void* B_k, const void* B_v, const precc_rope* rope,
+                                    const precc_cache* cache, void* out, void* workspace,
+                                    size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -22,6 +22,7 @@ EXPORTS = [
     "precc_poll_status", "precc_pack_kmajor", "precc_lr_precompute", "precc_rebase_project", "precc_turn_project",
     "precc_decode_workspace_bytes", "precc_workspace_init", "precc_lr_attend_decode",
     "precc_lr_attend_decode_static", "precc_lr_attend_prefill",
+    "precc_rebase_project_rope", "precc_turn_project_rope", "precc_lr_attend_decode_rope",
 ]
 
 
@@ -41,6 +42,10 @@ class CacheDesc(C.Structure):
 
 
 _lib = None
+
+
+class RopeDesc(C.Structure):
+    _fields_ = [("table", C.c_void_p), ("max_pos", C.c_int32), ("positions", C.c_void_p), ("start_pos", C.c_int64)]
 
 
 def load_library() -> C.CDLL:
@@ -75,6 +80,11 @@ def load_library() -> C.CDLL:
                                                   C.POINTER(CacheDesc), vp, vp]
     lib.precc_lr_attend_prefill.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp,
                                             C.POINTER(CacheDesc), vp, vp]
+    rp = C.POINTER(RopeDesc)
+    lib.precc_rebase_project_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, rp, C.POINTER(CacheDesc), vp]
+    lib.precc_turn_project_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, u64, rp, C.POINTER(CacheDesc), vp]
+    lib.precc_lr_attend_decode_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, i32, vp, i32, vp, vp, rp,
+                                                C.POINTER(CacheDesc), vp, vp, sz, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is C.c_int:  # default restype: the int32 status code
@@ -100,6 +110,14 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
+
+
+def rope_table(max_pos: int, hd: int, theta: float = 10000.0, device="cuda") -> torch.Tensor:
+    """The rotary table the *_rope calls take: fp32 [max_pos][hd/2][2] = (cos, sin) of t * theta^(-2c/hd)
+    (angles evaluated in fp64, then rounded once)."""
+    inv = torch.pow(torch.tensor(theta, dtype=torch.float64), -torch.arange(hd // 2, dtype=torch.float64) * 2.0 / hd)
+    ang = torch.arange(max_pos, dtype=torch.float64)[:, None] * inv[None, :]
+    return torch.stack([torch.cos(ang), torch.sin(ang)], dim=-1).to(torch.float32).contiguous().to(device)
 
 
 class Cache:
@@ -230,6 +248,40 @@ class Precc:
         self._check(self.lib.precc_rebase_project(self.h, C.byref(desc), _ptr(H), H.shape[0], _ptr(W_packed),
                                                   _ptr(slot_mapping), start_slot, C.byref(cd), _stream()),
                     "precc_rebase_project")
+
+    # ------------------------------------------------------------------ rotary-key variant
+    @staticmethod
+    def _rope(table: torch.Tensor, positions: Optional[torch.Tensor] = None, start_pos: int = 0) -> RopeDesc:
+        if table.dtype != torch.float32 or table.dim() != 3 or table.shape[2] != 2:
+            raise PreccError("rope table must be fp32 [max_pos][hd/2][2]")
+        return RopeDesc(_ptr(table), table.shape[0], _ptr(positions), start_pos)
+
+    def rebase_project_rope(self, desc: LayerDesc, H: torch.Tensor, W_packed: torch.Tensor, cache: Cache, rope: torch.Tensor,
+                            start_slot: int = 0, slot_mapping: Optional[torch.Tensor] = None, start_pos: int = 0,
+                            positions: Optional[torch.Tensor] = None):
+        cd, rd = cache.desc(), self._rope(rope, positions, start_pos)
+        self._check(self.lib.precc_rebase_project_rope(self.h, C.byref(desc), _ptr(H), H.shape[0], _ptr(W_packed),
+                                                       _ptr(slot_mapping), start_slot, C.byref(rd), C.byref(cd), _stream()),
+                    "precc_rebase_project_rope")
+
+    def turn_project_rope(self, desc: LayerDesc, H: torch.Tensor, WA_packed: torch.Tensor, cache: Cache, rope: torch.Tensor,
+                          start_slot: int = 0, slot_mapping: Optional[torch.Tensor] = None, agent_mask: int = (1 << 64) - 1,
+                          start_pos: int = 0, positions: Optional[torch.Tensor] = None):
+        cd, rd = cache.desc(), self._rope(rope, positions, start_pos)
+        self._check(self.lib.precc_turn_project_rope(self.h, C.byref(desc), _ptr(H), H.shape[0], _ptr(WA_packed),
+                                                     _ptr(slot_mapping), start_slot, agent_mask & ((1 << 64) - 1),
+                                                     C.byref(rd), C.byref(cd), _stream()), "precc_turn_project_rope")
+
+    def lr_attend_decode_rope(self, desc: LayerDesc, q: torch.Tensor, agent_id: torch.Tensor, ctx_len: torch.Tensor,
+                              max_ctx: int, B_k, B_v, rope: torch.Tensor, cache: Cache, out: torch.Tensor,
+                              workspace: torch.Tensor, block_table: Optional[torch.Tensor] = None,
+                              first_block: Optional[torch.Tensor] = None):
+        cd, rd = cache.desc(), self._rope(rope)
+        stride = block_table.shape[1] if block_table is not None else 0
+        self._check(self.lib.precc_lr_attend_decode_rope(
+            self.h, C.byref(desc), _ptr(q), q.shape[0], _ptr(agent_id), _ptr(ctx_len), _ptr(block_table), stride,
+            _ptr(first_block), max_ctx, _ptr(B_k), _ptr(B_v), C.byref(rd), C.byref(cd), _ptr(out), _ptr(workspace),
+            workspace.numel(), _stream()), "precc_lr_attend_decode_rope")
 
     def decode_workspace(self, desc: LayerDesc, max_batch: int, max_ctx: int) -> torch.Tensor:
         n = self.lib.precc_decode_workspace_bytes(C.byref(desc), max_batch, max_ctx, self.sm_count)

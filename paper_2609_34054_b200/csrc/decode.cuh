@@ -6,6 +6,13 @@
 // (q~ = s_k q B^K_{a,g}^T, contraction length head_dim + r_k) and the value-side adapter into r extra
 // output coordinates (U = P L^V_a, then out += s_v U B^V_{a,g}).
 //
+// Rotary variant (ROPE = true, Appendix D.2): the base cache holds rotated keys, the LR-K rows are not
+// rotated, and a rotated key cannot take the fold because the rotation sits between L^K and q.  Per
+// page the warp expands E = L^K B^K_{a,g} on the tensor cores (16 x hd), rotates E by the tokens'
+// positions (token t of a request sits at position t; rotate-half pairing (c, c + hd/2)), and adds
+// s_k E to the key fragments before the score MMA; nothing of K_a is written anywhere.  The value side
+// is unchanged.
+//
 // Streaming core (decode_stream_block): a thread block owns consecutive 16-token pages of one (b, g);
 // its warps take pages round-robin, each with a private cp.async ring (no block-wide barrier inside
 // the stream loop).  Tokens sit on the MMA M axis:
@@ -44,6 +51,9 @@ struct DecodeParams {
   int32_t* tickets;   // ticket kernel: [B][n_kv], zero between calls
   uint32_t* status;
   unsigned long long* trace;   // optional [blocks][16] phase timestamps (ns), or null
+  const float4* rope;          // rotary variant: [max_pos][hd/4] of (cos c, sin c, cos c+1, sin c+1), c even
+  int max_pos;                 // rows of `rope`; a context longer than this raises BAD_INDEX
+  int bk_off;                  // rotary variant: byte offset of the B_k slice in dynamic shared memory
   int64_t n_blocks;
   int table_stride;
   int n_q, n_kv, group, n_agents;
@@ -63,6 +73,8 @@ struct DecodeCfg {
   static constexpr int STAGE_BYTES = 2 * KV_BYTES + LK_BYTES + LV_BYTES;
   static constexpr int OW = HD + RV;                 // accumulated output width
   static constexpr int PART_STRIDE = 8 * OW + 16;     // floats: m[8], l[8], O'[8][OW]
+  static constexpr int BK_ROWS = RK > 16 ? RK : 16;   // rotary variant: B_k[a][:, g] slice, rows padded to 16
+  static constexpr int BK_BYTES = BK_ROWS * HD * 2;
   // shared memory of a block with `warps` warps and `stages` ring slots per warp
   __host__ __device__ static constexpr int ring_bytes(int warps, int stages) { return warps * stages * STAGE_BYTES; }
   __host__ __device__ static constexpr int merge_bytes(int warps) { return warps * (OW * 8 + 16) * 4; }
@@ -114,10 +126,11 @@ __device__ __forceinline__ void load_q_frags(const DecodeParams& p, int b, int g
 // (m = running maximum in the log2 domain, l = softmax denominator, O' = unnormalised output with the
 // r_v LR-V coordinates appended).  Ends with a __syncthreads().  A block with no pages yields
 // m = NEG_BIG, l = 0, O' = 0.
-template <int HD, int RK, int RV, int NW>
+template <int HD, int RK, int RV, int NW, bool ROPE>
 __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsigned char* smem, int b, int g, int ctx,
                                                     int agent, bool use_lr, int tile0, int tile_end,
                                                     const uint32_t (&qb)[HD / 16][2], const DecodeTrace& mark) {
+  static_assert(!ROPE || RK > 0, "the rotary variant only differs when there is a key-side adapter");
   using C = DecodeCfg<HD, RK, RV>;
   constexpr int OW = C::OW;
   constexpr int KC = HD / 16;                         // k-chunks of the base part
@@ -192,7 +205,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
 
   // ---- B_k fragments for the query fold are requested first (a few small loads), so that they do
   //      not queue behind the page stream; large ranks would need too many registers and load later
-  constexpr bool PRELOAD_BK = RK > 0 && KX * KC * 4 <= 32;
+  constexpr bool PRELOAD_BK = !ROPE && RK > 0 && KX * KC * 4 <= 32;
   const __nv_bfloat16* Bk = RK > 0 ? p.B_k + ((size_t)agent * RK) * ((size_t)p.n_kv * HD) + (size_t)g * HD : nullptr;
   const size_t bk_rs = (size_t)p.n_kv * HD;     // row stride of B_k
   auto load_bk = [&](int jt, int kc, uint32_t (&a)[4]) {
@@ -217,15 +230,38 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
         for (int kc = 0; kc < KC; ++kc) load_bk(jt, kc, bk_pre[jt * KC + kc]);
     }
   }
+  // ---- rotary variant: the B_k[a][:, g] slice goes to shared memory ([BK_ROWS][HD], swizzled like a
+  //      key page; rows >= RK are zero); requested before the page stream, stored after it is issued
+  constexpr int BK_CHUNKS = ROPE ? C::BK_ROWS * CPR_KV : 0;
+  constexpr int BK_PER_THREAD = ROPE ? (BK_CHUNKS + NT - 1) / NT : 1;
+  uint4 bk_stage[BK_PER_THREAD];
+  if constexpr (ROPE) {
+#pragma unroll
+    for (int k = 0; k < BK_PER_THREAD; ++k) {
+      const int c = threadIdx.x + k * NT;
+      const int j = c / CPR_KV, ch = c % CPR_KV;
+      bk_stage[k] = (c < BK_CHUNKS && j < RK && use_lr) ? __ldg(reinterpret_cast<const uint4*>(Bk + (size_t)j * bk_rs + ch * 8))
+                                                        : make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
   // ---- start the stream: every ring slot is filled at once
   for (int i = 0; i < p.stages; ++i) issue_tile(i);
   mark(2);
+  const uint32_t bk_u32 = smem_u32(smem + p.bk_off);
+  if constexpr (ROPE) {
+#pragma unroll
+    for (int k = 0; k < BK_PER_THREAD; ++k) {
+      const int c = threadIdx.x + k * NT;
+      if (c < BK_CHUNKS) *reinterpret_cast<uint4*>(smem + p.bk_off + swz_off<CPR_KV>(c / CPR_KV, c % CPR_KV)) = bk_stage[k];
+    }
+    __syncthreads();
+  }
 
   // ---- folded key-side adapter q~ = s_k q B_k[a][:, g]^T, computed on the tensor cores as
   //      q~^T[j x q] = B_k[j x c] . q^T[c x q]; the accumulator fragment, transposed with movmatrix,
   //      is exactly the B operand (k = j, n = query) needed by the score MMA.
   uint32_t qxb[KX > 0 ? KX : 1][2];
-  if constexpr (RK > 0) {
+  if constexpr (RK > 0 && !ROPE) {
     __shared__ uint32_t qx_share[KX > 0 ? KX : 1][2][32];
 #pragma unroll
     for (int jt = 0; jt < KX; ++jt) { qxb[jt][0] = 0u; qxb[jt][1] = 0u; }
@@ -267,6 +303,28 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   const int v_row = (lane & 7) + (lane >> 4) * 8;         // V'^T A-operand (transposed load)
   const int v_cpar = (lane >> 3) & 1;
 
+  // ---- rotary variant: (cos, sin) of this lane's tokens (rows lane>>2 and +8 of the page) and columns
+  //      (n-tiles 2kc and 2kc+1 of the lower half), fetched one page ahead
+  constexpr int KH = KC / 2;
+  float4 cs[ROPE ? KH : 1][2][2];                       // [chunk pair][n-tile][row]
+  auto load_cs = [&](int i) {
+    if constexpr (ROPE) {
+      if (i < my_n && use_lr) {
+        const int t = tile0 + warp + NW * i;
+        const int pos0 = min(t * PAGE + (lane >> 2), p.max_pos - 1), pos1 = min(t * PAGE + (lane >> 2) + 8, p.max_pos - 1);
+#pragma unroll
+        for (int kc = 0; kc < KH; ++kc)
+#pragma unroll
+          for (int n2 = 0; n2 < 2; ++n2) {
+            const int c4 = (kc * 16 + n2 * 8 + qk) >> 1;           // float4 index: two columns per entry
+            cs[kc][n2][0] = __ldg(p.rope + (size_t)pos0 * (HD / 4) + c4);
+            cs[kc][n2][1] = __ldg(p.rope + (size_t)pos1 * (HD / 4) + c4);
+          }
+      }
+    }
+  };
+  load_cs(0);
+
   mark(3);
   for (int i = 0; i < my_n; ++i) {
     switch (p.stages) {
@@ -281,13 +339,67 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     const int valid = ctx - t * PAGE;   // >= 1; tokens >= valid are masked
 
     float s[4] = {0.f, 0.f, 0.f, 0.f};
+    if (ROPE && use_lr) {
+      if constexpr (ROPE) {
+        // L^K fragments of the page (A operand of the expansion), all rank chunks
+        uint32_t la[KX][4];
 #pragma unroll
-    for (int kc = 0; kc < KC; ++kc) {
-      uint32_t a[4];
-      ldsm_x4(a, st + swz_off<CPR_KV>(a_row, 2 * kc + a_cpar));
-      mma_bf16_16816(s, a, qb[kc][0], qb[kc][1]);
+        for (int jx = 0; jx < KX; ++jx) {
+          if constexpr (RK >= 16) {
+            ldsm_x4(la[jx], st + 2 * C::KV_BYTES + swz_off<CPR_LK>(a_row, 2 * jx + a_cpar));
+          } else {
+            la[jx][2] = 0u; la[jx][3] = 0u;
+            ldsm_x2(la[jx][0], la[jx][1], st + 2 * C::KV_BYTES + swz_off<1>(a_row, 0));
+          }
+        }
+#pragma unroll
+        for (int kc = 0; kc < KH; ++kc) {
+          // E for columns [16kc, 16kc+16) and their rotation partners [16kc + hd/2, ...)
+          float e[2][2][4];                              // [half][n-tile][c]
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+            for (int n2 = 0; n2 < 2; ++n2) { e[hf][n2][0] = e[hf][n2][1] = e[hf][n2][2] = e[hf][n2][3] = 0.f; }
+#pragma unroll
+            for (int jx = 0; jx < KX; ++jx) {
+              uint32_t bf[4];
+              ldsm_x4_t(bf, bk_u32 + swz_off<CPR_KV>(16 * jx + a_row, 2 * (kc + hf * KH) + a_cpar));
+              mma_bf16_16816(e[hf][0], la[jx], bf[0], bf[1]);
+              mma_bf16_16816(e[hf][1], la[jx], bf[2], bf[3]);
+            }
+          }
+          uint32_t alo[4], ahi[4];
+          ldsm_x4(alo, st + swz_off<CPR_KV>(a_row, 2 * kc + a_cpar));
+          ldsm_x4(ahi, st + swz_off<CPR_KV>(a_row, 2 * (kc + KH) + a_cpar));
+#pragma unroll
+          for (int n2 = 0; n2 < 2; ++n2)
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+              const float4 c4 = cs[kc][n2][r];           // (cos c, sin c, cos c+1, sin c+1)
+              const float lo0 = e[0][n2][2 * r], lo1 = e[0][n2][2 * r + 1];
+              const float hi0 = e[1][n2][2 * r], hi1 = e[1][n2][2 * r + 1];
+              const float rl0 = (lo0 * c4.x - hi0 * c4.y) * p.s_k, rl1 = (lo1 * c4.z - hi1 * c4.w) * p.s_k;
+              const float rh0 = (hi0 * c4.x + lo0 * c4.y) * p.s_k, rh1 = (hi1 * c4.z + lo1 * c4.w) * p.s_k;
+              const int f = n2 * 2 + r;                  // A fragment register: (n-tile, row half)
+              const float2 kl = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&alo[f]));
+              const float2 kh = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ahi[f]));
+              alo[f] = pack_bf16(kl.x + rl0, kl.y + rl1);
+              ahi[f] = pack_bf16(kh.x + rh0, kh.y + rh1);
+            }
+          mma_bf16_16816(s, alo, qb[kc][0], qb[kc][1]);
+          mma_bf16_16816(s, ahi, qb[kc + KH][0], qb[kc + KH][1]);
+        }
+        load_cs(i + 1);
+      }
+    } else {
+#pragma unroll
+      for (int kc = 0; kc < KC; ++kc) {
+        uint32_t a[4];
+        ldsm_x4(a, st + swz_off<CPR_KV>(a_row, 2 * kc + a_cpar));
+        mma_bf16_16816(s, a, qb[kc][0], qb[kc][1]);
+      }
     }
-    if (!use_lr) {
+    if (!use_lr || ROPE) {
     } else if constexpr (RK >= 16) {
 #pragma unroll
       for (int kc = 0; kc < KX; ++kc) {
@@ -405,7 +517,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
 
 // ------------------------------------------------------------------------------------------------
 // Ticket kernel: grid (split, kv head, request), DEC_WARPS warps.
-template <int HD, int RK, int RV>
+template <int HD, int RK, int RV, bool ROPE = false>
 __global__ void __launch_bounds__(DEC_WARPS * 32)
 lr_attend_decode_kernel(const DecodeParams p) {
   using C = DecodeCfg<HD, RK, RV>;
@@ -440,7 +552,8 @@ lr_attend_decode_kernel(const DecodeParams p) {
   const int tile0 = split * p.chunk_tiles;
   const int tile_end = min(n_tiles, tile0 + p.chunk_tiles);
   mark(1);
-  decode_stream_block<HD, RK, RV, DEC_WARPS>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, qb, mark);
+  if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
+  decode_stream_block<HD, RK, RV, DEC_WARPS, ROPE>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, qb, mark);
 
   float* res = reinterpret_cast<float*>(smem);          // [m[8] | l[8] | O'[G][OW]]
   const int n_el = G * OW;
@@ -586,8 +699,8 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
 }
 
-template <int HD, int RK, int RV, int NW>
-__global__ void __launch_bounds__(NW * 32)
+template <int HD, int RK, int RV, int NW, bool ROPE = false>
+__global__ void __launch_bounds__(NW * 32, (NW == 8 && HD == 64) ? 2 : 1)   // 16-block clusters need two blocks per SM
 lr_attend_decode_cluster_kernel(const DecodeParams p) {
   using C = DecodeCfg<HD, RK, RV>;
   constexpr int OW = C::OW;
@@ -631,7 +744,8 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
       bv_pre[k] = (i < RV * cols_) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);
     }
   }
-  decode_stream_block<HD, RK, RV, NW>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, qb, mark);
+  if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
+  decode_stream_block<HD, RK, RV, NW, ROPE>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, qb, mark);
 
   // own result res = [m[8] | l[8] | O'[G][OW]] sits at the start of shared memory in every block
   float* res = reinterpret_cast<float*>(smem);

@@ -37,6 +37,12 @@ struct GemmParams {
   int n_agents, rank_k, rank_v;
   unsigned long long agent_mask;
   int n_kv, hd;
+  // rotary keys (modes 1, 2; null = none): the key columns of a row are rotated by the row's position
+  // before they are stored (rotate-half pairing (c, c + hd/2)); needs BN % hd == 0
+  const float4* rope;             // [max_pos][hd/4] of (cos c, sin c, cos c+1, sin c+1), c even
+  const int32_t* positions;       // [M] or null (start_pos + row)
+  int64_t start_pos;
+  int max_pos;
   uint32_t* status;
 };
 
@@ -213,9 +219,41 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       }
       const long long blk = slot / PAGE;
       const int off = (int)(slot % PAGE);
+      long long pos = 0;
+      if (p.rope && row_ok) {
+        pos = p.positions ? (long long)p.positions[gm] : p.start_pos + gm;
+        if (pos < 0 || pos >= p.max_pos) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
+      }
       mbar_wait(acc_full + 8 * buf, (i >> 1) & 1, p.status);
       asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
       for (int c0 = 0; c0 < p.BN; c0 += 16) {
+        if (p.rope && n0 + c0 < w) {
+          // key columns: chunk [c, c+16) of the lower half of a head together with its partner chunk
+          const int gc = n0 + c0;
+          const int g = gc / p.hd, c = gc % p.hd;
+          if (c >= p.hd / 2) continue;                  // done with its partner
+          uint32_t lo[16], hi[16];
+          tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + buf * p.BN + c0, lo);
+          tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + buf * p.BN + c0 + p.hd / 2, hi);
+          asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+          if (!row_ok) continue;
+          const float4* cs = p.rope + pos * (p.hd / 4) + c / 2;
+          uint32_t ol[8], oh[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float4 t4 = __ldg(cs + k);
+            const float l0 = __uint_as_float(lo[2 * k]), l1 = __uint_as_float(lo[2 * k + 1]);
+            const float h0 = __uint_as_float(hi[2 * k]), h1 = __uint_as_float(hi[2 * k + 1]);
+            ol[k] = pack_bf16(l0 * t4.x - h0 * t4.y, l1 * t4.z - h1 * t4.w);
+            oh[k] = pack_bf16(h0 * t4.x + l0 * t4.y, h1 * t4.z + l1 * t4.w);
+          }
+          __nv_bfloat16* dst = p.base_k + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
+          reinterpret_cast<uint4*>(dst)[0] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+          reinterpret_cast<uint4*>(dst)[1] = make_uint4(ol[4], ol[5], ol[6], ol[7]);
+          reinterpret_cast<uint4*>(dst + p.hd / 2)[0] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+          reinterpret_cast<uint4*>(dst + p.hd / 2)[1] = make_uint4(oh[4], oh[5], oh[6], oh[7]);
+          continue;
+        }
         uint32_t r[16];
         tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + buf * p.BN + c0, r);
         asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");

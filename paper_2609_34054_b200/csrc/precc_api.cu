@@ -147,7 +147,8 @@ int pick_bn(int n_out, int m_tiles, int sm_count) {
 
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
   const int m_tiles = (M + GEMM_BM - 1) / GEMM_BM;
-  const int bn = pick_bn(n_out, m_tiles, ctx->sm_count);
+  int bn = pick_bn(n_out, m_tiles, ctx->sm_count);
+  if (gp.rope && bn % gp.hd != 0) bn = gp.hd;        // a head's two halves must sit in one tile
   const int n_tiles = (n_out + bn - 1) / bn;
   const int stage_bytes = GEMM_A_BYTES + bn * GEMM_BK * 2;
   int stages = (ctx->max_smem_optin - 4096) / stage_bytes;
@@ -190,15 +191,16 @@ int32_t dispatch_shape(precc_ctx* ctx, int hd, int rk, int rv, Args&&... args) {
 // otherwise the ticket kernel with up to max_splits blocks per (request, kv head).
 struct DecodePlan { int cluster, warps, chunk_tiles, max_splits, stages, smem; };
 
+// `extra`: bytes of shared memory appended after the usual layout (the rotary variant's B_k slice).
 template <int HD, int RK, int RV>
-DecodePlan plan_ticket(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
+DecodePlan plan_ticket(int sm_count, int max_smem, int B, int n_kv, int max_ctx, int extra = 0) {
   using C = DecodeCfg<HD, RK, RV>;
   DecodePlan pl{};
   // ring depth: as deep as possible (<= 4) while two blocks still fit on an SM
   int stages = 4;
-  while (stages > 2 && 2 * (C::ticket_smem(stages) + 1024) > max_smem) --stages;
+  while (stages > 2 && 2 * (C::ticket_smem(stages) + extra + 1024) > max_smem) --stages;
   pl.stages = stages;
-  pl.smem = C::ticket_smem(stages);
+  pl.smem = C::ticket_smem(stages) + extra;
   const int per_sm = (2 * (pl.smem + 1024) <= max_smem) ? 2 : 1;
   const long long slots = (long long)sm_count * per_sm;
   const int max_tiles = (max_ctx + PAGE - 1) / PAGE;
@@ -219,7 +221,7 @@ DecodePlan plan_ticket(int sm_count, int max_smem, int B, int n_kv, int max_ctx)
 // The cluster kernel serves the latency-bound regime: few (request, kv head) units, each worth
 // splitting, the whole grid co-resident in one wave.  Returns cluster = 0 when it does not apply.
 template <int HD, int RK, int RV>
-DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
+DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx, int extra = 0) {
   using C = DecodeCfg<HD, RK, RV>;
   DecodePlan pl{};
   const int max_tiles = (max_ctx + PAGE - 1) / PAGE;
@@ -228,7 +230,7 @@ DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx
   if (units * max_tiles > 32768) return pl;              // bandwidth-bound: all SMs matter more than the short tail
   // two blocks per SM must fit (a 16-block cluster needs 16 free slots inside one GPC, and not every
   // GPC has 16 SMs): 8 warps with a 2-deep ring if that fits, else 4 warps with the deepest ring that does
-  const int budget = max_smem / 2 - 1024;
+  const int budget = max_smem / 2 - 1024 - extra;
   int warps = 8, stages = 2;
   if (C::cluster_smem(8, 2) > budget) {
     warps = 4; stages = 4;
@@ -241,7 +243,7 @@ DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx
   pl.cluster = cs;
   pl.warps = warps;
   pl.stages = stages;
-  pl.smem = C::cluster_smem(warps, stages);
+  pl.smem = C::cluster_smem(warps, stages) + extra;
   pl.chunk_tiles = (max_tiles + cs - 1) / cs;
   pl.max_splits = cs;
   return pl;
@@ -251,12 +253,14 @@ struct DecodeArgs {
   const precc_layer_desc* d; const void* q; int B; const int32_t* agent_id; const int32_t* ctx_len;
   const int32_t* block_table; int table_stride; const int32_t* first_block; int max_ctx;
   const void* B_k; const void* B_v; const precc_cache* cache; void* out; void* ws; size_t ws_bytes; cudaStream_t stream;
+  const float* rope = nullptr; int max_pos = 0;      // rotary variant when rope != null
 };
 
-template <int HD, int RK, int RV>
-struct DecodeRun {
+template <int HD, int RK, int RV, bool ROPE = false>
+struct DecodeRunT {
+  // (the rotary variant never needs more than the plain one: its larger blocks only lower the split count)
   static size_t ws_bytes(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
-    const DecodePlan pl = plan_ticket<HD, RK, RV>(sm_count, max_smem, B, n_kv, max_ctx);
+    const DecodePlan pl = plan_ticket<HD, RK, RV>(sm_count, max_smem, B, n_kv, max_ctx, ROPE ? DecodeCfg<HD, RK, RV>::BK_BYTES + 128 : 0);
     const size_t tickets = ((size_t)B * n_kv * 4 + 255) / 256 * 256;
     return tickets + (size_t)B * n_kv * pl.max_splits * DecodeCfg<HD, RK, RV>::PART_STRIDE * 4;
   }
@@ -265,7 +269,7 @@ struct DecodeRun {
   static bool cluster_fits(precc_ctx* ctx, const DecodePlan& pl, int need) {
     static int cached[DEC_MAX_CLUSTER + 1] = {0};      // 0 = unknown, else max active clusters + 1
     if (cached[pl.cluster] == 0) {
-      auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW>;
+      auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
       int n = 0;
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess ||
           cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
@@ -288,10 +292,11 @@ struct DecodeRun {
   }
   static int32_t run(precc_ctx* ctx, const DecodeArgs& a) {
     const precc_layer_desc* d = a.d;
-    DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
+    constexpr int extra = ROPE ? DecodeCfg<HD, RK, RV>::BK_BYTES + 128 : 0;
+    DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);
     if (pl.cluster && !(pl.warps == 8 ? cluster_fits<8>(ctx, pl, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, pl, a.B * d->n_kv_heads))) pl.cluster = 0;
     if (!pl.cluster) {
-      pl = plan_ticket<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
+      pl = plan_ticket<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);
       const size_t need = ws_bytes(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
       if (!a.ws || a.ws_bytes < need) return fail(ctx, PRECC_ERR_WORKSPACE, "decode workspace: need %zu bytes, got %zu", need, a.ws_bytes);
     }
@@ -310,6 +315,8 @@ struct DecodeRun {
     p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = d->n_q_heads / d->n_kv_heads; p.n_agents = d->n_agents;
     p.chunk_tiles = pl.chunk_tiles; p.max_splits = pl.max_splits; p.stages = pl.stages;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
+    p.rope = reinterpret_cast<const float4*>(a.rope); p.max_pos = a.max_pos;
+    p.bk_off = ROPE ? ((pl.smem - extra + 127) / 128) * 128 : 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(pl.max_splits, d->n_kv_heads, a.B);
     cfg.dynamicSmemBytes = pl.smem;
@@ -324,15 +331,27 @@ struct DecodeRun {
       attr[1].id = cudaLaunchAttributeClusterDimension;
       attr[1].val.clusterDim.x = pl.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
       cfg.numAttrs = 2;
-      if (pl.warps == 8) PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 8>, p));
-      else PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 4>, p));
+      if (pl.warps == 8) PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 8, ROPE>, p));
+      else PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 4, ROPE>, p));
     } else {
-      auto kern = lr_attend_decode_kernel<HD, RK, RV>;
+      auto kern = lr_attend_decode_kernel<HD, RK, RV, ROPE>;
       cfg.blockDim = dim3(DEC_WARPS * 32);
       PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem));
       PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, p));
     }
     return PRECC_OK;
+  }
+};
+
+template <int HD, int RK, int RV>
+struct DecodeRun : DecodeRunT<HD, RK, RV, false> {};
+// Rotary keys: without a key-side adapter (or for the adapter-free view) the rotated base cache is all
+// there is, and the position-free kernel is already exact.
+template <int HD, int RK, int RV>
+struct DecodeRunRope {
+  static int32_t run(precc_ctx* ctx, const DecodeArgs& a) {
+    if constexpr (RK > 0) return DecodeRunT<HD, RK, RV, true>::run(ctx, a);
+    else return DecodeRunT<HD, RK, RV, false>::run(ctx, a);
   }
 };
 
@@ -542,8 +561,22 @@ int32_t precc_lr_precompute(precc_ctx* ctx, const precc_layer_desc* desc, const 
   return launch_gemm(ctx, H, M, desc->d_model, A_packed, n_out, gp, (cudaStream_t)stream);
 }
 
-int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* W_packed,
-                             const int32_t* slot_mapping, int64_t start_slot, const precc_cache* cache, void* stream) {
+static int32_t set_rope(precc_ctx* ctx, const precc_layer_desc* desc, const precc_rope* rope, GemmParams* gp) {
+  if (!rope) return PRECC_OK;
+  if (!rope->table || rope->max_pos < 1) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table is null or empty");
+  if (!aligned16(rope->table)) return fail(ctx, PRECC_ERR_MISALIGNED, "rope table not 16-byte aligned");
+  if (!rope->positions && (rope->start_pos < 0 || rope->start_pos + gp->M > rope->max_pos))
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "positions [%lld, %lld) outside the rope table", (long long)rope->start_pos,
+                (long long)rope->start_pos + gp->M);
+  (void)desc;
+  gp->rope = reinterpret_cast<const float4*>(rope->table); gp->positions = rope->positions;
+  gp->start_pos = rope->start_pos; gp->max_pos = rope->max_pos;
+  return PRECC_OK;
+}
+
+static int32_t rebase_entry(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* W_packed,
+                            const int32_t* slot_mapping, int64_t start_slot, const precc_rope* rope, const precc_cache* cache,
+                            void* stream) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (M < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "M < 0");
@@ -559,12 +592,28 @@ int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const
   gp.base_k = (__nv_bfloat16*)cache->k_base; gp.base_v = (__nv_bfloat16*)cache->v_base;
   gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = ~0ull;
   gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
+  gp.M = M;
+  rc = set_rope(ctx, desc, rope, &gp);
+  if (rc) return rc;
   return launch_gemm(ctx, H, M, desc->d_model, W_packed, 2 * desc->n_kv_heads * desc->head_dim, gp, (cudaStream_t)stream);
 }
 
-int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
-                           const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_cache* cache,
-                           void* stream) {
+int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* W_packed,
+                             const int32_t* slot_mapping, int64_t start_slot, const precc_cache* cache, void* stream) {
+  return rebase_entry(ctx, desc, H, M, W_packed, slot_mapping, start_slot, nullptr, cache, stream);
+}
+
+int32_t precc_rebase_project_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* W_packed,
+                                  const int32_t* slot_mapping, int64_t start_slot, const precc_rope* rope,
+                                  const precc_cache* cache, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!rope) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope is null");
+  return rebase_entry(ctx, desc, H, M, W_packed, slot_mapping, start_slot, rope, cache, stream);
+}
+
+static int32_t turn_entry(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
+                          const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_rope* rope,
+                          const precc_cache* cache, void* stream) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (M < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "M < 0");
@@ -582,7 +631,24 @@ int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const v
   gp.lr_k = (__nv_bfloat16*)cache->lr_k; gp.lr_v = (__nv_bfloat16*)cache->lr_v;
   gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = agent_mask;
   gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
+  gp.M = M;
+  rc = set_rope(ctx, desc, rope, &gp);
+  if (rc) return rc;
   return launch_gemm(ctx, H, M, desc->d_model, WA_packed, 2 * desc->n_kv_heads * desc->head_dim + n_lr, gp, (cudaStream_t)stream);
+}
+
+int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
+                           const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_cache* cache,
+                           void* stream) {
+  return turn_entry(ctx, desc, H, M, WA_packed, slot_mapping, start_slot, agent_mask, nullptr, cache, stream);
+}
+
+int32_t precc_turn_project_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
+                                const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_rope* rope,
+                                const precc_cache* cache, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!rope) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope is null");
+  return turn_entry(ctx, desc, H, M, WA_packed, slot_mapping, start_slot, agent_mask, rope, cache, stream);
 }
 
 size_t precc_decode_workspace_bytes(const precc_layer_desc* desc, int32_t max_batch, int32_t max_ctx, int32_t sm_count) {
@@ -602,10 +668,11 @@ int32_t precc_workspace_init(precc_ctx* ctx, void* workspace, size_t workspace_b
   return PRECC_OK;
 }
 
-int32_t precc_lr_attend_decode(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B, const int32_t* agent_id,
-                               const int32_t* ctx_len, const int32_t* block_table, int32_t table_stride,
-                               const int32_t* first_block, int32_t max_ctx, const void* B_k, const void* B_v,
-                               const precc_cache* cache, void* out, void* workspace, size_t workspace_bytes, void* stream) {
+static int32_t decode_entry(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B, const int32_t* agent_id,
+                            const int32_t* ctx_len, const int32_t* block_table, int32_t table_stride,
+                            const int32_t* first_block, int32_t max_ctx, const void* B_k, const void* B_v,
+                            const precc_cache* cache, void* out, void* workspace, size_t workspace_bytes, void* stream,
+                            const float* rope, int32_t max_pos) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (B < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "B < 0");
@@ -626,7 +693,30 @@ int32_t precc_lr_attend_decode(precc_ctx* ctx, const precc_layer_desc* desc, con
   }
   DecodeArgs a{desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, B_v, cache, out,
                workspace, workspace_bytes, (cudaStream_t)stream};
-  return dispatch_shape<DecodeRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
+  if (!rope) return dispatch_shape<DecodeRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
+  if (!aligned16(rope)) return fail(ctx, PRECC_ERR_MISALIGNED, "rope table not 16-byte aligned");
+  if (max_pos < max_ctx) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table covers %d positions, max_ctx is %d", max_pos, max_ctx);
+  a.rope = rope; a.max_pos = max_pos;
+  return dispatch_shape<DecodeRunRope>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
+}
+
+int32_t precc_lr_attend_decode(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B, const int32_t* agent_id,
+                               const int32_t* ctx_len, const int32_t* block_table, int32_t table_stride,
+                               const int32_t* first_block, int32_t max_ctx, const void* B_k, const void* B_v,
+                               const precc_cache* cache, void* out, void* workspace, size_t workspace_bytes, void* stream) {
+  return decode_entry(ctx, desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, B_v, cache, out,
+                      workspace, workspace_bytes, stream, nullptr, 0);
+}
+
+int32_t precc_lr_attend_decode_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,
+                                    const int32_t* agent_id, const int32_t* ctx_len, const int32_t* block_table,
+                                    int32_t table_stride, const int32_t* first_block, int32_t max_ctx, const void* B_k,
+                                    const void* B_v, const precc_rope* rope, const precc_cache* cache, void* out,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!rope || !rope->table) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table is null");
+  return decode_entry(ctx, desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, B_v, cache, out,
+                      workspace, workspace_bytes, stream, rope->table, rope->max_pos);
 }
 
 int32_t precc_lr_attend_decode_static(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,

@@ -1,0 +1,177 @@
+"""Parity of the rotary-key variant (Appendix D.2): rotated base keys written by the projection kernels,
+un-rotated LR-K rows, and decode that expands, rotates and adds the rank-r key term page by page.
+Expected values come from the merged-weight definition K_a[t] = RoPE_t(H_t (W_k + s A B))."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lrkv_oracle as O
+from paper_2609_34054_b200 import inputs as I
+from paper_2609_34054_b200.binding import PreccError, rope_table
+
+from harness import Layer, assert_close, base_rows, f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def px():
+    from paper_2609_34054_b200.binding import Precc
+    p = Precc(0)
+    yield p
+    assert p.poll_status() == 0
+    p.close()
+
+
+def _decode_rope(L, q, agent_id, ctx_len, table, max_ctx=None, block_table=None):
+    qd = q.cuda()
+    aid = torch.as_tensor(agent_id, dtype=torch.int32).cuda()
+    cl = torch.as_tensor(ctx_len, dtype=torch.int32).cuda()
+    max_ctx = int(max(ctx_len)) if max_ctx is None else max_ctx
+    ws = L.px.decode_workspace(L.desc, qd.shape[0], max_ctx)
+    out = torch.full_like(qd, float("nan"))
+    bt = None if block_table is None else block_table.cuda()
+    L.px.lr_attend_decode_rope(L.desc, qd, aid, cl, max_ctx, L.B_k, L.B_v, table, L.cache, out, ws, bt)
+    torch.cuda.synchronize()
+    return out
+
+
+def test_rope_table_matches_the_definition():
+    """The library-side table generator against the oracle's (independent code, same definition)."""
+    t = rope_table(300, 64, device="cpu").double().numpy()
+    cos, sin = O.rope_tables(300, 64)
+    np.testing.assert_allclose(t[..., 0], cos, atol=1e-7)
+    np.testing.assert_allclose(t[..., 1], sin, atol=1e-7)
+
+
+@pytest.mark.parametrize("hd,n_kv,M", [(64, 2, 300), (128, 1, 130), (128, 4, 517)])
+def test_projection_rotates_keys_only(px, hd, n_kv, M):
+    geo = I.Geometry(d_model=256, n_q=2 * n_kv, n_kv=n_kv, hd=hd, n_agents=2, rank_k=16, rank_v=16, alpha=32.0)
+    nb = (M + 15) // 16 + 2
+    L = Layer(px, geo, seed=3, n_blocks=nb, tag="rp", fill=0.0)
+    H = I.hidden_states(M, geo, 3, "rp.H")
+    table = rope_table(1024, hd)
+    cos, sin = O.rope_tables(1024, hd)
+    # plain projection first (keeps V for the bitwise check), then the rotary one with explicit positions
+    px.rebase_project(L.desc, H.cuda(), L.W_packed, L.cache, 0)
+    torch.cuda.synchronize()
+    v_plain = L.cache.v_base.clone()
+    pos = I.uniform_int(0, 1023, M, 3, "rp.pos").to(torch.int32)
+    px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0, positions=pos.cuda())
+    torch.cuda.synchronize()
+    assert torch.equal(L.cache.v_base, v_plain)
+    got = base_rows(L.cache.k_base)[:M]
+    ref = O.rope_rotate(O.base_cache(f64(H), L.w_np["W_k"]), pos.numpy(), n_kv, cos, sin)
+    err = np.abs(got - ref)
+    assert (err <= 2.0 ** -8 * np.abs(ref) + 2e-3).all(), f"max err {err.max()}"
+    # consecutive positions from start_pos, through the fused projection: bitwise equal to the two-call form
+    px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0, start_pos=7)
+    px.lr_precompute(L.desc, H.cuda(), L.A_packed, L.cache, 0)
+    torch.cuda.synchronize()
+    k2, lk2 = L.cache.k_base.clone(), L.cache.lr_k.clone()
+    ref2 = O.rope_rotate(O.base_cache(f64(H), L.w_np["W_k"]), np.arange(M) + 7, n_kv, cos, sin)
+    assert (np.abs(base_rows(k2)[:M] - ref2) <= 2.0 ** -8 * np.abs(ref2) + 2e-3).all()
+    WA = px.pack_turn_weights(geo, L.w["W_k"].cuda(), L.w["W_v"].cuda(), L.w["A_k"].cuda(), L.w["A_v"].cuda())
+    L.cache.k_base.zero_(); L.cache.lr_k.zero_()
+    px.turn_project_rope(L.desc, H.cuda(), WA, L.cache, table, 0, start_pos=7)
+    torch.cuda.synchronize()
+    assert torch.equal(L.cache.k_base, k2) and torch.equal(L.cache.lr_k, lk2)
+
+
+SHAPES = [
+    # hd, n_q, n_kv, rank, T, agents
+    (64, 8, 2, 16, 70, 2),
+    (64, 16, 2, 8, 333, 3),
+    (64, 4, 4, 32, 129, 2),
+    (64, 8, 1, 64, 100, 2),
+    (128, 8, 2, 8, 97, 3),
+    (128, 8, 2, 16, 260, 2),
+    (128, 4, 1, 32, 65, 2),
+    (128, 8, 8, 64, 48, 2),
+]
+
+
+@pytest.mark.parametrize("hd,n_q,n_kv,r,T,N", SHAPES)
+def test_decode_rope_small_shapes(px, hd, n_q, n_kv, r, T, N):
+    geo = I.Geometry(d_model=192, n_q=n_q, n_kv=n_kv, hd=hd, n_agents=N, rank_k=r, rank_v=r, alpha=2.0 * r)
+    L = Layer(px, geo, seed=5, n_blocks=(T + 15) // 16, tag="rd")
+    H = I.hidden_states(T, geo, 5, "rd.H")
+    table = rope_table(T + 5, hd)
+    cos, sin = O.rope_tables(T + 5, hd)
+    px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0)
+    px.lr_precompute(L.desc, H.cuda(), L.A_packed, L.cache, 0)
+    agents = [i % N for i in range(4)]
+    ctx = [T, max(1, T // 2), 17, 1]
+    w = L.w_np
+    for gain in (1.0, 4.0):
+        q = I.queries(4, geo, 5, f"rd.q{gain}", gain=gain)
+        out = f64(_decode_rope(L, q, agents, ctx, table))
+        ref = O.lr_decode_reference_rope(f64(q), agents, ctx, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                         geo.scale_k, geo.scale_v, n_kv, cos, sin)
+        assert_close(out, ref, f"rope decode hd{hd} r{r} gain {gain}")
+
+
+def test_decode_rope_differs_from_the_position_free_fold(px):
+    """Guards against a vacuous test: on rotated base keys the position-free kernel (which folds the
+    un-rotated rank-r term into the query) must NOT match the rotary definition."""
+    geo = I.Geometry(d_model=192, n_q=8, n_kv=2, hd=64, n_agents=2, rank_k=16, rank_v=16, alpha=64.0)
+    T = 200
+    L = Layer(px, geo, seed=6, n_blocks=(T + 15) // 16, tag="rf")
+    H = I.hidden_states(T, geo, 6, "rf.H")
+    table = rope_table(T, 64)
+    cos, sin = O.rope_tables(T, 64)
+    px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0)
+    px.lr_precompute(L.desc, H.cuda(), L.A_packed, L.cache, 0)
+    q = I.queries(2, geo, 6, "rf.q", gain=4.0)
+    w = L.w_np
+    ref = O.lr_decode_reference_rope(f64(q), [0, 1], [T, T], f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                     geo.scale_k, geo.scale_v, 2, cos, sin)
+    assert_close(f64(_decode_rope(L, q, [0, 1], [T, T], table)), ref, "rotary decode")
+    plain = f64(L.decode(q, [0, 1], [T, T]))
+    assert np.max(np.abs(plain - ref)) > 5e-2
+    # adapter-free view (agent -1) and position-free kernel agree bit for bit on the rotated base cache
+    a = _decode_rope(L, q, [-1, -1], [T, T], table)
+    b = L.decode(q, [-1, -1], [T, T])
+    assert torch.equal(a, b)
+
+
+def test_decode_rope_long_context_split_and_paged(px):
+    """Benchmark-layer shape, 8192 tokens: batch 1 takes the cluster path, batch 24 over shuffled pages the
+    ticket path with several splits; both against the definition."""
+    geo, T = I.C2, 8192
+    L = Layer(px, geo, seed=0, n_blocks=T // 16, tag="L0")
+    H = I.hidden_states(T, geo, 0, "L0.H")
+    table = rope_table(T, geo.hd)
+    cos, sin = O.rope_tables(T, geo.hd)
+    perm = I.permutation(T // 16, 0, "rope.perm").to(torch.int32)          # logical block -> physical block
+    slots = (perm.long()[:, None] * 16 + torch.arange(16)[None, :]).reshape(-1).to(torch.int32)
+    WA = px.pack_turn_weights(geo, L.w["W_k"].cuda(), L.w["W_v"].cuda(), L.w["A_k"].cuda(), L.w["A_v"].cuda())
+    px.turn_project_rope(L.desc, H.cuda(), WA, L.cache, table, 0, slot_mapping=slots.cuda())
+    w, Hn = L.w_np, f64(H)
+    q = I.queries(1, geo, 0, "rope.q1", gain=4.0)
+    out = f64(_decode_rope(L, q, [2], [T], table, block_table=perm[None, :]))
+    ref = O.lr_decode_reference_rope(f64(q), [2], [T], Hn, w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                     geo.scale_k, geo.scale_v, geo.n_kv, cos, sin)
+    assert_close(out, ref, "rope C2 batch 1")
+    Bn = 24
+    agents = [i % geo.n_agents for i in range(Bn)]
+    ctx = [int(x) for x in I.uniform_int(1500, T, Bn, 0, "rope.ctx")]
+    q = I.queries(Bn, geo, 0, "rope.q24", gain=4.0)
+    out = f64(_decode_rope(L, q, agents, ctx, table, block_table=perm[None, :].repeat(Bn, 1)))
+    sel = [0, 7, 23]
+    ref = O.lr_decode_reference_rope(f64(q)[sel], [agents[i] for i in sel], [ctx[i] for i in sel], Hn, w["W_k"], w["W_v"],
+                                     w["A_k"], w["B_k"], w["A_v"], w["B_v"], geo.scale_k, geo.scale_v, geo.n_kv, cos, sin)
+    assert_close(out[sel], ref, "rope C2 batch 24")
+
+
+def test_rope_invalid_arguments(px):
+    geo = I.Geometry(d_model=192, n_q=8, n_kv=2, hd=64, n_agents=2, rank_k=16, rank_v=16, alpha=32.0)
+    L = Layer(px, geo, seed=7, n_blocks=8, tag="ri", fill=0.0)
+    H = I.hidden_states(100, geo, 7, "ri.H")
+    table = rope_table(64, 64)
+    with pytest.raises(PreccError):                      # positions 0..99 do not fit a 64-row table
+        px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0)
+    q = I.queries(1, geo, 7, "ri.q")
+    with pytest.raises(PreccError):                      # max_ctx beyond the table
+        _decode_rope(L, q, [0], [100], table)
+    assert px.poll_status() == 0
