@@ -244,6 +244,11 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
                                                         : make_uint4(0u, 0u, 0u, 0u);
     }
   }
+  // the LoRA scale is folded into the slice (one bf16 rounding of s_k B; exact for power-of-two scales)
+  auto scale2 = [&](uint32_t v) -> uint32_t {
+    const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v));
+    return pack_bf16(f.x * p.s_k, f.y * p.s_k);
+  };
   // ---- start the stream: every ring slot is filled at once
   for (int i = 0; i < p.stages; ++i) issue_tile(i);
   mark(2);
@@ -252,7 +257,9 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
 #pragma unroll
     for (int k = 0; k < BK_PER_THREAD; ++k) {
       const int c = threadIdx.x + k * NT;
-      if (c < BK_CHUNKS) *reinterpret_cast<uint4*>(smem + p.bk_off + swz_off<CPR_KV>(c / CPR_KV, c % CPR_KV)) = bk_stage[k];
+      if (c < BK_CHUNKS)
+        *reinterpret_cast<uint4*>(smem + p.bk_off + swz_off<CPR_KV>(c / CPR_KV, c % CPR_KV)) =
+            make_uint4(scale2(bk_stage[k].x), scale2(bk_stage[k].y), scale2(bk_stage[k].z), scale2(bk_stage[k].w));
     }
     __syncthreads();
   }
@@ -306,9 +313,10 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   // ---- rotary variant: (cos, sin) of this lane's tokens (rows lane>>2 and +8 of the page) and columns
   //      (n-tiles 2kc and 2kc+1 of the lower half), fetched one page ahead
   constexpr int KH = KC / 2;
-  float4 cs[ROPE ? KH : 1][2][2];                       // [chunk pair][n-tile][row]
+  constexpr bool CS_AHEAD = true;                      // wider heads: the table entries are loaded at their use
+  float4 cs[ROPE && CS_AHEAD ? KH : 1][2][2];           // [chunk pair][n-tile][row]
   auto load_cs = [&](int i) {
-    if constexpr (ROPE) {
+    if constexpr (ROPE && CS_AHEAD) {
       if (i < my_n && use_lr) {
         const int t = tile0 + warp + NW * i;
         const int pos0 = min(t * PAGE + (lane >> 2), p.max_pos - 1), pos1 = min(t * PAGE + (lane >> 2) + 8, p.max_pos - 1);
@@ -371,20 +379,31 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
           uint32_t alo[4], ahi[4];
           ldsm_x4(alo, st + swz_off<CPR_KV>(a_row, 2 * kc + a_cpar));
           ldsm_x4(ahi, st + swz_off<CPR_KV>(a_row, 2 * (kc + KH) + a_cpar));
+          float4 csl[2][2];
+          if constexpr (!CS_AHEAD) {
+            const int pos0 = min(t * PAGE + (lane >> 2), p.max_pos - 1), pos1 = min(t * PAGE + (lane >> 2) + 8, p.max_pos - 1);
+#pragma unroll
+            for (int n2 = 0; n2 < 2; ++n2) {
+              const int c4i = (kc * 16 + n2 * 8 + qk) >> 1;
+              csl[n2][0] = __ldg(p.rope + (size_t)pos0 * (HD / 4) + c4i);
+              csl[n2][1] = __ldg(p.rope + (size_t)pos1 * (HD / 4) + c4i);
+            }
+          }
 #pragma unroll
           for (int n2 = 0; n2 < 2; ++n2)
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
-              const float4 c4 = cs[kc][n2][r];           // (cos c, sin c, cos c+1, sin c+1)
+              const float4 c4 = CS_AHEAD ? cs[CS_AHEAD ? kc : 0][n2][r] : csl[n2][r];   // (cos c, sin c, cos c+1, sin c+1)
               const float lo0 = e[0][n2][2 * r], lo1 = e[0][n2][2 * r + 1];
               const float hi0 = e[1][n2][2 * r], hi1 = e[1][n2][2 * r + 1];
-              const float rl0 = (lo0 * c4.x - hi0 * c4.y) * p.s_k, rl1 = (lo1 * c4.z - hi1 * c4.w) * p.s_k;
-              const float rh0 = (hi0 * c4.x + lo0 * c4.y) * p.s_k, rh1 = (hi1 * c4.z + lo1 * c4.w) * p.s_k;
+              const uint32_t rl = pack_bf16(lo0 * c4.x - hi0 * c4.y, lo1 * c4.z - hi1 * c4.w);
+              const uint32_t rh = pack_bf16(hi0 * c4.x + lo0 * c4.y, hi1 * c4.z + lo1 * c4.w);
               const int f = n2 * 2 + r;                  // A fragment register: (n-tile, row half)
-              const float2 kl = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&alo[f]));
-              const float2 kh = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ahi[f]));
-              alo[f] = pack_bf16(kl.x + rl0, kl.y + rl1);
-              ahi[f] = pack_bf16(kh.x + rh0, kh.y + rh1);
+              // packed bf16 add: the rotated rank-r term is rounded to bf16 once before it joins the key
+              *reinterpret_cast<__nv_bfloat162*>(&alo[f]) = __hadd2(*reinterpret_cast<const __nv_bfloat162*>(&alo[f]),
+                                                                   *reinterpret_cast<const __nv_bfloat162*>(&rl));
+              *reinterpret_cast<__nv_bfloat162*>(&ahi[f]) = __hadd2(*reinterpret_cast<const __nv_bfloat162*>(&ahi[f]),
+                                                                   *reinterpret_cast<const __nv_bfloat162*>(&rh));
             }
           mma_bf16_16816(s, alo, qb[kc][0], qb[kc][1]);
           mma_bf16_16816(s, ahi, qb[kc + KH][0], qb[kc + KH][1]);
