@@ -113,17 +113,20 @@ int32_t precc_set_trace_buffer(precc_ctx* ctx, void* buffer, size_t n_blocks);
  * word is zero, PRECC_ERR_DEVICE_STATUS otherwise. */
 int32_t precc_poll_status(precc_ctx* ctx, void* stream, uint32_t* status_out);
 
-/* Transpose-pack a row-major [d_model][n_cols] matrix (paper layout d_in x d_out) into rows
- * [dst_row0, dst_row0 + n_cols) of a [dst_rows][d_model] matrix, i.e. dst[dst_row0 + c][i] = src[i][c].
- * Used to build the packed A (all agents' down-projections side by side, Section 3.1) and the
- * packed W.  src, dst device; d_model % 8 == 0. */
+/* Pack a row-major [d_model][n_cols] matrix (paper layout d_in x d_out) as rows [dst_row0, dst_row0 +
+ * n_cols) of a packed matrix of dst_rows rows, the operand format of the projection kernels: k-blocked
+ * K-major, element (row, i) at ((i / 64) * dst_rows + row) * 64 + i % 64, holding src[i][row - dst_row0]
+ * (the 64-deep k step of any run of rows is contiguous, one TMA box).  dst has dst_rows * d_model
+ * elements and must be packed with the dst_rows it is later used with.  Used to build the packed A (all
+ * agents' down-projections side by side, Section 3.1), the packed W and the two together.  src, dst
+ * device; d_model % 64 == 0. */
 int32_t precc_pack_kmajor(precc_ctx* ctx, const void* src, int32_t d_model, int32_t n_cols,
                           void* dst, int32_t dst_rows, int32_t dst_row0, void* stream);
 
 /* LR-cache precompute (Section 3.1, PreLRShared): L_k^p = H A_k^p for every agent k whose bit is set
  * in agent_mask and both projections p, written to the LR caches at the tokens' slots.
  *   H            [M][d_model]
- *   A_packed     [n_agents*(rank_k+rank_v)][d_model]  (precc_pack_kmajor output)
+ *   A_packed     n_agents*(rank_k+rank_v) packed rows (precc_pack_kmajor output): agent-major K rows, then V rows
  *   slot_mapping [M] physical token slots, or NULL for slots start_slot .. start_slot+M-1
  *   agent_mask   bit k = write agent k (all agents: PreLRShared; all but the current one: the
  *                adapter-free pass of ReBaseShared; only the current one: its adapted pass)
@@ -134,7 +137,8 @@ int32_t precc_lr_precompute(precc_ctx* ctx, const precc_layer_desc* desc, const 
 
 /* Base-cache (re-)projection (Section 3.2, ReBaseShared; also the in-turn append): K_base[slot] = H W_k,
  * V_base[slot] = H W_v for each of the M rows; existing slots are overwritten.
- *   H [M][d_model];  W_packed [2*n_kv_heads*head_dim][d_model];  slot_mapping / start_slot as above. */
+ *   H [M][d_model];  W_packed: 2*n_kv_heads*head_dim packed rows (W_k columns, then W_v columns);
+ *   slot_mapping / start_slot as above. */
 int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
                              const void* W_packed, const int32_t* slot_mapping, int64_t start_slot,
                              const precc_cache* cache, void* stream);
@@ -142,8 +146,8 @@ int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const
 /* Both of the above in one pass over H (Section 3.1: the hidden states of a newly processed segment
  * feed the base cache and every agent's LR cache; Section 3.2: the adapter-free pass writes the neutral
  * base rows and the other agents' LR rows).  H is read from HBM once and one kernel runs instead of two.
- *   WA_packed  [2*n_kv_heads*head_dim + n_agents*(rank_k+rank_v)][d_model]: the packed W rows followed by
- *              the packed A rows (precc_pack_kmajor into one buffer)
+ *   WA_packed  2*n_kv_heads*head_dim + n_agents*(rank_k+rank_v) packed rows: the W rows followed by the A
+ *              rows (precc_pack_kmajor into one buffer of that many rows)
  *   agent_mask selects the LR caches written; the base rows are always written.
  * Results are bit-identical to precc_rebase_project followed by precc_lr_precompute. */
 int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,

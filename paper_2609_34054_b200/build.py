@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libprecc.so")
 SOURCES = ["precc_api.cu"]
-HEADERS = ["common.cuh", "decode.cuh", "prefill.cuh", "prefill_tc.cuh", "gemm_tc.cuh", os.path.join("..", "..", "include", "precc.h")]
+HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith(".cuh")) + [os.path.join("..", "..", "include", "precc.h")]
 
 
 def _stale() -> bool:

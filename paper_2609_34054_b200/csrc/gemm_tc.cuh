@@ -88,6 +88,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
 // 1024 bytes apart (start >> 4 | LBO(ignored) | SBO = 1024 >> 4 | version 1 | layout SWIZZLE_128B).
 __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
@@ -119,6 +125,37 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
+}
+
+// Routes eight consecutive output columns [gc, gc+8) of one row (cache block `blk`, offset `off`) to
+// their place in the paged caches: column -> (projection, head, c) for base columns, (projection, agent,
+// r) for LR columns (skipped when the agent is masked out).  Pieces never straddle a destination row
+// because head_dim and the ranks are multiples of 8.
+__device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, int off, int gc, const float (&v8)[8]) {
+  const int w = p.n_kv * p.hd;
+  __nv_bfloat16* dst;
+  const bool to_base = p.mode == 1 || (p.mode == 2 && gc < 2 * w);
+  if (!to_base) {
+    const int n_k = p.n_agents * p.rank_k;
+    const int gl = p.mode == 2 ? gc - 2 * w : gc;
+    const bool is_v = gl >= n_k;
+    const int rr = is_v ? p.rank_v : p.rank_k;
+    const int cc = is_v ? gl - n_k : gl;
+    const int agent = cc / rr, ri = cc % rr;
+    if (!((p.agent_mask >> agent) & 1ull)) return;
+    dst = (is_v ? p.lr_v : p.lr_k) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
+  } else {
+    const bool is_v = gc >= w;
+    const int cc = is_v ? gc - w : gc;
+    const int g = cc / p.hd, c = cc % p.hd;
+    dst = (is_v ? p.base_v : p.base_k) + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
+  }
+  uint4 v;
+  v.x = pack_bf16(v8[0], v8[1]);
+  v.y = pack_bf16(v8[2], v8[3]);
+  v.z = pack_bf16(v8[4], v8[5]);
+  v.w = pack_bf16(v8[6], v8[7]);
+  *reinterpret_cast<uint4*>(dst) = v;
 }
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -172,7 +209,7 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
           const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
           mbar_expect_tx(full0 + 8 * s, stage_bytes);
           tma_load_2d(sa, &map_x, kb * GEMM_BK, m0, full0 + 8 * s);
-          tma_load_2d(sa + GEMM_A_BYTES, &map_w, kb * GEMM_BK, n0, full0 + 8 * s);
+          tma_load_3d(sa + GEMM_A_BYTES, &map_w, 0, n0, kb, full0 + 8 * s);      // packed weights are k-blocked
         }
       }
     }
@@ -204,7 +241,6 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // ---- epilogue: TMEM lane = tile row; this warp may touch lanes 32*(warp%4) .. +31
     const int lane_base = (warp & 3) * 32;
     const int row = lane_base + lane;
-    const int n_k = p.n_agents * p.rank_k;
     const int w = p.n_kv * p.hd;
     int i = 0;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
@@ -261,28 +297,10 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int h = 0; h < 2; ++h) {
           const int gc = n0 + c0 + 8 * h;
           if (!row_ok || gc >= p.N_out) continue;
-          __nv_bfloat16* dst;
-          const bool to_base = p.mode == 1 || (p.mode == 2 && gc < 2 * w);
-          if (!to_base) {
-            const int gl = p.mode == 2 ? gc - 2 * w : gc;
-            const bool is_v = gl >= n_k;
-            const int rr = is_v ? p.rank_v : p.rank_k;
-            const int cc = is_v ? gl - n_k : gl;
-            const int agent = cc / rr, ri = cc % rr;
-            if (!((p.agent_mask >> agent) & 1ull)) continue;
-            dst = (is_v ? p.lr_v : p.lr_k) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
-          } else {
-            const bool is_v = gc >= w;
-            const int cc = is_v ? gc - w : gc;
-            const int g = cc / p.hd, c = cc % p.hd;
-            dst = (is_v ? p.base_v : p.base_k) + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
-          }
-          uint4 v;
-          v.x = pack_bf16(__uint_as_float(r[8 * h + 0]), __uint_as_float(r[8 * h + 1]));
-          v.y = pack_bf16(__uint_as_float(r[8 * h + 2]), __uint_as_float(r[8 * h + 3]));
-          v.z = pack_bf16(__uint_as_float(r[8 * h + 4]), __uint_as_float(r[8 * h + 5]));
-          v.w = pack_bf16(__uint_as_float(r[8 * h + 6]), __uint_as_float(r[8 * h + 7]));
-          *reinterpret_cast<uint4*>(dst) = v;
+          float v8[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(r[8 * h + k]);
+          store_piece(p, blk, off, gc, v8);
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");

@@ -12,6 +12,7 @@
 #include "../../include/precc.h"
 #include "decode.cuh"
 #include "gemm_tc.cuh"
+#include "proj_small.cuh"
 #include "prefill.cuh"
 #include "prefill_tc.cuh"
 
@@ -25,6 +26,7 @@ struct precc_ctx {
   unsigned long long* trace = nullptr; // optional caller-owned trace buffer
   size_t trace_blocks = 0;
   bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
+  bool force_tiled_gemm = false;       // PRECC_GEMM=tiled in the environment: never take the few-row kernel
   char err[512] = {0};
   CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                            const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -94,7 +96,10 @@ float softmax_scale_log2(const precc_layer_desc* d) {
 }
 
 // ------------------------------------------------------------------------------------------ pack
-__global__ void pack_kmajor_kernel(const __nv_bfloat16* __restrict__ src, int d, int n, __nv_bfloat16* __restrict__ dst, int row0) {
+// dst is k-blocked: element (row, i) lives at ((i / 64) * dst_rows + row) * 64 + i % 64, so the 64-deep k
+// step of any range of rows is one contiguous run in memory (what a TMA box of the GEMMs fetches).
+__global__ void pack_kmajor_kernel(const __nv_bfloat16* __restrict__ src, int d, int n, __nv_bfloat16* __restrict__ dst, int dst_rows,
+                                   int row0) {
   __shared__ __nv_bfloat16 tile[32][33];
   const int c0 = blockIdx.x * 32, i0 = blockIdx.y * 32;
   for (int r = threadIdx.y; r < 32; r += blockDim.y) {
@@ -104,7 +109,7 @@ __global__ void pack_kmajor_kernel(const __nv_bfloat16* __restrict__ src, int d,
   __syncthreads();
   for (int r = threadIdx.y; r < 32; r += blockDim.y) {
     const int c = c0 + r, i = i0 + threadIdx.x;
-    if (c < n && i < d) dst[(size_t)(row0 + c) * d + i] = tile[threadIdx.x][r];
+    if (c < n && i < d) dst[((size_t)(i / GEMM_BK) * dst_rows + row0 + c) * GEMM_BK + i % GEMM_BK] = tile[threadIdx.x][r];
   }
 }
 
@@ -118,6 +123,19 @@ int32_t make_map(precc_ctx* ctx, CUtensorMap* map, const void* base, int rows, i
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(ctx, PRECC_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  return PRECC_OK;
+}
+
+// Tensor map over a k-blocked packed weight matrix [K/64][rows][64]: box = `box_rows` rows of one k block.
+int32_t make_map_w(precc_ctx* ctx, CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+  const cuuint64_t dims[3] = {(cuuint64_t)GEMM_BK, (cuuint64_t)rows, (cuuint64_t)(K / GEMM_BK)};
+  const cuuint64_t strides[2] = {(cuuint64_t)GEMM_BK * 2, (cuuint64_t)rows * GEMM_BK * 2};
+  const cuuint32_t box[3] = {(cuuint32_t)GEMM_BK, (cuuint32_t)box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, PRECC_ERR_CUDA, "cuTensorMapEncodeTiled (packed weights) failed (%d)", (int)r);
   return PRECC_OK;
 }
 
@@ -145,7 +163,51 @@ int pick_bn(int n_out, int m_tiles, int sm_count) {
   return 64;
 }
 
+// Few rows (decode steps): the weight-streaming split-K kernel.  The K split depends on K alone, so a
+// column's summation order - and with it every output bit - is the same whichever entry point (LR only,
+// base only, fused) produced it.
+int32_t launch_small(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
+  int cs = 8;
+  while (cs > 1 && (K / cs < 512 || K % (PS_BK * cs) != 0)) cs >>= 1;
+  const int k_slice = K / cs;
+  const int steps = k_slice / PS_BK;
+  const int mt = M <= 16 ? 1 : (M <= 32 ? 2 : 4);
+  const int smem = ps_smem_bytes(mt);
+  if (steps < 1 || smem > ctx->max_smem_optin) return -1;                // caller falls back to the tiled kernel
+  gp.M = M; gp.N_out = n_out; gp.K = K; gp.status = ctx->status;
+  const int cols = ps_cols(mt);
+  CUtensorMap map_x, map_w;
+  int32_t rc = make_map(ctx, &map_x, X, M, K, mt * 16);
+  if (rc) return rc;
+  rc = make_map_w(ctx, &map_w, Wt, n_out, K, cols);
+  if (rc) return rc;
+  const int groups = (n_out + cols - 1) / cols;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(groups * cs);
+  cfg.blockDim = dim3(PS_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = cs; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  auto go = [&](auto kern) -> int32_t {
+    PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, map_x, map_w, gp, k_slice));
+    return PRECC_OK;
+  };
+  if (mt == 1) return go(proj_small_kernel<1>);
+  if (mt == 2) return go(proj_small_kernel<2>);
+  return go(proj_small_kernel<4>);
+}
+
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
+  if (M <= PS_MAX_M && !gp.rope && !ctx->force_tiled_gemm) {
+    const int32_t rc = launch_small(ctx, X, M, K, Wt, n_out, gp, stream);
+    if (rc >= 0) return rc;
+  }
   const int m_tiles = (M + GEMM_BM - 1) / GEMM_BM;
   int bn = pick_bn(n_out, m_tiles, ctx->sm_count);
   if (gp.rope && bn % gp.hd != 0) bn = gp.hd;        // a head's two halves must sit in one tile
@@ -161,7 +223,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   CUtensorMap map_x, map_w;
   int32_t rc = make_map(ctx, &map_x, X, M, K, GEMM_BM);
   if (rc) return rc;
-  rc = make_map(ctx, &map_w, Wt, n_out, K, bn);
+  rc = make_map_w(ctx, &map_w, Wt, n_out, K, bn);
   if (rc) return rc;
   gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
   gp.status = ctx->status;
@@ -471,6 +533,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
     ctx->encode_tiled = reinterpret_cast<decltype(ctx->encode_tiled)>(fn);
   }
   if (const char* v = getenv("PRECC_PREFILL")) ctx->force_simple_prefill = (strcmp(v, "simple") == 0);
+  if (const char* v = getenv("PRECC_GEMM")) ctx->force_tiled_gemm = (strcmp(v, "tiled") == 0);
   if (e != cudaSuccess) {
     fprintf(stderr, "precc_create: %s\n", cudaGetErrorString(e));
     if (ctx->status) cudaFree(ctx->status);
@@ -532,9 +595,9 @@ int32_t precc_pack_kmajor(precc_ctx* ctx, const void* src, int32_t d_model, int3
   if (n_cols == 0) return PRECC_OK;
   if (!src || !dst || d_model <= 0 || n_cols < 0 || dst_row0 < 0 || dst_row0 + n_cols > dst_rows)
     return fail(ctx, PRECC_ERR_INVALID_ARG, "pack_kmajor: bad arguments");
-  if (d_model % 8) return fail(ctx, PRECC_ERR_UNSUPPORTED, "pack_kmajor: d_model %% 8 != 0");
+  if (d_model % GEMM_BK) return fail(ctx, PRECC_ERR_UNSUPPORTED, "pack_kmajor: d_model %% 64 != 0");
   dim3 grid((n_cols + 31) / 32, (d_model + 31) / 32), block(32, 8);
-  pack_kmajor_kernel<<<grid, block, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)src, d_model, n_cols, (__nv_bfloat16*)dst, dst_row0);
+  pack_kmajor_kernel<<<grid, block, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)src, d_model, n_cols, (__nv_bfloat16*)dst, dst_rows, dst_row0);
   PRECC_CUDA(ctx, cudaGetLastError());
   return PRECC_OK;
 }

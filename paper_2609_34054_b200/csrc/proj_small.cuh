@@ -1,0 +1,165 @@
+// Projection for a handful of rows (decode steps, M <= 64): Y[M x n_out] = X[M x K] . Wt^T with the same
+// routing epilogue as the tensor-memory GEMM (LR caches, base caches, or both).
+//
+// With M this small the work is one pass over the packed weights (n_out x K bf16), so the kernel is a
+// weight-streaming kernel: HBM-bound at n_out*K*2 bytes.  A 128-row tcgen05 tile would leave all but
+// n_out/BN blocks idle; here the grid covers every SM:
+//   block  = 64 output columns (128 when M > 16) x one K slice; the K slices of a column group form a
+//            thread-block cluster (split-K, up to 8);
+//   loads  = TMA: per 64-deep k step one box of W rows (contiguous in memory: the packed weights are
+//            k-blocked, [K/64][n_out][64]) and one box of X rows (rows past M are zero-filled
+//            by the out-of-bounds rule) into a 4-slot ring of 128-byte-swizzled shared memory, issued by
+//            a producer warp (full/empty mbarriers).  The ring is kept small on purpose: every cluster of
+//            the grid must be resident at once, or the launch runs in two waves;
+//   math   = mma.sync m16n8k16 (bf16 -> fp32): X rows on the M axis, a warp owns 8 (16 when M > 16)
+//            output columns; fragments come from shared memory with ldmatrix;
+//   reduce = partial tiles go to shared memory; after a cluster barrier each block sums one slice of the
+//            columns over its peers through distributed shared memory (rank order: deterministic) and
+//            scatters bf16 pieces into the paged caches.  No global scratch, no atomics.
+// The K split depends on K alone, so an output value does not depend on which entry point, which other
+// columns or how many other rows were in the call.
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace precc {
+
+constexpr int PS_WARPS = 8;
+constexpr int PS_BK = 64;                   // k elements per step: one 128-byte swizzle row
+constexpr int PS_MAX_M = 64;
+constexpr int PS_STAGES = 4;
+constexpr int PS_THREADS = (PS_WARPS + 1) * 32;       // consumer warps + one producer warp
+__host__ __device__ constexpr int ps_nt(int mt) { return mt > 1 ? 2 : 1; }               // 8-column n-tiles per warp
+__host__ __device__ constexpr int ps_cols(int mt) { return PS_WARPS * 8 * ps_nt(mt); }   // output columns per block
+__host__ __device__ constexpr int ps_step_bytes(int mt) { return (ps_cols(mt) + mt * 16) * PS_BK * 2; }
+__host__ __device__ constexpr int ps_smem_bytes(int mt) {
+  return PS_STAGES * ps_step_bytes(mt) + 2 * PS_STAGES * 8 + 1024;   // ring | mbarriers | alignment slack
+}
+
+template <int MT>
+__global__ void __launch_bounds__(PS_THREADS)
+proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const GemmParams p,
+                  const int k_slice) {
+  constexpr int NT = ps_nt(MT);
+  constexpr int COLS = ps_cols(MT);
+  constexpr int W_BYTES = COLS * PS_BK * 2;
+  constexpr int STEP_BYTES = ps_step_bytes(MT);
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint32_t rank, CS;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(rank));
+  asm volatile("mov.u32 %0, %%cluster_nctaid.x;\n" : "=r"(CS));
+  const int group = blockIdx.x / CS;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k0 = rank * k_slice;
+  const int steps = k_slice / PS_BK;
+  const uint32_t tiles = smem_u32(smem);
+  const uint32_t full0 = tiles + PS_STAGES * STEP_BYTES, empty0 = full0 + 8 * PS_STAGES;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < PS_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, PS_WARPS); }
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+  }
+  pdl_wait();                 // X may be the previous kernel's output
+  pdl_launch_dependents();
+  __syncthreads();
+
+  float acc[MT][NT][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int t = 0; t < NT; ++t) { acc[mt][t][0] = acc[mt][t][1] = acc[mt][t][2] = acc[mt][t][3] = 0.f; }
+
+  if (warp == PS_WARPS) {
+    // ---- producer: one lane walks the k steps of this block's slice
+    if (lane == 0) {
+      for (int s = 0; s < steps; ++s) {
+        const int slot = s % PS_STAGES;
+        if (s >= PS_STAGES) mbar_wait(empty0 + 8 * slot, ((s / PS_STAGES) - 1) & 1, p.status);
+        const uint32_t dst = tiles + slot * STEP_BYTES;
+        mbar_expect_tx(full0 + 8 * slot, STEP_BYTES);
+        tma_load_3d(dst, &map_w, 0, group * COLS, k0 / PS_BK + s, full0 + 8 * slot);   // one contiguous run of the k-blocked weights
+        tma_load_2d(dst + W_BYTES, &map_x, k0 + s * PS_BK, 0, full0 + 8 * slot);
+      }
+    }
+  } else {
+    const int mi = lane >> 3, ri = lane & 7;
+    for (int s = 0; s < steps; ++s) {
+      const int slot = s % PS_STAGES;
+      mbar_wait(full0 + 8 * slot, (s / PS_STAGES) & 1, p.status);
+      const uint32_t wt = tiles + slot * STEP_BYTES, xt = wt + W_BYTES;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {                      // two k steps of 16 per ldmatrix of W
+        uint32_t b[NT][4];
+#pragma unroll
+        for (int t = 0; t < NT; ++t) ldsm_x4(b[t], wt + swz_off<8>((warp * NT + t) * 8 + ri, 4 * j + mi));
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t a[4];
+            ldsm_x4(a, xt + swz_off<8>(mt * 16 + ri + (mi & 1) * 8, 2 * (2 * j + h) + (mi >> 1)));
+#pragma unroll
+            for (int t = 0; t < NT; ++t) mma_bf16_16816(acc[mt][t], a, b[t][2 * h], b[t][2 * h + 1]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(empty0 + 8 * slot) : "memory");
+    }
+  }
+  __syncthreads();                                     // all reads of the tiles are done; the region is reused
+
+  // ---- partial tile [MT*16][COLS] fp32 -> shared memory
+  float* part = reinterpret_cast<float*>(smem);
+  if (warp < PS_WARPS) {
+    const int r = lane >> 2, q = lane & 3;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int t = 0; t < NT; ++t) {
+        const int col = (warp * NT + t) * 8 + 2 * q;
+        *reinterpret_cast<float2*>(part + (mt * 16 + r) * COLS + col) = make_float2(acc[mt][t][0], acc[mt][t][1]);
+        *reinterpret_cast<float2*>(part + (mt * 16 + r + 8) * COLS + col) = make_float2(acc[mt][t][2], acc[mt][t][3]);
+      }
+  }
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+
+  // ---- this block finishes columns [rank*COLS/CS, (rank+1)*COLS/CS) of its group: 8-column pieces,
+  //      all peers' values requested at once, added in rank order
+  const int pieces_per_row = COLS / 8 / CS;             // CS in {1,2,4,8}
+  const uint32_t part_u32 = smem_u32(part);
+  for (int it = threadIdx.x; it < p.M * pieces_per_row; it += PS_THREADS) {
+    const int row = it / pieces_per_row, pc = it % pieces_per_row;
+    const int col = (rank * pieces_per_row + pc) * 8;
+    const int gc = group * COLS + col;
+    if (gc >= p.N_out) continue;
+    float4 x0[8], x1[8];
+#pragma unroll
+    for (uint32_t s = 0; s < 8; ++s) {
+      if (s < CS) {
+        uint32_t remote;
+        asm("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(part_u32 + (row * COLS + col) * 4), "r"(s));
+        asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(x0[s].x), "=f"(x0[s].y), "=f"(x0[s].z), "=f"(x0[s].w) : "r"(remote));
+        asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(x1[s].x), "=f"(x1[s].y), "=f"(x1[s].z), "=f"(x1[s].w) : "r"(remote + 16));
+      } else {
+        x0[s] = make_float4(0.f, 0.f, 0.f, 0.f); x1[s] = x0[s];
+      }
+    }
+    float v8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      v8[0] += x0[s].x; v8[1] += x0[s].y; v8[2] += x0[s].z; v8[3] += x0[s].w;
+      v8[4] += x1[s].x; v8[5] += x1[s].y; v8[6] += x1[s].z; v8[7] += x1[s].w;
+    }
+    long long slot = p.slot_mapping ? (long long)p.slot_mapping[row] : p.start_slot + row;
+    if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); continue; }
+    store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8);
+  }
+  // nobody leaves while a peer may still read its partial tile
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+
+}  // namespace precc

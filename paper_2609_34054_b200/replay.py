@@ -1,0 +1,221 @@
+"""Turn-loop replay of controlled multi-agent traces through the KV-path kernels (Sections 3.1-3.2, 4.1).
+
+A trace is a list of agent turns over one growing shared trajectory: turn = (agent j, n_in tokens that
+arrive as input, n_out tokens the agent decodes).  For every layer the replay issues exactly the KV-path
+work a sharing policy implies and nothing else (no MLP, no query/output projections, random hidden
+states and queries), so its times are the KV-path share of a turn, not model latencies:
+
+  prelr       PreLRShared: new tokens -> base rows + LR rows of ALL agents (one fused projection), then
+              attention of agent j over base + own LR cache; the same per decoded token.
+  rebase_lp   ReBaseShared with lazy prefill: during the turn only agent j's LR rows are written; after
+              the turn one contiguous adapter-free pass over the turn's n_in + n_out tokens rewrites the
+              base rows from neutral hidden states, writes the other agents' LR rows and runs plain
+              attention over the neutral base cache.  That pass is outside TTFT and inside total time.
+  fullshared  one shared full-width cache, no agent-specific part (the lower bound the paper compares to).
+  nonshared   every agent keeps a private full-width cache and first processes all tokens it has not
+              seen (everything the other agents appended since its last turn).
+
+TTFT of a turn = its prefill phase (projection + prefill attention over all layers); the trace's TTFT is
+the sum over turns; throughput = trajectory tokens / total time (Section 4.1).  Decode steps are one
+CUDA graph per turn (all layers, device-side context length and slot), replayed n_out times.
+
+Run:  python -m paper_2609_34054_b200.replay --lengths 1900,17300,66400 --layers 32
+"""
+from __future__ import annotations
+
+import argparse
+import json
+from dataclasses import dataclass
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+from . import inputs as I
+from .binding import Cache, Precc, layer_desc
+
+POLICIES = ("prelr", "rebase_lp", "fullshared", "nonshared")
+
+
+@dataclass(frozen=True)
+class Turn:
+    agent: int
+    n_in: int
+    n_out: int
+
+
+def three_agent_trace(total_tokens: int, cycles: int = 2, prompt: int = 256, short_in: int = 64, n_out: int = 64) -> List[Turn]:
+    """plan -> action -> reflect cycles; the action agent receives the retrieved context, which is the
+    part that varies with the trajectory length; every call decodes a short segment."""
+    fixed = prompt + cycles * (3 * n_out + 2 * short_in)
+    retrieved = max(16, (total_tokens - fixed) // cycles)
+    turns: List[Turn] = []
+    for c in range(cycles):
+        turns.append(Turn(0, (prompt if c == 0 else 0) + short_in, n_out))    # plan
+        turns.append(Turn(1, retrieved, n_out))                               # action: tool observation arrives
+        turns.append(Turn(2, short_in, n_out))                                # reflect
+    return turns
+
+
+def round_robin_trace(n_agents: int, n_turns: int = 8, retrieved: int = 8192, n_out: int = 64) -> List[Turn]:
+    """Fixed retrieved context per turn, agents in round-robin order (the agent-count experiment)."""
+    return [Turn(t % n_agents, retrieved, n_out) for t in range(n_turns)]
+
+
+def trace_tokens(turns: Sequence[Turn]) -> int:
+    return sum(t.n_in + t.n_out for t in turns)
+
+
+class Stack:
+    """Per-layer device state: caches, packed weights, B factors (distinct per layer unless
+    ``shared_weights``, so that a layer's weights are not found in L2 by the next one).  Hidden states and
+    queries are random buffers shared by all layers (their values do not affect the work done)."""
+
+    def __init__(self, px: Precc, geo: I.Geometry, n_layers: int, max_tokens: int, max_rows: int, seed: int = 0,
+                 shared_weights: bool = False):
+        self.px, self.geo, self.n_layers = px, geo, n_layers
+        self.desc = layer_desc(geo)
+        n_blocks = (max_tokens + I.PAGE - 1) // I.PAGE
+        self.caches = [Cache(geo, n_blocks, fill=0.0) for _ in range(n_layers)]
+        n_w = 1 if shared_weights else n_layers
+        self.WA, self.W, self.B_k, self.B_v = [], [], [], []
+        for l in range(n_w):
+            w = {k: v.cuda() for k, v in I.layer_weights(geo, seed, f"L{l}").items()}
+            self.WA.append(px.pack_turn_weights(geo, w["W_k"], w["W_v"], w["A_k"], w["A_v"]))
+            self.W.append(px.pack_base_weights(geo, w["W_k"], w["W_v"]))
+            self.B_k.append(w["B_k"] if geo.rank_k else None)
+            self.B_v.append(w["B_v"] if geo.rank_v else None)
+        self.H = I.normal_bf16((max_rows, geo.d_model), 1.0, seed, "replay.H").cuda()
+        self.q = I.queries(max_rows, geo, seed, "replay.q").cuda()
+        self.out = torch.empty_like(self.q)
+        self.ws = px.decode_workspace(self.desc, 1, max_tokens)
+        self.max_tokens = max_tokens
+
+    def w(self, l: int) -> int:
+        return l if len(self.WA) > 1 else 0
+
+
+def _project(st: Stack, l: int, n: int, start: int, mask: Optional[int], slot_map=None):
+    """mask None: base rows only; else base rows + LR rows of the agents in `mask`."""
+    px, k = st.px, st.w(l)
+    if mask is None or (st.geo.rank_k == 0 and st.geo.rank_v == 0):
+        px.rebase_project(st.desc, st.H[:n], st.W[k], st.caches[l], start, slot_map)
+    else:
+        px.turn_project(st.desc, st.H[:n], st.WA[k], st.caches[l], start, slot_map, mask)
+
+
+def _prefill_phase(st: Stack, n: int, T: int, agent: int, mask: Optional[int]):
+    for l in range(st.n_layers):
+        _project(st, l, n, T, mask)
+        k = st.w(l)
+        st.px.lr_attend_prefill(st.desc, st.q[:n], agent, T, st.B_k[k], st.B_v[k], st.caches[l], st.out[:n])
+
+
+class _DecodeGraph:
+    """One decode step over all layers with device-side position; replayed once per generated token."""
+
+    def __init__(self, st: Stack, agent: int, mask: Optional[int], ctx0: int, max_ctx: int):
+        dev = st.q.device
+        self.ctx = torch.tensor([ctx0], dtype=torch.int32, device=dev)        # tokens attended (incl. the new one)
+        self.slot = torch.tensor([ctx0 - 1], dtype=torch.int32, device=dev)   # where the new token's rows go
+        self.agent = torch.tensor([agent], dtype=torch.int32, device=dev)
+        self.first = torch.zeros(1, dtype=torch.int32, device=dev)
+
+        def step():
+            for l in range(st.n_layers):
+                _project(st, l, 1, 0, mask, self.slot)
+                k = st.w(l)
+                st.px.lr_attend_decode(st.desc, st.q[:1], self.agent, self.ctx, max_ctx, st.B_k[k], st.B_v[k], st.caches[l],
+                                       st.out[:1], st.ws, None, self.first)
+            self.ctx.add_(1)
+            self.slot.add_(1)
+
+        step()                                       # warm-up outside capture (also the first real step)
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            step()
+
+    def run(self, n: int):
+        for _ in range(n):
+            self.graph.replay()
+
+
+def _timed(fn) -> float:
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    fn()
+    e1.record()
+    e1.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def replay(st: Stack, turns: Sequence[Turn], policy: str) -> Dict[str, float]:
+    """Replays one trace under one policy; returns milliseconds and token counts."""
+    if policy not in POLICIES:
+        raise ValueError(f"policy must be one of {POLICIES}")
+    geo = st.geo
+    all_mask = (1 << geo.n_agents) - 1
+    ttft = decode_ms = rebase_ms = 0.0
+    P = 0                                            # shared trajectory length so far
+    seen = [0] * geo.n_agents                        # nonshared: tokens each agent's private cache covers
+    prefilled = 0
+    for t in turns:
+        j = t.agent
+        if policy == "nonshared":
+            start, n_pref, agent, mask = seen[j], P - seen[j] + t.n_in, -1, None
+        elif policy == "fullshared":
+            start, n_pref, agent, mask = P, t.n_in, -1, None
+        elif policy == "prelr":
+            start, n_pref, agent, mask = P, t.n_in, j, all_mask
+        else:
+            start, n_pref, agent, mask = P, t.n_in, j, 1 << j
+        prefilled += n_pref
+        ttft += _timed(lambda: _prefill_phase(st, n_pref, start, agent, mask))
+        ctx0 = P + t.n_in + 1
+        if t.n_out > 0:
+            g = _DecodeGraph(st, agent, mask, ctx0, P + t.n_in + t.n_out)     # runs the first decode step itself
+            decode_ms += _timed(lambda: g.run(t.n_out - 1)) * t.n_out / max(1, t.n_out - 1)
+        if policy == "rebase_lp":
+            n_c = t.n_in + t.n_out
+            rebase_ms += _timed(lambda: _prefill_phase(st, n_c, P, -1, all_mask & ~(1 << j)))
+        P += t.n_in + t.n_out
+        seen[j] = P
+    total = ttft + decode_ms + rebase_ms
+    per_tok = 2 * geo.n_kv * geo.hd * 2
+    lr_tok = (geo.rank_k + geo.rank_v) * 2 * geo.n_agents
+    cache_bytes = {"nonshared": per_tok * geo.n_agents, "fullshared": per_tok}.get(policy, per_tok + lr_tok) * P * st.n_layers
+    return {"policy": policy, "tokens": P, "turns": len(turns), "prefilled_tokens": prefilled, "ttft_ms": ttft,
+            "decode_ms": decode_ms, "rebase_ms": rebase_ms, "total_ms": total, "tokens_per_s": P / total * 1e3,
+            "cache_gb": cache_bytes / 1e9}
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
+    ap.add_argument("--lengths", default="1900,3000,5000,9100,17300,33700,66400")
+    ap.add_argument("--layers", type=int, default=32)
+    ap.add_argument("--agents", type=int, default=3)
+    ap.add_argument("--rank", type=int, default=32)
+    ap.add_argument("--policies", default=",".join(POLICIES))
+    ap.add_argument("--round-robin", type=int, default=0, help="instead of the length sweep: N agents, 8 turns x 8192 tokens")
+    args = ap.parse_args(argv)
+    px = Precc(0)
+    n_agents = args.round_robin or args.agents
+    geo = I.Geometry(d_model=4096, n_q=32, n_kv=8, hd=128, n_agents=n_agents, rank_k=args.rank, rank_v=args.rank,
+                     alpha=2.0 * args.rank)
+    traces = [round_robin_trace(n_agents)] if args.round_robin else [three_agent_trace(int(x)) for x in args.lengths.split(",")]
+    for turns in traces:
+        total = trace_tokens(turns)
+        rows = max(total, 64)                         # nonshared may prefill nearly the whole trajectory at once
+        st = Stack(px, geo, args.layers, total + I.PAGE, rows)
+        for pol in args.policies.split(","):
+            r = replay(st, turns, pol)
+            r.update({"layers": args.layers, "n_agents": n_agents, "rank": args.rank})
+            print(json.dumps({k: (round(v, 3) if isinstance(v, float) else v) for k, v in r.items()}), flush=True)
+        del st
+        torch.cuda.empty_cache()
+    if px.poll_status() != 0:
+        raise SystemExit("device status flagged an error")
+
+
+if __name__ == "__main__":
+    main()
