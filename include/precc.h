@@ -240,7 +240,7 @@ int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, co
  *   - q must already be rotated by the caller (the query projection is outside this library).
  * Convention: rotate-half pairing, coordinates (c, c + head_dim/2) of a head turn by angle(t, c):
  *   x'[c] = x[c] cos - x[c + hd/2] sin,   x'[c + hd/2] = x[c + hd/2] cos + x[c] sin.
- * Prefill over rotary keys has no entry point yet. */
+ * Cached token t sits at position t in decode and prefill (the new tokens of a turn at ctx_len + i). */
 typedef struct precc_rope {
   const float* table;        /* device fp32 [max_pos][head_dim/2][2]: (cos, sin) of angle(t, c); 16-byte aligned */
   int32_t max_pos;           /* rows of `table` */
@@ -272,6 +272,15 @@ int32_t precc_lr_attend_decode_rope(precc_ctx* ctx, const precc_layer_desc* desc
                                     const void* B_k, const void* B_v, const precc_rope* rope,
                                     const precc_cache* cache, void* out, void* workspace,
                                     size_t workspace_bytes, void* stream);
+
+/* precc_lr_attend_prefill over rotated base keys (rope->max_pos >= ctx_len + S).  The rank-r key term of
+ * every 64-token tile is expanded, rotated and added to the tile in shared memory before the scores are
+ * taken.  With rank_k == 0, or for agent -1, the result equals precc_lr_attend_prefill. */
+int32_t precc_lr_attend_prefill_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S,
+                                     int32_t agent, int32_t ctx_len, const int32_t* block_table,
+                                     int32_t table_stride, int32_t first_block,
+                                     const void* B_k, const void* B_v, const precc_rope* rope,
+                                     const precc_cache* cache, void* out, void* stream);
 
 #ifdef __cplusplus
 }

@@ -255,6 +255,18 @@ def lr_decode_reference_rope(q, agent_id, ctx_len, H, W_k, W_v, A_k, B_k, A_v, B
     return out
 
 
+def lr_prefill_reference_rope(q, agent: int, T: int, H, W_k, W_v, A_k, B_k, A_v, B_v, s_k: float, s_v: float,
+                              n_kv: int, cos, sin, sigma=None, rows=None) -> np.ndarray:
+    """New-turn prefill with rotary keys from first principles: the agent's keys of all T + S tokens are
+    RoPE_t(H_t (W_k + s_k A B)) (token t at position t), values un-rotated, then ``attend_prefill``."""
+    q = as_f64(q)
+    S = q.shape[0]
+    H = as_f64(H)[:T + S]
+    K = rope_rotate(H @ merged_weight(W_k, A_k[agent], B_k[agent], s_k), np.arange(T + S), n_kv, cos, sin)
+    V = H @ merged_weight(W_v, A_v[agent], B_v[agent], s_v)
+    return attend_prefill(q, K, V, T, n_kv, sigma, rows)
+
+
 # ------------------------------------------------------------------ cache accounting
 
 def cache_bytes_per_token(n_kv: int, hd: int, n_agents: int, rank_k: int, rank_v: int,

@@ -22,7 +22,7 @@ EXPORTS = [
     "precc_poll_status", "precc_pack_kmajor", "precc_lr_precompute", "precc_rebase_project", "precc_turn_project",
     "precc_decode_workspace_bytes", "precc_workspace_init", "precc_lr_attend_decode",
     "precc_lr_attend_decode_static", "precc_lr_attend_prefill",
-    "precc_rebase_project_rope", "precc_turn_project_rope", "precc_lr_attend_decode_rope",
+    "precc_rebase_project_rope", "precc_turn_project_rope", "precc_lr_attend_decode_rope", "precc_lr_attend_prefill_rope",
 ]
 
 
@@ -85,6 +85,8 @@ def load_library() -> C.CDLL:
     lib.precc_turn_project_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, u64, rp, C.POINTER(CacheDesc), vp]
     lib.precc_lr_attend_decode_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, i32, vp, i32, vp, vp, rp,
                                                 C.POINTER(CacheDesc), vp, vp, sz, vp]
+    lib.precc_lr_attend_prefill_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp, rp,
+                                                 C.POINTER(CacheDesc), vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is C.c_int:  # default restype: the int32 status code
@@ -282,6 +284,14 @@ class Precc:
             self.h, C.byref(desc), _ptr(q), q.shape[0], _ptr(agent_id), _ptr(ctx_len), _ptr(block_table), stride,
             _ptr(first_block), max_ctx, _ptr(B_k), _ptr(B_v), C.byref(rd), C.byref(cd), _ptr(out), _ptr(workspace),
             workspace.numel(), _stream()), "precc_lr_attend_decode_rope")
+
+    def lr_attend_prefill_rope(self, desc: LayerDesc, q: torch.Tensor, agent: int, ctx_len: int, B_k, B_v, rope: torch.Tensor,
+                               cache: Cache, out: torch.Tensor, block_table: Optional[torch.Tensor] = None, first_block: int = 0):
+        cd, rd = cache.desc(), self._rope(rope)
+        stride = block_table.numel() if block_table is not None else 0
+        self._check(self.lib.precc_lr_attend_prefill_rope(
+            self.h, C.byref(desc), _ptr(q), q.shape[0], agent, ctx_len, _ptr(block_table), stride, first_block,
+            _ptr(B_k), _ptr(B_v), C.byref(rd), C.byref(cd), _ptr(out), _stream()), "precc_lr_attend_prefill_rope")
 
     def decode_workspace(self, desc: LayerDesc, max_batch: int, max_ctx: int) -> torch.Tensor:
         n = self.lib.precc_decode_workspace_bytes(C.byref(desc), max_batch, max_ctx, self.sm_count)

@@ -420,6 +420,7 @@ struct DecodeRunRope {
 struct PrefillArgs {
   const precc_layer_desc* d; const void* q; int S; int agent; int T; const int32_t* block_table; int first_block;
   const void* B_k; const void* B_v; const precc_cache* cache; void* out; cudaStream_t stream;
+  const float* rope = nullptr; int max_pos = 0;      // rotary variant when rope != null
 };
 
 template <int HD, int RK, int RV>
@@ -470,15 +471,16 @@ struct PrefillRun {
                                 reinterpret_cast<uintptr_t>(a.cache->lr_k) | reinterpret_cast<uintptr_t>(a.cache->lr_v)) & 127u) == 0;
       if (kv_rows < (1ll << 31) && aligned128 && !ctx->force_simple_prefill) return run_tc(ctx, a);
     }
-    return run_simple(ctx, a);
+    return run_simple<false>(ctx, a);
   }
-  // mma.sync kernel: ranks 8 and 64, oversized or unaligned caches
+  // mma.sync kernel: ranks 8 and 64, oversized or unaligned caches, and the rotary variant
+  template <bool ROPE = false>
   static int32_t run_simple(precc_ctx* ctx, const PrefillArgs& a) {
     using C = PrefillCfg<HD, RK, RV>;
     const precc_layer_desc* d = a.d;
     int stages = 3;
-    while (stages > 2 && 2 * (C::smem_bytes(stages) + 1024) > ctx->max_smem_optin) --stages;
-    const int smem = C::smem_bytes(stages);
+    while (stages > 2 && 2 * (C::smem_bytes(stages, ROPE) + 1024) > ctx->max_smem_optin) --stages;
+    const int smem = C::smem_bytes(stages, ROPE);
     PrefillParams p;
     const size_t kvw = (size_t)d->n_kv_heads * HD;
     p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;
@@ -491,12 +493,23 @@ struct PrefillRun {
     p.S = a.S; p.T = a.T; p.first_block = a.first_block;
     p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = d->n_q_heads / d->n_kv_heads; p.stages = stages;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
-    auto kern = lr_attend_prefill_kernel<HD, RK, RV>;
+    p.rope = reinterpret_cast<const float4*>(a.rope); p.max_pos = a.max_pos;
+    auto kern = lr_attend_prefill_kernel<HD, RK, RV, ROPE>;
     PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int row_tiles = (a.S * p.group + PF_ROWS - 1) / PF_ROWS;
     kern<<<dim3(row_tiles, d->n_kv_heads), PF_THREADS, smem, a.stream>>>(p);
     PRECC_CUDA(ctx, cudaGetLastError());
     return PRECC_OK;
+  }
+};
+
+// Rotary keys: without a key-side adapter the rotated base cache is all there is (the position-free
+// kernels are exact); with one, the mma.sync kernel expands and rotates the rank-r key term per tile.
+template <int HD, int RK, int RV>
+struct PrefillRunRope {
+  static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
+    if constexpr (RK > 0) return PrefillRun<HD, RK, RV>::template run_simple<true>(ctx, a);
+    else return PrefillRun<HD, RK, RV>::run(ctx, a);
   }
 };
 
@@ -813,9 +826,10 @@ int32_t precc_lr_attend_decode_static(precc_ctx* ctx, const precc_layer_desc* de
                                 cache, out, scratch, PRECC_STATIC_SCRATCH_BYTES, stream);
 }
 
-int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
-                                int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
-                                const void* B_k, const void* B_v, const precc_cache* cache, void* out, void* stream) {
+static int32_t prefill_entry(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
+                             int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
+                             const void* B_k, const void* B_v, const precc_rope* rope, const precc_cache* cache, void* out,
+                             void* stream) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (S < 0 || ctx_len < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "S < 0 or ctx_len < 0");
@@ -833,7 +847,27 @@ int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, co
     return fail(ctx, PRECC_ERR_INVALID_ARG, "blocks [%d, %lld) outside the cache", first_block, first_block + need_blocks);
   if ((long long)S * (desc->n_q_heads / desc->n_kv_heads) > (long long)PF_ROWS * 65535) return fail(ctx, PRECC_ERR_UNSUPPORTED, "S too large");
   PrefillArgs a{desc, q, S, neutral ? 0 : agent, ctx_len, block_table, first_block, B_k, B_v, cache, out, (cudaStream_t)stream};
-  return dispatch_shape<PrefillRun>(ctx, desc->head_dim, neutral ? 0 : desc->rank_k, neutral ? 0 : desc->rank_v, a);
+  if (!rope) return dispatch_shape<PrefillRun>(ctx, desc->head_dim, neutral ? 0 : desc->rank_k, neutral ? 0 : desc->rank_v, a);
+  if (!rope->table || !aligned16(rope->table)) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table is null or not 16-byte aligned");
+  if ((long long)rope->max_pos < (long long)ctx_len + S)
+    return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table covers %d positions, the turn ends at %lld", rope->max_pos, (long long)ctx_len + S);
+  a.rope = rope->table; a.max_pos = rope->max_pos;
+  return dispatch_shape<PrefillRunRope>(ctx, desc->head_dim, neutral ? 0 : desc->rank_k, neutral ? 0 : desc->rank_v, a);
+}
+
+int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
+                                int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
+                                const void* B_k, const void* B_v, const precc_cache* cache, void* out, void* stream) {
+  return prefill_entry(ctx, desc, q, S, agent, ctx_len, block_table, table_stride, first_block, B_k, B_v, nullptr, cache, out, stream);
+}
+
+int32_t precc_lr_attend_prefill_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
+                                     int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
+                                     const void* B_k, const void* B_v, const precc_rope* rope, const precc_cache* cache,
+                                     void* out, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!rope) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope is null");
+  return prefill_entry(ctx, desc, q, S, agent, ctx_len, block_table, table_stride, first_block, B_k, B_v, rope, cache, out, stream);
 }
 
 }  // extern "C"

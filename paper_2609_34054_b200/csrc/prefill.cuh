@@ -7,6 +7,12 @@
 // group): row = i*G + hg.  Four warps x 16 rows; 64-token tiles of {K, V, L^K, L^V} stream through
 // a cp.async ring shared by the block; S = Q'K'^T and O' += P V' run on mma.sync m16n8k16 with the
 // FlashAttention-2 register reuse of P.
+//
+// Rotary variant (ROPE = true, Appendix D.2: rotated base keys, un-rotated LR-K rows): before a tile
+// is used, each warp expands E = L^K (s_k B^K_g) for 16 of the tile's tokens on the tensor cores, rotates
+// it by the tokens' positions (cached token t sits at position t) and adds it onto the key rows in
+// shared memory, so that the score MMA sees the agent's rotated keys; the fold q~ is not used.  The
+// agent's keys exist only in that shared-memory tile.
 #pragma once
 #include "common.cuh"
 
@@ -28,6 +34,8 @@ struct PrefillParams {
   int n_q, n_kv, group;
   int stages;
   float scale_log2, s_k, s_v;
+  const float4* rope;          // rotary variant: [max_pos][hd/4] of (cos c, sin c, cos c+1, sin c+1), c even
+  int max_pos;
 };
 
 constexpr int PF_ROWS = 64;
@@ -44,16 +52,18 @@ struct PrefillCfg {
   static constexpr int LV_BYTES = PF_TOK * RV * 2;
   static constexpr int STAGE_BYTES = 2 * KV_BYTES + LK_BYTES + LV_BYTES;
   static constexpr int OW = HD + RV;
-  __host__ __device__ static constexpr int smem_bytes(int stages) {
-    int stream = Q_BYTES + QX_BYTES + stages * STAGE_BYTES;
+  static constexpr int BK_BYTES = (RK > 16 ? RK : 16) * HD * 2;   // rotary variant: s_k B^K_g slice, rows padded to 16
+  __host__ __device__ static constexpr int smem_bytes(int stages, bool rope = false) {
+    int stream = Q_BYTES + QX_BYTES + stages * STAGE_BYTES + (rope ? BK_BYTES : 0);
     int epi = PF_ROWS * (OW + 1) * 4;
     return (stream > epi ? stream : epi) + 16;
   }
 };
 
-template <int HD, int RK, int RV>
+template <int HD, int RK, int RV, bool ROPE = false>
 __global__ void __launch_bounds__(PF_THREADS)
 lr_attend_prefill_kernel(const PrefillParams p) {
+  static_assert(!ROPE || RK > 0, "the rotary variant only differs when there is a key-side adapter");
   using C = PrefillCfg<HD, RK, RV>;
   constexpr int OW = C::OW;
   constexpr int KC = HD / 16;
@@ -137,7 +147,22 @@ lr_attend_prefill_kernel(const PrefillParams p) {
     }
     *reinterpret_cast<uint4*>(smem + swz_off<CPR_KV>(r, ch)) = v;
   }
-  if constexpr (RK > 0) {
+  const uint32_t bk_u32 = ring_u32 + p.stages * C::STAGE_BYTES;
+  if constexpr (ROPE) {
+    // s_k B^K[:, g] -> shared memory, [max(RK,16)][HD], swizzled like a key tile (rows >= RK are zero)
+    constexpr int ROWS = RK > 16 ? RK : 16;
+    for (int c = threadIdx.x; c < ROWS * CPR_KV; c += PF_THREADS) {
+      const int j = c / CPR_KV, ch = c % CPR_KV;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (j < RK) v = __ldg(reinterpret_cast<const uint4*>(p.B_k + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
+      auto sc = [&](uint32_t x) -> uint32_t {
+        const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x));
+        return pack_bf16(f.x * p.s_k, f.y * p.s_k);
+      };
+      *reinterpret_cast<uint4*>(smem + (bk_u32 - q_u32) + swz_off<CPR_KV>(j, ch)) = make_uint4(sc(v.x), sc(v.y), sc(v.z), sc(v.w));
+    }
+  }
+  if constexpr (RK > 0 && !ROPE) {
     for (int e = threadIdx.x; e < PF_ROWS * C::RKP; e += PF_THREADS) {
       const int r = e / C::RKP, j = e % C::RKP;
       const int row = row0 + r;
@@ -191,6 +216,59 @@ lr_attend_prefill_kernel(const PrefillParams p) {
     const uint32_t st = ring_u32 + (uint32_t)(it % p.stages) * C::STAGE_BYTES;
     const int t0 = it * PF_TOK;
 
+    if constexpr (ROPE) {
+      // this warp's 16 tokens of the tile: K[tok] += RoPE_tok(L^K[tok] . s_k B^K_g), in shared memory
+      constexpr int KH = KC / 2;
+      constexpr int KXR = (RK + 15) / 16;
+      const int ar = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, ac = lane >> 4;   // A operand rows / chunk parity
+      const int br = (lane & 7) + ((lane >> 3) & 1) * 8, bc = lane >> 4;                // B^K slice rows / chunk parity
+      const int r0 = warp * 16 + (lane >> 2), qk = (lane & 3) * 2;
+      uint32_t la[KXR][4];
+#pragma unroll
+      for (int jx = 0; jx < KXR; ++jx) {
+        if constexpr (RK >= 16) {
+          ldsm_x4(la[jx], st + 2 * C::KV_BYTES + swz_off<CPR_LK>(ar, 2 * jx + ac));
+        } else {
+          la[jx][2] = 0u; la[jx][3] = 0u;
+          ldsm_x2(la[jx][0], la[jx][1], st + 2 * C::KV_BYTES + swz_off<1>(ar, 0));
+        }
+      }
+      const int pos0 = min(t0 + r0, p.max_pos - 1), pos1 = min(t0 + r0 + 8, p.max_pos - 1);
+#pragma unroll
+      for (int kc = 0; kc < KH; ++kc) {
+        float e[2][2][4];                               // [half][n-tile][c]
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+          for (int n2 = 0; n2 < 2; ++n2) { e[hf][n2][0] = e[hf][n2][1] = e[hf][n2][2] = e[hf][n2][3] = 0.f; }
+#pragma unroll
+          for (int jx = 0; jx < KXR; ++jx) {
+            uint32_t bf[4];
+            ldsm_x4_t(bf, bk_u32 + swz_off<CPR_KV>(16 * jx + br, 2 * (kc + hf * KH) + bc));
+            mma_bf16_16816(e[hf][0], la[jx], bf[0], bf[1]);
+            mma_bf16_16816(e[hf][1], la[jx], bf[2], bf[3]);
+          }
+        }
+#pragma unroll
+        for (int n2 = 0; n2 < 2; ++n2)
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const int col = kc * 16 + n2 * 8 + qk;                       // lower-half column (even)
+            const float4 c4 = __ldg(p.rope + (size_t)(r ? pos1 : pos0) * (HD / 4) + (col >> 1));
+            const float lo0 = e[0][n2][2 * r], lo1 = e[0][n2][2 * r + 1];
+            const float hi0 = e[1][n2][2 * r], hi1 = e[1][n2][2 * r + 1];
+            const uint32_t rl = pack_bf16(lo0 * c4.x - hi0 * c4.y, lo1 * c4.z - hi1 * c4.w);
+            const uint32_t rh = pack_bf16(hi0 * c4.x + lo0 * c4.y, hi1 * c4.z + lo1 * c4.w);
+            const int row = r0 + 8 * r;
+            __nv_bfloat162* klo = reinterpret_cast<__nv_bfloat162*>(smem + (st - q_u32) + swz_off<CPR_KV>(row, col >> 3) + (col & 7) * 2);
+            __nv_bfloat162* khi = reinterpret_cast<__nv_bfloat162*>(smem + (st - q_u32) + swz_off<CPR_KV>(row, (col + HD / 2) >> 3) + (col & 7) * 2);
+            *klo = __hadd2(*klo, *reinterpret_cast<const __nv_bfloat162*>(&rl));
+            *khi = __hadd2(*khi, *reinterpret_cast<const __nv_bfloat162*>(&rh));
+          }
+      }
+      __syncthreads();                                   // every warp's 16 tokens are updated before any warp reads keys
+    }
+
     float s[PF_TOK / 8][4];
 #pragma unroll
     for (int nt = 0; nt < PF_TOK / 8; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
@@ -206,7 +284,7 @@ lr_attend_prefill_kernel(const PrefillParams p) {
         mma_bf16_16816(s[2 * n2 + 1], a, b[2], b[3]);
       }
     }
-    if constexpr (RK > 0) {
+    if constexpr (RK > 0 && !ROPE) {
 #pragma unroll
       for (int kc = 0; kc < KX; ++kc) {
         uint32_t a[4];

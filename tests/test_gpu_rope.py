@@ -164,6 +164,34 @@ def test_decode_rope_long_context_split_and_paged(px):
     assert_close(out[sel], ref, "rope C2 batch 24")
 
 
+@pytest.mark.parametrize("hd,n_q,n_kv,r,T,S", [(64, 8, 2, 16, 150, 37), (64, 4, 4, 8, 0, 70), (128, 8, 2, 32, 70, 64),
+                                              (128, 8, 1, 64, 33, 20), (64, 16, 2, 32, 333, 5)])
+def test_prefill_rope_shapes(px, hd, n_q, n_kv, r, T, S):
+    geo = I.Geometry(d_model=192, n_q=n_q, n_kv=n_kv, hd=hd, n_agents=2, rank_k=r, rank_v=r, alpha=2.0 * r)
+    L = Layer(px, geo, seed=8, n_blocks=(T + S + 15) // 16, tag="rpf")
+    H = I.hidden_states(T + S, geo, 8, "rpf.H")
+    table = rope_table(T + S + 3, hd)
+    cos, sin = O.rope_tables(T + S + 3, hd)
+    px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0)
+    px.lr_precompute(L.desc, H.cuda(), L.A_packed, L.cache, 0)
+    w = L.w_np
+    q = I.queries(S, geo, 8, "rpf.q", gain=3.0)
+    out = torch.full_like(q, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope(L.desc, q.cuda(), 1, T, L.B_k, L.B_v, table, L.cache, out)
+    torch.cuda.synchronize()
+    ref = O.lr_prefill_reference_rope(f64(q), 1, T, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                      geo.scale_k, geo.scale_v, n_kv, cos, sin)
+    assert_close(f64(out), ref, f"rope prefill hd{hd} r{r}")
+    # last row against the rotary decode kernel at the same context (two different kernels, same definition)
+    dec = f64(_decode_rope(L, q[S - 1:], [1], [T + S], table))
+    assert_close(dec, ref[S - 1:], "rope decode at the turn's last token")
+    # adapter-free view: identical to the position-free prefill over the rotated base
+    a = torch.full_like(q, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope(L.desc, q.cuda(), -1, T, L.B_k, L.B_v, table, L.cache, a)
+    b = L.prefill(q, -1, T)
+    assert torch.equal(a, b)
+
+
 def test_rope_invalid_arguments(px):
     geo = I.Geometry(d_model=192, n_q=8, n_kv=2, hd=64, n_agents=2, rank_k=16, rank_v=16, alpha=32.0)
     L = Layer(px, geo, seed=7, n_blocks=8, tag="ri", fill=0.0)

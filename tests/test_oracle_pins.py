@@ -424,3 +424,15 @@ def test_rope_decode_reference_brute_force():
             m = max(z); e = [math.exp(v - m) for v in z]; den = sum(e)
             for c in range(hd):
                 assert abs(got[b, h, c] - sum(e[t] * V[t][c] for t in range(T)) / den) < 1e-11
+
+
+def test_rope_prefill_row_equals_rope_decode():
+    p = _tiny(T=9, d=8, n_q=4, n_kv=2, hd=4, N=2, rk=2, rv=2, B=3)
+    cos, sin = O.rope_tables(16, 4)
+    T, S = 6, 3
+    got = O.lr_prefill_reference_rope(p["q"], 1, T, p["H"], p["W_k"], p["W_v"], p["A_k"], p["B_k"], p["A_v"], p["B_v"],
+                                      1.5, 0.5, 2, cos, sin)
+    for i in range(S):
+        ref = O.lr_decode_reference_rope(p["q"][i:i + 1], [1], [T + i + 1], p["H"], p["W_k"], p["W_v"], p["A_k"], p["B_k"],
+                                         p["A_v"], p["B_v"], 1.5, 0.5, 2, cos, sin)
+        np.testing.assert_allclose(got[i], ref[0], rtol=1e-12, atol=1e-14)
