@@ -417,6 +417,19 @@ struct DecodeRunRope {
   }
 };
 
+// 4-D map over a base cache [n_blocks][n_kv][16][hd]: box = 64 columns x 16 rows x 1 head x `box_blocks` blocks.
+int32_t make_map_cache4(precc_ctx* ctx, CUtensorMap* map, const void* base, long long n_blocks, int n_kv, int hd, int box_blocks) {
+  const cuuint64_t dims[4] = {(cuuint64_t)hd, (cuuint64_t)PAGE, (cuuint64_t)n_kv, (cuuint64_t)n_blocks};
+  const cuuint64_t strides[3] = {(cuuint64_t)hd * 2, (cuuint64_t)PAGE * hd * 2, (cuuint64_t)n_kv * PAGE * hd * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)PAGE, 1, (cuuint32_t)box_blocks};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, PRECC_ERR_CUDA, "cuTensorMapEncodeTiled (4-D cache) failed (%d)", (int)r);
+  return PRECC_OK;
+}
+
 struct PrefillArgs {
   const precc_layer_desc* d; const void* q; int S; int agent; int T; const int32_t* block_table; int first_block;
   const void* B_k; const void* B_v; const precc_cache* cache; void* out; cudaStream_t stream;
@@ -442,21 +455,28 @@ struct PrefillRun {
     const long long kv_rows = (long long)a.cache->n_blocks * d->n_kv_heads * PAGE;
     const long long lr_rows = (long long)a.cache->n_blocks * PAGE;
     CUtensorMap mk, mv, mlk, mlv;
-    int32_t rc = make_map2(ctx, &mk, a.cache->k_base, kv_rows, HD, PAGE, 64);
+    // without a block table the pages of a 128-token stage are consecutive: whole-stage boxes (one TMA
+    // instruction per 64-column slab instead of one per page)
+    const bool contig = a.block_table == nullptr;
+    const int box_rows = contig ? PTC_TOK : PAGE;
+    int32_t rc = contig ? make_map_cache4(ctx, &mk, a.cache->k_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
+                        : make_map2(ctx, &mk, a.cache->k_base, kv_rows, HD, PAGE, 64);
     if (rc) return rc;
-    rc = make_map2(ctx, &mv, a.cache->v_base, kv_rows, HD, PAGE, 64);
+    rc = contig ? make_map_cache4(ctx, &mv, a.cache->v_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
+                : make_map2(ctx, &mv, a.cache->v_base, kv_rows, HD, PAGE, 64);
     if (rc) return rc;
     mlk = mk; mlv = mv;     // placeholders when a rank is zero (never dereferenced)
-    if (RK) { rc = make_map2(ctx, &mlk, (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * lr_rows * RK, lr_rows, RK, PAGE, RK); if (rc) return rc; }
-    if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, PAGE, 64); if (rc) return rc; }
+    if (RK) { rc = make_map2(ctx, &mlk, (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * lr_rows * RK, lr_rows, RK, box_rows, RK); if (rc) return rc; }
+    if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, box_rows, 64); if (rc) return rc; }
     PrefillTcParams p;
     p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;
     p.B_k = RK ? (const __nv_bfloat16*)a.B_k + (size_t)a.agent * RK * kvw : nullptr;
     p.B_v = RV ? (const __nv_bfloat16*)a.B_v + (size_t)a.agent * RV * kvw : nullptr;
     p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
-    p.S = a.S; p.T = a.T; p.first_block = a.first_block;
+    p.S = a.S; p.T = a.T; p.first_block = a.first_block; p.contig = contig ? 1 : 0;
     p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.k_stages = ks; p.v_stages = vs;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
+    p.trace = (ctx->trace && ctx->trace_blocks >= 32) ? ctx->trace : nullptr;
     auto kern = lr_attend_prefill_tc_kernel<HD, RK, RV>;
     PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int row_tiles = (a.S + p.tok_per_tile - 1) / p.tok_per_tile;

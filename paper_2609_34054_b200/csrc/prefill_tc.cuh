@@ -3,19 +3,30 @@
 // One thread block = up to 128 query rows of one kv head (row = new token i * G + head-in-group) against
 // the whole visible context, 128 tokens per step:
 //   S  = Q K_base^T + Q~ L_K^T                 tcgen05.mma, A/B from shared memory, S in TMEM (2 buffers)
-//   P  = exp2(S*scale - m)                     4 softmax warps, one TMEM lane (= query row) per thread,
-//                                              written back over S as packed bf16
-//   O' += P [V_base | L_V]                      tcgen05.mma with A = P from TMEM, O' (hd + r_v columns) in TMEM
+//   P  = exp2(S*scale - m)                     8 softmax warps, two threads per TMEM lane (= query row);
+//                                              packed bf16 in its own 64 TMEM columns
+//   O' += P [V_base | L_V | 1]                  tcgen05.mma with A = P from TMEM; O' in TMEM holds the numerator
+//                                              (hd columns), U = P L_V (r_v columns) and, through a column of
+//                                              ones written into the zero-padded L_V slab, the denominator
 // and finally out = (O + s_v U B_v) / l on the CUDA cores.  The key-side fold Q~ = s_k Q B_k^T is
-// computed once per block by the softmax threads.  Pages of the caches arrive by TMA (one box per page
-// and 64-column slab, 128/64/32-byte swizzle) into a ring of stages guarded by mbarriers.
+// computed once per block by the softmax threads.  The caches arrive by TMA into rings of stages
+// guarded by mbarriers: one box per page and 64-column slab when a block table scatters the pages, one
+// box per slab for the whole 128-token stage (4-D tensor map) when the pages are consecutive.
+//
+// TMEM columns: S0 [0,128) | S1 [128,256) | P [256,320) | O' [320, 320 + 192).  Because P does not
+// overlay S, an S buffer is free as soon as the softmax threads have pulled it into registers, so
+// Q K^T runs two steps ahead of the softmax; P has one buffer and is rewritten once the previous P V'
+// has retired (that MMA was issued a whole step earlier).
 //
 // Warp roles: warp 0 = TMA producer of the key ring, the last warp = TMA producer of the value ring
 // (keys are released right after S is computed, values only after O' is updated, so the two rings run
-// at different distances ahead), warp 1 = TMEM owner + MMA issuer, the 16 warps in between = softmax /
-// correction / epilogue, four threads per query row.  The running maximum is only raised when it grows by more than 8
-// (log2 domain), so O' is rescaled a handful of times per row instead of at every step; P stays
-// below 2^8.  Every mbarrier wait is bounded and falls through with PRECC_STATUS_TIMEOUT.
+// at different distances ahead), warp 1 = TMEM owner + Q K^T issuer, warp 2 = P V' issuer (an MMA costs
+// its issuing thread about a hundred cycles, so the two streams are issued by different threads), the
+// 8 warps in between = softmax / correction / epilogue.  The row maximum of a step is taken one step
+// ahead (in the middle of the previous step's exponentials) and the reference maximum is only raised
+// when it grows by more than 8 (log2 domain), so O' is rescaled a handful of times per row instead of
+// at every step; P stays below 2^8.  Every mbarrier wait is bounded and falls through with
+// PRECC_STATUS_TIMEOUT.
 #pragma once
 #include <type_traits>
 
@@ -35,8 +46,20 @@ struct PrefillTcParams {
   int n_q, n_kv, group;
   int tok_per_tile;            // 128 / group
   int k_stages, v_stages;      // depth of the key ring and of the value ring
+  int contig;                  // 1: no block table; the tensor maps fetch a whole 128-token stage per box
   float scale_log2, s_k, s_v;
+  unsigned long long* trace;   // PRECC_PF_TRACE builds only: [steps][16] clock stamps of block (0, 0)
 };
+
+// Timeline stamps for tuning (compiled in with -DPRECC_PF_TRACE; slot meanings at the call sites).
+#ifdef PRECC_PF_TRACE
+#define PTC_STAMP(p, j, slot)                                                                    \
+  do {                                                                                           \
+    if ((p).trace && blockIdx.x == 0 && blockIdx.y == 0 && (j) < 64) (p).trace[(j) * 16 + (slot)] = clock64(); \
+  } while (0)
+#else
+#define PTC_STAMP(p, j, slot) do { } while (0)
+#endif
 
 constexpr int PTC_PARTS_MAX = 4;
 constexpr int PTC_PARTS = 2;                         // softmax threads per query row
@@ -61,10 +84,18 @@ struct PrefillTcCfg {
   static constexpr int VSTAGE = VSLABS * SLAB_BYTES;          // {V_base slabs | L_V slab}
   static constexpr int K_PAGE_TX = PAGE * (HD + RK) * 2;      // bytes one page contributes to a key stage
   static constexpr int V_PAGE_TX = PAGE * VSLABS * 128;
-  static constexpr int TMEM_O = 2 * PTC_TOK;                  // O' starts after the two S buffers
+  static constexpr bool L_IN_MMA = RV > 0 && RV < 64;         // a spare column of the L_V slab carries the denominator
+  static constexpr int TMEM_P = 2 * PTC_TOK;                  // packed bf16 P (64 columns) after the two S buffers
+  static constexpr int TMEM_O = TMEM_P + PTC_TOK / 2;         // O' (at most 192 columns): 320 + 192 = 512
   __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 320 + 2 * PTC_PARTS_MAX * 512 + 1024; }
   static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 16 || RK == 32) && (RV == 0 || RV == 16 || RV == 32);
 };
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
 
 // layout_type field of a shared-memory matrix descriptor for rows of `row_bytes`
 __device__ __forceinline__ constexpr uint64_t umma_layout_for(int row_bytes) {
@@ -176,7 +207,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     mbar_init(s_full, 1); mbar_init(s_full + 8, 1);
     mbar_init(p_full, PTC_SOFTMAX_WARPS); mbar_init(p_full + 8, PTC_SOFTMAX_WARPS);
     mbar_init(pv_done, 1);
-    mbar_init(s_free, 1); mbar_init(s_free + 8, 1);
+    mbar_init(s_free, PTC_SOFTMAX_WARPS); mbar_init(s_free + 8, PTC_SOFTMAX_WARPS);
     mbar_init(q_ready, PTC_SOFTMAX_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     fence_async_smem();
@@ -200,10 +231,30 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       if (j >= NS) mbar_wait(emptyb + 8 * s, ((j / NS) - 1) & 1, p.status);
       // the last key stage doubles as the staging area of B_k until the query fold is done
       if (RK > 0 && is_k && j == KS - 1) mbar_wait(q_ready, 0, p.status);
+      if (lane == 0) PTC_STAMP(p, j, is_k ? 8 : 9);               // stage of step j free: loads go out now
       const int t0 = j * PTC_TOK;
       const int live = min(PTC_TOK / PAGE, (t_end - t0 + PAGE - 1) / PAGE);
       const uint32_t st = is_k ? kring_u32 + (uint32_t)s * C::KSTAGE : vring_u32 + (uint32_t)s * C::VSTAGE;
       const uint32_t full = fullb + 8 * s;
+      if (p.contig) {
+        // consecutive physical blocks: one box per 64-column slab covers all eight pages of the stage
+        // (4-D map [block][kv head][16][hd]); blocks past the cache end arrive as zeros
+        if (lane == 0) {
+          mbar_expect_tx(full, (PTC_TOK / PAGE) * (is_k ? C::K_PAGE_TX : C::V_PAGE_TX));
+          const int blk0 = p.first_block + j * (PTC_TOK / PAGE);
+          if (is_k) {
+#pragma unroll
+            for (int sl = 0; sl < C::SLABS; ++sl) tma_load_4d(st + sl * C::SLAB_BYTES, &map_k, sl * 64, 0, g, blk0, full);
+            if constexpr (RK > 0) tma_load_2d(st + C::KV_BYTES, &map_lk, 0, blk0 * PAGE, full);
+          } else {
+#pragma unroll
+            for (int sl = 0; sl < C::SLABS; ++sl) tma_load_4d(st + sl * C::SLAB_BYTES, &map_v, sl * 64, 0, g, blk0, full);
+            if constexpr (RV > 0) tma_load_2d(st + C::SLABS * C::SLAB_BYTES, &map_lv, 0, blk0 * PAGE, full);
+          }
+        }
+        __syncwarp();
+        continue;
+      }
       if (lane == 0) mbar_expect_tx(full, live * (is_k ? C::K_PAGE_TX : C::V_PAGE_TX));
       __syncwarp();
       if (lane < live) {
@@ -237,12 +288,13 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     mbar_wait(q_ready, 0, p.status);
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j % KS;
-      // S buffer j&1 still holds P of step j-2 until that step's P V' has been executed (one barrier
-      // per buffer, so this wait is never more than one phase behind)
+      // S buffer j&1 is free once the softmax threads have pulled the scores of step j-2 into registers
+      // (P has its own columns), so Q K^T runs up to two steps ahead of the softmax
       if (j >= 2) mbar_wait(s_free + 8 * (j & 1), ((j >> 1) - 1) & 1, p.status);
       mbar_wait(k_full + 8 * s, (j / KS) & 1, p.status);
       tc_fence_after();
       if (lane == 0) {
+        PTC_STAMP(p, j, 10);                     // keys of step j have landed (seen by the issuer)
         const uint64_t so = (uint64_t)((s * C::KSTAGE) >> 4);
         const uint32_t d = tmem_base + (j & 1) * PTC_TOK;
 #pragma unroll
@@ -256,6 +308,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         }
         umma_commit(k_empty + 8 * s);            // the key stage is free as soon as S is computed
         umma_commit(s_full + 8 * (j & 1));
+        PTC_STAMP(p, j, 2);                      // QK^T of step j issued
       }
       __syncwarp();
     }
@@ -267,10 +320,22 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       const int s = j % VS;
       const int n_live = min(PTC_TOK, t_end - j * PTC_TOK);       // tokens of this step that exist
       mbar_wait(v_full + 8 * s, (j / VS) & 1, p.status);
-      if (n_live < PTC_TOK && (n_live % PAGE) != 0) {
-        // the last page is only partly written: value rows past the end may hold anything, and
-        // 0 * NaN would poison the accumulators, so clear them before the MMA reads the page
-        const int r0 = n_live, r1 = (n_live + PAGE - 1) / PAGE * PAGE;
+      if (lane == 0) PTC_STAMP(p, j, 11);                          // values of step j have landed
+      if constexpr (C::L_IN_MMA) {
+        // column RV of the zero-padded L_V slab is set to one for the live tokens: the P V' MMA then
+        // accumulates the softmax denominator sum_t p_t in column HD + RV of O' (same bf16 p as the numerator)
+        unsigned char* slab = vring + (size_t)s * C::VSTAGE + C::SLABS * C::SLAB_BYTES;
+        constexpr int CH = (RV * 2) / 16;                          // 16-byte chunk holding column RV
+        for (int r = lane; r < PTC_TOK; r += 32)
+          *reinterpret_cast<__nv_bfloat16*>(slab + r * 128 + ((CH ^ (r & 7)) * 16)) = __float2bfloat16(r < n_live ? 1.f : 0.f);
+        fence_async_smem();
+        __syncwarp();
+      }
+      if (n_live < PTC_TOK && (p.contig || (n_live % PAGE) != 0)) {
+        // value rows past the end may hold anything (the rest of a partly written page; with whole-stage
+        // boxes also the pages behind it), and 0 * NaN would poison the accumulators: clear them
+        // before the MMA reads the stage
+        const int r0 = n_live, r1 = p.contig ? PTC_TOK : (n_live + PAGE - 1) / PAGE * PAGE;
         unsigned char* base = vring + (size_t)s * C::VSTAGE;
         for (int r = r0; r < r1; ++r)
           for (int sl = 0; sl < C::VSLABS; ++sl)
@@ -281,7 +346,8 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       mbar_wait(p_full + 8 * (j & 1), (j >> 1) & 1, p.status);
       tc_fence_after();
       if (lane == 0) {
-        const uint32_t a = tmem_base + (j & 1) * PTC_TOK;          // P overlays S (packed bf16, 2 per column)
+        PTC_STAMP(p, j, 0);                                        // P of step j seen by the PV issuer
+        const uint32_t a = tmem_base + C::TMEM_P;                  // packed bf16 P, 2 per column
         const uint64_t so = (uint64_t)((s * C::VSTAGE) >> 4);
         const uint32_t od = tmem_base + C::TMEM_O;
         if (n_live == PTC_TOK) {
@@ -292,8 +358,8 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           for (int ks = 0; ks < n_ks; ++ks) umma_bf16_ts(od, a + ks * 8, vd0 + so + (uint64_t)(ks * 128), id_o, (j | ks) ? 1u : 0u);
         }
         umma_commit(v_empty + 8 * s);
-        umma_commit(s_free + 8 * (j & 1));
         umma_commit(pv_done);
+        PTC_STAMP(p, j, 1);                                        // P V' of step j issued
       }
       __syncwarp();
     }
@@ -368,34 +434,65 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     __syncwarp();
     if (lane == 0) mbar_arrive(q_ready);
 
-    constexpr int OCH = (HD + RV) / 16;                           // 16-column chunks of O' that carry data
+    constexpr int OCH = (HD + RV) / 16 + (C::L_IN_MMA ? 1 : 0);   // 16-column chunks of O' that carry data (numerator, U, denominator)
     float m_used = NEG_BIG, l_sum = 0.f;
+    constexpr int NCH = COLS / 32;
+    // This thread's maximum (log2 domain) over its COLS scores of step j, read straight from TMEM.  It is
+    // taken one step ahead, in the middle of the previous step's exponentials, so that its latency chain
+    // (TMEM read, compare chain, exchange between the row's threads) is off the critical path.
+    auto local_max = [&](int j) -> float {
+      const int b = j & 1;
+      const int nvis = lim - (j * PTC_TOK + part * COLS) + 1;     // visible tokens among this thread's
+      const bool masked = j * PTC_TOK + PTC_TOK > full_vis;
+      float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        uint32_t x[32];
+        tmem_ld32(lane_addr + b * PTC_TOK + part * COLS + c * 32, x);
+        tmem_wait_ld();
+        if (masked) {
+#pragma unroll
+          for (int k = 0; k < 32; ++k)
+            if (c * 32 + k >= nvis) x[k] = 0xff800000u;          // -inf
+        }
+#pragma unroll
+        for (int k = 0; k < 32; k += 2)                            // two elements per step: the three-input maximum
+          tm[(k >> 1) & 3] = fmaxf(tm[(k >> 1) & 3], fmaxf(__uint_as_float(x[k]), __uint_as_float(x[k + 1])));
+      }
+      return fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])) * p.scale_log2;
+    };
+    // row maximum from the per-thread maxima of the row's NP threads
+    auto exchange_max = [&](int j, float own) -> float {
+      const int b = j & 1;
+      xch[(b * NP + part) * 128 + row] = own;
+      row_sync();
+      float t = own;
+#pragma unroll
+      for (int q2 = 0; q2 < NP; ++q2) t = fmaxf(t, xch[(b * NP + q2) * 128 + row]);
+      return t;
+    };
+    float tmax = NEG_BIG;                                         // row maximum of the step about to run
     // One step of the online softmax for this thread's COLS scores.  MASKED is a compile-time flag so
     // that the common step (far from the causal edge) carries no per-element compare/select.
     auto step = [&](int j, auto masked_tag) {
       constexpr bool MASKED = decltype(masked_tag)::value;
       const int b = j & 1;
-      const int t0 = j * PTC_TOK + part * COLS;
-      constexpr int NCH = COLS / 32;
       uint32_t sv[NCH][32];
 #pragma unroll
       for (int c = 0; c < NCH; ++c) tmem_ld32(lane_addr + b * PTC_TOK + part * COLS + c * 32, sv[c]);
       tmem_wait_ld();
-      // row maximum of the raw scores (the scale is positive, so it commutes with max)
-      const int nvis = lim - t0 + 1;                              // visible tokens among this thread's
-      float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (tid == 0) PTC_STAMP(p, j, 7);                            // scores in registers
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_free + 8 * b);                  // the S buffer may be overwritten
+      if constexpr (MASKED) {
+        const int nvis = lim - (j * PTC_TOK + part * COLS) + 1;
 #pragma unroll
-      for (int c = 0; c < NCH; ++c)
+        for (int c = 0; c < NCH; ++c)
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          if (MASKED && c * 32 + k >= nvis) sv[c][k] = 0xff800000u;   // -inf
-          tm[k & 3] = fmaxf(tm[k & 3], __uint_as_float(sv[c][k]));
-        }
-      float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])) * p.scale_log2;
-      xch[(b * NP + part) * 128 + row] = tmax;
-      row_sync();
-#pragma unroll
-      for (int q2 = 0; q2 < NP; ++q2) tmax = fmaxf(tmax, xch[(b * NP + q2) * 128 + row]);
+          for (int k = 0; k < 32; ++k)
+            if (c * 32 + k >= nvis) sv[c][k] = 0xff800000u;      // -inf: weight zero
+      }
       float m_new = m_used;
       if (tmax > m_used + PTC_RAISE) m_new = tmax;                 // all threads of the row decide alike
       const bool raise = m_new != m_used;
@@ -418,34 +515,53 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         l_sum *= alpha;
         m_used = m_new;
       }
+      if (tid == 0) PTC_STAMP(p, j, 5);                            // reference maximum settled
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
       const float neg_m = -m_used;
+      uint32_t pk[NCH][16];
+      float next_own = NEG_BIG;
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
-        uint32_t pk[16];
 #pragma unroll
         for (int k = 0; k < 32; k += 2) {
           const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c][k]), p.scale_log2, neg_m));
           const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c][k + 1]), p.scale_log2, neg_m));
-          ls[(k >> 1) & 3] += p0 + p1;
-          pk[k / 2] = pack_bf16(p0, p1);
+          if constexpr (!C::L_IN_MMA) ls[(k >> 1) & 3] += p0 + p1;
+          pk[c][k / 2] = pack_bf16(p0, p1);
         }
-        tmem_st16(lane_addr + b * PTC_TOK + part * (COLS / 2) + c * 16, pk);
+        if (c == 0 && j + 1 < n_tiles) {
+          if (tid == 0) PTC_STAMP(p, j, 12);                       // first half of the exponentials done
+          // between the two halves of the exponentials: the next step's scores are normally there already
+          mbar_wait(s_full + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, p.status);
+          tc_fence_after();
+          next_own = local_max(j + 1);
+          if (tid == 0) PTC_STAMP(p, j, 13);                       // next step's local maximum taken
+        }
       }
       l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      // P has one buffer: it may be overwritten once the previous step's P V' has read it (that MMA was
+      // issued a whole softmax step ago, so this wait normally falls through)
+      if (tid == 0) PTC_STAMP(p, j, 14);                           // all exponentials done
+      if (j > 0) { mbar_wait(pv_done, (j - 1) & 1, p.status); tc_fence_after(); }
+      if (tid == 0) PTC_STAMP(p, j, 15);                           // previous P V' has retired
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) tmem_st16(lane_addr + C::TMEM_P + part * (COLS / 2) + c * 16, pk[c]);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(p_full + 8 * b);
-      // observe every phase of pv_done (a parity wait must never lag two phases behind); by now the
-      // previous step's MMAs have normally retired, so this does not stall the pipeline
-      if (j > 0) mbar_wait(pv_done, (j - 1) & 1, p.status);
+      if (tid == 0) PTC_STAMP(p, j, 6);                            // P published
+      if (j + 1 < n_tiles) tmax = exchange_max(j + 1, next_own);
     };
+    if (tid == 0) PTC_STAMP(p, 0, 3);
+    mbar_wait(s_full, 0, p.status);
+    tc_fence_after();
+    tmax = exchange_max(0, local_max(0));
     for (int j = 0; j < n_tiles; ++j) {
-      mbar_wait(s_full + 8 * (j & 1), (j >> 1) & 1, p.status);
-      tc_fence_after();
+      if (tid == 0) PTC_STAMP(p, j, 4);                            // step j starts (its scores were awaited a step earlier)
       if (j * PTC_TOK + PTC_TOK > full_vis) step(j, std::true_type{});     // only the last few steps reach the causal edge
       else step(j, std::false_type{});
+      if (tid == 0) PTC_STAMP(p, j + 1, 3);
     }
     // ---- epilogue: out = (O + s_v U B_v) / l ; the threads of a row share its output columns
     mbar_wait(pv_done, (n_tiles - 1) & 1, p.status);
@@ -461,8 +577,15 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     xch[part * 128 + row] = l_sum;
     asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
     float l_tot = 0.f;
+    if constexpr (C::L_IN_MMA) {
+      uint32_t lv16[16];
+      tmem_ld16(lane_addr + C::TMEM_O + HD + (RV / 16) * 16, lv16);   // RV is a multiple of 16: column HD + RV leads its chunk
+      tmem_wait_ld();
+      l_tot = __uint_as_float(lv16[0]);
+    } else {
 #pragma unroll
-    for (int q2 = 0; q2 < NP; ++q2) l_tot += xch[q2 * 128 + row];
+      for (int q2 = 0; q2 < NP; ++q2) l_tot += xch[q2 * 128 + row];
+    }
     const float inv = 1.f / l_tot;
     float u[RV > 0 ? RV : 1];
     if constexpr (RV > 0) {
