@@ -282,6 +282,32 @@ int32_t precc_lr_attend_prefill_rope(precc_ctx* ctx, const precc_layer_desc* des
                                      const void* B_k, const void* B_v, const precc_rope* rope,
                                      const precc_cache* cache, void* out, void* stream);
 
+/* ------------------------------------------------------------- context-sharded decode (no paper counterpart)
+ * When the tokens of a request are spread over several GPUs (each holds base and LR rows of a contiguous
+ * token range in its own caches), softmax attention over the union is the split-KV merge taken once more
+ * across GPUs.  Each shard calls precc_lr_attend_decode_partial over its LOCAL tokens; the records of all
+ * shards are gathered (e.g. an NCCL all-gather) into [n_shards][B][n_kv_heads][R] floats, R =
+ * precc_partial_record_floats(desc); precc_combine_partials merges them in shard order and applies the
+ * value-side epilogue.  The result equals precc_lr_attend_decode over the concatenated context up to fp32
+ * summation order.  Position-free path only.
+ *   record = [ m[8] | l[8] | O'[group][head_dim + rank_v] ] fp32: running maximum (log2 domain), softmax
+ *            denominator and un-normalised output (with the rank_v LR-V coordinates appended) per query head
+ *   ctx_len [B] local token counts; 0 is allowed (the shard holds nothing of that request) and yields the
+ *            neutral record; max_ctx >= 1 bounds them
+ *   agent ids, q, B_k, block tables, workspace: as for precc_lr_attend_decode (B_v is not needed here) */
+size_t precc_partial_record_floats(const precc_layer_desc* desc);
+int32_t precc_lr_attend_decode_partial(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,
+                                       const int32_t* agent_id, const int32_t* ctx_len,
+                                       const int32_t* block_table, int32_t table_stride,
+                                       const int32_t* first_block, int32_t max_ctx, const void* B_k,
+                                       const precc_cache* cache, float* records, void* workspace,
+                                       size_t workspace_bytes, void* stream);
+/*   records  device fp32 [n_shards][B][n_kv_heads][R], 1 <= n_shards <= 64;  out [B][n_q_heads][head_dim].
+ * A request with no token on any shard gets zeros. */
+int32_t precc_combine_partials(precc_ctx* ctx, const precc_layer_desc* desc, const float* records,
+                               int32_t n_shards, int32_t B, const int32_t* agent_id, const void* B_v,
+                               void* out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,6 +23,7 @@ EXPORTS = [
     "precc_decode_workspace_bytes", "precc_workspace_init", "precc_lr_attend_decode",
     "precc_lr_attend_decode_static", "precc_lr_attend_prefill",
     "precc_rebase_project_rope", "precc_turn_project_rope", "precc_lr_attend_decode_rope", "precc_lr_attend_prefill_rope",
+    "precc_partial_record_floats", "precc_lr_attend_decode_partial", "precc_combine_partials",
 ]
 
 
@@ -87,6 +88,11 @@ def load_library() -> C.CDLL:
                                                 C.POINTER(CacheDesc), vp, vp, sz, vp]
     lib.precc_lr_attend_prefill_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp, rp,
                                                  C.POINTER(CacheDesc), vp, vp]
+    lib.precc_partial_record_floats.argtypes = [C.POINTER(LayerDesc)]
+    lib.precc_partial_record_floats.restype = sz
+    lib.precc_lr_attend_decode_partial.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, i32, vp, i32, vp,
+                                                   C.POINTER(CacheDesc), vp, vp, sz, vp]
+    lib.precc_combine_partials.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, vp, vp, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is C.c_int:  # default restype: the int32 status code
@@ -292,6 +298,28 @@ class Precc:
         self._check(self.lib.precc_lr_attend_prefill_rope(
             self.h, C.byref(desc), _ptr(q), q.shape[0], agent, ctx_len, _ptr(block_table), stride, first_block,
             _ptr(B_k), _ptr(B_v), C.byref(rd), C.byref(cd), _ptr(out), _stream()), "precc_lr_attend_prefill_rope")
+
+    # ------------------------------------------------------------------ context-sharded decode
+    def partial_record_floats(self, desc: LayerDesc) -> int:
+        return int(self.lib.precc_partial_record_floats(C.byref(desc)))
+
+    def lr_attend_decode_partial(self, desc: LayerDesc, q: torch.Tensor, agent_id: torch.Tensor, ctx_len: torch.Tensor,
+                                 max_ctx: int, B_k, cache: Cache, records: torch.Tensor, workspace: torch.Tensor,
+                                 block_table: Optional[torch.Tensor] = None, first_block: Optional[torch.Tensor] = None):
+        """This shard's split-KV record per (request, kv head) over its local tokens: records fp32 [B][n_kv][R]."""
+        if records.dtype != torch.float32:
+            raise PreccError("records must be fp32")
+        cd = cache.desc()
+        stride = block_table.shape[1] if block_table is not None else 0
+        self._check(self.lib.precc_lr_attend_decode_partial(
+            self.h, C.byref(desc), _ptr(q), q.shape[0], _ptr(agent_id), _ptr(ctx_len), _ptr(block_table), stride,
+            _ptr(first_block), max_ctx, _ptr(B_k), C.byref(cd), _ptr(records), _ptr(workspace), workspace.numel(), _stream()),
+            "precc_lr_attend_decode_partial")
+
+    def combine_partials(self, desc: LayerDesc, records: torch.Tensor, agent_id: torch.Tensor, B_v, out: torch.Tensor):
+        """records fp32 [n_shards][B][n_kv][R] (as an all-gather leaves them) -> out [B][n_q][hd]."""
+        self._check(self.lib.precc_combine_partials(self.h, C.byref(desc), _ptr(records), records.shape[0], out.shape[0],
+                                                    _ptr(agent_id), _ptr(B_v), _ptr(out), _stream()), "precc_combine_partials")
 
     def decode_workspace(self, desc: LayerDesc, max_batch: int, max_ctx: int) -> torch.Tensor:
         n = self.lib.precc_decode_workspace_bytes(C.byref(desc), max_batch, max_ctx, self.sm_count)

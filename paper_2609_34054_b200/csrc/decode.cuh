@@ -49,6 +49,7 @@ struct DecodeParams {
   const __nv_bfloat16* B_v;
   float* part;        // ticket kernel: [B][n_kv][max_splits][PART_STRIDE]
   int32_t* tickets;   // ticket kernel: [B][n_kv], zero between calls
+  float* raw;         // partial-output mode (ticket kernel): [B][n_kv][PART_STRIDE] records instead of `out`, or null
   uint32_t* status;
   unsigned long long* trace;   // optional [blocks][16] phase timestamps (ns), or null
   const float4* rope;          // rotary variant: [max_pos][hd/4] of (cos c, sin c, cos c+1, sin c+1), c even
@@ -560,7 +561,13 @@ lr_attend_decode_kernel(const DecodeParams p) {
   __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
   if (ctx < 1 || agent_raw < -1 || agent_raw >= p.n_agents) {
     if (split == 0) {
-      for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
+      if (p.raw) {
+        // an empty shard (or a rejected request) contributes the neutral record: m = -big, l = 0, O' = 0
+        float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
+        for (int i = threadIdx.x; i < C::PART_STRIDE; i += NT) rec[i] = i < 8 ? NEG_BIG : 0.f;
+      } else {
+        for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
+      }
       if (threadIdx.x == 0 && ctx >= 1) atomicOr(p.status, StatusBits::BAD_INDEX);
     }
     return;
@@ -591,6 +598,7 @@ lr_attend_decode_kernel(const DecodeParams p) {
   };
   float* fo = res + 16;                                 // final O' [G][OW]
   __shared__ float fin_l[8];
+  __shared__ float fin_m[8];
   if (n_splits > 1) {
     float* rec = p.part + (((size_t)b * p.n_kv + g) * p.max_splits + split) * C::PART_STRIDE;
     for (int i = threadIdx.x; i < rec_f / 4; i += NT)
@@ -614,7 +622,7 @@ lr_attend_decode_kernel(const DecodeParams p) {
     const float* base = p.part + (((size_t)b * p.n_kv + g) * p.max_splits) * C::PART_STRIDE;
     float* recs = res + 16 + 8 * OW;                    // [n_splits][rec_f] (staged) or [n_splits][16]
     const bool staged = (16 + 8 * OW + n_splits * rec_f + DEC_WARPS * n_el) * 4 + bv_bytes <= region;
-    stage_bv();
+    if (!p.raw) stage_bv();
     if (staged) {
       const int cpr = rec_f / 4;                        // 16-byte chunks per record
       for (int c = threadIdx.x; c < n_splits * cpr; c += NT) {
@@ -644,7 +652,7 @@ lr_attend_decode_kernel(const DecodeParams p) {
       }
 #pragma unroll
       for (int d = 16; d >= 1; d >>= 1) L += __shfl_xor_sync(0xffffffffu, L, d);   // fixed tree: deterministic
-      if (lane == 0) fin_l[h] = L;
+      if (lane == 0) { fin_l[h] = L; fin_m[h] = M; }
     }
     __syncthreads();
     mark(9);
@@ -679,13 +687,27 @@ lr_attend_decode_kernel(const DecodeParams p) {
     for (int e = threadIdx.x; e < n_el; e += NT)
       fo[e] = ((wsum[e] + wsum[n_el + e]) + wsum[2 * n_el + e]) + wsum[3 * n_el + e];
   } else {
-    stage_bv();
+    if (!p.raw) stage_bv();
     cp_async_commit();
-    if (threadIdx.x < 8) fin_l[threadIdx.x] = res[8 + threadIdx.x];
+    if (threadIdx.x < 8) { fin_l[threadIdx.x] = res[8 + threadIdx.x]; fin_m[threadIdx.x] = res[threadIdx.x]; }
     cp_async_wait<0>();
   }
   __syncthreads();
   mark(10);
+  if (p.raw) {
+    // partial-output mode: the merged record of this (request, kv head) over the LOCAL tokens, not
+    // normalised and without the value-side epilogue; a later combine step merges such records
+    float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
+    for (int i = threadIdx.x; i < C::PART_STRIDE; i += NT) {
+      float v = 0.f;
+      if (i < 8) v = i < G ? fin_m[i] : NEG_BIG;
+      else if (i < 16) v = i - 8 < G ? fin_l[i - 8] : 0.f;
+      else if (i - 16 < n_el) v = fo[i - 16];
+      rec[i] = v;
+    }
+    mark(7);
+    return;
+  }
   const __nv_bfloat16* bvs = reinterpret_cast<const __nv_bfloat16*>(bv_s);
   for (int e = threadIdx.x; e < G * HD; e += NT) {
     const int h = e / HD, c = e % HD;

@@ -11,6 +11,7 @@
 
 #include "../../include/precc.h"
 #include "decode.cuh"
+#include "combine.cuh"
 #include "gemm_tc.cuh"
 #include "proj_small.cuh"
 #include "prefill.cuh"
@@ -316,6 +317,7 @@ struct DecodeArgs {
   const int32_t* block_table; int table_stride; const int32_t* first_block; int max_ctx;
   const void* B_k; const void* B_v; const precc_cache* cache; void* out; void* ws; size_t ws_bytes; cudaStream_t stream;
   const float* rope = nullptr; int max_pos = 0;      // rotary variant when rope != null
+  float* raw = nullptr;                              // partial-output mode: records instead of `out`
 };
 
 template <int HD, int RK, int RV, bool ROPE = false>
@@ -356,6 +358,7 @@ struct DecodeRunT {
     const precc_layer_desc* d = a.d;
     constexpr int extra = ROPE ? DecodeCfg<HD, RK, RV>::BK_BYTES + 128 : 0;
     DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);
+    if (a.raw) pl.cluster = 0;                        // records are written by the ticket kernel
     if (pl.cluster && !(pl.warps == 8 ? cluster_fits<8>(ctx, pl, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, pl, a.B * d->n_kv_heads))) pl.cluster = 0;
     if (!pl.cluster) {
       pl = plan_ticket<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);
@@ -371,6 +374,7 @@ struct DecodeRunT {
     const size_t tickets = ((size_t)a.B * d->n_kv_heads * 4 + 255) / 256 * 256;
     p.tickets = (int32_t*)a.ws;
     p.part = a.ws ? (float*)((char*)a.ws + tickets) : nullptr;
+    p.raw = a.raw;
     p.status = ctx->status;
     p.trace = (ctx->trace && (size_t)pl.max_splits * d->n_kv_heads * a.B <= ctx->trace_blocks) ? ctx->trace : nullptr;
     p.n_blocks = a.cache->n_blocks; p.table_stride = a.table_stride;
@@ -530,6 +534,31 @@ struct PrefillRunRope {
   static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
     if constexpr (RK > 0) return PrefillRun<HD, RK, RV>::template run_simple<true>(ctx, a);
     else return PrefillRun<HD, RK, RV>::run(ctx, a);
+  }
+};
+
+struct CombineArgs {
+  const precc_layer_desc* d; const float* recs; int n_shards; int B; const int32_t* agent_id; const void* B_v; void* out;
+  cudaStream_t stream;
+};
+template <int HD, int RK, int RV>
+struct CombineRun {
+  static int32_t run(precc_ctx* ctx, const CombineArgs& a) {
+    CombineParams p;
+    p.recs = a.recs; p.agent_id = a.agent_id; p.B_v = (const __nv_bfloat16*)a.B_v; p.out = (__nv_bfloat16*)a.out;
+    p.status = ctx->status; p.n_shards = a.n_shards; p.B = a.B;
+    p.n_q = a.d->n_q_heads; p.n_kv = a.d->n_kv_heads; p.group = a.d->n_q_heads / a.d->n_kv_heads; p.n_agents = a.d->n_agents;
+    p.s_v = a.d->lora_scale_v;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.d->n_kv_heads, a.B);
+    cfg.blockDim = dim3(COMBINE_THREADS);
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_combine_kernel<HD, RV>, p));
+    return PRECC_OK;
   }
 };
 
@@ -768,7 +797,7 @@ static int32_t decode_entry(precc_ctx* ctx, const precc_layer_desc* desc, const 
                             const int32_t* ctx_len, const int32_t* block_table, int32_t table_stride,
                             const int32_t* first_block, int32_t max_ctx, const void* B_k, const void* B_v,
                             const precc_cache* cache, void* out, void* workspace, size_t workspace_bytes, void* stream,
-                            const float* rope, int32_t max_pos) {
+                            const float* rope, int32_t max_pos, float* raw = nullptr) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (B < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "B < 0");
@@ -776,7 +805,7 @@ static int32_t decode_entry(precc_ctx* ctx, const precc_layer_desc* desc, const 
   rc = check_cache(ctx, desc, cache, true, true);
   if (rc) return rc;
   if (!q || !out || !agent_id || !ctx_len) return fail(ctx, PRECC_ERR_INVALID_ARG, "q / out / agent_id / ctx_len is null");
-  if ((desc->rank_k > 0 && !B_k) || (desc->rank_v > 0 && !B_v)) return fail(ctx, PRECC_ERR_INVALID_ARG, "B_k / B_v is null");
+  if ((desc->rank_k > 0 && !B_k) || (desc->rank_v > 0 && !B_v && !raw)) return fail(ctx, PRECC_ERR_INVALID_ARG, "B_k / B_v is null");
   if (!aligned16(q) || !aligned16(out) || !aligned16(B_k) || !aligned16(B_v) || !aligned16(workspace))
     return fail(ctx, PRECC_ERR_MISALIGNED, "q / out / B_k / B_v / workspace not 16-byte aligned");
   if (max_ctx < 1) return fail(ctx, PRECC_ERR_INVALID_ARG, "max_ctx < 1");
@@ -789,6 +818,7 @@ static int32_t decode_entry(precc_ctx* ctx, const precc_layer_desc* desc, const 
   }
   DecodeArgs a{desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, B_v, cache, out,
                workspace, workspace_bytes, (cudaStream_t)stream};
+  a.raw = raw;
   if (!rope) return dispatch_shape<DecodeRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
   if (!aligned16(rope)) return fail(ctx, PRECC_ERR_MISALIGNED, "rope table not 16-byte aligned");
   if (max_pos < max_ctx) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table covers %d positions, max_ctx is %d", max_pos, max_ctx);
@@ -813,6 +843,38 @@ int32_t precc_lr_attend_decode_rope(precc_ctx* ctx, const precc_layer_desc* desc
   if (!rope || !rope->table) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table is null");
   return decode_entry(ctx, desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, B_v, cache, out,
                       workspace, workspace_bytes, stream, rope->table, rope->max_pos);
+}
+
+size_t precc_partial_record_floats(const precc_layer_desc* desc) {
+  if (!desc) return 0;
+  return (size_t)16 + 8 * (size_t)(desc->head_dim + desc->rank_v);
+}
+
+int32_t precc_lr_attend_decode_partial(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,
+                                       const int32_t* agent_id, const int32_t* ctx_len, const int32_t* block_table,
+                                       int32_t table_stride, const int32_t* first_block, int32_t max_ctx, const void* B_k,
+                                       const precc_cache* cache, float* records, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!records || !aligned16(records)) return fail(ctx, PRECC_ERR_INVALID_ARG, "records is null or not 16-byte aligned");
+  // `out` is not written in this mode (the records pointer stands in for it); B_v is not needed: the
+  // value-side epilogue belongs to the combine step
+  return decode_entry(ctx, desc, q, B, agent_id, ctx_len, block_table, table_stride, first_block, max_ctx, B_k, nullptr, cache,
+                      records, workspace, workspace_bytes, stream, nullptr, 0, records);
+}
+
+int32_t precc_combine_partials(precc_ctx* ctx, const precc_layer_desc* desc, const float* records, int32_t n_shards, int32_t B,
+                               const int32_t* agent_id, const void* B_v, void* out, void* stream) {
+  int32_t rc = check_desc(ctx, desc);
+  if (rc) return rc;
+  if (B < 0 || n_shards < 1 || n_shards > 64) return fail(ctx, PRECC_ERR_INVALID_ARG, "B < 0 or n_shards outside [1, 64]");
+  if (B == 0) return PRECC_OK;
+  if (!records || !agent_id || !out) return fail(ctx, PRECC_ERR_INVALID_ARG, "records / agent_id / out is null");
+  if (desc->rank_v > 0 && !B_v) return fail(ctx, PRECC_ERR_INVALID_ARG, "B_v is null");
+  if (!aligned16(records) || !aligned16(out) || !aligned16(B_v)) return fail(ctx, PRECC_ERR_MISALIGNED, "records / out / B_v not 16-byte aligned");
+  if (B > 65535) return fail(ctx, PRECC_ERR_UNSUPPORTED, "B > 65535");
+  CombineArgs a{desc, records, n_shards, B, agent_id, B_v, out, (cudaStream_t)stream};
+  return dispatch_shape<CombineRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
 }
 
 int32_t precc_lr_attend_decode_static(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,

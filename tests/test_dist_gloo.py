@@ -61,3 +61,50 @@ def test_reference_arm_is_silent_on_nonzero_ranks(monkeypatch, capsys):
     monkeypatch.setenv("RANK", "1")
     assert bench.run_reference(argparse.Namespace(gpus=2, steps=1, warmup=0)) == 0
     assert capsys.readouterr().out == ""
+
+
+# ---------------------------------------------------------------- context-sharded decode: host logic
+
+def test_shard_ranges_cover_every_token_once():
+    sys.path.insert(0, ROOT)
+    from paper_2609_34054_b200.sharded import shard_ranges
+    ctx = [0, 1, 15, 16, 17, 100, 4097, 32768]
+    for world in (1, 2, 3, 4, 8):
+        ranges = shard_ranges(ctx, world)
+        assert len(ranges) == world and all(len(r) == len(ctx) for r in ranges)
+        for i, c in enumerate(ctx):
+            pos = 0
+            for r in range(world):
+                s, e = ranges[r][i]
+                assert s == pos and e >= s and (s % 16 == 0 or s == c)      # contiguous, rank order, page-aligned starts
+                pos = e
+            assert pos == c                                                 # exactly [0, ctx)
+        sizes = [ranges[r][-1][1] - ranges[r][-1][0] for r in range(world)]
+        assert max(sizes) - min(sizes) <= 16                                # balanced to within a page
+
+
+def _gather_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2609_34054_b200.sharded import gather_records
+    local = torch.full((3, 2, 24), float(rank + 1), dtype=torch.float32)
+    local[0, 0, 0] = 100.0 + rank
+    got = gather_records(local)
+    reuse = torch.empty((world, 3, 2, 24), dtype=torch.float32)
+    again = gather_records(local, None, reuse)
+    out[rank] = (tuple(got.shape), [float(got[s, 1, 1, 5]) for s in range(world)], [float(got[s, 0, 0, 0]) for s in range(world)],
+                 again.data_ptr() == reuse.data_ptr() and bool(torch.equal(again, got)))
+    dist.destroy_process_group()
+
+
+def test_gather_records_layout_world_size_2():
+    world = 2
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_gather_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+        res = dict(out)
+    for r in range(world):
+        shape, vals, tags, reused = res[r]
+        assert shape == (2, 3, 2, 24) and vals == [1.0, 2.0] and tags == [100.0, 101.0] and reused   # slot s holds rank s's records
