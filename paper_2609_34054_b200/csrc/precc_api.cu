@@ -172,7 +172,8 @@ int32_t launch_small(precc_ctx* ctx, const void* X, int M, int K, const void* Wt
   while (cs > 1 && (K / cs < 512 || K % (PS_BK * cs) != 0)) cs >>= 1;
   const int k_slice = K / cs;
   const int steps = k_slice / PS_BK;
-  const int mt = M <= 16 ? 1 : (M <= 32 ? 2 : 4);
+  int mt = M <= 16 ? 1 : (M <= 32 ? 2 : 4);
+  if (gp.rope && ps_cols(mt) % gp.hd != 0) mt = 2;     // a head's two halves must sit in one block tile (128 columns)
   const int smem = ps_smem_bytes(mt);
   if (steps < 1 || smem > ctx->max_smem_optin) return -1;                // caller falls back to the tiled kernel
   gp.M = M; gp.N_out = n_out; gp.K = K; gp.status = ctx->status;
@@ -205,7 +206,7 @@ int32_t launch_small(precc_ctx* ctx, const void* X, int M, int K, const void* Wt
 }
 
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
-  if (M <= PS_MAX_M && !gp.rope && !ctx->force_tiled_gemm) {
+  if (M <= PS_MAX_M && !ctx->force_tiled_gemm) {
     const int32_t rc = launch_small(ctx, X, M, K, Wt, n_out, gp, stream);
     if (rc >= 0) return rc;
   }

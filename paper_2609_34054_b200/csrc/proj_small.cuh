@@ -16,6 +16,8 @@
 //   reduce = partial tiles go to shared memory; after a cluster barrier each block sums one slice of the
 //            columns over its peers through distributed shared memory (rank order: deterministic) and
 //            scatters bf16 pieces into the paged caches.  No global scratch, no atomics.
+// Rotary keys (GemmParams::rope): the reducing thread of the lower half of a head also gathers the partner
+// piece hd/2 columns further and writes both rotated; the block tile therefore holds whole heads.
 // The K split depends on K alone, so an output value does not depend on which entry point, which other
 // columns or how many other rows were in the call.
 #pragma once
@@ -130,11 +132,8 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   //      all peers' values requested at once, added in rank order
   const int pieces_per_row = COLS / 8 / CS;             // CS in {1,2,4,8}
   const uint32_t part_u32 = smem_u32(part);
-  for (int it = threadIdx.x; it < p.M * pieces_per_row; it += PS_THREADS) {
-    const int row = it / pieces_per_row, pc = it % pieces_per_row;
-    const int col = (rank * pieces_per_row + pc) * 8;
-    const int gc = group * COLS + col;
-    if (gc >= p.N_out) continue;
+  // eight columns [col, col+8) of one row, summed over the cluster's partial tiles
+  auto gather = [&](int row, int col, float (&v8)[8]) {
     float4 x0[8], x1[8];
 #pragma unroll
     for (uint32_t s = 0; s < 8; ++s) {
@@ -147,14 +146,46 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         x0[s] = make_float4(0.f, 0.f, 0.f, 0.f); x1[s] = x0[s];
       }
     }
-    float v8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v8[k] = 0.f;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
       v8[0] += x0[s].x; v8[1] += x0[s].y; v8[2] += x0[s].z; v8[3] += x0[s].w;
       v8[4] += x1[s].x; v8[5] += x1[s].y; v8[6] += x1[s].z; v8[7] += x1[s].w;
     }
+  };
+  const int kw = (p.rope && p.mode != 0) ? p.n_kv * p.hd : 0;   // width of the key columns that get rotated
+  for (int it = threadIdx.x; it < p.M * pieces_per_row; it += PS_THREADS) {
+    const int row = it / pieces_per_row, pc = it % pieces_per_row;
+    const int col = (rank * pieces_per_row + pc) * 8;
+    const int gc = group * COLS + col;
+    if (gc >= p.N_out) continue;
+    if (gc < kw && (gc % p.hd) >= p.hd / 2) continue;   // upper half of a rotated head: written with its lower partner
     long long slot = p.slot_mapping ? (long long)p.slot_mapping[row] : p.start_slot + row;
     if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); continue; }
+    float v8[8];
+    gather(row, col, v8);
+    if (gc < kw) {
+      // rotary keys: columns (c, c + hd/2) of a head turn by the row's position; the block tile holds whole
+      // heads (COLS % hd == 0), so the partner piece sits hd/2 columns further in the same tiles
+      long long pos = p.positions ? (long long)p.positions[row] : p.start_pos + row;
+      if (pos < 0 || pos >= p.max_pos) { atomicOr(p.status, StatusBits::BAD_INDEX); continue; }
+      float h8[8];
+      gather(row, col + p.hd / 2, h8);
+      const float4* cs = p.rope + pos * (p.hd / 4) + (gc % p.hd) / 2;
+      float lo[8], hi[8];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float4 t4 = __ldg(cs + k);                // (cos c, sin c, cos c+1, sin c+1)
+        lo[2 * k] = v8[2 * k] * t4.x - h8[2 * k] * t4.y;
+        lo[2 * k + 1] = v8[2 * k + 1] * t4.z - h8[2 * k + 1] * t4.w;
+        hi[2 * k] = h8[2 * k] * t4.x + v8[2 * k] * t4.y;
+        hi[2 * k + 1] = h8[2 * k + 1] * t4.z + v8[2 * k + 1] * t4.w;
+      }
+      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, lo);
+      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc + p.hd / 2, hi);
+      continue;
+    }
     store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8);
   }
   // nobody leaves while a peer may still read its partial tile

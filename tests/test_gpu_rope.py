@@ -44,7 +44,8 @@ def test_rope_table_matches_the_definition():
     np.testing.assert_allclose(t[..., 1], sin, atol=1e-7)
 
 
-@pytest.mark.parametrize("hd,n_kv,M", [(64, 2, 300), (128, 1, 130), (128, 4, 517)])
+@pytest.mark.parametrize("hd,n_kv,M", [(64, 2, 300), (128, 1, 130), (128, 4, 517),
+                                      (64, 2, 1), (128, 2, 7), (128, 1, 40), (64, 4, 64), (128, 2, 16)])   # the last five: few-row kernel
 def test_projection_rotates_keys_only(px, hd, n_kv, M):
     geo = I.Geometry(d_model=256, n_q=2 * n_kv, n_kv=n_kv, hd=hd, n_agents=2, rank_k=16, rank_v=16, alpha=32.0)
     nb = (M + 15) // 16 + 2
