@@ -764,7 +764,12 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
   if (ctx < 1 || agent_raw < -1 || agent_raw >= p.n_agents) {   // the same decision in every block of the cluster
     if (rank == 0) {
-      for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
+      if (p.raw) {
+        float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;   // neutral record: m = -big, l = 0, O' = 0
+        for (int i = threadIdx.x; i < C::PART_STRIDE; i += NT) rec[i] = i < 8 ? NEG_BIG : 0.f;
+      } else {
+        for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
+      }
       if (threadIdx.x == 0 && ctx >= 1) atomicOr(p.status, StatusBits::BAD_INDEX);
     }
     return;
@@ -782,7 +787,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
 #pragma unroll
     for (int k = 0; k < BV_PER_THREAD; ++k) {
       const int i = threadIdx.x + k * NT;
-      bv_pre[k] = (i < RV * cols_) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);
+      bv_pre[k] = (i < RV * cols_ && !p.raw) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);   // partial-output mode has no B_v
     }
   }
   if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
@@ -802,6 +807,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   }
   mark(6);
   cluster_sync_all();                                   // every block's result is complete and visible
+  __shared__ float fin_m[8];
   // One pass over distributed shared memory: a thread owns one merged element (for every h < G my
   // `cols` base columns and all r_v LR-V coordinates, plus the denominators) and reads the peers'
   // running maxima and values with all loads in flight at once; peers are added in rank order.
@@ -825,10 +831,30 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
 #pragma unroll
     for (int r = 0; r < DEC_MAX_CLUSTER; ++r) v += xr[r] * fast_exp2(mr[r] - M);
     mine[is_l ? 8 * (HD + RV) + h : e] = v;
+    if (is_l) fin_m[h] = M;
   }
   __syncthreads();
   mark(10);
   const float* fin_l = mine + 8 * (HD + RV);
+  if (p.raw) {
+    // partial-output mode: this block's column slice of the merged, un-normalised record; block 0 adds the
+    // LR-V coordinates, the denominators and the maxima
+    float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
+    for (int e = threadIdx.x; e < G * cols; e += NT) rec[16 + (e / cols) * OW + c0 + (e % cols)] = mine[(e / cols) * sw + (e % cols)];
+    if (rank == 0) {
+      if constexpr (RV > 0) {
+        for (int e = threadIdx.x; e < G * RV; e += NT) rec[16 + (e / RV) * OW + HD + (e % RV)] = mine[(e / RV) * sw + cols + (e % RV)];
+      }
+      for (int e = G * OW + threadIdx.x; e < 8 * OW; e += NT) rec[16 + e] = 0.f;   // unused query-head slots: defined
+      if (threadIdx.x < 8) {
+        rec[threadIdx.x] = threadIdx.x < G ? fin_m[threadIdx.x] : NEG_BIG;
+        rec[8 + threadIdx.x] = threadIdx.x < G ? fin_l[threadIdx.x] : 0.f;
+      }
+    }
+    mark(7);
+    cluster_sync_all();                                 // nobody leaves while a peer may still read its result
+    return;
+  }
   for (int e = threadIdx.x; e < G * cols; e += NT) {
     const int h = e / cols, c = e % cols;
     float v = mine[h * sw + c];

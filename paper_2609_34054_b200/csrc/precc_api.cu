@@ -359,7 +359,6 @@ struct DecodeRunT {
     const precc_layer_desc* d = a.d;
     constexpr int extra = ROPE ? DecodeCfg<HD, RK, RV>::BK_BYTES + 128 : 0;
     DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);
-    if (a.raw) pl.cluster = 0;                        // records are written by the ticket kernel
     if (pl.cluster && !(pl.warps == 8 ? cluster_fits<8>(ctx, pl, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, pl, a.B * d->n_kv_heads))) pl.cluster = 0;
     if (!pl.cluster) {
       pl = plan_ticket<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);

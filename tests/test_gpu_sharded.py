@@ -97,3 +97,19 @@ def test_one_shard_reproduces_the_plain_kernel_and_empty_requests_give_zeros(px)
     with pytest.raises(PreccError):
         px.combine_partials(L.desc, recs.new_zeros((65,) + tuple(recs.shape[1:])), torch.tensor(agents, dtype=torch.int32).cuda(),
                             L.B_v, out)
+
+
+def test_long_context_shards_take_the_cluster_path(px):
+    """Benchmark-layer shape, one request, 8192 tokens over 2 shards: each shard's launch is the cluster
+    kernel (few units, long context), whose blocks write column slices of the record."""
+    geo, T = I.C2, 8192
+    H = I.hidden_states(T, geo, 0, "L0.H")
+    q = I.queries(2, geo, 0, "sh.q2", gain=4.0)
+    agents, ctx = [3, -1], [T, 5000]
+    out, recs, L = _sharded_decode(px, geo, 0, H, q, agents, ctx, 2)
+    assert torch.isfinite(recs).all()
+    w = L.w_np
+    args = (f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"])
+    ref0 = O.lr_decode_reference(f64(q[:1]), [3], [T], *args, geo.scale_k, geo.scale_v, geo.n_kv)
+    ref1 = O.lr_decode_reference(f64(q[1:]), [0], [5000], *args, 0.0, 0.0, geo.n_kv)
+    assert_close(f64(out), np.concatenate([ref0, ref1]), "sharded C2 decode")
