@@ -782,12 +782,13 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   constexpr int BV_PER_THREAD = RV > 0 ? (RV * (HD / 2) + NT - 1) / NT : 1;
   __nv_bfloat16 bv_pre[BV_PER_THREAD];
   if constexpr (RV > 0) {
-    const int cols_ = HD / CS;
+    const int cols_ = (HD + CS - 1) / CS;                 // the cluster size need not divide the head dimension:
+    const int ncol_ = max(0, min(cols_, HD - rank * cols_));   // the last blocks own fewer (or no) columns
     const __nv_bfloat16* Bv = p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD + rank * cols_;
 #pragma unroll
     for (int k = 0; k < BV_PER_THREAD; ++k) {
       const int i = threadIdx.x + k * NT;
-      bv_pre[k] = (i < RV * cols_ && !p.raw) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);   // partial-output mode has no B_v
+      bv_pre[k] = (i < RV * cols_ && (i % cols_) < ncol_ && !p.raw) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);   // partial-output mode has no B_v
     }
   }
   if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
@@ -797,8 +798,9 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   float* res = reinterpret_cast<float*>(smem);
   float* mine = res + C::PART_STRIDE;                   // merged slice [G][cols + RV], then l[8]
   __nv_bfloat16* bvs = reinterpret_cast<__nv_bfloat16*>(mine + 8 * (HD + RV) + 8);   // B_v[:, my columns], [RV][cols]
-  const int cols = HD / CS;                             // output columns finished by this block
+  const int cols = (HD + CS - 1) / CS;                  // output columns finished by a block (stride of the slices)
   const int c0 = rank * cols;
+  const int ncol = max(0, min(cols, HD - c0));          // columns this block really owns
   if constexpr (RV > 0) {                               // B_v column slice (bv_pre was requested before the stream)
     for (int k = 0; k < BV_PER_THREAD; ++k) {
       const int i = threadIdx.x + k * NT;
@@ -817,6 +819,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     const bool is_l = e >= G * sw;
     const int h = is_l ? e - G * sw : e / sw;
     const int k = e % sw;
+    if (!is_l && k < cols && k >= ncol) { mine[e] = 0.f; continue; }   // slice padding past the head dimension
     const int src = is_l ? 8 + h : 16 + h * OW + (k < cols ? c0 + k : HD + (k - cols));
     float mr[DEC_MAX_CLUSTER], xr[DEC_MAX_CLUSTER];
 #pragma unroll
@@ -840,7 +843,8 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     // partial-output mode: this block's column slice of the merged, un-normalised record; block 0 adds the
     // LR-V coordinates, the denominators and the maxima
     float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
-    for (int e = threadIdx.x; e < G * cols; e += NT) rec[16 + (e / cols) * OW + c0 + (e % cols)] = mine[(e / cols) * sw + (e % cols)];
+    for (int e = threadIdx.x; e < G * cols; e += NT)
+      if ((e % cols) < ncol) rec[16 + (e / cols) * OW + c0 + (e % cols)] = mine[(e / cols) * sw + (e % cols)];
     if (rank == 0) {
       if constexpr (RV > 0) {
         for (int e = threadIdx.x; e < G * RV; e += NT) rec[16 + (e / RV) * OW + HD + (e % RV)] = mine[(e / RV) * sw + cols + (e % RV)];
@@ -857,6 +861,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   }
   for (int e = threadIdx.x; e < G * cols; e += NT) {
     const int h = e / cols, c = e % cols;
+    if (c >= ncol) continue;
     float v = mine[h * sw + c];
     if constexpr (RV > 0) {
       float u[4] = {0.f, 0.f, 0.f, 0.f};

@@ -271,7 +271,8 @@ DecodePlan plan_ticket(int sm_count, int max_smem, int B, int n_kv, int max_ctx,
   const long long units = (long long)B * n_kv;
   // blocks per (request, kv head): fill the machine once; with plenty of work use 4 waves of
   // blocks so that requests of different length balance out
-  long long want = (slots + units - 1) / units;
+  long long want = slots / units;                       // rounded down: one full wave, never a wave and a bit
+  if (want < 1) want = 1;
   const long long total_tiles = units * max_tiles;
   if (total_tiles >= slots * 4 * 64) want = (4 * slots + units - 1) / units;
   int chunk = (int)((max_tiles + want - 1) / want);
@@ -291,7 +292,6 @@ DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx
   const int max_tiles = (max_ctx + PAGE - 1) / PAGE;
   const long long units = (long long)B * n_kv;
   if (units * 2 > sm_count || max_tiles <= 16) return pl;  // too many units, or nothing worth splitting
-  if (units * max_tiles > 32768) return pl;              // bandwidth-bound: all SMs matter more than the short tail
   // two blocks per SM must fit (a 16-block cluster needs 16 free slots inside one GPC, and not every
   // GPC has 16 SMs): 8 warps with a 2-deep ring if that fits, else 4 warps with the deepest ring that does
   const int budget = max_smem / 2 - 1024 - extra;
@@ -301,9 +301,15 @@ DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx
     while (stages > 2 && C::cluster_smem(4, stages) > budget) --stages;
     if (C::cluster_smem(4, stages) > budget) return pl;
   }
+  // as many blocks per unit as keep the whole grid in one wave (any size up to 16, not only powers of two:
+  // 3 requests x 8 heads take 6 blocks each = 144 blocks, where 4 would leave a third of the SMs idle)
   int cs = DEC_MAX_CLUSTER;
-  while (cs > 1 && (units * cs > sm_count || max_tiles < cs * warps)) cs >>= 1;
+  if ((long long)cs * units > sm_count) cs = (int)(sm_count / units);
+  if (cs * warps > max_tiles) cs = max_tiles / warps;
   if (cs < 2) return pl;
+  // bandwidth-bound sizes: wide clusters (few units) leave SMs idle and pay a wider merge, where the ticket
+  // kernel fills every SM; narrow ones (measured up to 4) still win over it
+  if (units * max_tiles > 32768 && cs > 4) return pl;
   pl.cluster = cs;
   pl.warps = warps;
   pl.stages = stages;

@@ -401,3 +401,40 @@ def test_device_side_bad_indices_are_flagged_not_fatal(px):
     assert px.poll_status() & 1
     assert (out[1] == 0).all() and torch.isfinite(out[0]).all()
     assert px.poll_status() == 0
+
+
+@pytest.mark.parametrize("B,hd,n_kv", [(3, 64, 8), (5, 64, 8), (6, 128, 8), (9, 128, 4), (2, 128, 5)])
+def test_decode_cluster_sizes_that_do_not_divide_the_head_dimension(px, B, hd, n_kv):
+    """Few requests, long contexts: the splits of a (request, kv head) form a cluster of as many blocks as fit
+    the machine in one wave (6, 3, 3, 4, 14 here), each finishing a slice of the output columns; the slices
+    are uneven when the cluster size does not divide head_dim."""
+    geo = I.Geometry(1024, 2 * n_kv, n_kv, hd, 3, 16, 16, alpha=32.0)
+    T = 4096 + 16 * B + 5
+    nb = (T + 15) // 16
+    c = I.direct_caches(nb, geo, 51, f"cl.{B}")
+    from paper_2609_34054_b200.binding import Cache, layer_desc
+    cache = Cache.from_tensors(geo, c["k_base"].cuda(), c["v_base"].cuda(), c["lr_k"].cuda(), c["lr_v"].cuda())
+    w = I.layer_weights(geo, 51, "cl")
+    desc = layer_desc(geo)
+    q = I.queries(B, geo, 51, f"cl.q{B}", gain=4.0)
+    agents = [i % 3 for i in range(B)]
+    ctx = [T - 37 * i for i in range(B)]
+    out = torch.full_like(q, float("nan"), device="cuda")
+    ws = px.decode_workspace(desc, B, T)
+    args = (desc, q.cuda(), torch.tensor(agents, dtype=torch.int32).cuda(), torch.tensor(ctx, dtype=torch.int32).cuda(), T,
+            w["B_k"].cuda(), w["B_v"].cuda(), cache, out, ws)
+    px.lr_attend_decode(*args)
+    torch.cuda.synchronize()
+    first = out.clone()
+    px.lr_attend_decode(*args)
+    torch.cuda.synchronize()
+    assert torch.equal(first, out)                                   # deterministic
+    G = geo.group
+    for b, g in ((0, 0), (B - 1, n_kv - 1), (B // 2, n_kv // 2)):
+        t, a = ctx[b], agents[b]
+        rows = lambda x: f64(x.reshape(-1, x.shape[-1]))[:t]
+        cols = slice(g * hd, (g + 1) * hd)
+        ref = O.attend_from_caches(f64(q[b, g * G:(g + 1) * G]), rows(c["k_base"][:, g]), rows(c["v_base"][:, g]),
+                                   rows(c["lr_k"][a]), rows(c["lr_v"][a]), f64(w["B_k"][a][:, cols]), f64(w["B_v"][a][:, cols]),
+                                   geo.scale_k, geo.scale_v, 1)
+        assert_close(f64(out)[b, g * G:(g + 1) * G], ref, f"B={B} request {b} head {g}")
