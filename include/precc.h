@@ -155,7 +155,8 @@ int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const v
                            uint64_t agent_mask, const precc_cache* cache, void* stream);
 
 /* Workspace size for precc_lr_attend_decode with at most max_batch requests of at most max_ctx tokens
- * on a device with `sm_count` SMs.  The workspace must be zeroed once (precc_workspace_init) before its
+ * on a device with `sm_count` SMs: an upper bound over every such call (a smaller batch splits each request
+ * further, so the bound is taken over all batch sizes up to max_batch).  The workspace must be zeroed once (precc_workspace_init) before its
  * first use; calls leave it ready for the next call.  Two calls that may run concurrently need
  * separate workspaces. */
 size_t precc_decode_workspace_bytes(const precc_layer_desc* desc, int32_t max_batch, int32_t max_ctx,

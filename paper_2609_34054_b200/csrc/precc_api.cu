@@ -330,10 +330,34 @@ struct DecodeArgs {
 template <int HD, int RK, int RV, bool ROPE = false>
 struct DecodeRunT {
   // (the rotary variant never needs more than the plain one: its larger blocks only lower the split count)
-  static size_t ws_bytes(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
-    const DecodePlan pl = plan_ticket<HD, RK, RV>(sm_count, max_smem, B, n_kv, max_ctx, ROPE ? DecodeCfg<HD, RK, RV>::BK_BYTES + 128 : 0);
+  // exact need of one call
+  static size_t ws_need(int B, int n_kv, int max_splits) {
     const size_t tickets = ((size_t)B * n_kv * 4 + 255) / 256 * 256;
-    return tickets + (size_t)B * n_kv * pl.max_splits * DecodeCfg<HD, RK, RV>::PART_STRIDE * 4;
+    return tickets + (size_t)B * n_kv * max_splits * DecodeCfg<HD, RK, RV>::PART_STRIDE * 4;
+  }
+  // Upper bound over EVERY call with at most B requests of at most max_ctx tokens (a smaller batch gets more
+  // splits per request, so the need is not monotone in B).  Mirrors plan_ticket: splits <= blocks wanted per
+  // unit, splits <= pages / DEC_WARPS, and the four-wave mode can only switch on as the context grows.
+  static size_t ws_bytes(int sm_count, int max_smem, int B, int n_kv, int max_ctx) {
+    using C = DecodeCfg<HD, RK, RV>;
+    int stages = 4;
+    while (stages > 2 && 2 * (C::ticket_smem(stages) + 1024) > max_smem) --stages;
+    const long long slots = (long long)sm_count * ((2 * (C::ticket_smem(stages) + 1024) <= max_smem) ? 2 : 1);
+    const long long max_tiles = (max_ctx + PAGE - 1) / PAGE;
+    size_t best = 0;
+    for (int b = 1; b <= B; ++b) {
+      const long long units = (long long)b * n_kv;
+      long long want = slots / units;
+      if (want < 1) want = 1;
+      if (units * max_tiles >= slots * 4 * 64) want = (4 * slots + units - 1) / units;
+      long long bound = (max_tiles + DEC_WARPS - 1) / DEC_WARPS;
+      if (bound > want) bound = want;
+      if (bound > DEC_MAX_SPLITS) bound = DEC_MAX_SPLITS;
+      if (bound < 1) bound = 1;
+      const size_t need = ws_need(b, n_kv, (int)bound);
+      if (need > best) best = need;
+    }
+    return best;
   }
   // Can `need` clusters of `cs` blocks be resident at once?  Asked once per (shape, warps, cluster size).
   template <int NW>
@@ -368,7 +392,7 @@ struct DecodeRunT {
     if (pl.cluster && !(pl.warps == 8 ? cluster_fits<8>(ctx, pl, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, pl, a.B * d->n_kv_heads))) pl.cluster = 0;
     if (!pl.cluster) {
       pl = plan_ticket<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);
-      const size_t need = ws_bytes(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx);
+      const size_t need = ws_need(a.B, d->n_kv_heads, pl.max_splits);
       if (!a.ws || a.ws_bytes < need) return fail(ctx, PRECC_ERR_WORKSPACE, "decode workspace: need %zu bytes, got %zu", need, a.ws_bytes);
     }
     DecodeParams p;

@@ -14,6 +14,12 @@ states and queries), so its times are the KV-path share of a turn, not model lat
   fullshared  one shared full-width cache, no agent-specific part (the lower bound the paper compares to).
   nonshared   every agent keeps a private full-width cache and first processes all tokens it has not
               seen (everything the other agents appended since its last turn).
+  rebase_db   ReBaseShared with double batching: every step of the turn carries two sequences over the same
+              tokens, the adapted one (agent j: its LR rows, and adapted base rows in private blocks that
+              its block table splices in after the shared context) and the adapter-free one (neutral base
+              rows into the shared cache, the other agents' LR rows).  Prefill runs both; every decode step
+              is two one-row projections and ONE attention launch of two requests (agent j and the
+              adapter-free view, each with its own block table).  Nothing is left to do after the turn.
 
 TTFT of a turn = its prefill phase (projection + prefill attention over all layers); the trace's TTFT is
 the sum over turns; throughput = trajectory tokens / total time (Section 4.1).  Decode steps are one
@@ -33,7 +39,7 @@ import torch
 from . import inputs as I
 from .binding import Cache, Precc, layer_desc
 
-POLICIES = ("prelr", "rebase_lp", "fullshared", "nonshared")
+POLICIES = ("prelr", "rebase_lp", "rebase_db", "fullshared", "nonshared")
 
 
 @dataclass(frozen=True)
@@ -71,11 +77,15 @@ class Stack:
     queries are random buffers shared by all layers (their values do not affect the work done)."""
 
     def __init__(self, px: Precc, geo: I.Geometry, n_layers: int, max_tokens: int, max_rows: int, seed: int = 0,
-                 shared_weights: bool = False):
+                 shared_weights: bool = False, private_tokens: int = 0):
         self.px, self.geo, self.n_layers = px, geo, n_layers
         self.desc = layer_desc(geo)
         n_blocks = (max_tokens + I.PAGE - 1) // I.PAGE
-        self.caches = [Cache(geo, n_blocks, fill=0.0) for _ in range(n_layers)]
+        # blocks [0, shared_blocks) hold the shared trajectory; the rest are private to the adapted sequence
+        # of the current turn (double batching only)
+        self.shared_blocks = n_blocks
+        self.private_blocks = (private_tokens + I.PAGE - 1) // I.PAGE + 1 if private_tokens else 0
+        self.caches = [Cache(geo, n_blocks + self.private_blocks, fill=0.0) for _ in range(n_layers)]
         n_w = 1 if shared_weights else n_layers
         self.WA, self.W, self.B_k, self.B_v = [], [], [], []
         for l in range(n_w):
@@ -87,7 +97,7 @@ class Stack:
         self.H = I.normal_bf16((max_rows, geo.d_model), 1.0, seed, "replay.H").cuda()
         self.q = I.queries(max_rows, geo, seed, "replay.q").cuda()
         self.out = torch.empty_like(self.q)
-        self.ws = px.decode_workspace(self.desc, 1, max_tokens)
+        self.ws = px.decode_workspace(self.desc, 2, max_tokens)      # up to two requests per launch (double batching)
         self.max_tokens = max_tokens
 
     def w(self, l: int) -> int:
@@ -149,10 +159,80 @@ def _timed(fn) -> float:
     return e0.elapsed_time(e1)
 
 
+def _adapted_table(st: Stack, P: int, n_c: int) -> torch.Tensor:
+    """Block table of the adapted sequence: the shared blocks of the context, then private blocks from the
+    page that holds position P on (that boundary page is private too, so that the two sequences never
+    write the same page)."""
+    n_ctx = P // I.PAGE
+    n_priv = (P % I.PAGE + n_c + I.PAGE - 1) // I.PAGE
+    if n_priv > st.private_blocks:
+        raise ValueError("turn longer than the private region of the stack")
+    return torch.cat([torch.arange(n_ctx, dtype=torch.int32), st.shared_blocks + torch.arange(n_priv, dtype=torch.int32)]).cuda()
+
+
+def _replay_db(st: Stack, turns: Sequence[Turn]) -> Dict[str, float]:
+    geo, px = st.geo, st.px
+    all_mask = (1 << geo.n_agents) - 1
+    ttft = decode_ms = 0.0
+    P = 0
+    dev = st.q.device
+    for t in turns:
+        j, n, n_c = t.agent, t.n_in, t.n_in + t.n_out
+        others = all_mask & ~(1 << j)
+        table_a = _adapted_table(st, P, n_c)
+        priv0 = st.shared_blocks * I.PAGE + P % I.PAGE                  # slot of position P in the private region
+        slots_a = (priv0 + torch.arange(n, dtype=torch.int32)).to(dev)
+
+        def prefill_both():
+            for l in range(st.n_layers):
+                k = st.w(l)
+                px.turn_project(st.desc, st.H[:n], st.WA[k], st.caches[l], 0, slots_a, 1 << j)      # adapted rows
+                px.turn_project(st.desc, st.H[:n], st.WA[k], st.caches[l], P, None, others)         # adapter-free rows
+                px.lr_attend_prefill(st.desc, st.q[:n], j, P, st.B_k[k], st.B_v[k], st.caches[l], st.out[:n], table_a)
+                px.lr_attend_prefill(st.desc, st.q[:n], -1, P, st.B_k[k], st.B_v[k], st.caches[l], st.out[:n])
+
+        ttft += _timed(prefill_both)
+        if t.n_out > 0:
+            max_ctx = P + n_c
+            width = (max_ctx + I.PAGE - 1) // I.PAGE
+            table2 = torch.zeros((2, width), dtype=torch.int32)
+            table2[0, :table_a.numel()] = table_a.cpu()[:width]
+            table2[1] = torch.arange(width, dtype=torch.int32)
+            table2 = table2.to(dev)
+            ctx = torch.full((2,), P + n + 1, dtype=torch.int32, device=dev)
+            agent2 = torch.tensor([j, -1], dtype=torch.int32, device=dev)
+            slot_a = torch.tensor([priv0 + n], dtype=torch.int32, device=dev)
+            slot_n = torch.tensor([P + n], dtype=torch.int32, device=dev)
+
+            def step():
+                for l in range(st.n_layers):
+                    k = st.w(l)
+                    px.turn_project(st.desc, st.H[:1], st.WA[k], st.caches[l], 0, slot_a, 1 << j)
+                    px.turn_project(st.desc, st.H[1:2], st.WA[k], st.caches[l], 0, slot_n, others)
+                    px.lr_attend_decode(st.desc, st.q[:2], agent2, ctx, max_ctx, st.B_k[k], st.B_v[k], st.caches[l], st.out[:2],
+                                        st.ws, table2)
+                ctx.add_(1); slot_a.add_(1); slot_n.add_(1)
+
+            step()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                step()
+            decode_ms += _timed(lambda: [g.replay() for _ in range(t.n_out - 1)]) * t.n_out / max(1, t.n_out - 1)
+        P += n_c
+    total = ttft + decode_ms
+    per_tok = 2 * geo.n_kv * geo.hd * 2 + (geo.rank_k + geo.rank_v) * 2 * geo.n_agents
+    return {"policy": "rebase_db", "tokens": P, "turns": len(turns), "prefilled_tokens": 2 * sum(t.n_in for t in turns),
+            "ttft_ms": ttft, "decode_ms": decode_ms, "rebase_ms": 0.0, "total_ms": total, "tokens_per_s": P / total * 1e3,
+            "cache_gb": per_tok * P * st.n_layers / 1e9}
+
+
 def replay(st: Stack, turns: Sequence[Turn], policy: str) -> Dict[str, float]:
     """Replays one trace under one policy; returns milliseconds and token counts."""
     if policy not in POLICIES:
         raise ValueError(f"policy must be one of {POLICIES}")
+    if policy == "rebase_db":
+        return _replay_db(st, turns)
     geo = st.geo
     all_mask = (1 << geo.n_agents) - 1
     ttft = decode_ms = rebase_ms = 0.0
@@ -206,7 +286,7 @@ def main(argv=None):
     for turns in traces:
         total = trace_tokens(turns)
         rows = max(total, 64)                         # nonshared may prefill nearly the whole trajectory at once
-        st = Stack(px, geo, args.layers, total + I.PAGE, rows)
+        st = Stack(px, geo, args.layers, total + I.PAGE, rows, private_tokens=max(t.n_in + t.n_out for t in turns) + I.PAGE)
         for pol in args.policies.split(","):
             r = replay(st, turns, pol)
             r.update({"layers": args.layers, "n_agents": n_agents, "rank": args.rank})

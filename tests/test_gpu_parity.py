@@ -438,3 +438,26 @@ def test_decode_cluster_sizes_that_do_not_divide_the_head_dimension(px, B, hd, n
                                    rows(c["lr_k"][a]), rows(c["lr_v"][a]), f64(w["B_k"][a][:, cols]), f64(w["B_v"][a][:, cols]),
                                    geo.scale_k, geo.scale_v, 1)
         assert_close(f64(out)[b, g * G:(g + 1) * G], ref, f"B={B} request {b} head {g}")
+
+
+def test_one_workspace_serves_every_smaller_batch_and_context(px):
+    """The workspace query is an upper bound: a buffer sized for (max_batch, max_ctx) must be accepted for any
+    batch <= max_batch and any max_ctx below (smaller batches split each request further, so the need is not
+    monotone in the batch size)."""
+    geo = I.Geometry(256, 8, 2, 128, 2, 16, 16, alpha=32.0)
+    T = 40000
+    L = Layer(px, geo, seed=61, n_blocks=T // 16 + 1, fill=0.0)
+    ws = px.decode_workspace(L.desc, 8, T)
+    from paper_2609_34054_b200.binding import load_library
+    import ctypes
+    lib = load_library()
+    q8 = I.queries(8, geo, 61, "ws.q").cuda()
+    for B in (1, 2, 3, 5, 8):
+        for ctx in (T, 33333, 8200, 4096, 100, 1):
+            assert lib.precc_decode_workspace_bytes(ctypes.byref(L.desc), B, ctx, px.sm_count) <= ws.numel()
+            out = torch.empty_like(q8[:B])
+            px.lr_attend_decode(L.desc, q8[:B], torch.zeros(B, dtype=torch.int32, device="cuda"),
+                                torch.full((B,), ctx, dtype=torch.int32, device="cuda"), ctx, L.B_k, L.B_v, L.cache, out, ws,
+                                None, torch.zeros(B, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert px.poll_status() == 0
