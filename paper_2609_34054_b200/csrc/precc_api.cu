@@ -28,6 +28,7 @@ struct precc_ctx {
   size_t trace_blocks = 0;
   bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
   bool force_tiled_gemm = false;       // PRECC_GEMM=tiled in the environment: never take the few-row kernel
+  bool no_prefill_split = false;       // PRECC_PREFILL_SPLIT=0 in the environment: never split a turn's context over a cluster
   char err[512] = {0};
   CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                            const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -514,8 +515,45 @@ struct PrefillRun {
     auto kern = lr_attend_prefill_tc_kernel<HD, RK, RV>;
     PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int row_tiles = (a.S + p.tok_per_tile - 1) / p.tok_per_tile;
-    kern<<<dim3(row_tiles, d->n_kv_heads), PTC_THREADS, smem, a.stream>>>(mk, mv, mlk, mlv, p);
-    PRECC_CUDA(ctx, cudaGetLastError());
+    // Short turn over a long context: too few (row tile, kv head) blocks to fill the machine, so the
+    // context of each is split over a cluster of up to 8 blocks whose partial results merge over DSMEM.
+    int ns = 1;
+    const long long base_blocks = (long long)row_tiles * d->n_kv_heads;
+    const int steps = (a.T + a.S + PTC_TOK - 1) / PTC_TOK;
+    if (!ctx->no_prefill_split && C::SPLIT_BYTES <= ks * C::KSTAGE + vs * C::VSTAGE) {
+      ns = (int)(ctx->sm_count / base_blocks);          // as many as keep the grid within one block per SM
+      if (ns > 8) ns = 8;
+      if (ns > steps / 8) ns = steps / 8;               // at least eight steps per block
+      if (ns < 1) ns = 1;
+      // every cluster must be resident at once (one block per SM, and a cluster lives inside one GPC): ask
+      // the occupancy calculator once per cluster size, and shrink the clusters until the grid fits in one wave
+      static int max_clusters[9] = {0};               // 0 = unknown, else max active clusters + 1
+      while (ns > 1) {
+        if (max_clusters[ns] == 0) {
+          cudaLaunchConfig_t qc = {};
+          qc.gridDim = dim3(1, 1, ns * (ctx->sm_count / ns)); qc.blockDim = dim3(PTC_THREADS); qc.dynamicSmemBytes = smem;
+          cudaLaunchAttribute qa[1];
+          qa[0].id = cudaLaunchAttributeClusterDimension;
+          qa[0].val.clusterDim.x = 1; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = ns;
+          qc.attrs = qa; qc.numAttrs = 1;
+          int n = 0;
+          if (cudaOccupancyMaxActiveClusters(&n, kern, &qc) != cudaSuccess) { cudaGetLastError(); n = 0; }
+          max_clusters[ns] = n + 1;
+        }
+        if (max_clusters[ns] - 1 >= base_blocks) break;
+        --ns;
+      }
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(row_tiles, d->n_kv_heads, ns);
+    cfg.blockDim = dim3(PTC_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = ns;
+    cfg.attrs = attr; cfg.numAttrs = ns > 1 ? 1 : 0;
+    PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, mk, mv, mlk, mlv, p));
     return PRECC_OK;
   }
   static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
@@ -626,6 +664,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   }
   if (const char* v = getenv("PRECC_PREFILL")) ctx->force_simple_prefill = (strcmp(v, "simple") == 0);
   if (const char* v = getenv("PRECC_GEMM")) ctx->force_tiled_gemm = (strcmp(v, "tiled") == 0);
+  if (const char* v = getenv("PRECC_PREFILL_SPLIT")) ctx->no_prefill_split = (strcmp(v, "0") == 0);
   if (e != cudaSuccess) {
     fprintf(stderr, "precc_create: %s\n", cudaGetErrorString(e));
     if (ctx->status) cudaFree(ctx->status);

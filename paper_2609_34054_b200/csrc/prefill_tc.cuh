@@ -84,6 +84,9 @@ struct PrefillTcCfg {
   static constexpr int VSTAGE = VSLABS * SLAB_BYTES;          // {V_base slabs | L_V slab}
   static constexpr int K_PAGE_TX = PAGE * (HD + RK) * 2;      // bytes one page contributes to a key stage
   static constexpr int V_PAGE_TX = PAGE * VSLABS * 128;
+  static constexpr int SPLIT_XS = HD + RV + 4;                // row stride (floats) of a partial in shared memory
+  // split-context merge area (laid over the rings): partial | m | l | merged rows | weights | 1/l | B_v slice
+  static constexpr int SPLIT_BYTES = (128 * SPLIT_XS + 256 + 64 * SPLIT_XS + 16 * 64 + 64) * 4 + RV * HD * 2;
   static constexpr bool L_IN_MMA = RV > 0 && RV < 64;         // a spare column of the L_V slab carries the denominator
   static constexpr int TMEM_P = 2 * PTC_TOK;                  // packed bf16 P (64 columns) after the two S buffers
   static constexpr int TMEM_O = TMEM_P + PTC_TOK / 2;         // O' (at most 192 columns): 320 + 192 = 512
@@ -198,8 +201,18 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   const int tok0 = blockIdx.x * p.tok_per_tile;
   const int n_tok = min(p.tok_per_tile, p.S - tok0);             // new tokens handled by this block
   const int t_end = p.T + tok0 + n_tok;                          // context + causal reach of the last row
-  const int n_tiles = (t_end + PTC_TOK - 1) / PTC_TOK;
   const int full_vis = p.T + tok0 + 1;                           // tokens visible to every row of the block
+  // Short turns over long contexts: the 128-token steps of a (row tile, kv head) are split over the NS
+  // blocks of a cluster (grid/cluster z; any size from 2 to 8), each producing a partial (m, l, O') that the cluster merges
+  // over distributed shared memory.  `jb` is this block's first step, `n_tiles` its number of steps
+  // (possibly zero); loop indices below are local, token positions use jb + j.
+  uint32_t split, NS;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(split));
+  asm volatile("mov.u32 %0, %%cluster_nctaid.z;\n" : "=r"(NS));
+  const int n_total = (t_end + PTC_TOK - 1) / PTC_TOK;
+  const int chunk_steps = (n_total + (int)NS - 1) / (int)NS;
+  const int jb = min(n_total, (int)split * chunk_steps);
+  const int n_tiles = min(n_total, jb + chunk_steps) - jb;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < KS; ++s) { mbar_init(k_full + 8 * s, 1); mbar_init(k_empty + 8 * s, 1); }
@@ -232,7 +245,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       // the last key stage doubles as the staging area of B_k until the query fold is done
       if (RK > 0 && is_k && j == KS - 1) mbar_wait(q_ready, 0, p.status);
       if (lane == 0) PTC_STAMP(p, j, is_k ? 8 : 9);               // stage of step j free: loads go out now
-      const int t0 = j * PTC_TOK;
+      const int t0 = (jb + j) * PTC_TOK;
       const int live = min(PTC_TOK / PAGE, (t_end - t0 + PAGE - 1) / PAGE);
       const uint32_t st = is_k ? kring_u32 + (uint32_t)s * C::KSTAGE : vring_u32 + (uint32_t)s * C::VSTAGE;
       const uint32_t full = fullb + 8 * s;
@@ -241,7 +254,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         // (4-D map [block][kv head][16][hd]); blocks past the cache end arrive as zeros
         if (lane == 0) {
           mbar_expect_tx(full, (PTC_TOK / PAGE) * (is_k ? C::K_PAGE_TX : C::V_PAGE_TX));
-          const int blk0 = p.first_block + j * (PTC_TOK / PAGE);
+          const int blk0 = p.first_block + (jb + j) * (PTC_TOK / PAGE);
           if (is_k) {
 #pragma unroll
             for (int sl = 0; sl < C::SLABS; ++sl) tma_load_4d(st + sl * C::SLAB_BYTES, &map_k, sl * 64, 0, g, blk0, full);
@@ -258,7 +271,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       if (lane == 0) mbar_expect_tx(full, live * (is_k ? C::K_PAGE_TX : C::V_PAGE_TX));
       __syncwarp();
       if (lane < live) {
-        const int lt = j * (PTC_TOK / PAGE) + lane;
+        const int lt = (jb + j) * (PTC_TOK / PAGE) + lane;
         int ph = p.block_table ? __ldg(p.block_table + lt) : p.first_block + lt;
         if (ph < 0 || ph >= p.n_blocks) { atomicOr(p.status, StatusBits::BAD_INDEX); ph = 0; }
         const int row_kv = (ph * p.n_kv + g) * PAGE;
@@ -318,7 +331,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const uint64_t vd0 = umma_desc_mnmajor(vring_u32, 128, C::SLAB_BYTES);
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j % VS;
-      const int n_live = min(PTC_TOK, t_end - j * PTC_TOK);       // tokens of this step that exist
+      const int n_live = min(PTC_TOK, t_end - (jb + j) * PTC_TOK);       // tokens of this step that exist
       mbar_wait(v_full + 8 * s, (j / VS) & 1, p.status);
       if (lane == 0) PTC_STAMP(p, j, 11);                          // values of step j have landed
       if constexpr (C::L_IN_MMA) {
@@ -442,8 +455,8 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // (TMEM read, compare chain, exchange between the row's threads) is off the critical path.
     auto local_max = [&](int j) -> float {
       const int b = j & 1;
-      const int nvis = lim - (j * PTC_TOK + part * COLS) + 1;     // visible tokens among this thread's
-      const bool masked = j * PTC_TOK + PTC_TOK > full_vis;
+      const int nvis = lim - ((jb + j) * PTC_TOK + part * COLS) + 1;   // visible tokens among this thread's
+      const bool masked = (jb + j) * PTC_TOK + PTC_TOK > full_vis;
       float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
@@ -486,7 +499,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       __syncwarp();
       if (lane == 0) mbar_arrive(s_free + 8 * b);                  // the S buffer may be overwritten
       if constexpr (MASKED) {
-        const int nvis = lim - (j * PTC_TOK + part * COLS) + 1;
+        const int nvis = lim - ((jb + j) * PTC_TOK + part * COLS) + 1;
 #pragma unroll
         for (int c = 0; c < NCH; ++c)
 #pragma unroll
@@ -554,18 +567,53 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       if (j + 1 < n_tiles) tmax = exchange_max(j + 1, next_own);
     };
     if (tid == 0) PTC_STAMP(p, 0, 3);
-    mbar_wait(s_full, 0, p.status);
-    tc_fence_after();
-    tmax = exchange_max(0, local_max(0));
+    if (n_tiles > 0) {
+      mbar_wait(s_full, 0, p.status);
+      tc_fence_after();
+      tmax = exchange_max(0, local_max(0));
+    }
     for (int j = 0; j < n_tiles; ++j) {
       if (tid == 0) PTC_STAMP(p, j, 4);                            // step j starts (its scores were awaited a step earlier)
-      if (j * PTC_TOK + PTC_TOK > full_vis) step(j, std::true_type{});     // only the last few steps reach the causal edge
+      if ((jb + j) * PTC_TOK + PTC_TOK > full_vis) step(j, std::true_type{});   // only the last few steps reach the causal edge
       else step(j, std::false_type{});
       if (tid == 0) PTC_STAMP(p, j + 1, 3);
     }
     // ---- epilogue: out = (O + s_v U B_v) / l ; the threads of a row share its output columns
-    mbar_wait(pv_done, (n_tiles - 1) & 1, p.status);
-    tc_fence_after();
+    if (n_tiles > 0) { mbar_wait(pv_done, (n_tiles - 1) & 1, p.status); tc_fence_after(); }
+    if (NS > 1) {
+      // ---- split context: this block's partial (m, l, O') goes to shared memory for the cluster merge below
+      constexpr int XS = C::SPLIT_XS;
+      float* xo = reinterpret_cast<float*>(kring);
+      float* xm = xo + 128 * XS;
+      float* xl = xm + 128;
+      float l_loc = 0.f;
+      if constexpr (!C::L_IN_MMA) {
+        xch[part * 128 + row] = l_sum;
+        asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+#pragma unroll
+        for (int q2 = 0; q2 < NP; ++q2) l_loc += xch[q2 * 128 + row];
+      } else if (n_tiles > 0) {
+        uint32_t lv16[16];
+        tmem_ld16(lane_addr + C::TMEM_O + HD + (RV / 16) * 16, lv16);
+        tmem_wait_ld();
+        l_loc = __uint_as_float(lv16[0]);
+      }
+#pragma unroll 1
+      for (int c = part; c < (HD + RV) / 16; c += NP) {
+        uint32_t ov[16];
+        if (n_tiles > 0) {
+          tmem_ld16(lane_addr + C::TMEM_O + c * 16, ov);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int k = 0; k < 16; ++k) ov[k] = 0u;
+        }
+#pragma unroll
+        for (int k = 0; k < 16; k += 4)
+          *reinterpret_cast<uint4*>(xo + row * XS + c * 16 + k) = make_uint4(ov[k], ov[k + 1], ov[k + 2], ov[k + 3]);
+      }
+      if (part == 0) { xm[row] = n_tiles > 0 ? m_used : NEG_BIG; xl[row] = n_tiles > 0 ? l_loc : 0.f; }
+    } else {
     unsigned char* bv_s = vring;                                  // value stage 0 is free now
     if constexpr (RV > 0) {
       for (int c = tid; c < RV * (HD / 8); c += NSM) {
@@ -630,6 +678,100 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         }
       }
     }
+    }   // NS == 1
+  }
+  if (NS > 1) {
+    // ---- cluster merge of the context splits: block `split` finishes rows [split*R, (split+1)*R) of the tile
+    constexpr int XS = C::SPLIT_XS;
+    constexpr int NSM = PTC_SOFTMAX_WARPS * 32;
+    const int R = (128 + (int)NS - 1) / (int)NS;        // rows per block (the last block may own fewer); 2 <= NS <= 16
+    float* xo = reinterpret_cast<float*>(kring);
+    float* xm = xo + 128 * XS;
+    float* xl = xm + 128;
+    float* mo = xl + 128;                               // merged rows [R][XS]
+    float* wts = mo + 64 * XS;                          // [NS][R] weights of the splits
+    float* linv = wts + 16 * 64;                        // [R]
+    unsigned char* bvs = reinterpret_cast<unsigned char*>(linv + 64);   // B_v[:, g] slice, [RV][HD] bf16
+    asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+    if (warp >= PTC_FIRST_SM_WARP && warp < PTC_FIRST_SM_WARP + PTC_SOFTMAX_WARPS) {
+      const int tid = (warp - PTC_FIRST_SM_WARP) * 32 + lane;
+      const int r0 = (int)split * R;
+      const int nrows = max(0, min(R, 128 - r0));
+      auto peer = [&](const float* local, uint32_t s) -> uint32_t {
+        uint32_t remote;
+        asm("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(smem_u32(local)), "r"(s));
+        return remote;
+      };
+      auto ld1 = [&](uint32_t a) -> float { float v; asm volatile("ld.shared::cluster.f32 %0, [%1];\n" : "=f"(v) : "r"(a)); return v; };
+      if constexpr (RV > 0) {
+        for (int c = tid; c < RV * (HD / 8); c += NSM) {
+          const int j = c / (HD / 8), ch = c % (HD / 8);
+          *reinterpret_cast<uint4*>(bvs + (j * HD + ch * 8) * 2) =
+              __ldg(reinterpret_cast<const uint4*>(p.B_v + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
+        }
+      }
+      if (tid < nrows) {
+        float ms[16], M = NEG_BIG, L = 0.f;
+#pragma unroll
+        for (uint32_t s2 = 0; s2 < 16; ++s2) { ms[s2] = s2 < NS ? ld1(peer(xm + r0 + tid, s2)) : NEG_BIG; M = fmaxf(M, ms[s2]); }
+#pragma unroll
+        for (uint32_t s2 = 0; s2 < 16; ++s2) {
+          if (s2 < NS) {
+            const float wv = fast_exp2(ms[s2] - M);
+            wts[s2 * R + tid] = wv;
+            L += wv * ld1(peer(xl + r0 + tid, s2));               // split order: deterministic
+          }
+        }
+        linv[tid] = L > 0.f ? 1.f / L : 0.f;
+      }
+      asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+      constexpr int F4 = (HD + RV) / 4;                   // float4 columns of a merged row
+      for (int it = tid; it < nrows * F4; it += NSM) {
+        const int rl = it / F4, c4 = it % F4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint32_t s2 = 0; s2 < NS; ++s2) {
+          const uint32_t a = peer(xo + (r0 + rl) * XS + c4 * 4, s2);
+          float4 x;
+          asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w) : "r"(a));
+          const float wv = wts[s2 * R + rl];
+          acc.x += wv * x.x; acc.y += wv * x.y; acc.z += wv * x.z; acc.w += wv * x.w;
+        }
+        *reinterpret_cast<float4*>(mo + rl * XS + c4 * 4) = acc;
+      }
+      asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+      // out = (O + s_v U B_v) / l for my rows, eight columns per item
+      for (int it = tid; it < nrows * (HD / 8); it += NSM) {
+        const int rl = it / (HD / 8), c8 = (it % (HD / 8)) * 8;
+        const int rowg = r0 + rl;
+        if (rowg >= n_tok * G) continue;
+        float o[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) o[k] = mo[rl * XS + c8 + k];
+        if constexpr (RV > 0) {
+#pragma unroll 4
+          for (int jv = 0; jv < RV; ++jv) {
+            const float uj = mo[rl * XS + HD + jv] * p.s_v;
+            const uint4 y = *reinterpret_cast<const uint4*>(bvs + (jv * HD + c8) * 2);
+            const uint32_t ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              o[2 * k] += uj * bf16_bits_to_float(ys[k] & 0xffff);
+              o[2 * k + 1] += uj * bf16_bits_to_float(ys[k] >> 16);
+            }
+          }
+        }
+        const float inv = linv[rl];
+        const int i_new = tok0 + rowg / G, hg = rowg % G;
+        uint4 w;
+        w.x = pack_bf16(o[0] * inv, o[1] * inv); w.y = pack_bf16(o[2] * inv, o[3] * inv);
+        w.z = pack_bf16(o[4] * inv, o[5] * inv); w.w = pack_bf16(o[6] * inv, o[7] * inv);
+        *reinterpret_cast<uint4*>(p.out + ((size_t)i_new * p.n_q + (size_t)g * G + hg) * HD + c8) = w;
+      }
+    }
+    // nobody leaves while a peer may still read its partial
+    asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();

@@ -461,3 +461,25 @@ def test_one_workspace_serves_every_smaller_batch_and_context(px):
                                 None, torch.zeros(B, dtype=torch.int32, device="cuda"))
     torch.cuda.synchronize()
     assert px.poll_status() == 0
+
+
+@pytest.mark.parametrize("hd,n_q,n_kv,r,T,S,agent", [(128, 8, 2, 32, 2100, 40, 1), (128, 8, 2, 16, 4200, 33, 0), (64, 16, 4, 16, 9000, 20, 1),
+                                                       (128, 8, 2, 32, 8300, 64, -1), (64, 8, 1, 32, 5000, 130, 0)])
+def test_prefill_short_turn_over_long_context_is_split_over_a_cluster(px, hd, n_q, n_kv, r, T, S, agent):
+    """Few (row tile, kv head) blocks and many 128-token steps: the context is split over a cluster of 2, 4 or
+    8 blocks and merged over distributed shared memory.  Against the definition, and bit-identical runs."""
+    geo = I.Geometry(256, n_q, n_kv, hd, 2, r, r, alpha=2.0 * r)
+    L = Layer(px, geo, seed=71, n_blocks=(T + S + 15) // 16, tag="sp")
+    H = I.hidden_states(T + S, geo, 71, "sp.H")
+    L.append(H)
+    qs = I.queries(S, geo, 71, "sp.q", gain=4.0)
+    got = L.prefill(qs, agent, T)
+    again = L.prefill(qs, agent, T)
+    assert torch.equal(got, again)
+    w = L.w_np
+    rows = sorted(set([0, 1, S // 2, S - 2, S - 1]))
+    a = max(agent, 0)
+    sk, sv = (geo.scale_k, geo.scale_v) if agent >= 0 else (0.0, 0.0)
+    ref = O.lr_prefill_reference(f64(qs), a, T, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"], sk, sv, n_kv,
+                                 rows=rows)
+    assert_close(f64(got), ref, f"split prefill hd{hd} T{T} S{S}")
