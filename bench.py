@@ -37,7 +37,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch of this workload, from the ncu
 # capture summarised under profiles/ (None until a capture exists)
-NCU_DECODE_TRAFFIC_BYTES = 17370112   # profiles/decode_cluster_c2_layer.md
+NCU_DECODE_TRAFFIC_BYTES = 17378560   # profiles/decode_cluster_c2_layer.md
 
 
 def decode_bytes_per_launch(geo, ctx: int, batch: int = 1, distinct_agents: int = 1) -> int:

@@ -28,6 +28,7 @@ struct precc_ctx {
   size_t trace_blocks = 0;
   bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
   bool force_tiled_gemm = false;       // PRECC_GEMM=tiled in the environment: never take the few-row kernel
+  bool deep_clusters = true;           // PRECC_DEEP=0 in the environment: never use the one-block-per-SM deep-ring clusters
   bool no_prefill_split = false;       // PRECC_PREFILL_SPLIT=0 in the environment: never split a turn's context over a cluster
   char err[512] = {0};
   CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -254,7 +255,7 @@ int32_t dispatch_shape(precc_ctx* ctx, int hd, int rk, int rv, Args&&... args) {
 
 // Split schedule of decode.  cluster > 0: the cluster kernel with that many blocks per (request, kv head);
 // otherwise the ticket kernel with up to max_splits blocks per (request, kv head).
-struct DecodePlan { int cluster, warps, chunk_tiles, max_splits, stages, smem; };
+struct DecodePlan { int cluster, warps, chunk_tiles, max_splits, stages, smem, deep; };
 
 // `extra`: bytes of shared memory appended after the usual layout (the rotary variant's B_k slice).
 template <int HD, int RK, int RV>
@@ -287,7 +288,7 @@ DecodePlan plan_ticket(int sm_count, int max_smem, int B, int n_kv, int max_ctx,
 // The cluster kernel serves the latency-bound regime: few (request, kv head) units, each worth
 // splitting, the whole grid co-resident in one wave.  Returns cluster = 0 when it does not apply.
 template <int HD, int RK, int RV>
-DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx, int extra = 0) {
+DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx, int extra = 0, bool deep_ok = true) {
   using C = DecodeCfg<HD, RK, RV>;
   DecodePlan pl{};
   const int max_tiles = (max_ctx + PAGE - 1) / PAGE;
@@ -308,9 +309,24 @@ DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx
   if ((long long)cs * units > sm_count) cs = (int)(sm_count / units);
   if (cs * warps > max_tiles) cs = max_tiles / warps;
   if (cs < 2) return pl;
-  // bandwidth-bound sizes: wide clusters (few units) leave SMs idle and pay a wider merge, where the ticket
-  // kernel fills every SM; narrow ones (measured up to 4) still win over it
-  if (units * max_tiles > 32768 && cs > 4) return pl;
+  // Wide clusters (very few units) with more than a few pages per warp: one block per SM with the whole
+  // shared memory as page rings, i.e. two to three times the bytes in flight per SM and fewer dependent DRAM
+  // round trips per warp; the run-time occupancy check then shrinks the cluster until all clusters are
+  // resident (a 16-block cluster at one block per SM does not fit every GPC).  Measured against the
+  // two-blocks-per-SM layout: 8192 tokens x 8 units 9.3 -> 9.0 us, 32768 tokens 31 -> 27 us, 65536 tokens
+  // 53 -> 46 us.  With the deep rings switched off, bandwidth-bound sizes go to the ticket kernel instead.
+  if (units * max_tiles > (deep_ok ? 2048 : 32768) && cs > 4) {
+    if (!deep_ok) return pl;
+    const int big = max_smem - 2048 - extra;
+    warps = 8; stages = 4;
+    while (stages > 2 && C::cluster_smem(8, stages) > big) --stages;
+    if (C::cluster_smem(8, stages) > big) {
+      warps = 4; stages = 4;
+      while (stages > 2 && C::cluster_smem(4, stages) > big) --stages;
+      if (C::cluster_smem(4, stages) > big) return pl;
+    }
+    pl.deep = 1;
+  }
   pl.cluster = cs;
   pl.warps = warps;
   pl.stages = stages;
@@ -363,7 +379,8 @@ struct DecodeRunT {
   // Can `need` clusters of `cs` blocks be resident at once?  Asked once per (shape, warps, cluster size).
   template <int NW>
   static bool cluster_fits(precc_ctx* ctx, const DecodePlan& pl, int need) {
-    static int cached[DEC_MAX_CLUSTER + 1] = {0};      // 0 = unknown, else max active clusters + 1
+    static int cache2[2][DEC_MAX_CLUSTER + 1] = {{0}};  // 0 = unknown, else max active clusters + 1
+    int* cached = cache2[pl.deep ? 1 : 0];
     if (cached[pl.cluster] == 0) {
       auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
       int n = 0;
@@ -389,8 +406,15 @@ struct DecodeRunT {
   static int32_t run(precc_ctx* ctx, const DecodeArgs& a) {
     const precc_layer_desc* d = a.d;
     constexpr int extra = ROPE ? DecodeCfg<HD, RK, RV>::BK_BYTES + 128 : 0;
-    DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);
-    if (pl.cluster && !(pl.warps == 8 ? cluster_fits<8>(ctx, pl, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, pl, a.B * d->n_kv_heads))) pl.cluster = 0;
+    DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra, ctx->deep_clusters);
+    auto fits = [&](const DecodePlan& q) { return q.warps == 8 ? cluster_fits<8>(ctx, q, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, q, a.B * d->n_kv_heads); };
+    if (pl.cluster && pl.deep) {
+      const int max_tiles = (a.max_ctx + PAGE - 1) / PAGE;
+      while (pl.cluster > 4 && !fits(pl)) { --pl.cluster; pl.chunk_tiles = (max_tiles + pl.cluster - 1) / pl.cluster; pl.max_splits = pl.cluster; }
+      if (pl.cluster <= 4) pl.cluster = 0;
+    } else if (pl.cluster && !fits(pl)) {
+      pl.cluster = 0;
+    }
     if (!pl.cluster) {
       pl = plan_ticket<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra);
       const size_t need = ws_need(a.B, d->n_kv_heads, pl.max_splits);
@@ -664,6 +688,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   }
   if (const char* v = getenv("PRECC_PREFILL")) ctx->force_simple_prefill = (strcmp(v, "simple") == 0);
   if (const char* v = getenv("PRECC_GEMM")) ctx->force_tiled_gemm = (strcmp(v, "tiled") == 0);
+  if (const char* v = getenv("PRECC_DEEP")) ctx->deep_clusters = (strcmp(v, "0") != 0);
   if (const char* v = getenv("PRECC_PREFILL_SPLIT")) ctx->no_prefill_split = (strcmp(v, "0") == 0);
   if (e != cudaSuccess) {
     fprintf(stderr, "precc_create: %s\n", cudaGetErrorString(e));
