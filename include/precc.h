@@ -154,6 +154,15 @@ int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const v
                            const void* WA_packed, const int32_t* slot_mapping, int64_t start_slot,
                            uint64_t agent_mask, const precc_cache* cache, void* stream);
 
+/* precc_turn_project with one agent mask per row (double batching, Section 3.2: the adapted and the
+ * adapter-free sequence of a turn ride in one batch — the adapted rows write only the current agent's LR
+ * rows, the adapter-free rows write the other agents').  Every row writes its base rows at its own slot, so
+ * the two sequences must map to different slots (e.g. private blocks for the adapted one).
+ *   slot_mapping     [M] required;  row_agent_masks  device uint64 [M], bit k = write agent k for that row */
+int32_t precc_turn_project_rows(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
+                                const void* WA_packed, const int32_t* slot_mapping,
+                                const uint64_t* row_agent_masks, const precc_cache* cache, void* stream);
+
 /* Workspace size for precc_lr_attend_decode with at most max_batch requests of at most max_ctx tokens
  * on a device with `sm_count` SMs: an upper bound over every such call (a smaller batch splits each request
  * further, so the bound is taken over all batch sizes up to max_batch).  The workspace must be zeroed once (precc_workspace_init) before its

@@ -23,7 +23,7 @@ EXPORTS = [
     "precc_decode_workspace_bytes", "precc_workspace_init", "precc_lr_attend_decode",
     "precc_lr_attend_decode_static", "precc_lr_attend_prefill",
     "precc_rebase_project_rope", "precc_turn_project_rope", "precc_lr_attend_decode_rope", "precc_lr_attend_prefill_rope",
-    "precc_partial_record_floats", "precc_lr_attend_decode_partial", "precc_combine_partials",
+    "precc_turn_project_rows", "precc_partial_record_floats", "precc_lr_attend_decode_partial", "precc_combine_partials",
 ]
 
 
@@ -88,6 +88,7 @@ def load_library() -> C.CDLL:
                                                 C.POINTER(CacheDesc), vp, vp, sz, vp]
     lib.precc_lr_attend_prefill_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp, rp,
                                                  C.POINTER(CacheDesc), vp, vp]
+    lib.precc_turn_project_rows.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, C.POINTER(CacheDesc), vp]
     lib.precc_partial_record_floats.argtypes = [C.POINTER(LayerDesc)]
     lib.precc_partial_record_floats.restype = sz
     lib.precc_lr_attend_decode_partial.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, i32, vp, i32, vp,
@@ -241,6 +242,16 @@ class Precc:
         self._check(self.lib.precc_turn_project(self.h, C.byref(desc), _ptr(H), H.shape[0], _ptr(WA_packed),
                                                 _ptr(slot_mapping), start_slot, agent_mask & ((1 << 64) - 1),
                                                 C.byref(cd), _stream()), "precc_turn_project")
+
+    def turn_project_rows(self, desc: LayerDesc, H: torch.Tensor, WA_packed: torch.Tensor, cache: Cache,
+                          slot_mapping: torch.Tensor, row_masks: torch.Tensor):
+        """Fused projection with one agent mask per row (row_masks: int64 tensor holding the uint64 bit masks)."""
+        if row_masks.dtype != torch.int64:
+            raise PreccError("row_masks must be int64 (bit patterns of uint64 masks)")
+        cd = cache.desc()
+        self._check(self.lib.precc_turn_project_rows(self.h, C.byref(desc), _ptr(H), H.shape[0], _ptr(WA_packed),
+                                                     _ptr(slot_mapping), _ptr(row_masks), C.byref(cd), _stream()),
+                    "precc_turn_project_rows")
 
     # ------------------------------------------------------------------ the four entry points
     def lr_precompute(self, desc: LayerDesc, H: torch.Tensor, A_packed: torch.Tensor, cache: Cache,

@@ -36,6 +36,7 @@ struct GemmParams {
   __nv_bfloat16* lr_v;
   int n_agents, rank_k, rank_v;
   unsigned long long agent_mask;
+  const unsigned long long* row_masks;   // optional [M]: per-row agent masks (double batching), overrides agent_mask
   int n_kv, hd;
   // rotary keys (modes 1, 2; null = none): the key columns of a row are rotated by the row's position
   // before they are stored (rotate-half pairing (c, c + hd/2)); needs BN % hd == 0
@@ -129,9 +130,10 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 
 // Routes eight consecutive output columns [gc, gc+8) of one row (cache block `blk`, offset `off`) to
 // their place in the paged caches: column -> (projection, head, c) for base columns, (projection, agent,
-// r) for LR columns (skipped when the agent is masked out).  Pieces never straddle a destination row
+// r) for LR columns (skipped when the agent's bit in `mask` — the call's mask or the row's own — is clear).  Pieces never straddle a destination row
 // because head_dim and the ranks are multiples of 8.
-__device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, int off, int gc, const float (&v8)[8]) {
+__device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, int off, int gc, const float (&v8)[8],
+                                            unsigned long long mask) {
   const int w = p.n_kv * p.hd;
   __nv_bfloat16* dst;
   const bool to_base = p.mode == 1 || (p.mode == 2 && gc < 2 * w);
@@ -142,7 +144,7 @@ __device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, 
     const int rr = is_v ? p.rank_v : p.rank_k;
     const int cc = is_v ? gl - n_k : gl;
     const int agent = cc / rr, ri = cc % rr;
-    if (!((p.agent_mask >> agent) & 1ull)) return;
+    if (!((mask >> agent) & 1ull)) return;
     dst = (is_v ? p.lr_v : p.lr_k) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
   } else {
     const bool is_v = gc >= w;
@@ -255,6 +257,7 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       }
       const long long blk = slot / PAGE;
       const int off = (int)(slot % PAGE);
+      const unsigned long long row_mask = (p.row_masks && row_ok) ? p.row_masks[gm] : p.agent_mask;
       long long pos = 0;
       if (p.rope && row_ok) {
         pos = p.positions ? (long long)p.positions[gm] : p.start_pos + gm;
@@ -300,7 +303,7 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
           float v8[8];
 #pragma unroll
           for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(r[8 * h + k]);
-          store_piece(p, blk, off, gc, v8);
+          store_piece(p, blk, off, gc, v8, row_mask);
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");

@@ -832,7 +832,7 @@ int32_t precc_rebase_project_rope(precc_ctx* ctx, const precc_layer_desc* desc, 
 
 static int32_t turn_entry(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
                           const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_rope* rope,
-                          const precc_cache* cache, void* stream) {
+                          const precc_cache* cache, void* stream, const uint64_t* row_masks = nullptr) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (M < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "M < 0");
@@ -849,6 +849,7 @@ static int32_t turn_entry(precc_ctx* ctx, const precc_layer_desc* desc, const vo
   gp.base_k = (__nv_bfloat16*)cache->k_base; gp.base_v = (__nv_bfloat16*)cache->v_base;
   gp.lr_k = (__nv_bfloat16*)cache->lr_k; gp.lr_v = (__nv_bfloat16*)cache->lr_v;
   gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = agent_mask;
+  gp.row_masks = reinterpret_cast<const unsigned long long*>(row_masks);
   gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
   gp.M = M;
   rc = set_rope(ctx, desc, rope, &gp);
@@ -860,6 +861,15 @@ int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const v
                            const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_cache* cache,
                            void* stream) {
   return turn_entry(ctx, desc, H, M, WA_packed, slot_mapping, start_slot, agent_mask, nullptr, cache, stream);
+}
+
+int32_t precc_turn_project_rows(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
+                                const int32_t* slot_mapping, const uint64_t* row_agent_masks, const precc_cache* cache,
+                                void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!slot_mapping || !row_agent_masks) return fail(ctx, PRECC_ERR_INVALID_ARG, "slot_mapping / row_agent_masks is null");
+  if (reinterpret_cast<uintptr_t>(row_agent_masks) & 7u) return fail(ctx, PRECC_ERR_MISALIGNED, "row_agent_masks not 8-byte aligned");
+  return turn_entry(ctx, desc, H, M, WA_packed, slot_mapping, 0, 0, nullptr, cache, stream, row_agent_masks);
 }
 
 int32_t precc_turn_project_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,

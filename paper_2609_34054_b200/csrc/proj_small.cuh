@@ -163,6 +163,7 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     if (gc < kw && (gc % p.hd) >= p.hd / 2) continue;   // upper half of a rotated head: written with its lower partner
     long long slot = p.slot_mapping ? (long long)p.slot_mapping[row] : p.start_slot + row;
     if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); continue; }
+    const unsigned long long mask = p.row_masks ? p.row_masks[row] : p.agent_mask;
     float v8[8];
     gather(row, col, v8);
     if (gc < kw) {
@@ -182,11 +183,11 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         hi[2 * k] = h8[2 * k] * t4.x + v8[2 * k] * t4.y;
         hi[2 * k + 1] = h8[2 * k + 1] * t4.z + v8[2 * k + 1] * t4.w;
       }
-      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, lo);
-      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc + p.hd / 2, hi);
+      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, lo, mask);
+      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc + p.hd / 2, hi, mask);
       continue;
     }
-    store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8);
+    store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8, mask);
   }
   // nobody leaves while a peer may still read its partial tile
   asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");

@@ -18,7 +18,7 @@ states and queries), so its times are the KV-path share of a turn, not model lat
               tokens, the adapted one (agent j: its LR rows, and adapted base rows in private blocks that
               its block table splices in after the shared context) and the adapter-free one (neutral base
               rows into the shared cache, the other agents' LR rows).  Prefill runs both; every decode step
-              is two one-row projections and ONE attention launch of two requests (agent j and the
+              is ONE two-row projection (per-row agent masks) and ONE attention launch of two requests (agent j and the
               adapter-free view, each with its own block table).  Nothing is left to do after the turn.
 
 TTFT of a turn = its prefill phase (projection + prefill attention over all layers); the trace's TTFT is
@@ -183,11 +183,14 @@ def _replay_db(st: Stack, turns: Sequence[Turn]) -> Dict[str, float]:
         priv0 = st.shared_blocks * I.PAGE + P % I.PAGE                  # slot of position P in the private region
         slots_a = (priv0 + torch.arange(n, dtype=torch.int32)).to(dev)
 
+        slots_2n = torch.cat([slots_a, (P + torch.arange(n, dtype=torch.int32)).to(dev)])
+        masks_2n = torch.tensor([1 << j] * n + [others] * n, dtype=torch.int64, device=dev)
+
         def prefill_both():
             for l in range(st.n_layers):
                 k = st.w(l)
-                px.turn_project(st.desc, st.H[:n], st.WA[k], st.caches[l], 0, slots_a, 1 << j)      # adapted rows
-                px.turn_project(st.desc, st.H[:n], st.WA[k], st.caches[l], P, None, others)         # adapter-free rows
+                # adapted rows and adapter-free rows of the turn in ONE projection (per-row agent masks)
+                px.turn_project_rows(st.desc, st.H[:2 * n], st.WA[k], st.caches[l], slots_2n, masks_2n)
                 px.lr_attend_prefill(st.desc, st.q[:n], j, P, st.B_k[k], st.B_v[k], st.caches[l], st.out[:n], table_a)
                 px.lr_attend_prefill(st.desc, st.q[:n], -1, P, st.B_k[k], st.B_v[k], st.caches[l], st.out[:n])
 
@@ -201,17 +204,16 @@ def _replay_db(st: Stack, turns: Sequence[Turn]) -> Dict[str, float]:
             table2 = table2.to(dev)
             ctx = torch.full((2,), P + n + 1, dtype=torch.int32, device=dev)
             agent2 = torch.tensor([j, -1], dtype=torch.int32, device=dev)
-            slot_a = torch.tensor([priv0 + n], dtype=torch.int32, device=dev)
-            slot_n = torch.tensor([P + n], dtype=torch.int32, device=dev)
+            slot2 = torch.tensor([priv0 + n, P + n], dtype=torch.int32, device=dev)
+            mask2 = torch.tensor([1 << j, others], dtype=torch.int64, device=dev)
 
             def step():
                 for l in range(st.n_layers):
                     k = st.w(l)
-                    px.turn_project(st.desc, st.H[:1], st.WA[k], st.caches[l], 0, slot_a, 1 << j)
-                    px.turn_project(st.desc, st.H[1:2], st.WA[k], st.caches[l], 0, slot_n, others)
+                    px.turn_project_rows(st.desc, st.H[:2], st.WA[k], st.caches[l], slot2, mask2)
                     px.lr_attend_decode(st.desc, st.q[:2], agent2, ctx, max_ctx, st.B_k[k], st.B_v[k], st.caches[l], st.out[:2],
                                         st.ws, table2)
-                ctx.add_(1); slot_a.add_(1); slot_n.add_(1)
+                ctx.add_(1); slot2.add_(1)
 
             step()
             torch.cuda.synchronize()
@@ -285,7 +287,7 @@ def main(argv=None):
     traces = [round_robin_trace(n_agents)] if args.round_robin else [three_agent_trace(int(x)) for x in args.lengths.split(",")]
     for turns in traces:
         total = trace_tokens(turns)
-        rows = max(total, 64)                         # nonshared may prefill nearly the whole trajectory at once
+        rows = max(total, 64, 2 * max(t.n_in for t in turns))   # nonshared prefills nearly the whole trajectory at once; double batching 2 x n_in rows
         st = Stack(px, geo, args.layers, total + I.PAGE, rows, private_tokens=max(t.n_in + t.n_out for t in turns) + I.PAGE)
         for pol in args.policies.split(","):
             r = replay(st, turns, pol)

@@ -483,3 +483,31 @@ def test_prefill_short_turn_over_long_context_is_split_over_a_cluster(px, hd, n_
     ref = O.lr_prefill_reference(f64(qs), a, T, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"], sk, sv, n_kv,
                                  rows=rows)
     assert_close(f64(got), ref, f"split prefill hd{hd} T{T} S{S}")
+
+
+@pytest.mark.parametrize("n", [1, 10, 100])
+def test_per_row_agent_masks_equal_two_separate_projections(px, n):
+    """Double batching: adapted rows (current agent's LR rows, private slots) and adapter-free rows (the other
+    agents' LR rows, shared slots) in one fused projection, bit-equal to one call per sequence."""
+    geo = I.Geometry(256, 8, 2, 128, 3, 16, 16, alpha=32.0)
+    nb = 40
+    cur = 1
+    others = 0b111 & ~(1 << cur)
+    H_ad = I.hidden_states(n, geo, 81, f"db.ad{n}")
+    H_nt = I.hidden_states(n, geo, 81, f"db.nt{n}")
+    slots_ad = (20 * 16 + 3 + torch.arange(n)).to(torch.int32)          # private region, mid-page start
+    slots_nt = (5 * 16 + 3 + torch.arange(n)).to(torch.int32)
+    La = Layer(px, geo, seed=81, n_blocks=nb, fill=float("nan"))
+    dev = {k: v.cuda() for k, v in La.w.items()}
+    WA = px.pack_turn_weights(geo, dev["W_k"], dev["W_v"], dev["A_k"], dev["A_v"])
+    px.turn_project(La.desc, H_ad.cuda(), WA, La.cache, 0, slots_ad.cuda(), 1 << cur)
+    px.turn_project(La.desc, H_nt.cuda(), WA, La.cache, 0, slots_nt.cuda(), others)
+    Lb = Layer(px, geo, seed=81, n_blocks=nb, fill=float("nan"))
+    masks = torch.tensor([1 << cur] * n + [others] * n, dtype=torch.int64)
+    px.turn_project_rows(Lb.desc, torch.cat([H_ad, H_nt]).cuda(), WA, Lb.cache, torch.cat([slots_ad, slots_nt]).cuda(), masks.cuda())
+    torch.cuda.synchronize()
+    for name in ("k_base", "v_base", "lr_k", "lr_v"):
+        a, b = getattr(La.cache, name).view(torch.int16), getattr(Lb.cache, name).view(torch.int16)
+        assert torch.equal(a, b), name
+    assert not torch.isnan(Lb.cache.lr_k[cur].reshape(nb * 16, -1)[slots_ad.long()]).any()
+    assert torch.isnan(Lb.cache.lr_k[cur].reshape(nb * 16, -1)[slots_nt.long()]).all()      # the neutral rows left agent `cur` alone

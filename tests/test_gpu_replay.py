@@ -23,7 +23,7 @@ def test_replay_policies_small():
     geo = I.Geometry(d_model=256, n_q=8, n_kv=2, hd=64, n_agents=3, rank_k=16, rank_v=16, alpha=32.0)
     turns = [R.Turn(0, 70, 5), R.Turn(1, 200, 4), R.Turn(2, 33, 3), R.Turn(0, 64, 2)]
     total = R.trace_tokens(turns)
-    st = R.Stack(px, geo, n_layers=2, max_tokens=total + 16, max_rows=total, private_tokens=220)
+    st = R.Stack(px, geo, n_layers=2, max_tokens=total + 16, max_rows=2 * total, private_tokens=220)
     res = {p: R.replay(st, turns, p) for p in R.POLICIES}
     for p, r in res.items():
         assert r["tokens"] == total and r["ttft_ms"] > 0 and r["decode_ms"] > 0 and r["total_ms"] >= r["ttft_ms"]
