@@ -525,7 +525,7 @@ struct PrefillRun {
                 : make_map2(ctx, &mv, a.cache->v_base, kv_rows, HD, PAGE, 64);
     if (rc) return rc;
     mlk = mk; mlv = mv;     // placeholders when a rank is zero (never dereferenced)
-    if (RK) { rc = make_map2(ctx, &mlk, (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * lr_rows * RK, lr_rows, RK, box_rows, RK); if (rc) return rc; }
+    if (RK) { rc = make_map2(ctx, &mlk, (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * lr_rows * RK, lr_rows, RK, box_rows, C::RKP); if (rc) return rc; }
     if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, box_rows, 64); if (rc) return rc; }
     PrefillTcParams p;
     p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;

@@ -74,24 +74,25 @@ struct PrefillTcCfg {
   static constexpr int SLABS = HD / 64;                      // 64-column slabs of a base row
   static constexpr int SLAB_BYTES = PTC_TOK * 128;            // 128 rows x 128 bytes
   static constexpr int Q_BYTES = SLABS * SLAB_BYTES;
-  static constexpr int QX_BYTES = RK > 0 ? PTC_TOK * RK * 2 : 0;
+  static constexpr int RKP = RK == 8 ? 16 : RK;               // rank 8 rides as a zero-padded k step of 16
+  static constexpr int QX_BYTES = RK > 0 ? PTC_TOK * RKP * 2 : 0;
   static constexpr int KV_BYTES = SLABS * SLAB_BYTES;
-  static constexpr int LK_BYTES = PTC_TOK * RK * 2;
+  static constexpr int LK_BYTES = PTC_TOK * RKP * 2;
   static constexpr int LV_BYTES = PTC_TOK * RV * 2;
   static constexpr int KSTAGE = KV_BYTES + LK_BYTES;          // {K_base slabs | L_K} of 128 tokens
   static constexpr int VSLABS = SLABS + (RV > 0 ? 1 : 0);     // L_V rides as one more 64-column slab (zero padded)
   static constexpr int OW = VSLABS * 64;                      // columns of O' in TMEM: [O | U | padding]
   static constexpr int VSTAGE = VSLABS * SLAB_BYTES;          // {V_base slabs | L_V slab}
-  static constexpr int K_PAGE_TX = PAGE * (HD + RK) * 2;      // bytes one page contributes to a key stage
+  static constexpr int K_PAGE_TX = PAGE * (HD + RKP) * 2;      // bytes one page contributes to a key stage
   static constexpr int V_PAGE_TX = PAGE * VSLABS * 128;
-  static constexpr int SPLIT_XS = HD + RV + 4;                // row stride (floats) of a partial in shared memory
+  static constexpr int SPLIT_XS = (HD + RV + 15) / 16 * 16 + 4;                // row stride (floats) of a partial in shared memory
   // split-context merge area (laid over the rings): partial | m | l | merged rows | weights | 1/l | B_v slice
   static constexpr int SPLIT_BYTES = (128 * SPLIT_XS + 256 + 64 * SPLIT_XS + 16 * 64 + 64) * 4 + RV * HD * 2;
   static constexpr bool L_IN_MMA = RV > 0 && RV < 64;         // a spare column of the L_V slab carries the denominator
   static constexpr int TMEM_P = 2 * PTC_TOK;                  // packed bf16 P (64 columns) after the two S buffers
   static constexpr int TMEM_O = TMEM_P + PTC_TOK / 2;         // O' (at most 192 columns): 320 + 192 = 512
   __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 320 + 2 * PTC_PARTS_MAX * 512 + 1024; }
-  static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 16 || RK == 32) && (RV == 0 || RV == 16 || RV == 32);
+  static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 8 || RK == 16 || RK == 32) && (RV == 0 || RV == 8 || RV == 16 || RV == 32);
 };
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
@@ -278,7 +279,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         if (is_k) {
 #pragma unroll
           for (int sl = 0; sl < C::SLABS; ++sl) tma_load_2d(st + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_k, sl * 64, row_kv, full);
-          if constexpr (RK > 0) tma_load_2d(st + C::KV_BYTES + lane * PAGE * RK * 2, &map_lk, 0, ph * PAGE, full);
+          if constexpr (RK > 0) tma_load_2d(st + C::KV_BYTES + lane * PAGE * C::RKP * 2, &map_lk, 0, ph * PAGE, full);
         } else {
 #pragma unroll
           for (int sl = 0; sl < C::SLABS; ++sl) tma_load_2d(st + sl * C::SLAB_BYTES + lane * PAGE * 128, &map_v, sl * 64, row_kv, full);
@@ -295,9 +296,9 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // stage, slab or k-step is one 64-bit add of a small constant).
     const uint32_t id_s = umma_idesc(PTC_TOK, 0);
     const uint64_t qd0 = umma_desc_kmajor(q_u32, 128);
-    const uint64_t qxd0 = RK > 0 ? umma_desc_kmajor(qx_u32, RK * 2) : 0;
+    const uint64_t qxd0 = RK > 0 ? umma_desc_kmajor(qx_u32, C::RKP * 2) : 0;
     const uint64_t kd0 = umma_desc_kmajor(kring_u32, 128);
-    const uint64_t lkd0 = RK > 0 ? umma_desc_kmajor(kring_u32 + C::KV_BYTES, RK * 2) : 0;
+    const uint64_t lkd0 = RK > 0 ? umma_desc_kmajor(kring_u32 + C::KV_BYTES, C::RKP * 2) : 0;
     mbar_wait(q_ready, 0, p.status);
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j % KS;
@@ -317,7 +318,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         }
         if constexpr (RK > 0) {
 #pragma unroll
-          for (int ks = 0; ks < RK / 16; ++ks) umma_bf16(d, qxd0 + (uint64_t)(ks * 2), lkd0 + so + (uint64_t)(ks * 2), id_s, 1u);
+          for (int ks = 0; ks < C::RKP / 16; ++ks) umma_bf16(d, qxd0 + (uint64_t)(ks * 2), lkd0 + so + (uint64_t)(ks * 2), id_s, 1u);
         }
         umma_commit(k_empty + 8 * s);            // the key stage is free as soon as S is computed
         umma_commit(s_full + 8 * (j & 1));
@@ -415,7 +416,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       }
       asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");      // B_k slice and the Q tile are visible
       if constexpr (RK > 0) {
-        constexpr int CPR = RK / 8;
+        constexpr int CPR = C::RKP / 8;
 #pragma unroll 1
         for (int j0 = part * 8; j0 < RK; j0 += NP * 8) {           // this thread folds coordinates j0 .. j0+7
           float acc[8];
@@ -440,6 +441,10 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, j0 / 8)) =
               make_uint4(pack_bf16(acc[0] * p.s_k, acc[1] * p.s_k), pack_bf16(acc[2] * p.s_k, acc[3] * p.s_k),
                          pack_bf16(acc[4] * p.s_k, acc[5] * p.s_k), pack_bf16(acc[6] * p.s_k, acc[7] * p.s_k));
+        }
+        // rank 8: the upper half of the padded k step is zero on the query side (the key side is zero-filled by TMA)
+        if constexpr (C::RKP > RK) {
+          if (part == 0) *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, 1)) = make_uint4(0u, 0u, 0u, 0u);
         }
       }
     }
@@ -596,10 +601,10 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         uint32_t lv16[16];
         tmem_ld16(lane_addr + C::TMEM_O + HD + (RV / 16) * 16, lv16);
         tmem_wait_ld();
-        l_loc = __uint_as_float(lv16[0]);
+        l_loc = __uint_as_float(lv16[RV % 16]);
       }
 #pragma unroll 1
-      for (int c = part; c < (HD + RV) / 16; c += NP) {
+      for (int c = part; c < (HD + RV + 15) / 16; c += NP) {
         uint32_t ov[16];
         if (n_tiles > 0) {
           tmem_ld16(lane_addr + C::TMEM_O + c * 16, ov);
@@ -627,9 +632,9 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     float l_tot = 0.f;
     if constexpr (C::L_IN_MMA) {
       uint32_t lv16[16];
-      tmem_ld16(lane_addr + C::TMEM_O + HD + (RV / 16) * 16, lv16);   // RV is a multiple of 16: column HD + RV leads its chunk
+      tmem_ld16(lane_addr + C::TMEM_O + HD + (RV / 16) * 16, lv16);   // column HD + RV sits at index RV % 16 of its chunk
       tmem_wait_ld();
-      l_tot = __uint_as_float(lv16[0]);
+      l_tot = __uint_as_float(lv16[RV % 16]);
     } else {
 #pragma unroll
       for (int q2 = 0; q2 < NP; ++q2) l_tot += xch[q2 * 128 + row];
@@ -639,11 +644,12 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     if constexpr (RV > 0) {
       uint32_t uv[16];
 #pragma unroll
-      for (int c = 0; c < RV / 16; ++c) {
+      for (int c = 0; c < (RV + 15) / 16; ++c) {
         tmem_ld16(lane_addr + C::TMEM_O + HD + c * 16, uv);
         tmem_wait_ld();
 #pragma unroll
-        for (int k = 0; k < 16; ++k) u[c * 16 + k] = __uint_as_float(uv[k]) * p.s_v;
+        for (int k = 0; k < 16; ++k)
+          if (c * 16 + k < RV) u[c * 16 + k] = __uint_as_float(uv[k]) * p.s_v;
       }
     }
     __nv_bfloat16* orow = p.out + ((size_t)i_new * p.n_q + (size_t)g * G + hg) * HD;
