@@ -589,7 +589,7 @@ struct PrefillRun {
     }
     return run_simple<false>(ctx, a);
   }
-  // mma.sync kernel: ranks 8 and 64, oversized or unaligned caches, and the rotary variant
+  // mma.sync kernel: rank 64, oversized or unaligned caches, and the rotary variant
   template <bool ROPE = false>
   static int32_t run_simple(precc_ctx* ctx, const PrefillArgs& a) {
     using C = PrefillCfg<HD, RK, RV>;
