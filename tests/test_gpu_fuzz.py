@@ -1,0 +1,117 @@
+"""Seeded random shapes: head_dim, group size, kv heads, ranks, agents, batch, context lengths (ragged, around
+page and tile boundaries), paged or contiguous caches, adapter-free requests mixed in.  Decode and prefill
+over directly filled caches against the oracle's cache-content form."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lrkv_oracle as O
+from paper_2609_34054_b200 import inputs as I
+from paper_2609_34054_b200.binding import Cache, Precc, layer_desc
+
+from harness import assert_close, f64
+
+pytestmark = pytest.mark.gpu
+
+N_CASES = 36
+
+
+def _case(i: int):
+    rng = np.random.default_rng(1000 + i)
+    hd = int(rng.choice([64, 128]))
+    G = int(rng.choice([1, 2, 4, 7, 8]))
+    n_kv = int(rng.choice([1, 2, 3, 5]))
+    r = int(rng.choice([0, 8, 16, 32, 64]))
+    rk = r if rng.random() < 0.7 else 0
+    N = int(rng.integers(1, 5))
+    B = int(rng.integers(1, 6))
+    edge = [1, 15, 16, 17, 127, 128, 129, 255, 257]
+    ctx = [int(rng.choice(edge)) if rng.random() < 0.3 else int(rng.integers(1, 900)) for _ in range(B)]
+    if i % 6 == 0:
+        ctx[0] = int(rng.integers(3000, 6000))          # long enough for the split paths
+    agents = [int(rng.integers(-1, N)) for _ in range(B)]
+    paged = bool(rng.random() < 0.5)
+    S = int(rng.integers(1, 90))
+    T = int(rng.integers(0, 700)) if i % 5 else int(rng.integers(2000, 5000))
+    return hd, G, n_kv, rk, r, N, B, ctx, agents, paged, S, T
+
+
+@pytest.fixture(scope="module")
+def px():
+    p = Precc(0)
+    yield p
+    assert p.poll_status() == 0
+    p.close()
+
+
+@pytest.mark.parametrize("i", range(N_CASES))
+def test_random_shapes(px, i):
+    hd, G, n_kv, rk, rv, N, B, ctx, agents, paged, S, T = _case(i)
+    geo = I.Geometry(d_model=64, n_q=G * n_kv, n_kv=n_kv, hd=hd, n_agents=N, rank_k=rk, rank_v=rv, alpha=2.0 * max(rv, 1))
+    desc = layer_desc(geo)
+    need = [(c + 15) // 16 for c in ctx]
+    pool = sum(need) + 3
+    c = I.direct_caches(pool, geo, 100 + i, f"fz{i}")
+    dev = lambda t: None if t is None else t.cuda()
+    cache = Cache.from_tensors(geo, c["k_base"].cuda(), c["v_base"].cuda(), dev(c.get("lr_k")), dev(c.get("lr_v")))
+    w = I.layer_weights(geo, 100 + i, f"fz{i}")
+    Bk = w["B_k"].cuda() if rk else None
+    Bv = w["B_v"].cuda() if rv else None
+    # ---------------------------------------------------------------- decode
+    perm = I.permutation(pool, 100 + i, f"fz.perm{i}")
+    table = torch.zeros((B, max(need)), dtype=torch.int32)
+    first, at = [], 0
+    for b, n in enumerate(need):
+        table[b, :n] = perm[at:at + n] if paged else torch.arange(at, at + n)
+        first.append(at)
+        at += n
+    q = I.queries(B, geo, 100 + i, f"fz.q{i}", gain=3.0)
+    out = torch.full_like(q, float("nan"), device="cuda")
+    mx = max(ctx)
+    ws = px.decode_workspace(desc, B, mx)
+    px.lr_attend_decode(desc, q.cuda(), torch.tensor(agents, dtype=torch.int32).cuda(), torch.tensor(ctx, dtype=torch.int32).cuda(),
+                        mx, Bk, Bv, cache, out, ws, table.cuda() if paged else None,
+                        None if paged else torch.tensor(first, dtype=torch.int32).cuda())
+    torch.cuda.synchronize()
+    out = f64(out)
+
+    def rows(x, b, t):
+        blocks = table[b, :need[b]].long()
+        return f64(x[blocks].reshape(-1, x.shape[-1]))[:t]
+
+    def base_rows_of(x, b, t):                              # [blocks, n_kv, 16, hd] -> [t, n_kv*hd]
+        blocks = table[b, :need[b]].long()
+        return f64(x[blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))[:t]
+
+    zero_k = np.zeros((rk, n_kv * hd)); zero_v = np.zeros((rv, n_kv * hd))
+    for b in range(B):
+        t, a = ctx[b], agents[b]
+        Lk = rows(c["lr_k"][max(a, 0)], b, t) if rk else np.zeros((t, 0))
+        Lv = rows(c["lr_v"][max(a, 0)], b, t) if rv else np.zeros((t, 0))
+        Bk_a = f64(w["B_k"][a]) if (rk and a >= 0) else zero_k
+        Bv_a = f64(w["B_v"][a]) if (rv and a >= 0) else zero_v
+        ref = O.attend_from_caches(f64(q[b]), base_rows_of(c["k_base"], b, t), base_rows_of(c["v_base"], b, t), Lk, Lv, Bk_a, Bv_a,
+                                   geo.scale_k, geo.scale_v, n_kv)
+        assert_close(out[b], ref, f"case {i} decode request {b} (hd{hd} G{G} kv{n_kv} r{rk}/{rv} ctx{t} agent{a} paged={paged})")
+    # ---------------------------------------------------------------- prefill over a second, contiguous-or-paged sequence
+    nb2 = (T + S + 15) // 16
+    c2 = I.direct_caches(nb2 + 2, geo, 200 + i, f"fzp{i}")
+    cache2 = Cache.from_tensors(geo, c2["k_base"].cuda(), c2["v_base"].cuda(), dev(c2.get("lr_k")), dev(c2.get("lr_v")))
+    tab2 = I.permutation(nb2 + 2, 200 + i, f"fzp.perm{i}")[:nb2].to(torch.int32) if paged else torch.arange(1, nb2 + 1, dtype=torch.int32)
+    agent = agents[0]
+    qs = I.queries(S, geo, 200 + i, f"fzp.q{i}", gain=3.0)
+    outp = torch.full_like(qs, float("nan"), device="cuda")
+    px.lr_attend_prefill(desc, qs.cuda(), agent, T, Bk, Bv, cache2, outp, tab2.cuda() if paged else None, 0 if paged else 1)
+    torch.cuda.synchronize()
+    outp = f64(outp)
+    blocks = tab2.long()
+    kb = f64(c2["k_base"][blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))
+    vb = f64(c2["v_base"][blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))
+    Lk2 = f64(c2["lr_k"][max(agent, 0)][blocks].reshape(-1, rk)) if rk else np.zeros((nb2 * 16, 0))
+    Lv2 = f64(c2["lr_v"][max(agent, 0)][blocks].reshape(-1, rv)) if rv else np.zeros((nb2 * 16, 0))
+    Bk_a = f64(w["B_k"][agent]) if (rk and agent >= 0) else zero_k
+    Bv_a = f64(w["B_v"][agent]) if (rv and agent >= 0) else zero_v
+    for srow in sorted(set([0, S // 2, S - 1])):
+        t = T + srow + 1
+        ref = O.attend_from_caches(f64(qs[srow]), kb[:t], vb[:t], Lk2[:t], Lv2[:t], Bk_a, Bv_a, geo.scale_k, geo.scale_v, n_kv)
+        assert_close(outp[srow], ref, f"case {i} prefill row {srow} (hd{hd} G{G} kv{n_kv} r{rk}/{rv} T{T} S{S} agent{agent} paged={paged})")
