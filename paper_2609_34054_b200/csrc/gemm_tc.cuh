@@ -26,6 +26,7 @@ namespace precc {
 struct GemmParams {
   int M, N_out, K;
   int BN, stages, tmem_cols;
+  int spread_rows;                // 1: even row-tile spreading allowed (rows may be written twice, identically)
   int mode;                       // 0 = LR caches, 1 = base caches, 2 = base columns then LR columns
   const int32_t* slot_mapping;    // [M] or null
   int64_t start_slot;
@@ -178,7 +179,19 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb = p.K / GEMM_BK;
   const int n_tiles_n = (p.N_out + p.BN - 1) / p.BN;
-  const int n_tiles = ((p.M + GEMM_BM - 1) / GEMM_BM) * n_tiles_n;
+  // Row tiles.  With a single column tile the kernel is HBM-bound on X, and a row-tile count that is not a
+  // multiple of the grid leaves part of the machine idle in the last round (256 tiles on 148 blocks = 1.73
+  // rounds).  Then the count is rounded up to a multiple of the grid and the tiles are spread evenly over
+  // the rows: neighbours overlap by a few rows, which are computed twice with identical results (the
+  // overlap is re-read from L2, not from DRAM), and every block streams the same number of rows.
+  const int m_plain = (p.M + GEMM_BM - 1) / GEMM_BM;
+  const bool spread = p.spread_rows && n_tiles_n == 1 && m_plain > (int)gridDim.x && p.M >= GEMM_BM;
+  const int m_tiles = spread ? ((m_plain + (int)gridDim.x - 1) / (int)gridDim.x) * (int)gridDim.x : m_plain;
+  const int n_tiles = m_tiles * n_tiles_n;
+  auto row0_of = [&](int mt) -> int {
+    if (!spread) return mt * GEMM_BM;
+    return (int)(((long long)mt * (p.M - GEMM_BM)) / (m_tiles - 1));   // first tile at 0, last one ends at M
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -204,7 +217,7 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (lane == 0) {
       int it = 0;
       for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-        const int m0 = (t / n_tiles_n) * GEMM_BM, n0 = (t % n_tiles_n) * p.BN;
+        const int m0 = row0_of(t / n_tiles_n), n0 = (t % n_tiles_n) * p.BN;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % p.stages;
           if (it >= p.stages) mbar_wait(empty0 + 8 * s, ((it / p.stages) - 1) & 1, p.status);
@@ -247,7 +260,7 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     int i = 0;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
       const int buf = i & 1;
-      const int m0 = (t / n_tiles_n) * GEMM_BM, n0 = (t % n_tiles_n) * p.BN;
+      const int m0 = row0_of(t / n_tiles_n), n0 = (t % n_tiles_n) * p.BN;
       const int gm = m0 + row;
       bool row_ok = gm < p.M;
       long long slot = 0;

@@ -230,6 +230,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   rc = make_map_w(ctx, &map_w, Wt, n_out, K, bn);
   if (rc) return rc;
   gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
+  gp.spread_rows = 1;
   gp.status = ctx->status;
   PRECC_CUDA(ctx, cudaFuncSetAttribute(proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const int total_tiles = m_tiles * n_tiles;
