@@ -29,6 +29,7 @@ struct precc_ctx {
   bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
   bool force_tiled_gemm = false;       // PRECC_GEMM=tiled in the environment: never take the few-row kernel
   bool deep_clusters = true;           // PRECC_DEEP=0 in the environment: never use the one-block-per-SM deep-ring clusters
+  bool prefill_forward = false;        // PRECC_PREFILL_ORDER=forward: row tiles in ascending order (default: longest causal reach first)
   bool no_prefill_split = false;       // PRECC_PREFILL_SPLIT=0 in the environment: never split a turn's context over a cluster
   char err[512] = {0};
   CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -534,6 +535,7 @@ struct PrefillRun {
     p.B_v = RV ? (const __nv_bfloat16*)a.B_v + (size_t)a.agent * RV * kvw : nullptr;
     p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
     p.S = a.S; p.T = a.T; p.first_block = a.first_block; p.contig = contig ? 1 : 0;
+    p.longest_first = ctx->prefill_forward ? 0 : 1;
     p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.k_stages = ks; p.v_stages = vs;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
     p.trace = (ctx->trace && ctx->trace_blocks >= 32) ? ctx->trace : nullptr;
@@ -690,6 +692,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   if (const char* v = getenv("PRECC_PREFILL")) ctx->force_simple_prefill = (strcmp(v, "simple") == 0);
   if (const char* v = getenv("PRECC_GEMM")) ctx->force_tiled_gemm = (strcmp(v, "tiled") == 0);
   if (const char* v = getenv("PRECC_DEEP")) ctx->deep_clusters = (strcmp(v, "0") != 0);
+  if (const char* v = getenv("PRECC_PREFILL_ORDER")) ctx->prefill_forward = (strcmp(v, "forward") == 0);
   if (const char* v = getenv("PRECC_PREFILL_SPLIT")) ctx->no_prefill_split = (strcmp(v, "0") == 0);
   if (e != cudaSuccess) {
     fprintf(stderr, "precc_create: %s\n", cudaGetErrorString(e));

@@ -79,7 +79,8 @@ lr_attend_prefill_kernel(const PrefillParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.y;
   const int G = p.group;
-  const int row0 = blockIdx.x * PF_ROWS;      // first (token, head) row of this block
+  // block x = 0 takes the LAST row tile: blocks with the longest causal reach start first, the grid's tail is short blocks
+  const int row0 = (int)(gridDim.x - 1 - blockIdx.x) * PF_ROWS;      // first (token, head) row of this block
   const int n_rows = p.S * G;
 
   const uint32_t q_u32 = smem_u32(smem);

@@ -47,6 +47,7 @@ struct PrefillTcParams {
   int tok_per_tile;            // 128 / group
   int k_stages, v_stages;      // depth of the key ring and of the value ring
   int contig;                  // 1: no block table; the tensor maps fetch a whole 128-token stage per box
+  int longest_first;           // 1: block x = 0 takes the LAST row tile (longest causal reach), so the tail of the grid is short blocks
   float scale_log2, s_k, s_v;
   unsigned long long* trace;   // PRECC_PF_TRACE builds only: [steps][16] clock stamps of block (0, 0)
 };
@@ -199,7 +200,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.y, G = p.group;
-  const int tok0 = blockIdx.x * p.tok_per_tile;
+  const int tok0 = (p.longest_first ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x) * p.tok_per_tile;
   const int n_tok = min(p.tok_per_tile, p.S - tok0);             // new tokens handled by this block
   const int t_end = p.T + tok0 + n_tok;                          // context + causal reach of the last row
   const int full_vis = p.T + tok0 + 1;                           // tokens visible to every row of the block
