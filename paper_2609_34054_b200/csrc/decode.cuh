@@ -735,10 +735,9 @@ __device__ __forceinline__ float dsmem_ld(uint32_t addr) {
   asm volatile("ld.shared::cluster.f32 %0, [%1];\n" : "=f"(v) : "r"(addr) : "memory");
   return v;
 }
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
-}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_sync_all() { cluster_arrive(); cluster_wait(); }
 
 template <int HD, int RK, int RV, int NW, bool ROPE = false>
 __global__ void __launch_bounds__(NW * 32, (NW == 8 && HD == 64) ? 2 : 1)   // 16-block clusters need two blocks per SM
@@ -801,6 +800,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   const int cols = (HD + CS - 1) / CS;                  // output columns finished by a block (stride of the slices)
   const int c0 = rank * cols;
   const int ncol = max(0, min(cols, HD - c0));          // columns this block really owns
+  cluster_arrive();                                     // this block's result is complete (the stream ends with a block barrier)
   if constexpr (RV > 0) {                               // B_v column slice (bv_pre was requested before the stream)
     for (int k = 0; k < BV_PER_THREAD; ++k) {
       const int i = threadIdx.x + k * NT;
@@ -808,7 +808,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     }
   }
   mark(6);
-  cluster_sync_all();                                   // every block's result is complete and visible
+  cluster_wait();                                       // every block's result is complete and visible
   __shared__ float fin_m[8];
   // One pass over distributed shared memory: a thread owns one merged element (for every h < G my
   // `cols` base columns and all r_v LR-V coordinates, plus the denominators) and reads the peers'
@@ -837,6 +837,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     if (is_l) fin_m[h] = M;
   }
   __syncthreads();
+  cluster_arrive();                                     // this block has finished reading its peers; the wait is at the exit
   mark(10);
   const float* fin_l = mine + 8 * (HD + RV);
   if (p.raw) {
@@ -856,7 +857,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
       }
     }
     mark(7);
-    cluster_sync_all();                                 // nobody leaves while a peer may still read its result
+    cluster_wait();                                     // nobody leaves while a peer may still read its result
     return;
   }
   for (int e = threadIdx.x; e < G * cols; e += NT) {
@@ -872,7 +873,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     out_bg[h * HD + c0 + c] = __float2bfloat16(v / fin_l[h]);
   }
   mark(7);
-  cluster_sync_all();                                   // nobody leaves while a peer may still read its result
+  cluster_wait();                                       // nobody leaves while a peer may still read its result
 }
 
 }  // namespace precc
