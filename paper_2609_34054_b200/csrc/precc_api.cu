@@ -379,6 +379,19 @@ struct DecodeRunT {
     return best;
   }
   // Can `need` clusters of `cs` blocks be resident at once?  Asked once per (shape, warps, cluster size).
+  // The cluster kernel's shared-memory limit is only ever raised: the two ring layouts of one shape (two blocks
+  // per SM / one block per SM) need different amounts, and lowering the attribute for the smaller one would
+  // make a later launch of the larger one fail.
+  template <int NW>
+  static cudaError_t ensure_cluster_smem(int bytes) {
+    static int have = 0;
+    if (bytes <= have) return cudaSuccess;
+    auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e == cudaSuccess) have = bytes;
+    return e;
+  }
   template <int NW>
   static bool cluster_fits(precc_ctx* ctx, const DecodePlan& pl, int need) {
     static int cache2[2][DEC_MAX_CLUSTER + 1] = {{0}};  // 0 = unknown, else max active clusters + 1
@@ -386,8 +399,7 @@ struct DecodeRunT {
     if (cached[pl.cluster] == 0) {
       auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
       int n = 0;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess ||
-          cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+      if (ensure_cluster_smem<NW>(pl.smem) != cudaSuccess) {
         cudaGetLastError();
         cached[pl.cluster] = 1;
         return false;
@@ -454,8 +466,13 @@ struct DecodeRunT {
       attr[1].id = cudaLaunchAttributeClusterDimension;
       attr[1].val.clusterDim.x = pl.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
       cfg.numAttrs = 2;
-      if (pl.warps == 8) PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 8, ROPE>, p));
-      else PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 4, ROPE>, p));
+      if (pl.warps == 8) {
+        PRECC_CUDA(ctx, ensure_cluster_smem<8>(pl.smem));
+        PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 8, ROPE>, p));
+      } else {
+        PRECC_CUDA(ctx, ensure_cluster_smem<4>(pl.smem));
+        PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 4, ROPE>, p));
+      }
     } else {
       auto kern = lr_attend_decode_kernel<HD, RK, RV, ROPE>;
       cfg.blockDim = dim3(DEC_WARPS * 32);

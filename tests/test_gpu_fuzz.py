@@ -1,6 +1,8 @@
 """Seeded random shapes: head_dim, group size, kv heads, ranks, agents, batch, context lengths (ragged, around
 page and tile boundaries), paged or contiguous caches, adapter-free requests mixed in.  Decode and prefill
 over directly filled caches against the oracle's cache-content form."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -13,7 +15,7 @@ from harness import assert_close, f64
 
 pytestmark = pytest.mark.gpu
 
-N_CASES = 36
+N_CASES = int(os.environ.get("PRECC_FUZZ_CASES", "36"))      # a longer soak: PRECC_FUZZ_CASES=400
 
 
 def _case(i: int):

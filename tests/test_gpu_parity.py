@@ -533,3 +533,22 @@ def test_mma_sync_prefill_kernel_matches_too(monkeypatch, hd, r):
     assert_close(got, ref, f"mma.sync prefill hd{hd} r{r}")
     assert px2.poll_status() == 0
     px2.close()
+
+
+def test_decode_alternating_between_ring_layouts_of_one_shape(px):
+    """A long context takes the one-block-per-SM ring layout of the cluster kernel, a short one the
+    two-blocks-per-SM layout of the same kernel; going back and forth must keep working (the kernel's
+    shared-memory limit may only grow)."""
+    geo = I.Geometry(128, 6, 2, 64, 2, 0, 8, alpha=16.0)
+    T = 5200
+    L = Layer(px, geo, seed=63, n_blocks=(T + 15) // 16, tag="alt")
+    H = I.hidden_states(T, geo, 63, "alt.H")
+    L.append(H)
+    q = I.queries(1, geo, 63, "alt.q", gain=3.0)
+    w = L.w_np
+    args = (f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"])
+    for ctx in (T, 600, T - 3, 777, 4100, 290):
+        got = f64(L.decode(q, [1], [ctx]))
+        ref = O.lr_decode_reference(f64(q), [1], [ctx], *args, geo.scale_k, geo.scale_v, geo.n_kv)
+        assert_close(got, ref, f"alternating layouts, ctx {ctx}")
+    assert px.poll_status() == 0
