@@ -117,3 +117,111 @@ def test_random_shapes(px, i):
         t = T + srow + 1
         ref = O.attend_from_caches(f64(qs[srow]), kb[:t], vb[:t], Lk2[:t], Lv2[:t], Bk_a, Bv_a, geo.scale_k, geo.scale_v, n_kv)
         assert_close(outp[srow], ref, f"case {i} prefill row {srow} (hd{hd} G{G} kv{n_kv} r{rk}/{rv} T{T} S{S} agent{agent} paged={paged})")
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Projections and the rotary path, through the library's own calls (hidden states -> caches -> attention)
+
+from harness import Layer, base_rows, lr_rows                     # noqa: E402
+from paper_2609_34054_b200.binding import rope_table              # noqa: E402
+
+N_PROJ = max(12, N_CASES // 3)
+
+
+def _proj_case(i: int):
+    rng = np.random.default_rng(5000 + i)
+    d = int(rng.choice([64, 128, 192, 320, 1024]))
+    hd = int(rng.choice([64, 128]))
+    n_kv = int(rng.choice([1, 2, 3]))
+    r = int(rng.choice([8, 16, 32, 64]))
+    N = int(rng.integers(1, 6))
+    kind = int(rng.integers(0, 4))
+    M = [int(rng.integers(1, 65)), int(rng.integers(65, 400)), int(rng.integers(400, 1500)),
+         int(rng.choice([1, 16, 17, 64, 65, 127, 128, 129, 256]))][kind]
+    scattered = bool(rng.random() < 0.5)
+    mask = int(rng.integers(1, 1 << N))
+    return d, hd, n_kv, r, N, M, scattered, mask
+
+
+@pytest.mark.parametrize("i", range(N_PROJ))
+def test_random_projections(px, i):
+    """rebase_project + lr_precompute against the definition on every row; the fused turn_project bit-equal
+    to the two separate calls; masked-out agents and unaddressed slots untouched."""
+    d, hd, n_kv, r, N, M, scattered, mask = _proj_case(i)
+    geo = I.Geometry(d, 2 * n_kv, n_kv, hd, N, r, r, alpha=2.0 * r)
+    H = I.hidden_states(M, geo, seed=300 + i, tag=f"pz{i}")
+    nb = (M + 15) // 16 + 3
+    start = 5 if not scattered else 0
+    slots = I.permutation(nb * 16, 300 + i, f"pz.slots{i}")[:M].to(torch.int32) if scattered else None
+    La = Layer(px, geo, seed=300 + i, n_blocks=nb, fill=float("nan"), tag=f"pz{i}")
+    La.append(H, start_slot=start, slot_mapping=None if slots is None else slots.cuda(), agent_mask=mask)
+    torch.cuda.synchronize()
+    sl = slots.long() if scattered else torch.arange(start, start + M)
+    w, Hn = La.w_np, f64(H)
+    tol = lambda ref: 2.0 ** -8 * np.abs(ref) + 2e-3 * np.sqrt(d / 256)
+    for got, ref in ((base_rows(La.cache.k_base)[sl], O.base_cache(Hn, w["W_k"])),
+                     (base_rows(La.cache.v_base)[sl], O.base_cache(Hn, w["W_v"]))):
+        assert (np.abs(got - ref) <= tol(ref)).all(), f"case {i} base (d{d} hd{hd} kv{n_kv} M{M})"
+    for a in range(N):
+        if mask >> a & 1:
+            for name, A in (("lr_k", w["A_k"]), ("lr_v", w["A_v"])):
+                got, ref = lr_rows(getattr(La.cache, name), a)[sl], O.lr_cache(Hn, A[a])
+                assert (np.abs(got - ref) <= tol(ref)).all(), f"case {i} {name}[{a}] (d{d} r{r} M{M})"
+        else:
+            assert torch.isnan(La.cache.lr_k[a]).all() and torch.isnan(La.cache.lr_v[a]).all(), f"case {i}: masked agent {a} written"
+    untouched = torch.ones(nb * 16, dtype=torch.bool); untouched[sl] = False
+    assert torch.isnan(La.cache.k_base.permute(0, 2, 1, 3).reshape(nb * 16, -1)[untouched]).all()
+    Lb = Layer(px, geo, seed=300 + i, n_blocks=nb, fill=float("nan"), tag=f"pz{i}")
+    dev = {k: v.cuda() for k, v in Lb.w.items()}
+    WA = px.pack_turn_weights(geo, dev["W_k"], dev["W_v"], dev["A_k"], dev["A_v"])
+    px.turn_project(Lb.desc, H.cuda(), WA, Lb.cache, start, None if slots is None else slots.cuda(), mask)
+    torch.cuda.synchronize()
+    for name in ("k_base", "v_base", "lr_k", "lr_v"):
+        a_, b_ = getattr(La.cache, name).view(torch.int16), getattr(Lb.cache, name).view(torch.int16)
+        assert torch.equal(a_, b_), f"case {i}: fused projection differs in {name}"
+
+
+def _rope_case(i: int):
+    rng = np.random.default_rng(9000 + i)
+    hd = int(rng.choice([64, 128]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    n_kv = int(rng.choice([1, 2, 3]))
+    r = int(rng.choice([8, 16, 32, 64]))
+    T = int(rng.integers(1, 700)) if i % 4 else int(rng.integers(1500, 2600))
+    S = int(rng.integers(1, 60))
+    B = int(rng.integers(1, 4))
+    ctx = [T + S] + [int(rng.integers(1, T + S + 1)) for _ in range(B - 1)]
+    agents = [int(rng.integers(-1, 2)) for _ in range(B)]
+    return hd, G, n_kv, r, T, S, ctx, agents
+
+
+@pytest.mark.parametrize("i", range(N_PROJ))
+def test_random_rope_shapes(px, i):
+    """Rotary keys end to end: rotated base projection, un-rotated LR rows, rotary decode and prefill against
+    the oracle's definition (adapted key = rotation of the full-width adapted projection)."""
+    hd, G, n_kv, r, T, S, ctx, agents = _rope_case(i)
+    geo = I.Geometry(d_model=128, n_q=G * n_kv, n_kv=n_kv, hd=hd, n_agents=2, rank_k=r, rank_v=r, alpha=2.0 * r)
+    L = Layer(px, geo, seed=600 + i, n_blocks=(T + S + 15) // 16, tag=f"rz{i}")
+    H = I.hidden_states(T + S, geo, 600 + i, f"rz.H{i}")
+    table = rope_table(T + S + 1, hd)
+    cos, sin = O.rope_tables(T + S + 1, hd)
+    px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0)
+    px.lr_precompute(L.desc, H.cuda(), L.A_packed, L.cache, 0)
+    w = L.w_np
+    args = (f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"])
+    q = I.queries(len(ctx), geo, 600 + i, f"rz.q{i}", gain=3.0)
+    out = torch.full_like(q, float("nan"), device="cuda")
+    ws = px.decode_workspace(L.desc, len(ctx), max(ctx))
+    px.lr_attend_decode_rope(L.desc, q.cuda(), torch.tensor(agents, dtype=torch.int32).cuda(), torch.tensor(ctx, dtype=torch.int32).cuda(),
+                             max(ctx), L.B_k, L.B_v, table, L.cache, out, ws)
+    torch.cuda.synchronize()
+    adapted = O.lr_decode_reference_rope(f64(q), [max(a, 0) for a in agents], ctx, *args, geo.scale_k, geo.scale_v, n_kv, cos, sin)
+    neutral = O.lr_decode_reference_rope(f64(q), [0] * len(ctx), ctx, *args, 0.0, 0.0, n_kv, cos, sin)
+    ref = np.where(np.array(agents)[:, None, None] < 0, neutral, adapted)
+    assert_close(f64(out), ref, f"case {i} rope decode (hd{hd} G{G} kv{n_kv} r{r} ctx{ctx} agents{agents})")
+    qs = I.queries(S, geo, 600 + i, f"rz.qs{i}", gain=3.0)
+    outp = torch.full_like(qs, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope(L.desc, qs.cuda(), 1, T, L.B_k, L.B_v, table, L.cache, outp)
+    torch.cuda.synchronize()
+    refp = O.lr_prefill_reference_rope(f64(qs), 1, T, *args, geo.scale_k, geo.scale_v, n_kv, cos, sin)
+    assert_close(f64(outp), refp, f"case {i} rope prefill (hd{hd} G{G} kv{n_kv} r{r} T{T} S{S})")
