@@ -86,6 +86,7 @@ def test_random_shapes(px, i):
         return f64(x[blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))[:t]
 
     zero_k = np.zeros((rk, n_kv * hd)); zero_v = np.zeros((rv, n_kv * hd))
+    refs = []
     for b in range(B):
         t, a = ctx[b], agents[b]
         Lk = rows(c["lr_k"][max(a, 0)], b, t) if rk else np.zeros((t, 0))
@@ -94,7 +95,19 @@ def test_random_shapes(px, i):
         Bv_a = f64(w["B_v"][a]) if (rv and a >= 0) else zero_v
         ref = O.attend_from_caches(f64(q[b]), base_rows_of(c["k_base"], b, t), base_rows_of(c["v_base"], b, t), Lk, Lv, Bk_a, Bv_a,
                                    geo.scale_k, geo.scale_v, n_kv)
+        refs.append(ref)
         assert_close(out[b], ref, f"case {i} decode request {b} (hd{hd} G{G} kv{n_kv} r{rk}/{rv} ctx{t} agent{a} paged={paged})")
+    if B > 1:
+        # the same workspace serves a sub-batch (another split plan, possibly the other kernel)
+        out2 = torch.full_like(q[1:], float("nan"), device="cuda")
+        mx2 = max(ctx[1:])
+        px.lr_attend_decode(desc, q[1:].cuda(), torch.tensor(agents[1:], dtype=torch.int32).cuda(),
+                            torch.tensor(ctx[1:], dtype=torch.int32).cuda(), mx2, Bk, Bv, cache, out2, ws,
+                            table[1:].contiguous().cuda() if paged else None,
+                            None if paged else torch.tensor(first[1:], dtype=torch.int32).cuda())
+        torch.cuda.synchronize()
+        for b in range(1, B):
+            assert_close(f64(out2[b - 1]), refs[b], f"case {i} sub-batch request {b}")
     # ---------------------------------------------------------------- prefill over a second, contiguous-or-paged sequence
     nb2 = (T + S + 15) // 16
     c2 = I.direct_caches(nb2 + 2, geo, 200 + i, f"fzp{i}")
@@ -225,3 +238,61 @@ def test_random_rope_shapes(px, i):
     torch.cuda.synchronize()
     refp = O.lr_prefill_reference_rope(f64(qs), 1, T, *args, geo.scale_k, geo.scale_v, n_kv, cos, sin)
     assert_close(f64(outp), refp, f"case {i} rope prefill (hd{hd} G{G} kv{n_kv} r{r} T{T} S{S})")
+
+
+def _shard_case(i: int):
+    rng = np.random.default_rng(13000 + i)
+    hd = int(rng.choice([64, 128]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    n_kv = int(rng.choice([1, 2, 3]))
+    r = int(rng.choice([0, 8, 16, 32, 64]))
+    world = int(rng.integers(1, 9))
+    T = int(rng.integers(40, 900)) if i % 4 else int(rng.integers(2500, 4500))
+    B = int(rng.integers(1, 5))
+    ctx = [T] + [int(rng.integers(0, T + 1)) for _ in range(B - 1)]
+    agents = [int(rng.integers(-1, 2)) for _ in range(B)]
+    return hd, G, n_kv, r, world, T, ctx, agents
+
+
+@pytest.mark.parametrize("i", range(N_PROJ))
+def test_random_context_shards(px, i):
+    """Context-sharded decode (shards run one after another on this GPU): partial records merged by the
+    combine kernel equal attention over the whole context."""
+    from paper_2609_34054_b200.sharded import shard_ranges
+    hd, G, n_kv, r, world, T, ctx, agents = _shard_case(i)
+    geo = I.Geometry(d_model=128, n_q=G * n_kv, n_kv=n_kv, hd=hd, n_agents=2, rank_k=r, rank_v=r, alpha=2.0 * max(r, 1))
+    H = I.hidden_states(T, geo, 800 + i, f"sz.H{i}")
+    q = I.queries(len(ctx), geo, 800 + i, f"sz.q{i}", gain=3.0)
+    ranges = shard_ranges(ctx, world)
+    aid = torch.tensor(agents, dtype=torch.int32).cuda()
+    recs, first_layer = None, None
+    for rk_ in range(world):
+        local = [e - s for s, e in ranges[rk_]]
+        L = Layer(px, geo, seed=800 + i, n_blocks=sum((l + 15) // 16 for l in local) + 1, tag=f"sz{i}")
+        first, at = [], 0
+        for (s, e) in ranges[rk_]:
+            first.append(at)
+            if e > s:
+                L.append(H[s:e], start_slot=at * 16)
+            at += (e - s + 15) // 16
+        if recs is None:
+            recs = torch.full((world, len(ctx), n_kv, px.partial_record_floats(L.desc)), float("nan"), dtype=torch.float32, device="cuda")
+            first_layer = L
+        mx = max(1, max(local))
+        ws = px.decode_workspace(L.desc, len(ctx), mx)
+        px.lr_attend_decode_partial(L.desc, q.cuda(), aid, torch.tensor(local, dtype=torch.int32).cuda(), mx, L.B_k, L.cache,
+                                    recs[rk_], ws, None, torch.tensor(first, dtype=torch.int32).cuda())
+    out = torch.full_like(q, float("nan"), device="cuda")
+    px.combine_partials(first_layer.desc, recs, aid, first_layer.B_v, out)
+    torch.cuda.synchronize()
+    assert torch.isfinite(recs).all()
+    w = first_layer.w_np
+    args = (f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"])
+    live = [b for b, t in enumerate(ctx) if t > 0]
+    adapted = O.lr_decode_reference(f64(q)[live], [max(agents[b], 0) for b in live], [ctx[b] for b in live], *args, geo.scale_k, geo.scale_v, n_kv)
+    neutral = O.lr_decode_reference(f64(q)[live], [0] * len(live), [ctx[b] for b in live], *args, 0.0, 0.0, n_kv)
+    ref = np.where(np.array([agents[b] for b in live])[:, None, None] < 0, neutral, adapted)
+    assert_close(f64(out)[live], ref, f"case {i} sharded decode (hd{hd} G{G} kv{n_kv} r{r} world{world} ctx{ctx} agents{agents})")
+    for b, t in enumerate(ctx):
+        if t == 0:
+            assert (out[b] == 0).all(), f"case {i}: empty request {b} not zero"
