@@ -382,9 +382,11 @@ struct DecodeRunT {
   // The cluster kernel's shared-memory limit is only ever raised: the two ring layouts of one shape (two blocks
   // per SM / one block per SM) need different amounts, and lowering the attribute for the smaller one would
   // make a later launch of the larger one fail.
+  // (Function attributes and occupancy answers belong to a device: the caches are indexed by its ordinal.)
   template <int NW>
-  static cudaError_t ensure_cluster_smem(int bytes) {
-    static int have = 0;
+  static cudaError_t ensure_cluster_smem(precc_ctx* ctx, int bytes) {
+    static int have_dev[kMaxDevices] = {0};
+    int& have = have_dev[ctx->device % kMaxDevices];
     if (bytes <= have) return cudaSuccess;
     auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
@@ -394,12 +396,12 @@ struct DecodeRunT {
   }
   template <int NW>
   static bool cluster_fits(precc_ctx* ctx, const DecodePlan& pl, int need) {
-    static int cache2[2][DEC_MAX_CLUSTER + 1] = {{0}};  // 0 = unknown, else max active clusters + 1
-    int* cached = cache2[pl.deep ? 1 : 0];
+    static int cache2[kMaxDevices][2][DEC_MAX_CLUSTER + 1] = {{{0}}};  // 0 = unknown, else max active clusters + 1
+    int* cached = cache2[ctx->device % kMaxDevices][pl.deep ? 1 : 0];
     if (cached[pl.cluster] == 0) {
       auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
       int n = 0;
-      if (ensure_cluster_smem<NW>(pl.smem) != cudaSuccess) {
+      if (ensure_cluster_smem<NW>(ctx, pl.smem) != cudaSuccess) {
         cudaGetLastError();
         cached[pl.cluster] = 1;
         return false;
@@ -467,10 +469,10 @@ struct DecodeRunT {
       attr[1].val.clusterDim.x = pl.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
       cfg.numAttrs = 2;
       if (pl.warps == 8) {
-        PRECC_CUDA(ctx, ensure_cluster_smem<8>(pl.smem));
+        PRECC_CUDA(ctx, ensure_cluster_smem<8>(ctx, pl.smem));
         PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 8, ROPE>, p));
       } else {
-        PRECC_CUDA(ctx, ensure_cluster_smem<4>(pl.smem));
+        PRECC_CUDA(ctx, ensure_cluster_smem<4>(ctx, pl.smem));
         PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 4, ROPE>, p));
       }
     } else {
@@ -571,7 +573,8 @@ struct PrefillRun {
       if (ns < 1) ns = 1;
       // every cluster must be resident at once (one block per SM, and a cluster lives inside one GPC): ask
       // the occupancy calculator once per cluster size, and shrink the clusters until the grid fits in one wave
-      static int max_clusters[9] = {0};               // 0 = unknown, else max active clusters + 1
+      static int max_clusters_dev[kMaxDevices][9] = {{0}};   // 0 = unknown, else max active clusters + 1
+      int* max_clusters = max_clusters_dev[ctx->device % kMaxDevices];
       while (ns > 1) {
         if (max_clusters[ns] == 0) {
           cudaLaunchConfig_t qc = {};
