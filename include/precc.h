@@ -25,9 +25,8 @@
  *     host and can be captured into a CUDA graph (none synchronises, none allocates).
  *   - Return value: PRECC_OK or an error code.  On a host-detected error nothing is launched and no
  *     output is touched.  Text for the last error of a context: precc_last_error().
- *   - A context may be used from one host thread at a time.  Contexts of different threads must not
- *     make their FIRST call for a given shape concurrently: launch limits and occupancy answers are
- *     cached per device in the library image (warm each shape up from one thread).
+ *   - A context may be used from one host thread at a time; different contexts may be used from
+ *     different threads (kernel launch limits shared by all contexts of a device are kept under a lock).
  *
  * HBM layouts (PRECC_PAGE = 16 tokens per block; token slot s lives in block s / 16 at offset s % 16)
  *   base K, base V : [n_blocks][n_kv_heads][16][head_dim]

@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "../../include/precc.h"
@@ -62,6 +63,28 @@ int32_t fail(precc_ctx* ctx, int32_t code, const char* fmt, ...) {
     cudaError_t e__ = (expr);                                                                   \
     if (e__ != cudaSuccess) return fail(ctx, PRECC_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
   } while (0)
+
+// Dynamic shared-memory limit of a kernel on the context's device: only ever raised (a kernel serves
+// several configurations; lowering the limit for a small one would make a later large launch fail), and
+// set under a lock so that contexts on several host threads cannot interleave a set and a launch badly.
+struct SmemLimit { const void* fn; int dev; int bytes; };
+std::mutex g_limits_mu;
+SmemLimit g_limits[1024];
+int g_n_limits = 0;
+template <typename K>
+cudaError_t raise_smem_limit(precc_ctx* ctx, K kern, int bytes) {
+  const void* fn = reinterpret_cast<const void*>(kern);
+  std::lock_guard<std::mutex> lk(g_limits_mu);
+  SmemLimit* e = nullptr;
+  for (int i = 0; i < g_n_limits; ++i)
+    if (g_limits[i].fn == fn && g_limits[i].dev == ctx->device) { e = &g_limits[i]; break; }
+  if (e && bytes <= e->bytes) return cudaSuccess;
+  const cudaError_t rc = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (rc != cudaSuccess) return rc;
+  if (!e && g_n_limits < 1024) { e = &g_limits[g_n_limits++]; e->fn = fn; e->dev = ctx->device; e->bytes = 0; }
+  if (e) e->bytes = bytes;
+  return cudaSuccess;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -199,7 +222,7 @@ int32_t launch_small(precc_ctx* ctx, const void* X, int M, int K, const void* Wt
   attr[1].val.clusterDim.x = cs; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
   auto go = [&](auto kern) -> int32_t {
-    PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, smem));
     PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, map_x, map_w, gp, k_slice));
     return PRECC_OK;
   };
@@ -233,7 +256,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
   gp.spread_rows = 1;
   gp.status = ctx->status;
-  PRECC_CUDA(ctx, cudaFuncSetAttribute(proj_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  PRECC_CUDA(ctx, raise_smem_limit(ctx, proj_gemm_kernel, (int)smem));
   const int total_tiles = m_tiles * n_tiles;
   proj_gemm_kernel<<<dim3(total_tiles < ctx->sm_count ? total_tiles : ctx->sm_count), GEMM_THREADS, smem, stream>>>(map_x, map_w, gp);
   PRECC_CUDA(ctx, cudaGetLastError());
@@ -385,13 +408,14 @@ struct DecodeRunT {
   // (Function attributes and occupancy answers belong to a device: the caches are indexed by its ordinal.)
   template <int NW>
   static cudaError_t ensure_cluster_smem(precc_ctx* ctx, int bytes) {
-    static int have_dev[kMaxDevices] = {0};
-    int& have = have_dev[ctx->device % kMaxDevices];
-    if (bytes <= have) return cudaSuccess;
+    static bool nonportable_dev[kMaxDevices] = {false};
     auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-    if (e == cudaSuccess) have = bytes;
+    cudaError_t e = raise_smem_limit(ctx, kern, bytes);
+    bool& np = nonportable_dev[ctx->device % kMaxDevices];
+    if (e == cudaSuccess && !np) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      if (e == cudaSuccess) np = true;
+    }
     return e;
   }
   template <int NW>
@@ -478,7 +502,7 @@ struct DecodeRunT {
     } else {
       auto kern = lr_attend_decode_kernel<HD, RK, RV, ROPE>;
       cfg.blockDim = dim3(DEC_WARPS * 32);
-      PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem));
+      PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, pl.smem));
       PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, p));
     }
     return PRECC_OK;
@@ -559,7 +583,7 @@ struct PrefillRun {
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
     p.trace = (ctx->trace && ctx->trace_blocks >= 32) ? ctx->trace : nullptr;
     auto kern = lr_attend_prefill_tc_kernel<HD, RK, RV>;
-    PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, smem));
     const int row_tiles = (a.S + p.tok_per_tile - 1) / p.tok_per_tile;
     // Short turn over a long context: too few (row tile, kv head) blocks to fill the machine, so the
     // context of each is split over a cluster of up to 8 blocks whose partial results merge over DSMEM.
@@ -634,7 +658,7 @@ struct PrefillRun {
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
     p.rope = reinterpret_cast<const float4*>(a.rope); p.max_pos = a.max_pos;
     auto kern = lr_attend_prefill_kernel<HD, RK, RV, ROPE>;
-    PRECC_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, smem));
     const int row_tiles = (a.S * p.group + PF_ROWS - 1) / PF_ROWS;
     kern<<<dim3(row_tiles, d->n_kv_heads), PF_THREADS, smem, a.stream>>>(p);
     PRECC_CUDA(ctx, cudaGetLastError());
