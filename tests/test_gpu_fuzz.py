@@ -192,6 +192,25 @@ def test_random_projections(px, i):
     for name in ("k_base", "v_base", "lr_k", "lr_v"):
         a_, b_ = getattr(La.cache, name).view(torch.int16), getattr(Lb.cache, name).view(torch.int16)
         assert torch.equal(a_, b_), f"case {i}: fused projection differs in {name}"
+    # one mask per row (double batching): a row's LR columns land only in the agents its mask names, with the
+    # same bits as above; the base columns of every row are written
+    rng = np.random.default_rng(7000 + i)
+    row_masks = torch.from_numpy(rng.integers(0, 1 << N, size=M).astype(np.int64))
+    Lc = Layer(px, geo, seed=300 + i, n_blocks=nb, fill=float("nan"), tag=f"pz{i}")
+    slots_c = (slots if scattered else torch.arange(start, start + M, dtype=torch.int32)).cuda()
+    px.turn_project_rows(Lc.desc, H.cuda(), WA, Lc.cache, slots_c, row_masks.cuda())
+    full = Layer(px, geo, seed=300 + i, n_blocks=nb, fill=float("nan"), tag=f"pz{i}")
+    px.turn_project(full.desc, H.cuda(), WA, full.cache, start, None if slots is None else slots.cuda())      # every agent
+    torch.cuda.synchronize()
+    assert torch.equal(Lc.cache.k_base.view(torch.int16), full.cache.k_base.view(torch.int16))
+    assert torch.equal(Lc.cache.v_base.view(torch.int16), full.cache.v_base.view(torch.int16))
+    for a in range(N):
+        named = ((row_masks >> a) & 1).bool()
+        for name in ("lr_k", "lr_v"):
+            got = getattr(Lc.cache, name)[a].reshape(nb * 16, -1)[sl]
+            want = getattr(full.cache, name)[a].reshape(nb * 16, -1)[sl]
+            assert torch.equal(got[named].view(torch.int16), want[named].view(torch.int16)), f"case {i}: {name}[{a}] rows"
+            assert torch.isnan(got[~named]).all(), f"case {i}: {name}[{a}] written for rows that do not name it"
 
 
 def _rope_case(i: int):
