@@ -153,6 +153,24 @@ def direct_caches(n_blocks: int, geo: Geometry, seed: int, tag: str = "cache") -
     }
 
 
+def direct_caches_device(n_blocks: int, geo: Geometry, seed: int, tag: str = "cache", device: str = "cuda") -> Dict[str, torch.Tensor]:
+    """``direct_caches`` drawn on the device (large pools: seconds on the host, milliseconds there); same
+    distributions and layouts, another stream of numbers.  Ranks of zero give no LR tensors."""
+    g = torch.Generator(device=device)
+    g.manual_seed((zlib.crc32(tag.encode()) * 1_000_003 + seed * 7_919 + 54_321) % (2**63 - 1))
+    sig = 0.02 * geo.d_model ** 0.5
+
+    def draw(shape, std):
+        return (torch.randn(shape, device=device, generator=g) * std).to(torch.bfloat16)
+
+    out = {"k_base": draw((n_blocks, geo.n_kv, PAGE, geo.hd), sig), "v_base": draw((n_blocks, geo.n_kv, PAGE, geo.hd), sig)}
+    if geo.rank_k:
+        out["lr_k"] = draw((geo.n_agents, n_blocks, PAGE, geo.rank_k), 1.0)
+    if geo.rank_v:
+        out["lr_v"] = draw((geo.n_agents, n_blocks, PAGE, geo.rank_v), 1.0)
+    return out
+
+
 def serving_batch(batch: int, ctx_min: int, ctx_max: int, n_agents: int, seed: int):
     """Agent ids uniform over the agents, context lengths uniform (inclusive)."""
     agent_id = uniform_int(0, n_agents - 1, batch, seed, "serve.agent_id")

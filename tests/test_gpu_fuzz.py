@@ -315,3 +315,98 @@ def test_random_context_shards(px, i):
     for b, t in enumerate(ctx):
         if t == 0:
             assert (out[b] == 0).all(), f"case {i}: empty request {b} not zero"
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Large shapes (caches drawn on the device): batches up to 64 requests, contexts up to 70k tokens, turns of
+# up to 2047 new tokens over up to 66k; sampled requests / rows against the oracle.
+
+N_LARGE = max(6, N_CASES // 6)
+
+
+def _weights_small(geo, seed, tag):
+    w = I.layer_weights(geo, seed, tag)
+    return (w["B_k"].cuda() if geo.rank_k else None, w["B_v"].cuda() if geo.rank_v else None, w)
+
+
+@pytest.mark.parametrize("i", range(N_LARGE))
+def test_random_large_decode(px, i):
+    rng = np.random.default_rng(20000 + i)
+    hd = int(rng.choice([64, 128])); G = int(rng.choice([1, 2, 4, 7, 8])); n_kv = int(rng.choice([1, 2, 4, 8]))
+    r = int(rng.choice([0, 8, 16, 32, 64])); N = int(rng.integers(1, 5))
+    B = int(rng.choice([1, 1, 2, 3, 5, 8, 16, 33, 64]))
+    tmax = int(rng.choice([3000, 9000, 20000, 70000]))
+    ctx = [int(rng.integers(1, tmax + 1)) for _ in range(B)]
+    while sum(ctx) > 400000:
+        ctx = [max(1, c // 2) for c in ctx]
+    agents = [int(rng.integers(-1, N)) for _ in range(B)]
+    paged = bool(rng.random() < 0.6)
+    geo = I.Geometry(64, G * n_kv, n_kv, hd, N, r, r, alpha=2.0 * max(r, 1))
+    desc = layer_desc(geo)
+    need = [(c + 15) // 16 for c in ctx]
+    pool = sum(need) + 5
+    c = I.direct_caches_device(pool, geo, 400 + i, f"lz{i}")
+    cache = Cache.from_tensors(geo, c["k_base"], c["v_base"], c.get("lr_k"), c.get("lr_v"))
+    Bk, Bv, w = _weights_small(geo, 400 + i, f"lz{i}")
+    perm = I.permutation(pool, 400 + i, f"lz.perm{i}")
+    table = torch.zeros((B, max(need)), dtype=torch.int32)
+    first, at = [], 0
+    for b, n in enumerate(need):
+        table[b, :n] = perm[at:at + n] if paged else torch.arange(at, at + n)
+        first.append(at)
+        at += n
+    q = I.queries(B, geo, 400 + i, f"lz.q{i}", gain=3.0)
+    out = torch.full_like(q, float("nan"), device="cuda")
+    mx = max(ctx)
+    ws = px.decode_workspace(desc, B, mx)
+    px.lr_attend_decode(desc, q.cuda(), torch.tensor(agents, dtype=torch.int32).cuda(), torch.tensor(ctx, dtype=torch.int32).cuda(),
+                        mx, Bk, Bv, cache, out, ws, table.cuda() if paged else None,
+                        None if paged else torch.tensor(first, dtype=torch.int32).cuda())
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
+    for b in sorted(set([0, B // 2, B - 1, int(np.argmax(ctx))])):
+        t, a = ctx[b], agents[b]
+        blocks = table[b, :need[b]].long().cuda()
+        rows = lambda x: f64(x[blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))[:t]
+        Lk = f64(c["lr_k"][max(a, 0)][blocks].reshape(-1, r))[:t] if r else np.zeros((t, 0))
+        Lv = f64(c["lr_v"][max(a, 0)][blocks].reshape(-1, r))[:t] if r else np.zeros((t, 0))
+        Bka = f64(w["B_k"][a]) if (r and a >= 0) else np.zeros((r, n_kv * hd))
+        Bva = f64(w["B_v"][a]) if (r and a >= 0) else np.zeros((r, n_kv * hd))
+        ref = O.attend_from_caches(f64(q[b]), rows(c["k_base"]), rows(c["v_base"]), Lk, Lv, Bka, Bva, geo.scale_k, geo.scale_v, n_kv)
+        assert_close(f64(out[b]), ref, f"case {i} large decode request {b} (hd{hd} G{G} kv{n_kv} r{r} B{B} ctx{t} agent{a} paged={paged})")
+
+
+@pytest.mark.parametrize("i", range(N_LARGE))
+def test_random_large_prefill(px, i):
+    rng = np.random.default_rng(40000 + i)
+    hd = int(rng.choice([64, 128])); G = int(rng.choice([1, 2, 4, 8])); n_kv = int(rng.choice([1, 2, 4, 8]))
+    r = int(rng.choice([0, 8, 16, 32, 64])); N = int(rng.integers(1, 4))
+    S = int(rng.choice([1, 7, 16, 31, 32, 33, 64, 100, 128, 200, 256, 500, 512, 1000, 2047]))
+    T = int(rng.choice([0, 1, 100, 127, 128, 1000, 4000, 9000, 30000, 66000]))
+    if T > 100:
+        T = int(rng.integers(T // 2, T + 1))
+    agent = int(rng.integers(-1, N))
+    paged = bool(rng.random() < 0.5)
+    geo = I.Geometry(64, G * n_kv, n_kv, hd, N, r, r, alpha=2.0 * max(r, 1))
+    desc = layer_desc(geo)
+    nb = (T + S + 15) // 16
+    c = I.direct_caches_device(nb + 3, geo, 500 + i, f"lp{i}")
+    cache = Cache.from_tensors(geo, c["k_base"], c["v_base"], c.get("lr_k"), c.get("lr_v"))
+    Bk, Bv, w = _weights_small(geo, 500 + i, f"lp{i}")
+    tab = I.permutation(nb + 3, 500 + i, f"lp.perm{i}")[:nb].to(torch.int32) if paged else torch.arange(2, nb + 2, dtype=torch.int32)
+    q = I.queries(S, geo, 500 + i, f"lp.q{i}", gain=3.0)
+    out = torch.full_like(q, float("nan"), device="cuda")
+    px.lr_attend_prefill(desc, q.cuda(), agent, T, Bk, Bv, cache, out, tab.cuda() if paged else None, 0 if paged else 2)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
+    blocks = tab.long().cuda()
+    K = f64(c["k_base"][blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))
+    V = f64(c["v_base"][blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))
+    Lk = f64(c["lr_k"][max(agent, 0)][blocks].reshape(-1, r)) if r else np.zeros((nb * 16, 0))
+    Lv = f64(c["lr_v"][max(agent, 0)][blocks].reshape(-1, r)) if r else np.zeros((nb * 16, 0))
+    Bka = f64(w["B_k"][agent]) if (r and agent >= 0) else np.zeros((r, n_kv * hd))
+    Bva = f64(w["B_v"][agent]) if (r and agent >= 0) else np.zeros((r, n_kv * hd))
+    for srow in sorted(set([0, S // 3, S // 2, S - 1])):
+        t = T + srow + 1
+        ref = O.attend_from_caches(f64(q[srow]), K[:t], V[:t], Lk[:t], Lv[:t], Bka, Bva, geo.scale_k, geo.scale_v, n_kv)
+        assert_close(f64(out[srow]), ref, f"case {i} large prefill row {srow} (hd{hd} G{G} kv{n_kv} r{r} S{S} T{T} agent{agent} paged={paged})")
