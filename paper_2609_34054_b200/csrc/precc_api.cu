@@ -548,7 +548,9 @@ struct PrefillRun {
     const precc_layer_desc* d = a.d;
     const int G = d->n_q_heads / d->n_kv_heads;
     // as deep as shared memory allows, keys first (they are needed one step earlier)
-    int ks = 2, vs = 2;
+    // (head_dim 128 with rank 64 has room for a single value stage: 48 KB per stage of either kind)
+    int ks = 2, vs = 1;
+    if (C::smem_bytes(ks, vs) > ctx->max_smem_optin) return run_simple<false>(ctx, a);
     while (ks + vs < 8) {
       if (ks <= vs && C::smem_bytes(ks + 1, vs) <= ctx->max_smem_optin) ++ks;
       else if (C::smem_bytes(ks, vs + 1) <= ctx->max_smem_optin) ++vs;
@@ -590,7 +592,7 @@ struct PrefillRun {
     int ns = 1;
     const long long base_blocks = (long long)row_tiles * d->n_kv_heads;
     const int steps = (a.T + a.S + PTC_TOK - 1) / PTC_TOK;
-    if (!ctx->no_prefill_split && C::SPLIT_BYTES <= ks * C::KSTAGE + vs * C::VSTAGE) {
+    if (!ctx->no_prefill_split && C::SPLIT_BYTES <= C::Q_BYTES + C::QX_BYTES + ks * C::KSTAGE + vs * C::VSTAGE) {
       ns = (int)(ctx->sm_count / base_blocks);          // as many as keep the grid within one block per SM
       if (ns > 8) ns = 8;
       if (ns > steps / 8) ns = steps / 8;               // at least eight steps per block
@@ -636,7 +638,7 @@ struct PrefillRun {
     }
     return run_simple<false>(ctx, a);
   }
-  // mma.sync kernel: rank 64, oversized or unaligned caches, and the rotary variant
+  // mma.sync kernel: oversized or unaligned caches, and the rotary variant
   template <bool ROPE = false>
   static int32_t run_simple(precc_ctx* ctx, const PrefillArgs& a) {
     using C = PrefillCfg<HD, RK, RV>;

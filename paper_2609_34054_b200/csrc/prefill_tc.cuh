@@ -87,13 +87,14 @@ struct PrefillTcCfg {
   static constexpr int K_PAGE_TX = PAGE * (HD + RKP) * 2;      // bytes one page contributes to a key stage
   static constexpr int V_PAGE_TX = PAGE * VSLABS * 128;
   static constexpr int SPLIT_XS = (HD + RV + 15) / 16 * 16 + 4;                // row stride (floats) of a partial in shared memory
-  // split-context merge area (laid over the rings): partial | m | l | merged rows | weights | 1/l | B_v slice
+  // split-context merge area (laid over the Q tile, the folded-query tile and the rings): partial | m | l | merged rows | weights | 1/l | B_v slice
   static constexpr int SPLIT_BYTES = (128 * SPLIT_XS + 256 + 64 * SPLIT_XS + 16 * 64 + 64) * 4 + RV * HD * 2;
   static constexpr bool L_IN_MMA = RV > 0 && RV < 64;         // a spare column of the L_V slab carries the denominator
   static constexpr int TMEM_P = 2 * PTC_TOK;                  // packed bf16 P (64 columns) after the two S buffers
   static constexpr int TMEM_O = TMEM_P + PTC_TOK / 2;         // O' (at most 192 columns): 320 + 192 = 512
   __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 320 + 2 * PTC_PARTS_MAX * 512 + 1024; }
-  static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 8 || RK == 16 || RK == 32) && (RV == 0 || RV == 8 || RV == 16 || RV == 32);
+  static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 8 || RK == 16 || RK == 32 || RK == 64) &&
+                                    (RV == 0 || RV == 8 || RV == 16 || RV == 32 || RV == 64);
 };
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
@@ -589,7 +590,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     if (NS > 1) {
       // ---- split context: this block's partial (m, l, O') goes to shared memory for the cluster merge below
       constexpr int XS = C::SPLIT_XS;
-      float* xo = reinterpret_cast<float*>(kring);
+      float* xo = reinterpret_cast<float*>(smem);          // the merge area starts at the Q tile: every MMA has completed
       float* xm = xo + 128 * XS;
       float* xl = xm + 128;
       float l_loc = 0.f;
@@ -692,7 +693,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     constexpr int XS = C::SPLIT_XS;
     constexpr int NSM = PTC_SOFTMAX_WARPS * 32;
     const int R = (128 + (int)NS - 1) / (int)NS;        // rows per block (the last block may own fewer); 2 <= NS <= 16
-    float* xo = reinterpret_cast<float*>(kring);
+    float* xo = reinterpret_cast<float*>(smem);          // the merge area starts at the Q tile: every MMA has completed
     float* xm = xo + 128 * XS;
     float* xl = xm + 128;
     float* mo = xl + 128;                               // merged rows [R][XS]

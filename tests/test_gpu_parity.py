@@ -465,7 +465,8 @@ def test_one_workspace_serves_every_smaller_batch_and_context(px):
 
 @pytest.mark.parametrize("hd,n_q,n_kv,r,T,S,agent", [(128, 8, 2, 32, 2100, 40, 1), (128, 8, 2, 16, 4200, 33, 0), (64, 16, 4, 16, 9000, 20, 1),
                                                        (128, 8, 2, 32, 8300, 64, -1), (64, 8, 1, 32, 5000, 130, 0),
-                                                       (128, 8, 2, 8, 3000, 50, 1)])
+                                                       (128, 8, 2, 8, 3000, 50, 1), (128, 8, 2, 64, 4100, 45, 1), (64, 8, 2, 64, 2600, 70, 0),
+                                                       (128, 16, 2, 64, 300, 500, 1)])
 def test_prefill_short_turn_over_long_context_is_split_over_a_cluster(px, hd, n_q, n_kv, r, T, S, agent):
     """Few (row tile, kv head) blocks and many 128-token steps: the context is split over a cluster of 2, 4 or
     8 blocks and merged over distributed shared memory.  Against the definition, and bit-identical runs."""
@@ -514,10 +515,10 @@ def test_per_row_agent_masks_equal_two_separate_projections(px, n):
     assert torch.isnan(Lb.cache.lr_k[cur].reshape(nb * 16, -1)[slots_nt.long()]).all()      # the neutral rows left agent `cur` alone
 
 
-@pytest.mark.parametrize("hd,r", [(128, 8), (64, 16), (128, 32)])
+@pytest.mark.parametrize("hd,r", [(128, 8), (64, 16), (128, 32), (128, 64), (64, 64)])
 def test_mma_sync_prefill_kernel_matches_too(monkeypatch, hd, r):
-    """The tensor-memory kernel serves these shapes by default; the mma.sync kernel behind it (used for rank
-    64, rotary keys, oversized or unaligned caches) is forced here through the environment switch."""
+    """The tensor-memory kernel serves these shapes by default; the mma.sync kernel behind it (used for
+    rotary keys and for oversized or unaligned caches) is forced here through the environment switch."""
     monkeypatch.setenv("PRECC_PREFILL", "simple")
     px2 = Precc(0)
     geo = I.Geometry(256, 8, 2, hd, 2, r, r, alpha=2.0 * r)
