@@ -1,8 +1,8 @@
 """Sweep on Llama-3-8B layer shapes (d_model 4096, 32 q / 8 kv heads, head_dim 128): decode attention over
-rank r x context T x batch, and the LR precompute over agents N x rank r.  Seeded synthetic inputs generated
+rank r x context T x batch, the LR precompute over agents N x rank r, and turn prefill over rank r x (S, T).  Seeded synthetic inputs generated
 on the device; one JSON line per cell and a Markdown table at the end.
 
-    python -m paper_2609_34054_b200.sweep [--decode-only | --precompute-only] [--peak-gbs 6451.2] [--peak-tflops 1652.6]
+    python -m paper_2609_34054_b200.sweep [--decode-only | --precompute-only | --prefill-only] [--peak-gbs 6451.2] [--peak-tflops 1652.6]
 
 Decode bytes per request do not depend on the number of agents (a request reads the base rows and its own
 agent's LR rows), so the decode grid fixes N = 4; N enters through the precompute.  Small cells rotate over
@@ -23,6 +23,7 @@ RANKS = (8, 16, 32, 64)
 AGENTS = (2, 4, 8, 16)
 CONTEXTS = (1024, 8192, 32768, 131072)
 BATCHES = (1, 32)
+TURNS = ((512, 32768), (2048, 8192), (64, 65536))      # (new tokens S, context T)
 L2_BYTES = 126e6
 
 
@@ -112,16 +113,40 @@ def precompute_cell(px: Precc, N: int, r: int, M: int = 32768, seed: int = 0) ->
     return {"kind": "precompute", "N": N, "r": r, "n_out": n_out, "M": M, "us": us, "TFLOPs": flops / us / 1e6, "GBps": byt / us / 1e3}
 
 
+def prefill_cell(px: Precc, r: int, S: int, T: int, seed: int = 0) -> dict:
+    geo = I.c5_geometry(r, 4)
+    desc = layer_desc(geo)
+    c = I.direct_caches_device((T + S) // I.PAGE, geo, seed, "sweep.pf")
+    cache = Cache.from_tensors(geo, c["k_base"], c["v_base"], c["lr_k"], c["lr_v"])
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    B_k = _randn((geo.n_agents, r, geo.kv_width), 0.02, gen)
+    B_v = _randn((geo.n_agents, r, geo.kv_width), 0.02, gen)
+    q = _randn((S, geo.n_q, geo.hd), 1.0, gen)
+    out = torch.empty_like(q)
+    us = _graph_time_us(lambda: px.lr_attend_prefill(desc, q, 1, T, B_k, B_v, cache, out), 2, 5)
+    flops = 4.0 * geo.n_q * (geo.hd + r) * (S * T + S * (S + 1) / 2)      # scores + weighted sum over hd + r coordinates
+    assert px.poll_status() == 0 and torch.isfinite(out.float()).all()
+    return {"kind": "prefill", "r": r, "S": S, "T": T, "us": us, "TFLOPs": flops / us / 1e6}
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
     ap.add_argument("--decode-only", action="store_true")
     ap.add_argument("--precompute-only", action="store_true")
+    ap.add_argument("--prefill-only", action="store_true")
     ap.add_argument("--peak-gbs", type=float, default=6451.2, help="measured copy bandwidth the fractions refer to")
     ap.add_argument("--peak-tflops", type=float, default=1652.6, help="measured dense bf16 burst rate")
     args = ap.parse_args(argv)
     px = Precc(0)
-    dec, pre = [], []
-    if not args.precompute_only:
+    dec, pre, pf = [], [], []
+    if not (args.decode_only or args.precompute_only):
+        for r in RANKS:
+            for (S, T) in TURNS:
+                c = prefill_cell(px, r, S, T)
+                pf.append(c)
+                print(json.dumps({k: (round(v, 2) if isinstance(v, float) else v) for k, v in c.items()}), flush=True)
+                torch.cuda.empty_cache()
+    if not (args.precompute_only or args.prefill_only):
         for r in RANKS:
             for B in BATCHES:
                 for T in CONTEXTS:
@@ -129,7 +154,7 @@ def main(argv=None):
                     dec.append(c)
                     print(json.dumps({k: (round(v, 2) if isinstance(v, float) else v) for k, v in c.items()}), flush=True)
                     torch.cuda.empty_cache()
-    if not args.decode_only:
+    if not (args.decode_only or args.prefill_only):
         for N in AGENTS:
             for r in RANKS:
                 c = precompute_cell(px, N, r)
@@ -143,6 +168,11 @@ def main(argv=None):
                 cells = [c for c in dec if c["r"] == r and c["B"] == B]
                 print(f"| {r} | {B} | " + " | ".join(
                     f"{c['us']:.1f} us, {c['GBps']:.0f} GB/s ({c['GBps'] / args.peak_gbs * 100:.0f} %)" for c in cells) + " |")
+    if pf:
+        print("\n| r | " + " | ".join(f"S={S}, T={T}" for (S, T) in TURNS) + " |\n|---|" + "---|" * len(TURNS))
+        for r in RANKS:
+            cells = [c for c in pf if c["r"] == r]
+            print(f"| {r} | " + " | ".join(f"{c['us']:.0f} us, {c['TFLOPs']:.0f} TF/s ({c['TFLOPs'] / args.peak_tflops * 100:.0f} %)" for c in cells) + " |")
     if pre:
         print("\n| N | " + " | ".join(f"r={r}" for r in RANKS) + " |\n|---|" + "---|" * len(RANKS))
         for N in AGENTS:
