@@ -739,8 +739,10 @@ __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_sync_all() { cluster_arrive(); cluster_wait(); }
 
-template <int HD, int RK, int RV, int NW, bool ROPE = false>
-__global__ void __launch_bounds__(NW * 32, (NW == 8 && HD == 64) ? 2 : 1)   // 16-block clusters need two blocks per SM
+// MINB = 2 (8 warps, head_dim 64): 16-block clusters need two blocks per SM, which caps the kernel at 128
+// registers; the one-block-per-SM ring layout uses the MINB = 1 instance, free of that cap.
+template <int HD, int RK, int RV, int NW, bool ROPE = false, int MINB = 1>
+__global__ void __launch_bounds__(NW * 32, MINB)
 lr_attend_decode_cluster_kernel(const DecodeParams p) {
   using C = DecodeCfg<HD, RK, RV>;
   constexpr int OW = C::OW;

@@ -406,12 +406,21 @@ struct DecodeRunT {
   // per SM / one block per SM) need different amounts, and lowering the attribute for the smaller one would
   // make a later launch of the larger one fail.
   // (Function attributes and occupancy answers belong to a device: the caches are indexed by its ordinal.)
+  using ClusterKernel = void (*)(const DecodeParams);
+  // two blocks per SM (8 warps, head_dim 64) unless the plan uses the one-block-per-SM ring layout
   template <int NW>
-  static cudaError_t ensure_cluster_smem(precc_ctx* ctx, int bytes) {
-    static bool nonportable_dev[kMaxDevices] = {false};
-    auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
+  static ClusterKernel cluster_kernel(bool deep) {
+    if constexpr (NW == 8 && HD == 64) {
+      if (!deep) return lr_attend_decode_cluster_kernel<HD, RK, RV, 8, ROPE, 2>;
+    }
+    return lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE, 1>;
+  }
+  template <int NW>
+  static cudaError_t ensure_cluster_smem(precc_ctx* ctx, int bytes, bool deep) {
+    static bool nonportable_dev[kMaxDevices][2] = {{false}};
+    ClusterKernel kern = cluster_kernel<NW>(deep);
     cudaError_t e = raise_smem_limit(ctx, kern, bytes);
-    bool& np = nonportable_dev[ctx->device % kMaxDevices];
+    bool& np = nonportable_dev[ctx->device % kMaxDevices][deep ? 1 : 0];
     if (e == cudaSuccess && !np) {
       e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       if (e == cudaSuccess) np = true;
@@ -423,9 +432,9 @@ struct DecodeRunT {
     static int cache2[kMaxDevices][2][DEC_MAX_CLUSTER + 1] = {{{0}}};  // 0 = unknown, else max active clusters + 1
     int* cached = cache2[ctx->device % kMaxDevices][pl.deep ? 1 : 0];
     if (cached[pl.cluster] == 0) {
-      auto kern = lr_attend_decode_cluster_kernel<HD, RK, RV, NW, ROPE>;
+      ClusterKernel kern = cluster_kernel<NW>(pl.deep != 0);
       int n = 0;
-      if (ensure_cluster_smem<NW>(ctx, pl.smem) != cudaSuccess) {
+      if (ensure_cluster_smem<NW>(ctx, pl.smem, pl.deep != 0) != cudaSuccess) {
         cudaGetLastError();
         cached[pl.cluster] = 1;
         return false;
@@ -493,11 +502,11 @@ struct DecodeRunT {
       attr[1].val.clusterDim.x = pl.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
       cfg.numAttrs = 2;
       if (pl.warps == 8) {
-        PRECC_CUDA(ctx, ensure_cluster_smem<8>(ctx, pl.smem));
-        PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 8, ROPE>, p));
+        PRECC_CUDA(ctx, ensure_cluster_smem<8>(ctx, pl.smem, pl.deep != 0));
+        PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, cluster_kernel<8>(pl.deep != 0), p));
       } else {
-        PRECC_CUDA(ctx, ensure_cluster_smem<4>(ctx, pl.smem));
-        PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, lr_attend_decode_cluster_kernel<HD, RK, RV, 4, ROPE>, p));
+        PRECC_CUDA(ctx, ensure_cluster_smem<4>(ctx, pl.smem, pl.deep != 0));
+        PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, cluster_kernel<4>(pl.deep != 0), p));
       }
     } else {
       auto kern = lr_attend_decode_kernel<HD, RK, RV, ROPE>;
