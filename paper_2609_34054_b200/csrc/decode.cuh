@@ -541,6 +541,9 @@ template <int HD, int RK, int RV, bool ROPE = false>
 __global__ void __launch_bounds__(DEC_WARPS * 32)
 lr_attend_decode_kernel(const DecodeParams p) {
   using C = DecodeCfg<HD, RK, RV>;
+  // partial-output mode has no rotary entry point: compiled out of the rotary instances (which sit at the
+  // register limit; the extra branches cost them 14 % through register allocation alone)
+  float* const raw_out = ROPE ? nullptr : p.raw;
   constexpr int OW = C::OW;
   constexpr int NT = DEC_WARPS * 32;
   extern __shared__ __align__(128) unsigned char smem[];
@@ -561,9 +564,9 @@ lr_attend_decode_kernel(const DecodeParams p) {
   __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
   if (ctx < 1 || agent_raw < -1 || agent_raw >= p.n_agents) {
     if (split == 0) {
-      if (p.raw) {
+      if (raw_out) {
         // an empty shard (or a rejected request) contributes the neutral record: m = -big, l = 0, O' = 0
-        float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
+        float* rec = raw_out + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
         for (int i = threadIdx.x; i < C::PART_STRIDE; i += NT) rec[i] = i < 8 ? NEG_BIG : 0.f;
       } else {
         for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
@@ -622,7 +625,7 @@ lr_attend_decode_kernel(const DecodeParams p) {
     const float* base = p.part + (((size_t)b * p.n_kv + g) * p.max_splits) * C::PART_STRIDE;
     float* recs = res + 16 + 8 * OW;                    // [n_splits][rec_f] (staged) or [n_splits][16]
     const bool staged = (16 + 8 * OW + n_splits * rec_f + DEC_WARPS * n_el) * 4 + bv_bytes <= region;
-    if (!p.raw) stage_bv();
+    if (!raw_out) stage_bv();
     if (staged) {
       const int cpr = rec_f / 4;                        // 16-byte chunks per record
       for (int c = threadIdx.x; c < n_splits * cpr; c += NT) {
@@ -687,17 +690,17 @@ lr_attend_decode_kernel(const DecodeParams p) {
     for (int e = threadIdx.x; e < n_el; e += NT)
       fo[e] = ((wsum[e] + wsum[n_el + e]) + wsum[2 * n_el + e]) + wsum[3 * n_el + e];
   } else {
-    if (!p.raw) stage_bv();
+    if (!raw_out) stage_bv();
     cp_async_commit();
     if (threadIdx.x < 8) { fin_l[threadIdx.x] = res[8 + threadIdx.x]; fin_m[threadIdx.x] = res[threadIdx.x]; }
     cp_async_wait<0>();
   }
   __syncthreads();
   mark(10);
-  if (p.raw) {
+  if (raw_out) {
     // partial-output mode: the merged record of this (request, kv head) over the LOCAL tokens, not
     // normalised and without the value-side epilogue; a later combine step merges such records
-    float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
+    float* rec = raw_out + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
     for (int i = threadIdx.x; i < C::PART_STRIDE; i += NT) {
       float v = 0.f;
       if (i < 8) v = i < G ? fin_m[i] : NEG_BIG;
@@ -745,6 +748,7 @@ template <int HD, int RK, int RV, int NW, bool ROPE = false, int MINB = 1>
 __global__ void __launch_bounds__(NW * 32, MINB)
 lr_attend_decode_cluster_kernel(const DecodeParams p) {
   using C = DecodeCfg<HD, RK, RV>;
+  float* const raw_out = ROPE ? nullptr : p.raw;      // no rotary partial-output entry point: compiled out there
   constexpr int OW = C::OW;
   constexpr int NT = NW * 32;
   extern __shared__ __align__(128) unsigned char smem[];
@@ -765,8 +769,8 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
   if (ctx < 1 || agent_raw < -1 || agent_raw >= p.n_agents) {   // the same decision in every block of the cluster
     if (rank == 0) {
-      if (p.raw) {
-        float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;   // neutral record: m = -big, l = 0, O' = 0
+      if (raw_out) {
+        float* rec = raw_out + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;   // neutral record: m = -big, l = 0, O' = 0
         for (int i = threadIdx.x; i < C::PART_STRIDE; i += NT) rec[i] = i < 8 ? NEG_BIG : 0.f;
       } else {
         for (int i = threadIdx.x; i < G * HD; i += NT) out_bg[i] = __float2bfloat16(0.f);
@@ -789,7 +793,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
 #pragma unroll
     for (int k = 0; k < BV_PER_THREAD; ++k) {
       const int i = threadIdx.x + k * NT;
-      bv_pre[k] = (i < RV * cols_ && (i % cols_) < ncol_ && !p.raw) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);   // partial-output mode has no B_v
+      bv_pre[k] = (i < RV * cols_ && (i % cols_) < ncol_ && !raw_out) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);   // partial-output mode has no B_v
     }
   }
   if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
@@ -842,10 +846,10 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   cluster_arrive();                                     // this block has finished reading its peers; the wait is at the exit
   mark(10);
   const float* fin_l = mine + 8 * (HD + RV);
-  if (p.raw) {
+  if (raw_out) {
     // partial-output mode: this block's column slice of the merged, un-normalised record; block 0 adds the
     // LR-V coordinates, the denominators and the maxima
-    float* rec = p.raw + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
+    float* rec = raw_out + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
     for (int e = threadIdx.x; e < G * cols; e += NT)
       if ((e % cols) < ncol) rec[16 + (e / cols) * OW + c0 + (e % cols)] = mine[(e / cols) * sw + (e % cols)];
     if (rank == 0) {

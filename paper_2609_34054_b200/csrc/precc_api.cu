@@ -340,6 +340,9 @@ DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx
   // resident (a 16-block cluster at one block per SM does not fit every GPC).  Measured against the
   // two-blocks-per-SM layout: 8192 tokens x 8 units 9.3 -> 9.0 us, 32768 tokens 31 -> 27 us, 65536 tokens
   // 53 -> 46 us.  With the deep rings switched off, bandwidth-bound sizes go to the ticket kernel instead.
+  // Narrow clusters over a lot of data (e.g. 8 requests x 8 kv heads x 32768 tokens: clusters of 2): the work is
+  // bandwidth-bound and the ticket kernel, which spreads it over every SM, is faster (rotary keys: 252 against 350 us).
+  if (units * max_tiles > 32768 && cs <= 4) return pl;
   if (units * max_tiles > (deep_ok ? 2048 : 32768) && cs > 4) {
     if (!deep_ok) return pl;
     const int big = max_smem - 2048 - extra;
@@ -455,7 +458,10 @@ struct DecodeRunT {
   static int32_t run(precc_ctx* ctx, const DecodeArgs& a) {
     const precc_layer_desc* d = a.d;
     constexpr int extra = ROPE ? DecodeCfg<HD, RK, RV>::BK_BYTES + 128 : 0;
-    DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra, ctx->deep_clusters);
+    // The rotary kernel at head_dim 128 is issue-bound (255 registers, 8 warps per SM at most): it gains more from
+    // the 128 blocks of the two-blocks-per-SM layout than from deeper rings on 80 SMs (131072 tokens: 141 against 238 us).
+    const bool deep_ok = ctx->deep_clusters && !(ROPE && HD == 128);
+    DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra, deep_ok);
     auto fits = [&](const DecodePlan& q) { return q.warps == 8 ? cluster_fits<8>(ctx, q, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, q, a.B * d->n_kv_heads); };
     if (pl.cluster && pl.deep) {
       const int max_tiles = (a.max_ctx + PAGE - 1) / PAGE;
@@ -983,6 +989,7 @@ static int32_t decode_entry(precc_ctx* ctx, const precc_layer_desc* desc, const 
                workspace, workspace_bytes, (cudaStream_t)stream};
   a.raw = raw;
   if (!rope) return dispatch_shape<DecodeRun>(ctx, desc->head_dim, desc->rank_k, desc->rank_v, a);
+  if (raw) return fail(ctx, PRECC_ERR_UNSUPPORTED, "partial records with rotary keys");   // compiled out of the rotary kernels
   if (!aligned16(rope)) return fail(ctx, PRECC_ERR_MISALIGNED, "rope table not 16-byte aligned");
   if (max_pos < max_ctx) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table covers %d positions, max_ctx is %d", max_pos, max_ctx);
   a.rope = rope; a.max_pos = max_pos;
