@@ -29,6 +29,7 @@ struct precc_ctx {
   size_t trace_blocks = 0;
   bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
   bool force_tiled_gemm = false;       // PRECC_GEMM=tiled in the environment: never take the few-row kernel
+  bool force_ticket_decode = false;    // PRECC_DECODE=ticket in the environment: never use the cluster decode kernel
   bool deep_clusters = true;           // PRECC_DEEP=0 in the environment: never use the one-block-per-SM deep-ring clusters
   bool prefill_forward = false;        // PRECC_PREFILL_ORDER=forward: row tiles in ascending order (default: longest causal reach first)
   bool no_prefill_split = false;       // PRECC_PREFILL_SPLIT=0 in the environment: never split a turn's context over a cluster
@@ -343,6 +344,10 @@ DecodePlan plan_cluster(int sm_count, int max_smem, int B, int n_kv, int max_ctx
   // Narrow clusters over a lot of data (e.g. 8 requests x 8 kv heads x 32768 tokens: clusters of 2): the work is
   // bandwidth-bound and the ticket kernel, which spreads it over every SM, is faster (rotary keys: 252 against 350 us).
   if (units * max_tiles > 32768 && cs <= 4) return pl;
+  // Wide pages (head_dim 128 with rank 32 or 64) leave the two-blocks-per-SM layout only 4 warps with 2-page
+  // rings; narrow clusters of such blocks lose to the ticket kernel's larger grid from a few thousand pages on
+  // (rank 32, 8192 tokens, 4..8 requests: 35..58 us against 33..51 us; ranks 8 and 16 keep three-page rings and win).
+  if (warps == 4 && stages == 2 && cs <= 4 && units * max_tiles >= 6000) return pl;
   if (units * max_tiles > (deep_ok ? 2048 : 32768) && cs > 4) {
     if (!deep_ok) return pl;
     const int big = max_smem - 2048 - extra;
@@ -462,6 +467,7 @@ struct DecodeRunT {
     // the 128 blocks of the two-blocks-per-SM layout than from deeper rings on 80 SMs (131072 tokens: 141 against 238 us).
     const bool deep_ok = ctx->deep_clusters && !(ROPE && HD == 128);
     DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra, deep_ok);
+    if (ctx->force_ticket_decode) pl.cluster = 0;
     auto fits = [&](const DecodePlan& q) { return q.warps == 8 ? cluster_fits<8>(ctx, q, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, q, a.B * d->n_kv_heads); };
     if (pl.cluster && pl.deep) {
       const int max_tiles = (a.max_ctx + PAGE - 1) / PAGE;
@@ -753,6 +759,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   if (const char* v = getenv("PRECC_PREFILL")) ctx->force_simple_prefill = (strcmp(v, "simple") == 0);
   if (const char* v = getenv("PRECC_GEMM")) ctx->force_tiled_gemm = (strcmp(v, "tiled") == 0);
   if (const char* v = getenv("PRECC_DEEP")) ctx->deep_clusters = (strcmp(v, "0") != 0);
+  if (const char* v = getenv("PRECC_DECODE")) ctx->force_ticket_decode = (strcmp(v, "ticket") == 0);
   if (const char* v = getenv("PRECC_PREFILL_ORDER")) ctx->prefill_forward = (strcmp(v, "forward") == 0);
   if (const char* v = getenv("PRECC_PREFILL_SPLIT")) ctx->no_prefill_split = (strcmp(v, "0") == 0);
   if (e != cudaSuccess) {
