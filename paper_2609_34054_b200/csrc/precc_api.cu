@@ -183,12 +183,23 @@ int32_t make_map2(precc_ctx* ctx, CUtensorMap* map, const void* base, long long 
   return PRECC_OK;
 }
 
+// Column tile width.  A block's time per 64-deep k-block hardly depends on the width below 256 columns (the
+// thread that issues the MMAs needs about a hundred cycles per instruction, four per k-block: measured 0.52 us
+// per k-block at 256 columns, 0.45 at 128, 0.42 at 64 and still 0.40 at 16), so a launch costs about
+// rounds x that, rounds = ceil(tiles / SMs): the widest tile that does not add a round wins
+// (2048 rows x 2304 columns: 144 tiles of 256 in one round, 35 us, against 288 tiles of 128 in two, 55 us).
 int pick_bn(int n_out, int m_tiles, int sm_count) {
   if (n_out <= 256) return (n_out + 15) / 16 * 16;
   const int cands[3] = {256, 128, 64};
-  for (int bn : cands)
-    if ((long long)m_tiles * ((n_out + bn - 1) / bn) >= sm_count) return bn;
-  return 64;
+  const double per_kblock[3] = {0.52, 0.45, 0.42};
+  int best = 256;
+  double best_cost = 1e30;
+  for (int i = 0; i < 3; ++i) {
+    const long long tiles = (long long)m_tiles * ((n_out + cands[i] - 1) / cands[i]);
+    const double cost = (double)((tiles + sm_count - 1) / sm_count) * per_kblock[i];
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = cands[i]; }
+  }
+  return best;
 }
 
 // Few rows (decode steps): the weight-streaming split-K kernel.  The K split depends on K alone, so a
