@@ -51,6 +51,7 @@ struct GemmParams {
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;                 // 64 bf16 = one 128-byte swizzle row
 constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_MAX_KS = 8;            // largest K split of the split-K kernel (cluster size)
 constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -324,6 +325,187 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(acc_empty + 8 * buf) : "memory");
     }
   }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+  }
+}
+
+
+// Reduce step of the split-K kernel: thread t of the 128 epilogue threads takes the 16-byte pieces t, t + 128, ...
+// of this block's slice (piece f = row * cw/4 + q), 16 / KS of them at a time, so that sixteen loads over
+// distributed shared memory are in flight per thread; consecutive lanes read consecutive pieces of a peer; the
+// peers are summed in rank order.  The odd piece of a pair hands its four columns to the even one, which
+// stores eight.
+template <int KS>
+__device__ __forceinline__ void splitk_reduce(const GemmParams& p, uint32_t smem_base, int rank, int cw, int m0, int n0, int t) {
+  constexpr int G = 16 / KS;
+  const int XS = cw + 4, qpr = cw / 4;
+  const uint32_t slice = smem_base + (uint32_t)rank * GEMM_BM * XS * 4;
+  const int total = GEMM_BM * qpr;                              // a multiple of 128
+  for (int f0 = t; f0 < total; f0 += 128 * G) {
+    float4 a[G][KS];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const int f = f0 + g * 128;
+      const int row = f / qpr, q = f % qpr;
+#pragma unroll
+      for (int r = 0; r < KS; ++r) {
+        if (f < total) {
+          uint32_t remote;
+          asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(slice + (uint32_t)(row * XS + 4 * q) * 4), "r"(r));
+          asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];\n" : "=f"(a[g][r].x), "=f"(a[g][r].y), "=f"(a[g][r].z), "=f"(a[g][r].w) : "r"(remote));
+        } else {
+          a[g][r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const int f = f0 + g * 128;
+      const int row = f / qpr, q = f % qpr;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int r = 0; r < KS; ++r) { v.x += a[g][r].x; v.y += a[g][r].y; v.z += a[g][r].z; v.w += a[g][r].w; }
+      const float4 hi = make_float4(__shfl_down_sync(0xffffffffu, v.x, 1), __shfl_down_sync(0xffffffffu, v.y, 1),
+                                    __shfl_down_sync(0xffffffffu, v.z, 1), __shfl_down_sync(0xffffffffu, v.w, 1));
+      if ((q & 1) == 0 && f < total) {
+        const int gm = m0 + row, c = rank * cw + 4 * q, gc = n0 + c;
+        if (gm < p.M && c < p.BN && gc < p.N_out) {
+          const long long slot = p.slot_mapping ? (long long)p.slot_mapping[gm] : p.start_slot + gm;
+          if (slot < 0 || slot >= p.n_blocks * PAGE) {
+            atomicOr(p.status, StatusBits::BAD_INDEX);
+          } else {
+            const float v8[8] = {v.x, v.y, v.z, v.w, hi.x, hi.y, hi.z, hi.w};
+            store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8, p.row_masks ? p.row_masks[gm] : p.agent_mask);
+          }
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Split-K form for a few row tiles (64 < M <= 512: the tokens of a short turn).  A block of the kernel
+// above needs about 0.4 us per 64-deep k-block whatever its tile width, so the whole K extent costs one
+// block 25 us at d_model 4096 even when there is almost no work.  Here the K extent of one 128 x BN tile is
+// divided over the KS = 4 or 8 blocks of a cluster (grid = (KS, column tiles, row tiles)); each block accumulates its
+// K slice in TMEM exactly as above, writes the fp32 accumulator into its own shared memory (over the ring,
+// which is idle by then), and after a cluster barrier block r adds up columns [r*cw, (r+1)*cw) of all KS
+// partial tiles over distributed shared memory — in rank order, so the result does not depend on timing —
+// and routes them to the caches with the same epilogue.  No rotary epilogue here (a head's two halves would
+// have to land in one block's slice); rotary calls use the kernel above.
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
+proj_gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const GemmParams p) {
+  // The declared alignment places the dynamic shared memory on a 1024-byte boundary (the swizzle atoms need it and
+  // the peers' addresses must correspond).  Should the base ever be unaligned, every block of the grid says so and leaves.
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw;
+  if ((smem_u32(smem_raw) & 1023u) != 0) {
+    if (threadIdx.x == 0) atomicOr(p.status, StatusBits::TIMEOUT);
+    return;
+  }
+  const int b_bytes = p.BN * GEMM_BK * 2;
+  const int stage_bytes = GEMM_A_BYTES + b_bytes;
+  // The dumped accumulator is laid out slice by slice: block r of the cluster will reduce columns
+  // [r*cw, (r+1)*cw), and finds them in every peer as one block of 128 rows x (cw + 4) floats (the 4 floats
+  // of padding keep the row-per-thread dump free of bank conflicts), which it can read with consecutive lanes
+  // on consecutive 16-byte pieces.
+  const int cw = (((p.BN + (int)gridDim.x - 1) / (int)gridDim.x) + 7) / 8 * 8;   // columns reduced by one block (a multiple of 8)
+  const int XS = cw + 4;                                        // row stride (floats) inside a slice
+  const int ring_bytes = p.stages * stage_bytes, dump_bytes = (int)gridDim.x * GEMM_BM * XS * 4;
+  const int data_bytes = ((ring_bytes > dump_bytes ? ring_bytes : dump_bytes) + 1023) & ~1023;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + data_bytes);
+  // barrier map: full[stages] | empty[stages] | acc_full
+  const uint32_t full0 = smem_u32(bars);
+  const uint32_t empty0 = full0 + 8 * p.stages;
+  const uint32_t acc_full = empty0 + 8 * p.stages;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * p.stages + 2);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KS = gridDim.x, rank = blockIdx.x;                  // the cluster spans grid.x
+  const int nkb_s = (p.K / GEMM_BK) / KS;                       // k-blocks of this block's slice
+  const int kb0 = rank * nkb_s;
+  const int m0 = blockIdx.z * GEMM_BM, n0 = blockIdx.y * p.BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(acc_full, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_holder)), "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = *tmem_holder;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int it = 0; it < nkb_s; ++it) {
+        const int s = it % p.stages;
+        if (it >= p.stages) mbar_wait(empty0 + 8 * s, ((it / p.stages) - 1) & 1, p.status);
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        mbar_expect_tx(full0 + 8 * s, stage_bytes);
+        tma_load_2d(sa, &map_x, (kb0 + it) * GEMM_BK, m0, full0 + 8 * s);
+        tma_load_3d(sa + GEMM_A_BYTES, &map_w, 0, n0, kb0 + it, full0 + 8 * s);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(p.BN);
+      const uint64_t da0 = umma_desc_sw128(smem_u32(smem));
+      const uint64_t db0 = umma_desc_sw128(smem_u32(smem) + GEMM_A_BYTES);
+      for (int it = 0; it < nkb_s; ++it) {
+        const int s = it % p.stages;
+        mbar_wait(full0 + 8 * s, (it / p.stages) & 1, p.status);
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const uint64_t so = (uint64_t)((s * stage_bytes) >> 4);
+#pragma unroll
+        for (int k = 0; k < GEMM_BK / 16; ++k)
+          umma_bf16(tmem_base, da0 + so + 2 * k, db0 + so + 2 * k, idesc, (it | k) ? 1u : 0u);
+        umma_commit(empty0 + 8 * s);
+      }
+      umma_commit(acc_full);                       // every MMA of the slice has completed: the ring is idle too
+    }
+  } else {
+    // ---- this block's partial tile: TMEM (lane = row) -> shared memory, fp32 [128][XS]
+    const int lane_base = (warp & 3) * 32;
+    const int row = lane_base + lane;
+    float* dump = reinterpret_cast<float*>(smem);
+    mbar_wait(acc_full, 0, p.status);
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    for (int c0 = 0; c0 < p.BN; c0 += 16) {
+      uint32_t r[16];
+      tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + c0, r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+      for (int k = 0; k < 16; k += 4) {
+        const int c = c0 + k, sl = c / cw;
+        *reinterpret_cast<uint4*>(dump + ((size_t)sl * GEMM_BM + row) * XS + (c - sl * cw)) = make_uint4(r[k], r[k + 1], r[k + 2], r[k + 3]);
+      }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  }
+  // every block's partial tile is complete and visible
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+  if (warp >= 2) {
+    const int t = (warp - 2) * 32 + lane;
+    if (KS == 8) splitk_reduce<8>(p, smem_u32(smem), rank, cw, m0, n0, t);
+    else if (KS == 4) splitk_reduce<4>(p, smem_u32(smem), rank, cw, m0, n0, t);
+    else splitk_reduce<2>(p, smem_u32(smem), rank, cw, m0, n0, t);
+  }
+  // nobody leaves while a peer may still read its partial tile
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
   __syncthreads();
   if (warp == 1) {

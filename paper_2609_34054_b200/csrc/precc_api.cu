@@ -29,6 +29,7 @@ struct precc_ctx {
   size_t trace_blocks = 0;
   bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
   bool force_tiled_gemm = false;       // PRECC_GEMM=tiled in the environment: never take the few-row kernel
+  bool no_gemm_splitk = false;         // PRECC_GEMM_SPLITK=0 in the environment: short turns stay on the one-block-per-tile GEMM
   bool force_ticket_decode = false;    // PRECC_DECODE=ticket in the environment: never use the cluster decode kernel
   bool deep_clusters = true;           // PRECC_DEEP=0 in the environment: never use the one-block-per-SM deep-ring clusters
   bool prefill_forward = false;        // PRECC_PREFILL_ORDER=forward: row tiles in ascending order (default: longest causal reach first)
@@ -244,11 +245,84 @@ int32_t launch_small(precc_ctx* ctx, const void* X, int M, int K, const void* Wt
 }
 
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
-  if (M <= PS_MAX_M && !ctx->force_tiled_gemm) {
+  // Up to 40 rows the weight-streaming few-row kernel is the fastest (fused C3 projection: 8.7 us at 16 rows, 11.6 at
+  // 32); from there to 384 rows the split-K kernel (15..22 us; the few-row kernel needs 16.5 us at 48 rows and 18.4 at
+  // 64, the one-block-per-tile GEMM 27 us throughout); the few-row kernel still takes 41..64 rows when the split does
+  // not apply (rotary epilogue, short K).
+  if (M <= 40 && !ctx->force_tiled_gemm) {
     const int32_t rc = launch_small(ctx, X, M, K, Wt, n_out, gp, stream);
     if (rc >= 0) return rc;
   }
   const int m_tiles = (M + GEMM_BM - 1) / GEMM_BM;
+  // A few row tiles (the tokens of a short turn): the K extent of every tile is split over a cluster.  The split
+  // depends on M and K alone, so a column's summation order is the same whichever entry point produced it.
+  if (m_tiles <= 4 && !gp.rope && !ctx->no_gemm_splitk) {
+    const int nkb = K / GEMM_BK;
+    // planned for the width of the FUSED projection of this layer, whatever this call projects, so that the base-only,
+    // LR-only and fused calls of one M take the same decision (and with it the same summation order)
+    const int n_fused = 2 * gp.n_kv * gp.hd + gp.n_agents * (gp.rank_k + gp.rank_v);
+    // 256-column tiles, one block per SM (a kernel that allocates tensor memory is given one block per SM)
+    const int bn = n_out >= 256 ? 256 : (n_out + 15) / 16 * 16;
+    const int stage_bytes = GEMM_A_BYTES + 256 * GEMM_BK * 2;
+    const int dump_max = GEMM_MAX_KS * GEMM_BM * (256 / GEMM_MAX_KS + 4) * 4;             // widest tile, finest split
+    const int ring_max = 3 * stage_bytes;
+    const int smem_plan = (((ring_max > dump_max ? ring_max : dump_max) + 1023) & ~1023) + (2 * 3 + 4) * 8;   // the same for every width
+    const long long clusters = (long long)m_tiles * ((n_fused + 255) / 256);
+    int ks = 8;
+    for (; ks > 2; ks >>= 1) {                                   // a two-way split does not pay for its merge
+      if (nkb % ks != 0 || nkb / ks < 2) continue;
+      // every cluster must be resident at once (a second wave would cost more than the split gains)
+      static int max_clusters_dev[kMaxDevices][GEMM_MAX_KS + 1] = {{0}};   // 0 = unknown, else max active clusters + 1
+      int& cached = max_clusters_dev[ctx->device % kMaxDevices][ks];
+      if (cached == 0) {
+        int n = 0;
+        if (raise_smem_limit(ctx, proj_gemm_splitk_kernel, smem_plan) == cudaSuccess) {
+          cudaLaunchConfig_t qc = {};
+          qc.gridDim = dim3(ks, ctx->sm_count, 1); qc.blockDim = dim3(GEMM_THREADS); qc.dynamicSmemBytes = smem_plan;
+          cudaLaunchAttribute qa[1];
+          qa[0].id = cudaLaunchAttributeClusterDimension;
+          qa[0].val.clusterDim.x = ks; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+          qc.attrs = qa; qc.numAttrs = 1;
+          if (cudaOccupancyMaxActiveClusters(&n, proj_gemm_splitk_kernel, &qc) != cudaSuccess) { cudaGetLastError(); n = 0; }
+        } else {
+          cudaGetLastError();
+        }
+        cached = n + 1;
+      }
+      if (cached - 1 >= clusters) break;
+    }
+    if (ks > 2) {
+      const int n_tiles = (n_out + bn - 1) / bn;
+      int stages = 3;
+      if (stages > nkb / ks) stages = nkb / ks;
+      int tmem_cols = 32;
+      while (tmem_cols < bn) tmem_cols <<= 1;
+      CUtensorMap map_x, map_w;
+      int32_t rc = make_map(ctx, &map_x, X, M, K, GEMM_BM);
+      if (rc) return rc;
+      rc = make_map_w(ctx, &map_w, Wt, n_out, K, bn);
+      if (rc) return rc;
+      gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
+      gp.spread_rows = 0;
+      gp.status = ctx->status;
+      PRECC_CUDA(ctx, raise_smem_limit(ctx, proj_gemm_splitk_kernel, smem_plan));
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(ks, n_tiles, m_tiles);
+      cfg.blockDim = dim3(GEMM_THREADS);
+      cfg.dynamicSmemBytes = smem_plan;
+      cfg.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = ks; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+      PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, proj_gemm_splitk_kernel, map_x, map_w, gp));
+      return PRECC_OK;
+    }
+  }
+  if (M <= PS_MAX_M && !ctx->force_tiled_gemm) {
+    const int32_t rc = launch_small(ctx, X, M, K, Wt, n_out, gp, stream);
+    if (rc >= 0) return rc;
+  }
   int bn = pick_bn(n_out, m_tiles, ctx->sm_count);
   if (gp.rope && bn % gp.hd != 0) bn = gp.hd;        // a head's two halves must sit in one tile
   const int n_tiles = (n_out + bn - 1) / bn;
@@ -770,6 +844,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   if (const char* v = getenv("PRECC_PREFILL")) ctx->force_simple_prefill = (strcmp(v, "simple") == 0);
   if (const char* v = getenv("PRECC_GEMM")) ctx->force_tiled_gemm = (strcmp(v, "tiled") == 0);
   if (const char* v = getenv("PRECC_DEEP")) ctx->deep_clusters = (strcmp(v, "0") != 0);
+  if (const char* v = getenv("PRECC_GEMM_SPLITK")) ctx->no_gemm_splitk = (strcmp(v, "0") == 0);
   if (const char* v = getenv("PRECC_DECODE")) ctx->force_ticket_decode = (strcmp(v, "ticket") == 0);
   if (const char* v = getenv("PRECC_PREFILL_ORDER")) ctx->prefill_forward = (strcmp(v, "forward") == 0);
   if (const char* v = getenv("PRECC_PREFILL_SPLIT")) ctx->no_prefill_split = (strcmp(v, "0") == 0);

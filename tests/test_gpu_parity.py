@@ -553,3 +553,43 @@ def test_decode_alternating_between_ring_layouts_of_one_shape(px):
         ref = O.lr_decode_reference(f64(q), [1], [ctx], *args, geo.scale_k, geo.scale_v, geo.n_kv)
         assert_close(got, ref, f"alternating layouts, ctx {ctx}")
     assert px.poll_status() == 0
+
+
+@pytest.mark.parametrize("M,d", [(41, 1024), (64, 2048), (100, 1024), (129, 2048), (300, 1024), (384, 4096)])
+def test_short_turn_projection_split_over_a_cluster(monkeypatch, px, M, d):
+    """41 to 384 rows (the tokens of a short turn): the K extent of every 128 x 256 tile is split over a cluster
+    of 4 or 8 blocks whose partial accumulators are merged over distributed shared memory.  Against the
+    definition, fused call bit-equal to the two separate ones, scattered slots, agent mask, untouched slots; and
+    within one bf16 ulp (plus fp32 summation noise near zero) of the one-block-per-tile kernel."""
+    geo = I.Geometry(d, 8, 2, 128, 3, 32, 32, alpha=64.0)
+    H = I.hidden_states(M, geo, seed=81, tag=f"sk.{M}.{d}")
+    nb = (M + 15) // 16 + 4
+    slots = I.permutation(nb * 16, 81, f"sk.slots.{M}")[:M].to(torch.int32)
+    La = Layer(px, geo, seed=81, n_blocks=nb, fill=float("nan"))
+    La.append(H, slot_mapping=slots.cuda(), agent_mask=0b101)
+    torch.cuda.synchronize()
+    w, Hn, sl = La.w_np, f64(H), slots.long()
+    tol = lambda ref: 2.0 ** -8 * np.abs(ref) + 2e-3 * np.sqrt(d / 256)
+    for got, ref in ((base_rows(La.cache.k_base)[sl], O.base_cache(Hn, w["W_k"])), (base_rows(La.cache.v_base)[sl], O.base_cache(Hn, w["W_v"])),
+                     (lr_rows(La.cache.lr_k, 0)[sl], O.lr_cache(Hn, w["A_k"][0])), (lr_rows(La.cache.lr_v, 2)[sl], O.lr_cache(Hn, w["A_v"][2]))):
+        assert (np.abs(got - ref) <= tol(ref)).all()
+    assert torch.isnan(La.cache.lr_k[1]).all()
+    untouched = torch.ones(nb * 16, dtype=torch.bool); untouched[sl] = False
+    assert torch.isnan(La.cache.v_base.permute(0, 2, 1, 3).reshape(nb * 16, -1)[untouched]).all()
+    Lb = Layer(px, geo, seed=81, n_blocks=nb, fill=float("nan"))
+    dev = {k: v.cuda() for k, v in Lb.w.items()}
+    WA = px.pack_turn_weights(geo, dev["W_k"], dev["W_v"], dev["A_k"], dev["A_v"])
+    px.turn_project(Lb.desc, H.cuda(), WA, Lb.cache, 0, slots.cuda(), 0b101)
+    torch.cuda.synchronize()
+    for name in ("k_base", "v_base", "lr_k", "lr_v"):
+        assert torch.equal(getattr(La.cache, name).view(torch.int16), getattr(Lb.cache, name).view(torch.int16)), name
+    monkeypatch.setenv("PRECC_GEMM_SPLITK", "0")
+    monkeypatch.setenv("PRECC_GEMM", "tiled")
+    px2 = Precc(0)
+    Lc = Layer(px2, geo, seed=81, n_blocks=nb, fill=float("nan"))
+    px2.turn_project(Lc.desc, H.cuda(), WA, Lc.cache, 0, slots.cuda(), 0b101)
+    torch.cuda.synchronize()
+    a, b = base_rows(Lb.cache.k_base)[sl], base_rows(Lc.cache.k_base)[sl]
+    assert (np.abs(a - b) <= 2.0 ** -7 * np.abs(b) + 2e-4).all()      # another summation order: one bf16 ulp, or fp32 noise near zero
+    assert px.poll_status() == 0 and px2.poll_status() == 0
+    px2.close()
