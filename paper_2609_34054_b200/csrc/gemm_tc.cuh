@@ -334,7 +334,7 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 }
 
 
-// Reduce step of the split-K kernel: thread t of the 128 epilogue threads takes the 16-byte pieces t, t + 128, ...
+// Reduce step of the split-K kernel: thread t of the block's 192 threads takes the 16-byte pieces t, t + 192, ...
 // of this block's slice (piece f = row * cw/4 + q), 16 / KS of them at a time, so that sixteen loads over
 // distributed shared memory are in flight per thread; consecutive lanes read consecutive pieces of a peer; the
 // peers are summed in rank order.  The odd piece of a pair hands its four columns to the even one, which
@@ -345,15 +345,15 @@ __device__ __forceinline__ void splitk_reduce(const GemmParams& p, uint32_t smem
   const int XS = cw + 4, qpr = cw / 4;
   const uint32_t slice = smem_base + (uint32_t)rank * GEMM_BM * XS * 4;
   const int total = GEMM_BM * qpr;                              // a multiple of 128
-  for (int f0 = t; f0 < total; f0 += 128 * G) {
+  for (int f0 = t; f0 < total; f0 += GEMM_THREADS * G) {
     float4 a[G][KS];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const int f = f0 + g * 128;
+      const int f = f0 + g * GEMM_THREADS;
       const int row = f / qpr, q = f % qpr;
 #pragma unroll
       for (int r = 0; r < KS; ++r) {
-        if (f < total) {
+        if (f < total && m0 + row < p.M) {                        // rows past M are never stored: not fetched either
           uint32_t remote;
           asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(slice + (uint32_t)(row * XS + 4 * q) * 4), "r"(r));
           asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];\n" : "=f"(a[g][r].x), "=f"(a[g][r].y), "=f"(a[g][r].z), "=f"(a[g][r].w) : "r"(remote));
@@ -364,7 +364,7 @@ __device__ __forceinline__ void splitk_reduce(const GemmParams& p, uint32_t smem
     }
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const int f = f0 + g * 128;
+      const int f = f0 + g * GEMM_THREADS;
       const int row = f / qpr, q = f % qpr;
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -496,8 +496,8 @@ proj_gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   __syncwarp();
   asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
-  if (warp >= 2) {
-    const int t = (warp - 2) * 32 + lane;
+  {
+    const int t = threadIdx.x;                                  // the producer and MMA warps help with the merge
     if (KS == 8) splitk_reduce<8>(p, smem_u32(smem), rank, cw, m0, n0, t);
     else if (KS == 4) splitk_reduce<4>(p, smem_u32(smem), rank, cw, m0, n0, t);
     else splitk_reduce<2>(p, smem_u32(smem), rank, cw, m0, n0, t);

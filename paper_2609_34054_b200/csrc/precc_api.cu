@@ -246,7 +246,7 @@ int32_t launch_small(precc_ctx* ctx, const void* X, int M, int K, const void* Wt
 
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
   // Up to 40 rows the weight-streaming few-row kernel is the fastest (fused C3 projection: 8.7 us at 16 rows, 11.6 at
-  // 32); from there to 384 rows the split-K kernel (15..22 us; the few-row kernel needs 16.5 us at 48 rows and 18.4 at
+  // 32); from there to 384 rows the split-K kernel (14..20 us; the few-row kernel needs 16.5 us at 48 rows and 18.4 at
   // 64, the one-block-per-tile GEMM 27 us throughout); the few-row kernel still takes 41..64 rows when the split does
   // not apply (rotary epilogue, short K).
   if (M <= 40 && !ctx->force_tiled_gemm) {
