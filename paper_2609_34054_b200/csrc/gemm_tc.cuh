@@ -435,6 +435,14 @@ proj_gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     mbar_init(acc_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    // the ring's first fill is requested right away (this thread is the producer): its latency then overlaps the
+    // tensor-memory allocation and the block barrier below
+    for (int it = 0; it < min(p.stages, nkb_s); ++it) {
+      const uint32_t sa = smem_u32(smem + (size_t)it * stage_bytes);
+      mbar_expect_tx(full0 + 8 * it, stage_bytes);
+      tma_load_2d(sa, &map_x, (kb0 + it) * GEMM_BK, m0, full0 + 8 * it);
+      tma_load_3d(sa + GEMM_A_BYTES, &map_w, 0, n0, kb0 + it, full0 + 8 * it);
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_holder)), "r"(p.tmem_cols) : "memory");
@@ -447,9 +455,9 @@ proj_gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
 
   if (warp == 0) {
     if (lane == 0) {
-      for (int it = 0; it < nkb_s; ++it) {
+      for (int it = p.stages; it < nkb_s; ++it) {          // the first fill was issued above
         const int s = it % p.stages;
-        if (it >= p.stages) mbar_wait(empty0 + 8 * s, ((it / p.stages) - 1) & 1, p.status);
+        mbar_wait(empty0 + 8 * s, ((it / p.stages) - 1) & 1, p.status);
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
         mbar_expect_tx(full0 + 8 * s, stage_bytes);
         tma_load_2d(sa, &map_x, (kb0 + it) * GEMM_BK, m0, full0 + 8 * s);
