@@ -143,7 +143,7 @@ N_PROJ = max(12, N_CASES // 3)
 
 def _proj_case(i: int):
     rng = np.random.default_rng(5000 + i)
-    d = int(rng.choice([64, 128, 192, 320, 1024]))
+    d = int(rng.choice([64, 128, 192, 320, 1024, 2048]))           # 1024 and 2048: deep enough for the split-K kernel
     hd = int(rng.choice([64, 128]))
     n_kv = int(rng.choice([1, 2, 3]))
     r = int(rng.choice([8, 16, 32, 64]))
