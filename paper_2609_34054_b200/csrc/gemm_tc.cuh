@@ -391,7 +391,7 @@ __device__ __forceinline__ void splitk_reduce(const GemmParams& p, uint32_t smem
 // Split-K form for a few row tiles (64 < M <= 512: the tokens of a short turn).  A block of the kernel
 // above needs about 0.4 us per 64-deep k-block whatever its tile width, so the whole K extent costs one
 // block 25 us at d_model 4096 even when there is almost no work.  Here the K extent of one 128 x BN tile is
-// divided over the KS = 4 or 8 blocks of a cluster (grid = (KS, column tiles, row tiles)); each block accumulates its
+// divided over the KS = 3 ... 8 blocks of a cluster (grid = (KS, column tiles, row tiles)); each block accumulates its
 // K slice in TMEM exactly as above, writes the fp32 accumulator into its own shared memory (over the ring,
 // which is idle by then), and after a cluster barrier block r adds up columns [r*cw, (r+1)*cw) of all KS
 // partial tiles over distributed shared memory — in rank order, so the result does not depend on timing —
@@ -426,8 +426,9 @@ proj_gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KS = gridDim.x, rank = blockIdx.x;                  // the cluster spans grid.x
-  const int nkb_s = (p.K / GEMM_BK) / KS;                       // k-blocks of this block's slice
-  const int kb0 = rank * nkb_s;
+  const int nkb = p.K / GEMM_BK;                                // K slices need not be equal (KS = 3, 5, 6, 7 are allowed):
+  const int kb0 = (rank * nkb) / KS;                            // slice r = [r nkb / KS, (r+1) nkb / KS), each at least
+  const int nkb_s = ((rank + 1) * nkb) / KS - kb0;              // floor(nkb / KS) >= 2 k-blocks (the host sees to that)
   const int m0 = blockIdx.z * GEMM_BM, n0 = blockIdx.y * p.BN;
 
   if (threadIdx.x == 0) {
@@ -506,9 +507,15 @@ proj_gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
   {
     const int t = threadIdx.x;                                  // the producer and MMA warps help with the merge
-    if (KS == 8) splitk_reduce<8>(p, smem_u32(smem), rank, cw, m0, n0, t);
-    else if (KS == 4) splitk_reduce<4>(p, smem_u32(smem), rank, cw, m0, n0, t);
-    else splitk_reduce<2>(p, smem_u32(smem), rank, cw, m0, n0, t);
+    switch (KS) {
+      case 8: splitk_reduce<8>(p, smem_u32(smem), rank, cw, m0, n0, t); break;
+      case 7: splitk_reduce<7>(p, smem_u32(smem), rank, cw, m0, n0, t); break;
+      case 6: splitk_reduce<6>(p, smem_u32(smem), rank, cw, m0, n0, t); break;
+      case 5: splitk_reduce<5>(p, smem_u32(smem), rank, cw, m0, n0, t); break;
+      case 4: splitk_reduce<4>(p, smem_u32(smem), rank, cw, m0, n0, t); break;
+      case 3: splitk_reduce<3>(p, smem_u32(smem), rank, cw, m0, n0, t); break;
+      default: splitk_reduce<2>(p, smem_u32(smem), rank, cw, m0, n0, t); break;
+    }
   }
   // nobody leaves while a peer may still read its partial tile
   __syncwarp();

@@ -246,7 +246,7 @@ int32_t launch_small(precc_ctx* ctx, const void* X, int M, int K, const void* Wt
 
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
   // Up to 40 rows the weight-streaming few-row kernel is the fastest (fused C3 projection: 8.7 us at 16 rows, 11.6 at
-  // 32); from there to 384 rows the split-K kernel (14..20 us; the few-row kernel needs 16.5 us at 48 rows and 18.4 at
+  // 32); from there to 512 rows the split-K kernel (13..24 us; the few-row kernel needs 16.5 us at 48 rows and 18.4 at
   // 64, the one-block-per-tile GEMM 27 us throughout); the few-row kernel still takes 41..64 rows when the split does
   // not apply (rotary epilogue, short K).
   if (M <= 40 && !ctx->force_tiled_gemm) {
@@ -264,14 +264,17 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
     // 256-column tiles, one block per SM (a kernel that allocates tensor memory is given one block per SM)
     const int bn = n_out >= 256 ? 256 : (n_out + 15) / 16 * 16;
     const int stage_bytes = GEMM_A_BYTES + 256 * GEMM_BK * 2;
-    const int dump_max = GEMM_MAX_KS * GEMM_BM * (256 / GEMM_MAX_KS + 4) * 4;             // widest tile, finest split
     const int ring_max = 3 * stage_bytes;
-    const int smem_plan = (((ring_max > dump_max ? ring_max : dump_max) + 1023) & ~1023) + (2 * 3 + 4) * 8;   // the same for every width
     const long long clusters = (long long)m_tiles * ((n_fused + 255) / 256);
-    int ks = 8;
-    for (; ks > 2; ks >>= 1) {                                   // a two-way split does not pay for its merge
-      if (nkb % ks != 0 || nkb / ks < 2) continue;
-      // every cluster must be resident at once (a second wave would cost more than the split gains)
+    // the finest split whose clusters are all resident at once (a second wave would cost more than the split gains);
+    // cluster sizes need not be powers of two: 18 clusters fit as 6-block clusters, 36 as 3-block clusters
+    int ks = GEMM_MAX_KS, smem_plan = 0;
+    for (; ks > 2; --ks) {                                       // a two-way split does not pay for its merge
+      if (nkb / ks < 2) continue;
+      const int cw = ((256 + ks - 1) / ks + 7) / 8 * 8;          // planned for the widest tile, whatever this call's width
+      const int dump = ks * GEMM_BM * (cw + 4) * 4;
+      smem_plan = (((ring_max > dump ? ring_max : dump) + 1023) & ~1023) + (2 * 3 + 4) * 8;
+      if (smem_plan > ctx->max_smem_optin) continue;
       static int max_clusters_dev[kMaxDevices][GEMM_MAX_KS + 1] = {{0}};   // 0 = unknown, else max active clusters + 1
       int& cached = max_clusters_dev[ctx->device % kMaxDevices][ks];
       if (cached == 0) {

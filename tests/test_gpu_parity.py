@@ -555,10 +555,10 @@ def test_decode_alternating_between_ring_layouts_of_one_shape(px):
     assert px.poll_status() == 0
 
 
-@pytest.mark.parametrize("M,d", [(41, 1024), (64, 2048), (100, 1024), (129, 2048), (300, 1024), (384, 4096)])
+@pytest.mark.parametrize("M,d", [(41, 1024), (64, 2048), (100, 1024), (129, 2048), (300, 1024), (384, 4096), (450, 2048), (512, 4096)])
 def test_short_turn_projection_split_over_a_cluster(monkeypatch, px, M, d):
-    """41 to 384 rows (the tokens of a short turn): the K extent of every 128 x 256 tile is split over a cluster
-    of 4 or 8 blocks whose partial accumulators are merged over distributed shared memory.  Against the
+    """41 to 512 rows (the tokens of a short turn): the K extent of every 128 x 256 tile is split over a cluster
+    of 3 to 8 blocks (K slices need not be equal) whose partial accumulators are merged over distributed shared memory.  Against the
     definition, fused call bit-equal to the two separate ones, scattered slots, agent mask, untouched slots; and
     within one bf16 ulp (plus fp32 summation noise near zero) of the one-block-per-tile kernel."""
     geo = I.Geometry(d, 8, 2, 128, 3, 32, 32, alpha=64.0)
