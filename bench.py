@@ -290,7 +290,27 @@ def extra_turn(px, T: int, S: int, seed: int = 0):
     us_attn = _event_us(torch, lambda: px.lr_attend_prefill(desc, q, cur, T, w["B_k"], w["B_v"], cache, out), 5)
     us_reb = _event_us(torch, rebase, 10)
     fl_attn = 4.0 * geo.n_q * S * (geo.hd + (geo.rank_k + geo.rank_v) / 2) * (T + S / 2)
+    # a short turn over the same context (a tool observation of 128 tokens): the projection takes the split-K
+    # kernel and the prefill splits its context over clusters
+    S2 = 128
+    H_short = [I.hidden_states(S2, geo, seed + i, "C3.H_short").cuda() for i in range(32)]
+    q2 = I.queries(S2, geo, seed, "C3.q_short").cuda()
+    out2 = torch.empty_like(q2)
+
+    def short_proj():
+        h = H_short[it[0] % 32]; it[0] += 1
+        px.turn_project(desc, h, WA_packed, cache, T)
+
+    def short_turn():
+        short_proj()
+        px.lr_attend_prefill(desc, q2, cur, T, w["B_k"], w["B_v"], cache, out2)
+    us_sproj = _event_us(torch, short_proj, 10)
+    us_sattn = _event_us(torch, lambda: px.lr_attend_prefill(desc, q2, cur, T, w["B_k"], w["B_v"], cache, out2), 10)
+    us_sturn = _event_us(torch, short_turn, 10)
+    short = {"S": S2, "projection_us": us_sproj, "prefill_attention_us": us_sattn, "turn_us_per_layer": us_sturn,
+             "turn_ttft_ms_32_layers": us_sturn * C3_LAYERS_FOR_TTFT / 1e3}
     return {"workload": f"C3 turn, one layer: d=4096 32q/8kv hd=128, N=4 r=32, T={T}, S={S}",
+            "short_turn": short,
             "lr_precompute_context": {"us": us_pre, "tflops": fl_pre / us_pre / 1e6, "n_out": n_lr,
                                       "GBps": 2.0 * (T * geo.d_model + T * n_lr) / us_pre / 1e3},
             "base_projection_context": {"us": us_base, "tflops": 2.0 * T * geo.d_model * 2 * geo.kv_width / us_base / 1e6},
