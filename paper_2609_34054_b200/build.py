@@ -1,43 +1,67 @@
-"""Build libprecc.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+"""Build libprecc.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+The library is split into several translation units (the attention kernels per head dimension, the
+projection kernels, the entry points) that are compiled side by side and linked into one shared object.
+"""
 from __future__ import annotations
 
+import concurrent.futures
 import os
 import subprocess
 import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libprecc.so")
-SOURCES = ["precc_api.cu"]
-HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith(".cuh")) + [os.path.join("..", "..", "include", "precc.h")]
+SOURCES = sorted(f for f in os.listdir(CSRC) if f.endswith(".cu"))
+HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))) + [os.path.join("..", "..", "include", "precc.h")]
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--use_fast_math",
+              "-Xcompiler", "-fPIC"]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _newest_header() -> float:
+    return max(os.path.getmtime(os.path.join(CSRC, h)) for h in HEADERS)
+
+
+def _obj(src: str) -> str:
+    return os.path.join(OBJ, src[:-3] + ".o")
+
+
+def _stale(src: str, hdr_time: float) -> bool:
+    o = _obj(src)
+    if not os.path.exists(o):
         return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, s) for s in SOURCES + HEADERS]
-    return any(os.path.getmtime(d) > t for d in deps)
+    t = os.path.getmtime(o)
+    return os.path.getmtime(os.path.join(CSRC, src)) > t or hdr_time > t
+
+
+def _compile(nvcc: str, src: str, verbose: bool) -> str:
+    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas=-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", _obj(src)]
+    r = subprocess.run(cmd, capture_output=True, text=True)
+    if r.returncode != 0:
+        raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}{r.stderr}")
+    return r.stderr
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile if missing or out of date; returns the library path."""
-    if not force and not _stale():
-        return LIB
+    """Compile what is missing or out of date, link, and return the library path."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "--use_fast_math", "-shared", "-Xcompiler", "-fPIC", "-t", "0",
-           "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
-    if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    r = subprocess.run(cmd, capture_output=True, text=True)
+    os.makedirs(OBJ, exist_ok=True)
+    hdr_time = _newest_header()
+    todo = [s for s in SOURCES if force or _stale(s, hdr_time)]
+    if not todo and os.path.exists(LIB) and all(os.path.getmtime(_obj(s)) <= os.path.getmtime(LIB) for s in SOURCES):
+        return LIB
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(len(todo), os.cpu_count() or 1) or 1) as pool:
+        for log in pool.map(lambda s: _compile(nvcc, s, verbose), todo):
+            if verbose:
+                sys.stderr.write(log)
+    r = subprocess.run([nvcc, "-shared", "-o", LIB] + [_obj(s) for s in SOURCES], capture_output=True, text=True)
     if r.returncode != 0:
         sys.stderr.write(r.stdout + r.stderr)
-        raise RuntimeError("nvcc failed building libprecc.so")
-    if verbose:
-        sys.stderr.write(r.stderr)
+        raise RuntimeError("linking libprecc.so failed")
     return LIB
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force="-f" in sys.argv, verbose="-v" in sys.argv))

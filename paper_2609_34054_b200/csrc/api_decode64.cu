@@ -1,0 +1,3 @@
+// Decode attention kernels and their launch logic for head_dim 64.
+#include "decode_run.cuh"
+PRECC_DEFINE_DECODE_UNIT(64)

@@ -1,0 +1,3 @@
+// New-turn prefill attention kernels and their launch logic for head_dim 64.
+#include "prefill_run.cuh"
+PRECC_DEFINE_PREFILL_UNIT(64)

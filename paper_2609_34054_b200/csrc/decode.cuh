@@ -59,12 +59,18 @@ struct DecodeParams {
   int table_stride;
   int n_q, n_kv, group, n_agents;
   int chunk_tiles, max_splits, stages;
+  int max_ctx;                 // the host's bound on ctx_len[b]: it sized the grid, the split and the block table
   float scale_log2, s_k, s_v;
 };
 
 constexpr int DEC_WARPS = 4;            // ticket kernel
 constexpr int DEC_MAX_SPLITS = 512;
 constexpr int DEC_MAX_CLUSTER = 16;
+// Overlap with the preceding kernel (programmatic dependent launch): before the kernel waits for its
+// predecessor it already reads the index arrays, the adapter matrices and every cache page that holds
+// none of the request's last DEC_PDL_TAIL tokens.  The newest tokens (the in-turn append of the preceding
+// few-row projection), q and every store stay behind the wait.
+constexpr int DEC_PDL_TAIL = 64;
 
 template <int HD, int RK, int RV>
 struct DecodeCfg {
@@ -129,8 +135,7 @@ __device__ __forceinline__ void load_q_frags(const DecodeParams& p, int b, int g
 // m = NEG_BIG, l = 0, O' = 0.
 template <int HD, int RK, int RV, int NW, bool ROPE>
 __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsigned char* smem, int b, int g, int ctx,
-                                                    int agent, bool use_lr, int tile0, int tile_end,
-                                                    const uint32_t (&qb)[HD / 16][2], const DecodeTrace& mark) {
+                                                    int agent, bool use_lr, int tile0, int tile_end, const DecodeTrace& mark) {
   static_assert(!ROPE || RK > 0, "the rotary variant only differs when there is a key-side adapter");
   using C = DecodeCfg<HD, RK, RV>;
   constexpr int OW = C::OW;
@@ -250,8 +255,20 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v));
     return pack_bf16(f.x * p.s_k, f.y * p.s_k);
   };
-  // ---- start the stream: every ring slot is filled at once
-  for (int i = 0; i < p.stages; ++i) issue_tile(i);
+  // ---- start the stream: every ring slot is filled at once.  Pages that cannot hold one of the request's
+  //      last DEC_PDL_TAIL tokens are requested while the preceding kernel may still be running; the wait
+  //      for that kernel comes next, and the pages it may have appended to are requested after it.
+  const int safe_tiles = max(0, ctx - DEC_PDL_TAIL) / PAGE;
+  int n_pre = 0;
+  for (; n_pre < p.stages; ++n_pre) {
+    if (n_pre < my_n && tile0 + warp + NW * n_pre >= safe_tiles) break;
+    issue_tile(n_pre);
+  }
+  pdl_wait();                 // the predecessor has completed: its q, its cache rows and its workspace are visible
+  pdl_launch_dependents();
+  uint32_t qb[HD / 16][2];
+  load_q_frags<HD>(p, b, g, qb);
+  for (int i = n_pre; i < p.stages; ++i) issue_tile(i);
   mark(2);
   const uint32_t bk_u32 = smem_u32(smem + p.bk_off);
   if constexpr (ROPE) {
@@ -336,10 +353,14 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
 
   mark(3);
   for (int i = 0; i < my_n; ++i) {
-    switch (p.stages) {
+    switch (p.stages) {                // ring depth 2 .. 8: all but the newest (depth - 1) groups have landed
       case 2: cp_async_wait<1>(); break;
       case 3: cp_async_wait<2>(); break;
-      default: cp_async_wait<3>(); break;
+      case 4: cp_async_wait<3>(); break;
+      case 5: cp_async_wait<4>(); break;
+      case 6: cp_async_wait<5>(); break;
+      case 7: cp_async_wait<6>(); break;
+      default: cp_async_wait<7>(); break;
     }
     __syncwarp();                      // page i is visible to all lanes
     if (i == 0) mark(4);
@@ -553,16 +574,18 @@ lr_attend_decode_kernel(const DecodeParams p) {
   const int cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
   const DecodeTrace mark{p.trace ? p.trace + (size_t)cta_lin * 16 : nullptr};
   mark(0);
-  pdl_wait();                 // nothing of the predecessor's output is touched before this point
-  pdl_launch_dependents();
-  uint32_t qb[HD / 16][2];    // independent of the index arrays: same round trip
-  load_q_frags<HD>(p, b, g, qb);
+  // The index arrays are read before the wait for the preceding kernel (see DEC_PDL_TAIL): they are inputs
+  // of the whole call chain, not something the kernel just before this one produces.
   const int ctx = __ldg(p.ctx_len + b);
   const int agent_raw = __ldg(p.agent_id + b);
   const bool use_lr = agent_raw >= 0;          // agent id -1: adapter-free view, base cache only
   const int agent = use_lr ? agent_raw : 0;
   __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
-  if (ctx < 1 || agent_raw < -1 || agent_raw >= p.n_agents) {
+  // A context longer than the host's bound would index past the grid, the split and the block table:
+  // rejected like a bad agent id (the same decision in every block of the request).
+  if (ctx < 1 || ctx > p.max_ctx || agent_raw < -1 || agent_raw >= p.n_agents) {
+    pdl_wait();               // `out` may still be read by the predecessor's consumers: store after the wait
+    pdl_launch_dependents();
     if (split == 0) {
       if (raw_out) {
         // an empty shard (or a rejected request) contributes the neutral record: m = -big, l = 0, O' = 0
@@ -582,7 +605,7 @@ lr_attend_decode_kernel(const DecodeParams p) {
   const int tile_end = min(n_tiles, tile0 + p.chunk_tiles);
   mark(1);
   if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
-  decode_stream_block<HD, RK, RV, DEC_WARPS, ROPE>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, qb, mark);
+  decode_stream_block<HD, RK, RV, DEC_WARPS, ROPE>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, mark);
 
   float* res = reinterpret_cast<float*>(smem);          // [m[8] | l[8] | O'[G][OW]]
   const int n_el = G * OW;
@@ -758,16 +781,14 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   const int cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
   const DecodeTrace mark{p.trace ? p.trace + (size_t)cta_lin * 16 : nullptr};
   mark(0);
-  pdl_wait();
-  pdl_launch_dependents();
-  uint32_t qb[HD / 16][2];
-  load_q_frags<HD>(p, b, g, qb);
-  const int ctx = __ldg(p.ctx_len + b);
+  const int ctx = __ldg(p.ctx_len + b);        // index arrays: read before the wait for the preceding kernel
   const int agent_raw = __ldg(p.agent_id + b);
   const bool use_lr = agent_raw >= 0;          // agent id -1: adapter-free view, base cache only
   const int agent = use_lr ? agent_raw : 0;
   __nv_bfloat16* out_bg = p.out + ((size_t)b * p.n_q + (size_t)g * G) * HD;
-  if (ctx < 1 || agent_raw < -1 || agent_raw >= p.n_agents) {   // the same decision in every block of the cluster
+  if (ctx < 1 || ctx > p.max_ctx || agent_raw < -1 || agent_raw >= p.n_agents) {   // the same decision in every block of the cluster
+    pdl_wait();
+    pdl_launch_dependents();
     if (rank == 0) {
       if (raw_out) {
         float* rec = raw_out + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;   // neutral record: m = -big, l = 0, O' = 0
@@ -797,7 +818,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     }
   }
   if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
-  decode_stream_block<HD, RK, RV, NW, ROPE>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, qb, mark);
+  decode_stream_block<HD, RK, RV, NW, ROPE>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, mark);
 
   // own result res = [m[8] | l[8] | O'[G][OW]] sits at the start of shared memory in every block
   float* res = reinterpret_cast<float*>(smem);

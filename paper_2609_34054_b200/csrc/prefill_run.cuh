@@ -1,0 +1,158 @@
+// Host side of new-turn prefill attention: kernel choice (tcgen05 kernel or the mma.sync kernel), tensor maps,
+// the cluster split of short turns and the launch.  Included by one translation unit per head dimension.
+#pragma once
+#include "api_internal.h"
+#include "prefill.cuh"
+#include "prefill_tc.cuh"
+
+namespace precc {
+
+template <int HD, int RK, int RV>
+struct PrefillRun {
+  // tensor-core kernel (tcgen05 + TMEM + TMA) for the shapes it supports
+  static int32_t run_tc(precc_ctx* ctx, const PrefillArgs& a) {
+    using C = PrefillTcCfg<HD, RK, RV>;
+    const precc_layer_desc* d = a.d;
+    const int G = d->n_q_heads / d->n_kv_heads;
+    // as deep as shared memory allows, keys first (they are needed one step earlier)
+    // (head_dim 128 with rank 64 has room for a single value stage: 48 KB per stage of either kind)
+    int ks = 2, vs = 1;
+    if (C::smem_bytes(ks, vs) > ctx->max_smem_optin) return run_simple<false>(ctx, a);
+    while (ks + vs < 8) {
+      if (ks <= vs && C::smem_bytes(ks + 1, vs) <= ctx->max_smem_optin) ++ks;
+      else if (C::smem_bytes(ks, vs + 1) <= ctx->max_smem_optin) ++vs;
+      else break;
+    }
+    const int smem = C::smem_bytes(ks, vs);
+    const size_t kvw = (size_t)d->n_kv_heads * HD;
+    const long long kv_rows = (long long)a.cache->n_blocks * d->n_kv_heads * PAGE;
+    const long long lr_rows = (long long)a.cache->n_blocks * PAGE;
+    CUtensorMap mk, mv, mlk, mlv;
+    // without a block table the pages of a 128-token stage are consecutive: whole-stage boxes (one TMA
+    // instruction per 64-column slab instead of one per page)
+    const bool contig = a.block_table == nullptr;
+    const int box_rows = contig ? PTC_TOK : PAGE;
+    int32_t rc = contig ? make_map_cache4(ctx, &mk, a.cache->k_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
+                        : make_map2(ctx, &mk, a.cache->k_base, kv_rows, HD, PAGE, 64);
+    if (rc) return rc;
+    rc = contig ? make_map_cache4(ctx, &mv, a.cache->v_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
+                : make_map2(ctx, &mv, a.cache->v_base, kv_rows, HD, PAGE, 64);
+    if (rc) return rc;
+    mlk = mk; mlv = mv;     // placeholders when a rank is zero (never dereferenced)
+    if (RK) { rc = make_map2(ctx, &mlk, (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * lr_rows * RK, lr_rows, RK, box_rows, C::RKP); if (rc) return rc; }
+    if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, box_rows, 64); if (rc) return rc; }
+    PrefillTcParams p;
+    p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;
+    p.B_k = RK ? (const __nv_bfloat16*)a.B_k + (size_t)a.agent * RK * kvw : nullptr;
+    p.B_v = RV ? (const __nv_bfloat16*)a.B_v + (size_t)a.agent * RV * kvw : nullptr;
+    p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
+    p.S = a.S; p.T = a.T; p.first_block = a.first_block; p.contig = contig ? 1 : 0;
+    p.longest_first = ctx->prefill_forward ? 0 : 1;
+    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.k_stages = ks; p.v_stages = vs;
+    p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
+    p.trace = (ctx->trace && ctx->trace_blocks >= 32) ? ctx->trace : nullptr;
+    auto kern = lr_attend_prefill_tc_kernel<HD, RK, RV>;
+    PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, smem));
+    const int row_tiles = (a.S + p.tok_per_tile - 1) / p.tok_per_tile;
+    // Short turn over a long context: too few (row tile, kv head) blocks to fill the machine, so the
+    // context of each is split over a cluster of up to 8 blocks whose partial results merge over DSMEM.
+    int ns = 1;
+    const long long base_blocks = (long long)row_tiles * d->n_kv_heads;
+    const int steps = (a.T + a.S + PTC_TOK - 1) / PTC_TOK;
+    if (!ctx->no_prefill_split && C::SPLIT_BYTES <= C::Q_BYTES + C::QX_BYTES + ks * C::KSTAGE + vs * C::VSTAGE) {
+      ns = (int)(ctx->sm_count / base_blocks);          // as many as keep the grid within one block per SM
+      if (ns > 8) ns = 8;
+      if (ns > steps / 8) ns = steps / 8;               // at least eight steps per block
+      if (ns < 1) ns = 1;
+      // every cluster must be resident at once (one block per SM, and a cluster lives inside one GPC): ask
+      // the occupancy calculator once per cluster size, and shrink the clusters until the grid fits in one wave
+      static int max_clusters_dev[kMaxDevices][9] = {{0}};   // 0 = unknown, else max active clusters + 1
+      std::lock_guard<std::recursive_mutex> lk(lazy_mu());
+      int* max_clusters = max_clusters_dev[ctx->device % kMaxDevices];
+      while (ns > 1) {
+        if (max_clusters[ns] == 0) {
+          cudaLaunchConfig_t qc = {};
+          qc.gridDim = dim3(1, 1, ns * (ctx->sm_count / ns)); qc.blockDim = dim3(PTC_THREADS); qc.dynamicSmemBytes = smem;
+          cudaLaunchAttribute qa[1];
+          qa[0].id = cudaLaunchAttributeClusterDimension;
+          qa[0].val.clusterDim.x = 1; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = ns;
+          qc.attrs = qa; qc.numAttrs = 1;
+          int n = 0;
+          if (cudaOccupancyMaxActiveClusters(&n, kern, &qc) != cudaSuccess) { cudaGetLastError(); n = 0; }
+          max_clusters[ns] = n + 1;
+        }
+        if (max_clusters[ns] - 1 >= base_blocks) break;
+        --ns;
+      }
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(row_tiles, d->n_kv_heads, ns);
+    cfg.blockDim = dim3(PTC_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = ns;
+    cfg.attrs = attr; cfg.numAttrs = ns > 1 ? 1 : 0;
+    PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, mk, mv, mlk, mlv, p));
+    return PRECC_OK;
+  }
+  static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
+    if constexpr (PrefillTcCfg<HD, RK, RV>::supported) {
+      const long long kv_rows = (long long)a.cache->n_blocks * a.d->n_kv_heads * PAGE;
+      const bool aligned128 = ((reinterpret_cast<uintptr_t>(a.cache->k_base) | reinterpret_cast<uintptr_t>(a.cache->v_base) |
+                                reinterpret_cast<uintptr_t>(a.cache->lr_k) | reinterpret_cast<uintptr_t>(a.cache->lr_v)) & 127u) == 0;
+      if (kv_rows < (1ll << 31) && aligned128 && !ctx->force_simple_prefill) return run_tc(ctx, a);
+    }
+    return run_simple<false>(ctx, a);
+  }
+  // mma.sync kernel: oversized or unaligned caches, and the rotary variant
+  template <bool ROPE = false>
+  static int32_t run_simple(precc_ctx* ctx, const PrefillArgs& a) {
+    using C = PrefillCfg<HD, RK, RV>;
+    const precc_layer_desc* d = a.d;
+    int stages = 3;
+    while (stages > 2 && 2 * (C::smem_bytes(stages, ROPE) + 1024) > ctx->max_smem_optin) --stages;
+    const int smem = C::smem_bytes(stages, ROPE);
+    PrefillParams p;
+    const size_t kvw = (size_t)d->n_kv_heads * HD;
+    p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;
+    p.k_base = (const __nv_bfloat16*)a.cache->k_base; p.v_base = (const __nv_bfloat16*)a.cache->v_base;
+    p.lr_k = RK ? (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * a.cache->n_blocks * PAGE * RK : nullptr;
+    p.lr_v = RV ? (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * a.cache->n_blocks * PAGE * RV : nullptr;
+    p.B_k = RK ? (const __nv_bfloat16*)a.B_k + (size_t)a.agent * RK * kvw : nullptr;
+    p.B_v = RV ? (const __nv_bfloat16*)a.B_v + (size_t)a.agent * RV * kvw : nullptr;
+    p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
+    p.S = a.S; p.T = a.T; p.first_block = a.first_block;
+    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = d->n_q_heads / d->n_kv_heads; p.stages = stages;
+    p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
+    p.rope = reinterpret_cast<const float4*>(a.rope); p.max_pos = a.max_pos;
+    auto kern = lr_attend_prefill_kernel<HD, RK, RV, ROPE>;
+    PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, smem));
+    const int row_tiles = (a.S * p.group + PF_ROWS - 1) / PF_ROWS;
+    kern<<<dim3(row_tiles, d->n_kv_heads), PF_THREADS, smem, a.stream>>>(p);
+    PRECC_CUDA(ctx, cudaGetLastError());
+    return PRECC_OK;
+  }
+};
+
+// Rotary keys: without a key-side adapter the rotated base cache is all there is (the position-free
+// kernels are exact); with one, the mma.sync kernel expands and rotates the rank-r key term per tile.
+template <int HD, int RK, int RV>
+struct PrefillRunRope {
+  static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
+    if constexpr (RK > 0) return PrefillRun<HD, RK, RV>::template run_simple<true>(ctx, a);
+    else return PrefillRun<HD, RK, RV>::run(ctx, a);
+  }
+};
+
+
+}  // namespace precc
+
+#define PRECC_DEFINE_PREFILL_UNIT(HD)                                                                         \
+  namespace precc {                                                                                           \
+  int32_t prefill_run_hd##HD(precc_ctx* ctx, const PrefillArgs& a, int rk, int rv) {                          \
+    if (a.rope) return dispatch_ranks<PrefillRunRope, HD>(ctx, rk, rv, a);                                    \
+    return dispatch_ranks<PrefillRun, HD>(ctx, rk, rv, a);                                                    \
+  }                                                                                                           \
+  }

@@ -30,7 +30,7 @@
 #pragma once
 #include <type_traits>
 
-#include "gemm_tc.cuh"
+#include "tc_common.cuh"
 
 namespace precc {
 

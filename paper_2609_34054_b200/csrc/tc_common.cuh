@@ -1,0 +1,117 @@
+// Shared pieces of the tcgen05 / TMEM / TMA kernels: the projection parameters and tile constants, bounded
+// mbarrier waits, TMA loads, shared-memory matrix descriptors, tcgen05.mma / commit / ld wrappers.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace precc {
+
+struct GemmParams {
+  int M, N_out, K;
+  int BN, stages, tmem_cols;
+  int spread_rows;                // 1: even row-tile spreading allowed (rows may be written twice, identically)
+  int mode;                       // 0 = LR caches, 1 = base caches, 2 = base columns then LR columns
+  const int32_t* slot_mapping;    // [M] or null
+  int64_t start_slot;
+  int64_t n_blocks;
+  __nv_bfloat16* base_k;          // modes 1, 2
+  __nv_bfloat16* base_v;
+  __nv_bfloat16* lr_k;            // modes 0, 2
+  __nv_bfloat16* lr_v;
+  int n_agents, rank_k, rank_v;
+  unsigned long long agent_mask;
+  const unsigned long long* row_masks;   // optional [M]: per-row agent masks (double batching), overrides agent_mask
+  int n_kv, hd;
+  // rotary keys (modes 1, 2; null = none): the key columns of a row are rotated by the row's position
+  // before they are stored (rotate-half pairing (c, c + hd/2)); needs BN % hd == 0
+  const float4* rope;             // [max_pos][hd/4] of (cos c, sin c, cos c+1, sin c+1), c even
+  const int32_t* positions;       // [M] or null (start_pos + row)
+  int64_t start_pos;
+  int max_pos;
+  uint32_t* status;
+};
+
+constexpr int GEMM_BM = 128;
+constexpr int GEMM_BK = 64;                 // 64 bf16 = one 128-byte swizzle row
+constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_MAX_KS = 8;            // largest K split of the split-K kernel (cluster size)
+constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait (about a second of SM clock).  Returns false after recording a timeout.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (clock64() - t0 > 2000000000LL) break;
+    // once any wait in the grid has expired the results are void anyway: do not queue up more seconds
+    if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
+  }
+  atomicOr(status, StatusBits::TIMEOUT);
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
+// 1024 bytes apart (start >> 4 | LBO(ignored) | SBO = 1024 >> 4 | version 1 | layout SWIZZLE_128B).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(GEMM_BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+
+}  // namespace precc
