@@ -19,10 +19,11 @@
  * Conventions
  *   - All tensors are bf16 in DEVICE memory unless stated; all accumulation is fp32; stores round to
  *     nearest even.  Index arrays are int32 in DEVICE memory unless stated.
- *   - Every buffer is owned by the caller.  The library allocates no device memory; it keeps no
- *     pointer after the work it enqueued on `stream` has completed.  `stream` is a cudaStream_t
- *     passed as void* (NULL = the default stream).  All calls are asynchronous with respect to the
- *     host and can be captured into a CUDA graph (none synchronises, none allocates).
+ *   - Every buffer is owned by the caller.  Apart from the 4-byte status word that precc_create obtains
+ *     (and precc_destroy releases) the library allocates no device memory; it keeps no pointer after the
+ *     work it enqueued on `stream` has completed.  `stream` is a cudaStream_t passed as void* (NULL = the
+ *     default stream).  The compute calls are asynchronous with respect to the host and can be captured
+ *     into a CUDA graph (they neither synchronise nor allocate; precc_poll_status synchronises).
  *   - Return value: PRECC_OK or an error code.  On a host-detected error nothing is launched and no
  *     output is touched.  Text for the last error of a context: precc_last_error().
  *   - A context may be used from one host thread at a time; different contexts may be used from
@@ -150,7 +151,10 @@ int32_t precc_rebase_project(precc_ctx* ctx, const precc_layer_desc* desc, const
  *   WA_packed  2*n_kv_heads*head_dim + n_agents*(rank_k+rank_v) packed rows: the W rows followed by the A
  *              rows (precc_pack_kmajor into one buffer of that many rows)
  *   agent_mask selects the LR caches written; the base rows are always written.
- * Results are bit-identical to precc_rebase_project followed by precc_lr_precompute. */
+ * Results are bit-identical to precc_rebase_project followed by precc_lr_precompute with the same M (the
+ * three calls pick their kernel from M, d_model and the layer's fused width alone, so they agree).  The same
+ * row projected in calls of different M may differ in the last bf16 bit: few rows (a decode step), a short
+ * turn and a long segment run on three kernels whose fp32 summation orders differ. */
 int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
                            const void* WA_packed, const int32_t* slot_mapping, int64_t start_slot,
                            uint64_t agent_mask, const precc_cache* cache, void* stream);
@@ -159,10 +163,18 @@ int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const v
  * adapter-free sequence of a turn ride in one batch — the adapted rows write only the current agent's LR
  * rows, the adapter-free rows write the other agents').  Every row writes its base rows at its own slot, so
  * the two sequences must map to different slots (e.g. private blocks for the adapted one).
- *   slot_mapping     [M] required;  row_agent_masks  device uint64 [M], bit k = write agent k for that row */
+ *   slot_mapping     [M] required;  row_agent_masks  device uint64 [M], bit k = write agent k for that row
+ *   lr_copy_slots    optional device int32 [M] (NULL = none): a second slot that also receives the LR rows the
+ *                    row writes (entry < 0: none for that row).  The adapted sequence keeps its base rows in
+ *                    private blocks, which are dropped after the turn, but its own LR rows (built from the
+ *                    adapted hidden states, Section 3.2) belong to the shared trajectory for good: they are
+ *                    written at the private slot, where this turn's attention finds them through the adapted
+ *                    block table, and at the token's shared slot.  A slot >= 16*n_blocks raises
+ *                    PRECC_STATUS_BAD_INDEX. */
 int32_t precc_turn_project_rows(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M,
                                 const void* WA_packed, const int32_t* slot_mapping,
-                                const uint64_t* row_agent_masks, const precc_cache* cache, void* stream);
+                                const uint64_t* row_agent_masks, const int32_t* lr_copy_slots,
+                                const precc_cache* cache, void* stream);
 
 /* Workspace size for precc_lr_attend_decode with at most max_batch requests of at most max_ctx tokens
  * on a device with `sm_count` SMs: an upper bound over every such call (a smaller batch splits each request
@@ -188,7 +200,18 @@ int32_t precc_workspace_init(precc_ctx* ctx, void* workspace, size_t workspace_b
  *                 the context across thread blocks, so results are bit-identical for any block
  *                 placement given the same (B, max_ctx)
  *   B_k, B_v      [n_agents][rank][n_kv_heads*head_dim]
- * B == 0 is a no-op. */
+ * A request whose ctx_len exceeds max_ctx is rejected on the device: zeros, PRECC_STATUS_BAD_INDEX.
+ * B == 0 is a no-op.
+ * Overlap with the kernel before it on the stream.  The launch is a programmatic dependent launch: where the
+ * preceding kernel permits it (of this library: another decode or combine launch, and the few-row projection
+ * that serves calls of at most 64 rows; kernels of other libraries normally do not) the decode kernel starts
+ * while that kernel still runs and, before it waits for it to finish, already reads ctx_len, agent_id, the block
+ * table / first_block, B_k, B_v and every cache page that holds none of the request's last 64 tokens (logical
+ * positions ctx_len-64 .. ctx_len-1).  q, the pages holding those last 64 tokens and every store come after the
+ * wait.  So the immediately preceding kernel may produce q and may append or overwrite the request's newest
+ * tokens (the in-turn append of Section 3.1, the ReBaseShared overwrite of a just-appended short segment), but
+ * if it is one of the kernels named above it must not write the index arrays, the B matrices or older cache
+ * rows of the attended requests; put any other kernel or an event between the two otherwise. */
 int32_t precc_lr_attend_decode(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t B,
                                const int32_t* agent_id, const int32_t* ctx_len,
                                const int32_t* block_table, int32_t table_stride,

@@ -88,7 +88,7 @@ def load_library() -> C.CDLL:
                                                 C.POINTER(CacheDesc), vp, vp, sz, vp]
     lib.precc_lr_attend_prefill_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp, rp,
                                                  C.POINTER(CacheDesc), vp, vp]
-    lib.precc_turn_project_rows.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, C.POINTER(CacheDesc), vp]
+    lib.precc_turn_project_rows.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, vp, C.POINTER(CacheDesc), vp]
     lib.precc_partial_record_floats.argtypes = [C.POINTER(LayerDesc)]
     lib.precc_partial_record_floats.restype = sz
     lib.precc_lr_attend_decode_partial.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, i32, vp, i32, vp,
@@ -119,14 +119,6 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
-
-
-def rope_table(max_pos: int, hd: int, theta: float = 10000.0, device="cuda") -> torch.Tensor:
-    """The rotary table the *_rope calls take: fp32 [max_pos][hd/2][2] = (cos, sin) of t * theta^(-2c/hd)
-    (angles evaluated in fp64, then rounded once)."""
-    inv = torch.pow(torch.tensor(theta, dtype=torch.float64), -torch.arange(hd // 2, dtype=torch.float64) * 2.0 / hd)
-    ang = torch.arange(max_pos, dtype=torch.float64)[:, None] * inv[None, :]
-    return torch.stack([torch.cos(ang), torch.sin(ang)], dim=-1).to(torch.float32).contiguous().to(device)
 
 
 class Cache:
@@ -244,13 +236,17 @@ class Precc:
                                                 C.byref(cd), _stream()), "precc_turn_project")
 
     def turn_project_rows(self, desc: LayerDesc, H: torch.Tensor, WA_packed: torch.Tensor, cache: Cache,
-                          slot_mapping: torch.Tensor, row_masks: torch.Tensor):
-        """Fused projection with one agent mask per row (row_masks: int64 tensor holding the uint64 bit masks)."""
+                          slot_mapping: torch.Tensor, row_masks: torch.Tensor, lr_copy_slots: Optional[torch.Tensor] = None):
+        """Fused projection with one agent mask per row (row_masks: int64 tensor holding the uint64 bit masks);
+        lr_copy_slots: optional int32 [M], a second slot that also receives each row's LR rows (< 0: none)."""
         if row_masks.dtype != torch.int64:
             raise PreccError("row_masks must be int64 (bit patterns of uint64 masks)")
+        if lr_copy_slots is not None and lr_copy_slots.dtype != torch.int32:
+            raise PreccError("lr_copy_slots must be int32")
         cd = cache.desc()
         self._check(self.lib.precc_turn_project_rows(self.h, C.byref(desc), _ptr(H), H.shape[0], _ptr(WA_packed),
-                                                     _ptr(slot_mapping), _ptr(row_masks), C.byref(cd), _stream()),
+                                                     _ptr(slot_mapping), _ptr(row_masks), _ptr(lr_copy_slots),
+                                                     C.byref(cd), _stream()),
                     "precc_turn_project_rows")
 
     # ------------------------------------------------------------------ the four entry points

@@ -255,7 +255,8 @@ int32_t precc_rebase_project_rope(precc_ctx* ctx, const precc_layer_desc* desc, 
 
 static int32_t turn_entry(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
                           const int32_t* slot_mapping, int64_t start_slot, uint64_t agent_mask, const precc_rope* rope,
-                          const precc_cache* cache, void* stream, const uint64_t* row_masks = nullptr) {
+                          const precc_cache* cache, void* stream, const uint64_t* row_masks = nullptr,
+                          const int32_t* lr_copy_slots = nullptr) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (M < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "M < 0");
@@ -273,6 +274,7 @@ static int32_t turn_entry(precc_ctx* ctx, const precc_layer_desc* desc, const vo
   gp.lr_k = (__nv_bfloat16*)cache->lr_k; gp.lr_v = (__nv_bfloat16*)cache->lr_v;
   gp.n_agents = desc->n_agents; gp.rank_k = desc->rank_k; gp.rank_v = desc->rank_v; gp.agent_mask = agent_mask;
   gp.row_masks = reinterpret_cast<const unsigned long long*>(row_masks);
+  gp.lr_copy_slots = lr_copy_slots;
   gp.n_kv = desc->n_kv_heads; gp.hd = desc->head_dim;
   gp.M = M;
   rc = set_rope(ctx, desc, rope, &gp);
@@ -287,12 +289,12 @@ int32_t precc_turn_project(precc_ctx* ctx, const precc_layer_desc* desc, const v
 }
 
 int32_t precc_turn_project_rows(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,
-                                const int32_t* slot_mapping, const uint64_t* row_agent_masks, const precc_cache* cache,
-                                void* stream) {
+                                const int32_t* slot_mapping, const uint64_t* row_agent_masks, const int32_t* lr_copy_slots,
+                                const precc_cache* cache, void* stream) {
   if (!ctx) return PRECC_ERR_INVALID_ARG;
   if (!slot_mapping || !row_agent_masks) return fail(ctx, PRECC_ERR_INVALID_ARG, "slot_mapping / row_agent_masks is null");
   if (reinterpret_cast<uintptr_t>(row_agent_masks) & 7u) return fail(ctx, PRECC_ERR_MISALIGNED, "row_agent_masks not 8-byte aligned");
-  return turn_entry(ctx, desc, H, M, WA_packed, slot_mapping, 0, 0, nullptr, cache, stream, row_agent_masks);
+  return turn_entry(ctx, desc, H, M, WA_packed, slot_mapping, 0, 0, nullptr, cache, stream, row_agent_masks, lr_copy_slots);
 }
 
 int32_t precc_turn_project_rope(precc_ctx* ctx, const precc_layer_desc* desc, const void* H, int32_t M, const void* WA_packed,

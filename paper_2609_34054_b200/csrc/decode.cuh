@@ -84,7 +84,9 @@ struct DecodeCfg {
   static constexpr int BK_BYTES = BK_ROWS * HD * 2;
   // shared memory of a block with `warps` warps and `stages` ring slots per warp
   __host__ __device__ static constexpr int ring_bytes(int warps, int stages) { return warps * stages * STAGE_BYTES; }
-  __host__ __device__ static constexpr int merge_bytes(int warps) { return warps * (OW * 8 + 16) * 4; }
+  static constexpr int OWP = OW + 4;                  // padded head stride of a warp's record in the block merge (OW % 8 == 0)
+  static constexpr int WREC = 8 * OWP + 16;           // floats per warp record: m[8], l[8], O'[8 heads][OWP]
+  __host__ __device__ static constexpr int merge_bytes(int warps) { return warps * WREC * 4; }
   __host__ __device__ static constexpr int ticket_smem(int stages) {
     int a = ring_bytes(DEC_WARPS, stages), b = merge_bytes(DEC_WARPS);
     int c = (16 + 8 * OW + 16 * DEC_MAX_SPLITS + DEC_WARPS * 8 * OW) * 4 + RV * HD * 2;   // final merge without staging
@@ -171,41 +173,90 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   const __nv_bfloat16* lrk_a = RK > 0 ? p.lr_k + (size_t)agent * p.n_blocks * PAGE * RK : nullptr;
   const __nv_bfloat16* lrv_a = RV > 0 ? p.lr_v + (size_t)agent * p.n_blocks * PAGE * RV : nullptr;
 
+  // ---- page copies.  Everything that does not change from page to page is computed once: lane l moves the
+  //      16-byte chunks l + 32 j of each tile; the source of chunk j is (page base + 16 l) + 512 j, its swizzled
+  //      destination repeats with the period of (row & 7), so two (or four) offsets cover all j.  Per page that
+  //      leaves one 64-bit multiply-add per cache array and one cp.async per chunk.
+  constexpr int KV_PER_LANE = PAGE * CPR_KV / 32;        // 4 (head_dim 64) or 8 (128)
+  constexpr int KV_PERIOD = CPR_KV / 4;                  // 2 or 4: rows advance by 32 / CPR_KV per j, the swizzle by row & 7
+  uint32_t kv_dst[KV_PERIOD];
+#pragma unroll
+  for (int jj = 0; jj < KV_PERIOD; ++jj) {
+    const int c = lane + 32 * jj;
+    kv_dst[jj] = swz_off<CPR_KV>(c / CPR_KV, c % CPR_KV);
+  }
+  const int kv_row0 = lane / CPR_KV;                     // row of chunk j: kv_row0 + j * (32 / CPR_KV)
+  constexpr int LK_PER_LANE = RK > 0 ? (PAGE * CPR_LK + 31) / 32 : 0;   // 1, 1, 2, 4 for rank 8, 16, 32, 64
+  constexpr int LV_PER_LANE = RV > 0 ? (PAGE * CPR_LV + 31) / 32 : 0;
+  constexpr int LK_PERIOD = CPR_LK >= 8 ? 2 : 1, LV_PERIOD = CPR_LV >= 8 ? 2 : 1;
+  uint32_t lk_dst[LK_PERIOD], lv_dst[LV_PERIOD];
+#pragma unroll
+  for (int jj = 0; jj < LK_PERIOD; ++jj) { const int c = lane + 32 * jj; lk_dst[jj] = swz_off<CPR_LK>(c / CPR_LK, c % CPR_LK); }
+#pragma unroll
+  for (int jj = 0; jj < LV_PERIOD; ++jj) { const int c = lane + 32 * jj; lv_dst[jj] = swz_off<CPR_LV>(c / CPR_LV, c % CPR_LV); }
+  const bool lr_lane_k = RK > 0 && use_lr && lane < PAGE * CPR_LK;     // rank 8: 16 chunks, lanes 0..15 only
+  const bool lr_lane_v = RV > 0 && use_lr && lane < PAGE * CPR_LV;
+  const int lv_row0 = lane / CPR_LV;
+  const unsigned char* const k_lane = reinterpret_cast<const unsigned char*>(p.k_base) + (size_t)g * C::KV_BYTES + lane * 16;
+  const ptrdiff_t v_minus_k = reinterpret_cast<const unsigned char*>(p.v_base) - reinterpret_cast<const unsigned char*>(p.k_base);
+  const unsigned char* const lk_lane = reinterpret_cast<const unsigned char*>(lrk_a) + lane * 16;
+  const unsigned char* const lv_lane = reinterpret_cast<const unsigned char*>(lrv_a) + lane * 16;
+  const size_t kv_block_bytes = (size_t)p.n_kv * C::KV_BYTES;
+  int issue_slot = 0;                                   // ring slot of the next page to request: i % stages, kept incrementally
+
   auto issue_tile = [&](int i) {
     if (i < my_n) {
       if ((i & 31) == 0 && i > 0) { phys_cur = phys_nxt; phys_nxt = load_phys((i >> 5) + 1); }
       const int ph = __shfl_sync(0xffffffffu, phys_cur, i & 31);
       const int t = tile0 + warp + NW * i;
-      const int valid = min(PAGE, ctx - t * PAGE);
-      const uint32_t st = ring_u32 + (uint32_t)(i % p.stages) * C::STAGE_BYTES;
-      const unsigned char* ksrc = reinterpret_cast<const unsigned char*>(p.k_base + ((size_t)ph * p.n_kv + g) * PAGE * HD);
-      const unsigned char* vsrc = reinterpret_cast<const unsigned char*>(p.v_base + ((size_t)ph * p.n_kv + g) * PAGE * HD);
+      const int valid = ctx - t * PAGE;                 // >= PAGE for every page but the request's last one
+      const uint32_t st = ring_u32 + (uint32_t)issue_slot * C::STAGE_BYTES;
+      const unsigned char* ksrc = k_lane + (size_t)ph * kv_block_bytes;
+      const unsigned char* vsrc = ksrc + v_minus_k;
+      if (valid >= PAGE) {
 #pragma unroll
-      for (int c = lane; c < PAGE * CPR_KV; c += 32) {
-        const int row = c / CPR_KV, ch = c % CPR_KV;
-        const int off = swz_off<CPR_KV>(row, ch);
-        cp_async16(st + off, ksrc + c * 16, 16);
-        // value rows past the context are zero-filled: their weight is zero, but 0 * garbage
-        // (an unwritten slot may hold NaN) must not reach the accumulators
-        cp_async16(st + C::KV_BYTES + off, vsrc + c * 16, row < valid ? 16 : 0);
-      }
-      if (RK > 0 && use_lr) {
-        const unsigned char* src = reinterpret_cast<const unsigned char*>(lrk_a + (size_t)ph * PAGE * RK);
-#pragma unroll
-        for (int c = lane; c < PAGE * CPR_LK; c += 32) {
-          const int row = c / CPR_LK, ch = c % CPR_LK;
-          cp_async16(st + 2 * C::KV_BYTES + swz_off<CPR_LK>(row, ch), src + c * 16, 16);
+        for (int j = 0; j < KV_PER_LANE; ++j) {
+          const uint32_t dst = st + kv_dst[j % KV_PERIOD] + (j / KV_PERIOD) * (KV_PERIOD * 512);
+          cp_async16(dst, ksrc + j * 512, 16);
+          cp_async16(dst + C::KV_BYTES, vsrc + j * 512, 16);
         }
-      }
-      if (RV > 0 && use_lr) {
-        const unsigned char* src = reinterpret_cast<const unsigned char*>(lrv_a + (size_t)ph * PAGE * RV);
+        if (lr_lane_k) {
+          const unsigned char* src = lk_lane + (size_t)ph * C::LK_BYTES;
 #pragma unroll
-        for (int c = lane; c < PAGE * CPR_LV; c += 32) {
-          const int row = c / CPR_LV, ch = c % CPR_LV;
-          cp_async16(st + 2 * C::KV_BYTES + C::LK_BYTES + swz_off<CPR_LV>(row, ch), src + c * 16, row < valid ? 16 : 0);
+          for (int j = 0; j < LK_PER_LANE; ++j)
+            cp_async16(st + 2 * C::KV_BYTES + lk_dst[j % LK_PERIOD] + (j / LK_PERIOD) * (LK_PERIOD * 512), src + j * 512, 16);
+        }
+        if (lr_lane_v) {
+          const unsigned char* src = lv_lane + (size_t)ph * C::LV_BYTES;
+#pragma unroll
+          for (int j = 0; j < LV_PER_LANE; ++j)
+            cp_async16(st + 2 * C::KV_BYTES + C::LK_BYTES + lv_dst[j % LV_PERIOD] + (j / LV_PERIOD) * (LV_PERIOD * 512), src + j * 512, 16);
+        }
+      } else {
+        // the request's last, partial page: value rows past the context are zero-filled - their weight is zero,
+        // but 0 * garbage (an unwritten slot may hold NaN) must not reach the accumulators
+#pragma unroll
+        for (int j = 0; j < KV_PER_LANE; ++j) {
+          const uint32_t dst = st + kv_dst[j % KV_PERIOD] + (j / KV_PERIOD) * (KV_PERIOD * 512);
+          cp_async16(dst, ksrc + j * 512, 16);
+          cp_async16(dst + C::KV_BYTES, vsrc + j * 512, kv_row0 + j * (32 / CPR_KV) < valid ? 16 : 0);
+        }
+        if (lr_lane_k) {
+          const unsigned char* src = lk_lane + (size_t)ph * C::LK_BYTES;
+#pragma unroll
+          for (int j = 0; j < LK_PER_LANE; ++j)
+            cp_async16(st + 2 * C::KV_BYTES + lk_dst[j % LK_PERIOD] + (j / LK_PERIOD) * (LK_PERIOD * 512), src + j * 512, 16);
+        }
+        if (lr_lane_v) {
+          const unsigned char* src = lv_lane + (size_t)ph * C::LV_BYTES;
+#pragma unroll
+          for (int j = 0; j < LV_PER_LANE; ++j)
+            cp_async16(st + 2 * C::KV_BYTES + C::LK_BYTES + lv_dst[j % LV_PERIOD] + (j / LV_PERIOD) * (LV_PERIOD * 512), src + j * 512,
+                       lv_row0 + j * (32 / CPR_LV) < valid ? 16 : 0);
         }
       }
     }
+    if (++issue_slot == p.stages) issue_slot = 0;
     cp_async_commit();
   };
 
@@ -352,6 +403,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   load_cs(0);
 
   mark(3);
+  int use_slot = 0;                    // ring slot of page i: i % stages, kept incrementally
   for (int i = 0; i < my_n; ++i) {
     switch (p.stages) {                // ring depth 2 .. 8: all but the newest (depth - 1) groups have landed
       case 2: cp_async_wait<1>(); break;
@@ -364,7 +416,8 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     }
     __syncwarp();                      // page i is visible to all lanes
     if (i == 0) mark(4);
-    const uint32_t st = ring_u32 + (uint32_t)(i % p.stages) * C::STAGE_BYTES;
+    const uint32_t st = ring_u32 + (uint32_t)use_slot * C::STAGE_BYTES;
+    if (++use_slot == p.stages) use_slot = 0;
     const int t = tile0 + warp + NW * i;
     const int valid = ctx - t * PAGE;   // >= 1; tokens >= valid are masked
 
@@ -506,19 +559,23 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   }
   mark(5);
 
-  // ---- merge the warps of this block: smem [warp][ m[8] | l[8] | O'[OW][8] ]
+  // ---- merge the warps of this block: smem [warp][ m[8] | l[8] | O'[8 heads][OWP] ], OWP = OW + 4: a store
+  //      instruction touches heads cq = 0, 2, 4, 6 (2 OWP = 8 mod 32 banks apart) at rows r = 0..7, i.e. 32 different
+  //      banks, and the merging threads load consecutive columns: both free of bank conflicts
   __syncthreads();
   float* mg = reinterpret_cast<float*>(smem);
-  constexpr int WREC = OW * 8 + 16;
+  constexpr int OWP = C::OWP;
+  constexpr int WREC = C::WREC;
   {
     float* w = mg + warp * WREC;
     if (lane < 4) { w[2 * lane] = m0; w[2 * lane + 1] = m1; w[8 + 2 * lane] = l0; w[8 + 2 * lane + 1] = l1; }
     const int r = lane >> 2, cq = (lane & 3) * 2;
+    float* w0 = w + 16 + cq * OWP;         // query head cq, cq + 1
 #pragma unroll
     for (int mt = 0; mt < MT + MX; ++mt) {
       const int row = mt * 16 + r;
-      if (row < OW) { w[16 + row * 8 + cq] = o[mt][0]; w[16 + row * 8 + cq + 1] = o[mt][1]; }
-      if (row + 8 < OW) { w[16 + (row + 8) * 8 + cq] = o[mt][2]; w[16 + (row + 8) * 8 + cq + 1] = o[mt][3]; }
+      if (row < OW) { w0[row] = o[mt][0]; w0[OWP + row] = o[mt][1]; }
+      if (row + 8 < OW) { w0[row + 8] = o[mt][2]; w0[OWP + row + 8] = o[mt][3]; }
     }
   }
   __syncthreads();
@@ -535,7 +592,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     if (e < n_el + 8) {
       const bool is_ml = e >= n_el;
       const int h = is_ml ? e - n_el : e / OW;
-      const int src = is_ml ? 8 + h : 16 + (e % OW) * 8 + h;
+      const int src = is_ml ? 8 + h : 16 + h * OWP + (e % OW);
       float mw[NW], xw[NW];
 #pragma unroll
       for (int w = 0; w < NW; ++w) { mw[w] = mg[w * WREC + h]; xw[w] = mg[w * WREC + src]; }

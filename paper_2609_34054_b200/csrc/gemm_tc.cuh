@@ -25,10 +25,12 @@ namespace precc {
 // their place in the paged caches: column -> (projection, head, c) for base columns, (projection, agent,
 // r) for LR columns (skipped when the agent's bit in `mask` — the call's mask or the row's own — is clear).  Pieces never straddle a destination row
 // because head_dim and the ranks are multiples of 8.
+// `gm` is the row's index in the call (for the optional second LR destination of that row, see lr_copy_slots).
 __device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, int off, int gc, const float (&v8)[8],
-                                            unsigned long long mask) {
+                                            unsigned long long mask, int gm) {
   const int w = p.n_kv * p.hd;
   __nv_bfloat16* dst;
+  __nv_bfloat16* dst2 = nullptr;
   const bool to_base = p.mode == 1 || (p.mode == 2 && gc < 2 * w);
   if (!to_base) {
     const int n_k = p.n_agents * p.rank_k;
@@ -39,6 +41,11 @@ __device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, 
     const int agent = cc / rr, ri = cc % rr;
     if (!((mask >> agent) & 1ull)) return;
     dst = (is_v ? p.lr_v : p.lr_k) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
+    if (p.lr_copy_slots) {
+      const long long s2 = p.lr_copy_slots[gm];
+      if (s2 >= p.n_blocks * PAGE) atomicOr(p.status, StatusBits::BAD_INDEX);
+      else if (s2 >= 0) dst2 = (is_v ? p.lr_v : p.lr_k) + ((long long)agent * p.n_blocks * PAGE + s2) * rr + ri;
+    }
   } else {
     const bool is_v = gc >= w;
     const int cc = is_v ? gc - w : gc;
@@ -51,6 +58,7 @@ __device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, 
   v.z = pack_bf16(v8[4], v8[5]);
   v.w = pack_bf16(v8[6], v8[7]);
   *reinterpret_cast<uint4*>(dst) = v;
+  if (dst2) *reinterpret_cast<uint4*>(dst2) = v;
 }
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -208,7 +216,7 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
           float v8[8];
 #pragma unroll
           for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(r[8 * h + k]);
-          store_piece(p, blk, off, gc, v8, row_mask);
+          store_piece(p, blk, off, gc, v8, row_mask, gm);
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
@@ -270,7 +278,7 @@ __device__ __forceinline__ void splitk_reduce(const GemmParams& p, uint32_t smem
             atomicOr(p.status, StatusBits::BAD_INDEX);
           } else {
             const float v8[8] = {v.x, v.y, v.z, v.w, hi.x, hi.y, hi.z, hi.w};
-            store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8, p.row_masks ? p.row_masks[gm] : p.agent_mask);
+            store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8, p.row_masks ? p.row_masks[gm] : p.agent_mask, gm);
           }
         }
       }

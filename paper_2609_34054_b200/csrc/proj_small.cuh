@@ -183,11 +183,11 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         hi[2 * k] = h8[2 * k] * t4.x + v8[2 * k] * t4.y;
         hi[2 * k + 1] = h8[2 * k + 1] * t4.z + v8[2 * k + 1] * t4.w;
       }
-      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, lo, mask);
-      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc + p.hd / 2, hi, mask);
+      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, lo, mask, row);
+      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc + p.hd / 2, hi, mask, row);
       continue;
     }
-    store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8, mask);
+    store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8, mask, row);
   }
   // nobody leaves while a peer may still read its partial tile
   asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");

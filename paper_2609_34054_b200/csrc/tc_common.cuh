@@ -22,6 +22,7 @@ struct GemmParams {
   int n_agents, rank_k, rank_v;
   unsigned long long agent_mask;
   const unsigned long long* row_masks;   // optional [M]: per-row agent masks (double batching), overrides agent_mask
+  const int32_t* lr_copy_slots;          // optional [M]: a second slot that also receives the row's LR rows (< 0: none)
   int n_kv, hd;
   // rotary keys (modes 1, 2; null = none): the key columns of a row are rotated by the row's position
   // before they are stored (rotate-half pairing (c, c + hd/2)); needs BN % hd == 0

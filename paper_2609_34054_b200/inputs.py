@@ -195,3 +195,11 @@ def block_tables(ctx_len: torch.Tensor, n_phys_blocks: int, seed: int) -> torch.
         table[b, :n] = perm[at:at + n]
         at += n
     return table
+
+
+def rope_table(max_pos: int, hd: int, theta: float = 10000.0, device="cuda") -> torch.Tensor:
+    """The position table that callers of the rotary-key entry points pass in: fp32 [max_pos][hd/2][2] =
+    (cos, sin) of t * theta^(-2c/hd), angles evaluated in fp64 and rounded once."""
+    inv = torch.pow(torch.tensor(theta, dtype=torch.float64), -torch.arange(hd // 2, dtype=torch.float64) * 2.0 / hd)
+    ang = torch.arange(max_pos, dtype=torch.float64)[:, None] * inv[None, :]
+    return torch.stack([torch.cos(ang), torch.sin(ang)], dim=-1).to(torch.float32).contiguous().to(device)

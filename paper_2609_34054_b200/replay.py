@@ -15,8 +15,9 @@ states and queries), so its times are the KV-path share of a turn, not model lat
   nonshared   every agent keeps a private full-width cache and first processes all tokens it has not
               seen (everything the other agents appended since its last turn).
   rebase_db   ReBaseShared with double batching: every step of the turn carries two sequences over the same
-              tokens, the adapted one (agent j: its LR rows, and adapted base rows in private blocks that
-              its block table splices in after the shared context) and the adapter-free one (neutral base
+              tokens, the adapted one (agent j: adapted base rows and its LR rows in private blocks that its
+              block table splices in after the shared context; the LR rows are also written at the tokens' shared
+              slots, where they stay) and the adapter-free one (neutral base
               rows into the shared cache, the other agents' LR rows).  Prefill runs both; every decode step
               is ONE two-row projection (per-row agent masks) and ONE attention launch of two requests (agent j and the
               adapter-free view, each with its own block table).  Nothing is left to do after the turn.
@@ -73,8 +74,11 @@ def trace_tokens(turns: Sequence[Turn]) -> int:
 
 class Stack:
     """Per-layer device state: caches, packed weights, B factors (distinct per layer unless
-    ``shared_weights``, so that a layer's weights are not found in L2 by the next one).  Hidden states and
-    queries are random buffers shared by all layers (their values do not affect the work done)."""
+    ``shared_weights``, so that a layer's weights are not found in L2 by the next one).  Hidden states are
+    random and indexed by trajectory position: ``H_adpt[t]`` is what the layer sees for token t under the
+    current agent's adapter, ``H_neut[t]`` what it sees in the adapter-free pass; they and the queries are
+    shared by all layers (their values do not affect the work done, but they make the final cache contents
+    and outputs a function of the trace that a test can recompute)."""
 
     def __init__(self, px: Precc, geo: I.Geometry, n_layers: int, max_tokens: int, max_rows: int, seed: int = 0,
                  shared_weights: bool = False, private_tokens: int = 0):
@@ -94,7 +98,11 @@ class Stack:
             self.W.append(px.pack_base_weights(geo, w["W_k"], w["W_v"]))
             self.B_k.append(w["B_k"] if geo.rank_k else None)
             self.B_v.append(w["B_v"] if geo.rank_v else None)
-        self.H = I.normal_bf16((max_rows, geo.d_model), 1.0, seed, "replay.H").cuda()
+        rows = n_blocks * I.PAGE
+        self.H_adpt = I.normal_bf16((rows, geo.d_model), 1.0, seed, "replay.H_adpt").cuda()
+        self.H_neut = I.normal_bf16((rows, geo.d_model), 1.0, seed, "replay.H_neut").cuda()
+        self.H2 = torch.empty((max(max_rows, 2), geo.d_model), dtype=torch.bfloat16, device="cuda")   # two sequences in one batch
+        self.stage = torch.empty((2, geo.d_model), dtype=torch.bfloat16, device="cuda")              # rows of one decode step
         self.q = I.queries(max_rows, geo, seed, "replay.q").cuda()
         self.out = torch.empty_like(self.q)
         self.ws = px.decode_workspace(self.desc, 2, max_tokens)      # up to two requests per launch (double batching)
@@ -104,40 +112,46 @@ class Stack:
         return l if len(self.WA) > 1 else 0
 
 
-def _project(st: Stack, l: int, n: int, start: int, mask: Optional[int], slot_map=None):
-    """mask None: base rows only; else base rows + LR rows of the agents in `mask`."""
+def _project(st: Stack, l: int, H: torch.Tensor, start: int, mask: Optional[int], slot_map=None):
+    """Rows H -> slots start.. (or slot_map).  mask None: base rows only; else base rows + LR rows of the agents in `mask`."""
     px, k = st.px, st.w(l)
     if mask is None or (st.geo.rank_k == 0 and st.geo.rank_v == 0):
-        px.rebase_project(st.desc, st.H[:n], st.W[k], st.caches[l], start, slot_map)
+        px.rebase_project(st.desc, H, st.W[k], st.caches[l], start, slot_map)
     else:
-        px.turn_project(st.desc, st.H[:n], st.WA[k], st.caches[l], start, slot_map, mask)
+        px.turn_project(st.desc, H, st.WA[k], st.caches[l], start, slot_map, mask)
 
 
-def _prefill_phase(st: Stack, n: int, T: int, agent: int, mask: Optional[int]):
+def _prefill_phase(st: Stack, H: torch.Tensor, T: int, agent: int, mask: Optional[int]):
+    """The n = len(H) tokens at positions T.. : projection into the caches, then attention of `agent` over them."""
+    n = H.shape[0]
     for l in range(st.n_layers):
-        _project(st, l, n, T, mask)
+        _project(st, l, H, T, mask)
         k = st.w(l)
         st.px.lr_attend_prefill(st.desc, st.q[:n], agent, T, st.B_k[k], st.B_v[k], st.caches[l], st.out[:n])
 
 
 class _DecodeGraph:
-    """One decode step over all layers with device-side position; replayed once per generated token."""
+    """One decode step over all layers with device-side position; replayed once per generated token.  The
+    hidden state of the token at position t is H_src[t], fetched into a staging row by a gather inside the graph."""
 
-    def __init__(self, st: Stack, agent: int, mask: Optional[int], ctx0: int, max_ctx: int):
+    def __init__(self, st: Stack, H_src: torch.Tensor, agent: int, mask: Optional[int], ctx0: int, max_ctx: int):
         dev = st.q.device
         self.ctx = torch.tensor([ctx0], dtype=torch.int32, device=dev)        # tokens attended (incl. the new one)
         self.slot = torch.tensor([ctx0 - 1], dtype=torch.int32, device=dev)   # where the new token's rows go
+        self.pos = torch.tensor([ctx0 - 1], dtype=torch.int64, device=dev)    # its trajectory position (gather index)
         self.agent = torch.tensor([agent], dtype=torch.int32, device=dev)
         self.first = torch.zeros(1, dtype=torch.int32, device=dev)
 
         def step():
+            torch.index_select(H_src, 0, self.pos, out=st.stage[:1])
             for l in range(st.n_layers):
-                _project(st, l, 1, 0, mask, self.slot)
+                _project(st, l, st.stage[:1], 0, mask, self.slot)
                 k = st.w(l)
                 st.px.lr_attend_decode(st.desc, st.q[:1], self.agent, self.ctx, max_ctx, st.B_k[k], st.B_v[k], st.caches[l],
                                        st.out[:1], st.ws, None, self.first)
             self.ctx.add_(1)
             self.slot.add_(1)
+            self.pos.add_(1)
 
         step()                                       # warm-up outside capture (also the first real step)
         torch.cuda.synchronize()
@@ -185,12 +199,26 @@ def _replay_db(st: Stack, turns: Sequence[Turn]) -> Dict[str, float]:
 
         slots_2n = torch.cat([slots_a, (P + torch.arange(n, dtype=torch.int32)).to(dev)])
         masks_2n = torch.tensor([1 << j] * n + [others] * n, dtype=torch.int64, device=dev)
+        # agent j's own LR rows also go to the tokens' shared slots: they outlive the private blocks
+        copy_2n = torch.cat([P + torch.arange(n, dtype=torch.int32), torch.full((n,), -1, dtype=torch.int32)]).to(dev)
+
+        st.H2[:n].copy_(st.H_adpt[P:P + n])                           # the two sequences of the turn, one batch
+        st.H2[n:2 * n].copy_(st.H_neut[P:P + n])
 
         def prefill_both():
             for l in range(st.n_layers):
                 k = st.w(l)
+                if P % I.PAGE:
+                    # the page that holds position P is private to the adapted sequence: it starts as a copy of the
+                    # shared page, so that the context rows in front of P are there too
+                    c, src, dst = st.caches[l], P // I.PAGE, st.shared_blocks
+                    c.k_base[dst].copy_(c.k_base[src]); c.v_base[dst].copy_(c.v_base[src])
+                    if c.lr_k is not None:
+                        c.lr_k[:, dst].copy_(c.lr_k[:, src])
+                    if c.lr_v is not None:
+                        c.lr_v[:, dst].copy_(c.lr_v[:, src])
                 # adapted rows and adapter-free rows of the turn in ONE projection (per-row agent masks)
-                px.turn_project_rows(st.desc, st.H[:2 * n], st.WA[k], st.caches[l], slots_2n, masks_2n)
+                px.turn_project_rows(st.desc, st.H2[:2 * n], st.WA[k], st.caches[l], slots_2n, masks_2n, copy_2n)
                 px.lr_attend_prefill(st.desc, st.q[:n], j, P, st.B_k[k], st.B_v[k], st.caches[l], st.out[:n], table_a)
                 px.lr_attend_prefill(st.desc, st.q[:n], -1, P, st.B_k[k], st.B_v[k], st.caches[l], st.out[:n])
 
@@ -206,14 +234,18 @@ def _replay_db(st: Stack, turns: Sequence[Turn]) -> Dict[str, float]:
             agent2 = torch.tensor([j, -1], dtype=torch.int32, device=dev)
             slot2 = torch.tensor([priv0 + n, P + n], dtype=torch.int32, device=dev)
             mask2 = torch.tensor([1 << j, others], dtype=torch.int64, device=dev)
+            pos = torch.tensor([P + n], dtype=torch.int64, device=dev)
+            copy2 = torch.tensor([P + n, -1], dtype=torch.int32, device=dev)
 
             def step():
+                torch.index_select(st.H_adpt, 0, pos, out=st.stage[:1])
+                torch.index_select(st.H_neut, 0, pos, out=st.stage[1:2])
                 for l in range(st.n_layers):
                     k = st.w(l)
-                    px.turn_project_rows(st.desc, st.H[:2], st.WA[k], st.caches[l], slot2, mask2)
+                    px.turn_project_rows(st.desc, st.stage, st.WA[k], st.caches[l], slot2, mask2, copy2)
                     px.lr_attend_decode(st.desc, st.q[:2], agent2, ctx, max_ctx, st.B_k[k], st.B_v[k], st.caches[l], st.out[:2],
                                         st.ws, table2)
-                ctx.add_(1); slot2.add_(1)
+                ctx.add_(1); slot2.add_(1); pos.add_(1); copy2[:1].add_(1)
 
             step()
             torch.cuda.synchronize()
@@ -252,14 +284,14 @@ def replay(st: Stack, turns: Sequence[Turn], policy: str) -> Dict[str, float]:
         else:
             start, n_pref, agent, mask = P, t.n_in, j, 1 << j
         prefilled += n_pref
-        ttft += _timed(lambda: _prefill_phase(st, n_pref, start, agent, mask))
+        ttft += _timed(lambda: _prefill_phase(st, st.H_adpt[start:start + n_pref], start, agent, mask))
         ctx0 = P + t.n_in + 1
         if t.n_out > 0:
-            g = _DecodeGraph(st, agent, mask, ctx0, P + t.n_in + t.n_out)     # runs the first decode step itself
+            g = _DecodeGraph(st, st.H_adpt, agent, mask, ctx0, P + t.n_in + t.n_out)     # runs the first decode step itself
             decode_ms += _timed(lambda: g.run(t.n_out - 1)) * t.n_out / max(1, t.n_out - 1)
         if policy == "rebase_lp":
             n_c = t.n_in + t.n_out
-            rebase_ms += _timed(lambda: _prefill_phase(st, n_c, P, -1, all_mask & ~(1 << j)))
+            rebase_ms += _timed(lambda: _prefill_phase(st, st.H_neut[P:P + n_c], P, -1, all_mask & ~(1 << j)))
         P += t.n_in + t.n_out
         seen[j] = P
     total = ttft + decode_ms + rebase_ms

@@ -136,7 +136,7 @@ def test_random_shapes(px, i):
 # Projections and the rotary path, through the library's own calls (hidden states -> caches -> attention)
 
 from harness import Layer, base_rows, lr_rows                     # noqa: E402
-from paper_2609_34054_b200.binding import rope_table              # noqa: E402
+from paper_2609_34054_b200.inputs import rope_table               # noqa: E402
 
 N_PROJ = max(12, N_CASES // 3)
 

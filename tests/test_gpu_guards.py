@@ -5,7 +5,8 @@ import pytest
 import torch
 
 from paper_2609_34054_b200 import inputs as I
-from paper_2609_34054_b200.binding import Cache, Precc, layer_desc, rope_table
+from paper_2609_34054_b200.binding import Cache, Precc, layer_desc
+from paper_2609_34054_b200.inputs import rope_table
 
 pytestmark = pytest.mark.gpu
 

@@ -403,6 +403,77 @@ def test_device_side_bad_indices_are_flagged_not_fatal(px):
     assert px.poll_status() == 0
 
 
+@pytest.mark.parametrize("B,T", [(2, 4096), (40, 1200)])     # the cluster kernel and the ticket kernel
+def test_context_longer_than_the_host_bound_is_flagged_and_the_workspace_stays_usable(px, B, T):
+    """ctx_len is device data; the host's max_ctx sized the grid, the split and the block table.  A request whose
+    ctx_len exceeds it is rejected on the device like a bad agent id: zeros, BAD_INDEX, and the workspace is left
+    ready, so the next call on it is correct."""
+    geo = I.Geometry(256, 8, 2, 64, 2, 16, 16, alpha=32.0)
+    nb = (T + 15) // 16
+    c = I.direct_caches(nb, geo, 61, "over")
+    from paper_2609_34054_b200.binding import Cache, layer_desc
+    cache = Cache.from_tensors(geo, c["k_base"].cuda(), c["v_base"].cuda(), c["lr_k"].cuda(), c["lr_v"].cuda())
+    w = I.layer_weights(geo, 61, "over")
+    desc = layer_desc(geo)
+    q = I.queries(B, geo, 61, "over.q").cuda()
+    aid = torch.tensor([i % 2 for i in range(B)], dtype=torch.int32).cuda()
+    good = torch.full((B,), T - 3, dtype=torch.int32)
+    bad = good.clone()
+    bad[1] = 8 * T                                        # far beyond max_ctx (and beyond the cache)
+    ws = px.decode_workspace(desc, B, T)
+    Bk, Bv = w["B_k"].cuda(), w["B_v"].cuda()
+    ref = torch.full_like(q, float("nan"))
+    px.lr_attend_decode(desc, q, aid, good.cuda(), T, Bk, Bv, cache, ref, ws)
+    assert px.poll_status() == 0
+    out = torch.full_like(q, float("nan"))
+    px.lr_attend_decode(desc, q, aid, bad.cuda(), T, Bk, Bv, cache, out, ws)
+    assert px.poll_status() & 1
+    assert (out[1] == 0).all()
+    keep = [i for i in range(B) if i != 1]
+    assert torch.equal(out[keep], ref[keep])
+    again = torch.full_like(q, float("nan"))
+    px.lr_attend_decode(desc, q, aid, good.cuda(), T, Bk, Bv, cache, again, ws)      # same workspace, no re-init
+    assert px.poll_status() == 0
+    assert torch.equal(again, ref)
+
+
+@pytest.mark.parametrize("M", [1, 7, 40])
+def test_decode_launched_right_behind_the_append_of_its_newest_tokens(px, M):
+    """Decode starts fetching a request's older pages while the kernel before it on the stream - here the few-row
+    projection that appends the M newest tokens (Section 3.1: in-turn append) - may still be running.  The result
+    must be bit-equal to running the two one after the other, for every one of many back-to-back repetitions with
+    changing rows (a race on the appended rows, on q or on the output would show as a stale value)."""
+    geo = I.Geometry(512, 32, 8, 64, 4, 16, 16, alpha=32.0)
+    T = 4096 + 21
+    L = Layer(px, geo, seed=77, n_blocks=(T + 15) // 16)
+    dev = {k: v.cuda() for k, v in L.w.items()}
+    WA = px.pack_turn_weights(geo, dev["W_k"], dev["W_v"], dev["A_k"], dev["A_v"])
+    L.append(I.hidden_states(T, geo, 77, "pdl.H"))
+    ws = px.decode_workspace(L.desc, 1, T)
+    aid = torch.tensor([2], dtype=torch.int32).cuda()
+    cl = torch.tensor([T], dtype=torch.int32).cuda()
+    trials = 12
+    Hn = [I.hidden_states(M, geo, 100 + i, "pdl.new").cuda() for i in range(trials)]
+    qs = [I.queries(1, geo, 100 + i, "pdl.q", gain=3.0).cuda() for i in range(trials)]
+    ref = []
+    for i in range(trials):                                   # serialised order
+        px.turn_project(L.desc, Hn[i], WA, L.cache, T - M)
+        torch.cuda.synchronize()
+        o = torch.full_like(qs[i], float("nan"))
+        px.lr_attend_decode(L.desc, qs[i], aid, cl, T, L.B_k, L.B_v, L.cache, o, ws)
+        torch.cuda.synchronize()
+        ref.append(o)
+    assert not torch.equal(ref[0], ref[1])
+    got = [torch.full_like(qs[i], float("nan")) for i in range(trials)]
+    for i in range(trials):                                   # back to back, nothing in between
+        px.turn_project(L.desc, Hn[i], WA, L.cache, T - M)
+        px.lr_attend_decode(L.desc, qs[i], aid, cl, T, L.B_k, L.B_v, L.cache, got[i], ws)
+    torch.cuda.synchronize()
+    for i in range(trials):
+        assert torch.equal(got[i], ref[i]), f"repetition {i}"
+    assert px.poll_status() == 0
+
+
 @pytest.mark.parametrize("B,hd,n_kv", [(3, 64, 8), (5, 64, 8), (6, 128, 8), (9, 128, 4), (2, 128, 5)])
 def test_decode_cluster_sizes_that_do_not_divide_the_head_dimension(px, B, hd, n_kv):
     """Few requests, long contexts: the splits of a (request, kv head) form a cluster of as many blocks as fit

@@ -7,7 +7,8 @@ import torch
 
 from oracle import lrkv_oracle as O
 from paper_2609_34054_b200 import inputs as I
-from paper_2609_34054_b200.binding import PreccError, rope_table
+from paper_2609_34054_b200.binding import PreccError
+from paper_2609_34054_b200.inputs import rope_table
 
 from harness import Layer, assert_close, base_rows, f64
 
@@ -69,14 +70,27 @@ def test_projection_rotates_keys_only(px, hd, n_kv, M):
     px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0, start_pos=7)
     px.lr_precompute(L.desc, H.cuda(), L.A_packed, L.cache, 0)
     torch.cuda.synchronize()
-    k2, lk2 = L.cache.k_base.clone(), L.cache.lr_k.clone()
+    k2, lk2, v2, lv2 = L.cache.k_base.clone(), L.cache.lr_k.clone(), L.cache.v_base.clone(), L.cache.lr_v.clone()
     ref2 = O.rope_rotate(O.base_cache(f64(H), L.w_np["W_k"]), np.arange(M) + 7, n_kv, cos, sin)
     assert (np.abs(base_rows(k2)[:M] - ref2) <= 2.0 ** -8 * np.abs(ref2) + 2e-3).all()
     WA = px.pack_turn_weights(geo, L.w["W_k"].cuda(), L.w["W_v"].cuda(), L.w["A_k"].cuda(), L.w["A_v"].cuda())
-    L.cache.k_base.zero_(); L.cache.lr_k.zero_()
+    # the fused rotary projection (precc_turn_project_rope): every cache it writes equals the two-call form bit for
+    # bit - rotated base K rows (checked against the oracle above), plain V rows, un-rotated LR rows of both sides
+    for c in (L.cache.k_base, L.cache.v_base, L.cache.lr_k, L.cache.lr_v):
+        c.zero_()
     px.turn_project_rope(L.desc, H.cuda(), WA, L.cache, table, 0, start_pos=7)
     torch.cuda.synchronize()
     assert torch.equal(L.cache.k_base, k2) and torch.equal(L.cache.lr_k, lk2)
+    assert torch.equal(L.cache.v_base, v2) and torch.equal(L.cache.lr_v, lv2)
+    assert_close(f64(L.cache.lr_k[1].reshape(-1, 16))[:M], O.lr_cache(f64(H), L.w_np["A_k"][1]), "LR-K rows stay un-rotated",
+                 atol=2e-2, rtol=1e-2, norm_tol=1e-2)
+    # with an agent mask only the selected agents' LR rows are written; the rotated base rows always are
+    for c in (L.cache.k_base, L.cache.v_base, L.cache.lr_k, L.cache.lr_v):
+        c.zero_()
+    px.turn_project_rope(L.desc, H.cuda(), WA, L.cache, table, 0, None, 0b10, start_pos=7)
+    torch.cuda.synchronize()
+    assert torch.equal(L.cache.k_base, k2) and torch.equal(L.cache.lr_k[1], lk2[1]) and torch.equal(L.cache.lr_v[1], lv2[1])
+    assert (L.cache.lr_k[0] == 0).all() and (L.cache.lr_v[0] == 0).all()
 
 
 SHAPES = [
