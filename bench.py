@@ -4,8 +4,8 @@
 Workload (one "step" = one pass of the hot path over one synthetic trajectory, single stream):
 a Llama-3.2-1B-shaped stack (16 layers, d_model 2048, 32 q / 8 kv heads, head_dim 64), 4 agents,
 LoRA rank 16 on K and V (scale alpha/r = 2), shared trajectory of 8192 tokens:
-  phase A  per layer: base K/V projection of the 8192 hidden states into the shared cache
-           (precc_rebase_project) and the LR precompute for all 4 agents (precc_lr_precompute);
+  phase A  per layer: one fused projection of the 8192 hidden states (precc_turn_project): base K/V rows
+           into the shared cache and the LR rows of all 4 agents, the hidden states read once;
   phase B  per agent, 128 decode steps, each one LR-reconstructed decode attention per layer
            (precc_lr_attend_decode, batch 1, context 8192): 4 x 128 x 16 = 8192 launches,
            replayed from one CUDA graph.
@@ -15,6 +15,12 @@ divided by the WHOLE step time (phase A included).  Inputs are resident in HBM f
 repeats the step with the hidden states and queries copied from pinned host memory and the outputs
 copied back inside the timed region.
 
+Beside the timed step the line carries, at one GPU, the other rows of the metric with their own roofline
+records (`rooflines`): serving-shaped decode (64 requests, 2.4 GB of cache per launch), the new-turn prefill
+and the LR precompute of a Llama-3-8B-shaped layer, each with the oracle timed on a stated sample.
+
+`--gpus N` (N > 1) without a launcher starts N ranks itself (torch.distributed.run on 127.0.0.1): independent
+replicas, one per GPU; the only collective is the max-reduction of the step time.
 `--impl reference` times the CPU oracle (oracle/lrkv_oracle.py, numpy float64) on a bounded sample
 of the same workload.
 """
@@ -23,6 +29,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -35,9 +42,18 @@ METRIC = "lr_kv_decode_attention_GBps"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per decode launch of this workload, from the ncu
-# capture summarised under profiles/ (None until a capture exists)
-NCU_DECODE_TRAFFIC_BYTES = 17378560   # profiles/decode_cluster_c2_layer.md
+# DRAM bytes per launch of the profiled kernels (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture each), kept as data beside the profile summaries
+NCU_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
+
+
+def ncu_traffic(key: str):
+    """The recorded capture `key`: {"dram_bytes": per launch, "algorithmic_bytes": of the captured case, ...} or None."""
+    try:
+        with open(NCU_TRAFFIC_FILE) as f:
+            return json.load(f).get(key)
+    except Exception:
+        return None
 
 
 def decode_bytes_per_launch(geo, ctx: int, batch: int = 1, distinct_agents: int = 1) -> int:
@@ -204,7 +220,7 @@ def _event_us(torch, fn, iters, warm=3):
     return e0.elapsed_time(e1) / iters * 1e3
 
 
-def extra_serving_decode(px, batch: int, ctx_min: int, ctx_max: int, seed: int = 0):
+def extra_serving_decode(px, batch: int, ctx_min: int, ctx_max: int, seed: int = 0, cpu_seconds: float = 0.0):
     """C4-shaped decode: `batch` requests, agents uniform over 8, contexts uniform in [ctx_min, ctx_max],
     paged-16 caches with every logical block on its own physical block (a seeded CPU pool of 4096 blocks
     tiled over the physical pool: values repeat, addresses do not, so every launch streams from HBM)."""
@@ -232,13 +248,54 @@ def extra_serving_decode(px, batch: int, ctx_min: int, ctx_max: int, seed: int =
     byt = int(ctx_len.sum()) * per_tok + batch * 2 * geo.n_q * geo.hd * 2 + sum(need) * 4 + geo.n_agents * (geo.rank_k + geo.rank_v) * geo.kv_width * 2
     peak, kind = measured_peak()
     gbs = byt / us / 1e3
-    return {"workload": f"C4 serving decode: B={batch}, ctx~U[{ctx_min},{ctx_max}], 28q/4kv hd=128, N=8 r=16, paged-16",
-            "kernel": "lr_attend_decode_kernel<128,16,16> (ticket)", "us_per_launch": us, "algorithmic_bytes": byt,
-            "GBps": gbs, "frac_of_peak": gbs / peak, "peak_kind": kind, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
-            "l2_policy": f"{byt / 1e6:.0f} MB of distinct cache per launch >> 126 MB L2"}
+    # DRAM traffic of a full launch: the ncu capture is a 16-request reduction of this workload (same kernel, same
+    # page layout; traffic is proportional to the tokens streamed), scaled by the algorithmic bytes
+    cap = ncu_traffic("decode_ticket_c4_reduced")
+    traffic = int(cap["dram_bytes"] * byt / cap["algorithmic_bytes"]) if cap else None
+    res = {"workload": f"C4 serving decode: B={batch}, ctx~U[{ctx_min},{ctx_max}], 28q/4kv hd=128, N=8 r=16, paged-16",
+           "kernel": "lr_attend_decode_kernel<128,16,16> (ticket)", "us_per_launch": us, "algorithmic_bytes": byt,
+           "GBps": gbs, "frac_of_peak": gbs / peak, "peak_kind": kind, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+           "l2_policy": f"{byt / 1e6:.0f} MB of distinct cache per launch >> 126 MB L2",
+           "roofline": {"bound": "hbm", "kernel": "lr_attend_decode_kernel<128,16,16> (ticket)", "achieved": gbs, "peak": peak,
+                        "peak_kind": kind, "unit": "GB/s", "frac": gbs / peak, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+                        "traffic": traffic, "traffic_note": "ncu capture of a 16-request reduction, scaled by algorithmic bytes",
+                        "algorithmic_bytes_per_launch": byt, "avg_launch_us": us}}
+    if cpu_seconds > 0:
+        res["cpu_baseline"] = _oracle_serving_sample(geo, q, agent_id, ctx_len, table, cache, w, per_tok, cpu_seconds, out)
+    return res
 
 
-def extra_turn(px, T: int, S: int, seed: int = 0):
+def _oracle_serving_sample(geo, q, agent_id, ctx_len, table, cache, w, per_tok, budget_s, gpu_out):
+    """The oracle (attention from cache contents, float64) on whole requests of the batch until `budget_s` seconds
+    of CPU time are spent; also checks those requests' GPU outputs against it."""
+    import numpy as np
+    import torch
+    from oracle import lrkv_oracle as O
+    G = geo.group
+    f64 = lambda t: t.detach().float().cpu().numpy().astype(np.float64)
+    spent, done_bytes, n_req, worst = 0.0, 0, 0, 0.0
+    got = f64(gpu_out)
+    for b in range(q.shape[0]):
+        t, a = int(ctx_len[b]), int(agent_id[b])
+        blocks = table[b, :(t + 15) // 16].long()
+        kb = f64(cache.k_base[blocks].permute(0, 2, 1, 3).reshape(-1, geo.kv_width))[:t]
+        vb = f64(cache.v_base[blocks].permute(0, 2, 1, 3).reshape(-1, geo.kv_width))[:t]
+        lk = f64(cache.lr_k[a][blocks].reshape(-1, geo.rank_k))[:t]
+        lv = f64(cache.lr_v[a][blocks].reshape(-1, geo.rank_v))[:t]
+        t0 = time.perf_counter()
+        ref = O.attend_from_caches(f64(q[b]), kb, vb, lk, lv, f64(w["B_k"][a]), f64(w["B_v"][a]), geo.scale_k, geo.scale_v, geo.n_kv)
+        spent += time.perf_counter() - t0
+        worst = max(worst, float(np.abs(got[b] - ref).max()))
+        done_bytes += t * per_tok + 2 * geo.n_q * geo.hd * 2
+        n_req += 1
+        if spent >= budget_s:
+            break
+    return {"value": done_bytes / spent / 1e9, "unit": "GB/s", "cores": cpu_threads(), "kind": "oracle",
+            "sample": f"{n_req} whole requests of the batch (all kv heads; attention from cache contents in float64), {spent:.1f} s",
+            "gpu_max_abs_err_on_sample": worst}
+
+
+def extra_turn(px, T: int, S: int, seed: int = 0, cpu_seconds: float = 0.0):
     """C3-shaped turn of one layer: LR precompute over the context (throughput), then the turn itself
     (base append + LR precompute of the S new tokens + prefill attention) and the ReBase re-projection."""
     import torch
@@ -309,16 +366,75 @@ def extra_turn(px, T: int, S: int, seed: int = 0):
     us_sturn = _event_us(torch, short_turn, 10)
     short = {"S": S2, "projection_us": us_sproj, "prefill_attention_us": us_sattn, "turn_us_per_layer": us_sturn,
              "turn_ttft_ms_32_layers": us_sturn * C3_LAYERS_FOR_TTFT / 1e3}
-    return {"workload": f"C3 turn, one layer: d=4096 32q/8kv hd=128, N=4 r=32, T={T}, S={S}",
-            "short_turn": short,
-            "lr_precompute_context": {"us": us_pre, "tflops": fl_pre / us_pre / 1e6, "n_out": n_lr,
-                                      "GBps": 2.0 * (T * geo.d_model + T * n_lr) / us_pre / 1e3},
-            "base_projection_context": {"us": us_base, "tflops": 2.0 * T * geo.d_model * 2 * geo.kv_width / us_base / 1e6},
-            "fused_projection_context": {"us": us_cfused, "tflops": 2.0 * T * geo.d_model * (2 * geo.kv_width + n_lr) / us_cfused / 1e6},
-            "turn_projection_us": us_tproj,
-            "turn_us_per_layer": us_turn, "turn_ttft_ms_32_layers": us_turn * C3_LAYERS_FOR_TTFT / 1e3,
-            "prefill_attention": {"us": us_attn, "tflops": fl_attn / us_attn / 1e6},
-            "rebase_us_per_layer": us_reb, "peaks": measured_tensor_peaks()}
+    pk = measured_tensor_peaks()
+    hbm, hbm_kind = measured_peak()
+    tf_attn = fl_attn / us_attn / 1e6
+    tf_pre = fl_pre / us_pre / 1e6
+    pre_bytes = 2.0 * (T * geo.d_model + geo.d_model * n_lr + T * n_lr)
+    attainable = min(pk["bf16_tflops_burst"], fl_pre / pre_bytes * hbm / 1e3)      # min(tensor, intensity x HBM), TFLOP/s
+    cap_pf, cap_pre = ncu_traffic("prefill_tc_c3_layer"), ncu_traffic("proj_gemm_c3_context")
+    res = {"workload": f"C3 turn, one layer: d=4096 32q/8kv hd=128, N=4 r=32, T={T}, S={S}",
+           "short_turn": short,
+           "lr_precompute_context": {"us": us_pre, "tflops": tf_pre, "n_out": n_lr, "GBps": pre_bytes / us_pre / 1e3,
+                                     "attainable_tflops": attainable, "frac_of_attainable": tf_pre / attainable},
+           "base_projection_context": {"us": us_base, "tflops": 2.0 * T * geo.d_model * 2 * geo.kv_width / us_base / 1e6},
+           "fused_projection_context": {"us": us_cfused, "tflops": 2.0 * T * geo.d_model * (2 * geo.kv_width + n_lr) / us_cfused / 1e6},
+           "turn_projection_us": us_tproj,
+           "turn_us_per_layer": us_turn, "turn_ttft_ms_32_layers": us_turn * C3_LAYERS_FOR_TTFT / 1e3,
+           "prefill_attention": {"us": us_attn, "tflops": tf_attn},
+           "rebase_us_per_layer": us_reb, "peaks": pk,
+           "roofline_prefill": {"bound": "tensor", "kernel": "lr_attend_prefill_tc_kernel<128,32,32>", "achieved": tf_attn,
+                                "peak": pk["bf16_tflops_burst"], "peak_kind": pk["peak_kind"] + " (burst)", "unit": "TFLOP/s",
+                                "frac": tf_attn / pk["bf16_tflops_burst"], "frac_of_sustained": tf_attn / pk["bf16_tflops_sustained"],
+                                "traffic": cap_pf["dram_bytes"] if cap_pf else None, "algorithmic_flops_per_launch": fl_attn,
+                                "avg_launch_us": us_attn},
+           "roofline_precompute": {"bound": "tensor", "kernel": "proj_gemm_kernel (mode 0, n_out 256)", "achieved": tf_pre,
+                                   "peak": pk["bf16_tflops_burst"], "peak_kind": pk["peak_kind"] + " (burst)", "unit": "TFLOP/s",
+                                   "frac": tf_pre / pk["bf16_tflops_burst"], "attainable_min_tensor_hbm": attainable,
+                                   "frac_of_attainable": tf_pre / attainable,
+                                   "traffic": cap_pre["dram_bytes"] if cap_pre else None, "algorithmic_flops_per_launch": fl_pre,
+                                   "algorithmic_bytes_per_launch": pre_bytes, "avg_launch_us": us_pre}}
+    if cpu_seconds > 0:
+        res["cpu_baseline"] = _oracle_turn_sample(px, geo, desc, w, A_packed, W_packed, T, S, cur, seed, cpu_seconds)
+    return res
+
+
+def _oracle_turn_sample(px, geo, desc, w, A_packed, W_packed, T, S, cur, seed, budget_s):
+    """The oracle on a sample of the turn's prefill (merged-weight K/V of two kv heads over all T + S tokens, then
+    naive attention for a few query rows), timed; the GPU result for the same rows is checked against it."""
+    import numpy as np
+    import torch
+    from oracle import lrkv_oracle as O
+    from paper_2609_34054_b200 import inputs as I
+    from paper_2609_34054_b200.binding import Cache
+    f64 = lambda t: t.detach().float().cpu().numpy().astype(np.float64)
+    H = torch.cat([I.hidden_states(T, geo, seed, "C3.H_ctx"), I.hidden_states(S, geo, seed, "C3.H_new_adpt")])
+    cache = Cache(geo, (T + S + 15) // 16)
+    px.rebase_project(desc, H.cuda(), W_packed, cache, 0)
+    px.lr_precompute(desc, H.cuda(), A_packed, cache, 0)
+    q = I.queries(S, geo, seed, "C3.q", gain=4.0)
+    out = torch.empty_like(q, device="cuda")
+    px.lr_attend_prefill(desc, q.cuda(), cur, T, w["B_k"], w["B_v"], cache, out)
+    torch.cuda.synchronize()
+    heads = [0, 5]
+    rows = [0, 1, 17, 255, 256, 510, 511]
+    wn = {k: f64(v) for k, v in w.items()}
+    t0 = time.perf_counter()
+    ref = O.lr_prefill_reference(f64(q), cur, T, f64(H), wn["W_k"], wn["W_v"], wn["A_k"], wn["B_k"], wn["A_v"], wn["B_v"],
+                                 geo.scale_k, geo.scale_v, geo.n_kv, heads=heads, rows=rows)
+    dt = time.perf_counter() - t0
+    got = f64(out)
+    m = ~np.isnan(ref)
+    err = float(np.abs(got[m] - ref[m]).max())
+    G = geo.group
+    # work of the sample in the units of the GPU row: attention flops of the sampled (row, head) pairs, plus the
+    # projection of the sampled heads' K and V columns that the oracle needs first
+    fl_attn = sum(4.0 * G * len(heads) * (geo.hd + (geo.rank_k + geo.rank_v) / 2) * (T + r + 1) for r in rows)
+    fl_proj = 2.0 * (T + S) * geo.d_model * 2 * len(heads) * geo.hd
+    return {"value": (fl_attn + fl_proj) / dt / 1e12, "unit": "TFLOP/s", "cores": cpu_threads(), "kind": "oracle",
+            "sample": f"kv heads {heads} x query rows {rows} of the {S}-token turn over {T} tokens: merged-weight K/V projection "
+                      f"of those heads ({fl_proj / 1e9:.0f} GFLOP) + naive attention ({fl_attn / 1e9:.2f} GFLOP) in float64, {dt:.1f} s",
+            "gpu_max_abs_err_on_sample": err, "budget_s": budget_s}
 
 
 C3_LAYERS_FOR_TTFT = 32
@@ -335,12 +451,11 @@ class Workload:
         self.layers, self.dsteps, self.T = layers, steps, T
         self.desc = layer_desc(geo)
         nb = (T + 15) // 16
-        self.H_host, self.H, self.A_packed, self.W_packed, self.B_k, self.B_v, self.cache = [], [], [], [], [], [], []
+        self.H_host, self.H, self.WA_packed, self.B_k, self.B_v, self.cache = [], [], [], [], [], []
         for l in range(layers):
             w = I.layer_weights(geo, seed, f"L{l}")
             dev = {k: v.cuda() for k, v in w.items()}
-            self.A_packed.append(px.pack_adapters(geo, dev["A_k"], dev["A_v"]))
-            self.W_packed.append(px.pack_base_weights(geo, dev["W_k"], dev["W_v"]))
+            self.WA_packed.append(px.pack_turn_weights(geo, dev["W_k"], dev["W_v"], dev["A_k"], dev["A_v"]))
             self.B_k.append(dev["B_k"]); self.B_v.append(dev["B_v"])
             h = I.hidden_states(T, geo, seed, f"L{l}.H").pin_memory()
             self.H_host.append(h)
@@ -355,14 +470,13 @@ class Workload:
         self.ctx = torch.full((1,), T, dtype=torch.int32, device="cuda")
         self.ws = px.decode_workspace(self.desc, 1, T)
         self.graph = None
-        self.launches_a = 2 * layers
+        self.launches_a = layers
         self.launches_b = geo.n_agents * steps * layers
 
     def phase_a(self):
         px = self.px
-        for l in range(self.layers):
-            px.rebase_project(self.desc, self.H[l], self.W_packed[l], self.cache[l], 0)
-            px.lr_precompute(self.desc, self.H[l], self.A_packed[l], self.cache[l], 0)
+        for l in range(self.layers):           # base rows and all agents' LR rows in one pass over the hidden states
+            px.turn_project(self.desc, self.H[l], self.WA_packed[l], self.cache[l], 0)
 
     def phase_b_eager(self):
         px, geo = self.px, self.geo
@@ -437,6 +551,15 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    ranks = None
+    if world > 1:
+        # evidence of the ranks that really ran: every rank reports its device
+        mine = {"rank": rank, "local_rank": local, "device": torch.cuda.get_device_name(local)}
+        ranks = [None] * world
+        dist.all_gather_object(ranks, mine)
+        if rank == 0:
+            sys.stderr.write(f"bench.py: {world} ranks over NCCL: {ranks}\n")
+
     px = Precc(local)
     if args.extra_only:
         res = extra_serving_decode(px, args.c4_batch, args.c4_ctx_min, args.c4_ctx_max) if args.extra_only == "c4" \
@@ -503,11 +626,13 @@ def run_gpu(args):
             "dtype": "bf16", "data": "synthetic",
             "config": {
                 "workload": f"C2 llama-3.2-1B-shaped stack: {wl.layers} layers d=2048 32q/8kv hd=64, N=4 agents r=16 on K,V, "
-                            f"T={wl.T}: base projection + LR precompute, then {wl.dsteps} decode steps per agent (batch 1)",
+                            f"T={wl.T}: fused base projection + LR precompute of the trajectory, then {wl.dsteps} decode steps "
+                            f"per agent (batch 1)",
                 "parallelism": "replicas" if world > 1 else "single GPU",
                 "l2_policy": f"decode cycles over {wl.layers} layers' caches = "
                              f"{wl.layers * per_launch / 1e6:.0f} MB > 126 MB L2; no explicit flush",
                 "decode_launch": "CUDA graph replay" if not args.no_graph else "eager ctypes launches",
+                "ranks": ranks,
             },
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(), "d2h_bytes_per_step": wl.d2h_bytes(),
@@ -515,8 +640,9 @@ def run_gpu(args):
             "gpu_launches": (wl.launches_a + wl.launches_b) * args.steps,
             "roofline": {"bound": "hbm", "kernel": "lr_attend_decode_cluster_kernel<64,16,16,8>", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
-                         "traffic": NCU_DECODE_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": per_launch,
-                         "avg_launch_us": launch_us},
+                         "traffic": (ncu_traffic("decode_cluster_c2_layer") or {}).get("dram_bytes"),
+                         "algorithmic_bytes_per_launch": per_launch, "avg_launch_us": launch_us,
+                         "note": "batch-1 launch of 17 MB: latency-bound by construction; the bandwidth-bound decode row is rooflines.decode_serving"},
             "phases": {"precompute_ms_per_step": pa / args.steps, "decode_ms_per_step": pb / args.steps,
                        "projection_tflops": flops_a / (pa / args.steps * 1e-3) / 1e12,
                        "decode_only_GBps": step_bytes / (pb / args.steps * 1e-3) / 1e9},
@@ -524,13 +650,54 @@ def run_gpu(args):
         if world == 1 and not args.no_extra:
             del wl
             torch.cuda.empty_cache()
-            line["extra"] = {"serving_decode": extra_serving_decode(px, 64, 4096, 32768),
-                             "turn": extra_turn(px, 32768, 512)}
+            cpu_s = 0.0 if args.no_cpu else 6.0
+            line["extra"] = {"serving_decode": extra_serving_decode(px, 64, 4096, 32768, cpu_seconds=cpu_s),
+                             "turn": extra_turn(px, 32768, 512, cpu_seconds=cpu_s)}
+            # the other rows of the metric, each with its own roofline record (the timed step's is `roofline`)
+            line["rooflines"] = {"decode_c2_layer": line["roofline"],
+                                 "decode_serving": line["extra"]["serving_decode"]["roofline"],
+                                 "prefill_turn": line["extra"]["turn"]["roofline_prefill"],
+                                 "lr_precompute_context": line["extra"]["turn"]["roofline_precompute"]}
         if cpu_val is not None:
             line["cpu_baseline"] = {"value": cpu_val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                                     "sample": f"{args.cpu_requests} decode requests of layer 0 (all kv heads, context {I.C2_T}), "
                                               f"{cpu_dt:.1f} s of numpy float64"}
         print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def spawn_ranks(n: int, argv) -> int:
+    """`bench.py --gpus N` run by hand: start N ranks of this script (one per GPU) under torch.distributed.run on
+    127.0.0.1 and return the launcher's exit code.  Rank 0 prints the JSON line."""
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def run_stub(args) -> int:
+    """The multi-rank plumbing of the benchmark without a GPU: gloo ranks, a sleep of (rank + 1) ms as the step, the
+    same barrier / max-over-ranks / whole-job aggregation, one JSON line from rank 0."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(1e-3 * (rank + 1))
+    ms = reduce_max_ms((time.perf_counter() - t0) * 1e3)
+    ranks = [None] * world
+    if world > 1:
+        dist.all_gather_object(ranks, {"rank": rank, "pid": os.getpid()})
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": whole_job_value(1e6, args.steps, ms, world), "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "ms_per_step": ms / args.steps, "stub": True, "scaling": "weak",
+                          "config": {"workload": "stub", "parallelism": "replicas", "ranks": ranks}}))
     if world > 1:
         dist.destroy_process_group()
     return 0
@@ -555,9 +722,15 @@ def main():
     ap.add_argument("--c4-ctx-max", type=int, default=32768)
     ap.add_argument("--c3-ctx", type=int, default=32768)
     ap.add_argument("--c3-new", type=int, default=512)
+    ap.add_argument("--stub-workload", action="store_true",
+                    help="run the rank plumbing (launch, barrier, max-reduce, aggregation) on CPU over gloo with a sleep as the step")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args.gpus, sys.argv[1:])          # started without a launcher: become one
     if args.impl == "reference":
         return run_reference(args)
+    if args.stub_workload:
+        return run_stub(args)
     return run_gpu(args)
 
 

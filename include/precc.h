@@ -19,7 +19,7 @@
  * Conventions
  *   - All tensors are bf16 in DEVICE memory unless stated; all accumulation is fp32; stores round to
  *     nearest even.  Index arrays are int32 in DEVICE memory unless stated.
- *   - Every buffer is owned by the caller.  Apart from the 4-byte status word that precc_create obtains
+ *   - Every buffer is owned by the caller.  Apart from the 8 bytes (status word, wait limit) that precc_create obtains
  *     (and precc_destroy releases) the library allocates no device memory; it keeps no pointer after the
  *     work it enqueued on `stream` has completed.  `stream` is a cudaStream_t passed as void* (NULL = the
  *     default stream).  The compute calls are asynchronous with respect to the host and can be captured
@@ -93,8 +93,8 @@ typedef struct {
   int64_t n_blocks;            /* physical blocks in each of the four arrays */
 } precc_cache;
 
-/* Create a context for CUDA device `device` (host allocation only, plus a 4-byte device status
- * word obtained with cudaMalloc here and released in precc_destroy). */
+/* Create a context for CUDA device `device` (host allocation only, plus 8 bytes of device memory - the status
+ * word and the wait limit - obtained with cudaMalloc here and released in precc_destroy). */
 int32_t precc_create(precc_ctx** out, int32_t device);
 int32_t precc_destroy(precc_ctx* ctx);
 /* Text of the last error seen by `ctx` (owned by ctx, valid until the next call on it). */
@@ -114,6 +114,17 @@ int32_t precc_set_trace_buffer(precc_ctx* ctx, void* buffer, size_t n_blocks);
  * Synchronises `stream`.  *status_out receives an OR of PRECC_STATUS_* bits.  Returns PRECC_OK when the
  * word is zero, PRECC_ERR_DEVICE_STATUS otherwise. */
 int32_t precc_poll_status(precc_ctx* ctx, void* stream, uint32_t* status_out);
+
+/* Bounded waits (no paper counterpart).  Every wait inside a kernel of this library - on an mbarrier that a TMA
+ * copy or a tensor-core commit completes - gives up after a limit, records PRECC_STATUS_TIMEOUT and lets the kernel
+ * run to its end (freeing its tensor memory); results of that launch are void, the context stays usable.  The limit
+ * is a number of SM clock cycles, about one second by default (sm_cycles == 0 restores the default); it is rounded
+ * up to a multiple of 1024 cycles.  The call synchronises with nothing: set it while no kernel of this context runs. */
+int32_t precc_set_wait_limit(precc_ctx* ctx, uint64_t sm_cycles);
+/* Self-test of that mechanism: one tiny kernel waits on a barrier that is never completed.  It must end by itself
+ * after the wait limit; *done_flag (device uint32) then holds 2 and precc_poll_status reports
+ * PRECC_STATUS_TIMEOUT.  With the default limit this takes about a second of GPU time: lower the limit first. */
+int32_t precc_selftest_wait_timeout(precc_ctx* ctx, uint32_t* done_flag, void* stream);
 
 /* Pack a row-major [d_model][n_cols] matrix (paper layout d_in x d_out) as rows [dst_row0, dst_row0 +
  * n_cols) of a packed matrix of dst_rows rows, the operand format of the projection kernels: k-blocked

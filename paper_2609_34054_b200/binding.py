@@ -24,6 +24,7 @@ EXPORTS = [
     "precc_lr_attend_decode_static", "precc_lr_attend_prefill",
     "precc_rebase_project_rope", "precc_turn_project_rope", "precc_lr_attend_decode_rope", "precc_lr_attend_prefill_rope",
     "precc_turn_project_rows", "precc_partial_record_floats", "precc_lr_attend_decode_partial", "precc_combine_partials",
+    "precc_set_wait_limit", "precc_selftest_wait_timeout",
 ]
 
 
@@ -68,6 +69,8 @@ def load_library() -> C.CDLL:
     lib.precc_sm_count.argtypes = [vp]
     lib.precc_set_trace_buffer.argtypes = [vp, vp, sz]
     lib.precc_poll_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+    lib.precc_set_wait_limit.argtypes = [vp, u64]
+    lib.precc_selftest_wait_timeout.argtypes = [vp, vp, vp]
     lib.precc_pack_kmajor.argtypes = [vp, vp, i32, i32, vp, i32, i32, vp]
     lib.precc_lr_precompute.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, u64, C.POINTER(CacheDesc), vp]
     lib.precc_rebase_project.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, C.POINTER(CacheDesc), vp]
@@ -191,6 +194,14 @@ class Precc:
         st = C.c_uint32(0)
         self.lib.precc_poll_status(self.h, _stream(), C.byref(st))
         return st.value
+
+    def set_wait_limit(self, sm_cycles: int):
+        """Limit of the kernels' bounded waits in SM clock cycles (0 = the default of about a second)."""
+        self._check(self.lib.precc_set_wait_limit(self.h, sm_cycles), "precc_set_wait_limit")
+
+    def selftest_wait_timeout(self, done_flag: torch.Tensor):
+        """Launch the kernel that waits on a barrier nothing completes; done_flag: uint32/int32 CUDA tensor of one element."""
+        self._check(self.lib.precc_selftest_wait_timeout(self.h, _ptr(done_flag), _stream()), "precc_selftest_wait_timeout")
 
     def pack_kmajor(self, src: torch.Tensor, dst: torch.Tensor, dst_row0: int):
         d, n = src.shape

@@ -128,6 +128,22 @@ int32_t make_map_cache4(precc_ctx* ctx, CUtensorMap* map, const void* base, long
 
 
 namespace {
+// A barrier that nothing ever arrives on: the waiting lane must give up after the context's wait limit, record
+// PRECC_STATUS_TIMEOUT and let the kernel end normally (the self-test of the bounded waits every tcgen05 / TMA
+// kernel of the library uses).
+__global__ void wait_timeout_selftest_kernel(uint32_t* status, uint32_t* done_flag) {
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncwarp();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = mbar_wait(smem_u32(&bar), 0, status);
+  __syncwarp();
+  if (threadIdx.x == 0) *done_flag = ok ? 1u : 2u;      // 2: the wait expired and the kernel carried on to its end
+}
+
 // ------------------------------------------------------------------------------------------ pack
 // dst is k-blocked: element (row, i) lives at ((i / 64) * dst_rows + row) * 64 + i % 64, so the 64-deep k
 // step of any range of rows is one contiguous run in memory (what a TMA box of the GEMMs fetches).
@@ -163,8 +179,11 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->status, sizeof(uint32_t));
-  if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->status, 2 * sizeof(uint32_t));
+  if (e == cudaSuccess) {
+    const uint32_t init[2] = {0u, kDefaultWaitLimit};
+    e = cudaMemcpy(ctx->status, init, sizeof(init), cudaMemcpyHostToDevice);
+  }
   if (e == cudaSuccess) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -232,6 +251,23 @@ int32_t precc_poll_status(precc_ctx* ctx, void* stream, uint32_t* status_out) {
   if (status_out) *status_out = h;
   if (h) return fail(ctx, PRECC_ERR_DEVICE_STATUS, "device status 0x%x%s%s", h, (h & PRECC_STATUS_BAD_INDEX) ? " bad-index" : "",
                      (h & PRECC_STATUS_TIMEOUT) ? " timeout" : "");
+  return PRECC_OK;
+}
+
+int32_t precc_set_wait_limit(precc_ctx* ctx, uint64_t sm_cycles) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  uint64_t units = sm_cycles == 0 ? kDefaultWaitLimit : (sm_cycles + 1023) >> 10;
+  if (units > 0xffffffffull) units = 0xffffffffull;
+  const uint32_t v = static_cast<uint32_t>(units < 1 ? 1 : units);
+  PRECC_CUDA(ctx, cudaMemcpy(ctx->status + 1, &v, sizeof(v), cudaMemcpyHostToDevice));
+  return PRECC_OK;
+}
+
+int32_t precc_selftest_wait_timeout(precc_ctx* ctx, uint32_t* done_flag, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!done_flag) return fail(ctx, PRECC_ERR_INVALID_ARG, "done_flag is null");
+  wait_timeout_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(ctx->status, done_flag);
+  PRECC_CUDA(ctx, cudaGetLastError());
   return PRECC_OK;
 }
 

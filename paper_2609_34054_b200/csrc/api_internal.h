@@ -20,7 +20,7 @@ struct precc_ctx {
   int device = 0;
   int sm_count = 0;
   int max_smem_optin = 0;
-  uint32_t* status = nullptr;          // device status word
+  uint32_t* status = nullptr;          // two device words: [0] status bits, [1] limit of the bounded waits (x 1024 cycles)
   unsigned long long* trace = nullptr; // optional caller-owned trace buffer
   size_t trace_blocks = 0;
   bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
@@ -40,6 +40,7 @@ struct precc_ctx {
 namespace precc {
 
 constexpr int kMaxDevices = 64;
+constexpr uint32_t kDefaultWaitLimit = 2000000000u >> 10;   // about a second of SM clock, in units of 1024 cycles
 
 int32_t fail(precc_ctx* ctx, int32_t code, const char* fmt, ...);
 

@@ -54,15 +54,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait (about a second of SM clock).  Returns false after recording a timeout.
+// Bounded wait.  `status` points at the context's two device words: [0] the status bits, [1] the wait limit in
+// units of 1024 SM clock cycles (default: about a second).  Returns false after recording a timeout.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
+  const long long limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > 2000000000LL) break;
+    if (clock64() - t0 > limit) break;
     // once any wait in the grid has expired the results are void anyway: do not queue up more seconds
     if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
   }

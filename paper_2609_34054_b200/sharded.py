@@ -1,11 +1,18 @@
-"""Context-sharded decode over several GPUs (one process per GPU): each rank keeps a contiguous,
+"""Decode attention of one layer spread over several GPUs (one process per GPU), two ways.
+
+Context sharding: each rank keeps a contiguous,
 page-aligned range of every request's tokens in its own caches, computes the split-KV record of its range
 (``precc_lr_attend_decode_partial``), the records are all-gathered, and every rank merges them
 (``precc_combine_partials``).  The exchange is ``(16 + 8 (hd + r_v)) * 4`` bytes per (request, kv head) and
 rank, independent of the context length.  The paper is single-GPU; this is the natural way its path
 shards when one GPU's HBM no longer holds a trajectory.
 
-Only the plumbing lives here (range planning, the collective, buffer reuse); all arithmetic is in the two
+Head sharding: each rank keeps the base cache of ``n_kv / world`` kv heads (and the matching columns of B_k and
+B_v); the LR caches, a few percent of the bytes, are replicated.  A rank runs the ordinary decode call with the
+descriptor of its slice (no new kernel: the heads of a layer never interact inside attention) and the outputs
+``[B][n_q / world][hd]`` are all-gathered into ``[B][n_q][hd]``.
+
+Only the plumbing lives here (range and head planning, the collectives, buffer reuse); all arithmetic is in the
 kernels behind the C ABI.
 """
 from __future__ import annotations
@@ -16,7 +23,8 @@ import torch
 import torch.distributed as dist
 
 from .binding import Cache, LayerDesc, Precc
-from .inputs import PAGE
+from .binding import layer_desc
+from .inputs import PAGE, Geometry
 
 
 def shard_ranges(ctx_len: Sequence[int], world: int, page: int = PAGE) -> List[List[Tuple[int, int]]]:
@@ -70,3 +78,76 @@ class ShardedDecoder:
         gather_records(local, self.group, gathered)
         self.px.combine_partials(self.desc, gathered, agent_id, B_v, out)
         return out
+
+
+# --------------------------------------------------------------------------------------------- head sharding
+
+def head_shard_geometry(geo: Geometry, world: int) -> Geometry:
+    """Geometry of one rank's slice: n_kv / world kv heads with their query heads; everything else unchanged."""
+    if geo.n_kv % world:
+        raise ValueError(f"{geo.n_kv} kv heads do not divide over {world} ranks")
+    return Geometry(d_model=geo.d_model, n_q=geo.n_q // world, n_kv=geo.n_kv // world, hd=geo.hd, n_agents=geo.n_agents,
+                    rank_k=geo.rank_k, rank_v=geo.rank_v, alpha=geo.alpha)
+
+
+def head_slice(rank: int, world: int, n_heads: int) -> slice:
+    """The heads (kv or query) that rank `rank` owns: a contiguous run, in rank order."""
+    per = n_heads // world
+    return slice(rank * per, (rank + 1) * per)
+
+
+def shard_cache_heads(cache: Cache, geo: Geometry, rank: int, world: int) -> Cache:
+    """One rank's caches cut out of full-width ones (for tests and for loading a sharded layout from a replicated
+    one): base K/V of its kv heads (copied: the head axis is not the outermost), LR caches as they are."""
+    hs = head_slice(rank, world, geo.n_kv)
+    return Cache.from_tensors(head_shard_geometry(geo, world), cache.k_base[:, hs].contiguous(), cache.v_base[:, hs].contiguous(),
+                              cache.lr_k, cache.lr_v)
+
+
+def shard_b_heads(B: Optional[torch.Tensor], geo: Geometry, rank: int, world: int) -> Optional[torch.Tensor]:
+    """Columns of B_k / B_v ([n_agents][rank][n_kv*hd]) that belong to the rank's kv heads."""
+    if B is None:
+        return None
+    hs = head_slice(rank, world, geo.n_kv)
+    return B[:, :, hs.start * geo.hd:hs.stop * geo.hd].contiguous()
+
+
+def gather_heads(local_out: torch.Tensor, group: Optional[dist.ProcessGroup] = None,
+                 staging: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """local_out [B][n_q_local][hd] of every rank -> [B][world * n_q_local][hd], rank r's heads at [r * n_q_local, ...)."""
+    world = dist.get_world_size(group)
+    B, hq, hd = local_out.shape
+    if staging is None:
+        staging = torch.empty((world, B, hq, hd), dtype=local_out.dtype, device=local_out.device)
+    dist.all_gather_into_tensor(staging.view(-1), local_out.contiguous().view(-1), group=group)
+    res = staging.permute(1, 0, 2, 3).reshape(B, world * hq, hd)
+    if out is None:
+        return res.contiguous()
+    out.copy_(res)
+    return out
+
+
+class HeadShardedDecoder:
+    """Decode attention of one layer with the kv heads divided over the ranks of `group`."""
+
+    def __init__(self, px: Precc, geo: Geometry, group: Optional[dist.ProcessGroup] = None, softmax_scale: float = 0.0):
+        self.px, self.geo, self.group = px, geo, group
+        self.world = dist.get_world_size(group)
+        self.rank = dist.get_rank(group)
+        self.local_geo = head_shard_geometry(geo, self.world)
+        self.desc = layer_desc(self.local_geo, softmax_scale)
+        self._local = self._staging = None
+
+    def decode(self, q: torch.Tensor, agent_id: torch.Tensor, ctx_len: torch.Tensor, max_ctx: int, B_k_local, B_v_local,
+               cache_local: Cache, out: torch.Tensor, workspace: torch.Tensor, block_table: Optional[torch.Tensor] = None,
+               first_block: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """q [B][n_q][hd] (the same on every rank; the rank's heads are cut out here), caches and B matrices of the
+        rank's heads; out [B][n_q][hd]: the full result on every rank."""
+        hs = head_slice(self.rank, self.world, self.geo.n_q)
+        q_local = q[:, hs].contiguous()
+        if self._local is None or self._local.shape != q_local.shape:
+            self._local = torch.empty_like(q_local)
+            self._staging = torch.empty((self.world,) + tuple(q_local.shape), dtype=q.dtype, device=q.device)
+        self.px.lr_attend_decode(self.desc, q_local, agent_id, ctx_len, max_ctx, B_k_local, B_v_local, cache_local, self._local,
+                                 workspace, block_table, first_block)
+        return gather_heads(self._local, self.group, self._staging, out)

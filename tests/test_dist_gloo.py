@@ -47,6 +47,26 @@ def test_replica_aggregation_world_size_2():
     assert res[0][2] is False                             # replicas see different seeded inputs
 
 
+def test_bench_gpus_flag_starts_that_many_ranks():
+    """`python bench.py --gpus 2` without a launcher re-executes itself under torch.distributed.run with two ranks;
+    here with the stub step on gloo: the line must come from rank 0, count two ranks with different pids, take the
+    slower rank's time and sum the ranks' units."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "5", "--stub-workload"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                      # rank 0 alone prints
+    d = lines[0]
+    assert d["n_gpus"] == 2 and d["stub"] and d["scaling"] == "weak"
+    ranks = d["config"]["ranks"]
+    assert [x["rank"] for x in ranks] == [0, 1] and ranks[0]["pid"] != ranks[1]["pid"]
+    assert d["ms_per_step"] >= 2.0                              # rank 1 sleeps 2 ms per step: the max over ranks
+    assert abs(d["value"] - 2 * 1e6 * 5 / (d["ms_per_step"] * 5e-3) / 1e9) < 1e-9
+
+
 def test_single_process_is_identity():
     sys.path.insert(0, ROOT)
     import bench
@@ -108,3 +128,45 @@ def test_gather_records_layout_world_size_2():
     for r in range(world):
         shape, vals, tags, reused = res[r]
         assert shape == (2, 3, 2, 24) and vals == [1.0, 2.0] and tags == [100.0, 101.0] and reused   # slot s holds rank s's records
+
+
+def _gather_heads_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2609_34054_b200.sharded import gather_heads
+    B, hq, hd = 3, 2, 4
+    local = torch.arange(B * hq * hd, dtype=torch.float32).reshape(B, hq, hd) + 1000.0 * rank
+    got = gather_heads(local)
+    buf = torch.empty((B, world * hq, hd), dtype=torch.float32)
+    again = gather_heads(local, None, None, buf)
+    out[rank] = (tuple(got.shape), [float(got[1, r * hq + 1, 2]) for r in range(world)], bool(torch.equal(again, got)),
+                 again.data_ptr() == buf.data_ptr())
+    dist.destroy_process_group()
+
+
+def test_gather_heads_layout_world_size_2():
+    """Head-sharded decode: rank r's query heads land at [r * n_q_local, (r + 1) * n_q_local) of every request."""
+    world = 2
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_gather_heads_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+        res = dict(out)
+    for r in range(world):
+        shape, vals, same, reused = res[r]
+        assert shape == (3, 4, 4) and vals == [14.0, 1014.0] and same and reused
+
+
+def test_head_shard_planning():
+    sys.path.insert(0, ROOT)
+    from paper_2609_34054_b200 import inputs as I
+    from paper_2609_34054_b200.sharded import head_shard_geometry, head_slice
+    g = head_shard_geometry(I.C3, 4)
+    assert (g.n_q, g.n_kv, g.hd, g.rank_k, g.n_agents, g.d_model) == (8, 2, 128, 32, 4, 4096) and g.scale_k == I.C3.scale_k
+    assert [head_slice(r, 4, 8) for r in range(4)] == [slice(0, 2), slice(2, 4), slice(4, 6), slice(6, 8)]
+    try:
+        head_shard_geometry(I.C3, 3)
+        assert False
+    except ValueError:
+        pass

@@ -1,6 +1,8 @@
 """Out-of-bounds writes: every output and cache buffer sits between guard regions filled with a sentinel
 bit pattern; after each entry point has run at awkward sizes (ragged tails, partial pages, masked agents,
 scattered slots) the guards must be untouched, and so must every cache row that was not addressed."""
+import time
+
 import pytest
 import torch
 
@@ -86,4 +88,54 @@ def test_all_entry_points_stay_inside_their_buffers(hd, r, M, S):
     for name, raw in raws.items():
         assert guards_intact(raw), name
     assert px.poll_status() == 0
+    px.close()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """Failure detection without a fault: every wait inside the library's kernels has a limit.  A kernel whose
+    barrier is never completed must end by itself once the limit (lowered here to about a millisecond) has passed,
+    the status word must say TIMEOUT, nothing around the flag it writes may be touched, and the context must go on
+    working: the same projection + attention calls give the same bits before and after."""
+    px = Precc(0)
+    geo = I.Geometry(d_model=256, n_q=8, n_kv=2, hd=128, n_agents=2, rank_k=16, rank_v=16, alpha=32.0)
+    desc = layer_desc(geo)
+    w = {k: v.cuda() for k, v in I.layer_weights(geo, 4, "to").items()}
+    WA = px.pack_turn_weights(geo, w["W_k"], w["W_v"], w["A_k"], w["A_v"])
+    T, S = 600, 96
+    H = I.hidden_states(T, geo, 4, "to.H").cuda()
+    q, qs = I.queries(2, geo, 4, "to.q").cuda(), I.queries(S, geo, 4, "to.qs").cuda()
+    aid = torch.tensor([0, 1], dtype=torch.int32, device="cuda")
+    cl = torch.tensor([T, 77], dtype=torch.int32, device="cuda")
+
+    def ordinary():
+        cache = Cache(geo, (T + 15) // 16 + 1, fill=0.0)
+        px.turn_project(desc, H, WA, cache, 0)                      # tcgen05 GEMM: bounded mbarrier waits inside
+        out = torch.full_like(q, float("nan"))
+        px.lr_attend_decode(desc, q, aid, cl, T, w["B_k"], w["B_v"], cache, out, px.decode_workspace(desc, 2, T))
+        outp = torch.full_like(qs, float("nan"))
+        px.lr_attend_prefill(desc, qs, 1, T - S, w["B_k"], w["B_v"], cache, outp)   # tcgen05 prefill: bounded waits too
+        torch.cuda.synchronize()
+        return cache.k_base.clone(), out, outp
+
+    before = ordinary()
+    assert px.poll_status() == 0
+    px.set_wait_limit(2_000_000)                                     # about 1 ms of SM clock
+    raw = torch.full((2 * 64 + 1,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    flag = raw[64:65]
+    t0 = time.perf_counter()
+    px.selftest_wait_timeout(flag)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert dt < 0.5, f"the wait did not give up at its limit ({dt:.2f} s)"
+    assert flag.item() == 2                                          # expired, then ran to its end
+    assert (raw[:64] == 0x5A5A5A5A).all() and (raw[65:] == 0x5A5A5A5A).all()
+    assert px.poll_status() == 2                                     # PRECC_STATUS_TIMEOUT, nothing else
+    assert px.poll_status() == 0                                     # cleared by the read
+    after_low = ordinary()                                           # real kernels under the 1 ms limit: none of their waits runs out
+    assert px.poll_status() == 0
+    px.set_wait_limit(0)                                             # back to the default
+    after = ordinary()
+    assert px.poll_status() == 0
+    for a, b, c in zip(before, after_low, after):
+        assert torch.equal(a, b) and torch.equal(a, c)
     px.close()

@@ -8,7 +8,8 @@ import torch
 from oracle import lrkv_oracle as O
 from paper_2609_34054_b200 import inputs as I
 from paper_2609_34054_b200.binding import Precc, PreccError
-from paper_2609_34054_b200.sharded import shard_ranges
+from paper_2609_34054_b200.binding import layer_desc
+from paper_2609_34054_b200.sharded import head_shard_geometry, head_slice, shard_b_heads, shard_cache_heads, shard_ranges
 
 from harness import Layer, assert_close, f64
 
@@ -113,3 +114,43 @@ def test_long_context_shards_take_the_cluster_path(px):
     ref0 = O.lr_decode_reference(f64(q[:1]), [3], [T], *args, geo.scale_k, geo.scale_v, geo.n_kv)
     ref1 = O.lr_decode_reference(f64(q[1:]), [0], [5000], *args, 0.0, 0.0, geo.n_kv)
     assert_close(f64(out), np.concatenate([ref0, ref1]), "sharded C2 decode")
+
+
+@pytest.mark.parametrize("hd,n_q,n_kv,r,world", [(64, 16, 4, 16, 2), (128, 16, 8, 32, 4), (128, 8, 8, 8, 8), (64, 8, 2, 0, 2)])
+def test_head_sharded_equals_the_oracle_and_the_unsharded_call(px, hd, n_q, n_kv, r, world):
+    """Head sharding: every rank runs the ordinary decode call on the caches of its kv heads (LR caches replicated)
+    and the outputs are concatenated along the head axis.  The ranks are emulated one after another on one GPU; the
+    result must meet the oracle's bar, and each rank's slice must equal the oracle's slice for its heads."""
+    geo = I.Geometry(d_model=192, n_q=n_q, n_kv=n_kv, hd=hd, n_agents=2, rank_k=r, rank_v=r, alpha=2.0 * max(r, 1))
+    T = 1500
+    H = I.hidden_states(T, geo, 21, "hs.H")
+    L = Layer(px, geo, seed=21, n_blocks=(T + 15) // 16, tag="hs")
+    L.append(H)
+    agents, ctx = [0, 1, -1, 1], [T, 777, 300, 16]
+    q = I.queries(len(ctx), geo, 21, "hs.q", gain=4.0)
+    aid = torch.tensor(agents, dtype=torch.int32).cuda()
+    cl = torch.tensor(ctx, dtype=torch.int32).cuda()
+    local_geo = head_shard_geometry(geo, world)
+    desc = layer_desc(local_geo)
+    parts = []
+    for rank in range(world):
+        cache_r = shard_cache_heads(L.cache, geo, rank, world)
+        Bk, Bv = shard_b_heads(L.B_k, geo, rank, world), shard_b_heads(L.B_v, geo, rank, world)
+        q_r = q[:, head_slice(rank, world, geo.n_q)].contiguous().cuda()
+        out_r = torch.full_like(q_r, float("nan"))
+        ws = px.decode_workspace(desc, len(ctx), T)
+        px.lr_attend_decode(desc, q_r, aid, cl, T, Bk, Bv, cache_r, out_r, ws)
+        parts.append(out_r)
+    torch.cuda.synchronize()
+    out = torch.cat(parts, dim=1)                        # what gather_heads builds from the all-gathered slices
+    w, Hn = L.w_np, f64(H)
+    ref = np.zeros((len(ctx), n_q, hd))
+    for b, (a, t) in enumerate(zip(agents, ctx)):
+        if a >= 0 and r > 0:
+            ref[b] = O.lr_decode_reference(f64(q[b:b + 1]), [a], [t], Hn, w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                           geo.scale_k, geo.scale_v, geo.n_kv)[0]
+        else:
+            ref[b] = O.attend_decode_one(f64(q[b]), O.base_cache(Hn, w["W_k"]), O.base_cache(Hn, w["W_v"]), t, geo.n_kv)
+    assert_close(f64(out), ref, f"head-sharded decode over {world} ranks")
+    whole = f64(L.decode(q, agents, ctx))                # the unsharded call: same values up to fp32 summation order
+    assert np.abs(f64(out) - whole).max() <= 2e-2
