@@ -2,6 +2,7 @@
 // their rotary forms) and the choice among the three projection kernels.
 #include "api_internal.h"
 #include "gemm_tc.cuh"
+#include "gemm_pair.cuh"
 #include "proj_small.cuh"
 
 using namespace precc;
@@ -80,7 +81,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   const int m_tiles = (M + GEMM_BM - 1) / GEMM_BM;
   // A few row tiles (the tokens of a short turn): the K extent of every tile is split over a cluster.  The split
   // depends on M and K alone, so a column's summation order is the same whichever entry point produced it.
-  if (m_tiles <= 4 && !gp.rope && !ctx->no_gemm_splitk) {
+  if (m_tiles <= 8 && !gp.rope && !ctx->no_gemm_splitk) {
     const int nkb = K / GEMM_BK;
     // planned for the width of the FUSED projection of this layer, whatever this call projects, so that the base-only,
     // LR-only and fused calls of one M take the same decision (and with it the same summation order)
@@ -93,7 +94,11 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
     // the finest split whose clusters are all resident at once (a second wave would cost more than the split gains);
     // cluster sizes need not be powers of two: 18 clusters fit as 6-block clusters, 36 as 3-block clusters
     int ks = GEMM_MAX_KS, smem_plan = 0;
-    for (; ks > 2; --ks) {                                       // a two-way split does not pay for its merge
+    // a two-way split does not pay for its merge (measured at 768 and 1024 rows of the fused Llama-3-8B projection:
+    // 32.7 and 33.1 us against 31.4 and 32.1 us without a split), so the split must be three-way or finer; with nine
+    // column tiles that serves up to five row tiles (640 rows: 25 us against 30.5 us)
+    const int ks_min = 3;
+    for (; ks >= ks_min; --ks) {
       if (nkb / ks < 2) continue;
       const int cw = ((256 + ks - 1) / ks + 7) / 8 * 8;          // planned for the widest tile, whatever this call's width
       const int dump = ks * GEMM_BM * (cw + 4) * 4;
@@ -119,7 +124,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
       }
       if (cached - 1 >= clusters) break;
     }
-    if (ks > 2) {
+    if (ks >= ks_min) {
       const int n_tiles = (n_out + bn - 1) / bn;
       int stages = 3;
       if (stages > nkb / ks) stages = nkb / ks;
@@ -150,6 +155,43 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   if (M <= PS_MAX_M && !ctx->force_tiled_gemm) {
     const int32_t rc = launch_small(ctx, X, M, K, Wt, n_out, gp, stream);
     if (rc >= 0) return rc;
+  }
+  // Many rows: two SMs per 256 x 256 tile (each stages half of the weight tile), see gemm_pair.cuh.
+  if (ctx->gemm_pair && M >= 2 * GEMM_PAIR_BM) {
+    const int bn2 = n_out >= 256 ? 256 : (n_out + 15) / 16 * 16;
+    if (!(gp.rope && bn2 % gp.hd != 0)) {
+      const int stage2 = GEMM_A_BYTES + (bn2 / 2) * GEMM_BK * 2;
+      int st2 = (ctx->max_smem_optin - 4096) / stage2;
+      if (st2 > 8) st2 = 8;
+      if (st2 > K / GEMM_BK) st2 = K / GEMM_BK;
+      if (st2 >= 2) {
+        int tc2 = 32;
+        while (tc2 < 2 * bn2) tc2 <<= 1;
+        const size_t smem2 = (size_t)st2 * stage2 + (2 * st2 + 6) * 8 + 1024;
+        CUtensorMap map_x2, map_w2;
+        int32_t rc2 = make_map(ctx, &map_x2, X, M, K, GEMM_BM);
+        if (rc2) return rc2;
+        rc2 = make_map_w(ctx, &map_w2, Wt, n_out, K, bn2 / 2);
+        if (rc2) return rc2;
+        gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn2; gp.stages = st2; gp.tmem_cols = tc2;
+        gp.spread_rows = 1;
+        gp.status = ctx->status;
+        PRECC_CUDA(ctx, raise_smem_limit(ctx, proj_gemm_pair_kernel, (int)smem2));
+        const long long tiles2 = (long long)((M + GEMM_PAIR_BM - 1) / GEMM_PAIR_BM) * ((n_out + bn2 - 1) / bn2);
+        const int pairs = (int)(tiles2 < ctx->sm_count / 2 ? tiles2 : ctx->sm_count / 2);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * pairs);
+        cfg.blockDim = dim3(GEMM_THREADS);
+        cfg.dynamicSmemBytes = smem2;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, proj_gemm_pair_kernel, map_x2, map_w2, gp));
+        return PRECC_OK;
+      }
+    }
   }
   int bn = pick_bn(n_out, m_tiles, ctx->sm_count);
   if (gp.rope && bn % gp.hd != 0) bn = gp.hd;        // a head's two halves must sit in one tile

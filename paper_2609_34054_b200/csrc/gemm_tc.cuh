@@ -61,6 +61,74 @@ __device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, 
   if (dst2) *reinterpret_cast<uint4*>(dst2) = v;
 }
 
+// Epilogue of one output tile for one warp: TMEM lane = tile row (this warp owns lanes lane_base .. lane_base + 31 of
+// the accumulator at `tmem_tile`, which holds rows m0 .. m0 + 127 and columns n0 .. n0 + BN - 1).  Waits for the
+// accumulator (bounded), converts to bf16 and routes 16-byte pieces to the paged caches; key columns of the rotary
+// variant are rotated by the row's position first.
+__device__ __forceinline__ void gemm_epilogue_tile(const GemmParams& p, uint32_t tmem_tile, int m0, int n0, int lane_base, int lane,
+                                                   uint32_t acc_full_bar, uint32_t parity) {
+  const int row = lane_base + lane;
+  const int w = p.n_kv * p.hd;
+  const int gm = m0 + row;
+  bool row_ok = gm < p.M;
+  long long slot = 0;
+  if (row_ok) {
+    slot = p.slot_mapping ? (long long)p.slot_mapping[gm] : p.start_slot + gm;
+    if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
+  }
+  const long long blk = slot / PAGE;
+  const int off = (int)(slot % PAGE);
+  const unsigned long long row_mask = (p.row_masks && row_ok) ? p.row_masks[gm] : p.agent_mask;
+  long long pos = 0;
+  if (p.rope && row_ok) {
+    pos = p.positions ? (long long)p.positions[gm] : p.start_pos + gm;
+    if (pos < 0 || pos >= p.max_pos) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
+  }
+  mbar_wait(acc_full_bar, parity, p.status);
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  for (int c0 = 0; c0 < p.BN; c0 += 16) {
+    if (p.rope && n0 + c0 < w) {
+      // key columns: chunk [c, c+16) of the lower half of a head together with its partner chunk
+      const int gc = n0 + c0;
+      const int g = gc / p.hd, c = gc % p.hd;
+      if (c >= p.hd / 2) continue;                  // done with its partner
+      uint32_t lo[16], hi[16];
+      tmem_ld16(tmem_tile + (static_cast<uint32_t>(lane_base) << 16) + c0, lo);
+      tmem_ld16(tmem_tile + (static_cast<uint32_t>(lane_base) << 16) + c0 + p.hd / 2, hi);
+      asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+      if (!row_ok) continue;
+      const float4* cs = p.rope + pos * (p.hd / 4) + c / 2;
+      uint32_t ol[8], oh[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const float4 t4 = __ldg(cs + k);
+        const float l0 = __uint_as_float(lo[2 * k]), l1 = __uint_as_float(lo[2 * k + 1]);
+        const float h0 = __uint_as_float(hi[2 * k]), h1 = __uint_as_float(hi[2 * k + 1]);
+        ol[k] = pack_bf16(l0 * t4.x - h0 * t4.y, l1 * t4.z - h1 * t4.w);
+        oh[k] = pack_bf16(h0 * t4.x + l0 * t4.y, h1 * t4.z + l1 * t4.w);
+      }
+      __nv_bfloat16* dst = p.base_k + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
+      reinterpret_cast<uint4*>(dst)[0] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+      reinterpret_cast<uint4*>(dst)[1] = make_uint4(ol[4], ol[5], ol[6], ol[7]);
+      reinterpret_cast<uint4*>(dst + p.hd / 2)[0] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+      reinterpret_cast<uint4*>(dst + p.hd / 2)[1] = make_uint4(oh[4], oh[5], oh[6], oh[7]);
+      continue;
+    }
+    uint32_t r[16];
+    tmem_ld16(tmem_tile + (static_cast<uint32_t>(lane_base) << 16) + c0, r);
+    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int gc = n0 + c0 + 8 * h;
+      if (!row_ok || gc >= p.N_out) continue;
+      float v8[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(r[8 * h + k]);
+      store_piece(p, blk, off, gc, v8, row_mask, gm);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const GemmParams p) {
   extern __shared__ unsigned char smem_raw[];
@@ -155,70 +223,11 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   } else {
     // ---- epilogue: TMEM lane = tile row; this warp may touch lanes 32*(warp%4) .. +31
     const int lane_base = (warp & 3) * 32;
-    const int row = lane_base + lane;
-    const int w = p.n_kv * p.hd;
     int i = 0;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
       const int buf = i & 1;
       const int m0 = row0_of(t / n_tiles_n), n0 = (t % n_tiles_n) * p.BN;
-      const int gm = m0 + row;
-      bool row_ok = gm < p.M;
-      long long slot = 0;
-      if (row_ok) {
-        slot = p.slot_mapping ? (long long)p.slot_mapping[gm] : p.start_slot + gm;
-        if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
-      }
-      const long long blk = slot / PAGE;
-      const int off = (int)(slot % PAGE);
-      const unsigned long long row_mask = (p.row_masks && row_ok) ? p.row_masks[gm] : p.agent_mask;
-      long long pos = 0;
-      if (p.rope && row_ok) {
-        pos = p.positions ? (long long)p.positions[gm] : p.start_pos + gm;
-        if (pos < 0 || pos >= p.max_pos) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
-      }
-      mbar_wait(acc_full + 8 * buf, (i >> 1) & 1, p.status);
-      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-      for (int c0 = 0; c0 < p.BN; c0 += 16) {
-        if (p.rope && n0 + c0 < w) {
-          // key columns: chunk [c, c+16) of the lower half of a head together with its partner chunk
-          const int gc = n0 + c0;
-          const int g = gc / p.hd, c = gc % p.hd;
-          if (c >= p.hd / 2) continue;                  // done with its partner
-          uint32_t lo[16], hi[16];
-          tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + buf * p.BN + c0, lo);
-          tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + buf * p.BN + c0 + p.hd / 2, hi);
-          asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-          if (!row_ok) continue;
-          const float4* cs = p.rope + pos * (p.hd / 4) + c / 2;
-          uint32_t ol[8], oh[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const float4 t4 = __ldg(cs + k);
-            const float l0 = __uint_as_float(lo[2 * k]), l1 = __uint_as_float(lo[2 * k + 1]);
-            const float h0 = __uint_as_float(hi[2 * k]), h1 = __uint_as_float(hi[2 * k + 1]);
-            ol[k] = pack_bf16(l0 * t4.x - h0 * t4.y, l1 * t4.z - h1 * t4.w);
-            oh[k] = pack_bf16(h0 * t4.x + l0 * t4.y, h1 * t4.z + l1 * t4.w);
-          }
-          __nv_bfloat16* dst = p.base_k + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
-          reinterpret_cast<uint4*>(dst)[0] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-          reinterpret_cast<uint4*>(dst)[1] = make_uint4(ol[4], ol[5], ol[6], ol[7]);
-          reinterpret_cast<uint4*>(dst + p.hd / 2)[0] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
-          reinterpret_cast<uint4*>(dst + p.hd / 2)[1] = make_uint4(oh[4], oh[5], oh[6], oh[7]);
-          continue;
-        }
-        uint32_t r[16];
-        tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_base) << 16) + buf * p.BN + c0, r);
-        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int gc = n0 + c0 + 8 * h;
-          if (!row_ok || gc >= p.N_out) continue;
-          float v8[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(r[8 * h + k]);
-          store_piece(p, blk, off, gc, v8, row_mask, gm);
-        }
-      }
+      gemm_epilogue_tile(p, tmem_base + buf * p.BN, m0, n0, lane_base, lane, acc_full + 8 * buf, (i >> 1) & 1);
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(acc_empty + 8 * buf) : "memory");

@@ -664,3 +664,37 @@ def test_short_turn_projection_split_over_a_cluster(monkeypatch, px, M, d):
     assert (np.abs(a - b) <= 2.0 ** -7 * np.abs(b) + 2e-4).all()      # another summation order: one bf16 ulp, or fp32 noise near zero
     assert px.poll_status() == 0 and px2.poll_status() == 0
     px2.close()
+
+
+@pytest.mark.parametrize("M,d,hd,n_kv,r", [(1000, 512, 128, 2, 32), (2125, 1024, 64, 8, 16), (640, 256, 128, 1, 8)])
+def test_two_sm_projection_equals_the_one_block_kernel_bitwise(monkeypatch, px, M, d, hd, n_kv, r):
+    """The cta_group::2 form of the projection GEMM (two SMs per 256-row tile, each staging half of the weight tile;
+    opt-in) accumulates every output element over the same k steps in the same order as the one-block kernel: all
+    caches agree bit for bit - fused, LR-only with an agent mask, scattered slots, a ragged last tile, and the rotary
+    epilogue.  Run under a 20 ms wait limit so that a lost hand-off inside the pair would show as a timeout at once."""
+    from paper_2609_34054_b200.inputs import rope_table
+    geo = I.Geometry(d, 2 * n_kv, n_kv, hd, 3, r, r, alpha=2.0 * r)
+    H = I.hidden_states(M, geo, seed=97, tag=f"pair.{M}").cuda()
+    nb = (M + 15) // 16 + 3
+    slots = I.permutation(nb * 16, 97, f"pair.slots.{M}")[:M].to(torch.int32).cuda()
+    table = rope_table(M + 9, hd)
+    monkeypatch.setenv("PRECC_GEMM", "pair")
+    px2 = Precc(0)
+    px2.set_wait_limit(40_000_000)
+    out = []
+    for p in (px, px2):
+        L = Layer(p, geo, seed=97, n_blocks=nb, fill=float("nan"))
+        dev = {k: v.cuda() for k, v in L.w.items()}
+        WA = p.pack_turn_weights(geo, dev["W_k"], dev["W_v"], dev["A_k"], dev["A_v"])
+        p.turn_project(L.desc, H, WA, L.cache, 0, slots, 0b101)
+        Lr = Layer(p, geo, seed=97, n_blocks=nb, fill=float("nan"))
+        p.turn_project_rope(Lr.desc, H, WA, Lr.cache, table, 0, None, 0b011, start_pos=5)
+        Ll = Layer(p, geo, seed=97, n_blocks=nb, fill=float("nan"))
+        p.lr_precompute(Ll.desc, H, Ll.A_packed, Ll.cache, 16, None, 0b110)
+        torch.cuda.synchronize()
+        assert p.poll_status() == 0
+        out.append((L.cache, Lr.cache, Ll.cache))
+    for a, b in zip(out[0], out[1]):
+        for name in ("k_base", "v_base", "lr_k", "lr_v"):
+            assert torch.equal(getattr(a, name).view(torch.int16), getattr(b, name).view(torch.int16)), name
+    px2.close()
