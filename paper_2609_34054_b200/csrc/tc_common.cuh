@@ -59,11 +59,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  const long long limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
-  for (;;) {
+  long long limit = -1;                // fetched from global memory only once a whole batch of polls has failed:
+  for (;;) {                           // the common short wait must not pay a memory round trip before it polls
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
+    if (limit < 0) limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
     if (clock64() - t0 > limit) break;
     // once any wait in the grid has expired the results are void anyway: do not queue up more seconds
     if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
