@@ -164,6 +164,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
       int st2 = (ctx->max_smem_optin - 4096) / stage2;
       if (st2 > 8) st2 = 8;
       if (st2 > K / GEMM_BK) st2 = K / GEMM_BK;
+      if (ctx->gemm_stage_cap > 0 && st2 > ctx->gemm_stage_cap) st2 = ctx->gemm_stage_cap;
       if (st2 >= 2) {
         int tc2 = 32;
         while (tc2 < 2 * bn2) tc2 <<= 1;
@@ -200,6 +201,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   int stages = (ctx->max_smem_optin - 4096) / stage_bytes;
   if (stages > 8) stages = 8;
   if (stages > K / GEMM_BK) stages = K / GEMM_BK;
+  if (ctx->gemm_stage_cap > 0 && stages > ctx->gemm_stage_cap) stages = ctx->gemm_stage_cap;
   if (stages < 1) return fail(ctx, PRECC_ERR_CUDA, "not enough shared memory for one GEMM stage");
   int tmem_cols = 32;
   while (tmem_cols < 2 * bn) tmem_cols <<= 1;      // two accumulator buffers

@@ -24,6 +24,7 @@ struct precc_ctx {
   unsigned long long* trace = nullptr; // optional caller-owned trace buffer
   size_t trace_blocks = 0;
   bool force_simple_prefill = false;   // PRECC_PREFILL=simple in the environment
+  int gemm_stage_cap = 0;              // PRECC_GEMM_STAGES=n in the environment: ring depth of the tiled GEMMs at most n (experiments)
   bool gemm_pair = false;              // PRECC_GEMM=pair in the environment: two SMs per tile for projections of many rows
   bool force_tiled_gemm = false;       // PRECC_GEMM=tiled in the environment: never take the few-row kernel
   bool no_gemm_splitk = false;         // PRECC_GEMM_SPLITK=0 in the environment: short turns stay on the one-block-per-tile GEMM
