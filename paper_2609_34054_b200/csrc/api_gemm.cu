@@ -9,20 +9,20 @@ using namespace precc;
 
 namespace {
 
-// Column tile width.  A block's time per 64-deep k-block hardly depends on the width below 256 columns (the
-// thread that issues the MMAs needs about a hundred cycles per instruction, four per k-block: measured 0.52 us
-// per k-block at 256 columns, 0.45 at 128, 0.42 at 64 and still 0.40 at 16), so a launch costs about
-// rounds x that, rounds = ceil(tiles / SMs): the widest tile that does not add a round wins
-// (2048 rows x 2304 columns: 144 tiles of 256 in one round, 35 us, against 288 tiles of 128 in two, 55 us).
+// Column tile width.  A block's time per 64-deep k-block hardly depends on the width (measured 0.52 us per k-block
+// at 256 columns, 0.45 at 128, 0.42 at 64 and still 0.40 at 16: about 0.40 us + 0.47 ns per column), so a launch
+// costs about rounds x that, rounds = ceil(tiles / SMs): the widest tile that does not add a round wins
+// (2048 rows x 2304 columns: 144 tiles of 256 in one round, 35 us, against 288 tiles of 128 in two, 55 us), and a
+// width that divides the columns evenly beats one whose last tile is half empty (8192 x 1152: 384 tiles of 192
+// against 320 of 256, three rounds either way, the narrower ones cheaper).
 int pick_bn(int n_out, int m_tiles, int sm_count) {
   if (n_out <= 256) return (n_out + 15) / 16 * 16;
-  const int cands[3] = {256, 128, 64};
-  const double per_kblock[3] = {0.52, 0.45, 0.42};
+  const int cands[5] = {256, 192, 128, 96, 64};
   int best = 256;
   double best_cost = 1e30;
-  for (int i = 0; i < 3; ++i) {
+  for (int i = 0; i < 5; ++i) {
     const long long tiles = (long long)m_tiles * ((n_out + cands[i] - 1) / cands[i]);
-    const double cost = (double)((tiles + sm_count - 1) / sm_count) * per_kblock[i];
+    const double cost = (double)((tiles + sm_count - 1) / sm_count) * (0.40 + 0.00047 * cands[i]);
     if (cost < best_cost - 1e-9) { best_cost = cost; best = cands[i]; }
   }
   return best;
@@ -195,7 +195,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
     }
   }
   int bn = pick_bn(n_out, m_tiles, ctx->sm_count);
-  if (gp.rope && bn % gp.hd != 0) bn = gp.hd;        // a head's two halves must sit in one tile
+  if (gp.rope && bn % gp.hd != 0) bn = 256;          // a head's two halves must sit in one tile (head_dim 64 or 128 divides 256)
   const int n_tiles = (n_out + bn - 1) / bn;
   const int stage_bytes = GEMM_A_BYTES + bn * GEMM_BK * 2;
   int stages = (ctx->max_smem_optin - 4096) / stage_bytes;
