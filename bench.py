@@ -521,6 +521,54 @@ class Workload:
         self.step()
         self.out_host.copy_(self.out, non_blocking=True)
 
+    def run_host_pipelined(self, steps: int):
+        """`steps` steps whose inputs arrive from pinned host memory and whose outputs return to it, with the copies on
+        a second stream: the inputs of step i + 1 are uploaded (into the other of two device buffer sets) while step i
+        computes, and the outputs of step i go back while step i + 1 projects.  Every step still uploads all of its
+        inputs and downloads all of its outputs; only the first upload and the last download are not overlapped."""
+        torch = self.torch
+        cur = torch.cuda.current_stream()
+        if not hasattr(self, "_cs"):
+            self._cs = torch.cuda.Stream()
+            self._H2 = [self.H, [torch.empty_like(h) for h in self.H]]
+            self._q2 = [torch.empty_like(self.q), torch.empty_like(self.q)]
+        cs = self._cs
+        ready = [torch.cuda.Event(), torch.cuda.Event()]
+        done = [None, None]
+        d2h_done = None
+
+        def upload(slot):
+            with torch.cuda.stream(cs):
+                if done[slot] is not None:
+                    cs.wait_event(done[slot])           # the compute that last read this buffer set has finished
+                for l in range(self.layers):
+                    self._H2[slot][l].copy_(self.H_host[l], non_blocking=True)
+                self._q2[slot].copy_(self.q_host, non_blocking=True)
+                ready[slot].record(cs)
+
+        cs.wait_stream(cur)
+        upload(0)
+        for i in range(steps):
+            slot = i & 1
+            cur.wait_event(ready[slot])
+            if i + 1 < steps:
+                upload(slot ^ 1)
+            px = self.px
+            for l in range(self.layers):
+                px.turn_project(self.desc, self._H2[slot][l], self.WA_packed[l], self.cache[l], 0)
+            if d2h_done is not None:
+                cur.wait_event(d2h_done)                # the previous outputs have left `out`
+            self.q.copy_(self._q2[slot], non_blocking=True)   # the decode graph reads q at a fixed address
+            self.phase_b()
+            done[slot] = torch.cuda.Event()
+            done[slot].record(cur)
+            with torch.cuda.stream(cs):
+                cs.wait_event(done[slot])
+                self.out_host.copy_(self.out, non_blocking=True)
+                d2h_done = torch.cuda.Event()
+                d2h_done.record(cs)
+        cur.wait_stream(cs)
+
     def h2d_bytes(self):
         return sum(h.numel() * 2 for h in self.H_host) + self.q_host.numel() * 2
 
@@ -602,8 +650,17 @@ def run_gpu(args):
         sampler.start()
     ms, pa, pb = timed(wl.step, args.steps, args.warmup, phases=True)
     clocks = sampler.stop() if rank == 0 else None
-    ms_e2e, _, _ = timed(wl.step_host, max(1, min(args.steps, 3)), 1)
-    e2e_steps = max(1, min(args.steps, 3))
+    e2e_steps = max(1, min(args.steps, 4))
+    wl.step_host()                                                   # warm-up of the host path (pinned buffers touched)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    wl.run_host_pipelined(e2e_steps)
+    ev1.record()
+    barrier()
+    ms_e2e = reduce_max_ms(ev0.elapsed_time(ev1), "cuda")
+    if not torch.equal(wl.out_host, wl.out.cpu()):                   # the host path returns what the device holds
+        raise SystemExit("bench.py: the host-path outputs differ from the device-resident ones")
     status = px.poll_status()
     if status:
         raise SystemExit(f"bench.py: device status 0x{status:x}")
@@ -636,7 +693,9 @@ def run_gpu(args):
             },
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": wl.h2d_bytes(), "d2h_bytes_per_step": wl.d2h_bytes(),
-                    "ms_per_step": ms_e2e / e2e_steps},
+                    "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps,
+                    "how": "pinned host buffers -> device -> C-ABI calls -> pinned host; copies on a second stream, the next "
+                           "step's upload and the previous step's download overlap the compute"},
             "gpu_launches": (wl.launches_a + wl.launches_b) * args.steps,
             "roofline": {"bound": "hbm", "kernel": "lr_attend_decode_cluster_kernel<64,16,16,8>", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
