@@ -69,7 +69,10 @@ int32_t launch_small(precc_ctx* ctx, const void* X, int M, int K, const void* Wt
   return go(proj_small_kernel<4>);
 }
 
+int ilog2(int v) { int s = 0; while ((1 << s) < v) ++s; return s; }
+
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
+  gp.hd_shift = ilog2(gp.hd); gp.rk_shift = ilog2(gp.rank_k > 0 ? gp.rank_k : 1); gp.rv_shift = ilog2(gp.rank_v > 0 ? gp.rank_v : 1);
   // Up to 40 rows the weight-streaming few-row kernel is the fastest (fused C3 projection: 8.7 us at 16 rows, 11.6 at
   // 32); from there to 512 rows the split-K kernel (13..24 us; the few-row kernel needs 16.5 us at 48 rows and 18.4 at
   // 64, the one-block-per-tile GEMM 27 us throughout); the few-row kernel still takes 41..64 rows when the split does

@@ -38,7 +38,8 @@ __device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, 
     const bool is_v = gl >= n_k;
     const int rr = is_v ? p.rank_v : p.rank_k;
     const int cc = is_v ? gl - n_k : gl;
-    const int agent = cc / rr, ri = cc % rr;
+    const int sh = is_v ? p.rv_shift : p.rk_shift;
+    const int agent = cc >> sh, ri = cc & (rr - 1);
     if (!((mask >> agent) & 1ull)) return;
     dst = (is_v ? p.lr_v : p.lr_k) + (((long long)agent * p.n_blocks + blk) * PAGE + off) * rr + ri;
     if (p.lr_copy_slots) {
@@ -49,7 +50,7 @@ __device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, 
   } else {
     const bool is_v = gc >= w;
     const int cc = is_v ? gc - w : gc;
-    const int g = cc / p.hd, c = cc % p.hd;
+    const int g = cc >> p.hd_shift, c = cc & (p.hd - 1);
     dst = (is_v ? p.base_v : p.base_k) + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
   }
   uint4 v;
@@ -65,32 +66,47 @@ __device__ __forceinline__ void store_piece(const GemmParams& p, long long blk, 
 // the accumulator at `tmem_tile`, which holds rows m0 .. m0 + 127 and columns n0 .. n0 + BN - 1).  Waits for the
 // accumulator (bounded), converts to bf16 and routes 16-byte pieces to the paged caches; key columns of the rotary
 // variant are rotated by the row's position first.
+// The epilogue shares its SM's issue slots with the lanes that feed the tensor pipe, so it is kept lean: what depends
+// on the row (its slot -> element offsets into the base and LR arrays, its agent mask, its optional second LR
+// destination) is computed once per tile, what depends on the column (projection, head or agent, offset inside the
+// destination row) is the same for every lane and uses shifts (head_dim and the ranks are powers of two).
 __device__ __forceinline__ void gemm_epilogue_tile(const GemmParams& p, uint32_t tmem_tile, int m0, int n0, int lane_base, int lane,
                                                    uint32_t acc_full_bar, uint32_t parity) {
   const int row = lane_base + lane;
-  const int w = p.n_kv * p.hd;
+  const int hs = p.hd_shift;
+  const int w = p.n_kv << hs;
   const int gm = m0 + row;
   bool row_ok = gm < p.M;
   long long slot = 0;
   if (row_ok) {
     slot = p.slot_mapping ? (long long)p.slot_mapping[gm] : p.start_slot + gm;
-    if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
+    if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; slot = 0; }
   }
   const long long blk = slot / PAGE;
   const int off = (int)(slot % PAGE);
   const unsigned long long row_mask = (p.row_masks && row_ok) ? p.row_masks[gm] : p.agent_mask;
+  long long slot2 = -1;                               // second destination of this row's LR pieces, if any
+  if (p.lr_copy_slots && row_ok) {
+    slot2 = p.lr_copy_slots[gm];
+    if (slot2 >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); slot2 = -1; }
+  }
   long long pos = 0;
   if (p.rope && row_ok) {
     pos = p.positions ? (long long)p.positions[gm] : p.start_pos + gm;
     if (pos < 0 || pos >= p.max_pos) { atomicOr(p.status, StatusBits::BAD_INDEX); row_ok = false; }
   }
-  mbar_wait(acc_full_bar, parity, p.status);
+  // element offsets of this row inside the base arrays ([blk][g][off][c]: the head term is added per column) and
+  // inside one agent's LR arrays ([blk][off][r] = [slot][r])
+  const long long base_row = ((blk * p.n_kv * PAGE) + off) << hs;
+  const int n_k = p.n_agents << p.rk_shift;           // LR-K columns of the call (0 when rank_k == 0: n_agents << 0 is not used then)
+  const int n_lrk = p.rank_k > 0 ? n_k : 0;
+  mbar_wait_relaxed(acc_full_bar, parity, p.status);
   asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-  for (int c0 = 0; c0 < p.BN; c0 += 16) {
+  for (int c0 = 0; c0 < p.BN && n0 + c0 < p.N_out; c0 += 16) {
     if (p.rope && n0 + c0 < w) {
       // key columns: chunk [c, c+16) of the lower half of a head together with its partner chunk
       const int gc = n0 + c0;
-      const int g = gc / p.hd, c = gc % p.hd;
+      const int g = gc >> hs, c = gc & (p.hd - 1);
       if (c >= p.hd / 2) continue;                  // done with its partner
       uint32_t lo[16], hi[16];
       tmem_ld16(tmem_tile + (static_cast<uint32_t>(lane_base) << 16) + c0, lo);
@@ -107,7 +123,7 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmParams& p, uint32_t
         ol[k] = pack_bf16(l0 * t4.x - h0 * t4.y, l1 * t4.z - h1 * t4.w);
         oh[k] = pack_bf16(h0 * t4.x + l0 * t4.y, h1 * t4.z + l1 * t4.w);
       }
-      __nv_bfloat16* dst = p.base_k + ((blk * p.n_kv + g) * PAGE + off) * p.hd + c;
+      __nv_bfloat16* dst = p.base_k + base_row + ((long long)(g * PAGE) << hs) + c;
       reinterpret_cast<uint4*>(dst)[0] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
       reinterpret_cast<uint4*>(dst)[1] = make_uint4(ol[4], ol[5], ol[6], ol[7]);
       reinterpret_cast<uint4*>(dst + p.hd / 2)[0] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
@@ -117,14 +133,33 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmParams& p, uint32_t
     uint32_t r[16];
     tmem_ld16(tmem_tile + (static_cast<uint32_t>(lane_base) << 16) + c0, r);
     asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+    if (!row_ok) continue;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const int gc = n0 + c0 + 8 * h;
-      if (!row_ok || gc >= p.N_out) continue;
-      float v8[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(r[8 * h + k]);
-      store_piece(p, blk, off, gc, v8, row_mask, gm);
+      const int gc = n0 + c0 + 8 * h;               // the same for every lane: the routing below is warp-uniform
+      if (gc >= p.N_out) break;
+      uint4 v;
+      v.x = pack_bf16(__uint_as_float(r[8 * h + 0]), __uint_as_float(r[8 * h + 1]));
+      v.y = pack_bf16(__uint_as_float(r[8 * h + 2]), __uint_as_float(r[8 * h + 3]));
+      v.z = pack_bf16(__uint_as_float(r[8 * h + 4]), __uint_as_float(r[8 * h + 5]));
+      v.w = pack_bf16(__uint_as_float(r[8 * h + 6]), __uint_as_float(r[8 * h + 7]));
+      if (p.mode == 1 || (p.mode == 2 && gc < 2 * w)) {
+        const bool is_v = gc >= w;
+        const int cc = is_v ? gc - w : gc;
+        const int g = cc >> hs, c = cc & (p.hd - 1);
+        __nv_bfloat16* dst = (is_v ? p.base_v : p.base_k) + base_row + ((long long)(g * PAGE) << hs) + c;
+        *reinterpret_cast<uint4*>(dst) = v;
+      } else {
+        const int gl = p.mode == 2 ? gc - 2 * w : gc;
+        const bool is_v = gl >= n_lrk;
+        const int sh = is_v ? p.rv_shift : p.rk_shift;
+        const int cc = is_v ? gl - n_lrk : gl;
+        const int agent = cc >> sh, ri = cc & ((1 << sh) - 1);
+        if (!((row_mask >> agent) & 1ull)) continue;
+        __nv_bfloat16* arr = (is_v ? p.lr_v : p.lr_k) + (((long long)agent * p.n_blocks * PAGE) << sh) + ri;
+        *reinterpret_cast<uint4*>(arr + (slot << sh)) = v;
+        if (slot2 >= 0) *reinterpret_cast<uint4*>(arr + (slot2 << sh)) = v;
+      }
     }
   }
 }

@@ -24,6 +24,7 @@ struct GemmParams {
   const unsigned long long* row_masks;   // optional [M]: per-row agent masks (double batching), overrides agent_mask
   const int32_t* lr_copy_slots;          // optional [M]: a second slot that also receives the row's LR rows (< 0: none)
   int n_kv, hd;
+  int hd_shift, rk_shift, rv_shift;      // log2 of hd, rank_k, rank_v (all powers of two; 0 for an absent rank)
   // rotary keys (modes 1, 2; null = none): the key columns of a row are rotated by the row's position
   // before they are stored (rotate-half pairing (c, c + hd/2)); needs BN % hd == 0
   const float4* rope;             // [max_pos][hd/4] of (cos c, sin c, cos c+1, sin c+1), c even
@@ -67,6 +68,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
     if (limit < 0) limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
     if (clock64() - t0 > limit) break;
     // once any wait in the grid has expired the results are void anyway: do not queue up more seconds
+    if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
+  }
+  atomicOr(status, StatusBits::TIMEOUT);
+  return false;
+}
+
+// The same bounded wait for waiters that are not on the critical path (an epilogue waiting for a whole tile of
+// MMAs): it sleeps between polls, so that four warps of waiters do not compete with the issuing lanes for issue
+// slots - and for the power budget - while the tile is being computed.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  long long limit = -1;
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+      __nanosleep(200);
+      if (mbar_try_wait(bar, parity)) return true;
+    }
+    if (limit < 0) limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
+    if (clock64() - t0 > limit) break;
     if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
   }
   atomicOr(status, StatusBits::TIMEOUT);
