@@ -92,7 +92,8 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
     // 256-column tiles, one block per SM (a kernel that allocates tensor memory is given one block per SM)
     const int bn = n_out >= 256 ? 256 : (n_out + 15) / 16 * 16;
     const int stage_bytes = GEMM_A_BYTES + 256 * GEMM_BK * 2;
-    const int ring_max = 3 * stage_bytes;
+    constexpr int SK_STAGES = 4;                          // ring depth of the split-K kernel
+    const int ring_max = SK_STAGES * stage_bytes;
     const long long clusters = (long long)m_tiles * ((n_fused + 255) / 256);
     // the finest split whose clusters are all resident at once (a second wave would cost more than the split gains);
     // cluster sizes need not be powers of two: 18 clusters fit as 6-block clusters, 36 as 3-block clusters
@@ -105,7 +106,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
       if (nkb / ks < 2) continue;
       const int cw = ((256 + ks - 1) / ks + 7) / 8 * 8;          // planned for the widest tile, whatever this call's width
       const int dump = ks * GEMM_BM * (cw + 4) * 4;
-      smem_plan = (((ring_max > dump ? ring_max : dump) + 1023) & ~1023) + (2 * 3 + 4) * 8;
+      smem_plan = (((ring_max > dump ? ring_max : dump) + 1023) & ~1023) + (2 * SK_STAGES + 4) * 8;
       if (smem_plan > ctx->max_smem_optin) continue;
       static int max_clusters_dev[kMaxDevices][GEMM_MAX_KS + 1] = {{0}};   // 0 = unknown, else max active clusters + 1
       std::lock_guard<std::recursive_mutex> lk(lazy_mu());
@@ -129,7 +130,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
     }
     if (ks >= ks_min) {
       const int n_tiles = (n_out + bn - 1) / bn;
-      int stages = 3;
+      int stages = SK_STAGES;
       if (stages > nkb / ks) stages = nkb / ks;
       int tmem_cols = 32;
       while (tmem_cols < bn) tmem_cols <<= 1;
