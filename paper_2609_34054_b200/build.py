@@ -37,7 +37,8 @@ def _stale(src: str, hdr_time: float) -> bool:
 
 
 def _compile(nvcc: str, src: str, verbose: bool) -> str:
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas=-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", _obj(src)]
+    extra = os.environ.get("PRECC_NVCC_FLAGS", "").split()          # e.g. -DPRECC_PF_TRACE -DPRECC_GEMM_TRACE (timeline stamps)
+    cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas=-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", _obj(src)]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}{r.stderr}")

@@ -181,6 +181,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
         gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn2; gp.stages = st2; gp.tmem_cols = tc2;
         gp.spread_rows = 1;
         gp.status = ctx->status;
+        gp.trace = (ctx->trace && ctx->trace_blocks >= 128) ? ctx->trace : nullptr;     // used by PRECC_GEMM_TRACE builds only
         PRECC_CUDA(ctx, raise_smem_limit(ctx, proj_gemm_pair_kernel, (int)smem2));
         const long long tiles2 = (long long)((M + GEMM_PAIR_BM - 1) / GEMM_PAIR_BM) * ((n_out + bn2 - 1) / bn2);
         const int pairs = (int)(tiles2 < ctx->sm_count / 2 ? tiles2 : ctx->sm_count / 2);
@@ -218,6 +219,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
   gp.spread_rows = 1;
   gp.status = ctx->status;
+  gp.trace = (ctx->trace && ctx->trace_blocks >= 128) ? ctx->trace : nullptr;     // used by PRECC_GEMM_TRACE builds only
   PRECC_CUDA(ctx, raise_smem_limit(ctx, proj_gemm_kernel, (int)smem));
   const int total_tiles = m_tiles * n_tiles;
   proj_gemm_kernel<<<dim3(total_tiles < ctx->sm_count ? total_tiles : ctx->sm_count), GEMM_THREADS, smem, stream>>>(map_x, map_w, gp);

@@ -128,10 +128,12 @@ proj_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % p.stages;
           if (it >= p.stages) mbar_wait(empty0 + 8 * s, ((it / p.stages) - 1) & 1, p.status);
+          GEMM_STAMP(p, it, 0);
           const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
           if (rank == 0) mbar_expect_tx(full0 + 8 * s, 2 * stage_bytes);
           tma_pair_load_2d(sa, &map_x, kb * GEMM_BK, m0, full0_lead + 8 * s);
           tma_pair_load_3d(sa + GEMM_A_BYTES, &map_w, 0, n0, kb, full0_lead + 8 * s);      // packed weights are k-blocked
+          GEMM_STAMP(p, it, 1);
         }
       }
     }
@@ -149,12 +151,15 @@ proj_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % p.stages;
           mbar_wait(full0 + 8 * s, (it / p.stages) & 1, p.status);
+          GEMM_STAMP(p, it, 2);
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint64_t so = (uint64_t)((s * stage_bytes) >> 4);
 #pragma unroll
           for (int k = 0; k < GEMM_BK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
             umma_pair_bf16(d, da0 + so + 2 * k, db0 + so + 2 * k, idesc, (kb | k) ? 1u : 0u);
+          GEMM_STAMP(p, it, 3);
           umma_pair_commit_both(empty0 + 8 * s);   // the stage of both blocks is reusable once these MMAs have read it
+          GEMM_STAMP(p, it, 4);
         }
         umma_pair_commit_both(acc_full + 8 * buf); // accumulator of this tile complete in both blocks
       }

@@ -224,10 +224,12 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % p.stages;
           if (it >= p.stages) mbar_wait(empty0 + 8 * s, ((it / p.stages) - 1) & 1, p.status);
+          GEMM_STAMP(p, it, 0);
           const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
           mbar_expect_tx(full0 + 8 * s, stage_bytes);
           tma_load_2d(sa, &map_x, kb * GEMM_BK, m0, full0 + 8 * s);
           tma_load_3d(sa + GEMM_A_BYTES, &map_w, 0, n0, kb, full0 + 8 * s);      // packed weights are k-blocked
+          GEMM_STAMP(p, it, 1);
         }
       }
     }
@@ -245,12 +247,15 @@ proj_gemm_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % p.stages;
           mbar_wait(full0 + 8 * s, (it / p.stages) & 1, p.status);
+          GEMM_STAMP(p, it, 2);
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint64_t so = (uint64_t)((s * stage_bytes) >> 4);
 #pragma unroll
           for (int k = 0; k < GEMM_BK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
             umma_bf16(d, da0 + so + 2 * k, db0 + so + 2 * k, idesc, (kb | k) ? 1u : 0u);
+          GEMM_STAMP(p, it, 3);
           umma_commit(empty0 + 8 * s);             // stage reusable once these MMAs have read it
+          GEMM_STAMP(p, it, 4);
         }
         umma_commit(acc_full + 8 * buf);           // accumulator of this tile complete
       }

@@ -32,7 +32,20 @@ struct GemmParams {
   int64_t start_pos;
   int max_pos;
   uint32_t* status;
+  unsigned long long* trace;      // PRECC_GEMM_TRACE builds only: [k-blocks][8] clock stamps of block 0
 };
+
+// Timeline stamps of the persistent GEMM's block 0 for tuning (compiled in with -DPRECC_GEMM_TRACE): slot 0 the
+// producer sees the stage free, 1 its copies are issued, 2 the MMA lane sees the stage full, 3 its MMAs are issued,
+// 4 the commit is issued.
+#ifdef PRECC_GEMM_TRACE
+#define GEMM_STAMP(p, it, slot)                                                                   \
+  do {                                                                                            \
+    if ((p).trace && blockIdx.x == 0 && (it) < 256) (p).trace[(it) * 8 + (slot)] = clock64();     \
+  } while (0)
+#else
+#define GEMM_STAMP(p, it, slot) do { } while (0)
+#endif
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;                 // 64 bf16 = one 128-byte swizzle row
