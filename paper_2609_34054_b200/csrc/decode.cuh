@@ -276,11 +276,13 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
       a[1] = 0u; a[3] = 0u;
     }
   };
-  // Only warp 0 loads B_k and folds; the other warps pick the folded fragments up from shared memory
-  // (every warp needs the same ones, and the load/store unit is what limits the start of the stream).
+  // Small ranks: every warp holds the B_k fragments itself (requested here, before the wait for the preceding
+  // kernel) and folds on its own, so that nothing but the arrival of q stands between the wait and the first
+  // score MMA.  Large ranks: only warp 0 loads B_k (at the fold, the fragments do not fit in registers) and the
+  // other warps pick the folded fragments up from shared memory.
   uint32_t bk_pre[PRELOAD_BK ? KX * KC : 1][4];
   if constexpr (PRELOAD_BK) {
-    if (warp == 0 && use_lr) {
+    if (use_lr) {
 #pragma unroll
       for (int jt = 0; jt < KX; ++jt)
 #pragma unroll
@@ -315,6 +317,11 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     if (n_pre < my_n && tile0 + warp + NW * n_pre >= safe_tiles) break;
     issue_tile(n_pre);
   }
+  // q is the predecessor's to write, so it is read after the wait - but its lines can be brought into L2 now (L2 is
+  // the point of coherence: a later write by the predecessor lands there too), which turns the one load that stands
+  // between the wait and the first MMA from a DRAM round trip into an L2 hit
+  if (warp == 0 && lane * 128 < G * HD * 2)
+    asm volatile("prefetch.global.L2 [%0];\n" ::"l"(reinterpret_cast<const unsigned char*>(p.q + ((size_t)b * p.n_q + (size_t)g * G) * HD) + lane * 128));
   pdl_wait();                 // the predecessor has completed: its q, its cache rows and its workspace are visible
   pdl_launch_dependents();
   uint32_t qb[HD / 16][2];
@@ -341,7 +348,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     __shared__ uint32_t qx_share[KX > 0 ? KX : 1][2][32];
 #pragma unroll
     for (int jt = 0; jt < KX; ++jt) { qxb[jt][0] = 0u; qxb[jt][1] = 0u; }
-    if (warp == 0 && use_lr) {
+    if ((PRELOAD_BK || warp == 0) && use_lr) {
 #pragma unroll
       for (int jt = 0; jt < KX; ++jt) {
         float c[4] = {0.f, 0.f, 0.f, 0.f};
@@ -357,14 +364,18 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
         }
         qxb[jt][0] = movmatrix_t(pack_bf16(c[0] * p.s_k, c[1] * p.s_k));
         qxb[jt][1] = movmatrix_t(pack_bf16(c[2] * p.s_k, c[3] * p.s_k));
-        qx_share[jt][0][lane] = qxb[jt][0];
-        qx_share[jt][1][lane] = qxb[jt][1];
+        if constexpr (!PRELOAD_BK) {
+          qx_share[jt][0][lane] = qxb[jt][0];
+          qx_share[jt][1][lane] = qxb[jt][1];
+        }
       }
     }
-    __syncthreads();
-    if (warp != 0 && use_lr) {
+    if constexpr (!PRELOAD_BK) {
+      __syncthreads();
+      if (warp != 0 && use_lr) {
 #pragma unroll
-      for (int jt = 0; jt < KX; ++jt) { qxb[jt][0] = qx_share[jt][0][lane]; qxb[jt][1] = qx_share[jt][1][lane]; }
+        for (int jt = 0; jt < KX; ++jt) { qxb[jt][0] = qx_share[jt][0][lane]; qxb[jt][1] = qx_share[jt][1][lane]; }
+      }
     }
   }
 
