@@ -107,7 +107,9 @@ int32_t precc_sm_count(const precc_ctx* ctx);
  * while it is set, each thread block of precc_lr_attend_decode whose grid has at most n_blocks blocks
  * records the GPU nanosecond timer at points of its life at entry [block][point]: 0 start, 1 indices
  * read, 2 stream issued, 3 query fold ready, 4 first tile landed, 5 stream done, 6 record published,
- * 7 done, and for the merging block 8 partials gathered, 9 weights ready, 10 merged (others stay 0).  Pass NULL to switch tracing off (the default).  There is no paper counterpart. */
+ * 7 done, 11 all warps of the block have left the stream, and for the merging block 8 partials gathered, 9 weights
+ * ready, 10 merged (others stay 0); blocks of the cluster schedule also record 12 cluster barrier passed, and
+ * store the id of the SM they run on at entry 15.  Pass NULL to switch tracing off (the default).  There is no paper counterpart. */
 int32_t precc_set_trace_buffer(precc_ctx* ctx, void* buffer, size_t n_blocks);
 
 /* Read the device status word accumulated by kernels launched through `ctx`, then clear it.

@@ -111,6 +111,14 @@ struct DecodeTrace {
       buf[k] = t;
     }
   }
+  // slot 15: the SM the block runs on (placement of co-resident launches)
+  __device__ __forceinline__ void where() const {
+    if (buf && threadIdx.x == 0) {
+      unsigned int id;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(id));
+      buf[15] = id;
+    }
+  }
 };
 
 // Query fragments of one (b, g): B operand of the score MMA (k = head-dim coordinate, n = query head).
@@ -574,6 +582,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   //      instruction touches heads cq = 0, 2, 4, 6 (2 OWP = 8 mod 32 banks apart) at rows r = 0..7, i.e. 32 different
   //      banks, and the merging threads load consecutive columns: both free of bank conflicts
   __syncthreads();
+  mark(11);
   float* mg = reinterpret_cast<float*>(smem);
   constexpr int OWP = C::OWP;
   constexpr int WREC = C::WREC;
@@ -590,6 +599,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     }
   }
   __syncthreads();
+  mark(13);
   // every thread merges its own elements and derives the warp weights of its query row itself
   // (a few redundant shared-memory reads instead of a serial phase and a barrier); element
   // G*OW + h is the pair (m, l) of row h
@@ -614,6 +624,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     }
     acc[k] = v; acc_m[k] = M;
   }
+  mark(14);
   __syncthreads();   // all reads of the warp records are done; the region is reused for the result
 #pragma unroll
   for (int k = 0; k < PER_THREAD; ++k) {
@@ -849,6 +860,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   const int cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
   const DecodeTrace mark{p.trace ? p.trace + (size_t)cta_lin * 16 : nullptr};
   mark(0);
+  mark.where();
   const int ctx = __ldg(p.ctx_len + b);        // index arrays: read before the wait for the preceding kernel
   const int agent_raw = __ldg(p.agent_id + b);
   const bool use_lr = agent_raw >= 0;          // agent id -1: adapter-free view, base cache only
@@ -904,6 +916,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   }
   mark(6);
   cluster_wait();                                       // every block's result is complete and visible
+  mark(12);
   __shared__ float fin_m[8];
   // One pass over distributed shared memory: a thread owns one merged element (for every h < G my
   // `cols` base columns and all r_v LR-V coordinates, plus the denominators) and reads the peers'
