@@ -193,8 +193,9 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   }
   if (const char* v = getenv("PRECC_PREFILL")) ctx->force_simple_prefill = (strcmp(v, "simple") == 0);
   if (const char* v = getenv("PRECC_GEMM")) { ctx->force_tiled_gemm = (strcmp(v, "tiled") == 0); ctx->gemm_pair = (strcmp(v, "pair") == 0); }
-  if (const char* v = getenv("PRECC_DEEP")) ctx->deep_clusters = (strcmp(v, "0") != 0);
+  if (const char* v = getenv("PRECC_DEEP")) { ctx->deep_clusters = (strcmp(v, "0") != 0); ctx->deep_always = (strcmp(v, "2") == 0); }
   if (const char* v = getenv("PRECC_DECODE_CLUSTER")) ctx->decode_cluster_cap = atoi(v);
+  if (const char* v = getenv("PRECC_DECODE_STAGES")) ctx->decode_stage_cap = atoi(v);
   if (const char* v = getenv("PRECC_GEMM_STAGES")) ctx->gemm_stage_cap = atoi(v);
   if (const char* v = getenv("PRECC_GEMM_SPLITK")) ctx->no_gemm_splitk = (strcmp(v, "0") == 0);
   if (const char* v = getenv("PRECC_DECODE")) ctx->force_ticket_decode = (strcmp(v, "ticket") == 0);

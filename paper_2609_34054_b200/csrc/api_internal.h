@@ -30,6 +30,8 @@ struct precc_ctx {
   bool no_gemm_splitk = false;         // PRECC_GEMM_SPLITK=0 in the environment: short turns stay on the one-block-per-tile GEMM
   bool force_ticket_decode = false;    // PRECC_DECODE=ticket in the environment: never use the cluster decode kernel
   bool deep_clusters = true;           // PRECC_DEEP=0 in the environment: never use the one-block-per-SM deep-ring clusters
+  bool deep_always = false;            // PRECC_DEEP=2: take them wherever they fit, also where they leave many SMs without a block
+  int decode_stage_cap = 0;            // PRECC_DECODE_STAGES=n in the environment: at most n ring slots per warp in the cluster schedule (0 = planner's choice)
   int decode_cluster_cap = 0;          // PRECC_DECODE_CLUSTER=n in the environment: at most n blocks per decode cluster (0 = planner's choice)
   bool prefill_forward = false;        // PRECC_PREFILL_ORDER=forward: row tiles in ascending order (default: longest causal reach first)
   bool no_prefill_split = false;       // PRECC_PREFILL_SPLIT=0 in the environment: never split a turn's context over a cluster

@@ -77,6 +77,41 @@ __device__ __forceinline__ float fast_exp2(float x) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 
+// ---- mbarrier basics (shared-memory address of the barrier as a 32-bit value)
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  `status` points at the context's two device words: [0] the status bits, [1] the wait limit in
+// units of 1024 SM clock cycles (default: about a second).  Returns false after recording a timeout.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  long long limit = -1;                // fetched from global memory only once a whole batch of polls has failed:
+  for (;;) {                           // the common short wait must not pay a memory round trip before it polls
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (limit < 0) limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
+    if (clock64() - t0 > limit) break;
+    // once any wait in the grid has expired the results are void anyway: do not queue up more seconds
+    if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
+  }
+  atomicOr(status, StatusBits::TIMEOUT);
+  return false;
+}
+
 // XOR swizzle of 16-byte chunks inside a tile whose rows hold CPR chunks (CPR in {1,2,4,8,16}):
 // eight consecutive rows of the same logical chunk land in eight different 16-byte bank groups.
 template <int CPR>

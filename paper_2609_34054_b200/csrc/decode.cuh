@@ -93,13 +93,18 @@ struct DecodeCfg {
     int m = a > b ? a : b;
     return (m > c ? m : c) + 64;
   }
-  // cluster kernel tail: own result | merged slice + denominators | B_v column slice (at most hd/2 columns)
-  static constexpr int CL_TAIL_BYTES = PART_STRIDE * 4 + (8 * (HD + RV) + 8) * 4 + RV * HD;
-  __host__ __device__ static constexpr int cluster_smem(int warps, int stages) {
-    int a = ring_bytes(warps, stages), b = merge_bytes(warps);
-    int m = a > b ? a : b;
-    return (m > CL_TAIL_BYTES ? m : CL_TAIL_BYTES) + 64;
+  // Cluster kernel.  After the stream the ring region is reused as: warp records | B_v[a][:, g] slice ([RV][HD] bf16) |
+  // merged LR-V coordinates ([8][RV] floats).  Behind it sits the receive area that the peers fill with st.async:
+  // [CS sources][G heads][cols columns] merged values, then [CS][G] pairs (m, l), then the mbarrier that counts
+  // the bytes.  With cols = ceil(W / CS), W <= OW columns and G <= 8: CS G cols + 2 G CS + 1 <= 8 OW + 24 CS floats.
+  static constexpr int RECV_FLOATS = 8 * OW + 24 * DEC_MAX_CLUSTER;
+  static constexpr int RECV_BYTES = RECV_FLOATS * 4 + 16;
+  __host__ __device__ static constexpr int cluster_tail(int warps) { return merge_bytes(warps) + RV * HD * 2 + 8 * RV * 4; }
+  __host__ __device__ static constexpr int cluster_core(int warps, int stages) {   // offset of the receive area
+    int a = ring_bytes(warps, stages), b = cluster_tail(warps);
+    return ((a > b ? a : b) + 15) / 16 * 16;
   }
+  __host__ __device__ static constexpr int cluster_smem(int warps, int stages) { return cluster_core(warps, stages) + RECV_BYTES + 64; }
 };
 
 struct DecodeTrace {
@@ -142,8 +147,9 @@ __device__ __forceinline__ void load_q_frags(const DecodeParams& p, int b, int g
 // result in shared memory as floats  res = [ m[8] | l[8] | O'[G][OW] ]  at the start of `smem`
 // (m = running maximum in the log2 domain, l = softmax denominator, O' = unnormalised output with the
 // r_v LR-V coordinates appended).  Ends with a __syncthreads().  A block with no pages yields
-// m = NEG_BIG, l = 0, O' = 0.
-template <int HD, int RK, int RV, int NW, bool ROPE>
+// m = NEG_BIG, l = 0, O' = 0.  With MERGE = false it stops one step earlier: the warps' records
+// [warp][ m[8] | l[8] | O'[8][OWP] ] are written to the start of `smem`, no barrier follows.
+template <int HD, int RK, int RV, int NW, bool ROPE, bool MERGE = true>
 __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsigned char* smem, int b, int g, int ctx,
                                                     int agent, bool use_lr, int tile0, int tile_end, const DecodeTrace& mark) {
   static_assert(!ROPE || RK > 0, "the rotary variant only differs when there is a key-side adapter");
@@ -598,6 +604,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
       if (row + 8 < OW) { w0[row + 8] = o[mt][2]; w0[OWP + row + 8] = o[mt][3]; }
     }
   }
+  if constexpr (!MERGE) return;          // the caller merges the warp records itself (after a block barrier of its own)
   __syncthreads();
   mark(13);
   // every thread merges its own elements and derives the warp weights of its query row itself
@@ -830,19 +837,56 @@ lr_attend_decode_kernel(const DecodeParams p) {
 
 // ------------------------------------------------------------------------------------------------
 // Cluster kernel: grid (cluster size CS, kv head, request), cluster (CS,1,1), NW warps.
+//
+// Merge.  Block `o` finishes the output columns [o cols, o cols + ncol) of the (b, g) unit.  Every block
+// merges the records of its own warps, adds the value-side adapter term to its partial (the term is linear in
+// the partial: s_v U B_v of the merged sum equals the sum of the per-block terms), and SENDS each merged value
+// to the block that owns its column with st.async, which also counts the bytes on an mbarrier in the owner's
+// shared memory; (m, l) of every head go to every owner.  An owner waits for its byte count, then weighs and
+// adds the CS contributions in rank order and stores.  The only cluster-wide barrier is the one that makes the
+// mbarriers' initialisation visible: arrived at when the kernel starts, waited for before the first send, i.e.
+// long complete.  A block leaves once it has received everything addressed to it, so no send can reach the
+// shared memory of a block that is gone.
 __device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(local), "r"(rank));
   return r;
 }
-__device__ __forceinline__ float dsmem_ld(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];\n" : "=f"(v) : "r"(addr) : "memory");
-  return v;
+__device__ __forceinline__ void st_async_f32(uint32_t remote, float v, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];\n"
+               ::"r"(remote), "f"(v), "r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void st_async_f32x2(uint32_t remote, float a, float b, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];\n"
+               ::"r"(remote), "f"(a), "f"(b), "r"(remote_bar) : "memory");
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
-__device__ __forceinline__ void cluster_sync_all() { cluster_arrive(); cluster_wait(); }
+// Bounded wait for bytes sent by other blocks of the cluster (acquire at cluster scope); limit as in mbar_wait.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t* status) {
+  auto poll = [&]() -> bool {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+  };
+  if (poll()) return true;
+  const long long t0 = clock64();
+  long long limit = -1;
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (poll()) return true;
+    if (limit < 0) limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
+    if (clock64() - t0 > limit) break;
+    if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
+  }
+  atomicOr(status, StatusBits::TIMEOUT);
+  return false;
+}
 
 // MINB = 2 (8 warps, head_dim 64): 16-block clusters need two blocks per SM, which caps the kernel at 128
 // registers; the one-block-per-SM ring layout uses the MINB = 1 instance, free of that cap.
@@ -852,6 +896,8 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   using C = DecodeCfg<HD, RK, RV>;
   float* const raw_out = ROPE ? nullptr : p.raw;      // no rotary partial-output entry point: compiled out there
   constexpr int OW = C::OW;
+  constexpr int OWP = C::OWP;
+  constexpr int WREC = C::WREC;
   constexpr int NT = NW * 32;
   extern __shared__ __align__(128) unsigned char smem[];
   const int rank = blockIdx.x, CS = gridDim.x;          // the cluster spans grid.x
@@ -884,104 +930,152 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   const int tile0 = min(n_tiles, rank * p.chunk_tiles);
   const int tile_end = min(n_tiles, tile0 + p.chunk_tiles);
   mark(1);
-  // B_v column slice of this block: requested now (before the page stream), parked in registers
-  constexpr int BV_PER_THREAD = RV > 0 ? (RV * (HD / 2) + NT - 1) / NT : 1;
-  __nv_bfloat16 bv_pre[BV_PER_THREAD];
+  // Columns of the merged record that are divided over the blocks: the head dimension (the LR-V coordinates are
+  // spent inside each block), or the whole record in partial-output mode (no B_v there).
+  const int W = raw_out ? OW : HD;
+  const int cols = (W + CS - 1) / CS;                   // the cluster size need not divide W:
+  const int c0 = rank * cols;
+  const int ncol = max(0, min(cols, W - c0));           // the last blocks own fewer (or no) columns
+  float* recv = reinterpret_cast<float*>(smem + C::cluster_core(NW, p.stages));
+  const uint32_t recv_u32 = smem_u32(recv);
+  const uint32_t recv_bar = recv_u32 + C::RECV_FLOATS * 4;
+  const int ml_off = (CS * G * cols + 1) & ~1;          // floats; the (m, l) pairs are stored as 8-byte words
+  if (threadIdx.x == 0) {
+    mbar_init(recv_bar, 1);
+    if (ncol > 0) mbar_expect_tx(recv_bar, (uint32_t)(CS * G * (ncol + 2) * 4));   // the one arrival, and the bytes to come
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncwarp();
+  cluster_arrive();
+  // B_v[a][:, g] slice: requested now (before the page stream), parked in registers as bf16 pairs
+  constexpr int BVW = RV > 0 ? (RV * HD / 2 + NT - 1) / NT : 1;
+  uint32_t bv_pre[BVW];
+  const bool expand = RV > 0 && use_lr && !raw_out && p.B_v != nullptr;
   if constexpr (RV > 0) {
-    const int cols_ = (HD + CS - 1) / CS;                 // the cluster size need not divide the head dimension:
-    const int ncol_ = max(0, min(cols_, HD - rank * cols_));   // the last blocks own fewer (or no) columns
-    const __nv_bfloat16* Bv = p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD + rank * cols_;
+    const uint32_t* Bv = reinterpret_cast<const uint32_t*>(p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD);
 #pragma unroll
-    for (int k = 0; k < BV_PER_THREAD; ++k) {
+    for (int k = 0; k < BVW; ++k) {
       const int i = threadIdx.x + k * NT;
-      bv_pre[k] = (i < RV * cols_ && (i % cols_) < ncol_ && !raw_out) ? Bv[(size_t)(i / cols_) * p.n_kv * HD + (i % cols_)] : __float2bfloat16(0.f);   // partial-output mode has no B_v
+      bv_pre[k] = (expand && i < RV * HD / 2) ? __ldg(Bv + (size_t)(i / (HD / 2)) * (p.n_kv * (HD / 2)) + (i % (HD / 2))) : 0u;
     }
   }
   if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
-  decode_stream_block<HD, RK, RV, NW, ROPE>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, mark);
+  decode_stream_block<HD, RK, RV, NW, ROPE, false>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, mark);
 
-  // own result res = [m[8] | l[8] | O'[G][OW]] sits at the start of shared memory in every block
-  float* res = reinterpret_cast<float*>(smem);
-  float* mine = res + C::PART_STRIDE;                   // merged slice [G][cols + RV], then l[8]
-  __nv_bfloat16* bvs = reinterpret_cast<__nv_bfloat16*>(mine + 8 * (HD + RV) + 8);   // B_v[:, my columns], [RV][cols]
-  const int cols = (HD + CS - 1) / CS;                  // output columns finished by a block (stride of the slices)
-  const int c0 = rank * cols;
-  const int ncol = max(0, min(cols, HD - c0));          // columns this block really owns
-  cluster_arrive();                                     // this block's result is complete (the stream ends with a block barrier)
-  if constexpr (RV > 0) {                               // B_v column slice (bv_pre was requested before the stream)
-    for (int k = 0; k < BV_PER_THREAD; ++k) {
-      const int i = threadIdx.x + k * NT;
-      if (i < RV * cols) bvs[i] = bv_pre[k];
+  // ---- the warps' records are at the start of shared memory; behind them the B_v slice and the merged LR-V coordinates
+  float* mg = reinterpret_cast<float*>(smem);
+  uint32_t* bvs = reinterpret_cast<uint32_t*>(smem + C::merge_bytes(NW));           // [RV][HD / 2] bf16 pairs
+  float* lrm = reinterpret_cast<float*>(smem + C::merge_bytes(NW) + RV * HD * 2);   // [8][RV]
+  if constexpr (RV > 0) {
+    if (expand) {
+#pragma unroll
+      for (int k = 0; k < BVW; ++k) {
+        const int i = threadIdx.x + k * NT;
+        if (i < RV * HD / 2) bvs[i] = bv_pre[k];
+      }
+    }
+  }
+  __syncthreads();
+  mark(13);
+  // every thread merges its own elements and derives the warp weights of its query row itself; element
+  // G*OW + h is the pair (m, l) of row h
+  const int n_el = G * OW;
+  constexpr int PER_THREAD = (8 * OW + 8 + NT - 1) / NT;
+  float acc[PER_THREAD], acc_m[PER_THREAD];
+#pragma unroll
+  for (int k = 0; k < PER_THREAD; ++k) {
+    const int e = threadIdx.x + k * NT;
+    float v = 0.f, M = NEG_BIG;
+    if (e < n_el + G) {
+      const bool is_ml = e >= n_el;
+      const int h = is_ml ? e - n_el : e / OW;
+      const int src = is_ml ? 8 + h : 16 + h * OWP + (e % OW);
+      float mw[NW], xw[NW];
+#pragma unroll
+      for (int w = 0; w < NW; ++w) { mw[w] = mg[w * WREC + h]; xw[w] = mg[w * WREC + src]; }
+#pragma unroll
+      for (int w = 0; w < NW; ++w) M = fmaxf(M, mw[w]);
+#pragma unroll
+      for (int w = 0; w < NW; ++w) v += xw[w] * fast_exp2(mw[w] - M);   // warp order: deterministic
+      if constexpr (RV > 0) {
+        if (expand && !is_ml && (e % OW) >= HD) lrm[h * RV + (e % OW) - HD] = v;
+      }
+    }
+    acc[k] = v; acc_m[k] = M;
+  }
+  if constexpr (RV > 0) {
+    if (expand) __syncthreads();       // block-uniform: the merged LR-V coordinates are complete
+  }
+  mark(14);
+  cluster_wait();                      // the barrier arrived at when the kernel started: every peer's mbarrier is initialised
+#pragma unroll
+  for (int k = 0; k < PER_THREAD; ++k) {
+    const int e = threadIdx.x + k * NT;
+    if (e < n_el) {
+      const int h = e / OW, c = e % OW;
+      if (c < W) {
+        float v = acc[k];
+        if constexpr (RV > 0) {
+          if (expand) {                // value-side adapter term of this block's partial: s_v sum_j U[h][j] B_v[j][c]
+            const __nv_bfloat16* bcol = reinterpret_cast<const __nv_bfloat16*>(bvs) + c;
+            float u[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < RV; ++j) u[j & 3] += lrm[h * RV + j] * __bfloat162float(bcol[j * HD]);
+            v += p.s_v * ((u[0] + u[1]) + (u[2] + u[3]));
+          }
+        }
+        const int owner = c / cols;
+        st_async_f32(dsmem_addr(recv_u32 + (uint32_t)(((rank * G + h) * cols + (c - owner * cols)) * 4), owner), v,
+                     dsmem_addr(recv_bar, owner));
+      }
+    } else if (e < n_el + G) {
+      const int h = e - n_el;
+      const uint32_t dst = recv_u32 + (uint32_t)((ml_off + (rank * G + h) * 2) * 4);
+      for (int o = 0; o * cols < W; ++o)             // every block that owns columns needs every block's (m, l)
+        st_async_f32x2(dsmem_addr(dst, o), acc_m[k], acc[k], dsmem_addr(recv_bar, o));
     }
   }
   mark(6);
-  cluster_wait();                                       // every block's result is complete and visible
+  if (ncol == 0) { mark(7); return; }  // nothing is addressed to a block without columns
+  mbar_wait_cluster(recv_bar, 0, p.status);
   mark(12);
-  __shared__ float fin_m[8];
-  // One pass over distributed shared memory: a thread owns one merged element (for every h < G my
-  // `cols` base columns and all r_v LR-V coordinates, plus the denominators) and reads the peers'
-  // running maxima and values with all loads in flight at once; peers are added in rank order.
-  const uint32_t res_u32 = smem_u32(res);
-  const int sw = cols + RV;
-  for (int e = threadIdx.x; e < G * sw + G; e += NT) {
-    const bool is_l = e >= G * sw;
-    const int h = is_l ? e - G * sw : e / sw;
-    const int k = e % sw;
-    if (!is_l && k < cols && k >= ncol) { mine[e] = 0.f; continue; }   // slice padding past the head dimension
-    const int src = is_l ? 8 + h : 16 + h * OW + (k < cols ? c0 + k : HD + (k - cols));
-    float mr[DEC_MAX_CLUSTER], xr[DEC_MAX_CLUSTER];
+  const float* ml = recv + ml_off;
+  auto weigh = [&](int h, float (&wr)[DEC_MAX_CLUSTER], float& M, float& L) {
+    float mr[DEC_MAX_CLUSTER], lr[DEC_MAX_CLUSTER];
 #pragma unroll
     for (int r = 0; r < DEC_MAX_CLUSTER; ++r) {
-      if (r < CS) { mr[r] = dsmem_ld(dsmem_addr(res_u32 + h * 4, r)); xr[r] = dsmem_ld(dsmem_addr(res_u32 + src * 4, r)); }
-      else { mr[r] = NEG_BIG; xr[r] = 0.f; }
+      if (r < CS) { const float2 t = *reinterpret_cast<const float2*>(ml + (r * G + h) * 2); mr[r] = t.x; lr[r] = t.y; }
+      else { mr[r] = NEG_BIG; lr[r] = 0.f; }
     }
-    float M = NEG_BIG;
+    M = NEG_BIG;
 #pragma unroll
     for (int r = 0; r < DEC_MAX_CLUSTER; ++r) M = fmaxf(M, mr[r]);
+    L = 0.f;
+#pragma unroll
+    for (int r = 0; r < DEC_MAX_CLUSTER; ++r) { wr[r] = fast_exp2(mr[r] - M); L += lr[r] * wr[r]; }   // rank order: deterministic
+  };
+  float* rec = raw_out ? raw_out + ((size_t)b * p.n_kv + g) * C::PART_STRIDE : nullptr;
+  for (int e = threadIdx.x; e < G * ncol; e += NT) {
+    const int h = e / ncol, c = e % ncol;
+    float wr[DEC_MAX_CLUSTER], M, L;
+    weigh(h, wr, M, L);
     float v = 0.f;
 #pragma unroll
-    for (int r = 0; r < DEC_MAX_CLUSTER; ++r) v += xr[r] * fast_exp2(mr[r] - M);
-    mine[is_l ? 8 * (HD + RV) + h : e] = v;
-    if (is_l) fin_m[h] = M;
+    for (int r = 0; r < DEC_MAX_CLUSTER; ++r)
+      if (r < CS) v += recv[(r * G + h) * cols + c] * wr[r];
+    if (rec) rec[16 + h * OW + c0 + c] = v;            // partial-output mode: merged, un-normalised
+    else out_bg[h * HD + c0 + c] = __float2bfloat16(v / L);
   }
-  __syncthreads();
-  cluster_arrive();                                     // this block has finished reading its peers; the wait is at the exit
-  mark(10);
-  const float* fin_l = mine + 8 * (HD + RV);
-  if (raw_out) {
-    // partial-output mode: this block's column slice of the merged, un-normalised record; block 0 adds the
-    // LR-V coordinates, the denominators and the maxima
-    float* rec = raw_out + ((size_t)b * p.n_kv + g) * C::PART_STRIDE;
-    for (int e = threadIdx.x; e < G * cols; e += NT)
-      if ((e % cols) < ncol) rec[16 + (e / cols) * OW + c0 + (e % cols)] = mine[(e / cols) * sw + (e % cols)];
-    if (rank == 0) {
-      if constexpr (RV > 0) {
-        for (int e = threadIdx.x; e < G * RV; e += NT) rec[16 + (e / RV) * OW + HD + (e % RV)] = mine[(e / RV) * sw + cols + (e % RV)];
-      }
-      for (int e = G * OW + threadIdx.x; e < 8 * OW; e += NT) rec[16 + e] = 0.f;   // unused query-head slots: defined
-      if (threadIdx.x < 8) {
-        rec[threadIdx.x] = threadIdx.x < G ? fin_m[threadIdx.x] : NEG_BIG;
-        rec[8 + threadIdx.x] = threadIdx.x < G ? fin_l[threadIdx.x] : 0.f;
-      }
+  if (rec && rank == 0) {                               // block 0 adds the maxima, the denominators and the unused slots
+    for (int e = G * OW + threadIdx.x; e < 8 * OW; e += NT) rec[16 + e] = 0.f;
+    if (threadIdx.x < 8) {
+      float wr[DEC_MAX_CLUSTER], M = NEG_BIG, L = 0.f;
+      if (threadIdx.x < G) weigh(threadIdx.x, wr, M, L);
+      rec[threadIdx.x] = M;
+      rec[8 + threadIdx.x] = L;
     }
-    mark(7);
-    cluster_wait();                                     // nobody leaves while a peer may still read its result
-    return;
-  }
-  for (int e = threadIdx.x; e < G * cols; e += NT) {
-    const int h = e / cols, c = e % cols;
-    if (c >= ncol) continue;
-    float v = mine[h * sw + c];
-    if constexpr (RV > 0) {
-      float u[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int j = 0; j < RV; ++j) u[j & 3] += mine[h * sw + cols + j] * __bfloat162float(bvs[j * cols + c]);
-      v += p.s_v * ((u[0] + u[1]) + (u[2] + u[3]));
-    }
-    out_bg[h * HD + c0 + c] = __float2bfloat16(v / fin_l[h]);
   }
   mark(7);
-  cluster_wait();                                       // nobody leaves while a peer may still read its result
 }
 
 }  // namespace precc

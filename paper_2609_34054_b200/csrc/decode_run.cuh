@@ -38,6 +38,12 @@ DecodePlan plan_ticket(int sm_count, int max_smem, int B, int n_kv, int max_ctx,
   return pl;
 }
 
+// Warps of a cluster-schedule block when two blocks share an SM (8 if a two-page ring per warp fits, else 4).
+template <int HD, int RK, int RV>
+int two_per_sm_warps(int max_smem, int extra) {
+  return DecodeCfg<HD, RK, RV>::cluster_smem(8, 2) <= max_smem / 2 - 1024 - extra ? 8 : 4;
+}
+
 // The cluster kernel serves the latency-bound regime: few (request, kv head) units, each worth
 // splitting, the whole grid co-resident in one wave.  Returns cluster = 0 when it does not apply.
 template <int HD, int RK, int RV>
@@ -198,11 +204,25 @@ struct DecodeRunT {
       const int mt = (a.max_ctx + PAGE - 1) / PAGE;
       pl.cluster = ctx->decode_cluster_cap; pl.chunk_tiles = (mt + pl.cluster - 1) / pl.cluster; pl.max_splits = pl.cluster;
     }
+    if (pl.cluster > 1 && ctx->decode_stage_cap >= 2 && pl.stages > ctx->decode_stage_cap) {
+      pl.stages = ctx->decode_stage_cap;
+      pl.smem = DecodeCfg<HD, RK, RV>::cluster_smem(pl.warps, pl.stages) + extra;
+    }
     auto fits = [&](const DecodePlan& q) { return q.warps == 8 ? cluster_fits<8>(ctx, q, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, q, a.B * d->n_kv_heads); };
     if (pl.cluster && pl.deep) {
       const int max_tiles = (a.max_ctx + PAGE - 1) / PAGE;
       while (pl.cluster > 4 && !fits(pl)) { --pl.cluster; pl.chunk_tiles = (max_tiles + pl.cluster - 1) / pl.cluster; pl.max_splits = pl.cluster; }
       if (pl.cluster <= 4) pl.cluster = 0;
+      // One block per SM means at most one cluster of more than half a GPC per GPC: 8 units get 10-block clusters,
+      // 80 of 148 SMs.  Where two 8-warp blocks fit on an SM the two-blocks-per-SM layout (16-block clusters, or
+      // the ticket kernel for long contexts) reaches more SMs and is faster then (head_dim 64, one request:
+      // 8192 tokens 8.0 -> 7.1 us, 131072 tokens 60 -> 49 us); with 4-warp blocks (head_dim 128) the deep rings win.
+      if (!ctx->deep_always && pl.cluster * a.B * d->n_kv_heads * 4 < ctx->sm_count * 3 &&
+          two_per_sm_warps<HD, RK, RV>(ctx->max_smem_optin, extra) == 8) {
+        pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra, false);
+        if (ctx->force_ticket_decode) pl.cluster = 0;
+        if (pl.cluster && !fits(pl)) pl.cluster = 0;
+      }
     } else if (pl.cluster && !fits(pl)) {
       pl.cluster = 0;
     }
