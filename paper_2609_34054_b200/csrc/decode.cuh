@@ -947,16 +947,25 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   }
   __syncwarp();
   cluster_arrive();
-  // B_v[a][:, g] slice: requested now (before the page stream), parked in registers as bf16 pairs
-  constexpr int BVW = RV > 0 ? (RV * HD / 2 + NT - 1) / NT : 1;
-  uint32_t bv_pre[BVW];
+  // B_v[a][:, g] slice: requested now (before the page stream), parked in registers.  A unit is eight consecutive
+  // rank rows of one column (one 16-byte word of the layout [RV / 8][HD][8] that the adapter term reads below).
+  constexpr int BVU = RV > 0 ? ((RV / 8) * HD + NT - 1) / NT : 1;
+  uint4 bv_pre[BVU];
   const bool expand = RV > 0 && use_lr && !raw_out && p.B_v != nullptr;
   if constexpr (RV > 0) {
-    const uint32_t* Bv = reinterpret_cast<const uint32_t*>(p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD);
+    const unsigned short* Bv = reinterpret_cast<const unsigned short*>(p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD);
+    const size_t rs = (size_t)p.n_kv * HD;
 #pragma unroll
-    for (int k = 0; k < BVW; ++k) {
-      const int i = threadIdx.x + k * NT;
-      bv_pre[k] = (expand && i < RV * HD / 2) ? __ldg(Bv + (size_t)(i / (HD / 2)) * (p.n_kv * (HD / 2)) + (i % (HD / 2))) : 0u;
+    for (int k = 0; k < BVU; ++k) {
+      const int i = threadIdx.x + k * NT;                 // unit (q, c) = (i / HD, i % HD): rows 8q .. 8q+7 of column c
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      if (expand && i < (RV / 8) * HD) {
+        const unsigned short* src = Bv + (size_t)(i / HD) * 8 * rs + (i % HD);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          w[j] = (uint32_t)__ldg(src + (2 * j) * rs) | ((uint32_t)__ldg(src + (2 * j + 1) * rs) << 16);
+      }
+      bv_pre[k] = make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
   if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
@@ -964,14 +973,14 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
 
   // ---- the warps' records are at the start of shared memory; behind them the B_v slice and the merged LR-V coordinates
   float* mg = reinterpret_cast<float*>(smem);
-  uint32_t* bvs = reinterpret_cast<uint32_t*>(smem + C::merge_bytes(NW));           // [RV][HD / 2] bf16 pairs
+  uint4* bvs = reinterpret_cast<uint4*>(smem + C::merge_bytes(NW));                  // [RV / 8][HD] words of 8 bf16 (rank rows 8q .. 8q+7)
   float* lrm = reinterpret_cast<float*>(smem + C::merge_bytes(NW) + RV * HD * 2);   // [8][RV]
   if constexpr (RV > 0) {
     if (expand) {
 #pragma unroll
-      for (int k = 0; k < BVW; ++k) {
+      for (int k = 0; k < BVU; ++k) {
         const int i = threadIdx.x + k * NT;
-        if (i < RV * HD / 2) bvs[i] = bv_pre[k];
+        if (i < (RV / 8) * HD) bvs[i] = bv_pre[k];
       }
     }
   }
@@ -1017,10 +1026,21 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
         float v = acc[k];
         if constexpr (RV > 0) {
           if (expand) {                // value-side adapter term of this block's partial: s_v sum_j U[h][j] B_v[j][c]
-            const __nv_bfloat16* bcol = reinterpret_cast<const __nv_bfloat16*>(bvs) + c;
             float u[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int j = 0; j < RV; ++j) u[j & 3] += lrm[h * RV + j] * __bfloat162float(bcol[j * HD]);
+            for (int q = 0; q < RV / 8; ++q) {
+              const uint4 bw = bvs[q * HD + c];
+              const float4 ua = *reinterpret_cast<const float4*>(lrm + h * RV + q * 8);
+              const float4 ub = *reinterpret_cast<const float4*>(lrm + h * RV + q * 8 + 4);
+              u[0] += ua.x * __uint_as_float(bw.x << 16);
+              u[1] += ua.y * __uint_as_float(bw.x & 0xffff0000u);
+              u[2] += ua.z * __uint_as_float(bw.y << 16);
+              u[3] += ua.w * __uint_as_float(bw.y & 0xffff0000u);
+              u[0] += ub.x * __uint_as_float(bw.z << 16);
+              u[1] += ub.y * __uint_as_float(bw.z & 0xffff0000u);
+              u[2] += ub.z * __uint_as_float(bw.w << 16);
+              u[3] += ub.w * __uint_as_float(bw.w & 0xffff0000u);
+            }
             v += p.s_v * ((u[0] + u[1]) + (u[2] + u[3]));
           }
         }
@@ -1037,40 +1057,57 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   }
   mark(6);
   if (ncol == 0) { mark(7); return; }  // nothing is addressed to a block without columns
+  // Four lanes share an element (h, c) of this block's slice, lane `sub` taking the sources sub, sub + 4, sub + 8,
+  // sub + 12; the indices are worked out before the wait, so that loads, a short chain and two shuffle rounds are
+  // all that follows it.  The order of every sum is fixed: results do not depend on timing.
+  const float* ml = recv + ml_off;
+  const int sub = threadIdx.x & 3;
+  const int n_own = G * ncol;
+  int el = threadIdx.x >> 2;
+  int h = el / ncol, c = el - h * ncol;
   mbar_wait_cluster(recv_bar, 0, p.status);
   mark(12);
-  const float* ml = recv + ml_off;
-  auto weigh = [&](int h, float (&wr)[DEC_MAX_CLUSTER], float& M, float& L) {
-    float mr[DEC_MAX_CLUSTER], lr[DEC_MAX_CLUSTER];
-#pragma unroll
-    for (int r = 0; r < DEC_MAX_CLUSTER; ++r) {
-      if (r < CS) { const float2 t = *reinterpret_cast<const float2*>(ml + (r * G + h) * 2); mr[r] = t.x; lr[r] = t.y; }
-      else { mr[r] = NEG_BIG; lr[r] = 0.f; }
-    }
-    M = NEG_BIG;
-#pragma unroll
-    for (int r = 0; r < DEC_MAX_CLUSTER; ++r) M = fmaxf(M, mr[r]);
-    L = 0.f;
-#pragma unroll
-    for (int r = 0; r < DEC_MAX_CLUSTER; ++r) { wr[r] = fast_exp2(mr[r] - M); L += lr[r] * wr[r]; }   // rank order: deterministic
-  };
   float* rec = raw_out ? raw_out + ((size_t)b * p.n_kv + g) * C::PART_STRIDE : nullptr;
-  for (int e = threadIdx.x; e < G * ncol; e += NT) {
-    const int h = e / ncol, c = e % ncol;
-    float wr[DEC_MAX_CLUSTER], M, L;
-    weigh(h, wr, M, L);
-    float v = 0.f;
+  for (int base = 0; base < n_own; base += NT / 4) {
+    const bool live = el < n_own;
+    const int hh = live ? h : 0, cc = live ? c : 0;
+    float mr[4], lr[4], xr[4];
 #pragma unroll
-    for (int r = 0; r < DEC_MAX_CLUSTER; ++r)
-      if (r < CS) v += recv[(r * G + h) * cols + c] * wr[r];
-    if (rec) rec[16 + h * OW + c0 + c] = v;            // partial-output mode: merged, un-normalised
-    else out_bg[h * HD + c0 + c] = __float2bfloat16(v / L);
+    for (int i = 0; i < 4; ++i) {
+      const int r = sub + 4 * i;
+      if (r < CS) {
+        const float2 t = *reinterpret_cast<const float2*>(ml + (r * G + hh) * 2);
+        mr[i] = t.x; lr[i] = t.y; xr[i] = recv[(r * G + hh) * cols + cc];
+      } else {
+        mr[i] = NEG_BIG; lr[i] = 0.f; xr[i] = 0.f;
+      }
+    }
+    float M = fmaxf(fmaxf(mr[0], mr[1]), fmaxf(mr[2], mr[3]));
+    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));
+    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
+    float v = 0.f, L = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float w = fast_exp2(mr[i] - M); v += xr[i] * w; L += lr[i] * w; }
+    v += __shfl_xor_sync(0xffffffffu, v, 1); L += __shfl_xor_sync(0xffffffffu, L, 1);
+    v += __shfl_xor_sync(0xffffffffu, v, 2); L += __shfl_xor_sync(0xffffffffu, L, 2);
+    if (live && sub == 0) {
+      if (rec) rec[16 + hh * OW + c0 + cc] = v;          // partial-output mode: merged, un-normalised
+      else out_bg[hh * HD + c0 + cc] = __float2bfloat16(v / L);
+    }
+    el += NT / 4;
+    h = el / ncol; c = el - h * ncol;
   }
   if (rec && rank == 0) {                               // block 0 adds the maxima, the denominators and the unused slots
     for (int e = G * OW + threadIdx.x; e < 8 * OW; e += NT) rec[16 + e] = 0.f;
     if (threadIdx.x < 8) {
-      float wr[DEC_MAX_CLUSTER], M = NEG_BIG, L = 0.f;
-      if (threadIdx.x < G) weigh(threadIdx.x, wr, M, L);
+      float M = NEG_BIG, L = 0.f;
+      if (threadIdx.x < G) {
+        for (int r = 0; r < CS; ++r) M = fmaxf(M, ml[(r * G + threadIdx.x) * 2]);
+        // the same tree as above: sources r, r + 4, r + 8, r + 12 first, then pairs of those partial sums
+        float part[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int r = 0; r < CS; ++r) part[r & 3] += ml[(r * G + threadIdx.x) * 2 + 1] * fast_exp2(ml[(r * G + threadIdx.x) * 2] - M);
+        L = (part[0] + part[1]) + (part[2] + part[3]);
+      }
       rec[threadIdx.x] = M;
       rec[8 + threadIdx.x] = L;
     }
