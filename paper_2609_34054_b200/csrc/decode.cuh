@@ -93,18 +93,29 @@ struct DecodeCfg {
     int m = a > b ? a : b;
     return (m > c ? m : c) + 64;
   }
-  // Cluster kernel.  After the stream the ring region is reused as: warp records | B_v[a][:, g] slice ([RV][HD] bf16) |
-  // merged LR-V coordinates ([8][RV] floats).  Behind it sits the receive area that the peers fill with st.async:
-  // [CS sources][G heads][cols columns] merged values, then [CS][G] pairs (m, l), then the mbarrier that counts
-  // the bytes.  With cols = ceil(W / CS), W <= OW columns and G <= 8: CS G cols + 2 G CS + 1 <= 8 OW + 24 CS floats.
+  // Cluster kernel.  Behind the ring region sits the receive area that the peers fill with st.async:
+  // [CS sources][G heads][cols columns] merged values, then [CS][G] pairs (m, l), then two mbarriers (received
+  // bytes; arrival of the B_v slice).  With cols = ceil(W / CS), W <= OW columns and G <= 8:
+  // CS G cols + 2 G CS + 1 <= 8 OW + 24 CS floats.
   static constexpr int RECV_FLOATS = 8 * OW + 24 * DEC_MAX_CLUSTER;
   static constexpr int RECV_BYTES = RECV_FLOATS * 4 + 16;
-  __host__ __device__ static constexpr int cluster_tail(int warps) { return merge_bytes(warps) + RV * HD * 2 + 8 * RV * 4; }
+  // Value-side adapter term s_v U B_v.  WEXP: every warp adds it to its own partial on the tensor cores right
+  // after its last page (O^T += B_v^T (s_v U)^T: B_v[a][:, g] is staged like a value page of max(r_v, 16) "tokens"
+  // behind the receive area).  That takes r_v x hd x 2 bytes more per block; where two blocks of the smallest
+  // kind would no longer fit on an SM (head_dim 128 with rank 64) the term is added after the block merge
+  // instead, from a copy of B_v that is placed in the ring region once the stream is over.
+  static constexpr int BVP = RV > 16 ? RV : 16;
+  static constexpr bool WEXP = RV > 0 && ring_bytes(4, 2) + RECV_BYTES + 128 + BVP * HD * 2 + 64 <= 232448 / 2 - 1024;
+  static constexpr int BVS_BYTES = WEXP ? BVP * HD * 2 : 0;
+  __host__ __device__ static constexpr int cluster_tail(int warps) { return merge_bytes(warps) + (WEXP ? 0 : RV * HD * 2 + 8 * RV * 4); }
   __host__ __device__ static constexpr int cluster_core(int warps, int stages) {   // offset of the receive area
     int a = ring_bytes(warps, stages), b = cluster_tail(warps);
     return ((a > b ? a : b) + 15) / 16 * 16;
   }
-  __host__ __device__ static constexpr int cluster_smem(int warps, int stages) { return cluster_core(warps, stages) + RECV_BYTES + 64; }
+  __host__ __device__ static constexpr int cluster_bv(int warps, int stages) {     // offset of the staged B_v slice (WEXP)
+    return (cluster_core(warps, stages) + RECV_BYTES + 127) / 128 * 128;
+  }
+  __host__ __device__ static constexpr int cluster_smem(int warps, int stages) { return cluster_bv(warps, stages) + BVS_BYTES + 64; }
 };
 
 struct DecodeTrace {
@@ -149,9 +160,17 @@ __device__ __forceinline__ void load_q_frags(const DecodeParams& p, int b, int g
 // r_v LR-V coordinates appended).  Ends with a __syncthreads().  A block with no pages yields
 // m = NEG_BIG, l = 0, O' = 0.  With MERGE = false it stops one step earlier: the warps' records
 // [warp][ m[8] | l[8] | O'[8][OWP] ] are written to the start of `smem`, no barrier follows.
+// B_v slice staged in shared memory for the warps' own adapter term (cluster kernel): `bar` completes when
+// every thread's copies have landed.
+struct WarpExpand {
+  bool on;
+  uint32_t bv_u32, bar;
+};
+
 template <int HD, int RK, int RV, int NW, bool ROPE, bool MERGE = true>
 __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsigned char* smem, int b, int g, int ctx,
-                                                    int agent, bool use_lr, int tile0, int tile_end, const DecodeTrace& mark) {
+                                                    int agent, bool use_lr, int tile0, int tile_end, const DecodeTrace& mark,
+                                                    const WarpExpand wexp = WarpExpand{false, 0u, 0u}) {
   static_assert(!ROPE || RK > 0, "the rotary variant only differs when there is a key-side adapter");
   using C = DecodeCfg<HD, RK, RV>;
   constexpr int OW = C::OW;
@@ -326,17 +345,25 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   //      last DEC_PDL_TAIL tokens are requested while the preceding kernel may still be running; the wait
   //      for that kernel comes next, and the pages it may have appended to are requested after it.
   const int safe_tiles = max(0, ctx - DEC_PDL_TAIL) / PAGE;
-  int n_pre = 0;
-  for (; n_pre < p.stages; ++n_pre) {
-    if (n_pre < my_n && tile0 + warp + NW * n_pre >= safe_tiles) break;
-    issue_tile(n_pre);
-  }
+  // Cluster schedule: the last warp is the block's scout.  It requests only its first page before the wait, so
+  // that in a block that starts when its predecessor is already over - where filling the rings is throttled by
+  // the SM's limit on requests in flight and takes two DRAM round trips - the q lines are requested about one
+  // round trip earlier; the other warps' q loads then hit in L1.  A block that starts early has time to spare.
+  const bool scout = !MERGE && warp == NW - 1;
   // q is the predecessor's to write, so it is read after the wait - but its lines can be brought into L2 now (L2 is
   // the point of coherence: a later write by the predecessor lands there too), which turns the one load that stands
   // between the wait and the first MMA from a DRAM round trip into an L2 hit
-  if (warp == 0 && lane * 128 < G * HD * 2)
+  if (warp == NW - 1 && lane * 128 < G * HD * 2)
     asm volatile("prefetch.global.L2 [%0];\n" ::"l"(reinterpret_cast<const unsigned char*>(p.q + ((size_t)b * p.n_q + (size_t)g * G) * HD) + lane * 128));
+  const int pre_cap = scout ? 1 : p.stages;
+  int n_pre = 0;
+  for (; n_pre < pre_cap; ++n_pre) {
+    if (n_pre < my_n && tile0 + warp + NW * n_pre >= safe_tiles) break;
+    issue_tile(n_pre);
+  }
+  mark(8);
   pdl_wait();                 // the predecessor has completed: its q, its cache rows and its workspace are visible
+  mark(9);
   pdl_launch_dependents();
   uint32_t qb[HD / 16][2];
   load_q_frags<HD>(p, b, g, qb);
@@ -577,6 +604,28 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     issue_tile(i + p.stages);
   }
   cp_async_wait<0>();
+  if constexpr (!MERGE && C::WEXP) {
+    // value-side adapter term of this warp's partial, O^T += B_v^T (s_v U)^T: one more "value page" whose tokens
+    // are the rank coordinates; U (fp32 accumulators) enters as a bf16 pair hi + lo, i.e. with 16 mantissa bits
+    if (wexp.on) {
+      mbar_wait(wexp.bar, 0, p.status);
+#pragma unroll
+      for (int mx = 0; mx < MX; ++mx) {
+        const float u0 = o[MT + mx][0] * p.s_v, u1 = o[MT + mx][1] * p.s_v, u2 = o[MT + mx][2] * p.s_v, u3 = o[MT + mx][3] * p.s_v;
+        const uint32_t h01 = pack_bf16(u0, u1), h23 = pack_bf16(u2, u3);
+        const uint32_t l01 = pack_bf16(u0 - __uint_as_float(h01 << 16), u1 - __uint_as_float(h01 & 0xffff0000u));
+        const uint32_t l23 = pack_bf16(u2 - __uint_as_float(h23 << 16), u3 - __uint_as_float(h23 & 0xffff0000u));
+        const uint32_t bh0 = movmatrix_t(h01), bh1 = movmatrix_t(h23), bl0 = movmatrix_t(l01), bl1 = movmatrix_t(l23);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          uint32_t a[4];
+          ldsm_x4_t(a, wexp.bv_u32 + swz_off<CPR_KV>(16 * mx + v_row, 2 * mt + v_cpar));
+          mma_bf16_16816(o[mt], a, bh0, bh1);
+          mma_bf16_16816(o[mt], a, bl0, bl1);
+        }
+      }
+    }
+  }
 #pragma unroll
   for (int d = 4; d <= 16; d <<= 1) {
     l0 += __shfl_xor_sync(0xffffffffu, l0, d);
@@ -940,19 +989,34 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   const uint32_t recv_u32 = smem_u32(recv);
   const uint32_t recv_bar = recv_u32 + C::RECV_FLOATS * 4;
   const int ml_off = (CS * G * cols + 1) & ~1;          // floats; the (m, l) pairs are stored as 8-byte words
+  const uint32_t bv_bar = recv_bar + 8;
   if (threadIdx.x == 0) {
     mbar_init(recv_bar, 1);
+    if constexpr (C::WEXP) mbar_init(bv_bar, NT);         // every thread arrives once its copies of the B_v slice have landed
     if (ncol > 0) mbar_expect_tx(recv_bar, (uint32_t)(CS * G * (ncol + 2) * 4));   // the one arrival, and the bytes to come
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  __syncwarp();
+  if constexpr (C::WEXP) __syncthreads(); else __syncwarp();   // bv_bar is used by this block's own threads right below
   cluster_arrive();
-  // B_v[a][:, g] slice: requested now (before the page stream), parked in registers.  A unit is eight consecutive
-  // rank rows of one column (one 16-byte word of the layout [RV / 8][HD][8] that the adapter term reads below).
-  constexpr int BVU = RV > 0 ? ((RV / 8) * HD + NT - 1) / NT : 1;
-  uint4 bv_pre[BVU];
   const bool expand = RV > 0 && use_lr && !raw_out && p.B_v != nullptr;
-  if constexpr (RV > 0) {
+  // B_v[a][:, g] slice, requested now (before the page stream).  WEXP: copied to shared memory in the layout of a
+  // value page (rows = rank coordinates, padded with zero rows to 16); each thread's arrival on bv_bar fires when
+  // its copies have landed.  Otherwise: parked in registers, a unit being eight consecutive rank rows of one column
+  // (one 16-byte word of the layout [RV / 8][HD][8] that the adapter term reads below).
+  const uint32_t bv_u32 = smem_u32(smem + C::cluster_bv(NW, p.stages));
+  constexpr int BVU = (RV > 0 && !C::WEXP) ? ((RV / 8) * HD + NT - 1) / NT : 1;
+  uint4 bv_pre[BVU];
+  if constexpr (RV > 0 && C::WEXP) {
+    if (expand) {
+      constexpr int CPR = HD / 8;
+      const __nv_bfloat16* Bv = p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD;
+      for (int i = threadIdx.x; i < C::BVP * CPR; i += NT) {
+        const int j = i / CPR, ch = i % CPR;
+        cp_async16(bv_u32 + swz_off<CPR>(j, ch), Bv + (size_t)(j < RV ? j : 0) * p.n_kv * HD + ch * 8, j < RV ? 16 : 0);
+      }
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bv_bar) : "memory");
+    }
+  } else if constexpr (RV > 0) {
     const unsigned short* Bv = reinterpret_cast<const unsigned short*>(p.B_v + ((size_t)agent * RV) * ((size_t)p.n_kv * HD) + (size_t)g * HD);
     const size_t rs = (size_t)p.n_kv * HD;
 #pragma unroll
@@ -969,13 +1033,18 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     }
   }
   if (ROPE && ctx > p.max_pos && threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);   // positions are clamped
-  decode_stream_block<HD, RK, RV, NW, ROPE, false>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, mark);
+  decode_stream_block<HD, RK, RV, NW, ROPE, false>(p, smem, b, g, ctx, agent, use_lr, tile0, tile_end, mark,
+                                                   WarpExpand{C::WEXP && expand, bv_u32, bv_bar});
 
-  // ---- the warps' records are at the start of shared memory; behind them the B_v slice and the merged LR-V coordinates
+  // ---- the warps' records are at the start of shared memory.  WEXP: their first hd columns are final (the adapter
+  //      term is in), the LR-V columns matter in partial-output mode only.  Otherwise the B_v slice and the merged
+  //      LR-V coordinates are placed behind the records and the term is added after the block merge.
+  constexpr bool TAIL_EXPAND = RV > 0 && !C::WEXP;
+  const int Wm = (TAIL_EXPAND || raw_out) ? OW : HD;    // merged columns per head
   float* mg = reinterpret_cast<float*>(smem);
   uint4* bvs = reinterpret_cast<uint4*>(smem + C::merge_bytes(NW));                  // [RV / 8][HD] words of 8 bf16 (rank rows 8q .. 8q+7)
   float* lrm = reinterpret_cast<float*>(smem + C::merge_bytes(NW) + RV * HD * 2);   // [8][RV]
-  if constexpr (RV > 0) {
+  if constexpr (TAIL_EXPAND) {
     if (expand) {
 #pragma unroll
       for (int k = 0; k < BVU; ++k) {
@@ -987,8 +1056,11 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   __syncthreads();
   mark(13);
   // every thread merges its own elements and derives the warp weights of its query row itself; element
-  // G*OW + h is the pair (m, l) of row h
-  const int n_el = G * OW;
+  // G*Wm + h is the pair (m, l) of row h
+  const int n_el = G * Wm;
+  auto head_col = [&](int e, int& h, int& c) {           // constant divisors
+    if (Wm == HD) { h = e / HD; c = e % HD; } else { h = e / OW; c = e % OW; }
+  };
   constexpr int PER_THREAD = (8 * OW + 8 + NT - 1) / NT;
   float acc[PER_THREAD], acc_m[PER_THREAD];
 #pragma unroll
@@ -997,8 +1069,10 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     float v = 0.f, M = NEG_BIG;
     if (e < n_el + G) {
       const bool is_ml = e >= n_el;
-      const int h = is_ml ? e - n_el : e / OW;
-      const int src = is_ml ? 8 + h : 16 + h * OWP + (e % OW);
+      int h, c;
+      head_col(e, h, c);
+      if (is_ml) h = e - n_el;
+      const int src = is_ml ? 8 + h : 16 + h * OWP + c;
       float mw[NW], xw[NW];
 #pragma unroll
       for (int w = 0; w < NW; ++w) { mw[w] = mg[w * WREC + h]; xw[w] = mg[w * WREC + src]; }
@@ -1006,13 +1080,13 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
       for (int w = 0; w < NW; ++w) M = fmaxf(M, mw[w]);
 #pragma unroll
       for (int w = 0; w < NW; ++w) v += xw[w] * fast_exp2(mw[w] - M);   // warp order: deterministic
-      if constexpr (RV > 0) {
-        if (expand && !is_ml && (e % OW) >= HD) lrm[h * RV + (e % OW) - HD] = v;
+      if constexpr (TAIL_EXPAND) {
+        if (expand && !is_ml && c >= HD) lrm[h * RV + c - HD] = v;
       }
     }
     acc[k] = v; acc_m[k] = M;
   }
-  if constexpr (RV > 0) {
+  if constexpr (TAIL_EXPAND) {
     if (expand) __syncthreads();       // block-uniform: the merged LR-V coordinates are complete
   }
   mark(14);
@@ -1021,10 +1095,11 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   for (int k = 0; k < PER_THREAD; ++k) {
     const int e = threadIdx.x + k * NT;
     if (e < n_el) {
-      const int h = e / OW, c = e % OW;
+      int h, c;
+      head_col(e, h, c);
       if (c < W) {
         float v = acc[k];
-        if constexpr (RV > 0) {
+        if constexpr (TAIL_EXPAND) {
           if (expand) {                // value-side adapter term of this block's partial: s_v sum_j U[h][j] B_v[j][c]
             float u[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll

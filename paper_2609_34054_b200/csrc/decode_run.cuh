@@ -198,16 +198,21 @@ struct DecodeRunT {
     // The rotary kernel at head_dim 128 is issue-bound (255 registers, 8 warps per SM at most): it gains more from
     // the 128 blocks of the two-blocks-per-SM layout than from deeper rings on 80 SMs (131072 tokens: 141 against 238 us).
     const bool deep_ok = ctx->deep_clusters && !(ROPE && HD == 128);
-    DecodePlan pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra, deep_ok);
-    if (ctx->force_ticket_decode) pl.cluster = 0;
-    if (pl.cluster > 1 && ctx->decode_cluster_cap > 1 && pl.cluster > ctx->decode_cluster_cap) {
-      const int mt = (a.max_ctx + PAGE - 1) / PAGE;
-      pl.cluster = ctx->decode_cluster_cap; pl.chunk_tiles = (mt + pl.cluster - 1) / pl.cluster; pl.max_splits = pl.cluster;
-    }
-    if (pl.cluster > 1 && ctx->decode_stage_cap >= 2 && pl.stages > ctx->decode_stage_cap) {
-      pl.stages = ctx->decode_stage_cap;
-      pl.smem = DecodeCfg<HD, RK, RV>::cluster_smem(pl.warps, pl.stages) + extra;
-    }
+    // planner's choice, then the experiment switches of the environment
+    auto plan = [&](bool deep) {
+      DecodePlan q = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra, deep);
+      if (ctx->force_ticket_decode) q.cluster = 0;
+      if (q.cluster > 1 && ctx->decode_cluster_cap > 1 && q.cluster > ctx->decode_cluster_cap) {
+        const int mt = (a.max_ctx + PAGE - 1) / PAGE;
+        q.cluster = ctx->decode_cluster_cap; q.chunk_tiles = (mt + q.cluster - 1) / q.cluster; q.max_splits = q.cluster;
+      }
+      if (q.cluster > 1 && ctx->decode_stage_cap >= 2 && q.stages > ctx->decode_stage_cap) {
+        q.stages = ctx->decode_stage_cap;
+        q.smem = DecodeCfg<HD, RK, RV>::cluster_smem(q.warps, q.stages) + extra;
+      }
+      return q;
+    };
+    DecodePlan pl = plan(deep_ok);
     auto fits = [&](const DecodePlan& q) { return q.warps == 8 ? cluster_fits<8>(ctx, q, a.B * d->n_kv_heads) : cluster_fits<4>(ctx, q, a.B * d->n_kv_heads); };
     if (pl.cluster && pl.deep) {
       const int max_tiles = (a.max_ctx + PAGE - 1) / PAGE;
@@ -219,8 +224,7 @@ struct DecodeRunT {
       // 8192 tokens 8.0 -> 7.1 us, 131072 tokens 60 -> 49 us); with 4-warp blocks (head_dim 128) the deep rings win.
       if (!ctx->deep_always && pl.cluster * a.B * d->n_kv_heads * 4 < ctx->sm_count * 3 &&
           two_per_sm_warps<HD, RK, RV>(ctx->max_smem_optin, extra) == 8) {
-        pl = plan_cluster<HD, RK, RV>(ctx->sm_count, ctx->max_smem_optin, a.B, d->n_kv_heads, a.max_ctx, extra, false);
-        if (ctx->force_ticket_decode) pl.cluster = 0;
+        pl = plan(false);
         if (pl.cluster && !fits(pl)) pl.cluster = 0;
       }
     } else if (pl.cluster && !fits(pl)) {
