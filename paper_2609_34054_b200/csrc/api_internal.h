@@ -31,6 +31,7 @@ struct precc_ctx {
   bool force_ticket_decode = false;    // PRECC_DECODE=ticket in the environment: never use the cluster decode kernel
   bool deep_clusters = true;           // PRECC_DEEP=0 in the environment: never use the one-block-per-SM deep-ring clusters
   bool deep_always = false;            // PRECC_DEEP=2: take them wherever they fit, also where they leave many SMs without a block
+  int decode_pre_stages = 0;           // PRECC_DECODE_PRE=n in the environment: ring slots filled before the dependency wait (0 = all)
   int decode_stage_cap = 0;            // PRECC_DECODE_STAGES=n in the environment: at most n ring slots per warp in the cluster schedule (0 = planner's choice)
   int decode_cluster_cap = 0;          // PRECC_DECODE_CLUSTER=n in the environment: at most n blocks per decode cluster (0 = planner's choice)
   bool prefill_forward = false;        // PRECC_PREFILL_ORDER=forward: row tiles in ascending order (default: longest causal reach first)

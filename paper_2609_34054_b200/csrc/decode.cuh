@@ -59,6 +59,7 @@ struct DecodeParams {
   int table_stride;
   int n_q, n_kv, group, n_agents;
   int chunk_tiles, max_splits, stages;
+  int pre_stages;              // ring slots a warp fills before it waits for the preceding kernel (the rest follow the wait)
   int max_ctx;                 // the host's bound on ctx_len[b]: it sized the grid, the split and the block table
   float scale_log2, s_k, s_v;
 };
@@ -355,7 +356,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
   // between the wait and the first MMA from a DRAM round trip into an L2 hit
   if (warp == NW - 1 && lane * 128 < G * HD * 2)
     asm volatile("prefetch.global.L2 [%0];\n" ::"l"(reinterpret_cast<const unsigned char*>(p.q + ((size_t)b * p.n_q + (size_t)g * G) * HD) + lane * 128));
-  const int pre_cap = scout ? 1 : p.stages;
+  const int pre_cap = scout ? 1 : p.pre_stages;
   int n_pre = 0;
   for (; n_pre < pre_cap; ++n_pre) {
     if (n_pre < my_n && tile0 + warp + NW * n_pre >= safe_tiles) break;
@@ -909,7 +910,7 @@ __device__ __forceinline__ void st_async_f32x2(uint32_t remote, float a, float b
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];\n"
                ::"r"(remote), "f"(a), "f"(b), "r"(remote_bar) : "memory");
 }
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
 // Bounded wait for bytes sent by other blocks of the cluster (acquire at cluster scope); limit as in mbar_wait.
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t* status) {
@@ -997,7 +998,10 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if constexpr (C::WEXP) __syncthreads(); else __syncwarp();   // bv_bar is used by this block's own threads right below
-  cluster_arrive();
+  cluster_arrive_relaxed();            // the fence above orders the initialisation; nothing else is published here
+  // divisions by the run-time cluster size and slice width, as multiplications (exact for numerators below 1024)
+  const uint32_t inv_cols = (65536u + (uint32_t)cols - 1u) / (uint32_t)cols;
+  const uint32_t inv_cs = (65536u + (uint32_t)CS - 1u) / (uint32_t)CS;
   const bool expand = RV > 0 && use_lr && !raw_out && p.B_v != nullptr;
   // B_v[a][:, g] slice, requested now (before the page stream).  WEXP: copied to shared memory in the layout of a
   // value page (rows = rank coordinates, padded with zero rows to 16); each thread's arrival on bv_bar fires when
@@ -1061,17 +1065,18 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   auto head_col = [&](int e, int& h, int& c) {           // constant divisors
     if (Wm == HD) { h = e / HD; c = e % HD; } else { h = e / OW; c = e % OW; }
   };
-  constexpr int PER_THREAD = (8 * OW + 8 + NT - 1) / NT;
+  // elements n_el + h CS + o: the pair (m, l) of row h, merged once per receiving block o (one send each)
+  constexpr int PER_THREAD = (8 * OW + 8 * DEC_MAX_CLUSTER + NT - 1) / NT;
   float acc[PER_THREAD], acc_m[PER_THREAD];
 #pragma unroll
   for (int k = 0; k < PER_THREAD; ++k) {
     const int e = threadIdx.x + k * NT;
     float v = 0.f, M = NEG_BIG;
-    if (e < n_el + G) {
+    if (e < n_el + G * CS) {
       const bool is_ml = e >= n_el;
       int h, c;
       head_col(e, h, c);
-      if (is_ml) h = e - n_el;
+      if (is_ml) h = (int)(((uint32_t)(e - n_el) * inv_cs) >> 16);
       const int src = is_ml ? 8 + h : 16 + h * OWP + c;
       float mw[NW], xw[NW];
 #pragma unroll
@@ -1119,15 +1124,15 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
             v += p.s_v * ((u[0] + u[1]) + (u[2] + u[3]));
           }
         }
-        const int owner = c / cols;
+        const int owner = (int)(((uint32_t)c * inv_cols) >> 16);
         st_async_f32(dsmem_addr(recv_u32 + (uint32_t)(((rank * G + h) * cols + (c - owner * cols)) * 4), owner), v,
                      dsmem_addr(recv_bar, owner));
       }
-    } else if (e < n_el + G) {
-      const int h = e - n_el;
-      const uint32_t dst = recv_u32 + (uint32_t)((ml_off + (rank * G + h) * 2) * 4);
-      for (int o = 0; o * cols < W; ++o)             // every block that owns columns needs every block's (m, l)
-        st_async_f32x2(dsmem_addr(dst, o), acc_m[k], acc[k], dsmem_addr(recv_bar, o));
+    } else if (e < n_el + G * CS) {
+      const int h = (int)(((uint32_t)(e - n_el) * inv_cs) >> 16), o = e - n_el - h * CS;
+      if (o * cols < W)                              // every block that owns columns needs every block's (m, l)
+        st_async_f32x2(dsmem_addr(recv_u32 + (uint32_t)((ml_off + (rank * G + h) * 2) * 4), o), acc_m[k], acc[k],
+                       dsmem_addr(recv_bar, o));
     }
   }
   mark(6);

@@ -250,6 +250,7 @@ struct DecodeRunT {
     p.n_blocks = a.cache->n_blocks; p.table_stride = a.table_stride;
     p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = d->n_q_heads / d->n_kv_heads; p.n_agents = d->n_agents;
     p.chunk_tiles = pl.chunk_tiles; p.max_splits = pl.max_splits; p.stages = pl.stages; p.max_ctx = a.max_ctx;
+    p.pre_stages = (ctx->decode_pre_stages >= 1 && ctx->decode_pre_stages < pl.stages) ? ctx->decode_pre_stages : pl.stages;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
     p.rope = reinterpret_cast<const float4*>(a.rope); p.max_pos = a.max_pos;
     p.bk_off = ROPE ? ((pl.smem - extra + 127) / 128) * 128 : 0;
