@@ -649,6 +649,7 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     float* w0 = w + 16 + cq * OWP;         // query head cq, cq + 1
 #pragma unroll
     for (int mt = 0; mt < MT + MX; ++mt) {
+      if (!MERGE && C::WEXP && mt >= MT && wexp.on) break;      // the LR-V coordinates are spent: nobody reads them
       const int row = mt * 16 + r;
       if (row < OW) { w0[row] = o[mt][0]; w0[OWP + row] = o[mt][1]; }
       if (row + 8 < OW) { w0[row + 8] = o[mt][2]; w0[OWP + row + 8] = o[mt][3]; }
@@ -999,9 +1000,8 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   }
   if constexpr (C::WEXP) __syncthreads(); else __syncwarp();   // bv_bar is used by this block's own threads right below
   cluster_arrive_relaxed();            // the fence above orders the initialisation; nothing else is published here
-  // divisions by the run-time cluster size and slice width, as multiplications (exact for numerators below 1024)
+  // division by the run-time slice width, as a multiplication (exact for numerators below 1024)
   const uint32_t inv_cols = (65536u + (uint32_t)cols - 1u) / (uint32_t)cols;
-  const uint32_t inv_cs = (65536u + (uint32_t)CS - 1u) / (uint32_t)CS;
   const bool expand = RV > 0 && use_lr && !raw_out && p.B_v != nullptr;
   // B_v[a][:, g] slice, requested now (before the page stream).  WEXP: copied to shared memory in the layout of a
   // value page (rows = rank coordinates, padded with zero rows to 16); each thread's arrival on bv_bar fires when
@@ -1065,31 +1065,36 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
   auto head_col = [&](int e, int& h, int& c) {           // constant divisors
     if (Wm == HD) { h = e / HD; c = e % HD; } else { h = e / OW; c = e % OW; }
   };
-  // elements n_el + h CS + o: the pair (m, l) of row h, merged once per receiving block o (one send each)
-  constexpr int PER_THREAD = (8 * OW + 8 * DEC_MAX_CLUSTER + NT - 1) / NT;
-  float acc[PER_THREAD], acc_m[PER_THREAD];
+  // The thread of element (h, c) with c < CS also merges the denominator of row h - its weights are at hand - and
+  // will send the pair (m, l) to block c (head_dim >= 64 > CS: such a thread exists for every receiving block).
+  constexpr int PER_THREAD = (8 * OW + NT - 1) / NT;
+  float acc[PER_THREAD], acc_m[PER_THREAD], acc_l[PER_THREAD];
 #pragma unroll
   for (int k = 0; k < PER_THREAD; ++k) {
     const int e = threadIdx.x + k * NT;
-    float v = 0.f, M = NEG_BIG;
-    if (e < n_el + G * CS) {
-      const bool is_ml = e >= n_el;
+    float v = 0.f, M = NEG_BIG, L = 0.f;
+    if (e < n_el) {
       int h, c;
       head_col(e, h, c);
-      if (is_ml) h = (int)(((uint32_t)(e - n_el) * inv_cs) >> 16);
-      const int src = is_ml ? 8 + h : 16 + h * OWP + c;
+      const int src = 16 + h * OWP + c;
       float mw[NW], xw[NW];
 #pragma unroll
       for (int w = 0; w < NW; ++w) { mw[w] = mg[w * WREC + h]; xw[w] = mg[w * WREC + src]; }
 #pragma unroll
       for (int w = 0; w < NW; ++w) M = fmaxf(M, mw[w]);
 #pragma unroll
-      for (int w = 0; w < NW; ++w) v += xw[w] * fast_exp2(mw[w] - M);   // warp order: deterministic
+      for (int w = 0; w < NW; ++w) mw[w] = fast_exp2(mw[w] - M);
+#pragma unroll
+      for (int w = 0; w < NW; ++w) v += xw[w] * mw[w];                  // warp order: deterministic
+      if (c < CS) {
+#pragma unroll
+        for (int w = 0; w < NW; ++w) L += mg[w * WREC + 8 + h] * mw[w];
+      }
       if constexpr (TAIL_EXPAND) {
-        if (expand && !is_ml && c >= HD) lrm[h * RV + c - HD] = v;
+        if (expand && c >= HD) lrm[h * RV + c - HD] = v;
       }
     }
-    acc[k] = v; acc_m[k] = M;
+    acc[k] = v; acc_m[k] = M; acc_l[k] = L;
   }
   if constexpr (TAIL_EXPAND) {
     if (expand) __syncthreads();       // block-uniform: the merged LR-V coordinates are complete
@@ -1102,6 +1107,9 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     if (e < n_el) {
       int h, c;
       head_col(e, h, c);
+      if (c < CS && c * cols < W)                    // every block that owns columns needs every block's (m, l)
+        st_async_f32x2(dsmem_addr(recv_u32 + (uint32_t)((ml_off + (rank * G + h) * 2) * 4), c), acc_m[k], acc_l[k],
+                       dsmem_addr(recv_bar, c));
       if (c < W) {
         float v = acc[k];
         if constexpr (TAIL_EXPAND) {
@@ -1128,11 +1136,6 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
         st_async_f32(dsmem_addr(recv_u32 + (uint32_t)(((rank * G + h) * cols + (c - owner * cols)) * 4), owner), v,
                      dsmem_addr(recv_bar, owner));
       }
-    } else if (e < n_el + G * CS) {
-      const int h = (int)(((uint32_t)(e - n_el) * inv_cs) >> 16), o = e - n_el - h * CS;
-      if (o * cols < W)                              // every block that owns columns needs every block's (m, l)
-        st_async_f32x2(dsmem_addr(recv_u32 + (uint32_t)((ml_off + (rank * G + h) * 2) * 4), o), acc_m[k], acc[k],
-                       dsmem_addr(recv_bar, o));
     }
   }
   mark(6);
