@@ -21,14 +21,15 @@
 // so no MMA row is wasted on padding.  The block's result (m, l, O') is left in shared memory.
 //
 // Two ways to combine the blocks of one (b, g):
-//   cluster kernel  the splits of a (b, g) form one thread-block cluster (up to 16 blocks); after a
-//                   cluster barrier every block merges its own slice of the output columns by reading
-//                   its peers' results over distributed shared memory.  No global scratch, no atomics:
-//                   the short-latency path for small batches.
+//   cluster kernel  the splits of a (b, g) form one thread-block cluster (up to 16 blocks); every block sends
+//                   the merged values of each output column to the block that owns the column (st.async into
+//                   the owner's shared memory, counted on the owner's mbarrier), and the owner adds what it
+//                   receives in rank order.  No global scratch, no atomics: the short-latency path for small
+//                   batches.
 //   ticket kernel   blocks publish their result to a global workspace; the last block to finish a
 //                   (b, g) (atomic ticket) merges the records in split order.  Any number of splits.
-// Neither waits on another block with a spin: the cluster barrier is a hardware barrier among
-// co-scheduled blocks, the ticket path never waits at all.
+// The ticket path never waits on another block.  In the cluster path a block waits (bounded, on its own
+// mbarrier) for the sends of blocks that are co-scheduled with it by the hardware.
 #pragma once
 #include "common.cuh"
 
