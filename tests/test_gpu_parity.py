@@ -698,3 +698,72 @@ def test_two_sm_projection_equals_the_one_block_kernel_bitwise(monkeypatch, px, 
         for name in ("k_base", "v_base", "lr_k", "lr_v"):
             assert torch.equal(getattr(a, name).view(torch.int16), getattr(b, name).view(torch.int16)), name
     px2.close()
+
+
+# ------------------------------------------------------------------ cluster merge under every layout switch
+
+_LAYOUTS = [
+    ({"PRECC_DECODE_CLUSTER": "15"}, 64, 8, 4, 16),                       # blocks 13, 14 own no output column
+    ({"PRECC_DECODE_CLUSTER": "13"}, 64, 8, 4, 16),                       # the last block owns 4 of 5 columns
+    ({"PRECC_DECODE_CLUSTER": "11", "PRECC_DEEP": "0"}, 64, 4, 3, 8),     # odd query group, rank 8 (half an MMA tile)
+    ({"PRECC_DEEP": "2"}, 64, 8, 4, 16),                                  # one block per SM, four-page rings
+    ({"PRECC_DEEP": "2", "PRECC_DECODE_CLUSTER": "7"}, 128, 8, 4, 64),    # adapter term after the block merge
+    ({"PRECC_DEEP": "0"}, 128, 8, 2, 64),
+    ({"PRECC_DECODE_PRE": "1"}, 64, 8, 4, 16),                            # one ring slot before the dependency wait
+    ({"PRECC_DECODE_STAGES": "2", "PRECC_DEEP": "2"}, 128, 4, 4, 32),
+    ({"PRECC_DEEP": "2", "PRECC_DECODE_CLUSTER": "6"}, 64, 8, 1, 0),      # no adapter at all, one query head per kv head
+]
+
+
+@pytest.mark.parametrize("env,hd,n_kv,G,r", _LAYOUTS, ids=lambda v: "-".join(f"{k[6:]}{x}" for k, x in v.items()) if isinstance(v, dict) else str(v))
+def test_cluster_merge_under_every_layout_switch(monkeypatch, env, hd, n_kv, G, r):
+    """The merge inside a cluster (sends to the block that owns a column) with cluster sizes that leave blocks
+    without columns, both ring layouts, both places of the value-side adapter term, and the partial-record mode
+    of the same kernel: every variant against the oracle, twice for determinism."""
+    from paper_2609_34054_b200.binding import Cache, layer_desc
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    p2 = Precc(0)                                        # the switches are read when a context is created
+    try:
+        geo = I.Geometry(1024, G * n_kv, n_kv, hd, 2, r, r, alpha=2.0 * max(r, 1))
+        T = 5000 + 16 * n_kv + 3
+        nb = (T + 15) // 16
+        c = I.direct_caches(nb, geo, 77, f"lay.{hd}.{n_kv}.{r}")
+        cache = Cache.from_tensors(geo, c["k_base"].cuda(), c["v_base"].cuda(), c["lr_k"].cuda() if r else None,
+                                   c["lr_v"].cuda() if r else None)
+        w = I.layer_weights(geo, 77, "lay")
+        desc = layer_desc(geo)
+        q = I.queries(1, geo, 77, "lay.q", gain=4.0)
+        aid = torch.tensor([1], dtype=torch.int32).cuda()
+        cl = torch.tensor([T], dtype=torch.int32).cuda()
+        B_k = w["B_k"].cuda() if r else None
+        B_v = w["B_v"].cuda() if r else None
+        out = torch.full_like(q, float("nan"), device="cuda")
+        ws = p2.decode_workspace(desc, 1, T)
+        p2.lr_attend_decode(desc, q.cuda(), aid, cl, T, B_k, B_v, cache, out, ws)
+        torch.cuda.synchronize()
+        first = out.clone()
+        p2.lr_attend_decode(desc, q.cuda(), aid, cl, T, B_k, B_v, cache, out, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(first, out)
+        # partial-record mode (one shard holding everything) + combine = the same attention
+        R = p2.partial_record_floats(desc)
+        rec = torch.full((1, 1, n_kv, R), float("nan"), dtype=torch.float32, device="cuda")
+        p2.lr_attend_decode_partial(desc, q.cuda(), aid, cl, T, B_k, cache, rec[0], ws)
+        out2 = torch.full_like(q, float("nan"), device="cuda")
+        p2.combine_partials(desc, rec, aid, B_v, out2)
+        torch.cuda.synchronize()
+        assert torch.isfinite(rec).all()
+        rows = lambda x: f64(x.reshape(-1, x.shape[-1]))[:T]
+        zero = np.zeros((1, hd))
+        for g in (0, n_kv - 1, n_kv // 2):
+            cols = slice(g * hd, (g + 1) * hd)
+            ref = O.attend_from_caches(f64(q[0, g * G:(g + 1) * G]), rows(c["k_base"][:, g]), rows(c["v_base"][:, g]),
+                                       rows(c["lr_k"][1]) if r else np.zeros((T, 1)), rows(c["lr_v"][1]) if r else np.zeros((T, 1)),
+                                       f64(w["B_k"][1][:, cols]) if r else zero, f64(w["B_v"][1][:, cols]) if r else zero,
+                                       geo.scale_k if r else 0.0, geo.scale_v if r else 0.0, 1)
+            assert_close(f64(out)[0, g * G:(g + 1) * G], ref, f"{env} head {g}")
+            assert_close(f64(out2)[0, g * G:(g + 1) * G], ref, f"{env} head {g}, partial records + combine")
+        assert p2.poll_status() == 0
+    finally:
+        p2.close()
