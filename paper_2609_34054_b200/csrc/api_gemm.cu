@@ -74,9 +74,9 @@ int ilog2(int v) { int s = 0; while ((1 << s) < v) ++s; return s; }
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
   gp.hd_shift = ilog2(gp.hd); gp.rk_shift = ilog2(gp.rank_k > 0 ? gp.rank_k : 1); gp.rv_shift = ilog2(gp.rank_v > 0 ? gp.rank_v : 1);
   // Up to 40 rows the weight-streaming few-row kernel is the fastest (fused C3 projection: 8.7 us at 16 rows, 11.6 at
-  // 32); from there to 512 rows the split-K kernel (13..24 us; the few-row kernel needs 16.5 us at 48 rows and 18.4 at
-  // 64, the one-block-per-tile GEMM 27 us throughout); the few-row kernel still takes 41..64 rows when the split does
-  // not apply (rotary epilogue, short K).
+  // 32); from there to about a thousand rows the split-K kernels (12.5 .. 23 us; the few-row kernel needs 16.5 us at
+  // 48 rows and 18.4 at 64, the one-block-per-tile GEMM 27 .. 30 us throughout); the few-row kernel still takes
+  // 41..64 rows when the split does not apply (rotary epilogue, short K).
   if (M <= 40 && !ctx->force_tiled_gemm) {
     const int32_t rc = launch_small(ctx, X, M, K, Wt, n_out, gp, stream);
     if (rc >= 0) return rc;
@@ -84,7 +84,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
   const int m_tiles = (M + GEMM_BM - 1) / GEMM_BM;
   // A few row tiles (the tokens of a short turn): the K extent of every tile is split over a cluster.  The split
   // depends on M and K alone, so a column's summation order is the same whichever entry point produced it.
-  if (m_tiles <= 8 && !gp.rope && !ctx->no_gemm_splitk) {
+  if (m_tiles <= 16 && !gp.rope && !ctx->no_gemm_splitk) {
     const int nkb = K / GEMM_BK;
     // planned for the width of the FUSED projection of this layer, whatever this call projects, so that the base-only,
     // LR-only and fused calls of one M take the same decision (and with it the same summation order)
@@ -97,30 +97,36 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
     const long long clusters = (long long)m_tiles * ((n_fused + 255) / 256);
     // the finest split whose clusters are all resident at once (a second wave would cost more than the split gains);
     // cluster sizes need not be powers of two: 18 clusters fit as 6-block clusters, 36 as 3-block clusters
-    int ks = GEMM_MAX_KS, smem_plan = 0;
-    // a two-way split does not pay for its merge (measured at 768 and 1024 rows of the fused Llama-3-8B projection:
-    // 32.7 and 33.1 us against 31.4 and 32.1 us without a split), so the split must be three-way or finer; with nine
-    // column tiles that serves up to five row tiles (640 rows: 25 us against 30.5 us)
-    const int ks_min = 3;
+    int ks = (ctx->gemm_ks_max >= 2 && ctx->gemm_ks_max < GEMM_MAX_KS) ? ctx->gemm_ks_max : GEMM_MAX_KS, smem_plan = 0;
+    const int push_max = (ctx->gemm_push_max >= 0 && ctx->gemm_push_max < GEMM_PUSH_MAX_KS) ? ctx->gemm_push_max : GEMM_PUSH_MAX_KS;
+    // Clusters of 2 .. 4 blocks merge by bulk sends (proj_gemm_splitk_push_kernel), larger ones by pulling over
+    // distributed shared memory (their slices do not fit twice beside each other).  Fused Llama-3-8B projection,
+    // graph replay over rotating weights: 384 / 512 / 640 rows (clusters of 4 / 4 / 3) 16.4 / 18.4 / 19.2 us against
+    // 19.3 / 22.1 / 22.5 us with the pulling merge; 768 / 896 / 1024 rows (clusters of 2) 22.4 / 22.6 / 23.2 us
+    // against 29.2 / 30.1 / 30.3 us on the one-block-per-tile kernel (a two-way split did not pay for a pulling merge).
+    const int ks_min = ctx->gemm_ks_min;
     for (; ks >= ks_min; --ks) {
-      if (nkb / ks < 2) continue;
+      const bool push = ks <= push_max;
+      if (nkb / ks < (push ? 4 : 2)) continue;                   // a coarse split of a short K is not worth a cluster
       const int cw = ((256 + ks - 1) / ks + 7) / 8 * 8;          // planned for the widest tile, whatever this call's width
-      const int dump = ks * GEMM_BM * (cw + 4) * 4;
-      smem_plan = (((ring_max > dump ? ring_max : dump) + 1023) & ~1023) + (2 * SK_STAGES + 4) * 8;
+      const int slice = GEMM_BM * (cw + 4) * 4;
+      const int dump = push ? 2 * (ks - 1) * slice : ks * slice;
+      smem_plan = (((ring_max > dump ? ring_max : dump) + 1023) & ~1023) + (2 * SK_STAGES + 8) * 8;
       if (smem_plan > ctx->max_smem_optin) continue;
-      static int max_clusters_dev[kMaxDevices][GEMM_MAX_KS + 1] = {{0}};   // 0 = unknown, else max active clusters + 1
+      static int max_clusters_dev[kMaxDevices][2][GEMM_MAX_KS + 1] = {{{0}}};   // 0 = unknown, else max active clusters + 1
       std::lock_guard<std::recursive_mutex> lk(lazy_mu());
-      int& cached = max_clusters_dev[ctx->device % kMaxDevices][ks];
+      int& cached = max_clusters_dev[ctx->device % kMaxDevices][push ? 1 : 0][ks];
       if (cached == 0) {
         int n = 0;
-        if (raise_smem_limit(ctx, proj_gemm_splitk_kernel, smem_plan) == cudaSuccess) {
+        auto kern = push ? proj_gemm_splitk_push_kernel : proj_gemm_splitk_kernel;
+        if (raise_smem_limit(ctx, kern, smem_plan) == cudaSuccess) {
           cudaLaunchConfig_t qc = {};
           qc.gridDim = dim3(ks, ctx->sm_count, 1); qc.blockDim = dim3(GEMM_THREADS); qc.dynamicSmemBytes = smem_plan;
           cudaLaunchAttribute qa[1];
           qa[0].id = cudaLaunchAttributeClusterDimension;
           qa[0].val.clusterDim.x = ks; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
           qc.attrs = qa; qc.numAttrs = 1;
-          if (cudaOccupancyMaxActiveClusters(&n, proj_gemm_splitk_kernel, &qc) != cudaSuccess) { cudaGetLastError(); n = 0; }
+          if (cudaOccupancyMaxActiveClusters(&n, kern, &qc) != cudaSuccess) { cudaGetLastError(); n = 0; }
         } else {
           cudaGetLastError();
         }
@@ -142,7 +148,8 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
       gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
       gp.spread_rows = 0;
       gp.status = ctx->status;
-      PRECC_CUDA(ctx, raise_smem_limit(ctx, proj_gemm_splitk_kernel, smem_plan));
+      auto kern = ks <= push_max ? proj_gemm_splitk_push_kernel : proj_gemm_splitk_kernel;
+      PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, smem_plan));
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3(ks, n_tiles, m_tiles);
       cfg.blockDim = dim3(GEMM_THREADS);
@@ -152,7 +159,7 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
       attr[0].id = cudaLaunchAttributeClusterDimension;
       attr[0].val.clusterDim.x = ks; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
       cfg.attrs = attr; cfg.numAttrs = 1;
-      PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, proj_gemm_splitk_kernel, map_x, map_w, gp));
+      PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, map_x, map_w, gp));
       return PRECC_OK;
     }
   }

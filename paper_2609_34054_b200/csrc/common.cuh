@@ -112,6 +112,32 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
   return false;
 }
 
+// Bounded wait for bytes sent by other blocks of the cluster (acquire at cluster scope); limit as in mbar_wait.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t* status) {
+  auto poll = [&]() -> bool {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+  };
+  if (poll()) return true;
+  const long long t0 = clock64();
+  long long limit = -1;
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (poll()) return true;
+    if (limit < 0) limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
+    if (clock64() - t0 > limit) break;
+    if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
+  }
+  atomicOr(status, StatusBits::TIMEOUT);
+  return false;
+}
+
 // XOR swizzle of 16-byte chunks inside a tile whose rows hold CPR chunks (CPR in {1,2,4,8,16}):
 // eight consecutive rows of the same logical chunk land in eight different 16-byte bank groups.
 template <int CPR>

@@ -914,32 +914,6 @@ __device__ __forceinline__ void st_async_f32x2(uint32_t remote, float a, float b
 }
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
-// Bounded wait for bytes sent by other blocks of the cluster (acquire at cluster scope); limit as in mbar_wait.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint32_t* status) {
-  auto poll = [&]() -> bool {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-  };
-  if (poll()) return true;
-  const long long t0 = clock64();
-  long long limit = -1;
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (poll()) return true;
-    if (limit < 0) limit = static_cast<long long>(*reinterpret_cast<volatile uint32_t*>(status + 1)) << 10;
-    if (clock64() - t0 > limit) break;
-    if (*reinterpret_cast<volatile uint32_t*>(status) & StatusBits::TIMEOUT) return false;
-  }
-  atomicOr(status, StatusBits::TIMEOUT);
-  return false;
-}
-
 // MINB = 2 (8 warps, head_dim 64): 16-block clusters need two blocks per SM, which caps the kernel at 128
 // registers; the one-block-per-SM ring layout uses the MINB = 1 instance, free of that cap.
 template <int HD, int RK, int RV, int NW, bool ROPE = false, int MINB = 1>

@@ -477,4 +477,278 @@ proj_gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Split-K with a merge by bulk sends (clusters of 2 .. 4 blocks: the turns of a few hundred to a thousand rows).
+// Same main loop as the kernel above.  Then block r dumps the column slices it does NOT own to shared memory
+// (over the idle ring), tells its peers that its ring is idle, and - once every peer has said the same - sends
+// slice j to block j with ONE cp.async.bulk (shared::cta -> shared::cluster), which counts the bytes on an
+// mbarrier of the receiver.  A receiver waits for its (KS - 1) slices, adds them to its own slice (re-read from
+// tensor memory) in rank order - the order of the pulling kernel, bit for bit - and stores through the same
+// epilogue routing.  The copy engine moves a slice (32 .. 66 KB) in well under a microsecond, where sixteen
+// 16-byte loads per thread over distributed shared memory moved the same bytes in 4 .. 6 us.
+// Shared memory: [ring | overlaid: dump of KS-1 slices, then receive area of KS-1 slices] [barriers].
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+}
+
+// What the routing of a row's 16-byte pieces needs to know about the row, worked out once (no rotary keys here).
+struct RowRoute {
+  bool ok;
+  long long slot, slot2, base_row;
+  unsigned long long mask;
+  __device__ __forceinline__ void init(const GemmParams& p, int gm) {
+    ok = gm < p.M;
+    slot = 0; slot2 = -1;
+    if (ok) {
+      slot = p.slot_mapping ? (long long)p.slot_mapping[gm] : p.start_slot + gm;
+      if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); ok = false; slot = 0; }
+    }
+    mask = (p.row_masks && ok) ? p.row_masks[gm] : p.agent_mask;
+    if (p.lr_copy_slots && ok) {
+      slot2 = p.lr_copy_slots[gm];
+      if (slot2 >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); slot2 = -1; }
+    }
+    base_row = (((slot / PAGE) * p.n_kv * PAGE) + (slot % PAGE)) << p.hd_shift;
+  }
+  // columns gc .. gc + 7 of the call's output (gc is the same in every lane: the branches are warp-uniform)
+  __device__ __forceinline__ void store8(const GemmParams& p, int gc, const float (&v8)[8]) const {
+    if (!ok) return;
+    const int hs = p.hd_shift, w = p.n_kv << hs;
+    uint4 v;
+    v.x = pack_bf16(v8[0], v8[1]); v.y = pack_bf16(v8[2], v8[3]); v.z = pack_bf16(v8[4], v8[5]); v.w = pack_bf16(v8[6], v8[7]);
+    if (p.mode == 1 || (p.mode == 2 && gc < 2 * w)) {
+      const bool is_v = gc >= w;
+      const int cc = is_v ? gc - w : gc;
+      const int g = cc >> hs, c = cc & (p.hd - 1);
+      *reinterpret_cast<uint4*>((is_v ? p.base_v : p.base_k) + base_row + ((long long)(g * PAGE) << hs) + c) = v;
+    } else {
+      const int n_lrk = p.rank_k > 0 ? (p.n_agents << p.rk_shift) : 0;
+      const int gl = p.mode == 2 ? gc - 2 * w : gc;
+      const bool is_v = gl >= n_lrk;
+      const int sh = is_v ? p.rv_shift : p.rk_shift;
+      const int cc = is_v ? gl - n_lrk : gl;
+      const int agent = cc >> sh, ri = cc & ((1 << sh) - 1);
+      if (!((mask >> agent) & 1ull)) return;
+      __nv_bfloat16* arr = (is_v ? p.lr_v : p.lr_k) + (((long long)agent * p.n_blocks * PAGE) << sh) + ri;
+      *reinterpret_cast<uint4*>(arr + (slot << sh)) = v;
+      if (slot2 >= 0) *reinterpret_cast<uint4*>(arr + (slot2 << sh)) = v;
+    }
+  }
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const GemmParams p) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw;
+  if ((smem_u32(smem_raw) & 1023u) != 0) {               // the peers' addresses must correspond
+    if (threadIdx.x == 0) atomicOr(p.status, StatusBits::TIMEOUT);
+    return;
+  }
+  const int KS = gridDim.x, rank = blockIdx.x;           // the cluster spans grid.x
+  const int b_bytes = p.BN * GEMM_BK * 2;
+  const int stage_bytes = GEMM_A_BYTES + b_bytes;
+  const int cw = (((p.BN + KS - 1) / KS) + 7) / 8 * 8;   // columns finished by one block (a multiple of 8)
+  const int XS = cw + 4;                                 // row stride (floats) inside a slice: conflict-free row-per-thread access
+  const int slice_bytes = GEMM_BM * XS * 4;              // a multiple of 16
+  const int ring_bytes = p.stages * stage_bytes, merge_bytes = 2 * (KS - 1) * slice_bytes;
+  const int data_bytes = ((ring_bytes > merge_bytes ? ring_bytes : merge_bytes) + 1023) & ~1023;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + data_bytes);
+  // barrier map: full[stages] | empty[stages] | acc_full | ready (peers whose ring is idle) | recv (bytes received)
+  const uint32_t full0 = smem_u32(bars);
+  const uint32_t empty0 = full0 + 8 * p.stages;
+  const uint32_t acc_full = empty0 + 8 * p.stages;
+  const uint32_t ready_bar = acc_full + 8, recv_bar = acc_full + 16;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * p.stages + 4);
+  float* dump = reinterpret_cast<float*>(smem);                                       // [KS-1][128][XS]
+  float* recv = reinterpret_cast<float*>(smem + (size_t)(KS - 1) * slice_bytes);      // [KS-1][128][XS]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nkb = p.K / GEMM_BK;
+  const int kb0 = (rank * nkb) / KS;
+  const int nkb_s = ((rank + 1) * nkb) / KS - kb0;
+  const int m0 = blockIdx.z * GEMM_BM, n0 = blockIdx.y * p.BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(acc_full, 1);
+    mbar_init(ready_bar, KS - 1);
+    mbar_init(recv_bar, 1);
+    mbar_expect_tx(recv_bar, (uint32_t)((KS - 1) * slice_bytes));     // the one arrival, and the bytes to come
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    for (int it = 0; it < min(p.stages, nkb_s); ++it) {
+      const uint32_t sa = smem_u32(smem + (size_t)it * stage_bytes);
+      mbar_expect_tx(full0 + 8 * it, stage_bytes);
+      tma_load_2d(sa, &map_x, (kb0 + it) * GEMM_BK, m0, full0 + 8 * it);
+      tma_load_3d(sa + GEMM_A_BYTES, &map_w, 0, n0, kb0 + it, full0 + 8 * it);
+    }
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_holder)), "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = *tmem_holder;
+  // every block's barriers exist before anybody arrives on them from outside (the wait comes with the first remote use)
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory");
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int it = p.stages; it < nkb_s; ++it) {
+        const int s = it % p.stages;
+        mbar_wait(empty0 + 8 * s, ((it / p.stages) - 1) & 1, p.status);
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        mbar_expect_tx(full0 + 8 * s, stage_bytes);
+        tma_load_2d(sa, &map_x, (kb0 + it) * GEMM_BK, m0, full0 + 8 * s);
+        tma_load_3d(sa + GEMM_A_BYTES, &map_w, 0, n0, kb0 + it, full0 + 8 * s);
+      }
+    }
+    __syncwarp();
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(p.BN);
+      const uint64_t da0 = umma_desc_sw128(smem_u32(smem));
+      const uint64_t db0 = umma_desc_sw128(smem_u32(smem) + GEMM_A_BYTES);
+      for (int it = 0; it < nkb_s; ++it) {
+        const int s = it % p.stages;
+        mbar_wait(full0 + 8 * s, (it / p.stages) & 1, p.status);
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const uint64_t so = (uint64_t)((s * stage_bytes) >> 4);
+#pragma unroll
+        for (int k = 0; k < GEMM_BK / 16; ++k)
+          umma_bf16(tmem_base, da0 + so + 2 * k, db0 + so + 2 * k, idesc, (it | k) ? 1u : 0u);
+        umma_commit(empty0 + 8 * s);
+      }
+      umma_commit(acc_full);                       // every MMA of the slice has completed: the ring is idle too
+    }
+    __syncwarp();
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+  } else {
+    const int lane_base = (warp & 3) * 32;
+    const int row = lane_base + lane;
+    const int et = threadIdx.x - 64;                // 0 .. 127 among the four epilogue warps
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");   // the peers' barriers are initialised
+    mbar_wait(acc_full, 0, p.status);
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    // this block's ring is idle: the peers may send into the receive area that overlays it
+    if (et < KS - 1) {
+      const int peer = et < rank ? et : et + 1;
+      uint32_t remote;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(ready_bar), "r"(peer));
+      asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(remote) : "memory");
+    }
+    RowRoute route;
+    route.init(p, m0 + row);
+    const uint32_t trow = tmem_base + (static_cast<uint32_t>(lane_base) << 16);
+    // ---- the peers' slices, one after the other: TMEM (lane = row) -> shared memory fp32 [slot][128][XS] (slot = the
+    //      peer's rank with the own rank left out), then one bulk copy into the peer's receive area while the next
+    //      slice is being dumped
+    for (int k = 1; k < KS; ++k) {
+      const int sl = rank + k < KS ? rank + k : rank + k - KS;
+      const int c_lo = sl * cw, vw = min(cw, p.BN - c_lo);           // valid width of the slice (a multiple of 8, may be <= 0)
+      float* drow = dump + ((size_t)(sl < rank ? sl : sl - 1) * GEMM_BM + row) * XS;
+      int c = 0;
+      for (; c + 32 <= vw; c += 32) {
+        uint32_t r0[16], r1[16];
+        tmem_ld16(trow + c_lo + c, r0);
+        tmem_ld16(trow + c_lo + c + 16, r1);
+        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          *reinterpret_cast<uint4*>(drow + c + 4 * q) = make_uint4(r0[4 * q], r0[4 * q + 1], r0[4 * q + 2], r0[4 * q + 3]);
+          *reinterpret_cast<uint4*>(drow + c + 16 + 4 * q) = make_uint4(r1[4 * q], r1[4 * q + 1], r1[4 * q + 2], r1[4 * q + 3]);
+        }
+      }
+      for (; c + 8 <= vw; c += 8) {
+        uint32_t r[8];
+        tmem_ld8(trow + c_lo + c, r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+        *reinterpret_cast<uint4*>(drow + c) = make_uint4(r[0], r[1], r[2], r[3]);
+        *reinterpret_cast<uint4*>(drow + c + 4) = make_uint4(r[4], r[5], r[6], r[7]);
+      }
+      asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");         // the copy engine reads what these threads wrote
+      asm volatile("bar.sync 1, 128;\n" ::: "memory");                       // the four epilogue warps
+      if (et == 0) {
+        if (k == 1) mbar_wait_cluster(ready_bar, 0, p.status);                // every peer's ring is idle
+        // slice sl of this block goes to slot (own rank, sl's rank left out) of block sl's receive area
+        const uint32_t src = smem_u32(dump) + (uint32_t)((sl < rank ? sl : sl - 1) * slice_bytes);
+        const uint32_t dst_local = smem_u32(recv) + (uint32_t)((rank < sl ? rank : rank - 1) * slice_bytes);
+        uint32_t dst, bar;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(dst) : "r"(dst_local), "r"(sl));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(bar) : "r"(recv_bar), "r"(sl));
+        asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                     ::"r"(dst), "r"(src), "r"(slice_bytes), "r"(bar) : "memory");
+      }
+    }
+    // ---- own slice (tensor memory) + received slices, in rank order, routed to the caches
+    mbar_wait_cluster(recv_bar, 0, p.status);
+    {
+      const int c_lo = rank * cw, vw = min(cw, p.BN - c_lo);
+      for (int c = 0; c + 8 <= vw; c += 16) {
+        const bool two = c + 16 <= vw;                // 16 columns at a time, 8 at a ragged end (the same in every lane)
+        uint32_t own[16];
+        if (two) {
+          tmem_ld16(trow + c_lo + c, own);
+        } else {
+          uint32_t o8[8];
+          tmem_ld8(trow + c_lo + c, o8);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) { own[q] = o8[q]; own[8 + q] = 0u; }
+        }
+        float4 pr[GEMM_PUSH_MAX_KS - 1][4];
+#pragma unroll
+        for (int j = 0; j < GEMM_PUSH_MAX_KS - 1; ++j) {
+          if (j < KS - 1) {
+            const float* src = recv + ((size_t)j * GEMM_BM + row) * XS + c;
+            pr[j][0] = *reinterpret_cast<const float4*>(src);
+            pr[j][1] = *reinterpret_cast<const float4*>(src + 4);
+            if (two) { pr[j][2] = *reinterpret_cast<const float4*>(src + 8); pr[j][3] = *reinterpret_cast<const float4*>(src + 12); }
+          }
+        }
+        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (h == 1 && !two) break;
+          float v8[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) v8[q] = 0.f;
+          // rank order: slot j of the receive area holds rank j (j < own rank) or j + 1, so the own slice goes in
+          // just before slot `rank` (or last)
+          auto add_own = [&]() {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v8[q] += __uint_as_float(own[8 * h + q]);
+          };
+#pragma unroll
+          for (int j = 0; j < GEMM_PUSH_MAX_KS - 1; ++j) {
+            if (j < KS - 1) {
+              if (j == rank) add_own();
+              const float4 a = pr[j][2 * h], b = pr[j][2 * h + 1];
+              v8[0] += a.x; v8[1] += a.y; v8[2] += a.z; v8[3] += a.w; v8[4] += b.x; v8[5] += b.y; v8[6] += b.z; v8[7] += b.w;
+            }
+          }
+          if (rank == KS - 1) add_own();
+          const int gc = n0 + c_lo + c + 8 * h;
+          if (gc < p.N_out) route.store8(p, gc, v8);
+        }
+      }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  }
+  // Nobody leaves before every block has received everything: a block's sends read its own shared memory until then.
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+  }
+}
+
 }  // namespace precc

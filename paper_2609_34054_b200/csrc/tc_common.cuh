@@ -50,7 +50,8 @@ struct GemmParams {
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;                 // 64 bf16 = one 128-byte swizzle row
 constexpr int GEMM_THREADS = 192;
-constexpr int GEMM_MAX_KS = 8;            // largest K split of the split-K kernel (cluster size)
+constexpr int GEMM_MAX_KS = 8;            // largest K split of the split-K kernels (cluster size)
+constexpr int GEMM_PUSH_MAX_KS = 4;       // up to this split the partial tiles are merged by bulk sends
 constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;
 
 // The same bounded wait for waiters that are not on the critical path (an epilogue waiting for a whole tile of

@@ -666,6 +666,42 @@ def test_short_turn_projection_split_over_a_cluster(monkeypatch, px, M, d):
     px2.close()
 
 
+@pytest.mark.parametrize("ks,M,d", [(2, 100, 1024), (2, 777, 2048), (3, 384, 4096), (3, 130, 1024), (4, 512, 2048), (4, 64, 4096), (4, 1000, 1024)])
+def test_split_k_merge_by_bulk_sends_equals_the_pulling_merge_bitwise(monkeypatch, ks, M, d):
+    """Clusters of 2 to 4 blocks merge their partial tiles by bulk copies into the owner's shared memory; the
+    summation order is that of the pulling merge, so the two kernels must agree bit for bit at the same split -
+    and with the definition.  Scattered slots, agent mask, a fused width that is not a multiple of the tile."""
+    geo = I.Geometry(d, 8, 2, 128, 3, 16, 16, alpha=32.0)          # fused width 2*256 + 3*32 = 608 columns: three tiles, the last 96 wide
+    H = I.hidden_states(M, geo, seed=91, tag=f"push.{M}.{d}")
+    nb = (M + 15) // 16 + 3
+    slots = I.permutation(nb * 16, 91, f"push.slots.{M}")[:M].to(torch.int32)
+    caches = []
+    for push_max in ("4", "0"):
+        monkeypatch.setenv("PRECC_GEMM_KS_MAX", str(ks))
+        monkeypatch.setenv("PRECC_GEMM_KS_MIN", str(ks))
+        monkeypatch.setenv("PRECC_GEMM_PUSH_MAX", push_max)
+        pz = Precc(0)
+        L = Layer(pz, geo, seed=91, n_blocks=nb, fill=float("nan"))
+        dev = {k: v.cuda() for k, v in L.w.items()}
+        WA = pz.pack_turn_weights(geo, dev["W_k"], dev["W_v"], dev["A_k"], dev["A_v"])
+        pz.turn_project(L.desc, H.cuda(), WA, L.cache, 0, slots.cuda(), 0b110)
+        torch.cuda.synchronize()
+        assert pz.poll_status() == 0
+        caches.append(L)
+        pz.close()
+    La, Lb = caches
+    for name in ("k_base", "v_base", "lr_k", "lr_v"):
+        assert torch.equal(getattr(La.cache, name).view(torch.int16), getattr(Lb.cache, name).view(torch.int16)), name
+    w, Hn, sl = La.w_np, f64(H), slots.long()
+    tol = lambda ref: 2.0 ** -8 * np.abs(ref) + 2e-3 * np.sqrt(d / 256)
+    for got, ref in ((base_rows(La.cache.k_base)[sl], O.base_cache(Hn, w["W_k"])), (base_rows(La.cache.v_base)[sl], O.base_cache(Hn, w["W_v"])),
+                     (lr_rows(La.cache.lr_k, 1)[sl], O.lr_cache(Hn, w["A_k"][1])), (lr_rows(La.cache.lr_v, 2)[sl], O.lr_cache(Hn, w["A_v"][2]))):
+        assert (np.abs(got - ref) <= tol(ref)).all()
+    assert torch.isnan(La.cache.lr_k[0]).all()                     # agent 0 is masked out
+    untouched = torch.ones(nb * 16, dtype=torch.bool); untouched[sl] = False
+    assert torch.isnan(La.cache.k_base.permute(0, 2, 1, 3).reshape(nb * 16, -1)[untouched]).all()
+
+
 @pytest.mark.parametrize("M,d,hd,n_kv,r", [(1000, 512, 128, 2, 32), (2125, 1024, 64, 8, 16), (640, 256, 128, 1, 8)])
 def test_two_sm_projection_equals_the_one_block_kernel_bitwise(monkeypatch, px, M, d, hd, n_kv, r):
     """The cta_group::2 form of the projection GEMM (two SMs per 256-row tile, each staging half of the weight tile;
