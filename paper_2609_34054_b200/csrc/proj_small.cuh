@@ -62,9 +62,19 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
   }
-  pdl_wait();                 // X may be the previous kernel's output
-  pdl_launch_dependents();
   __syncthreads();
+  // The weights are not the preceding kernel's to write: the first ring fill of W boxes is requested before the wait
+  // for that kernel (programmatic dependent launch), so a block that is resident early has them in shared memory
+  // when its predecessor ends.  X (the previous kernel's output) and every store stay behind the wait.
+  const int pre = steps < PS_STAGES ? steps : PS_STAGES;
+  if (warp == PS_WARPS && lane == 0) {
+    for (int s = 0; s < pre; ++s) {
+      mbar_expect_tx(full0 + 8 * s, STEP_BYTES);
+      tma_load_3d(tiles + s * STEP_BYTES, &map_w, 0, group * COLS, k0 / PS_BK + s, full0 + 8 * s);
+    }
+  }
+  pdl_wait();                 // X may be the previous kernel's output; the caches may still be read by it
+  pdl_launch_dependents();
 
   float acc[MT][NT][4];
 #pragma unroll
@@ -75,9 +85,11 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   if (warp == PS_WARPS) {
     // ---- producer: one lane walks the k steps of this block's slice
     if (lane == 0) {
-      for (int s = 0; s < steps; ++s) {
+      for (int s = 0; s < pre; ++s)                      // the X boxes of the steps whose W boxes are already on their way
+        tma_load_2d(tiles + s * STEP_BYTES + W_BYTES, &map_x, k0 + s * PS_BK, 0, full0 + 8 * s);
+      for (int s = pre; s < steps; ++s) {
         const int slot = s % PS_STAGES;
-        if (s >= PS_STAGES) mbar_wait(empty0 + 8 * slot, ((s / PS_STAGES) - 1) & 1, p.status);
+        mbar_wait(empty0 + 8 * slot, ((s / PS_STAGES) - 1) & 1, p.status);
         const uint32_t dst = tiles + slot * STEP_BYTES;
         mbar_expect_tx(full0 + 8 * slot, STEP_BYTES);
         tma_load_3d(dst, &map_w, 0, group * COLS, k0 / PS_BK + s, full0 + 8 * slot);   // one contiguous run of the k-blocked weights
