@@ -899,19 +899,6 @@ lr_attend_decode_kernel(const DecodeParams p) {
 // mbarriers' initialisation visible: arrived at when the kernel starts, waited for before the first send, i.e.
 // long complete.  A block leaves once it has received everything addressed to it, so no send can reach the
 // shared memory of a block that is gone.
-__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(local), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void st_async_f32(uint32_t remote, float v, uint32_t remote_bar) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];\n"
-               ::"r"(remote), "f"(v), "r"(remote_bar) : "memory");
-}
-__device__ __forceinline__ void st_async_f32x2(uint32_t remote, float a, float b, uint32_t remote_bar) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];\n"
-               ::"r"(remote), "f"(a), "f"(b), "r"(remote_bar) : "memory");
-}
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
 // MINB = 2 (8 warps, head_dim 64): 16-block clusters need two blocks per SM, which caps the kernel at 128

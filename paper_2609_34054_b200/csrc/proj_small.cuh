@@ -13,9 +13,13 @@
 //            the grid must be resident at once, or the launch runs in two waves;
 //   math   = mma.sync m16n8k16 (bf16 -> fp32): X rows on the M axis, a warp owns 8 (16 when M > 16)
 //            output columns; fragments come from shared memory with ldmatrix;
-//   reduce = partial tiles go to shared memory; after a cluster barrier each block sums one slice of the
-//            columns over its peers through distributed shared memory (rank order: deterministic) and
-//            scatters bf16 pieces into the paged caches.  No global scratch, no atomics.
+//   reduce = every block finishes one slice of its group's columns.  The consumer threads SEND their accumulator
+//            pairs to the block that owns the column (st.async into the owner's shared memory, bytes counted on
+//            the owner's mbarrier); the owner waits for its byte count, adds the partials in rank order
+//            (deterministic) and scatters bf16 pieces into the paged caches.  No global scratch, no atomics, and
+//            no cluster barrier on the critical path (one, relaxed, at the start makes the mbarriers visible).
+//            Rotary keys keep the earlier form: partial tiles in shared memory, a cluster barrier, and each block
+//            reads its slice - and the partner half of a head - from its peers over distributed shared memory.
 // Rotary keys (GemmParams::rope): the reducing thread of the lower half of a head also gathers the partner
 // piece hd/2 columns further and writes both rotated; the block tile therefore holds whole heads.
 // The K split depends on K alone, so an output value does not depend on which entry point, which other
@@ -33,8 +37,9 @@ constexpr int PS_THREADS = (PS_WARPS + 1) * 32;       // consumer warps + one pr
 __host__ __device__ constexpr int ps_nt(int mt) { return mt > 1 ? 2 : 1; }               // 8-column n-tiles per warp
 __host__ __device__ constexpr int ps_cols(int mt) { return PS_WARPS * 8 * ps_nt(mt); }   // output columns per block
 __host__ __device__ constexpr int ps_step_bytes(int mt) { return (ps_cols(mt) + mt * 16) * PS_BK * 2; }
+__host__ __device__ constexpr int ps_recv_bytes(int mt) { return mt * 16 * ps_cols(mt) * 4; }   // [cluster rank][row][own columns] fp32
 __host__ __device__ constexpr int ps_smem_bytes(int mt) {
-  return PS_STAGES * ps_step_bytes(mt) + 2 * PS_STAGES * 8 + 1024;   // ring | mbarriers | alignment slack
+  return PS_STAGES * ps_step_bytes(mt) + 128 + ps_recv_bytes(mt) + 1024;   // ring | mbarriers | receive area | alignment slack
 }
 
 template <int MT>
@@ -56,13 +61,20 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   const int steps = k_slice / PS_BK;
   const uint32_t tiles = smem_u32(smem);
   const uint32_t full0 = tiles + PS_STAGES * STEP_BYTES, empty0 = full0 + 8 * PS_STAGES;
+  const uint32_t recv_bar = empty0 + 8 * PS_STAGES;
+  const uint32_t recv_u32 = full0 + 128;                // behind the barriers; never overlaid: peers send while this block computes
+  const bool push = !p.rope;                            // the same in every block of the grid
+  const int cpb = COLS / CS;                            // columns finished by one block (a power of two >= 8)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < PS_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, PS_WARPS); }
+    mbar_init(recv_bar, 1);
+    if (push) mbar_expect_tx(recv_bar, (uint32_t)(CS * p.M * cpb * 4));   // the one arrival, and the bytes to come: rows < M of every peer
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
   }
   __syncthreads();
+  if (push) asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory");   // waited for before the first send
   // The weights are not the preceding kernel's to write: the first ring fill of W boxes is requested before the wait
   // for that kernel (programmatic dependent launch), so a block that is resident early has them in shared memory
   // when its predecessor ends.  X (the previous kernel's output) and every store stay behind the wait.
@@ -121,6 +133,61 @@ proj_small_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(empty0 + 8 * slot) : "memory");
     }
+  }
+  if (push) {
+    // ---- merge by sends: accumulator pairs go straight from registers to the owner of their column
+    __syncwarp();
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");   // every peer's mbarrier is initialised (long since)
+    const int cshift = 31 - __clz(cpb);
+    if (warp < PS_WARPS) {
+      const int r = lane >> 2, q = lane & 3;
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+          const int col = (warp * NT + t) * 8 + 2 * q;
+          const int owner = col >> cshift;
+          const uint32_t bar = dsmem_addr(recv_bar, owner);
+          const uint32_t dst = recv_u32 + (uint32_t)(((rank * (MT * 16) + mt * 16 + r) * cpb + (col & (cpb - 1))) * 4);
+          if (mt * 16 + r < p.M) st_async_f32x2(dsmem_addr(dst, owner), acc[mt][t][0], acc[mt][t][1], bar);
+          if (mt * 16 + r + 8 < p.M) st_async_f32x2(dsmem_addr(dst + 8 * cpb * 4, owner), acc[mt][t][2], acc[mt][t][3], bar);
+        }
+    }
+    // ---- this block finishes columns [rank*cpb, (rank+1)*cpb) of its group: 8-column pieces, partials added in rank order
+    const int ppr = cpb / 8;
+    const int n_items = p.M * ppr;
+    int it = threadIdx.x;
+    int row = it / ppr, pc = it - row * ppr;              // worked out before the wait
+    mbar_wait_cluster(recv_bar, 0, p.status);
+    const float* recv = reinterpret_cast<const float*>(smem + PS_STAGES * STEP_BYTES + 128);
+    for (; it < n_items; it += PS_THREADS, row = it / ppr, pc = it - row * ppr) {
+      const int gc = group * COLS + rank * cpb + pc * 8;
+      if (gc >= p.N_out) continue;
+      long long slot = p.slot_mapping ? (long long)p.slot_mapping[row] : p.start_slot + row;
+      if (slot < 0 || slot >= p.n_blocks * PAGE) { atomicOr(p.status, StatusBits::BAD_INDEX); continue; }
+      const unsigned long long mask = p.row_masks ? p.row_masks[row] : p.agent_mask;
+      float4 x0[8], x1[8];
+#pragma unroll
+      for (uint32_t s = 0; s < 8; ++s) {
+        if (s < CS) {
+          const float* src = recv + ((size_t)(s * (MT * 16) + row) * cpb + pc * 8);
+          x0[s] = *reinterpret_cast<const float4*>(src);
+          x1[s] = *reinterpret_cast<const float4*>(src + 4);
+        } else {
+          x0[s] = make_float4(0.f, 0.f, 0.f, 0.f); x1[s] = x0[s];
+        }
+      }
+      float v8[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v8[k] = 0.f;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        v8[0] += x0[s].x; v8[1] += x0[s].y; v8[2] += x0[s].z; v8[3] += x0[s].w;
+        v8[4] += x1[s].x; v8[5] += x1[s].y; v8[6] += x1[s].z; v8[7] += x1[s].w;
+      }
+      store_piece(p, slot / PAGE, (int)(slot % PAGE), gc, v8, mask, row);
+    }
+    return;     // a block leaves once everything addressed to it has arrived; its own sends carry their data with them
   }
   __syncthreads();                                     // all reads of the tiles are done; the region is reused
 
