@@ -134,7 +134,11 @@ int32_t precc_selftest_wait_timeout(precc_ctx* ctx, uint32_t* done_flag, void* s
  * (the 64-deep k step of any run of rows is contiguous, one TMA box).  dst has dst_rows * d_model
  * elements and must be packed with the dst_rows it is later used with.  Used to build the packed A (all
  * agents' down-projections side by side, Section 3.1), the packed W and the two together.  src, dst
- * device; d_model % 64 == 0. */
+ * device; d_model % 64 == 0.
+ * Packed matrices are constants of the projection calls: a projection of up to 64 rows is a programmatic
+ * dependent launch and requests its first weight boxes before it waits for the kernel ahead of it on the stream
+ * (H, the slot and mask arrays and every store come after that wait).  precc_pack_kmajor itself never lets a
+ * dependent launch start early, so packing and projecting back to back on one stream is ordered as usual. */
 int32_t precc_pack_kmajor(precc_ctx* ctx, const void* src, int32_t d_model, int32_t n_cols,
                           void* dst, int32_t dst_rows, int32_t dst_row0, void* stream);
 

@@ -73,10 +73,10 @@ int ilog2(int v) { int s = 0; while ((1 << s) < v) ++s; return s; }
 
 int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt, int n_out, GemmParams gp, cudaStream_t stream) {
   gp.hd_shift = ilog2(gp.hd); gp.rk_shift = ilog2(gp.rank_k > 0 ? gp.rank_k : 1); gp.rv_shift = ilog2(gp.rank_v > 0 ? gp.rank_v : 1);
-  // Up to 40 rows the weight-streaming few-row kernel is the fastest (fused C3 projection: 8.7 us at 16 rows, 11.6 at
-  // 32); from there to about a thousand rows the split-K kernels (12.5 .. 23 us; the few-row kernel needs 16.5 us at
-  // 48 rows and 18.4 at 64, the one-block-per-tile GEMM 27 .. 30 us throughout); the few-row kernel still takes
-  // 41..64 rows when the split does not apply (rotary epilogue, short K).
+  // Up to 40 rows the weight-streaming few-row kernel is the fastest (fused C3 projection: 5.8 us at 16 rows, 7.4 at
+  // 32, 12.7 at 40); from there to about a thousand rows the split-K kernels (12.3 .. 23 us; the few-row kernel needs
+  // 12.8 us at 41 rows and 13.7 at 64, the one-block-per-tile GEMM 27 .. 30 us throughout); the few-row kernel still
+  // takes 41..64 rows when the split does not apply (rotary epilogue, short K).
   if (M <= 40 && !ctx->force_tiled_gemm) {
     const int32_t rc = launch_small(ctx, X, M, K, Wt, n_out, gp, stream);
     if (rc >= 0) return rc;
