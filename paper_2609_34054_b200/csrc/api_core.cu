@@ -199,6 +199,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   if (const char* v = getenv("PRECC_DECODE_PRE")) ctx->decode_pre_stages = atoi(v);
   if (const char* v = getenv("PRECC_GEMM_STAGES")) ctx->gemm_stage_cap = atoi(v);
   if (const char* v = getenv("PRECC_GEMM_KS_MAX")) ctx->gemm_ks_max = atoi(v);
+  if (const char* v = getenv("PRECC_GEMM_DIRECT")) ctx->gemm_direct = atoi(v);
   if (const char* v = getenv("PRECC_GEMM_PUSH_MAX")) ctx->gemm_push_max = atoi(v);
   if (const char* v = getenv("PRECC_GEMM_KS_MIN")) { ctx->gemm_ks_min = atoi(v); if (ctx->gemm_ks_min < 2) ctx->gemm_ks_min = 2; }
   if (const char* v = getenv("PRECC_GEMM_SPLITK")) ctx->no_gemm_splitk = (strcmp(v, "0") == 0);

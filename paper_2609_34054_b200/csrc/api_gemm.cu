@@ -97,25 +97,32 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
     const long long clusters = (long long)m_tiles * ((n_fused + 255) / 256);
     // the finest split whose clusters are all resident at once (a second wave would cost more than the split gains);
     // cluster sizes need not be powers of two: 18 clusters fit as 6-block clusters, 36 as 3-block clusters
+    bool plan_direct = false, plan_push = false;
     int ks = (ctx->gemm_ks_max >= 2 && ctx->gemm_ks_max < GEMM_MAX_KS) ? ctx->gemm_ks_max : GEMM_MAX_KS, smem_plan = 0;
     const int push_max = (ctx->gemm_push_max >= 0 && ctx->gemm_push_max < GEMM_PUSH_MAX_KS) ? ctx->gemm_push_max : GEMM_PUSH_MAX_KS;
     // Clusters of 2 .. 4 blocks merge by bulk sends (proj_gemm_splitk_push_kernel), larger ones by pulling over
-    // distributed shared memory (their slices do not fit twice beside each other).  Fused Llama-3-8B projection,
-    // graph replay over rotating weights: 384 / 512 / 640 rows (clusters of 4 / 4 / 3) 16.4 / 18.4 / 19.2 us against
-    // 19.3 / 22.1 / 22.5 us with the pulling merge; 768 / 896 / 1024 rows (clusters of 2) 22.4 / 22.6 / 23.2 us
-    // against 29.2 / 30.1 / 30.3 us on the one-block-per-tile kernel (a two-way split did not pay for a pulling merge).
+    // distributed shared memory (their slices do not fit twice beside each other) or, for up to 64 rows, by direct
+    // sends.  Fused Llama-3-8B projection, graph replay over rotating weights: 384 / 512 / 640 rows (clusters of
+    // 4 / 4 / 3) 16.4 / 18.4 / 19.2 us against 19.3 / 22.1 / 22.5 us with the pulling merge; 768 / 896 / 1024 rows
+    // (clusters of 2) 22.4 / 22.6 / 23.2 us against 29.2 / 30.1 / 30.3 us on the one-block-per-tile kernel (a two-way
+    // split did not pay for a pulling merge).
     const int ks_min = ctx->gemm_ks_min;
     for (; ks >= ks_min; --ks) {
-      const bool push = ks <= push_max;
-      if (nkb / ks < (push ? 4 : 2)) continue;                   // a coarse split of a short K is not worth a cluster
+      const bool bulk = ks <= push_max && ctx->gemm_direct < 2;       // whole slices by bulk copy
+      // pieces straight from registers: pays only while few rows exist (fused Llama-3-8B projection, clusters of 8:
+      // 11.7 against 12.2 us at 41 rows, 12.6 against 13.0 at 64, but 16.5 against 15.6 at 128 and 21.8 against 17.0 at 256)
+      const bool direct = !bulk && (ctx->gemm_direct >= 2 || (ctx->gemm_direct == 1 && M <= 64));
+      const bool push = bulk || direct;
+      if (nkb / ks < (ks <= GEMM_PUSH_MAX_KS ? 4 : 2)) continue;       // a coarse split of a short K is not worth a cluster
       const int cw = ((256 + ks - 1) / ks + 7) / 8 * 8;          // planned for the widest tile, whatever this call's width
       const int slice = GEMM_BM * (cw + 4) * 4;
-      const int dump = push ? 2 * (ks - 1) * slice : ks * slice;
+      const int dump = bulk ? 2 * (ks - 1) * slice : (direct ? (ks - 1) * slice : ks * slice);
       smem_plan = (((ring_max > dump ? ring_max : dump) + 1023) & ~1023) + (2 * SK_STAGES + 8) * 8;
       if (smem_plan > ctx->max_smem_optin) continue;
       static int max_clusters_dev[kMaxDevices][2][GEMM_MAX_KS + 1] = {{{0}}};   // 0 = unknown, else max active clusters + 1
       std::lock_guard<std::recursive_mutex> lk(lazy_mu());
       int& cached = max_clusters_dev[ctx->device % kMaxDevices][push ? 1 : 0][ks];
+      plan_direct = direct; plan_push = push;
       if (cached == 0) {
         int n = 0;
         auto kern = push ? proj_gemm_splitk_push_kernel : proj_gemm_splitk_kernel;
@@ -148,7 +155,8 @@ int32_t launch_gemm(precc_ctx* ctx, const void* X, int M, int K, const void* Wt,
       gp.M = M; gp.N_out = n_out; gp.K = K; gp.BN = bn; gp.stages = stages; gp.tmem_cols = tmem_cols;
       gp.spread_rows = 0;
       gp.status = ctx->status;
-      auto kern = ks <= push_max ? proj_gemm_splitk_push_kernel : proj_gemm_splitk_kernel;
+      auto kern = plan_push ? proj_gemm_splitk_push_kernel : proj_gemm_splitk_kernel;
+      gp.direct_send = plan_direct ? 1 : 0;
       PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, smem_plan));
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3(ks, n_tiles, m_tiles);

@@ -29,6 +29,7 @@ struct precc_ctx {
   bool force_tiled_gemm = false;       // PRECC_GEMM=tiled in the environment: never take the few-row kernel
   int gemm_ks_max = 0;                 // PRECC_GEMM_KS_MAX=n: finest K split (0 = the largest the kernels support)
   int gemm_push_max = -1;              // PRECC_GEMM_PUSH_MAX=n: merge by bulk sends up to this split (-1 = the kernels' limit, 0 = never)
+  int gemm_direct = 1;                 // PRECC_GEMM_DIRECT=n: split-K merge by direct sends - 0 never, 1 finer splits of up to 64 rows, 2 every split
   int gemm_ks_min = 2;                 // PRECC_GEMM_KS_MIN=n in the environment: coarsest K split of short-turn projections (experiments)
   bool no_gemm_splitk = false;         // PRECC_GEMM_SPLITK=0 in the environment: short turns stay on the one-block-per-tile GEMM
   bool force_ticket_decode = false;    // PRECC_DECODE=ticket in the environment: never use the cluster decode kernel

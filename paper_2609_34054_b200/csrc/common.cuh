@@ -149,6 +149,10 @@ __device__ __forceinline__ void st_async_f32(uint32_t remote, float v, uint32_t 
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];\n"
                ::"r"(remote), "f"(v), "r"(remote_bar) : "memory");
 }
+__device__ __forceinline__ void st_async_b32x4(uint32_t remote, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];\n"
+               ::"r"(remote), "r"(a), "r"(b), "r"(c), "r"(d), "r"(remote_bar) : "memory");
+}
 __device__ __forceinline__ void st_async_f32x2(uint32_t remote, float a, float b, uint32_t remote_bar) {
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];\n"
                ::"r"(remote), "f"(a), "f"(b), "r"(remote_bar) : "memory");

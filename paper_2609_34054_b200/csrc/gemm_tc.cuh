@@ -487,6 +487,10 @@ proj_gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
 // epilogue routing.  The copy engine moves a slice (32 .. 66 KB) in well under a microsecond, where sixteen
 // 16-byte loads per thread over distributed shared memory moved the same bytes in 4 .. 6 us.
 // Shared memory: [ring | overlaid: dump of KS-1 slices, then receive area of KS-1 slices] [barriers].
+// Finer splits (GemmParams::direct_send; twice KS-1 slices would not fit): no dump at all - every epilogue thread
+// sends the 16-byte pieces of its row straight from registers (st.async.v4 into the owner's receive area, which
+// alone overlays the ring), only the rows of the tile that exist; no barrier at the end either, since a send
+// carries its data with it.
 __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];\n"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
@@ -552,7 +556,8 @@ proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __
   const int cw = (((p.BN + KS - 1) / KS) + 7) / 8 * 8;   // columns finished by one block (a multiple of 8)
   const int XS = cw + 4;                                 // row stride (floats) inside a slice: conflict-free row-per-thread access
   const int slice_bytes = GEMM_BM * XS * 4;              // a multiple of 16
-  const int ring_bytes = p.stages * stage_bytes, merge_bytes = 2 * (KS - 1) * slice_bytes;
+  const bool direct = p.direct_send != 0;               // the same in every block
+  const int ring_bytes = p.stages * stage_bytes, merge_bytes = (direct ? 1 : 2) * (KS - 1) * slice_bytes;
   const int data_bytes = ((ring_bytes > merge_bytes ? ring_bytes : merge_bytes) + 1023) & ~1023;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + data_bytes);
   // barrier map: full[stages] | empty[stages] | acc_full | ready (peers whose ring is idle) | recv (bytes received)
@@ -562,7 +567,9 @@ proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __
   const uint32_t ready_bar = acc_full + 8, recv_bar = acc_full + 16;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * p.stages + 4);
   float* dump = reinterpret_cast<float*>(smem);                                       // [KS-1][128][XS]
-  float* recv = reinterpret_cast<float*>(smem + (size_t)(KS - 1) * slice_bytes);      // [KS-1][128][XS]
+  float* recv = reinterpret_cast<float*>(smem + (direct ? (size_t)0 : (size_t)(KS - 1) * slice_bytes));   // [KS-1][128][XS]
+  const int rows_valid = min(GEMM_BM, p.M - blockIdx.z * GEMM_BM);                     // rows of this tile that exist
+  const int vw_own = max(0, min(cw, p.BN - rank * cw));                                // columns of this block's slice that exist
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb = p.K / GEMM_BK;
@@ -575,7 +582,8 @@ proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __
     mbar_init(acc_full, 1);
     mbar_init(ready_bar, KS - 1);
     mbar_init(recv_bar, 1);
-    mbar_expect_tx(recv_bar, (uint32_t)((KS - 1) * slice_bytes));     // the one arrival, and the bytes to come
+    // the one arrival, and the bytes to come: whole slices by bulk copy, or the existing rows and columns piece by piece
+    mbar_expect_tx(recv_bar, direct ? (uint32_t)((KS - 1) * rows_valid * vw_own * 4) : (uint32_t)((KS - 1) * slice_bytes));
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     for (int it = 0; it < min(p.stages, nkb_s); ++it) {
@@ -648,7 +656,39 @@ proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __
     // ---- the peers' slices, one after the other: TMEM (lane = row) -> shared memory fp32 [slot][128][XS] (slot = the
     //      peer's rank with the own rank left out), then one bulk copy into the peer's receive area while the next
     //      slice is being dumped
-    for (int k = 1; k < KS; ++k) {
+    if (direct) mbar_wait_cluster(ready_bar, 0, p.status);           // every peer's ring is idle
+    for (int k = 1; direct && k < KS; ++k) {
+      const int sl = rank + k < KS ? rank + k : rank + k - KS;
+      const int c_lo = sl * cw, vw = min(cw, p.BN - c_lo);
+      // this row of slice sl goes to slot (own rank, sl's rank left out) of block sl's receive area
+      const uint32_t dst_local = smem_u32(recv) + (uint32_t)((((rank < sl ? rank : rank - 1) * GEMM_BM + row) * XS) * 4);
+      const uint32_t dst = dsmem_addr(dst_local, sl), bar = dsmem_addr(recv_bar, sl);
+      const bool live = row < rows_valid;
+      int c = 0;
+      for (; c + 32 <= vw; c += 32) {
+        uint32_t r0[16], r1[16];
+        tmem_ld16(trow + c_lo + c, r0);
+        tmem_ld16(trow + c_lo + c + 16, r1);
+        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+        if (live) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            st_async_b32x4(dst + (c + 4 * q) * 4, r0[4 * q], r0[4 * q + 1], r0[4 * q + 2], r0[4 * q + 3], bar);
+            st_async_b32x4(dst + (c + 16 + 4 * q) * 4, r1[4 * q], r1[4 * q + 1], r1[4 * q + 2], r1[4 * q + 3], bar);
+          }
+        }
+      }
+      for (; c + 8 <= vw; c += 8) {
+        uint32_t r[8];
+        tmem_ld8(trow + c_lo + c, r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+        if (live) {
+          st_async_b32x4(dst + c * 4, r[0], r[1], r[2], r[3], bar);
+          st_async_b32x4(dst + (c + 4) * 4, r[4], r[5], r[6], r[7], bar);
+        }
+      }
+    }
+    for (int k = 1; !direct && k < KS; ++k) {
       const int sl = rank + k < KS ? rank + k : rank + k - KS;
       const int c_lo = sl * cw, vw = min(cw, p.BN - c_lo);           // valid width of the slice (a multiple of 8, may be <= 0)
       float* drow = dump + ((size_t)(sl < rank ? sl : sl - 1) * GEMM_BM + row) * XS;
@@ -689,8 +729,9 @@ proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __
     mbar_wait_cluster(recv_bar, 0, p.status);
     {
       const int c_lo = rank * cw, vw = min(cw, p.BN - c_lo);
-      for (int c = 0; c + 8 <= vw; c += 16) {
-        const bool two = c + 16 <= vw;                // 16 columns at a time, 8 at a ragged end (the same in every lane)
+      const bool wide = KS <= GEMM_PUSH_MAX_KS;         // 16 columns at a time while the peers' pieces fit in registers
+      for (int c = 0; c + 8 <= vw; c += wide ? 16 : 8) {
+        const bool two = wide && c + 16 <= vw;          // 8 at a ragged end (the same in every lane)
         uint32_t own[16];
         if (two) {
           tmem_ld16(trow + c_lo + c, own);
@@ -700,14 +741,16 @@ proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __
 #pragma unroll
           for (int q = 0; q < 8; ++q) { own[q] = o8[q]; own[8 + q] = 0u; }
         }
-        float4 pr[GEMM_PUSH_MAX_KS - 1][4];
+        float4 pr[GEMM_MAX_KS - 1][4];
 #pragma unroll
-        for (int j = 0; j < GEMM_PUSH_MAX_KS - 1; ++j) {
+        for (int j = 0; j < GEMM_MAX_KS - 1; ++j) {
           if (j < KS - 1) {
             const float* src = recv + ((size_t)j * GEMM_BM + row) * XS + c;
             pr[j][0] = *reinterpret_cast<const float4*>(src);
             pr[j][1] = *reinterpret_cast<const float4*>(src + 4);
-            if (two) { pr[j][2] = *reinterpret_cast<const float4*>(src + 8); pr[j][3] = *reinterpret_cast<const float4*>(src + 12); }
+            if (j < GEMM_PUSH_MAX_KS - 1) {
+              if (two) { pr[j][2] = *reinterpret_cast<const float4*>(src + 8); pr[j][3] = *reinterpret_cast<const float4*>(src + 12); }
+            }
           }
         }
         asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
@@ -724,10 +767,10 @@ proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __
             for (int q = 0; q < 8; ++q) v8[q] += __uint_as_float(own[8 * h + q]);
           };
 #pragma unroll
-          for (int j = 0; j < GEMM_PUSH_MAX_KS - 1; ++j) {
-            if (j < KS - 1) {
+          for (int j = 0; j < GEMM_MAX_KS - 1; ++j) {
+            if (j < KS - 1 && (h == 0 || j < GEMM_PUSH_MAX_KS - 1)) {
               if (j == rank) add_own();
-              const float4 a = pr[j][2 * h], b = pr[j][2 * h + 1];
+              const float4 a = pr[j][h == 0 ? 0 : 2], b = pr[j][h == 0 ? 1 : 3];
               v8[0] += a.x; v8[1] += a.y; v8[2] += a.z; v8[3] += a.w; v8[4] += b.x; v8[5] += b.y; v8[6] += b.z; v8[7] += b.w;
             }
           }
@@ -739,10 +782,13 @@ proj_gemm_splitk_push_kernel(const __grid_constant__ CUtensorMap map_x, const __
     }
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
   }
-  // Nobody leaves before every block has received everything: a block's sends read its own shared memory until then.
+  // Bulk sends read the sender's shared memory: nobody leaves before every block has received everything.  Direct
+  // sends carry their data with them, and a receiver stays until it has everything: no barrier.
   __syncwarp();
-  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+  if (!direct) {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+  }
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
   __syncthreads();
   if (warp == 1) {

@@ -11,6 +11,7 @@ struct GemmParams {
   int M, N_out, K;
   int BN, stages, tmem_cols;
   int spread_rows;                // 1: even row-tile spreading allowed (rows may be written twice, identically)
+  int direct_send;                // split-K merge by sends: 1 = pieces straight from registers (st.async), 0 = whole slices by bulk copy
   int mode;                       // 0 = LR caches, 1 = base caches, 2 = base columns then LR columns
   const int32_t* slot_mapping;    // [M] or null
   int64_t start_slot;

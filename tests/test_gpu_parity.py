@@ -666,20 +666,24 @@ def test_short_turn_projection_split_over_a_cluster(monkeypatch, px, M, d):
     px2.close()
 
 
-@pytest.mark.parametrize("ks,M,d", [(2, 100, 1024), (2, 777, 2048), (3, 384, 4096), (3, 130, 1024), (4, 512, 2048), (4, 64, 4096), (4, 1000, 1024)])
-def test_split_k_merge_by_bulk_sends_equals_the_pulling_merge_bitwise(monkeypatch, ks, M, d):
-    """Clusters of 2 to 4 blocks merge their partial tiles by bulk copies into the owner's shared memory; the
-    summation order is that of the pulling merge, so the two kernels must agree bit for bit at the same split -
-    and with the definition.  Scattered slots, agent mask, a fused width that is not a multiple of the tile."""
+@pytest.mark.parametrize("ks,M,d", [(2, 100, 1024), (2, 777, 2048), (3, 384, 4096), (3, 130, 1024), (4, 512, 2048), (4, 64, 4096), (4, 1000, 1024),
+                                    (5, 200, 2048), (6, 256, 4096), (7, 41, 2048), (8, 128, 1024), (8, 77, 4096)])
+def test_split_k_merge_by_sends_equals_the_pulling_merge_bitwise(monkeypatch, ks, M, d):
+    """The partial tiles of a split-K cluster are merged by sends into the owner's shared memory: whole slices by bulk
+    copy (clusters of 2 to 4 blocks), or 16-byte pieces straight from registers (any cluster size; the default for
+    finer splits of up to 64 rows).  The summation order is that of the pulling merge, so all three must agree bit for bit at the
+    same split - and with the definition.  Scattered slots, agent mask, a fused width that is not a multiple of the tile."""
     geo = I.Geometry(d, 8, 2, 128, 3, 16, 16, alpha=32.0)          # fused width 2*256 + 3*32 = 608 columns: three tiles, the last 96 wide
     H = I.hidden_states(M, geo, seed=91, tag=f"push.{M}.{d}")
     nb = (M + 15) // 16 + 3
     slots = I.permutation(nb * 16, 91, f"push.slots.{M}")[:M].to(torch.int32)
     caches = []
-    for push_max in ("4", "0"):
+    for push_max, direct in (("4", "1"), ("0", "2"), ("0", "0")):       # bulk copies where they apply | direct sends | pulling
+        monkeypatch.setenv("PRECC_GEMM", "tiled")                      # keep the few-row kernel out of it
         monkeypatch.setenv("PRECC_GEMM_KS_MAX", str(ks))
         monkeypatch.setenv("PRECC_GEMM_KS_MIN", str(ks))
         monkeypatch.setenv("PRECC_GEMM_PUSH_MAX", push_max)
+        monkeypatch.setenv("PRECC_GEMM_DIRECT", direct)
         pz = Precc(0)
         L = Layer(pz, geo, seed=91, n_blocks=nb, fill=float("nan"))
         dev = {k: v.cuda() for k, v in L.w.items()}
@@ -689,7 +693,9 @@ def test_split_k_merge_by_bulk_sends_equals_the_pulling_merge_bitwise(monkeypatc
         assert pz.poll_status() == 0
         caches.append(L)
         pz.close()
-    La, Lb = caches
+    La, Lb, Lc = caches
+    for name in ("k_base", "v_base", "lr_k", "lr_v"):
+        assert torch.equal(getattr(La.cache, name).view(torch.int16), getattr(Lc.cache, name).view(torch.int16)), name
     for name in ("k_base", "v_base", "lr_k", "lr_v"):
         assert torch.equal(getattr(La.cache, name).view(torch.int16), getattr(Lb.cache, name).view(torch.int16)), name
     w, Hn, sl = La.w_np, f64(H), slots.long()
