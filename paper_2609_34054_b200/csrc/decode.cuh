@@ -162,6 +162,9 @@ __device__ __forceinline__ void load_q_frags(const DecodeParams& p, int b, int g
 // r_v LR-V coordinates appended).  Ends with a __syncthreads().  A block with no pages yields
 // m = NEG_BIG, l = 0, O' = 0.  With MERGE = false it stops one step earlier: the warps' records
 // [warp][ m[8] | l[8] | O'[8][OWP] ] are written to the start of `smem`, no barrier follows.
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
+
 // B_v slice staged in shared memory for the warps' own adapter term (cluster kernel): `bar` completes when
 // every thread's copies have landed.
 struct WarpExpand {
@@ -634,6 +637,9 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     l1 += __shfl_xor_sync(0xffffffffu, l1, d);
   }
   mark(5);
+  // Cluster schedule: the cluster barrier that every block arrived at when the kernel started (it makes the peers'
+  // mbarriers visible) is waited for here, where a warp that is done early waits for the others anyway.
+  if constexpr (!MERGE) cluster_wait();
 
   // ---- merge the warps of this block: smem [warp][ m[8] | l[8] | O'[8 heads][OWP] ], OWP = OW + 4: a store
   //      instruction touches heads cq = 0, 2, 4, 6 (2 OWP = 8 mod 32 banks apart) at rows r = 0..7, i.e. 32 different
@@ -899,8 +905,6 @@ lr_attend_decode_kernel(const DecodeParams p) {
 // mbarriers' initialisation visible: arrived at when the kernel starts, waited for before the first send, i.e.
 // long complete.  A block leaves once it has received everything addressed to it, so no send can reach the
 // shared memory of a block that is gone.
-__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
 // MINB = 2 (8 warps, head_dim 64): 16-block clusters need two blocks per SM, which caps the kernel at 128
 // registers; the one-block-per-SM ring layout uses the MINB = 1 instance, free of that cap.
 template <int HD, int RK, int RV, int NW, bool ROPE = false, int MINB = 1>
@@ -1062,7 +1066,6 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
     if (expand) __syncthreads();       // block-uniform: the merged LR-V coordinates are complete
   }
   mark(14);
-  cluster_wait();                      // the barrier arrived at when the kernel started: every peer's mbarrier is initialised
 #pragma unroll
   for (int k = 0; k < PER_THREAD; ++k) {
     const int e = threadIdx.x + k * NT;
@@ -1140,7 +1143,7 @@ lr_attend_decode_cluster_kernel(const DecodeParams p) {
       else out_bg[hh * HD + c0 + cc] = __float2bfloat16(v / L);
     }
     el += NT / 4;
-    h = el / ncol; c = el - h * ncol;
+    if (base + NT / 4 < n_own) { h = el / ncol; c = el - h * ncol; }   // only if another pass follows
   }
   if (rec && rank == 0) {                               // block 0 adds the maxima, the denominators and the unused slots
     for (int e = G * OW + threadIdx.x; e < 8 * OW; e += NT) rec[16 + e] = 0.f;
