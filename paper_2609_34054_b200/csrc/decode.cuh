@@ -366,6 +366,29 @@ __device__ __forceinline__ void decode_stream_block(const DecodeParams& p, unsig
     if (n_pre < my_n && tile0 + warp + NW * n_pre >= safe_tiles) break;
     issue_tile(n_pre);
   }
+  // Cluster schedule: the pages that will be requested as soon as the first ring slots are free are brought into L2
+  // now (a hint, not a read: L2 is the point of coherence, so this is allowed ahead of the wait for any page), which
+  // turns the round trip that a shallow ring exposes in the loop from a DRAM access into an L2 hit.  Only for short
+  // streams (at most two ring generations per warp), which are bound by that latency; a longer stream hides it behind
+  // its ring, and the extra requests cost it 2 .. 6 % (measured at head_dim 128, 8192 .. 131072 tokens).
+  if (!MERGE && my_n <= 2 * p.stages) {
+    constexpr int KV_LINES = C::KV_BYTES / 128;
+    const unsigned char* kb = reinterpret_cast<const unsigned char*>(p.k_base) + (size_t)g * C::KV_BYTES;
+    for (int i = p.stages; i < my_n && i < 2 * p.stages && i < 32; ++i) {
+      const int ph = __shfl_sync(0xffffffffu, phys_cur, i);
+      const unsigned char* ksrc = kb + (size_t)ph * kv_block_bytes;
+      for (int l = lane; l < 2 * KV_LINES; l += 32) {
+        const unsigned char* a = l < KV_LINES ? ksrc + l * 128 : ksrc + v_minus_k + (l - KV_LINES) * 128;
+        asm volatile("prefetch.global.L2 [%0];\n" ::"l"(a));
+      }
+      if (use_lr) {
+        if (RK > 0 && lane * 128 < C::LK_BYTES)
+          asm volatile("prefetch.global.L2 [%0];\n" ::"l"(reinterpret_cast<const unsigned char*>(lrk_a) + (size_t)ph * C::LK_BYTES + lane * 128));
+        if (RV > 0 && lane * 128 < C::LV_BYTES)
+          asm volatile("prefetch.global.L2 [%0];\n" ::"l"(reinterpret_cast<const unsigned char*>(lrv_a) + (size_t)ph * C::LV_BYTES + lane * 128));
+      }
+    }
+  }
   mark(8);
   pdl_wait();                 // the predecessor has completed: its q, its cache rows and its workspace are visible
   mark(9);
