@@ -333,6 +333,26 @@ int32_t precc_lr_attend_prefill_rope(precc_ctx* ctx, const precc_layer_desc* des
                                      const void* B_k, const void* B_v, const precc_rope* rope,
                                      const precc_cache* cache, void* out, void* stream);
 
+/* The same attention as precc_lr_attend_prefill_rope, computed the fast way at the price of a scratch area
+ * (Appendix D.2 leaves the mechanics open; the paper's own path never materialises adapted keys).  The adapted rotary
+ * keys of THIS sequence - K_base_rot[t] + s_k RoPE_t(L^K_a[t] B^K_a) for its ctx_len + S tokens, all kv heads - are
+ * written once into `key_scratch` (device, 128-byte aligned, at least precc_prefill_rope_scratch_bytes(desc, ctx_len,
+ * S) bytes = the sequence's base-key bytes rounded up to whole 128-token steps), in logical block order, and the
+ * tensor-core prefill kernel then streams them as its key operand; values and the value-side adapter are used from
+ * the caches as usual.  The scratch is transient: its contents are unspecified after the call and it can be reused
+ * by the next layer or sequence on the same stream.  Results agree with precc_lr_attend_prefill_rope within the
+ * attention tolerance (the key term is rounded to bf16 once here, twice there).  With rank_k == 0, for agent -1,
+ * or where the tensor-core kernel does not apply (unaligned caches), the call behaves exactly like
+ * precc_lr_attend_prefill_rope and leaves the scratch untouched.  A scratch that is too small returns
+ * PRECC_ERR_WORKSPACE and launches nothing. */
+size_t precc_prefill_rope_scratch_bytes(const precc_layer_desc* desc, int32_t ctx_len, int32_t S);
+int32_t precc_lr_attend_prefill_rope_scratch(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S,
+                                             int32_t agent, int32_t ctx_len, const int32_t* block_table,
+                                             int32_t table_stride, int32_t first_block,
+                                             const void* B_k, const void* B_v, const precc_rope* rope,
+                                             const precc_cache* cache, void* out, void* key_scratch,
+                                             size_t key_scratch_bytes, void* stream);
+
 /* ------------------------------------------------------------- context-sharded decode (no paper counterpart)
  * When the tokens of a request are spread over several GPUs (each holds base and LR rows of a contiguous
  * token range in its own caches), softmax attention over the union is the split-KV merge taken once more

@@ -25,6 +25,7 @@ EXPORTS = [
     "precc_rebase_project_rope", "precc_turn_project_rope", "precc_lr_attend_decode_rope", "precc_lr_attend_prefill_rope",
     "precc_turn_project_rows", "precc_partial_record_floats", "precc_lr_attend_decode_partial", "precc_combine_partials",
     "precc_set_wait_limit", "precc_selftest_wait_timeout",
+    "precc_prefill_rope_scratch_bytes", "precc_lr_attend_prefill_rope_scratch",
 ]
 
 
@@ -91,6 +92,10 @@ def load_library() -> C.CDLL:
                                                 C.POINTER(CacheDesc), vp, vp, sz, vp]
     lib.precc_lr_attend_prefill_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp, rp,
                                                  C.POINTER(CacheDesc), vp, vp]
+    lib.precc_prefill_rope_scratch_bytes.argtypes = [C.POINTER(LayerDesc), i32, i32]
+    lib.precc_prefill_rope_scratch_bytes.restype = sz
+    lib.precc_lr_attend_prefill_rope_scratch.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp, rp,
+                                                         C.POINTER(CacheDesc), vp, vp, sz, vp]
     lib.precc_turn_project_rows.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, vp, vp, C.POINTER(CacheDesc), vp]
     lib.precc_partial_record_floats.argtypes = [C.POINTER(LayerDesc)]
     lib.precc_partial_record_floats.restype = sz
@@ -316,6 +321,20 @@ class Precc:
         self._check(self.lib.precc_lr_attend_prefill_rope(
             self.h, C.byref(desc), _ptr(q), q.shape[0], agent, ctx_len, _ptr(block_table), stride, first_block,
             _ptr(B_k), _ptr(B_v), C.byref(rd), C.byref(cd), _ptr(out), _stream()), "precc_lr_attend_prefill_rope")
+
+    def prefill_rope_scratch_bytes(self, desc: LayerDesc, ctx_len: int, S: int) -> int:
+        return int(self.lib.precc_prefill_rope_scratch_bytes(C.byref(desc), ctx_len, S))
+
+    def lr_attend_prefill_rope_scratch(self, desc: LayerDesc, q: torch.Tensor, agent: int, ctx_len: int, B_k, B_v, rope: torch.Tensor,
+                                       cache: Cache, out: torch.Tensor, key_scratch: torch.Tensor,
+                                       block_table: Optional[torch.Tensor] = None, first_block: int = 0):
+        """Rotary prefill through a caller-provided scratch for the sequence's adapted keys (uint8 or bf16 tensor)."""
+        cd, rd = cache.desc(), self._rope(rope)
+        stride = block_table.numel() if block_table is not None else 0
+        self._check(self.lib.precc_lr_attend_prefill_rope_scratch(
+            self.h, C.byref(desc), _ptr(q), q.shape[0], agent, ctx_len, _ptr(block_table), stride, first_block,
+            _ptr(B_k), _ptr(B_v), C.byref(rd), C.byref(cd), _ptr(out), _ptr(key_scratch),
+            key_scratch.numel() * key_scratch.element_size(), _stream()), "precc_lr_attend_prefill_rope_scratch")
 
     # ------------------------------------------------------------------ context-sharded decode
     def partial_record_floats(self, desc: LayerDesc) -> int:

@@ -4,6 +4,7 @@
 #include "api_internal.h"
 #include "combine.cuh"
 #include "prefill.cuh"   // PF_ROWS (the size check of the prefill entry)
+#include "rope_expand.cuh"
 
 using namespace precc;
 
@@ -193,7 +194,7 @@ int32_t precc_lr_attend_decode_static(precc_ctx* ctx, const precc_layer_desc* de
 static int32_t prefill_entry(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
                              int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
                              const void* B_k, const void* B_v, const precc_rope* rope, const precc_cache* cache, void* out,
-                             void* stream) {
+                             void* stream, void* k_scratch = nullptr, size_t k_scratch_bytes = 0) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (S < 0 || ctx_len < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "S < 0 or ctx_len < 0");
@@ -218,7 +219,32 @@ static int32_t prefill_entry(precc_ctx* ctx, const precc_layer_desc* desc, const
   if ((long long)rope->max_pos < (long long)ctx_len + S)
     return fail(ctx, PRECC_ERR_INVALID_ARG, "rope table covers %d positions, the turn ends at %lld", rope->max_pos, (long long)ctx_len + S);
   a.rope = rope->table; a.max_pos = rope->max_pos;
-  return run();
+  if (!k_scratch || rk == 0) return run();     // no key-side adapter in play: the rotated base cache is all there is
+  // Rotary prefill with scratch: write the adapted rotary keys of the sequence out once (logical block order), then run
+  // the tensor-memory kernel on them without a key-side adapter.  Falls back to the per-tile expansion of the
+  // mma.sync kernel where the tensor-memory kernel does not take the call.
+  const long long stage_blocks = 128 / PRECC_PAGE;            // whole 128-token stages of the tensor-memory kernel
+  const long long out_blocks = (need_blocks + stage_blocks - 1) / stage_blocks * stage_blocks;
+  const size_t need_bytes = (size_t)out_blocks * desc->n_kv_heads * PRECC_PAGE * desc->head_dim * 2;
+  if (k_scratch_bytes < need_bytes) return fail(ctx, PRECC_ERR_WORKSPACE, "key scratch: need %zu bytes, got %zu", need_bytes, k_scratch_bytes);
+  if ((reinterpret_cast<uintptr_t>(k_scratch) & 127u) != 0) return fail(ctx, PRECC_ERR_MISALIGNED, "key scratch not 128-byte aligned");
+  PrefillArgs b = a;
+  b.rope = nullptr; b.max_pos = 0; b.B_k = nullptr; b.k_scratch = k_scratch; b.k_scratch_blocks = out_blocks;
+  const int32_t ok = desc->head_dim == 64 ? prefill_tc_eligible_hd64(ctx, b, 0, rv) : prefill_tc_eligible_hd128(ctx, b, 0, rv);
+  if (ok < 0) return ok;
+  if (ok == 0) return run();
+  RopeExpandParams x;
+  const size_t kvw = (size_t)desc->n_kv_heads * desc->head_dim;
+  x.k_base = (const __nv_bfloat16*)cache->k_base;
+  x.lr_k = (const __nv_bfloat16*)cache->lr_k + (size_t)agent * cache->n_blocks * PRECC_PAGE * desc->rank_k;
+  x.B_k = (const __nv_bfloat16*)B_k + (size_t)agent * desc->rank_k * kvw;
+  x.rope = reinterpret_cast<const float4*>(rope->table);
+  x.block_table = block_table; x.scratch = (__nv_bfloat16*)k_scratch; x.status = ctx->status;
+  x.n_blocks = cache->n_blocks; x.first_block = first_block; x.n_tokens = ctx_len + S;
+  x.n_kv = desc->n_kv_heads; x.hd = desc->head_dim; x.rk = desc->rank_k; x.max_pos = rope->max_pos; x.s_k = desc->lora_scale_k;
+  rope_expand_keys_kernel<<<(unsigned)out_blocks, RX_THREADS, 0, (cudaStream_t)stream>>>(x);
+  PRECC_CUDA(ctx, cudaGetLastError());
+  return desc->head_dim == 64 ? prefill_run_hd64(ctx, b, 0, rv) : prefill_run_hd128(ctx, b, 0, rv);
 }
 
 int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
@@ -234,6 +260,24 @@ int32_t precc_lr_attend_prefill_rope(precc_ctx* ctx, const precc_layer_desc* des
   if (!ctx) return PRECC_ERR_INVALID_ARG;
   if (!rope) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope is null");
   return prefill_entry(ctx, desc, q, S, agent, ctx_len, block_table, table_stride, first_block, B_k, B_v, rope, cache, out, stream);
+}
+
+size_t precc_prefill_rope_scratch_bytes(const precc_layer_desc* desc, int32_t ctx_len, int32_t S) {
+  if (!desc || ctx_len < 0 || S < 0 || desc->n_kv_heads <= 0 || desc->head_dim <= 0) return 0;
+  const long long blocks = ((long long)ctx_len + S + PRECC_PAGE - 1) / PRECC_PAGE;
+  const long long stage = 128 / PRECC_PAGE;
+  return (size_t)((blocks + stage - 1) / stage * stage) * desc->n_kv_heads * PRECC_PAGE * desc->head_dim * 2;
+}
+
+int32_t precc_lr_attend_prefill_rope_scratch(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
+                                             int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
+                                             const void* B_k, const void* B_v, const precc_rope* rope, const precc_cache* cache,
+                                             void* out, void* key_scratch, size_t key_scratch_bytes, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  if (!rope) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope is null");
+  if (!key_scratch) return fail(ctx, PRECC_ERR_INVALID_ARG, "key scratch is null");
+  return prefill_entry(ctx, desc, q, S, agent, ctx_len, block_table, table_stride, first_block, B_k, B_v, rope, cache, out, stream,
+                       key_scratch, key_scratch_bytes);
 }
 
 }  // extern "C"

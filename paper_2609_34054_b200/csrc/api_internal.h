@@ -108,6 +108,8 @@ struct PrefillArgs {
   const precc_layer_desc* d; const void* q; int S; int agent; int T; const int32_t* block_table; int first_block;
   const void* B_k; const void* B_v; const precc_cache* cache; void* out; cudaStream_t stream;
   const float* rope = nullptr; int max_pos = 0;      // rotary variant when rope != null
+  const void* k_scratch = nullptr;                   // adapted keys of this sequence in logical block order (rotary prefill
+  long long k_scratch_blocks = 0;                    // with scratch): the keys come from here, the values from the cache
 };
 
 
@@ -120,5 +122,8 @@ int32_t decode_ws_hd64(precc_ctx* ctx, int rk, int rv, const WsQuery& w);
 int32_t decode_ws_hd128(precc_ctx* ctx, int rk, int rv, const WsQuery& w);
 int32_t prefill_run_hd64(precc_ctx* ctx, const PrefillArgs& a, int rk, int rv);
 int32_t prefill_run_hd128(precc_ctx* ctx, const PrefillArgs& a, int rk, int rv);
+// 1 when the tensor-memory prefill kernel would take the call, 0 when not, negative on an unsupported rank pair
+int32_t prefill_tc_eligible_hd64(precc_ctx* ctx, const PrefillArgs& a, int rk, int rv);
+int32_t prefill_tc_eligible_hd128(precc_ctx* ctx, const PrefillArgs& a, int rk, int rv);
 
 }  // namespace precc

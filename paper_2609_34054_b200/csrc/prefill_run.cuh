@@ -32,8 +32,9 @@ struct PrefillRun {
     // instruction per 64-column slab instead of one per page)
     const bool contig = a.block_table == nullptr;
     const int box_rows = contig ? PTC_TOK : PAGE;
-    int32_t rc = contig ? make_map_cache4(ctx, &mk, a.cache->k_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
-                        : make_map2(ctx, &mk, a.cache->k_base, kv_rows, HD, PAGE, 64);
+    int32_t rc = a.k_scratch ? make_map_cache4(ctx, &mk, a.k_scratch, a.k_scratch_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
+                 : contig    ? make_map_cache4(ctx, &mk, a.cache->k_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
+                             : make_map2(ctx, &mk, a.cache->k_base, kv_rows, HD, PAGE, 64);
     if (rc) return rc;
     rc = contig ? make_map_cache4(ctx, &mv, a.cache->v_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
                 : make_map2(ctx, &mv, a.cache->v_base, kv_rows, HD, PAGE, 64);
@@ -46,7 +47,7 @@ struct PrefillRun {
     p.B_k = RK ? (const __nv_bfloat16*)a.B_k + (size_t)a.agent * RK * kvw : nullptr;
     p.B_v = RV ? (const __nv_bfloat16*)a.B_v + (size_t)a.agent * RV * kvw : nullptr;
     p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
-    p.S = a.S; p.T = a.T; p.first_block = a.first_block; p.contig = contig ? 1 : 0;
+    p.S = a.S; p.T = a.T; p.first_block = a.first_block; p.contig = contig ? 1 : 0; p.k_logical = a.k_scratch ? 1 : 0;
     p.longest_first = ctx->prefill_forward ? 0 : 1;
     p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.k_stages = ks; p.v_stages = vs;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
@@ -97,13 +98,22 @@ struct PrefillRun {
     PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, mk, mv, mlk, mlv, p));
     return PRECC_OK;
   }
-  static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
+  // whether the tensor-memory kernel takes this call (shape, cache size, alignment, diagnostic switch)
+  static bool tc_eligible(precc_ctx* ctx, const PrefillArgs& a) {
     if constexpr (PrefillTcCfg<HD, RK, RV>::supported) {
       const long long kv_rows = (long long)a.cache->n_blocks * a.d->n_kv_heads * PAGE;
       const bool aligned128 = ((reinterpret_cast<uintptr_t>(a.cache->k_base) | reinterpret_cast<uintptr_t>(a.cache->v_base) |
-                                reinterpret_cast<uintptr_t>(a.cache->lr_k) | reinterpret_cast<uintptr_t>(a.cache->lr_v)) & 127u) == 0;
-      if (kv_rows < (1ll << 31) && aligned128 && !ctx->force_simple_prefill) return run_tc(ctx, a);
+                                reinterpret_cast<uintptr_t>(a.cache->lr_k) | reinterpret_cast<uintptr_t>(a.cache->lr_v) |
+                                reinterpret_cast<uintptr_t>(a.k_scratch)) & 127u) == 0;
+      return kv_rows < (1ll << 31) && aligned128 && !ctx->force_simple_prefill;
     }
+    return false;
+  }
+  static int32_t run(precc_ctx* ctx, const PrefillArgs& a) {
+    if (tc_eligible(ctx, a)) {
+      if constexpr (PrefillTcCfg<HD, RK, RV>::supported) return run_tc(ctx, a);
+    }
+    if (a.k_scratch) return fail(ctx, PRECC_ERR_UNSUPPORTED, "prefill from a key scratch needs the tensor-memory kernel");
     return run_simple<false>(ctx, a);
   }
   // mma.sync kernel: oversized or unaligned caches, and the rotary variant
@@ -147,10 +157,18 @@ struct PrefillRunRope {
 };
 
 
+template <int HD, int RK, int RV>
+struct PrefillEligible {
+  static int32_t run(precc_ctx* ctx, const PrefillArgs& a) { return PrefillRun<HD, RK, RV>::tc_eligible(ctx, a) ? 1 : 0; }
+};
+
 }  // namespace precc
 
 #define PRECC_DEFINE_PREFILL_UNIT(HD)                                                                         \
   namespace precc {                                                                                           \
+  int32_t prefill_tc_eligible_hd##HD(precc_ctx* ctx, const PrefillArgs& a, int rk, int rv) {                  \
+    return dispatch_ranks<PrefillEligible, HD>(ctx, rk, rv, a);                                               \
+  }                                                                                                           \
   int32_t prefill_run_hd##HD(precc_ctx* ctx, const PrefillArgs& a, int rk, int rv) {                          \
     if (a.rope) return dispatch_ranks<PrefillRunRope, HD>(ctx, rk, rv, a);                                    \
     return dispatch_ranks<PrefillRun, HD>(ctx, rk, rv, a);                                                    \

@@ -47,6 +47,8 @@ struct PrefillTcParams {
   int tok_per_tile;            // 128 / group
   int k_stages, v_stages;      // depth of the key ring and of the value ring
   int contig;                  // 1: no block table; the tensor maps fetch a whole 128-token stage per box
+  int k_logical;               // 1: the key map covers a scratch copy of this sequence's keys in logical block order (whole-stage boxes
+                               //    from block 0), whatever the layout of the value side
   int longest_first;           // 1: block x = 0 takes the LAST row tile (longest causal reach), so the tail of the grid is short blocks
   float scale_log2, s_k, s_v;
   unsigned long long* trace;   // PRECC_PF_TRACE builds only: [steps][16] clock stamps of block (0, 0)
@@ -252,12 +254,12 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       const int live = min(PTC_TOK / PAGE, (t_end - t0 + PAGE - 1) / PAGE);
       const uint32_t st = is_k ? kring_u32 + (uint32_t)s * C::KSTAGE : vring_u32 + (uint32_t)s * C::VSTAGE;
       const uint32_t full = fullb + 8 * s;
-      if (p.contig) {
+      if (p.contig || (is_k && p.k_logical)) {
         // consecutive physical blocks: one box per 64-column slab covers all eight pages of the stage
         // (4-D map [block][kv head][16][hd]); blocks past the cache end arrive as zeros
         if (lane == 0) {
           mbar_expect_tx(full, (PTC_TOK / PAGE) * (is_k ? C::K_PAGE_TX : C::V_PAGE_TX));
-          const int blk0 = p.first_block + (jb + j) * (PTC_TOK / PAGE);
+          const int blk0 = ((is_k && p.k_logical) ? 0 : p.first_block) + (jb + j) * (PTC_TOK / PAGE);
           if (is_k) {
 #pragma unroll
             for (int sl = 0; sl < C::SLABS; ++sl) tma_load_4d(st + sl * C::SLAB_BYTES, &map_k, sl * 64, 0, g, blk0, full);

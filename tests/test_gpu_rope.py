@@ -207,6 +207,69 @@ def test_prefill_rope_shapes(px, hd, n_q, n_kv, r, T, S):
     assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("hd,n_q,n_kv,r,T,S,paged", [(64, 8, 2, 16, 200, 40, False), (128, 8, 2, 32, 515, 130, True), (128, 4, 1, 8, 90, 7, False),
+                                                     (128, 8, 1, 64, 33, 20, True), (64, 16, 2, 32, 333, 5, False), (128, 8, 2, 16, 2300, 33, True)])
+def test_prefill_rope_through_a_key_scratch(px, hd, n_q, n_kv, r, T, S, paged):
+    """The fast rotary prefill: the sequence's adapted rotary keys are written to a scratch area once, then the
+    tensor-core kernel runs on them.  Against the definition, against the per-tile kernel, paged and contiguous,
+    a short turn over a longer context (split over a cluster), scratch reuse, and the error paths."""
+    geo = I.Geometry(d_model=192, n_q=n_q, n_kv=n_kv, hd=hd, n_agents=2, rank_k=r, rank_v=r, alpha=2.0 * r)
+    nb = (T + S + 15) // 16
+    pool = nb + 5 if paged else nb
+    L = Layer(px, geo, seed=18, n_blocks=pool, tag="rps")
+    H = I.hidden_states(T + S, geo, 18, "rps.H")
+    table = rope_table(T + S + 3, hd)
+    cos, sin = O.rope_tables(T + S + 3, hd)
+    bt = I.permutation(pool, 18, "rps.bt")[:nb].to(torch.int32).cuda() if paged else None
+    slots = (bt.long().cpu()[:, None] * 16 + torch.arange(16)[None, :]).reshape(-1)[:T + S].to(torch.int32).cuda() if paged else None
+    pos = torch.arange(T + S, dtype=torch.int32).cuda()
+    px.rebase_project_rope(L.desc, H.cuda(), L.W_packed, L.cache, table, 0, slots, positions=pos)
+    px.lr_precompute(L.desc, H.cuda(), L.A_packed, L.cache, 0, slots)
+    w = L.w_np
+    q = I.queries(S, geo, 18, "rps.q", gain=3.0)
+    nbytes = px.prefill_rope_scratch_bytes(L.desc, T, S)
+    assert nbytes == ((nb + 7) // 8 * 8) * n_kv * 16 * hd * 2
+    scratch = torch.full((nbytes + 256,), 0x7f, dtype=torch.uint8, device="cuda")       # NaN-ish fill, guard bytes behind
+    out = torch.full_like(q, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope_scratch(L.desc, q.cuda(), 1, T, L.B_k, L.B_v, table, L.cache, out, scratch[:nbytes], bt)
+    torch.cuda.synchronize()
+    assert (scratch[nbytes:] == 0x7f).all()                                              # nothing written behind the area
+    ref = O.lr_prefill_reference_rope(f64(q), 1, T, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                      geo.scale_k, geo.scale_v, n_kv, cos, sin)
+    assert_close(f64(out), ref, f"rope prefill through scratch hd{hd} r{r}")
+    slow = torch.full_like(q, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope(L.desc, q.cuda(), 1, T, L.B_k, L.B_v, table, L.cache, slow, bt)
+    torch.cuda.synchronize()
+    assert_close(f64(out), f64(slow), "scratch path against the per-tile kernel")
+    # the scratch holds the adapted rotary keys of the sequence in logical order: check a few rows against the definition
+    ks = scratch[:nbytes].view(torch.bfloat16).view(-1, n_kv, 16, hd)
+    Ka = O.rope_rotate(O.adapted_projection(f64(H), w["W_k"], w["A_k"][1], w["B_k"][1], geo.scale_k), np.arange(T + S), n_kv, cos, sin)
+    for t in (0, T - 1, T + S - 1):
+        got = f64(ks[t // 16, :, t % 16, :]).reshape(-1)
+        assert (np.abs(got - Ka[t]) <= 2.0 ** -7 * np.abs(Ka[t]) + 3e-3).all()
+    # second call on the same scratch (another agent): the area is simply overwritten
+    out2 = torch.full_like(q, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope_scratch(L.desc, q.cuda(), 0, T, L.B_k, L.B_v, table, L.cache, out2, scratch[:nbytes], bt)
+    torch.cuda.synchronize()
+    ref0 = O.lr_prefill_reference_rope(f64(q), 0, T, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"],
+                                       geo.scale_k, geo.scale_v, n_kv, cos, sin)
+    assert_close(f64(out2), ref0, "second agent through the same scratch")
+    # adapter-free view: the scratch is not needed and not touched
+    before = scratch.clone()
+    a = torch.full_like(q, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope_scratch(L.desc, q.cuda(), -1, T, L.B_k, L.B_v, table, L.cache, a, scratch[:nbytes], bt)
+    torch.cuda.synchronize()
+    assert torch.equal(scratch, before)
+    b = torch.full_like(q, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope(L.desc, q.cuda(), -1, T, L.B_k, L.B_v, table, L.cache, b, bt)
+    assert torch.equal(a, b)
+    with pytest.raises(PreccError):                      # too small
+        px.lr_attend_prefill_rope_scratch(L.desc, q.cuda(), 1, T, L.B_k, L.B_v, table, L.cache, out, scratch[:nbytes - 128], bt)
+    with pytest.raises(PreccError):                      # misaligned
+        px.lr_attend_prefill_rope_scratch(L.desc, q.cuda(), 1, T, L.B_k, L.B_v, table, L.cache, out, scratch[64:nbytes + 64], bt)
+    assert px.poll_status() == 0
+
+
 def test_rope_invalid_arguments(px):
     geo = I.Geometry(d_model=192, n_q=8, n_kv=2, hd=64, n_agents=2, rank_k=16, rank_v=16, alpha=32.0)
     L = Layer(px, geo, seed=7, n_blocks=8, tag="ri", fill=0.0)
