@@ -242,8 +242,23 @@ static int32_t prefill_entry(precc_ctx* ctx, const precc_layer_desc* desc, const
   x.block_table = block_table; x.scratch = (__nv_bfloat16*)k_scratch; x.status = ctx->status;
   x.n_blocks = cache->n_blocks; x.first_block = first_block; x.n_tokens = ctx_len + S;
   x.n_kv = desc->n_kv_heads; x.hd = desc->head_dim; x.rk = desc->rank_k; x.max_pos = rope->max_pos; x.s_k = desc->lora_scale_k;
-  rope_expand_keys_kernel<<<(unsigned)out_blocks, RX_THREADS, 0, (cudaStream_t)stream>>>(x);
-  PRECC_CUDA(ctx, cudaGetLastError());
+  x.n_out_blocks = (int)out_blocks;
+  const int n_tasks = desc->n_kv_heads * (desc->head_dim / 32);
+  auto launch = [&](auto kern, size_t xs, int group_tasks) -> int32_t {
+    PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, (int)xs));
+    const int groups = (n_tasks + group_tasks - 1) / group_tasks;
+    long long gx = 4ll * ctx->sm_count / groups;          // two resident blocks per SM, two rounds
+    if (gx < 1) gx = 1;
+    if (gx > out_blocks) gx = out_blocks;
+    kern<<<dim3((unsigned)gx, (unsigned)groups), RX_THREADS, xs, (cudaStream_t)stream>>>(x);
+    PRECC_CUDA(ctx, cudaGetLastError());
+    return PRECC_OK;
+  };
+  int32_t xrc;
+  if (desc->rank_k <= 16) xrc = launch(rope_expand_keys_kernel<1>, rope_expand_smem_bytes<1>(), RxCfg<1>::GROUP_TASKS);
+  else if (desc->rank_k == 32) xrc = launch(rope_expand_keys_kernel<2>, rope_expand_smem_bytes<2>(), RxCfg<2>::GROUP_TASKS);
+  else xrc = launch(rope_expand_keys_kernel<4>, rope_expand_smem_bytes<4>(), RxCfg<4>::GROUP_TASKS);
+  if (xrc) return xrc;
   return desc->head_dim == 64 ? prefill_run_hd64(ctx, b, 0, rv) : prefill_run_hd128(ctx, b, 0, rv);
 }
 

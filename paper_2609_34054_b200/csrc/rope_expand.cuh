@@ -5,8 +5,7 @@
 // with K_base_rot the cache's (already rotated) base keys, L^K the agent's unrotated LR rows and token t at
 // position t.  The result goes to a caller-provided scratch area in LOGICAL block order, layout
 // [block][kv head][16][hd] like the cache, so that the tensor-memory prefill kernel can stream it as its key
-// operand with whole-stage boxes and no key-side adapter at all.  One thread block per 16-token block; a thread
-// owns two adjacent columns of the lower half of a head and their partners in the upper half.
+// operand with whole-stage boxes and no key-side adapter at all.  One thread block per 16-token block.
 #pragma once
 #include "common.cuh"
 
@@ -23,73 +22,153 @@ struct RopeExpandParams {
   long long n_blocks;            // physical blocks of the cache
   int first_block;               // physical block of logical block 0 when block_table is null
   int n_tokens;                  // tokens of the sequence (context + turn); rows past it are written as zeros
+  int n_out_blocks;              // cache blocks to write (whole 128-token stages)
   int n_kv, hd, rk, max_pos;
   float s_k;
 };
 
 constexpr int RX_THREADS = 256;
+constexpr int RX_WARPS = RX_THREADS / 32;
 
-__global__ void __launch_bounds__(RX_THREADS)
+// E = L^K B^K on the tensor cores (mma.sync m16n8k16: the 16 tokens of a cache block on the M axis, rank on K, columns
+// on N).  A task is 16 adjacent columns of the lower half of one head together with their partners in the upper half;
+// a warp owns TPW tasks for the whole kernel and keeps their B^K fragments in registers, a thread block owns a group
+// of 8 TPW tasks (blockIdx.y) and walks over the sequence's cache blocks (blockIdx.x, persistent).  Per cache block:
+// L^K fragments straight from global memory, the MMAs, the rotation, the scaled term parked in shared memory, then
+// base keys + term -> scratch with 16-byte accesses, consecutive threads on consecutive pieces of a row.
+// KS = k steps of 16 (rank 8 and 16: 1, rank 32: 2, rank 64: 4).
+template <int KS>
+struct RxCfg {
+  static constexpr int TPW = KS <= 2 ? 2 : 1;            // tasks per warp: TPW * 4 tiles * KS * 2 fragment registers <= 32
+  static constexpr int GROUP_TASKS = RX_WARPS * TPW;
+};
+
+template <int KS>
+__global__ void __launch_bounds__(RX_THREADS, 2)
 rope_expand_keys_kernel(const RopeExpandParams p) {
-  __shared__ __align__(16) float Lf[64 * PAGE];          // s_k L^K of the block's tokens, [rank][token]
-  const int lb = blockIdx.x;
+  constexpr int TPW = RxCfg<KS>::TPW;
+  extern __shared__ __align__(16) float Es[];            // s_k RoPE(L^K B^K) of one cache block, [task of the group][token][32 columns]
   const int hd = p.hd, rk = p.rk;
   const int kvw = p.n_kv * hd;
-  __nv_bfloat16* dst_blk = p.scratch + (size_t)lb * p.n_kv * PAGE * hd;
-  const int t0 = lb * PAGE;
-  if (t0 >= p.n_tokens) {                                // padding up to a whole 128-token stage: defined contents
-    for (int i = threadIdx.x; i < p.n_kv * PAGE * hd / 8; i += RX_THREADS) reinterpret_cast<uint4*>(dst_blk)[i] = make_uint4(0u, 0u, 0u, 0u);
-    return;
-  }
-  int ph = p.block_table ? __ldg(p.block_table + lb) : p.first_block + lb;
-  if (ph < 0 || ph >= p.n_blocks) {
-    if (threadIdx.x == 0) atomicOr(p.status, StatusBits::BAD_INDEX);
-    ph = 0;
-  }
-  for (int i = threadIdx.x; i < PAGE * rk; i += RX_THREADS) {
-    const int tok = i / rk, j = i - tok * rk;
-    Lf[j * PAGE + tok] = p.s_k * __bfloat162float(p.lr_k[((size_t)ph * PAGE + tok) * rk + j]);
-  }
-  __syncthreads();
-  const int units = p.n_kv * (hd / 4);
-  for (int u = threadIdx.x; u < units; u += RX_THREADS) {
-    const int g = u / (hd / 4), cp = u - g * (hd / 4), c = 2 * cp;
-    const __nv_bfloat16* bcol = p.B_k + (size_t)g * hd + c;
-    const __nv_bfloat16* ksrc = p.k_base + ((size_t)ph * p.n_kv + g) * PAGE * hd + c;
-    __nv_bfloat16* kdst = dst_blk + (size_t)g * PAGE * hd + c;
-#pragma unroll 1
-    for (int half = 0; half < 2; ++half) {
-      float lo0[8], lo1[8], hi0[8], hi1[8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = lane >> 2, q2 = (lane & 3) * 2;          // accumulator rows r, r + 8; columns q2, q2 + 1 of an 8-column tile
+  const int tasks_per_head = hd / 32;                    // 16 lower-half columns per task
+  const int n_tasks = p.n_kv * tasks_per_head;
+  const int task0 = blockIdx.y * RxCfg<KS>::GROUP_TASKS + warp * TPW;
+  // ---- this warp's B^K fragments (k = rank, n = column), zero beyond the rank and beyond the last task
+  uint32_t bfr[TPW][4][KS][2];
 #pragma unroll
-      for (int t = 0; t < 8; ++t) { lo0[t] = lo1[t] = hi0[t] = hi1[t] = 0.f; }
-      for (int j = 0; j < rk; ++j) {
-        const float2 bl = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(bcol + (size_t)j * kvw));
-        const float2 bh = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(bcol + (size_t)j * kvw + hd / 2));
-        const float4 la = *reinterpret_cast<const float4*>(Lf + j * PAGE + half * 8);
-        const float4 lb4 = *reinterpret_cast<const float4*>(Lf + j * PAGE + half * 8 + 4);
-        const float l8[8] = {la.x, la.y, la.z, la.w, lb4.x, lb4.y, lb4.z, lb4.w};
+  for (int tw = 0; tw < TPW; ++tw) {
+    const int task = task0 + tw;
+    const int g = task / tasks_per_head, c0 = (task - g * tasks_per_head) * 16;
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-          lo0[t] += l8[t] * bl.x; lo1[t] += l8[t] * bl.y;
-          hi0[t] += l8[t] * bh.x; hi1[t] += l8[t] * bh.y;
-        }
-      }
+    for (int t = 0; t < 4; ++t) {
+      const int col = g * hd + c0 + (t & 1) * 8 + (t >> 1) * (hd / 2) + r;          // B operand: n = lane >> 2
 #pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        const int tok = half * 8 + t, pos = t0 + tok;
-        __nv_bfloat162 olo = __floats2bfloat162_rn(0.f, 0.f), ohi = olo;
-        if (pos < p.n_tokens) {
-          const float4 cs = __ldg(p.rope + (size_t)min(pos, p.max_pos - 1) * (hd / 4) + cp);
-          const float2 kl = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(ksrc + (size_t)tok * hd));
-          const float2 kh = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(ksrc + (size_t)tok * hd + hd / 2));
-          olo = __floats2bfloat162_rn(kl.x + (lo0[t] * cs.x - hi0[t] * cs.y), kl.y + (lo1[t] * cs.z - hi1[t] * cs.w));
-          ohi = __floats2bfloat162_rn(kh.x + (hi0[t] * cs.x + lo0[t] * cs.y), kh.y + (hi1[t] * cs.z + lo1[t] * cs.w));
-        }
-        *reinterpret_cast<__nv_bfloat162*>(kdst + (size_t)tok * hd) = olo;
-        *reinterpret_cast<__nv_bfloat162*>(kdst + (size_t)tok * hd + hd / 2) = ohi;
+      for (int ks = 0; ks < KS; ++ks) {
+        const int k0 = ks * 16 + q2;
+        auto bk = [&](int k) -> uint32_t {
+          return (task < n_tasks && k < rk) ? (uint32_t)__bfloat16_as_ushort(p.B_k[(size_t)k * kvw + col]) : 0u;
+        };
+        bfr[tw][t][ks][0] = bk(k0) | (bk(k0 + 1) << 16);
+        bfr[tw][t][ks][1] = bk(k0 + 8) | (bk(k0 + 9) << 16);
       }
     }
   }
+  const int n_out_blocks = gridDim.x ? p.n_out_blocks : 0;
+  for (int lb = blockIdx.x; lb < n_out_blocks; lb += gridDim.x) {
+    const int t0 = lb * PAGE;
+    __nv_bfloat16* dst_blk = p.scratch + (size_t)lb * p.n_kv * PAGE * hd;
+    const bool pad = t0 >= p.n_tokens;                   // padding up to a whole 128-token stage: zeros
+    int ph = 0;
+    if (!pad) {
+      ph = p.block_table ? __ldg(p.block_table + lb) : p.first_block + lb;
+      if (ph < 0 || ph >= p.n_blocks) {
+        if (threadIdx.x == 0 && blockIdx.y == 0) atomicOr(p.status, StatusBits::BAD_INDEX);
+        ph = 0;
+      }
+    }
+    // the base keys this thread will add the term to: requested first, so that their DRAM round trip runs under the MMAs
+    const __nv_bfloat16* src_blk = p.k_base + (size_t)ph * p.n_kv * PAGE * hd;
+    const int group_tasks = min(RxCfg<KS>::GROUP_TASKS, n_tasks - (int)blockIdx.y * RxCfg<KS>::GROUP_TASKS);
+    constexpr int PIECES = RxCfg<KS>::GROUP_TASKS * PAGE * 4 / RX_THREADS;
+    uint4 kb[PIECES];
+    size_t off[PIECES];
+#pragma unroll
+    for (int k = 0; k < PIECES; ++k) {
+      const int i = threadIdx.x + k * RX_THREADS;
+      const int pc = i & 3, tok = (i >> 2) % PAGE, tg = i / (4 * PAGE);               // piece, token, task in group
+      const int task = blockIdx.y * RxCfg<KS>::GROUP_TASKS + tg;
+      const int g = task / tasks_per_head, c0 = (task - g * tasks_per_head) * 16;
+      off[k] = ((size_t)g * PAGE + tok) * hd + c0 + (pc & 1) * 8 + (pc >> 1) * (hd / 2);
+      kb[k] = (tg < group_tasks && !pad && t0 + tok < p.n_tokens) ? __ldg(reinterpret_cast<const uint4*>(src_blk + off[k])) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    if (!pad) {
+      // A fragments: L^K rows r and r + 8 of the block (row-major [16][rk]); rank 8 fills half a k step
+      uint32_t afr[KS][4];
+      const __nv_bfloat16* lrow = p.lr_k + ((size_t)ph * PAGE + r) * rk;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int k = ks * 16 + q2;
+        afr[ks][0] = k < rk ? __ldg(reinterpret_cast<const uint32_t*>(lrow + k)) : 0u;
+        afr[ks][1] = k < rk ? __ldg(reinterpret_cast<const uint32_t*>(lrow + 8 * rk + k)) : 0u;
+        afr[ks][2] = k + 8 < rk ? __ldg(reinterpret_cast<const uint32_t*>(lrow + k + 8)) : 0u;
+        afr[ks][3] = k + 8 < rk ? __ldg(reinterpret_cast<const uint32_t*>(lrow + 8 * rk + k + 8)) : 0u;
+      }
+#pragma unroll
+      for (int tw = 0; tw < TPW; ++tw) {
+        const int task = task0 + tw;
+        if (task >= n_tasks) break;
+        const int g = task / tasks_per_head, c0 = (task - g * tasks_per_head) * 16;
+        float acc[4][4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
+#pragma unroll
+          for (int ks = 0; ks < KS; ++ks) mma_bf16_16816(acc[t], afr[ks], bfr[tw][t][ks][0], bfr[tw][t][ks][1]);
+        }
+        // rotate (lower tile t with upper tile t + 2), park the scaled term: [task in group][token][lower 16 | upper 16]
+        float* eb = Es + (size_t)(warp * TPW + tw) * PAGE * 32;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          const int cl = t * 8 + q2;                      // even column inside the task's lower 16
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int tok = r + 8 * h, pos = t0 + tok;
+            const float lo0 = p.s_k * acc[t][2 * h], lo1 = p.s_k * acc[t][2 * h + 1];
+            const float hi0 = p.s_k * acc[t + 2][2 * h], hi1 = p.s_k * acc[t + 2][2 * h + 1];
+            const float4 cs = __ldg(p.rope + (size_t)min(pos, p.max_pos - 1) * (hd / 4) + (c0 + cl) / 2);
+            *reinterpret_cast<float2*>(eb + tok * 32 + cl) = make_float2(lo0 * cs.x - hi0 * cs.y, lo1 * cs.z - hi1 * cs.w);
+            *reinterpret_cast<float2*>(eb + tok * 32 + 16 + cl) = make_float2(hi0 * cs.x + lo0 * cs.y, hi1 * cs.z + lo1 * cs.w);
+          }
+        }
+      }
+    }
+    __syncthreads();
+    // base keys + term -> scratch: a piece is 8 columns (16 bytes) of one token; per task and token 2 pieces of the
+    // lower half and 2 of the upper half
+#pragma unroll
+    for (int k = 0; k < PIECES; ++k) {
+      const int i = threadIdx.x + k * RX_THREADS;
+      const int pc = i & 3, tok = (i >> 2) % PAGE, tg = i / (4 * PAGE);
+      if (tg >= group_tasks) continue;
+      uint4 o = make_uint4(0u, 0u, 0u, 0u);
+      if (!pad && t0 + tok < p.n_tokens) {
+        const float* e = Es + (size_t)tg * PAGE * 32 + tok * 32 + pc * 8;
+        const float4 e0 = *reinterpret_cast<const float4*>(e), e1 = *reinterpret_cast<const float4*>(e + 4);
+        auto add2 = [](uint32_t k2, float a, float b) -> uint32_t {
+          const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&k2));
+          return pack_bf16(f.x + a, f.y + b);
+        };
+        o = make_uint4(add2(kb[k].x, e0.x, e0.y), add2(kb[k].y, e0.z, e0.w), add2(kb[k].z, e1.x, e1.y), add2(kb[k].w, e1.z, e1.w));
+      }
+      *reinterpret_cast<uint4*>(dst_blk + off[k]) = o;
+    }
+    __syncthreads();                                     // the parked term is reused by the next cache block
+  }
 }
+
+template <int KS>
+inline size_t rope_expand_smem_bytes() { return (size_t)RxCfg<KS>::GROUP_TASKS * PAGE * 32 * sizeof(float); }
 
 }  // namespace precc
