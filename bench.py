@@ -366,6 +366,15 @@ def extra_turn(px, T: int, S: int, seed: int = 0, cpu_seconds: float = 0.0):
     us_sturn = _event_us(torch, short_turn, 10)
     short = {"S": S2, "projection_us": us_sproj, "prefill_attention_us": us_sattn, "turn_us_per_layer": us_sturn,
              "turn_ttft_ms_32_layers": us_sturn * C3_LAYERS_FOR_TTFT / 1e3}
+    # rotary keys (Appendix D.2) on the same turn: the per-tile kernel, and the scratch form (adapted rotary keys of the
+    # sequence written once, then the tensor-memory kernel); the cache contents are taken as they are - only times matter here
+    table = I.rope_table(T + S, geo.hd)
+    scratch = torch.empty(px.prefill_rope_scratch_bytes(desc, T, S), dtype=torch.uint8, device="cuda")
+    us_rope_tile = _event_us(torch, lambda: px.lr_attend_prefill_rope(desc, q, cur, T, w["B_k"], w["B_v"], table, cache, out), 2)
+    us_rope_scr = _event_us(torch, lambda: px.lr_attend_prefill_rope_scratch(desc, q, cur, T, w["B_k"], w["B_v"], table, cache, out, scratch), 5)
+    rotary = {"prefill_per_tile_kernel_us": us_rope_tile, "prefill_through_scratch_us": us_rope_scr,
+              "scratch_bytes": scratch.numel(), "position_free_us": us_attn}
+    del scratch
     pk = measured_tensor_peaks()
     hbm, hbm_kind = measured_peak()
     tf_attn = fl_attn / us_attn / 1e6
@@ -382,6 +391,7 @@ def extra_turn(px, T: int, S: int, seed: int = 0, cpu_seconds: float = 0.0):
            "turn_projection_us": us_tproj,
            "turn_us_per_layer": us_turn, "turn_ttft_ms_32_layers": us_turn * C3_LAYERS_FOR_TTFT / 1e3,
            "prefill_attention": {"us": us_attn, "tflops": tf_attn},
+           "rotary_prefill": rotary,
            "rebase_us_per_layer": us_reb, "peaks": pk,
            "roofline_prefill": {"bound": "tensor", "kernel": "lr_attend_prefill_tc_kernel<128,32,32>", "achieved": tf_attn,
                                 "peak": pk["bf16_tflops_burst"], "peak_kind": pk["peak_kind"] + " (burst)", "unit": "TFLOP/s",
