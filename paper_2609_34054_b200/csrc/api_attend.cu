@@ -247,7 +247,7 @@ static int32_t prefill_entry(precc_ctx* ctx, const precc_layer_desc* desc, const
   auto launch = [&](auto kern, size_t xs, int group_tasks) -> int32_t {
     PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, (int)xs));
     const int groups = (n_tasks + group_tasks - 1) / group_tasks;
-    long long gx = 4ll * ctx->sm_count / groups;          // two resident blocks per SM, two rounds
+    long long gx = 2ll * ctx->sm_count / groups;          // two resident blocks per SM: each walks its share of the cache blocks
     if (gx < 1) gx = 1;
     if (gx > out_blocks) gx = out_blocks;
     kern<<<dim3((unsigned)gx, (unsigned)groups), RX_THREADS, xs, (cudaStream_t)stream>>>(x);
