@@ -257,6 +257,12 @@ def test_random_rope_shapes(px, i):
     torch.cuda.synchronize()
     refp = O.lr_prefill_reference_rope(f64(qs), 1, T, *args, geo.scale_k, geo.scale_v, n_kv, cos, sin)
     assert_close(f64(outp), refp, f"case {i} rope prefill (hd{hd} G{G} kv{n_kv} r{r} T{T} S{S})")
+    # the same turn through the key scratch (adapted rotary keys written once, then the tensor-core kernel)
+    scratch = torch.empty(px.prefill_rope_scratch_bytes(L.desc, T, S), dtype=torch.uint8, device="cuda")
+    outs = torch.full_like(qs, float("nan"), device="cuda")
+    px.lr_attend_prefill_rope_scratch(L.desc, qs.cuda(), 1, T, L.B_k, L.B_v, table, L.cache, outs, scratch)
+    torch.cuda.synchronize()
+    assert_close(f64(outs), refp, f"case {i} rope prefill through scratch (hd{hd} G{G} kv{n_kv} r{r} T{T} S{S})")
 
 
 def _shard_case(i: int):
