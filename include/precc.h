@@ -106,10 +106,12 @@ int32_t precc_sm_count(const precc_ctx* ctx);
 /* Tracing (optional).  Give the context a caller-owned DEVICE buffer of n_blocks * 16 uint64 entries;
  * while it is set, each thread block of precc_lr_attend_decode whose grid has at most n_blocks blocks
  * records the GPU nanosecond timer at points of its life at entry [block][point]: 0 start, 1 indices
- * read, 2 stream issued, 3 query fold ready, 4 first tile landed, 5 stream done, 6 record published,
- * 7 done, 11 all warps of the block have left the stream, and for the merging block 8 partials gathered, 9 weights
- * ready, 10 merged (others stay 0); blocks of the cluster schedule also record 12 cluster barrier passed, and
- * store the id of the SM they run on at entry 15.  Pass NULL to switch tracing off (the default).  There is no paper counterpart. */
+ * read, 2 stream issued, 3 query fold ready, 4 first tile landed, 5 stream done, 7 done, 8 / 9 just before and after
+ * the wait for the preceding kernel, 11 all warps of the block have left the stream, 13 warp records written, 14 block
+ * merge done.  Ticket schedule: 6 record published, and the merging block reuses 8 and 9 - partials gathered, weights
+ * ready - and records 10 merged.  Cluster schedule: 6 sends issued, 12 everything addressed to the block received, and the id of the SM
+ * the block runs on at entry 15.  Entries not written stay as they were.  Pass NULL to switch tracing off (the
+ * default).  There is no paper counterpart. */
 int32_t precc_set_trace_buffer(precc_ctx* ctx, void* buffer, size_t n_blocks);
 
 /* Read the device status word accumulated by kernels launched through `ctx`, then clear it.
