@@ -281,6 +281,28 @@ int32_t precc_lr_attend_prefill(precc_ctx* ctx, const precc_layer_desc* desc, co
                                 const void* B_k, const void* B_v, const precc_cache* cache,
                                 void* out, void* stream);
 
+/* precc_lr_attend_prefill with a caller-provided workspace (Section 3.1; the workspace has no counterpart
+ * in the paper).  A turn whose (row tile, kv head) blocks fill more than half of the SMs but not all of
+ * them - 512 new tokens of 8 kv heads are 128 blocks on 148 SMs - runs in one wave that leaves SMs idle.
+ * With a workspace each block stops some way before the end of its context and helper blocks on the idle
+ * SMs take the remaining steps of all tiles; the pieces of a tile are written to the workspace as fp32
+ * partial results (maximum, denominator, numerator) and merged, in a fixed order, by whichever block
+ * finishes last.  Same arguments and errors as precc_lr_attend_prefill, plus
+ *   ws, ws_bytes  device, 256-byte aligned (PRECC_ERR_MISALIGNED otherwise); precc_prefill_ws_bytes(ctx,
+ *                 desc, S) bytes are always enough; contents on entry do not matter, the call clears what
+ *                 must start at zero on `stream`; the caller owns it and may reuse it for the next call on
+ *                 the same stream.  Two calls that may overlap on the GPU need separate workspaces.
+ * With ws == NULL, a workspace that is too small, a turn length for which precc_prefill_ws_bytes returns 0,
+ * a short context, or where the tensor-memory kernel does not take the call, the call behaves exactly like
+ * precc_lr_attend_prefill.  Where helper blocks are used the result differs from precc_lr_attend_prefill
+ * in rounding only (another summation order over the context); it is the same from run to run. */
+size_t precc_prefill_ws_bytes(const precc_ctx* ctx, const precc_layer_desc* desc, int32_t S);
+int32_t precc_lr_attend_prefill_ws(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S,
+                                   int32_t agent, int32_t ctx_len, const int32_t* block_table,
+                                   int32_t table_stride, int32_t first_block,
+                                   const void* B_k, const void* B_v, const precc_cache* cache,
+                                   void* out, void* ws, size_t ws_bytes, void* stream);
+
 /* ---------------------------------------------------------------- rotary keys (Appendix D.2)
  * With a rotary position embedding the agent's key row of token t is RoPE_t(H_t (W_k + s_k A B)): the
  * rotation sits between the rank-r term and the query, so the rank-r term must be expanded to full

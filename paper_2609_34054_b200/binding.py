@@ -26,6 +26,7 @@ EXPORTS = [
     "precc_turn_project_rows", "precc_partial_record_floats", "precc_lr_attend_decode_partial", "precc_combine_partials",
     "precc_set_wait_limit", "precc_selftest_wait_timeout",
     "precc_prefill_rope_scratch_bytes", "precc_lr_attend_prefill_rope_scratch",
+    "precc_prefill_ws_bytes", "precc_lr_attend_prefill_ws",
 ]
 
 
@@ -85,6 +86,10 @@ def load_library() -> C.CDLL:
                                                   C.POINTER(CacheDesc), vp, vp]
     lib.precc_lr_attend_prefill.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp,
                                             C.POINTER(CacheDesc), vp, vp]
+    lib.precc_prefill_ws_bytes.argtypes = [vp, C.POINTER(LayerDesc), i32]
+    lib.precc_prefill_ws_bytes.restype = sz
+    lib.precc_lr_attend_prefill_ws.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, i32, i32, vp, i32, i32, vp, vp,
+                                               C.POINTER(CacheDesc), vp, vp, sz, vp]
     rp = C.POINTER(RopeDesc)
     lib.precc_rebase_project_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, rp, C.POINTER(CacheDesc), vp]
     lib.precc_turn_project_rope.argtypes = [vp, C.POINTER(LayerDesc), vp, i32, vp, vp, i64, u64, rp, C.POINTER(CacheDesc), vp]
@@ -397,3 +402,17 @@ class Precc:
         self._check(self.lib.precc_lr_attend_prefill(
             self.h, C.byref(desc), _ptr(q), q.shape[0], agent, ctx_len, _ptr(block_table), stride, first_block,
             _ptr(B_k), _ptr(B_v), C.byref(cd), _ptr(out), _stream()), "precc_lr_attend_prefill")
+
+    def prefill_ws_bytes(self, desc: LayerDesc, S: int) -> int:
+        return int(self.lib.precc_prefill_ws_bytes(self.h, C.byref(desc), S))
+
+    def lr_attend_prefill_ws(self, desc: LayerDesc, q: torch.Tensor, agent: int, ctx_len: int, B_k, B_v, cache: Cache,
+                             out: torch.Tensor, workspace: Optional[torch.Tensor], block_table: Optional[torch.Tensor] = None,
+                             first_block: int = 0):
+        """Prefill with a caller-provided workspace (uint8 tensor of prefill_ws_bytes, or None): helper blocks on idle SMs."""
+        cd = cache.desc()
+        stride = block_table.numel() if block_table is not None else 0
+        nbytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        self._check(self.lib.precc_lr_attend_prefill_ws(
+            self.h, C.byref(desc), _ptr(q), q.shape[0], agent, ctx_len, _ptr(block_table), stride, first_block,
+            _ptr(B_k), _ptr(B_v), C.byref(cd), _ptr(out), _ptr(workspace), nbytes, _stream()), "precc_lr_attend_prefill_ws")

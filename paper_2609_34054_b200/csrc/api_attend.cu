@@ -194,7 +194,8 @@ int32_t precc_lr_attend_decode_static(precc_ctx* ctx, const precc_layer_desc* de
 static int32_t prefill_entry(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
                              int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
                              const void* B_k, const void* B_v, const precc_rope* rope, const precc_cache* cache, void* out,
-                             void* stream, void* k_scratch = nullptr, size_t k_scratch_bytes = 0) {
+                             void* stream, void* k_scratch = nullptr, size_t k_scratch_bytes = 0, void* ws = nullptr,
+                             size_t ws_bytes = 0) {
   int32_t rc = check_desc(ctx, desc);
   if (rc) return rc;
   if (S < 0 || ctx_len < 0) return fail(ctx, PRECC_ERR_INVALID_ARG, "S < 0 or ctx_len < 0");
@@ -212,6 +213,10 @@ static int32_t prefill_entry(precc_ctx* ctx, const precc_layer_desc* desc, const
     return fail(ctx, PRECC_ERR_INVALID_ARG, "blocks [%d, %lld) outside the cache", first_block, first_block + need_blocks);
   if ((long long)S * (desc->n_q_heads / desc->n_kv_heads) > (long long)PF_ROWS * 65535) return fail(ctx, PRECC_ERR_UNSUPPORTED, "S too large");
   PrefillArgs a{desc, q, S, neutral ? 0 : agent, ctx_len, block_table, first_block, B_k, B_v, cache, out, (cudaStream_t)stream};
+  if (ws) {
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return fail(ctx, PRECC_ERR_MISALIGNED, "prefill workspace not 256-byte aligned");
+    a.ws = ws; a.ws_bytes = ws_bytes;
+  }
   const int rk = neutral ? 0 : desc->rank_k, rv = neutral ? 0 : desc->rank_v;
   auto run = [&]() { return desc->head_dim == 64 ? prefill_run_hd64(ctx, a, rk, rv) : prefill_run_hd128(ctx, a, rk, rv); };
   if (!rope) return run();
@@ -275,6 +280,27 @@ int32_t precc_lr_attend_prefill_rope(precc_ctx* ctx, const precc_layer_desc* des
   if (!ctx) return PRECC_ERR_INVALID_ARG;
   if (!rope) return fail(ctx, PRECC_ERR_INVALID_ARG, "rope is null");
   return prefill_entry(ctx, desc, q, S, agent, ctx_len, block_table, table_stride, first_block, B_k, B_v, rope, cache, out, stream);
+}
+
+size_t precc_prefill_ws_bytes(const precc_ctx* ctx, const precc_layer_desc* desc, int32_t S) {
+  if (!ctx || !desc || S <= 0 || desc->n_kv_heads <= 0 || desc->n_q_heads < desc->n_kv_heads || desc->head_dim <= 0) return 0;
+  const int G = desc->n_q_heads / desc->n_kv_heads;
+  if (G > 128) return 0;
+  const int tok_per_tile = 128 / G;
+  const long long tiles = (long long)((S + tok_per_tile - 1) / tok_per_tile) * desc->n_kv_heads;
+  if (tiles * 2 <= ctx->sm_count || tiles > (ctx->sm_count - tiles) * 14) return 0;   // no helper blocks for this turn length (at most 14 tiles per helper)
+  const size_t row = (size_t)((desc->head_dim + desc->rank_v + 15) / 16 * 16 + 4);
+  const size_t rec = (128 * row + 256) * 4;                                    // one partial: O' rows | m | l
+  return ((size_t)tiles * 4 + 255) / 256 * 256 + (size_t)(tiles + ctx->sm_count) * rec;
+}
+
+int32_t precc_lr_attend_prefill_ws(precc_ctx* ctx, const precc_layer_desc* desc, const void* q, int32_t S, int32_t agent,
+                                   int32_t ctx_len, const int32_t* block_table, int32_t table_stride, int32_t first_block,
+                                   const void* B_k, const void* B_v, const precc_cache* cache, void* out, void* ws,
+                                   size_t ws_bytes, void* stream) {
+  if (!ctx) return PRECC_ERR_INVALID_ARG;
+  return prefill_entry(ctx, desc, q, S, agent, ctx_len, block_table, table_stride, first_block, B_k, B_v, nullptr, cache, out, stream,
+                       nullptr, 0, ws, ws_bytes);
 }
 
 size_t precc_prefill_rope_scratch_bytes(const precc_layer_desc* desc, int32_t ctx_len, int32_t S) {

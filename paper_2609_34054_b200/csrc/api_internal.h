@@ -40,6 +40,9 @@ struct precc_ctx {
   int decode_cluster_cap = 0;          // PRECC_DECODE_CLUSTER=n in the environment: at most n blocks per decode cluster (0 = planner's choice)
   bool prefill_forward = false;        // PRECC_PREFILL_ORDER=forward: row tiles in ascending order (default: longest causal reach first)
   bool no_prefill_split = false;       // PRECC_PREFILL_SPLIT=0 in the environment: never split a turn's context over a cluster
+  bool no_prefill_helpers = false;     // PRECC_PREFILL_HELPERS=0 in the environment: prefill with a workspace never uses helper blocks
+  int prefill_helper_p = 0;            // PRECC_PREFILL_HELPER_P=n in the environment: the tiles' own blocks stop after n steps (experiments; 0 = planner's choice)
+  int prefill_helper_min_steps = 48;   // PRECC_PREFILL_HELPER_MIN=n in the environment: shortest context (128-token steps) that gets helper blocks
   char err[512] = {0};
   CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                            const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -110,6 +113,7 @@ struct PrefillArgs {
   const float* rope = nullptr; int max_pos = 0;      // rotary variant when rope != null
   const void* k_scratch = nullptr;                   // adapted keys of this sequence in logical block order (rotary prefill
   long long k_scratch_blocks = 0;                    // with scratch): the keys come from here, the values from the cache
+  void* ws = nullptr; size_t ws_bytes = 0;           // optional workspace of the work-list launch (helper blocks on idle SMs)
 };
 
 

@@ -1,6 +1,9 @@
 // Host side of new-turn prefill attention: kernel choice (tcgen05 kernel or the mma.sync kernel), tensor maps,
 // the cluster split of short turns and the launch.  Included by one translation unit per head dimension.
 #pragma once
+#include <algorithm>
+#include <vector>
+
 #include "api_internal.h"
 #include "prefill.cuh"
 #include "prefill_tc.cuh"
@@ -9,6 +12,68 @@ namespace precc {
 
 template <int HD, int RK, int RV>
 struct PrefillRun {
+  // ---- work-list launch of the tensor-core kernel: plan and workspace
+  struct WorkList { int p = 0, helpers = 0, tiles = 0; };
+  static size_t ticket_bytes(int tiles) { return ((size_t)tiles * 4 + 255) / 256 * 256; }
+  static size_t worklist_ws_bytes(int tiles, int helpers) {
+    return ticket_bytes(tiles) + (size_t)(2 * tiles + helpers) * PrefillTcCfg<HD, RK, RV>::REC_FLOATS * 4;
+  }
+  // Steps of row tile x; the tail of a tile is what lies beyond the first `p` steps.  Tails are laid end to end, kv
+  // head by kv head, and cut into `helpers` equal ranges (the kernel derives the same cuts from p and helpers).
+  // The cost of a plan, in steps: the longer of a tile's own block (p + its record and possibly the merge) and a
+  // helper (its range + a drain and refill per piece).  Returns p = 0 when the classic launch is as good.
+  static WorkList plan_worklist(precc_ctx* ctx, int S, int T, int tok_per_tile, int n_kv) {
+    WorkList best;
+    if (ctx->no_prefill_helpers) return best;
+    const int X = (S + tok_per_tile - 1) / tok_per_tile;
+    const long long tiles = (long long)X * n_kv;
+    const int H = ctx->sm_count - (int)tiles;
+    if (X >= PTC_MAX_XT || tiles * 2 <= ctx->sm_count || tiles > (long long)H * (PTC_MAX_SEG - 2)) return best;
+    auto steps_of = [&](int x) { return (int)(((long long)T + std::min(S, (x + 1) * tok_per_tile) + PTC_TOK - 1) / PTC_TOK); };
+    const int n_max = steps_of(X - 1);
+    if (n_max < ctx->prefill_helper_min_steps) return best;
+    // what a record + merge costs a tile's own block, and what a piece costs a helper beyond its steps (query tile,
+    // fold, pipeline fill, record), in steps: measured at head_dim 128, rank 32 (1.3 us per step), scaled for shorter steps
+    const int f100 = 100 * 160 / (HD + (RK + RV) / 2);
+    const int C_OWN = 14 * f100 / 100, C_PIECE = 12 * f100 / 100;
+    int best_cost = n_max - std::max(2, n_max / 25);   // a plan must win at least 4 % (and two steps)
+    for (int p = n_max - 1; p >= std::max(8, n_max / 2); --p) {
+      if (ctx->prefill_helper_p > 0 && p != ctx->prefill_helper_p) continue;
+      long long tail_sum = 0;
+      for (int x = 0; x < X; ++x) tail_sum += std::max(0, steps_of(x) - p);
+      const long long total = tail_sum * n_kv;
+      const long long per = std::max(1ll, (total + H - 1) / H);
+      if (p + C_OWN >= best_cost && ctx->prefill_helper_p <= 0) continue;
+      // walk the tails in the kernel's order: pieces per helper and pieces per tile
+      int max_seg = 0, max_src = 0;
+      long long pos = 0;
+      for (int g = 0; g < n_kv; ++g)
+        for (int x = 0; x < X; ++x) {
+          const int tl = std::max(0, steps_of(x) - p);
+          if (tl == 0) continue;
+          const long long hf = pos / per, hl = (pos + tl - 1) / per;
+          max_src = std::max(max_src, (int)(2 + hl - hf));
+          pos += tl;
+        }
+      {
+        // pieces of helper h = tiles whose tail range meets [h per, (h+1) per)
+        std::vector<int> cnt(H, 0);
+        pos = 0;
+        for (int g = 0; g < n_kv; ++g)
+          for (int x = 0; x < X; ++x) {
+            const int tl = std::max(0, steps_of(x) - p);
+            if (tl == 0) continue;
+            for (long long h = pos / per; h <= (pos + tl - 1) / per && h < H; ++h) ++cnt[(size_t)h];
+            pos += tl;
+          }
+        for (int h = 0; h < H; ++h) max_seg = std::max(max_seg, cnt[(size_t)h]);
+      }
+      if (max_seg > PTC_MAX_SEG || max_src > PTC_MAX_SRC) continue;
+      const int cost = (int)std::max<long long>(p + C_OWN, per + (long long)C_PIECE * max_seg);
+      if (cost < best_cost || ctx->prefill_helper_p > 0) { best_cost = cost; best.p = p; best.helpers = H; best.tiles = (int)tiles; }
+    }
+    return best;
+  }
   // tensor-core kernel (tcgen05 + TMEM + TMA) for the shapes it supports
   static int32_t run_tc(precc_ctx* ctx, const PrefillArgs& a) {
     using C = PrefillTcCfg<HD, RK, RV>;
@@ -84,6 +149,27 @@ struct PrefillRun {
         }
         if (max_clusters[ns] - 1 >= base_blocks) break;
         --ns;
+      }
+    }
+    p.helper_p = 0; p.n_helpers = 0; p.row_tiles = row_tiles; p.ws_rec = nullptr; p.ws_ticket = nullptr;
+    // One wave that leaves SMs without a block (a 512-token turn of 8 kv heads is 128 blocks on 148 SMs): with a
+    // workspace the blocks stop `helper_p` steps into their tile and helper blocks on the idle SMs share the tails.
+#ifdef PRECC_PF_TRACE
+    const bool wl_ok = !p.trace || ctx->trace_blocks >= 2048;   // room for every block's piece stamps
+#else
+    const bool wl_ok = !p.trace;
+#endif
+    if (a.ws && ns == 1 && wl_ok) {
+      const WorkList wl = plan_worklist(ctx, a.S, a.T, p.tok_per_tile, d->n_kv_heads);
+      if (wl.p > 0 && a.ws_bytes >= worklist_ws_bytes(wl.tiles, wl.helpers)) {
+        p.helper_p = wl.p; p.n_helpers = wl.helpers; p.longest_first = 0;
+        p.ws_ticket = reinterpret_cast<unsigned int*>(a.ws);
+        p.ws_rec = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(a.ws) + ticket_bytes(wl.tiles));
+        PRECC_CUDA(ctx, cudaMemsetAsync(a.ws, 0, ticket_bytes(wl.tiles), a.stream));
+        cudaLaunchConfig_t wc = {};
+        wc.gridDim = dim3(wl.tiles + wl.helpers); wc.blockDim = dim3(PTC_THREADS); wc.dynamicSmemBytes = smem; wc.stream = a.stream;
+        PRECC_CUDA(ctx, cudaLaunchKernelEx(&wc, kern, mk, mv, mlk, mlv, p));
+        return PRECC_OK;
       }
     }
     cudaLaunchConfig_t cfg = {};

@@ -52,6 +52,12 @@ struct PrefillTcParams {
   int longest_first;           // 1: block x = 0 takes the LAST row tile (longest causal reach), so the tail of the grid is short blocks
   float scale_log2, s_k, s_v;
   unsigned long long* trace;   // PRECC_PF_TRACE builds only: [steps][16] clock stamps of block (0, 0)
+  // Work-list launch (helper_p > 0; 1-D grid of tiles + n_helpers blocks, no cluster): block b < tiles takes steps
+  // [0, helper_p) of tile b, the n_helpers blocks behind them share the tails of all tiles; the pieces of a tile meet
+  // through records in `ws_rec`, and the block that arrives last at the tile's ticket merges them.
+  int helper_p, n_helpers, row_tiles;
+  float* ws_rec;               // [2 * tiles + n_helpers][PrefillTcCfg::REC_FLOATS]
+  unsigned int* ws_ticket;     // [tiles], zero before the launch and again after it
 };
 
 // Timeline stamps for tuning (compiled in with -DPRECC_PF_TRACE; slot meanings at the call sites).
@@ -60,8 +66,18 @@ struct PrefillTcParams {
   do {                                                                                           \
     if ((p).trace && blockIdx.x == 0 && blockIdx.y == 0 && (j) < 64) (p).trace[(j) * 16 + (slot)] = clock64(); \
   } while (0)
+// work-list launch: wall-clock stamps of every block's pieces (thread 0 of the softmax warps), behind the step stamps
+#define PTC_WL_STAMP(p, seg, slot)                                                               \
+  do {                                                                                           \
+    if ((p).trace && (p).helper_p > 0 && threadIdx.x == PTC_FIRST_SM_WARP * 32 && (seg) < 16) {   \
+      unsigned long long t__;                                                                    \
+      asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t__));                                 \
+      (p).trace[1024 + blockIdx.x * 128 + (seg) * 8 + (slot)] = t__;                             \
+    }                                                                                            \
+  } while (0)
 #else
 #define PTC_STAMP(p, j, slot) do { } while (0)
+#define PTC_WL_STAMP(p, seg, slot) do { } while (0)
 #endif
 
 constexpr int PTC_PARTS_MAX = 4;
@@ -69,8 +85,13 @@ constexpr int PTC_PARTS = 2;                         // softmax threads per quer
 constexpr int PTC_SOFTMAX_WARPS = 4 * PTC_PARTS;
 constexpr int PTC_FIRST_SM_WARP = 3;                 // warps 0..2: key producer, QK^T issuer, PV issuer
 constexpr int PTC_THREADS = (PTC_FIRST_SM_WARP + PTC_SOFTMAX_WARPS + 1) * 32;
+constexpr int PTC_FIXED_BARS = 10; // barriers besides the two per ring stage
 constexpr int PTC_TOK = 128;      // tokens per step
 constexpr float PTC_RAISE = 8.f;  // the running maximum is raised only when it grows by more than this
+constexpr int PTC_MAX_SRC = 8;    // work-list launch: pieces of one tile (its own block + helper pieces) at most
+constexpr int PTC_MAX_SEG = 16;   // work-list launch: tile pieces one helper block takes at most
+constexpr int PTC_MAX_XT = 160;   // work-list launch: row tiles at most
+constexpr int PTC_TAB_BYTES = (2 * PTC_MAX_XT + 8 + 4 * PTC_MAX_SEG) * 4;   // tail lengths | their prefix sums | scalars | piece list
 
 template <int HD, int RK, int RV>
 struct PrefillTcCfg {
@@ -91,10 +112,13 @@ struct PrefillTcCfg {
   static constexpr int SPLIT_XS = (HD + RV + 15) / 16 * 16 + 4;                // row stride (floats) of a partial in shared memory
   // split-context merge area (laid over the Q tile, the folded-query tile and the rings): partial | m | l | merged rows | weights | 1/l | B_v slice
   static constexpr int SPLIT_BYTES = (128 * SPLIT_XS + 256 + 64 * SPLIT_XS + 16 * 64 + 64) * 4 + RV * HD * 2;
+  static constexpr int REC_FLOATS = 128 * SPLIT_XS + 256;     // a tile's partial in global memory: O' rows | m[128] | l[128]
+  // work-list merge area (same place): merged rows | weights of up to PTC_MAX_SRC pieces | 1/l | B_v slice
+  static constexpr int WS_MERGE_BYTES = (128 * SPLIT_XS + PTC_MAX_SRC * 128 + 128) * 4 + RV * HD * 2;
   static constexpr bool L_IN_MMA = RV > 0 && RV < 64;         // a spare column of the L_V slab carries the denominator
   static constexpr int TMEM_P = 2 * PTC_TOK;                  // packed bf16 P (64 columns) after the two S buffers
   static constexpr int TMEM_O = TMEM_P + PTC_TOK / 2;         // O' (at most 192 columns): 320 + 192 = 512
-  __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 320 + 2 * PTC_PARTS_MAX * 512 + 1024; }
+  __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 320 + 2 * PTC_PARTS_MAX * 512 + PTC_TAB_BYTES + 1024; }
   static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 8 || RK == 16 || RK == 32 || RK == 64) &&
                                     (RV == 0 || RV == 8 || RV == 16 || RV == 32 || RV == 64);
 };
@@ -195,18 +219,22 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   const uint32_t vring_u32 = kring_u32 + KS * C::KSTAGE;
   uint64_t* bars = reinterpret_cast<uint64_t*>(vring + (size_t)VS * C::VSTAGE);
   const uint32_t bar0 = smem_u32(bars);
-  // barrier map: k_full[KS] | k_empty[KS] | v_full[VS] | v_empty[VS] | s_full[2] | p_full[2] | pv_done | q_ready | s_free[2]
+  // barrier map: k_full[KS] | k_empty[KS] | v_full[VS] | v_empty[VS] | s_full[2] | p_full[2] | pv_done | q_ready | s_free[2] | fold_go | fold_done
   const uint32_t k_full = bar0, k_empty = k_full + 8 * KS, v_full = k_empty + 8 * KS, v_empty = v_full + 8 * VS,
                  s_full = v_empty + 8 * VS, p_full = s_full + 16, pv_done = p_full + 16, q_ready = pv_done + 8,
-                 s_free = q_ready + 8;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * KS + 2 * VS + 8);
+                 s_free = q_ready + 8, fold_go = s_free + 16, fold_done = fold_go + 8;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * KS + 2 * VS + PTC_FIXED_BARS);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = blockIdx.y, G = p.group;
-  const int tok0 = (p.longest_first ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x) * p.tok_per_tile;
-  const int n_tok = min(p.tok_per_tile, p.S - tok0);             // new tokens handled by this block
-  const int t_end = p.T + tok0 + n_tok;                          // context + causal reach of the last row
-  const int full_vis = p.T + tok0 + 1;                           // tokens visible to every row of the block
+  const int G = p.group;
+  const bool worklist = p.helper_p > 0;
+  // What this block works on.  Classic launch: one (row tile, kv head) per block, fixed for the whole kernel.  Work-list
+  // launch: a short list of tile pieces, taken one after the other with the block drained in between.
+  int g = blockIdx.y;
+  int tok0 = (p.longest_first ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x) * p.tok_per_tile;
+  int n_tok = min(p.tok_per_tile, p.S - tok0);             // new tokens handled by this block
+  int t_end = p.T + tok0 + n_tok;                          // context + causal reach of the last row
+  int full_vis = p.T + tok0 + 1;                           // tokens visible to every row of the block
   // Short turns over long contexts: the 128-token steps of a (row tile, kv head) are split over the NS
   // blocks of a cluster (grid/cluster z; any size from 2 to 8), each producing a partial (m, l, O') that the cluster merges
   // over distributed shared memory.  `jb` is this block's first step, `n_tiles` its number of steps
@@ -214,12 +242,21 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   uint32_t split, NS;
   asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(split));
   asm volatile("mov.u32 %0, %%cluster_nctaid.z;\n" : "=r"(NS));
-  const int n_total = (t_end + PTC_TOK - 1) / PTC_TOK;
-  const int chunk_steps = (n_total + (int)NS - 1) / (int)NS;
-  const int jb = min(n_total, (int)split * chunk_steps);
-  const int n_tiles = min(n_total, jb + chunk_steps) - jb;
+  int jb = 0, n_tiles = 0;
+  if (!worklist) {
+    const int n_total = (t_end + PTC_TOK - 1) / PTC_TOK;
+    const int chunk_steps = (n_total + (int)NS - 1) / (int)NS;
+    jb = min(n_total, (int)split * chunk_steps);
+    n_tiles = min(n_total, jb + chunk_steps) - jb;
+  }
+  // work-list tables behind the maxima exchange area: tail[x] | pre[x] | scalars | pieces {tile, first step, steps, -}
+  int* tab_tail = reinterpret_cast<int*>(bars + 2 * KS + 2 * VS + PTC_FIXED_BARS + 2) + 2 * PTC_PARTS_MAX * 128;
+  int* tab_pre = tab_tail + PTC_MAX_XT;
+  int* tab_sc = tab_pre + PTC_MAX_XT;                      // [0] pieces of this block, [1] sum of the tails of one kv head, [2] tail steps per helper
+  int* tab_seg = tab_sc + 8;
+  auto steps_of = [&](int x) { return (p.T + min(p.S, (x + 1) * p.tok_per_tile) + PTC_TOK - 1) / PTC_TOK; };
 
-  if (threadIdx.x == 0) {
+  auto init_bars = [&]() {
     for (int s = 0; s < KS; ++s) { mbar_init(k_full + 8 * s, 1); mbar_init(k_empty + 8 * s, 1); }
     for (int s = 0; s < VS; ++s) { mbar_init(v_full + 8 * s, 1); mbar_init(v_empty + 8 * s, 1); }
     mbar_init(s_full, 1); mbar_init(s_full + 8, 1);
@@ -227,17 +264,89 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     mbar_init(pv_done, 1);
     mbar_init(s_free, PTC_SOFTMAX_WARPS); mbar_init(s_free + 8, PTC_SOFTMAX_WARPS);
     mbar_init(q_ready, PTC_SOFTMAX_WARPS);
+    mbar_init(fold_go, PTC_SOFTMAX_WARPS); mbar_init(fold_done, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     fence_async_smem();
-  }
+  };
+  if (threadIdx.x == 0) init_bars();
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_holder)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  if (worklist) {
+    for (int x = threadIdx.x; x < p.row_tiles; x += blockDim.x) tab_tail[x] = max(0, steps_of(x) - p.helper_p);
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  const int n_base_tiles = p.row_tiles * p.n_kv;           // work-list launch: blocks below this index own a tile
+  if (worklist) {
+    if (threadIdx.x == 0) {
+      const int X = p.row_tiles;
+      int acc = 0;
+      for (int x = 0; x < X; ++x) { tab_pre[x] = acc; acc += tab_tail[x]; }
+      const int tail_sum = acc, total = acc * p.n_kv;
+      const int per = max(1, (total + p.n_helpers - 1) / max(1, p.n_helpers));
+      int n = 0;
+      const int b = blockIdx.x;
+      if (b < n_base_tiles) {
+        const int x = b % X;
+        tab_seg[0] = b; tab_seg[1] = 0; tab_seg[2] = steps_of(x) - tab_tail[x];
+        n = 1;
+      } else {
+        const int h = b - n_base_tiles;
+        int pos = min(total, h * per);
+        const int hi = min(total, pos + per);
+        if (pos < hi) {
+          int gg = pos / tail_sum, off = pos - gg * tail_sum, x = 0;
+          while (tab_pre[x] + tab_tail[x] <= off) ++x;
+          while (pos < hi && n < PTC_MAX_SEG) {
+            const int take = min(hi - pos, tab_pre[x] + tab_tail[x] - off);
+            tab_seg[4 * n] = gg * X + x;
+            tab_seg[4 * n + 1] = steps_of(x) - tab_tail[x] + (off - tab_pre[x]);
+            tab_seg[4 * n + 2] = take;
+            ++n; pos += take; off += take;
+            while (x < X && tab_pre[x] + tab_tail[x] <= off) ++x;
+            if (x == X) { ++gg; off = 0; x = 0; while (x < X - 1 && tab_tail[x] == 0) ++x; off = tab_pre[x]; }
+          }
+        }
+      }
+      tab_sc[0] = n; tab_sc[1] = tail_sum; tab_sc[2] = per;
+    }
+    __syncthreads();
+  }
+  const int nseg = worklist ? tab_sc[0] : 1;
+  for (int seg = 0; seg < nseg; ++seg) {
+  // work-list launch: the tile of this piece, where its record goes and which records make up the tile
+  bool to_ws = false;
+  int tile_u = 0, rec_id = 0, n_src = 1, src_first = 0;
+  if (worklist) {
+    tile_u = tab_seg[4 * seg]; jb = tab_seg[4 * seg + 1]; n_tiles = tab_seg[4 * seg + 2];
+    const int x = tile_u % p.row_tiles;
+    g = tile_u / p.row_tiles;
+    tok0 = x * p.tok_per_tile;
+    n_tok = min(p.tok_per_tile, p.S - tok0);
+    t_end = p.T + tok0 + n_tok;
+    full_vis = p.T + tok0 + 1;
+    if (tab_tail[x] > 0) {
+      const int a_u = g * tab_sc[1] + tab_pre[x], per = tab_sc[2];
+      const int hf = a_u / per, hl = (a_u + tab_tail[x] - 1) / per;
+      to_ws = true;
+      n_src = 2 + hl - hf;
+      src_first = n_base_tiles + tile_u + hf;              // record of the first helper piece; the tile's own block writes record tile_u
+      rec_id = (int)blockIdx.x < n_base_tiles ? tile_u : n_base_tiles + tile_u + ((int)blockIdx.x - n_base_tiles);
+    }
+    if (seg > 0) {
+      // the block is drained (every load consumed, every MMA retired, all threads past the barrier that ended the
+      // previous piece): fresh barriers for the next piece
+      if (threadIdx.x == 0) {
+        for (int i = 0; i < 2 * KS + 2 * VS + PTC_FIXED_BARS; ++i) asm volatile("mbarrier.inval.shared::cta.b64 [%0];\n" ::"r"(bar0 + 8 * i) : "memory");
+        init_bars();
+      }
+      __syncthreads();
+    }
+  }
 
   if (warp == 0 || warp == PTC_FIRST_SM_WARP + PTC_SOFTMAX_WARPS) {
     // ------------------------------------------------------------------ TMA producers (keys / values)
@@ -303,6 +412,24 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const uint64_t qxd0 = RK > 0 ? umma_desc_kmajor(qx_u32, C::RKP * 2) : 0;
     const uint64_t kd0 = umma_desc_kmajor(kring_u32, 128);
     const uint64_t lkd0 = RK > 0 ? umma_desc_kmajor(kring_u32 + C::KV_BYTES, C::RKP * 2) : 0;
+    if constexpr (RK > 0) {
+      // the key-side fold Q B_k^T (128 x RKP x HD): Q tile and B_k slice are staged, the product lands in the first
+      // columns of S buffer 0, from where the softmax threads scale it into the folded-query tile
+      mbar_wait(fold_go, 0, p.status);
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t id_f = umma_idesc(C::RKP, 0);
+        const uint64_t bd0 = umma_desc_kmajor(kring_u32 + (uint32_t)(KS - 1) * C::KSTAGE, 128);
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint64_t qo = (uint64_t)(((ks / 4) * C::SLAB_BYTES + (ks % 4) * 32) >> 4);
+          const uint64_t bo = (uint64_t)(((ks / 4) * (C::RKP * 128) + (ks % 4) * 32) >> 4);
+          umma_bf16(tmem_base, qd0 + qo, bd0 + bo, id_f, ks ? 1u : 0u);
+        }
+        umma_commit(fold_done);
+      }
+      __syncwarp();
+    }
     mbar_wait(q_ready, 0, p.status);
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j % KS;
@@ -389,6 +516,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     constexpr int NP = PTC_PARTS;
     constexpr int COLS = PTC_TOK / NP;                            // score columns per thread (32)
     constexpr int NSM = PTC_SOFTMAX_WARPS * 32;                   // softmax threads
+    PTC_WL_STAMP(p, seg, 0);                                       // piece starts
     const int quad = warp & 3;                                    // TMEM lane quadrant this warp may touch
     const int part = (warp - PTC_FIRST_SM_WARP) >> 2;             // which tokens / which output columns
     const int row = quad * 32 + lane;                             // query row of this thread
@@ -397,15 +525,17 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const int i_new = tok0 + row / G, hg = row % G;
     const bool row_ok = row < n_tok * G;
     const int lim = row_ok ? p.T + i_new : -1;                    // last visible token of this row
-    float* xch = reinterpret_cast<float*>(bars + 2 * KS + 2 * VS + 10);   // [2][NP][128] row maxima exchanged by a row's threads
+    float* xch = reinterpret_cast<float*>(bars + 2 * KS + 2 * VS + PTC_FIXED_BARS + 2);   // [2][NP][128] row maxima exchanged by a row's threads
     auto row_sync = [&]() { asm volatile("bar.sync %0, %1;\n" ::"r"(2 + quad), "r"(32 * NP) : "memory"); };
-    // ---- B_k slice into the last key stage, Q row into the swizzled K-major tile, then the fold Q~
+    // ---- B_k slice into the last key stage and the Q rows into their tile, both as K-major swizzled operands; the
+    //      fold Q~ = s_k Q B_k^T is one small MMA chain (issued by warp 1), scaled and rounded here
     unsigned char* bk_s = kring + (size_t)(KS - 1) * C::KSTAGE;
     if constexpr (RK > 0) {
-      for (int c = tid; c < RK * (HD / 8); c += NSM) {
+      for (int c = tid; c < C::RKP * (HD / 8); c += NSM) {
         const int j = c / (HD / 8), ch = c % (HD / 8);
-        *reinterpret_cast<uint4*>(bk_s + (j * HD + ch * 8) * 2) =
-            __ldg(reinterpret_cast<const uint4*>(p.B_k + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
+        const uint4 v = j < RK ? __ldg(reinterpret_cast<const uint4*>(p.B_k + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8))
+                               : make_uint4(0u, 0u, 0u, 0u);    // rank 8 rides as a zero-padded step of 16
+        *reinterpret_cast<uint4*>(bk_s + (ch / 8) * (C::RKP * 128) + j * 128 + (((ch % 8) ^ (j & 7)) * 16)) = v;
       }
     }
     {
@@ -418,43 +548,31 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
               row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
         }
       }
-      asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");      // B_k slice and the Q tile are visible
       if constexpr (RK > 0) {
         constexpr int CPR = C::RKP / 8;
+        fence_async_smem();                                       // the staged operands -> visible to the MMA unit
+        __syncwarp();
+        if (lane == 0) mbar_arrive(fold_go);
+        mbar_wait(fold_done, 0, p.status);
+        tc_fence_after();
 #pragma unroll 1
-        for (int j0 = part * 8; j0 < RK; j0 += NP * 8) {           // this thread folds coordinates j0 .. j0+7
-          float acc[8];
+        for (int c = part; c < C::RKP / 16; c += NP) {             // 16 coordinates per pass
+          uint32_t fv[16];
+          tmem_ld16(lane_addr + c * 16, fv);
+          tmem_wait_ld();
+          uint32_t pk[8];
 #pragma unroll
-          for (int jj = 0; jj < 8; ++jj) acc[jj] = 0.f;
-#pragma unroll 2
-          for (int c = 0; c < HD / 8; ++c) {
-            const int sl = c / 8, ch = c % 8;
-            const uint4 qq = *reinterpret_cast<const uint4*>(smem + sl * C::SLAB_BYTES + row * 128 + ((ch ^ (row & 7)) * 16));
-            const uint32_t xs[4] = {qq.x, qq.y, qq.z, qq.w};
-#pragma unroll
-            for (int jj = 0; jj < 8; ++jj) {
-              const uint32_t* bb = reinterpret_cast<const uint32_t*>(bk_s + (size_t)(j0 + jj) * HD * 2) + c * 4;
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const uint32_t y = bb[k];
-                acc[jj] += bf16_bits_to_float(xs[k] & 0xffff) * bf16_bits_to_float(y & 0xffff) +
-                           bf16_bits_to_float(xs[k] >> 16) * bf16_bits_to_float(y >> 16);
-              }
-            }
-          }
-          *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, j0 / 8)) =
-              make_uint4(pack_bf16(acc[0] * p.s_k, acc[1] * p.s_k), pack_bf16(acc[2] * p.s_k, acc[3] * p.s_k),
-                         pack_bf16(acc[4] * p.s_k, acc[5] * p.s_k), pack_bf16(acc[6] * p.s_k, acc[7] * p.s_k));
+          for (int k = 0; k < 8; ++k) pk[k] = pack_bf16(__uint_as_float(fv[2 * k]) * p.s_k, __uint_as_float(fv[2 * k + 1]) * p.s_k);
+          *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, 2 * c)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, 2 * c + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
         }
-        // rank 8: the upper half of the padded k step is zero on the query side (the key side is zero-filled by TMA)
-        if constexpr (C::RKP > RK) {
-          if (part == 0) *reinterpret_cast<uint4*>(smem + C::Q_BYTES + swz_off<CPR>(row, 1)) = make_uint4(0u, 0u, 0u, 0u);
-        }
+        tc_fence_before();                                        // the reads of S buffer 0 precede the first Q K^T
       }
     }
     fence_async_smem();                                           // generic-proxy writes -> visible to the MMA unit
     __syncwarp();
     if (lane == 0) mbar_arrive(q_ready);
+    PTC_WL_STAMP(p, seg, 1);                                       // query tile loaded and folded
 
     constexpr int OCH = (HD + RV) / 16 + (C::L_IN_MMA ? 1 : 0);   // 16-column chunks of O' that carry data (numerator, U, denominator)
     float m_used = NEG_BIG, l_sum = 0.f;
@@ -581,6 +699,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       tc_fence_after();
       tmax = exchange_max(0, local_max(0));
     }
+    PTC_WL_STAMP(p, seg, 2);                                       // first scores seen
     for (int j = 0; j < n_tiles; ++j) {
       if (tid == 0) PTC_STAMP(p, j, 4);                            // step j starts (its scores were awaited a step earlier)
       if ((jb + j) * PTC_TOK + PTC_TOK > full_vis) step(j, std::true_type{});   // only the last few steps reach the causal edge
@@ -589,6 +708,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     }
     // ---- epilogue: out = (O + s_v U B_v) / l ; the threads of a row share its output columns
     if (n_tiles > 0) { mbar_wait(pv_done, (n_tiles - 1) & 1, p.status); tc_fence_after(); }
+    PTC_WL_STAMP(p, seg, 3);                                       // all steps done
     if (NS > 1) {
       // ---- split context: this block's partial (m, l, O') goes to shared memory for the cluster merge below
       constexpr int XS = C::SPLIT_XS;
@@ -622,6 +742,130 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           *reinterpret_cast<uint4*>(xo + row * XS + c * 16 + k) = make_uint4(ov[k], ov[k + 1], ov[k + 2], ov[k + 3]);
       }
       if (part == 0) { xm[row] = n_tiles > 0 ? m_used : NEG_BIG; xl[row] = n_tiles > 0 ? l_loc : 0.f; }
+    } else if (to_ws) {
+      // ---- work-list launch: this piece's partial (m, l, O') goes to its record in global memory; the block that
+      //      arrives last at the tile's ticket merges the tile's records in a fixed order and writes the output
+      constexpr int XS = C::SPLIT_XS;
+      float* rec = p.ws_rec + (size_t)rec_id * C::REC_FLOATS;
+      float l_loc = 0.f;
+      if constexpr (!C::L_IN_MMA) {
+        xch[part * 128 + row] = l_sum;
+        asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+#pragma unroll
+        for (int q2 = 0; q2 < NP; ++q2) l_loc += xch[q2 * 128 + row];
+      } else {
+        uint32_t lv16[16];
+        tmem_ld16(lane_addr + C::TMEM_O + HD + (RV / 16) * 16, lv16);
+        tmem_wait_ld();
+        l_loc = __uint_as_float(lv16[RV % 16]);
+      }
+#pragma unroll 1
+      for (int c = part; c < (HD + RV + 15) / 16; c += NP) {
+        uint32_t ov[16];
+        tmem_ld16(lane_addr + C::TMEM_O + c * 16, ov);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 16; k += 4)
+          __stcg(reinterpret_cast<uint4*>(rec + row * XS + c * 16 + k), make_uint4(ov[k], ov[k + 1], ov[k + 2], ov[k + 3]));
+      }
+      if (part == 0) { __stcg(rec + 128 * XS + row, m_used); __stcg(rec + 128 * XS + 128 + row, l_loc); }
+      __threadfence();
+      PTC_WL_STAMP(p, seg, 4);                                     // record written
+      asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+      int* flag = reinterpret_cast<int*>(xch) + 2 * PTC_PARTS_MAX * 128 - 1;   // last word of the exchange area
+      if (tid == 0) *flag = (int)atomicAdd(p.ws_ticket + tile_u, 1u);
+      asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+      if (*flag == n_src - 1) {
+        __threadfence();
+        // merge area over the Q tile and the rings: every load of this piece has been consumed, every MMA has retired
+        float* mo = reinterpret_cast<float*>(smem);         // merged rows [128][XS]
+        float* wts = mo + 128 * XS;                         // [n_src][128] weights of the pieces
+        float* linv = wts + PTC_MAX_SRC * 128;              // [128]
+        unsigned char* bvs = reinterpret_cast<unsigned char*>(linv + 128);   // B_v[:, g] slice, [RV][HD] bf16
+        auto src = [&](int k) -> const float* {
+          return p.ws_rec + (size_t)(k == 0 ? tile_u : src_first + k - 1) * C::REC_FLOATS;
+        };
+        if constexpr (RV > 0) {
+          for (int c = tid; c < RV * (HD / 8); c += NSM) {
+            const int j = c / (HD / 8), ch = c % (HD / 8);
+            *reinterpret_cast<uint4*>(bvs + (j * HD + ch * 8) * 2) =
+                __ldg(reinterpret_cast<const uint4*>(p.B_v + (size_t)j * p.n_kv * HD + (size_t)g * HD + ch * 8));
+          }
+        }
+        if (tid < 128) {
+          float ms[PTC_MAX_SRC], M = NEG_BIG, L = 0.f;
+#pragma unroll
+          for (int k = 0; k < PTC_MAX_SRC; ++k) { ms[k] = k < n_src ? __ldcg(src(k) + 128 * XS + tid) : NEG_BIG; M = fmaxf(M, ms[k]); }
+#pragma unroll
+          for (int k = 0; k < PTC_MAX_SRC; ++k) {
+            if (k < n_src) {
+              const float wv = fast_exp2(ms[k] - M);
+              wts[k * 128 + tid] = wv;
+              L += wv * __ldcg(src(k) + 128 * XS + 128 + tid);       // piece order: deterministic
+            }
+          }
+          linv[tid] = L > 0.f ? 1.f / L : 0.f;
+        }
+        asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+        constexpr int F4 = (HD + RV) / 4;                   // float4 columns of a merged row
+        constexpr int UN = 8;                               // items per thread in flight: the records come from L2
+        for (int it0 = tid; it0 < 128 * F4; it0 += NSM * UN) {
+          float4 acc[UN];
+#pragma unroll
+          for (int u = 0; u < UN; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int k = 0; k < n_src; ++k) {
+            const float* sk = src(k);
+            float4 x[UN];
+#pragma unroll
+            for (int u = 0; u < UN; ++u) {
+              const int it = it0 + u * NSM;
+              x[u] = it < 128 * F4 ? __ldcg(reinterpret_cast<const float4*>(sk + (it / F4) * XS + (it % F4) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < UN; ++u) {
+              const int it = it0 + u * NSM;
+              const float wv = it < 128 * F4 ? wts[k * 128 + it / F4] : 0.f;
+              acc[u].x += wv * x[u].x; acc[u].y += wv * x[u].y; acc[u].z += wv * x[u].z; acc[u].w += wv * x[u].w;
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < UN; ++u) {
+            const int it = it0 + u * NSM;
+            if (it < 128 * F4) *reinterpret_cast<float4*>(mo + (it / F4) * XS + (it % F4) * 4) = acc[u];
+          }
+        }
+        asm volatile("bar.sync 1, %0;\n" ::"r"(NSM) : "memory");
+        // out = (O + s_v U B_v) / l, eight columns per item
+        for (int it = tid; it < 128 * (HD / 8); it += NSM) {
+          const int rl = it / (HD / 8), c8 = (it % (HD / 8)) * 8;
+          if (rl >= n_tok * G) continue;
+          float o[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) o[k] = mo[rl * XS + c8 + k];
+          if constexpr (RV > 0) {
+#pragma unroll 4
+            for (int jv = 0; jv < RV; ++jv) {
+              const float uj = mo[rl * XS + HD + jv] * p.s_v;
+              const uint4 y = *reinterpret_cast<const uint4*>(bvs + (jv * HD + c8) * 2);
+              const uint32_t ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                o[2 * k] += uj * bf16_bits_to_float(ys[k] & 0xffff);
+                o[2 * k + 1] += uj * bf16_bits_to_float(ys[k] >> 16);
+              }
+            }
+          }
+          const float inv = linv[rl];
+          const int i_out = tok0 + rl / G, h_out = rl % G;
+          uint4 w;
+          w.x = pack_bf16(o[0] * inv, o[1] * inv); w.y = pack_bf16(o[2] * inv, o[3] * inv);
+          w.z = pack_bf16(o[4] * inv, o[5] * inv); w.w = pack_bf16(o[6] * inv, o[7] * inv);
+          *reinterpret_cast<uint4*>(p.out + ((size_t)i_out * p.n_q + (size_t)g * G + h_out) * HD + c8) = w;
+        }
+        if (tid == 0) p.ws_ticket[tile_u] = 0u;             // the workspace is ready for the next call
+        PTC_WL_STAMP(p, seg, 6);                                   // merged and stored
+      }
+      PTC_WL_STAMP(p, seg, 5);                                     // piece ends
     } else {
     unsigned char* bv_s = vring;                                  // value stage 0 is free now
     if constexpr (RV > 0) {
@@ -783,6 +1027,13 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
   }
+  if (worklist) {
+    // end of a piece: nothing of it is in flight any more once every warp is here
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+  }
+  }   // pieces of the work list (one pass in a classic launch)
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

@@ -92,3 +92,11 @@ class Layer:
         self.px.lr_attend_prefill(self.desc, qd, agent, T, self.B_k, self.B_v, self.cache, out, bt, first_block)
         torch.cuda.synchronize()
         return out
+
+    def prefill_ws(self, q: torch.Tensor, agent: int, T: int, ws, block_table=None, first_block=0):
+        qd = q.cuda()
+        out = torch.full_like(qd, float("nan"))
+        bt = None if block_table is None else block_table.cuda()
+        self.px.lr_attend_prefill_ws(self.desc, qd, agent, T, self.B_k, self.B_v, self.cache, out, ws, bt, first_block)
+        torch.cuda.synchronize()
+        return out

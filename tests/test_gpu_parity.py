@@ -558,6 +558,58 @@ def test_prefill_short_turn_over_long_context_is_split_over_a_cluster(px, hd, n_
     assert_close(f64(got), ref, f"split prefill hd{hd} T{T} S{S}")
 
 
+# (head_dim, q heads, kv heads, rank, context, new tokens, agent, paged): between 75 and 144 (row tile, kv head) blocks
+_HELPER_CASES = [(128, 32, 8, 32, 1500, 384, 1, False), (64, 32, 8, 16, 2300, 512, 0, True), (128, 32, 8, 64, 1300, 300, 1, False),
+                 (128, 32, 8, 8, 1100, 528, -1, False), (64, 16, 8, 0, 2000, 700, 0, True), (128, 28, 4, 16, 1800, 400, 1, False)]
+
+
+@pytest.mark.parametrize("hd,n_q,n_kv,r,T,S,agent,paged", _HELPER_CASES)
+def test_prefill_with_a_workspace_puts_helper_blocks_on_idle_sms(monkeypatch, hd, n_q, n_kv, r, T, S, agent, paged):
+    """One wave that leaves SMs idle: with a workspace every block stops short of its context's end and helper
+    blocks take the tails, several tile pieces each; the pieces meet through records in the workspace.  Against
+    the definition on rows at both ends of the turn and at tile borders, bit-identical from run to run, the
+    workspace reusable without clearing, and within rounding of the launch without a workspace."""
+    monkeypatch.setenv("PRECC_PREFILL_HELPER_MIN", "8")          # contexts the oracle finishes in seconds qualify:
+    n_steps = (T + S + 127) // 128                               # there the planner sees no gain, so the cut is given
+    monkeypatch.setenv("PRECC_PREFILL_HELPER_P", str(n_steps - 5))
+    p2 = Precc(0)
+    geo = I.Geometry(256, n_q, n_kv, hd, 2, r, r, alpha=2.0 * max(r, 1))
+    nb = (T + S + 15) // 16
+    L = Layer(p2, geo, seed=73, n_blocks=nb + 7, tag="hw")
+    H = I.hidden_states(T + S, geo, 73, "hw.H")
+    bt = None
+    if paged:
+        perm = I.permutation(nb + 7, 73, "hw.perm")[:nb].to(torch.int32)
+        slots = (perm.long()[:, None] * 16 + torch.arange(16)[None, :]).reshape(-1)[:T + S].to(torch.int32).cuda()
+        L.append(H, slot_mapping=slots)
+        bt = perm
+    else:
+        L.append(H)
+    qs = I.queries(S, geo, 73, "hw.q", gain=4.0)
+    nbytes = p2.prefill_ws_bytes(L.desc, S)
+    assert nbytes > 0
+    ws = torch.full((nbytes,), 0xA5, dtype=torch.uint8, device="cuda")     # contents on entry do not matter
+    got = L.prefill_ws(qs, agent, T, ws, bt)
+    again = L.prefill_ws(qs, agent, T, ws, bt)                             # the same workspace, not cleared
+    assert torch.equal(got, again)
+    plain = L.prefill(qs, agent, T, bt)
+    assert not torch.equal(got, plain)                                     # the helper blocks did run: another summation order
+    tol = 2e-2 + 1e-2 * plain.float().abs()
+    assert ((got.float() - plain.float()).abs() <= tol).all()
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")            # too small a workspace: the plain launch, bit for bit
+    assert torch.equal(L.prefill_ws(qs, agent, T, small, bt), plain)
+    assert torch.equal(L.prefill_ws(qs, agent, T, None, bt), plain)
+    w = L.w_np
+    tpt = 128 // geo.group
+    rows = sorted(set([0, 1, tpt - 1, tpt, S // 2, S - tpt, S - 2, S - 1]))
+    a = max(agent, 0)
+    sk, sv = (geo.scale_k, geo.scale_v) if agent >= 0 and r else (0.0, 0.0)
+    ref = O.lr_prefill_reference(f64(qs), a, T, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"], sk, sv, n_kv,
+                                 rows=rows)
+    assert_close(f64(got), ref, f"helper prefill hd{hd} T{T} S{S}")
+    assert p2.poll_status() == 0
+
+
 @pytest.mark.parametrize("n", [1, 10, 100])
 def test_per_row_agent_masks_equal_two_separate_projections(px, n):
     """Double batching: adapted rows (current agent's LR rows, private slots) and adapter-free rows (the other
