@@ -36,7 +36,7 @@ struct PrefillRun {
     // fold, pipeline fill, record), in steps: measured at head_dim 128, rank 32 (1.3 us per step), scaled for shorter steps
     const int f100 = 100 * 160 / (HD + (RK + RV) / 2);
     const int C_OWN = 14 * f100 / 100, C_PIECE = 12 * f100 / 100;
-    int best_cost = n_max - std::max(2, n_max / 25);   // a plan must win at least 4 % (and two steps)
+    int best_cost = n_max - std::max(2, n_max / 12);   // a plan must win at least 8 % on paper: with every SM busy a step takes about 4 % longer
     for (int p = n_max - 1; p >= std::max(8, n_max / 2); --p) {
       if (ctx->prefill_helper_p > 0 && p != ctx->prefill_helper_p) continue;
       long long tail_sum = 0;
