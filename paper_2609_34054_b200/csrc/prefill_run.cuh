@@ -88,7 +88,12 @@ struct PrefillRun {
       else if (C::smem_bytes(ks, vs + 1) <= ctx->max_smem_optin) ++vs;
       else break;
     }
-    const int smem = C::smem_bytes(ks, vs);
+    // room for one value stage but not for two (head_dim 128 with rank 64): a ring of three 64-token half stages
+    // lets the next step's values start loading while the current step's are still being read
+    bool v_half = false;
+    if (vs == 1 && !ctx->no_prefill_vhalf && C::smem_bytes(ks, 3, true) <= ctx->max_smem_optin) { v_half = true; vs = 3; }
+    else if (ctx->force_prefill_vhalf && vs <= 3) { v_half = true; vs = 2 * vs; }     // tests: the same bytes as units of half a step
+    const int smem = C::smem_bytes(ks, vs, v_half);
     const size_t kvw = (size_t)d->n_kv_heads * HD;
     const long long kv_rows = (long long)a.cache->n_blocks * d->n_kv_heads * PAGE;
     const long long lr_rows = (long long)a.cache->n_blocks * PAGE;
@@ -97,16 +102,17 @@ struct PrefillRun {
     // instruction per 64-column slab instead of one per page)
     const bool contig = a.block_table == nullptr;
     const int box_rows = contig ? PTC_TOK : PAGE;
+    const int v_box_blocks = (v_half ? PTC_TOK / 2 : PTC_TOK) / PAGE, v_box_rows = contig ? v_box_blocks * PAGE : PAGE;
     int32_t rc = a.k_scratch ? make_map_cache4(ctx, &mk, a.k_scratch, a.k_scratch_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
                  : contig    ? make_map_cache4(ctx, &mk, a.cache->k_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
                              : make_map2(ctx, &mk, a.cache->k_base, kv_rows, HD, PAGE, 64);
     if (rc) return rc;
-    rc = contig ? make_map_cache4(ctx, &mv, a.cache->v_base, a.cache->n_blocks, d->n_kv_heads, HD, PTC_TOK / PAGE)
+    rc = contig ? make_map_cache4(ctx, &mv, a.cache->v_base, a.cache->n_blocks, d->n_kv_heads, HD, v_box_blocks)
                 : make_map2(ctx, &mv, a.cache->v_base, kv_rows, HD, PAGE, 64);
     if (rc) return rc;
     mlk = mk; mlv = mv;     // placeholders when a rank is zero (never dereferenced)
     if (RK) { rc = make_map2(ctx, &mlk, (const __nv_bfloat16*)a.cache->lr_k + (size_t)a.agent * lr_rows * RK, lr_rows, RK, box_rows, C::RKP); if (rc) return rc; }
-    if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, box_rows, 64); if (rc) return rc; }
+    if (RV) { rc = make_map2(ctx, &mlv, (const __nv_bfloat16*)a.cache->lr_v + (size_t)a.agent * lr_rows * RV, lr_rows, RV, v_box_rows, 64); if (rc) return rc; }
     PrefillTcParams p;
     p.q = (const __nv_bfloat16*)a.q; p.out = (__nv_bfloat16*)a.out; p.block_table = a.block_table;
     p.B_k = RK ? (const __nv_bfloat16*)a.B_k + (size_t)a.agent * RK * kvw : nullptr;
@@ -114,7 +120,7 @@ struct PrefillRun {
     p.status = ctx->status; p.n_blocks = a.cache->n_blocks;
     p.S = a.S; p.T = a.T; p.first_block = a.first_block; p.contig = contig ? 1 : 0; p.k_logical = a.k_scratch ? 1 : 0;
     p.longest_first = ctx->prefill_forward ? 0 : 1;
-    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.k_stages = ks; p.v_stages = vs;
+    p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.k_stages = ks; p.v_stages = vs; p.v_half = v_half ? 1 : 0;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
     p.trace = (ctx->trace && ctx->trace_blocks >= 32) ? ctx->trace : nullptr;
     auto kern = lr_attend_prefill_tc_kernel<HD, RK, RV>;
@@ -125,7 +131,7 @@ struct PrefillRun {
     int ns = 1;
     const long long base_blocks = (long long)row_tiles * d->n_kv_heads;
     const int steps = (a.T + a.S + PTC_TOK - 1) / PTC_TOK;
-    if (!ctx->no_prefill_split && C::SPLIT_BYTES <= C::Q_BYTES + C::QX_BYTES + ks * C::KSTAGE + vs * C::VSTAGE) {
+    if (!ctx->no_prefill_split && C::SPLIT_BYTES <= C::Q_BYTES + C::QX_BYTES + ks * C::KSTAGE + vs * (v_half ? C::VSTAGE / 2 : C::VSTAGE)) {
       ns = (int)(ctx->sm_count / base_blocks);          // as many as keep the grid within one block per SM
       if (ns > 8) ns = 8;
       if (ns > steps / 8) ns = steps / 8;               // at least eight steps per block

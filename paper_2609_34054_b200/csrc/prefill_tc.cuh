@@ -46,6 +46,8 @@ struct PrefillTcParams {
   int n_q, n_kv, group;
   int tok_per_tile;            // 128 / group
   int k_stages, v_stages;      // depth of the key ring and of the value ring
+  int v_half;                  // 1: the value ring holds v_stages units of 64 tokens (half a step) instead of whole steps - where
+                               //    shared memory has room for one and a half value stages but not for two
   int contig;                  // 1: no block table; the tensor maps fetch a whole 128-token stage per box
   int k_logical;               // 1: the key map covers a scratch copy of this sequence's keys in logical block order (whole-stage boxes
                                //    from block 0), whatever the layout of the value side
@@ -118,7 +120,7 @@ struct PrefillTcCfg {
   static constexpr bool L_IN_MMA = RV > 0 && RV < 64;         // a spare column of the L_V slab carries the denominator
   static constexpr int TMEM_P = 2 * PTC_TOK;                  // packed bf16 P (64 columns) after the two S buffers
   static constexpr int TMEM_O = TMEM_P + PTC_TOK / 2;         // O' (at most 192 columns): 320 + 192 = 512
-  __host__ __device__ static constexpr int smem_bytes(int ks, int vs) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * VSTAGE + 320 + 2 * PTC_PARTS_MAX * 512 + PTC_TAB_BYTES + 1024; }
+  __host__ __device__ static constexpr int smem_bytes(int ks, int vs, bool v_half = false) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * (v_half ? VSTAGE / 2 : VSTAGE) + 320 + 2 * PTC_PARTS_MAX * 512 + PTC_TAB_BYTES + 1024; }
   static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 8 || RK == 16 || RK == 32 || RK == 64) &&
                                     (RV == 0 || RV == 8 || RV == 16 || RV == 32 || RV == 64);
 };
@@ -217,7 +219,8 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   unsigned char* kring = smem + C::Q_BYTES + C::QX_BYTES;
   unsigned char* vring = kring + (size_t)KS * C::KSTAGE;
   const uint32_t vring_u32 = kring_u32 + KS * C::KSTAGE;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(vring + (size_t)VS * C::VSTAGE);
+  const int vunit = p.v_half ? C::VSTAGE / 2 : C::VSTAGE;   // bytes of one slot of the value ring
+  uint64_t* bars = reinterpret_cast<uint64_t*>(vring + (size_t)VS * vunit);
   const uint32_t bar0 = smem_u32(bars);
   // barrier map: k_full[KS] | k_empty[KS] | v_full[VS] | v_empty[VS] | s_full[2] | p_full[2] | pv_done | q_ready | s_free[2] | fold_go | fold_done
   const uint32_t k_full = bar0, k_empty = k_full + 8 * KS, v_full = k_empty + 8 * KS, v_empty = v_full + 8 * VS,
@@ -353,6 +356,41 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const bool is_k = warp == 0;
     const int NS = is_k ? KS : VS;
     const uint32_t fullb = is_k ? k_full : v_full, emptyb = is_k ? k_empty : v_empty;
+    if (!is_k && p.v_half) {
+      // value ring in units of 64 tokens: two units per step, each freed as soon as its four k-steps of P V' retire
+      constexpr int UT = PTC_TOK / 2, UPG = UT / PAGE, HSLAB = C::SLAB_BYTES / 2;
+      for (int u = 0; u < 2 * n_tiles; ++u) {
+        const int s = u % VS;
+        if (u >= VS) mbar_wait(v_empty + 8 * s, ((u / VS) - 1) & 1, p.status);
+        const int t0 = (2 * jb + u) * UT;
+        const uint32_t st = vring_u32 + (uint32_t)s * (C::VSTAGE / 2);
+        const uint32_t full = v_full + 8 * s;
+        if (p.contig) {
+          if (lane == 0) {
+            mbar_expect_tx(full, UPG * C::V_PAGE_TX);
+            const int blk0 = p.first_block + (2 * jb + u) * UPG;
+#pragma unroll
+            for (int sl = 0; sl < C::SLABS; ++sl) tma_load_4d(st + sl * HSLAB, &map_v, sl * 64, 0, g, blk0, full);
+            if constexpr (RV > 0) tma_load_2d(st + C::SLABS * HSLAB, &map_lv, 0, blk0 * PAGE, full);
+          }
+          __syncwarp();
+          continue;
+        }
+        const int live = max(0, min(UPG, (t_end - t0 + PAGE - 1) / PAGE));
+        if (lane == 0) mbar_expect_tx(full, live * C::V_PAGE_TX);       // no live page: the phase completes at once
+        __syncwarp();
+        if (lane < live) {
+          const int lt = (2 * jb + u) * UPG + lane;
+          int ph = p.block_table ? __ldg(p.block_table + lt) : p.first_block + lt;
+          if (ph < 0 || ph >= p.n_blocks) { atomicOr(p.status, StatusBits::BAD_INDEX); ph = 0; }
+          const int row_kv = (ph * p.n_kv + g) * PAGE;
+#pragma unroll
+          for (int sl = 0; sl < C::SLABS; ++sl) tma_load_2d(st + sl * HSLAB + lane * PAGE * 128, &map_v, sl * 64, row_kv, full);
+          if constexpr (RV > 0) tma_load_2d(st + C::SLABS * HSLAB + lane * PAGE * 128, &map_lv, 0, ph * PAGE, full);
+        }
+        __syncwarp();
+      }
+    } else
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j % NS;
       if (j >= NS) mbar_wait(emptyb + 8 * s, ((j / NS) - 1) & 1, p.status);
@@ -461,6 +499,48 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // ------------------------------------------------------------------ O' += P V' issuer
     const uint32_t id_o = umma_idesc(C::OW, 1);
     const uint64_t vd0 = umma_desc_mnmajor(vring_u32, 128, C::SLAB_BYTES);
+    if (p.v_half) {
+      constexpr int UT = PTC_TOK / 2, HSLAB = C::SLAB_BYTES / 2;
+      const uint64_t vdh = umma_desc_mnmajor(vring_u32, 128, HSLAB);
+      for (int j = 0; j < n_tiles; ++j) {
+        const int n_live = min(PTC_TOK, t_end - (jb + j) * PTC_TOK);     // tokens of this step that exist
+        for (int half = 0; half < 2; ++half) {
+          const int u = 2 * j + half, s = u % VS;
+          const int live_u = max(0, min(UT, n_live - half * UT));        // tokens of this unit that exist
+          mbar_wait(v_full + 8 * s, (u / VS) & 1, p.status);
+          unsigned char* ub = vring + (size_t)s * (C::VSTAGE / 2);
+          if constexpr (C::L_IN_MMA) {
+            unsigned char* slab = ub + C::SLABS * HSLAB;
+            constexpr int CH = (RV * 2) / 16;
+            for (int r = lane; r < UT; r += 32)
+              *reinterpret_cast<__nv_bfloat16*>(slab + r * 128 + ((CH ^ (r & 7)) * 16)) = __float2bfloat16(r < live_u ? 1.f : 0.f);
+            fence_async_smem();
+            __syncwarp();
+          }
+          if (live_u < UT && (p.contig || (live_u % PAGE) != 0)) {
+            // rows past the end may hold anything: clear them before the MMA reads the unit
+            const int r1 = p.contig ? UT : (live_u + PAGE - 1) / PAGE * PAGE;
+            for (int r = live_u; r < r1; ++r)
+              for (int sl = 0; sl < C::VSLABS; ++sl)
+                for (int c = lane; c < 8; c += 32) *reinterpret_cast<uint4*>(ub + sl * HSLAB + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+            fence_async_smem();
+            __syncwarp();
+          }
+          if (half == 0) mbar_wait(p_full + 8 * (j & 1), (j >> 1) & 1, p.status);
+          tc_fence_after();
+          if (lane == 0) {
+            const uint32_t a = tmem_base + C::TMEM_P + half * (UT / 2);  // packed bf16 P, 2 per column
+            const uint64_t so = (uint64_t)((s * (C::VSTAGE / 2)) >> 4);
+            const uint32_t od = tmem_base + C::TMEM_O;
+            const int n_ks = (live_u + 15) / 16;
+            for (int ks = 0; ks < n_ks; ++ks) umma_bf16_ts(od, a + ks * 8, vdh + so + (uint64_t)(ks * 128), id_o, (j | half | ks) ? 1u : 0u);
+            umma_commit(v_empty + 8 * s);
+            if (half == 1) umma_commit(pv_done);
+          }
+          __syncwarp();
+        }
+      }
+    } else
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j % VS;
       const int n_live = min(PTC_TOK, t_end - (jb + j) * PTC_TOK);       // tokens of this step that exist

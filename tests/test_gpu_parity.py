@@ -558,6 +558,45 @@ def test_prefill_short_turn_over_long_context_is_split_over_a_cluster(px, hd, n_
     assert_close(f64(got), ref, f"split prefill hd{hd} T{T} S{S}")
 
 
+@pytest.mark.parametrize("hd,n_q,n_kv,r,T,S,agent,paged", [(128, 8, 2, 32, 700, 90, 1, False), (64, 16, 4, 16, 1203, 77, 0, True),
+                                                             (128, 8, 2, 8, 515, 130, 1, True), (64, 8, 2, 64, 300, 200, 1, False),
+                                                             (128, 8, 2, 0, 450, 64, -1, False), (128, 8, 2, 64, 2100, 40, 1, True),
+                                                             (128, 16, 2, 64, 1000, 260, 0, False)])
+def test_prefill_value_ring_in_half_steps_is_bit_identical(monkeypatch, hd, n_q, n_kv, r, T, S, agent, paged):
+    """Where shared memory holds one value stage but not two (head_dim 128, rank 64) the value ring works in units
+    of 64 tokens.  The same MMAs in the same order: bit-identical to whole-step stages, here on every kind of
+    shape (the switch forces half-step units), on contexts that end inside a unit, paged and contiguous."""
+    monkeypatch.setenv("PRECC_PREFILL_VHALF", "0")
+    p_whole = Precc(0)
+    monkeypatch.setenv("PRECC_PREFILL_VHALF", "1")
+    p_half = Precc(0)
+    geo = I.Geometry(256, n_q, n_kv, hd, 2, r, r, alpha=2.0 * max(r, 1))
+    nb = (T + S + 15) // 16
+    L = Layer(p_half, geo, seed=75, n_blocks=nb + 5, tag="vh")
+    H = I.hidden_states(T + S, geo, 75, "vh.H")
+    bt = None
+    if paged:
+        bt = I.permutation(nb + 5, 75, "vh.perm")[:nb].to(torch.int32)
+        slots = (bt.long()[:, None] * 16 + torch.arange(16)[None, :]).reshape(-1)[:T + S].to(torch.int32).cuda()
+        L.append(H, slot_mapping=slots)
+    else:
+        L.append(H)
+    qs = I.queries(S, geo, 75, "vh.q", gain=4.0)
+    got = L.prefill(qs, agent, T, bt)
+    ref = torch.full_like(got, float("nan"))
+    p_whole.lr_attend_prefill(L.desc, qs.cuda(), agent, T, L.B_k, L.B_v, L.cache, ref, None if bt is None else bt.cuda(), 0)
+    torch.cuda.synchronize()
+    assert torch.equal(got, ref)
+    w = L.w_np
+    rows = sorted(set([0, S // 2, S - 1]))
+    a = max(agent, 0)
+    sk, sv = (geo.scale_k, geo.scale_v) if agent >= 0 and r else (0.0, 0.0)
+    want = O.lr_prefill_reference(f64(qs), a, T, f64(H), w["W_k"], w["W_v"], w["A_k"], w["B_k"], w["A_v"], w["B_v"], sk, sv, n_kv,
+                                  rows=rows)
+    assert_close(f64(got), want, f"half-step value ring hd{hd} r{r} T{T} S{S}")
+    assert p_half.poll_status() == 0
+
+
 # (head_dim, q heads, kv heads, rank, context, new tokens, agent, paged): between 75 and 144 (row tile, kv head) blocks
 _HELPER_CASES = [(128, 32, 8, 32, 1500, 384, 1, False), (64, 32, 8, 16, 2300, 512, 0, True), (128, 32, 8, 64, 1300, 300, 1, False),
                  (128, 32, 8, 8, 1100, 528, -1, False), (64, 16, 8, 0, 2000, 700, 0, True), (128, 28, 4, 16, 1800, 400, 1, False)]
