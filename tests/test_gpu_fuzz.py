@@ -416,3 +416,66 @@ def test_random_large_prefill(px, i):
         t = T + srow + 1
         ref = O.attend_from_caches(f64(q[srow]), K[:t], V[:t], Lk[:t], Lv[:t], Bka, Bva, geo.scale_k, geo.scale_v, n_kv)
         assert_close(f64(out[srow]), ref, f"case {i} large prefill row {srow} (hd{hd} G{G} kv{n_kv} r{r} S{S} T{T} agent{agent} paged={paged})")
+
+
+@pytest.fixture(scope="module")
+def px_helpers():
+    """A context in which short contexts qualify for helper blocks too (the switch is read at creation)."""
+    old = os.environ.get("PRECC_PREFILL_HELPER_MIN")
+    os.environ["PRECC_PREFILL_HELPER_MIN"] = "8"
+    p = Precc(0)
+    if old is None:
+        del os.environ["PRECC_PREFILL_HELPER_MIN"]
+    else:
+        os.environ["PRECC_PREFILL_HELPER_MIN"] = old
+    yield p
+    assert p.poll_status() == 0
+    p.close()
+
+
+@pytest.mark.parametrize("i", range(N_LARGE))
+def test_random_prefill_with_helper_blocks(px_helpers, i):
+    """Turn lengths that leave between a sixteenth and a half of the SMs without a block, contexts of 1k .. 40k tokens:
+    the planner's own cuts (or its refusal), against the definition on rows across the turn, twice on one workspace."""
+    px = px_helpers
+    rng = np.random.default_rng(60000 + i)
+    hd = int(rng.choice([64, 128])); G = int(rng.choice([1, 2, 4, 8])); n_kv = int(rng.choice([2, 4, 8]))
+    r = int(rng.choice([0, 8, 16, 32, 64])); N = int(rng.integers(1, 4))
+    tpt = 128 // G
+    tiles = int(rng.integers(px.sm_count // 2 + 1, px.sm_count * 14 // 15))
+    X = max(1, tiles // n_kv)
+    S = int(min(4000, X * tpt - int(rng.integers(0, tpt))))
+    T = int(rng.choice([1000, 3000, 9000, 20000, 40000]))
+    T = int(rng.integers(T // 2, T + 1))
+    agent = int(rng.integers(-1, N))
+    paged = bool(rng.random() < 0.5)
+    geo = I.Geometry(64, G * n_kv, n_kv, hd, N, r, r, alpha=2.0 * max(r, 1))
+    desc = layer_desc(geo)
+    nb = (T + S + 15) // 16
+    c = I.direct_caches_device(nb + 3, geo, 600 + i, f"hp{i}")
+    cache = Cache.from_tensors(geo, c["k_base"], c["v_base"], c.get("lr_k"), c.get("lr_v"))
+    Bk, Bv, w = _weights_small(geo, 600 + i, f"hp{i}")
+    tab = I.permutation(nb + 3, 600 + i, f"hp.perm{i}")[:nb].to(torch.int32) if paged else torch.arange(2, nb + 2, dtype=torch.int32)
+    q = I.queries(S, geo, 600 + i, f"hp.q{i}", gain=3.0)
+    ws = torch.full((max(px.prefill_ws_bytes(desc, S), 256),), 0x5A, dtype=torch.uint8, device="cuda")
+    outs = []
+    for _ in range(2):
+        out = torch.full_like(q, float("nan"), device="cuda")
+        px.lr_attend_prefill_ws(desc, q.cuda(), agent, T, Bk, Bv, cache, out, ws, tab.cuda() if paged else None, 0 if paged else 2)
+        torch.cuda.synchronize()
+        outs.append(out)
+    assert torch.equal(outs[0], outs[1])
+    out = outs[0]
+    assert torch.isfinite(out.float()).all()
+    blocks = tab.long().cuda()
+    K = f64(c["k_base"][blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))
+    V = f64(c["v_base"][blocks].permute(0, 2, 1, 3).reshape(-1, n_kv * hd))
+    Lk = f64(c["lr_k"][max(agent, 0)][blocks].reshape(-1, r)) if r else np.zeros((nb * 16, 0))
+    Lv = f64(c["lr_v"][max(agent, 0)][blocks].reshape(-1, r)) if r else np.zeros((nb * 16, 0))
+    Bka = f64(w["B_k"][agent]) if (r and agent >= 0) else np.zeros((r, n_kv * hd))
+    Bva = f64(w["B_v"][agent]) if (r and agent >= 0) else np.zeros((r, n_kv * hd))
+    for srow in sorted(set([0, tpt - 1, S // 2, S - 1])):
+        srow = min(srow, S - 1)
+        t = T + srow + 1
+        ref = O.attend_from_caches(f64(q[srow]), K[:t], V[:t], Lk[:t], Lv[:t], Bka, Bva, geo.scale_k, geo.scale_v, n_kv)
+        assert_close(f64(out[srow]), ref, f"case {i} helper prefill row {srow} (hd{hd} G{G} kv{n_kv} r{r} S{S} T{T} agent{agent} paged={paged})")
