@@ -638,6 +638,8 @@ def test_prefill_with_a_workspace_puts_helper_blocks_on_idle_sms(monkeypatch, hd
     small = torch.empty(1024, dtype=torch.uint8, device="cuda")            # too small a workspace: the plain launch, bit for bit
     assert torch.equal(L.prefill_ws(qs, agent, T, small, bt), plain)
     assert torch.equal(L.prefill_ws(qs, agent, T, None, bt), plain)
+    with pytest.raises(PreccError, match="MISALIGNED|aligned"):
+        L.prefill_ws(qs, agent, T, ws[16:], bt)                            # a workspace must start on a 256-byte boundary
     w = L.w_np
     tpt = 128 // geo.group
     rows = sorted(set([0, 1, tpt - 1, tpt, S // 2, S - tpt, S - 2, S - 1]))
