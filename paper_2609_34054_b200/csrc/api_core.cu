@@ -206,7 +206,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   if (const char* v = getenv("PRECC_DECODE")) ctx->force_ticket_decode = (strcmp(v, "ticket") == 0);
   if (const char* v = getenv("PRECC_PREFILL_ORDER")) ctx->prefill_forward = (strcmp(v, "forward") == 0);
   if (const char* v = getenv("PRECC_PREFILL_SPLIT")) ctx->no_prefill_split = (strcmp(v, "0") == 0);
-  if (const char* v = getenv("PRECC_PREFILL_VHALF")) { ctx->no_prefill_vhalf = (strcmp(v, "0") == 0); ctx->force_prefill_vhalf = (strcmp(v, "1") == 0); }
+  if (const char* v = getenv("PRECC_PREFILL_VHALF")) ctx->no_prefill_vhalf = (strcmp(v, "0") == 0);
   if (const char* v = getenv("PRECC_PREFILL_HELPERS")) ctx->no_prefill_helpers = (strcmp(v, "0") == 0);
   if (const char* v = getenv("PRECC_PREFILL_HELPER_P")) ctx->prefill_helper_p = atoi(v);
   if (const char* v = getenv("PRECC_PREFILL_HELPER_MIN")) { const int n = atoi(v); if (n >= 8) ctx->prefill_helper_min_steps = n; }

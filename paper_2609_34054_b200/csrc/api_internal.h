@@ -41,7 +41,6 @@ struct precc_ctx {
   bool prefill_forward = false;        // PRECC_PREFILL_ORDER=forward: row tiles in ascending order (default: longest causal reach first)
   bool no_prefill_split = false;       // PRECC_PREFILL_SPLIT=0 in the environment: never split a turn's context over a cluster
   bool no_prefill_vhalf = false;       // PRECC_PREFILL_VHALF=0 in the environment: the value ring of the tcgen05 prefill kernel always holds whole steps
-  bool force_prefill_vhalf = false;    // PRECC_PREFILL_VHALF=1: half-step units wherever the ring has at most three stages (tests)
   bool no_prefill_helpers = false;     // PRECC_PREFILL_HELPERS=0 in the environment: prefill with a workspace never uses helper blocks
   int prefill_helper_p = 0;            // PRECC_PREFILL_HELPER_P=n in the environment: the tiles' own blocks stop after n steps (experiments; 0 = planner's choice)
   int prefill_helper_min_steps = 48;   // PRECC_PREFILL_HELPER_MIN=n in the environment: shortest context (128-token steps) that gets helper blocks

@@ -91,8 +91,9 @@ struct PrefillRun {
     // room for one value stage but not for two (head_dim 128 with rank 64): a ring of three 64-token half stages
     // lets the next step's values start loading while the current step's are still being read
     bool v_half = false;
-    if (vs == 1 && !ctx->no_prefill_vhalf && C::smem_bytes(ks, 3, true) <= ctx->max_smem_optin) { v_half = true; vs = 3; }
-    else if (ctx->force_prefill_vhalf && vs <= 3) { v_half = true; vs = 2 * vs; }     // tests: the same bytes as units of half a step
+    if constexpr (C::V_HALF_CAPABLE) {
+      if (vs == 1 && !ctx->no_prefill_vhalf && C::smem_bytes(ks, 3, true) <= ctx->max_smem_optin) { v_half = true; vs = 3; }
+    }
     const int smem = C::smem_bytes(ks, vs, v_half);
     const size_t kvw = (size_t)d->n_kv_heads * HD;
     const long long kv_rows = (long long)a.cache->n_blocks * d->n_kv_heads * PAGE;
@@ -123,7 +124,13 @@ struct PrefillRun {
     p.n_q = d->n_q_heads; p.n_kv = d->n_kv_heads; p.group = G; p.tok_per_tile = PTC_TOK / G; p.k_stages = ks; p.v_stages = vs; p.v_half = v_half ? 1 : 0;
     p.scale_log2 = softmax_scale_log2(d); p.s_k = d->lora_scale_k; p.s_v = d->lora_scale_v;
     p.trace = (ctx->trace && ctx->trace_blocks >= 32) ? ctx->trace : nullptr;
-    auto kern = lr_attend_prefill_tc_kernel<HD, RK, RV>;
+    // four instantiations at most: classic / work list, whole-step / half-step value ring (the latter only where it applies)
+    using KernT = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, PrefillTcParams);
+    KernT kern = lr_attend_prefill_tc_kernel<HD, RK, RV, false, false>;
+    KernT kern_wl = lr_attend_prefill_tc_kernel<HD, RK, RV, true, false>;
+    if constexpr (C::V_HALF_CAPABLE) {
+      if (v_half) { kern = lr_attend_prefill_tc_kernel<HD, RK, RV, false, true>; kern_wl = lr_attend_prefill_tc_kernel<HD, RK, RV, true, true>; }
+    }
     PRECC_CUDA(ctx, raise_smem_limit(ctx, kern, smem));
     const int row_tiles = (a.S + p.tok_per_tile - 1) / p.tok_per_tile;
     // Short turn over a long context: too few (row tile, kv head) blocks to fill the machine, so the
@@ -172,9 +179,10 @@ struct PrefillRun {
         p.ws_ticket = reinterpret_cast<unsigned int*>(a.ws);
         p.ws_rec = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(a.ws) + ticket_bytes(wl.tiles));
         PRECC_CUDA(ctx, cudaMemsetAsync(a.ws, 0, ticket_bytes(wl.tiles), a.stream));
+        PRECC_CUDA(ctx, raise_smem_limit(ctx, kern_wl, smem));
         cudaLaunchConfig_t wc = {};
         wc.gridDim = dim3(wl.tiles + wl.helpers); wc.blockDim = dim3(PTC_THREADS); wc.dynamicSmemBytes = smem; wc.stream = a.stream;
-        PRECC_CUDA(ctx, cudaLaunchKernelEx(&wc, kern, mk, mv, mlk, mlv, p));
+        PRECC_CUDA(ctx, cudaLaunchKernelEx(&wc, kern_wl, mk, mv, mlk, mlv, p));
         return PRECC_OK;
       }
     }

@@ -87,6 +87,7 @@ constexpr int PTC_PARTS = 2;                         // softmax threads per quer
 constexpr int PTC_SOFTMAX_WARPS = 4 * PTC_PARTS;
 constexpr int PTC_FIRST_SM_WARP = 3;                 // warps 0..2: key producer, QK^T issuer, PV issuer
 constexpr int PTC_THREADS = (PTC_FIRST_SM_WARP + PTC_SOFTMAX_WARPS + 1) * 32;
+constexpr int PTC_SMEM_LIMIT = 232448;   // dynamic shared memory a block can opt into on this architecture
 constexpr int PTC_FIXED_BARS = 10; // barriers besides the two per ring stage
 constexpr int PTC_TOK = 128;      // tokens per step
 constexpr float PTC_RAISE = 8.f;  // the running maximum is raised only when it grows by more than this
@@ -121,6 +122,8 @@ struct PrefillTcCfg {
   static constexpr int TMEM_P = 2 * PTC_TOK;                  // packed bf16 P (64 columns) after the two S buffers
   static constexpr int TMEM_O = TMEM_P + PTC_TOK / 2;         // O' (at most 192 columns): 320 + 192 = 512
   __host__ __device__ static constexpr int smem_bytes(int ks, int vs, bool v_half = false) { return Q_BYTES + QX_BYTES + ks * KSTAGE + vs * (v_half ? VSTAGE / 2 : VSTAGE) + 320 + 2 * PTC_PARTS_MAX * 512 + PTC_TAB_BYTES + 1024; }
+  // one whole value stage fits beside two key stages, two do not, three half-step units do (head_dim 128 with rank 64)
+  static constexpr bool V_HALF_CAPABLE = smem_bytes(2, 2) > PTC_SMEM_LIMIT && smem_bytes(2, 1) <= PTC_SMEM_LIMIT && smem_bytes(2, 3, true) <= PTC_SMEM_LIMIT;
   static constexpr bool supported = (HD == 64 || HD == 128) && (RK == 0 || RK == 8 || RK == 16 || RK == 32 || RK == 64) &&
                                     (RV == 0 || RV == 8 || RV == 16 || RV == 32 || RV == 64);
 };
@@ -204,7 +207,11 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
 }
 
-template <int HD, int RK, int RV>
+// WL: the work-list form (helper blocks; a block takes a list of tile pieces).  It is a separate instantiation so that
+// the classic launch carries none of its state through the step loop (the kernel sits at its register limit).
+// VH: the value ring holds units of 64 tokens (half a step) - instantiated only where shared memory has room for
+// one whole value stage but not for two.
+template <int HD, int RK, int RV, bool WL = false, bool VH = false>
 __global__ void __launch_bounds__(PTC_THREADS, 1)
 lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                             const __grid_constant__ CUtensorMap map_lk, const __grid_constant__ CUtensorMap map_lv,
@@ -219,7 +226,8 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   unsigned char* kring = smem + C::Q_BYTES + C::QX_BYTES;
   unsigned char* vring = kring + (size_t)KS * C::KSTAGE;
   const uint32_t vring_u32 = kring_u32 + KS * C::KSTAGE;
-  const int vunit = p.v_half ? C::VSTAGE / 2 : C::VSTAGE;   // bytes of one slot of the value ring
+  constexpr bool v_half = VH;
+  const int vunit = v_half ? C::VSTAGE / 2 : C::VSTAGE;   // bytes of one slot of the value ring
   uint64_t* bars = reinterpret_cast<uint64_t*>(vring + (size_t)VS * vunit);
   const uint32_t bar0 = smem_u32(bars);
   // barrier map: k_full[KS] | k_empty[KS] | v_full[VS] | v_empty[VS] | s_full[2] | p_full[2] | pv_done | q_ready | s_free[2] | fold_go | fold_done
@@ -230,7 +238,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.group;
-  const bool worklist = p.helper_p > 0;
+  constexpr bool worklist = WL;
   // What this block works on.  Classic launch: one (row tile, kv head) per block, fixed for the whole kernel.  Work-list
   // launch: a short list of tile pieces, taken one after the other with the block drained in between.
   int g = blockIdx.y;
@@ -246,7 +254,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(split));
   asm volatile("mov.u32 %0, %%cluster_nctaid.z;\n" : "=r"(NS));
   int jb = 0, n_tiles = 0;
-  if (!worklist) {
+  if constexpr (!worklist) {
     const int n_total = (t_end + PTC_TOK - 1) / PTC_TOK;
     const int chunk_steps = (n_total + (int)NS - 1) / (int)NS;
     jb = min(n_total, (int)split * chunk_steps);
@@ -276,7 +284,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_holder)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
-  if (worklist) {
+  if constexpr (worklist) {
     for (int x = threadIdx.x; x < p.row_tiles; x += blockDim.x) tab_tail[x] = max(0, steps_of(x) - p.helper_p);
   }
   tc_fence_before();
@@ -284,7 +292,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
   const int n_base_tiles = p.row_tiles * p.n_kv;           // work-list launch: blocks below this index own a tile
-  if (worklist) {
+  if constexpr (worklist) {
     if (threadIdx.x == 0) {
       const int X = p.row_tiles;
       int acc = 0;
@@ -324,7 +332,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
   // work-list launch: the tile of this piece, where its record goes and which records make up the tile
   bool to_ws = false;
   int tile_u = 0, rec_id = 0, n_src = 1, src_first = 0;
-  if (worklist) {
+  if constexpr (worklist) {
     tile_u = tab_seg[4 * seg]; jb = tab_seg[4 * seg + 1]; n_tiles = tab_seg[4 * seg + 2];
     const int x = tile_u % p.row_tiles;
     g = tile_u / p.row_tiles;
@@ -356,7 +364,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     const bool is_k = warp == 0;
     const int NS = is_k ? KS : VS;
     const uint32_t fullb = is_k ? k_full : v_full, emptyb = is_k ? k_empty : v_empty;
-    if (!is_k && p.v_half) {
+    if (v_half && !is_k) {
       // value ring in units of 64 tokens: two units per step, each freed as soon as its four k-steps of P V' retire
       constexpr int UT = PTC_TOK / 2, UPG = UT / PAGE, HSLAB = C::SLAB_BYTES / 2;
       for (int u = 0; u < 2 * n_tiles; ++u) {
@@ -499,7 +507,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     // ------------------------------------------------------------------ O' += P V' issuer
     const uint32_t id_o = umma_idesc(C::OW, 1);
     const uint64_t vd0 = umma_desc_mnmajor(vring_u32, 128, C::SLAB_BYTES);
-    if (p.v_half) {
+    if constexpr (v_half) {
       constexpr int UT = PTC_TOK / 2, HSLAB = C::SLAB_BYTES / 2;
       const uint64_t vdh = umma_desc_mnmajor(vring_u32, 128, HSLAB);
       for (int j = 0; j < n_tiles; ++j) {
@@ -822,7 +830,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           *reinterpret_cast<uint4*>(xo + row * XS + c * 16 + k) = make_uint4(ov[k], ov[k + 1], ov[k + 2], ov[k + 3]);
       }
       if (part == 0) { xm[row] = n_tiles > 0 ? m_used : NEG_BIG; xl[row] = n_tiles > 0 ? l_loc : 0.f; }
-    } else if (to_ws) {
+    } else if (WL && to_ws) {
       // ---- work-list launch: this piece's partial (m, l, O') goes to its record in global memory; the block that
       //      arrives last at the tile's ticket merges the tile's records in a fixed order and writes the output
       constexpr int XS = C::SPLIT_XS;
@@ -1107,7 +1115,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
   }
-  if (worklist) {
+  if constexpr (worklist) {
     // end of a piece: nothing of it is in flight any more once every warp is here
     tc_fence_before();
     __syncthreads();
