@@ -8,8 +8,9 @@
 //   O' += P [V_base | L_V | 1]                  tcgen05.mma with A = P from TMEM; O' in TMEM holds the numerator
 //                                              (hd columns), U = P L_V (r_v columns) and, through a column of
 //                                              ones written into the zero-padded L_V slab, the denominator
-// and finally out = (O + s_v U B_v) / l on the CUDA cores.  The key-side fold Q~ = s_k Q B_k^T is
-// computed once per block by the softmax threads.  The caches arrive by TMA into rings of stages
+// and finally out = (O + s_v U B_v) / l on the CUDA cores.  The key-side fold Q~ = s_k Q B_k^T is one
+// small MMA chain per block before the first step (product in the first columns of S buffer 0, scaled and
+// rounded to bf16 by the softmax threads).  The caches arrive by TMA into rings of stages
 // guarded by mbarriers: one box per page and 64-column slab when a block table scatters the pages, one
 // box per slab for the whole 128-token stage (4-D tensor map) when the pages are consecutive.
 //
@@ -27,6 +28,13 @@
 // when it grows by more than 8 (log2 domain), so O' is rescaled a handful of times per row instead of
 // at every step; P stays below 2^8.  Every mbarrier wait is bounded and falls through with
 // PRECC_STATUS_TIMEOUT.
+//
+// Two more instantiations of the same kernel.  VH: the value ring holds units of 64 tokens instead of whole
+// steps (where one value stage fits beside two key stages but two do not), a unit being freed as soon as its
+// four k-steps of P V' retire.  WL: the work-list launch - a 1-D grid in which the first (row tiles x kv heads)
+// blocks stop `helper_p` steps into their tile and the remaining blocks share the tails of all tiles, several
+// pieces each with the block drained in between; the pieces of a tile meet through fp32 records in a
+// caller-provided workspace, and the block that arrives last at the tile's ticket merges them in piece order.
 #pragma once
 #include <type_traits>
 
