@@ -729,6 +729,16 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           for (int k = 0; k < 32; ++k)
             if (c * 32 + k >= nvis) sv[c][k] = 0xff800000u;      // -inf: weight zero
       }
+      // The two warps of a row share a scheduler and its special-function unit.  They take the next step's maximum at
+      // different points of the step - one here, one between the halves of its exponentials - so that one warp's
+      // exponentials run while the other reads tensor memory and compares, instead of both queueing for the unit at once.
+      float next_own = NEG_BIG;
+      const bool max_first = !VH && part == 1;                     // (with the half-step value ring the skew measured slower)
+      if (max_first && j + 1 < n_tiles) {
+        mbar_wait(s_full + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, p.status);
+        tc_fence_after();
+        next_own = local_max(j + 1);
+      }
       float m_new = m_used;
       if (tmax > m_used + PTC_RAISE) m_new = tmax;                 // all threads of the row decide alike
       const bool raise = m_new != m_used;
@@ -755,7 +765,6 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
       const float neg_m = -m_used;
       uint32_t pk[NCH][16];
-      float next_own = NEG_BIG;
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
 #pragma unroll
@@ -765,7 +774,7 @@ lr_attend_prefill_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __g
           if constexpr (!C::L_IN_MMA) ls[(k >> 1) & 3] += p0 + p1;
           pk[c][k / 2] = pack_bf16(p0, p1);
         }
-        if (c == 0 && j + 1 < n_tiles) {
+        if (c == 0 && !max_first && j + 1 < n_tiles) {
           if (tid == 0) PTC_STAMP(p, j, 12);                       // first half of the exponentials done
           // between the two halves of the exponentials: the next step's scores are normally there already
           mbar_wait(s_full + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, p.status);
