@@ -195,6 +195,7 @@ int32_t precc_create(precc_ctx** out, int32_t device) {
   if (const char* v = getenv("PRECC_GEMM")) { ctx->force_tiled_gemm = (strcmp(v, "tiled") == 0); ctx->gemm_pair = (strcmp(v, "pair") == 0); }
   if (const char* v = getenv("PRECC_DEEP")) { ctx->deep_clusters = (strcmp(v, "0") != 0); ctx->deep_always = (strcmp(v, "2") == 0); }
   if (const char* v = getenv("PRECC_DECODE_CLUSTER")) ctx->decode_cluster_cap = atoi(v);
+  if (const char* v = getenv("PRECC_DECODE_POLICY")) ctx->decode_cluster_policy = atoi(v);
   if (const char* v = getenv("PRECC_DECODE_STAGES")) ctx->decode_stage_cap = atoi(v);
   if (const char* v = getenv("PRECC_DECODE_PRE")) ctx->decode_pre_stages = atoi(v);
   if (const char* v = getenv("PRECC_GEMM_STAGES")) ctx->gemm_stage_cap = atoi(v);

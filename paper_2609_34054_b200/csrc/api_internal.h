@@ -37,6 +37,7 @@ struct precc_ctx {
   bool deep_always = false;            // PRECC_DEEP=2: take them wherever they fit, also where they leave many SMs without a block
   int decode_pre_stages = 0;           // PRECC_DECODE_PRE=n in the environment: ring slots filled before the dependency wait (0 = all)
   int decode_stage_cap = 0;            // PRECC_DECODE_STAGES=n in the environment: at most n ring slots per warp in the cluster schedule (0 = planner's choice)
+  int decode_cluster_policy = 0;       // PRECC_DECODE_POLICY=n in the environment: cluster scheduling policy of the decode clusters - 0 the driver's default, 1 spread, 2 load balancing
   int decode_cluster_cap = 0;          // PRECC_DECODE_CLUSTER=n in the environment: at most n blocks per decode cluster (0 = planner's choice)
   bool prefill_forward = false;        // PRECC_PREFILL_ORDER=forward: row tiles in ascending order (default: longest causal reach first)
   bool no_prefill_split = false;       // PRECC_PREFILL_SPLIT=0 in the environment: never split a turn's context over a cluster

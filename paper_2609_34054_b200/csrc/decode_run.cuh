@@ -258,7 +258,7 @@ struct DecodeRunT {
     cfg.gridDim = dim3(pl.max_splits, d->n_kv_heads, a.B);
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = a.stream;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[3];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
@@ -268,6 +268,13 @@ struct DecodeRunT {
       attr[1].id = cudaLaunchAttributeClusterDimension;
       attr[1].val.clusterDim.x = pl.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
       cfg.numAttrs = 2;
+      if (ctx->decode_cluster_policy) {
+        // where the blocks of a cluster go inside their GPC: spread over as many SMs as possible, or packed
+        attr[2].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
+        attr[2].val.clusterSchedulingPolicyPreference =
+            ctx->decode_cluster_policy == 1 ? cudaClusterSchedulingPolicySpread : cudaClusterSchedulingPolicyLoadBalancing;
+        cfg.numAttrs = 3;
+      }
       if (pl.warps == 8) {
         PRECC_CUDA(ctx, ensure_cluster_smem<8>(ctx, pl.smem, pl.deep != 0));
         PRECC_CUDA(ctx, cudaLaunchKernelEx(&cfg, cluster_kernel<8>(pl.deep != 0), p));
