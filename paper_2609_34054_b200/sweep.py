@@ -114,16 +114,19 @@ def precompute_cell(px: Precc, N: int, r: int, M: int = 32768, seed: int = 0) ->
 
 
 def prefill_cell(px: Precc, r: int, S: int, T: int, seed: int = 0) -> dict:
-    geo = I.c5_geometry(r, 4)
+    """r == 0: the adapter-free view (agent -1) of a rank-8 layer, i.e. the same kernel without LR columns."""
+    agent = 1 if r else -1
+    rr = r if r else 8
+    geo = I.c5_geometry(rr, 4)
     desc = layer_desc(geo)
     c = I.direct_caches_device((T + S) // I.PAGE, geo, seed, "sweep.pf")
     cache = Cache.from_tensors(geo, c["k_base"], c["v_base"], c["lr_k"], c["lr_v"])
     gen = torch.Generator(device="cuda").manual_seed(seed)
-    B_k = _randn((geo.n_agents, r, geo.kv_width), 0.02, gen)
-    B_v = _randn((geo.n_agents, r, geo.kv_width), 0.02, gen)
+    B_k = _randn((geo.n_agents, rr, geo.kv_width), 0.02, gen)
+    B_v = _randn((geo.n_agents, rr, geo.kv_width), 0.02, gen)
     q = _randn((S, geo.n_q, geo.hd), 1.0, gen)
     out = torch.empty_like(q)
-    us = _graph_time_us(lambda: px.lr_attend_prefill(desc, q, 1, T, B_k, B_v, cache, out), 2, 5)
+    us = _graph_time_us(lambda: px.lr_attend_prefill(desc, q, agent, T, B_k, B_v, cache, out), 2, 5)
     flops = 4.0 * geo.n_q * (geo.hd + r) * (S * T + S * (S + 1) / 2)      # scores + weighted sum over hd + r coordinates
     assert px.poll_status() == 0 and torch.isfinite(out.float()).all()
     return {"kind": "prefill", "r": r, "S": S, "T": T, "us": us, "TFLOPs": flops / us / 1e6}
@@ -140,7 +143,7 @@ def main(argv=None):
     px = Precc(0)
     dec, pre, pf = [], [], []
     if not (args.decode_only or args.precompute_only):
-        for r in RANKS:
+        for r in (0,) + tuple(RANKS):               # rank 0: the adapter-free view, for the LR overhead of the other rows
             for (S, T) in TURNS:
                 c = prefill_cell(px, r, S, T)
                 pf.append(c)
@@ -170,7 +173,7 @@ def main(argv=None):
                     f"{c['us']:.1f} us, {c['GBps']:.0f} GB/s ({c['GBps'] / args.peak_gbs * 100:.0f} %)" for c in cells) + " |")
     if pf:
         print("\n| r | " + " | ".join(f"S={S}, T={T}" for (S, T) in TURNS) + " |\n|---|" + "---|" * len(TURNS))
-        for r in RANKS:
+        for r in (0,) + tuple(RANKS):
             cells = [c for c in pf if c["r"] == r]
             print(f"| {r} | " + " | ".join(f"{c['us']:.0f} us, {c['TFLOPs']:.0f} TF/s ({c['TFLOPs'] / args.peak_tflops * 100:.0f} %)" for c in cells) + " |")
     if pre:
